@@ -1,0 +1,184 @@
+"""ctypes wrapper of the CPU oracle (``qfmt_oracle.c``).
+
+TEST INFRASTRUCTURE ONLY: imported by tests, the smoke check and the benchmark's CPU-baseline
+leg.  The product package never imports this module, and this module never imports the
+product package.  Marshalling only: every piece of arithmetic lives in the C file.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from typing import Optional, Tuple
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "qfmt_oracle.c")
+_LIB = os.path.join(_HERE, "liboracle.so")
+
+STATS_WORDS = 264
+ST_TOTAL, ST_ZERO_IN, ST_DENORMAL, ST_UNDERFLOW, ST_OVERFLOW, ST_NAN, ST_INF_IN = range(256, 263)
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (OpenMP over independent outputs only)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        subprocess.check_call(["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-fopenmp", "-Wall",
+                               "-o", _LIB, _SRC, "-lm"])
+    return _LIB
+
+
+_lib: Optional[ctypes.CDLL] = None
+
+
+def _L() -> ctypes.CDLL:
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build())
+        u32, i32, i64, sz, vp = (ctypes.c_uint32, ctypes.c_int, ctypes.c_int64, ctypes.c_size_t,
+                                 ctypes.c_void_p)
+        for name in ("oracle_bias", "oracle_emax", "oracle_emin", "oracle_min_normal_log2"):
+            getattr(lib, name).argtypes = [i32]
+            getattr(lib, name).restype = i32
+        lib.oracle_min_denormal_log2.argtypes = [i32, i32]
+        lib.oracle_min_denormal_log2.restype = i32
+        lib.oracle_max_normal.argtypes = [i32, i32]
+        lib.oracle_max_normal.restype = ctypes.c_double
+        lib.oracle_scale_bits.argtypes = [u32, u32]
+        lib.oracle_scale_bits.restype = u32
+        lib.oracle_quantize_bits.argtypes = [u32, i32, i32, i32, ctypes.POINTER(ctypes.c_int)]
+        lib.oracle_quantize_bits.restype = u32
+        lib.oracle_decode_code.argtypes = [u32, i32, i32]
+        lib.oracle_decode_code.restype = u32
+        lib.oracle_encode_code.argtypes = [u32, i32, i32]
+        lib.oracle_encode_code.restype = u32
+        lib.oracle_quantize_stats.argtypes = [vp, vp, sz, i32, i32, i32, u32, vp]
+        lib.oracle_quantize_stats.restype = None
+        lib.oracle_gemm.argtypes = [vp, i64, i32, vp, i64, i32, i64, i64, i64, vp, vp]
+        lib.oracle_gemm.restype = None
+        lib.oracle_gemm_sampled.argtypes = [vp, i64, i32, vp, i64, i32, i64, vp, vp, i64, vp, vp]
+        lib.oracle_gemm_sampled.restype = None
+        lib.oracle_conv.argtypes = [i32, vp, vp, vp, vp, i64, vp, vp]
+        lib.oracle_conv.restype = None
+        _lib = lib
+    return _lib
+
+
+def _f32_bits(x: float) -> int:
+    return int(np.array([x], dtype=np.float32).view(np.uint32)[0])
+
+
+# ---- format constants -------------------------------------------------------------------------
+def bias(e: int) -> int:
+    return _L().oracle_bias(e)
+
+
+def emin(e: int) -> int:
+    return _L().oracle_emin(e)
+
+
+def emax(e: int) -> int:
+    return _L().oracle_emax(e)
+
+
+def min_denormal_log2(e: int, m: int) -> int:
+    return _L().oracle_min_denormal_log2(e, m)
+
+
+def max_normal(e: int, m: int) -> float:
+    return _L().oracle_max_normal(e, m)
+
+
+# ---- scalar entry points ----------------------------------------------------------------------
+def scale_bits(xbits: int, sbits: int) -> int:
+    return _L().oracle_scale_bits(xbits, sbits)
+
+
+def quantize_bits(ybits: int, e: int, m: int, denormals: int = 1) -> Tuple[int, int]:
+    flag = ctypes.c_int(0)
+    q = _L().oracle_quantize_bits(ybits, e, m, denormals, ctypes.byref(flag))
+    return q, flag.value
+
+
+def decode_code(code: int, e: int, m: int) -> int:
+    return _L().oracle_decode_code(code, e, m)
+
+
+def encode_code(qbits: int, e: int, m: int) -> int:
+    return _L().oracle_encode_code(qbits, e, m)
+
+
+# ---- tensors ----------------------------------------------------------------------------------
+def quantize_stats(x: np.ndarray, e: int, m: int, denormals: int = 1, loss_scale: float = 1.0,
+                   want_q: bool = True, want_stats: bool = True):
+    """Returns (q as float32 array shaped like x or None, stats as uint64[264] or None)."""
+    xf = np.ascontiguousarray(x, dtype=np.float32)
+    xb = xf.view(np.uint32).reshape(-1)
+    q = np.empty_like(xb) if want_q else None
+    st = np.zeros(STATS_WORDS, dtype=np.uint64) if want_stats else None
+    _L().oracle_quantize_stats(xb.ctypes.data, q.ctypes.data if want_q else None, xb.size, e, m,
+                               int(denormals), _f32_bits(loss_scale),
+                               st.ctypes.data if want_stats else None)
+    return (q.view(np.float32).reshape(xf.shape) if want_q else None), st
+
+
+def _mat(a: np.ndarray) -> np.ndarray:
+    a = np.ascontiguousarray(a, dtype=np.float32)
+    assert a.ndim == 2
+    return a
+
+
+def gemm(A: np.ndarray, B: np.ndarray, transA: bool = False, transB: bool = False):
+    """C = op(A) op(B) in fp64 and T = |op(A)||op(B)|; A, B are the STORED row-major matrices."""
+    A, B = _mat(A), _mat(B)
+    M, K = (A.shape[1], A.shape[0]) if transA else A.shape
+    K2, N = (B.shape[1], B.shape[0]) if transB else B.shape
+    assert K == K2
+    C = np.empty((M, N), dtype=np.float64)
+    T = np.empty((M, N), dtype=np.float64)
+    _L().oracle_gemm(A.ctypes.data, A.shape[1], int(transA), B.ctypes.data, B.shape[1], int(transB),
+                     M, N, K, C.ctypes.data, T.ctypes.data)
+    return C, T
+
+
+def gemm_sampled(A: np.ndarray, B: np.ndarray, ii: np.ndarray, jj: np.ndarray,
+                 transA: bool = False, transB: bool = False):
+    A, B = _mat(A), _mat(B)
+    K = A.shape[0] if transA else A.shape[1]
+    ii = np.ascontiguousarray(ii, dtype=np.int64)
+    jj = np.ascontiguousarray(jj, dtype=np.int64)
+    c = np.empty(ii.size, dtype=np.float64)
+    t = np.empty(ii.size, dtype=np.float64)
+    _L().oracle_gemm_sampled(A.ctypes.data, A.shape[1], int(transA), B.ctypes.data, B.shape[1],
+                             int(transB), K, ii.ctypes.data, jj.ctypes.data, ii.size, c.ctypes.data,
+                             t.ctypes.data)
+    return c, t
+
+
+CONV_FWD, CONV_DGRAD, CONV_WGRAD = 0, 1, 2
+
+
+def conv(which: int, P: np.ndarray, Q: np.ndarray, geom, idx: Optional[np.ndarray] = None):
+    """Direct convolution definitions on NCHW tensors.
+
+    geom = (n, ci, h, w, co, r, s, pad_h, pad_w).  Operands (P, Q): forward (X, W); data
+    gradient (dY, W); filter gradient (dY, X).  Returns (c, t) as flat fp64 arrays over the
+    output tensor ([n][co][oh][ow], [n][ci][h][w] or [co][ci][r][s]) or over ``idx``.
+    """
+    n, ci, h, w, co, r, s, ph, pw = [int(v) for v in geom]
+    oh, ow = h + 2 * ph - r + 1, w + 2 * pw - s + 1
+    total = {CONV_FWD: n * co * oh * ow, CONV_DGRAD: n * ci * h * w, CONV_WGRAD: co * ci * r * s}[which]
+    P = np.ascontiguousarray(P, dtype=np.float32)
+    Q = np.ascontiguousarray(Q, dtype=np.float32)
+    g = np.array([n, ci, h, w, co, r, s, ph, pw], dtype=np.int64)
+    if idx is not None:
+        idx = np.ascontiguousarray(idx, dtype=np.int64)
+        count = idx.size
+    else:
+        count = total
+    c = np.empty(count, dtype=np.float64)
+    t = np.empty(count, dtype=np.float64)
+    _L().oracle_conv(which, g.ctypes.data, P.ctypes.data, Q.ctypes.data,
+                     idx.ctypes.data if idx is not None else None, count, c.ctypes.data, t.ctypes.data)
+    return c, t

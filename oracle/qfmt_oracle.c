@@ -1,0 +1,410 @@
+/*
+ * CPU oracle for emulated 1/e/m floating-point training arithmetic.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the plain, slow reference the CUDA library is
+ * checked against.  It shares no code, header, table or helper with the CUDA path, and only
+ * tests, the smoke check and the benchmark's CPU-baseline leg may call it.
+ *
+ * What it follows (arXiv 2103.15940):
+ *   - Definition III.1, Eq. (1): a value is x = M * 2^(E-p+1) with E_min <= E <= E_max and an
+ *     integer significand M; normal numbers have |x| >= 2^E_min, all others are denormal with
+ *     E = E_min.
+ *   - Definition III.2: a format is 1/e/m/d with e exponent bits, m stored mantissa bits, and
+ *     "d" (denormals kept) or "n" (denormals flushed to zero).
+ *   - Table I: bias 2^(e-1)-1 gives E_min = 1-bias, E_max = bias, smallest denormal
+ *     2^(E_min-m).  The all-ones stored exponent field is reserved for inf/NaN and the
+ *     all-zero field for zero/denormals (Section III's list of special encodings, read the
+ *     IEEE way so that Table I's E_max stays the largest finite exponent).
+ *   - Section IV-A: roundfp rounds each element to the nearest representable value
+ *     (ties go to the even significand, the IEEE default), with e <= 8 and m <= 23.
+ *   - Section II: loss scaling multiplies the tensors by a factor before they are rounded.
+ *   - Section III-B: FMACS, a32 = round(a32 + x16*y16): exact products, wide accumulation.
+ *     The contraction is order dependent in fp32, so the oracle gives the exact result
+ *     (fp64 accumulation of exact products) together with sum |a||b| for the error bound.
+ *   - Section V: "denormal fraction" of each tensor is the logged statistic.
+ *
+ * Every number here is handled as an integer significand times a power of two.
+ *
+ * Pins: tests/test_oracle_*.py (all "not gpu").  FTZ-mode variants and formats other than
+ * 1/5/10, 1/8/7, 1/6/9 and 1/8/23 are pinned only by the brute-force invariants
+ * ("parity unpinned" beyond those).
+ */
+#include <math.h>
+#include <stddef.h>
+#include <stdint.h>
+#include <string.h>
+
+/* ------------------------------------------------------------------------------------------ */
+/* Format constants (Table I).                                                                  */
+/* ------------------------------------------------------------------------------------------ */
+int oracle_bias(int e) { return (1 << (e - 1)) - 1; }
+int oracle_emax(int e) { return oracle_bias(e); }
+int oracle_emin(int e) { return 1 - oracle_bias(e); }
+/* exponents of two of the smallest normal / smallest denormal */
+int oracle_min_normal_log2(int e) { return oracle_emin(e); }
+int oracle_min_denormal_log2(int e, int m) { return oracle_emin(e) - m; }
+/* largest normal = (2 - 2^-m) * 2^Emax, returned as a double (exact) */
+double oracle_max_normal(int e, int m) { return ldexp(2.0 - ldexp(1.0, -m), oracle_emax(e)); }
+
+/* ------------------------------------------------------------------------------------------ */
+/* A finite nonnegative magnitude as  sig * 2^exp2  (sig a 64-bit integer).                     */
+/* ------------------------------------------------------------------------------------------ */
+typedef struct {
+    uint64_t sig;
+    int exp2;
+} mag_t;
+
+/* classes of an fp32 word */
+enum { CLS_ZERO = 0, CLS_FINITE = 1, CLS_INF = 2, CLS_NAN = 3 };
+
+/* Decode an fp32 bit pattern: sign, class, and for finite nonzero values sig*2^exp2 exactly. */
+static int decode_f32(uint32_t u, int *sign, mag_t *mg) {
+    uint32_t E = (u >> 23) & 0xFFu, f = u & 0x7FFFFFu;
+    *sign = (int)(u >> 31);
+    mg->sig = 0;
+    mg->exp2 = 0;
+    if (E == 255) return f ? CLS_NAN : CLS_INF;
+    if (E == 0) {
+        if (f == 0) return CLS_ZERO;
+        mg->sig = f; /* fp32 denormal: f * 2^-149 */
+        mg->exp2 = -149;
+        return CLS_FINITE;
+    }
+    mg->sig = (uint64_t)f | 0x800000u; /* (2^23 + f) * 2^(E-150) */
+    mg->exp2 = (int)E - 150;
+    return CLS_FINITE;
+}
+
+static int floor_log2_u64(uint64_t v) { /* v > 0 */
+    int b = -1;
+    while (v) {
+        v >>= 1;
+        ++b;
+    }
+    return b;
+}
+
+/*
+ * Round the exact magnitude sig*2^exp2 (sig > 0) to the nearest value of format (e, m) with
+ * denormals, ties to even.  Result: Q * 2^g, where g is the exponent of the unit in the last
+ * place that applies at this magnitude: g = max(floor(log2 v), E_min) - m.  Q may come out as
+ * 2^(m+1) (carry into the next binade) or 0 (rounded to zero).  *is_inf is set when the rounded
+ * value reaches 2^(E_max+1), i.e. exceeds the largest normal.
+ */
+static mag_t round_to_format(mag_t v, int e, int m, int *is_inf) {
+    int emin = oracle_emin(e), emax = oracle_emax(e);
+    int lg = floor_log2_u64(v.sig) + v.exp2;       /* floor(log2 value) */
+    int g = (lg > emin ? lg : emin) - m;           /* quantum exponent */
+    int r = g - v.exp2;                            /* bits to drop (may be <= 0: exact) */
+    mag_t q;
+    q.exp2 = g;
+    *is_inf = 0;
+    if (r <= 0) {
+        q.sig = v.sig << (-r); /* already on the grid; callers keep sig small enough */
+    } else if (r >= 64) {
+        q.sig = 0; /* value is below a quarter of the quantum */
+    } else {
+        uint64_t keep = v.sig >> r;
+        uint64_t rem = v.sig & (((uint64_t)1 << r) - 1);
+        uint64_t half = (uint64_t)1 << (r - 1);
+        if (rem > half || (rem == half && (keep & 1))) keep += 1;
+        q.sig = keep;
+    }
+    if (q.sig != 0) {
+        int top = floor_log2_u64(q.sig) + q.exp2;
+        if (top > emax) *is_inf = 1;
+    }
+    return q;
+}
+
+/* Encode a finite magnitude Q*2^g (already a value of format (8,23) or coarser) as fp32 bits. */
+static uint32_t encode_f32_mag(mag_t q) {
+    if (q.sig == 0) return 0;
+    int top = floor_log2_u64(q.sig);
+    int lg = top + q.exp2;
+    if (lg < -126) { /* fp32 denormal: multiple of 2^-149 */
+        int sh = q.exp2 + 149;
+        uint64_t f = sh >= 0 ? (q.sig << sh) : (q.sig >> (-sh));
+        return (uint32_t)f;
+    }
+    uint64_t s24 = top >= 23 ? (q.sig >> (top - 23)) : (q.sig << (23 - top));
+    return ((uint32_t)(lg + 127) << 23) | (uint32_t)(s24 & 0x7FFFFFu);
+}
+
+/* ------------------------------------------------------------------------------------------ */
+/* Loss scale (Section II): y = fl32(x * S), IEEE single multiply, RNE, denormals honoured.     */
+/* ------------------------------------------------------------------------------------------ */
+uint32_t oracle_scale_bits(uint32_t xbits, uint32_t sbits) {
+    int sx, ss;
+    mag_t mx, ms;
+    int cx = decode_f32(xbits, &sx, &mx), cs = decode_f32(sbits, &ss, &ms);
+    uint32_t sign = (uint32_t)(sx ^ ss) << 31;
+    if (cx == CLS_NAN || cs == CLS_NAN) return sign | 0x7FC00000u;
+    if ((cx == CLS_INF && cs == CLS_ZERO) || (cx == CLS_ZERO && cs == CLS_INF)) return 0x7FC00000u;
+    if (cx == CLS_INF || cs == CLS_INF) return sign | 0x7F800000u;
+    if (cx == CLS_ZERO || cs == CLS_ZERO) return sign;
+    mag_t p;
+    p.sig = mx.sig * ms.sig; /* < 2^48, exact */
+    p.exp2 = mx.exp2 + ms.exp2;
+    int inf;
+    mag_t q = round_to_format(p, 8, 23, &inf);
+    if (inf) return sign | 0x7F800000u;
+    return sign | encode_f32_mag(q);
+}
+
+/* ------------------------------------------------------------------------------------------ */
+/* Quantize one fp32 word to 1/e/m (Section IV-A roundfp), result kept in an fp32 container.    */
+/* *was_denormal: the rounded value, before any flush, is a nonzero denormal of the format.     */
+/* ------------------------------------------------------------------------------------------ */
+uint32_t oracle_quantize_bits(uint32_t ybits, int e, int m, int keep_denormals, int *was_denormal) {
+    int s;
+    mag_t v;
+    int cls = decode_f32(ybits, &s, &v);
+    uint32_t sign = (uint32_t)s << 31;
+    if (was_denormal) *was_denormal = 0;
+    if (cls == CLS_NAN) return sign | 0x7FC00000u;
+    if (cls == CLS_INF) return sign | 0x7F800000u;
+    if (cls == CLS_ZERO) return sign;
+    int inf;
+    mag_t q = round_to_format(v, e, m, &inf);
+    if (inf) return sign | 0x7F800000u;
+    if (q.sig == 0) return sign;
+    /* below 2^E_min  <=>  Q < 2^m at the denormal quantum */
+    int is_den = (floor_log2_u64(q.sig) + q.exp2) < oracle_emin(e);
+    if (was_denormal) *was_denormal = is_den;
+    if (is_den && !keep_denormals) return sign; /* flushed formats: denormals become zero */
+    return sign | encode_f32_mag(q);
+}
+
+/* ------------------------------------------------------------------------------------------ */
+/* Packed (1+e+m)-bit encodings: sign | stored exponent | mantissa (used for brute force).      */
+/* ------------------------------------------------------------------------------------------ */
+/* Value of a packed code as fp32 bits (Eq. (1) plus the special encodings). */
+uint32_t oracle_decode_code(uint32_t code, int e, int m) {
+    uint32_t sign = (code >> (e + m)) & 1u;
+    uint32_t E = (code >> m) & ((1u << e) - 1u);
+    uint32_t f = code & ((1u << m) - 1u);
+    uint32_t sb = sign << 31;
+    if (E == (1u << e) - 1u) return f ? (sb | 0x7FC00000u) : (sb | 0x7F800000u);
+    mag_t q;
+    if (E == 0) {
+        q.sig = f;
+        q.exp2 = oracle_emin(e) - m;
+    } else {
+        q.sig = ((uint64_t)1 << m) | f;
+        q.exp2 = (int)E - oracle_bias(e) - m;
+    }
+    return sb | encode_f32_mag(q);
+}
+
+/* Packed code of an fp32 word that already holds a value of format (e, m). */
+uint32_t oracle_encode_code(uint32_t qbits, int e, int m) {
+    int s;
+    mag_t v;
+    int cls = decode_f32(qbits, &s, &v);
+    uint32_t sb = (uint32_t)s << (e + m);
+    uint32_t top = ((1u << e) - 1u) << m;
+    if (cls == CLS_NAN) return sb | top | (1u << (m - 1));
+    if (cls == CLS_INF) return sb | top;
+    if (cls == CLS_ZERO) return sb;
+    int lg = floor_log2_u64(v.sig) + v.exp2;
+    int emin = oracle_emin(e);
+    if (lg < emin) { /* denormal: mantissa = value / 2^(emin-m) */
+        int sh = v.exp2 - (emin - m);
+        uint64_t f = sh >= 0 ? (v.sig << sh) : (v.sig >> (-sh));
+        return sb | (uint32_t)f;
+    }
+    int sh = v.exp2 - (lg - m);
+    uint64_t sig = sh >= 0 ? (v.sig << sh) : (v.sig >> (-sh));
+    return sb | ((uint32_t)(lg + oracle_bias(e)) << m) | (uint32_t)(sig & (((uint64_t)1 << m) - 1));
+}
+
+/* ------------------------------------------------------------------------------------------ */
+/* Statistics record: 256 histogram bins followed by 8 counters (all 64-bit).                   */
+/* ------------------------------------------------------------------------------------------ */
+enum {
+    ST_TOTAL = 256, ST_ZERO_IN, ST_DENORMAL, ST_UNDERFLOW, ST_OVERFLOW, ST_NAN, ST_INF_IN, ST_RESERVED,
+    ST_WORDS
+};
+
+/* Stored exponent field of a quantized value: 0 zero/denormal, 1..2^e-2 normal, 2^e-1 inf/NaN. */
+static int exponent_code(uint32_t qbits, int e) {
+    int s;
+    mag_t v;
+    int cls = decode_f32(qbits, &s, &v);
+    if (cls == CLS_NAN || cls == CLS_INF) return (1 << e) - 1;
+    if (cls == CLS_ZERO) return 0;
+    int lg = floor_log2_u64(v.sig) + v.exp2;
+    if (lg < oracle_emin(e)) return 0;
+    return lg + oracle_bias(e);
+}
+
+/*
+ * Quantize n elements (after the loss-scale multiply) and count, one element at a time.
+ * q may be NULL (statistics only); stats may be NULL.  stats[] is ADDED to (caller zeroes).
+ */
+void oracle_quantize_stats(const uint32_t *x, uint32_t *q, size_t n, int e, int m, int keep_denormals,
+                           uint32_t scale_bits, uint64_t *stats) {
+    for (size_t i = 0; i < n; ++i) {
+        uint32_t xb = x[i];
+        uint32_t yb = (scale_bits == 0x3F800000u) ? xb : oracle_scale_bits(xb, scale_bits);
+        int was_den;
+        uint32_t qb = oracle_quantize_bits(yb, e, m, keep_denormals, &was_den);
+        if (q) q[i] = qb;
+        if (!stats) continue;
+        int sx;
+        mag_t mx;
+        int cx = decode_f32(xb, &sx, &mx);
+        int q_zero = (qb & 0x7FFFFFFFu) == 0;
+        int q_inf = (qb & 0x7FFFFFFFu) == 0x7F800000u;
+        stats[exponent_code(qb, e)] += 1;
+        stats[ST_TOTAL] += 1;
+        if (cx == CLS_ZERO) stats[ST_ZERO_IN] += 1;
+        if (cx == CLS_NAN) stats[ST_NAN] += 1;
+        if (cx == CLS_INF) stats[ST_INF_IN] += 1;
+        if (was_den) stats[ST_DENORMAL] += 1;
+        if (cx == CLS_FINITE && q_zero) stats[ST_UNDERFLOW] += 1;
+        if ((cx == CLS_FINITE || cx == CLS_ZERO) && q_inf) stats[ST_OVERFLOW] += 1;
+    }
+}
+
+/* ------------------------------------------------------------------------------------------ */
+/* Contractions (Section III-B, FMACS): exact products summed in fp64 in plain k order, with    */
+/* t = sum |a||b| beside each output for the accumulation-error bound.                          */
+/* Matrices are fp32, row-major with a leading dimension; trans != 0 reads the stored matrix    */
+/* transposed, so op(A) is M x K and op(B) is K x N.                                            */
+/* ------------------------------------------------------------------------------------------ */
+static double elemA(const float *A, int64_t lda, int transA, int64_t i, int64_t k) {
+    return transA ? (double)A[k * lda + i] : (double)A[i * lda + k];
+}
+static double elemB(const float *B, int64_t ldb, int transB, int64_t k, int64_t j) {
+    return transB ? (double)B[j * ldb + k] : (double)B[k * ldb + j];
+}
+
+static void dot_ab(const float *A, int64_t lda, int transA, const float *B, int64_t ldb, int transB,
+                   int64_t K, int64_t i, int64_t j, double *c, double *t) {
+    double acc = 0.0, abs_acc = 0.0;
+    for (int64_t k = 0; k < K; ++k) {
+        double a = elemA(A, lda, transA, i, k), b = elemB(B, ldb, transB, k, j);
+        acc += a * b;
+        abs_acc += fabs(a) * fabs(b);
+    }
+    *c = acc;
+    if (t) *t = abs_acc;
+}
+
+/* Full output: C and T are M x N fp64, dense row-major.  T may be NULL. */
+void oracle_gemm(const float *A, int64_t lda, int transA, const float *B, int64_t ldb, int transB,
+                 int64_t M, int64_t N, int64_t K, double *C, double *T) {
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < M; ++i)
+        for (int64_t j = 0; j < N; ++j)
+            dot_ab(A, lda, transA, B, ldb, transB, K, i, j, &C[i * N + j], T ? &T[i * N + j] : NULL);
+}
+
+/* Sampled outputs: c[s], t[s] for the pairs (ii[s], jj[s]). */
+void oracle_gemm_sampled(const float *A, int64_t lda, int transA, const float *B, int64_t ldb, int transB,
+                         int64_t K, const int64_t *ii, const int64_t *jj, int64_t nsamp, double *c,
+                         double *t) {
+#pragma omp parallel for schedule(static)
+    for (int64_t s = 0; s < nsamp; ++s)
+        dot_ab(A, lda, transA, B, ldb, transB, K, ii[s], jj[s], &c[s], t ? &t[s] : NULL);
+}
+
+/* ------------------------------------------------------------------------------------------ */
+/* Convolution layers (Section V: the matrix multiplies at the core of convolution layers),     */
+/* written as the direct definition on NCHW tensors: unit stride, zero padding, cross-          */
+/* correlation as deep-learning frameworks define it.                                            */
+/*   X [n][ci][h][w],  W [co][ci][r][s],  Y [n][co][oh][ow],  oh = h + 2*pad_h - r + 1.          */
+/* ------------------------------------------------------------------------------------------ */
+typedef struct {
+    int64_t n, ci, h, w, co, r, s, pad_h, pad_w;
+} conv_t;
+
+static int64_t conv_oh(const conv_t *g) { return g->h + 2 * g->pad_h - g->r + 1; }
+static int64_t conv_ow(const conv_t *g) { return g->w + 2 * g->pad_w - g->s + 1; }
+
+/* forward: Y[n,co,oh,ow] = sum_{ci,r,s} X[n,ci,oh+r-pad,ow+s-pad] * W[co,ci,r,s] */
+static void conv_fwd_one(const conv_t *g, const float *X, const float *Wt, int64_t n, int64_t co,
+                         int64_t oh, int64_t ow, double *c, double *t) {
+    double acc = 0.0, abs_acc = 0.0;
+    for (int64_t ci = 0; ci < g->ci; ++ci)
+        for (int64_t r = 0; r < g->r; ++r)
+            for (int64_t s = 0; s < g->s; ++s) {
+                int64_t ih = oh + r - g->pad_h, iw = ow + s - g->pad_w;
+                if (ih < 0 || ih >= g->h || iw < 0 || iw >= g->w) continue;
+                double a = X[((n * g->ci + ci) * g->h + ih) * g->w + iw];
+                double b = Wt[((co * g->ci + ci) * g->r + r) * g->s + s];
+                acc += a * b;
+                abs_acc += fabs(a) * fabs(b);
+            }
+    *c = acc;
+    if (t) *t = abs_acc;
+}
+
+/* data gradient: dX[n,ci,ih,iw] = sum_{co,r,s} dY[n,co,ih-r+pad,iw-s+pad] * W[co,ci,r,s] */
+static void conv_dgrad_one(const conv_t *g, const float *dY, const float *Wt, int64_t n, int64_t ci,
+                           int64_t ih, int64_t iw, double *c, double *t) {
+    int64_t OH = conv_oh(g), OW = conv_ow(g);
+    double acc = 0.0, abs_acc = 0.0;
+    for (int64_t co = 0; co < g->co; ++co)
+        for (int64_t r = 0; r < g->r; ++r)
+            for (int64_t s = 0; s < g->s; ++s) {
+                int64_t oh = ih - r + g->pad_h, ow = iw - s + g->pad_w;
+                if (oh < 0 || oh >= OH || ow < 0 || ow >= OW) continue;
+                double a = dY[((n * g->co + co) * OH + oh) * OW + ow];
+                double b = Wt[((co * g->ci + ci) * g->r + r) * g->s + s];
+                acc += a * b;
+                abs_acc += fabs(a) * fabs(b);
+            }
+    *c = acc;
+    if (t) *t = abs_acc;
+}
+
+/* filter gradient: dW[co,ci,r,s] = sum_{n,oh,ow} dY[n,co,oh,ow] * X[n,ci,oh+r-pad,ow+s-pad] */
+static void conv_wgrad_one(const conv_t *g, const float *dY, const float *X, int64_t co, int64_t ci,
+                           int64_t r, int64_t s, double *c, double *t) {
+    int64_t OH = conv_oh(g), OW = conv_ow(g);
+    double acc = 0.0, abs_acc = 0.0;
+    for (int64_t n = 0; n < g->n; ++n)
+        for (int64_t oh = 0; oh < OH; ++oh)
+            for (int64_t ow = 0; ow < OW; ++ow) {
+                int64_t ih = oh + r - g->pad_h, iw = ow + s - g->pad_w;
+                if (ih < 0 || ih >= g->h || iw < 0 || iw >= g->w) continue;
+                double a = dY[((n * g->co + co) * OH + oh) * OW + ow];
+                double b = X[((n * g->ci + ci) * g->h + ih) * g->w + iw];
+                acc += a * b;
+                abs_acc += fabs(a) * fabs(b);
+            }
+    *c = acc;
+    if (t) *t = abs_acc;
+}
+
+/*
+ * which: 0 forward (output index space [n][co][oh][ow]), 1 data gradient ([n][ci][h][w]),
+ * 2 filter gradient ([co][ci][r][s]).  P and Q are the two operands in the order of the
+ * formulas above: (X, W), (dY, W), (dY, X).  idx holds flat indices into the output tensor;
+ * idx == NULL means all outputs 0..count-1.
+ */
+void oracle_conv(int which, const int64_t *geom, const float *P, const float *Q, const int64_t *idx,
+                 int64_t count, double *c, double *t) {
+    conv_t g;
+    g.n = geom[0]; g.ci = geom[1]; g.h = geom[2]; g.w = geom[3]; g.co = geom[4];
+    g.r = geom[5]; g.s = geom[6]; g.pad_h = geom[7]; g.pad_w = geom[8];
+    int64_t OH = conv_oh(&g), OW = conv_ow(&g);
+#pragma omp parallel for schedule(static)
+    for (int64_t k = 0; k < count; ++k) {
+        int64_t f = idx ? idx[k] : k;
+        double *tk = t ? &t[k] : NULL;
+        if (which == 0) {
+            int64_t ow = f % OW, oh = (f / OW) % OH, co = (f / (OW * OH)) % g.co, n = f / (OW * OH * g.co);
+            conv_fwd_one(&g, P, Q, n, co, oh, ow, &c[k], tk);
+        } else if (which == 1) {
+            int64_t iw = f % g.w, ih = (f / g.w) % g.h, ci = (f / (g.w * g.h)) % g.ci, n = f / (g.w * g.h * g.ci);
+            conv_dgrad_one(&g, P, Q, n, ci, ih, iw, &c[k], tk);
+        } else {
+            int64_t s = f % g.s, r = (f / g.s) % g.r, ci = (f / (g.s * g.r)) % g.ci, co = f / (g.s * g.r * g.ci);
+            conv_wgrad_one(&g, P, Q, co, ci, r, s, &c[k], tk);
+        }
+    }
+}
