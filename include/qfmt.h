@@ -1,0 +1,114 @@
+/*
+ * qfmt — emulated 16-bit floating-point formats for mixed-precision training on one B200.
+ *
+ * C ABI of the hot path of "Representation range needs for 16-bit neural network training"
+ * (arXiv 2103.15940): rounding fp32 tensors to a 1/e/m/{d,n} format while recording range
+ * statistics, and contracting the rounded operands with wide accumulation.
+ *
+ * General rules
+ *   - Pointers named d_* are DEVICE pointers, h_* are HOST pointers.  Every buffer is
+ *     allocated, owned and freed by the caller; the library allocates no memory.
+ *   - All GPU work is enqueued on `stream` (a cudaStream_t passed as void*, NULL = default
+ *     stream) and the calls return without synchronising unless stated otherwise.
+ *   - Every function returns a qfmt_status_t (0 = success, negative = error); nothing throws,
+ *     prints or exits.  An error return means no GPU work was enqueued by that call.
+ *   - The device must be of compute capability 10.x (built for sm_100a).
+ */
+#ifndef QFMT_H_
+#define QFMT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    QFMT_OK = 0,
+    QFMT_ERR_BAD_FORMAT = -1,  /* e, m, rounding or loss_scale outside the supported domain   */
+    QFMT_ERR_BAD_ARG = -2,     /* NULL/misaligned pointer, bad dimension, workspace too small  */
+    QFMT_ERR_UNSUPPORTED_ARCH = -3, /* current device is not compute capability 10.x           */
+    QFMT_ERR_CUDA = -4,        /* a CUDA runtime/driver call failed (see qfmt_last_cuda_error)  */
+    QFMT_ERR_TIMEOUT = -5      /* a bounded device-side wait expired (reported via status word) */
+} qfmt_status_t;
+
+/*
+ * A floating-point system s/e/p/d in the sense of Definition III.2 with s = 1:
+ * e exponent bits, m explicitly stored mantissa bits (Table I's column "p"), and denormals
+ * kept ("d") or flushed to zero ("n").  Bias is 2^(e-1)-1, so E_min = 1-bias, E_max = bias and
+ * the smallest denormal is 2^(E_min-m) (Table I); the all-ones exponent field is inf/NaN.
+ * Section IV-A fixes the domain of the rounding kernel: e <= 8, m <= 23.
+ */
+typedef struct {
+    int32_t e;          /* exponent bits, 2..8                                               */
+    int32_t m;          /* stored mantissa bits, 1..23 (qfmt_gemm requires m <= 10)          */
+    int32_t denormals;  /* 1 = keep denormals ("d"), 0 = flush them to signed zero ("n")     */
+    int32_t rounding;   /* 0 = round to nearest, ties to even; any other value is rejected   */
+    float loss_scale;   /* finite and > 0; tensors are multiplied by it before rounding      */
+} qfmt_format_t;
+
+/*
+ * Per-tensor range statistics (Section V: the fraction of denormal elements of every layer's
+ * activations, weights and activation gradients is what the paper logs and tabulates).
+ * hist[c] counts elements by the stored exponent field c of the ROUNDED value in the target
+ * format: c = 0 zero or denormal, 1 .. 2^e-2 one bin per binade of normal numbers,
+ * 2^e-1 inf or NaN; bins >= 2^e stay zero.
+ *   n_total     elements seen
+ *   n_zero_in   inputs that are +-0
+ *   n_denormal  elements whose rounded value, before any flush, is a nonzero denormal of the
+ *               format (with denormals flushed these are exactly the flushed elements)
+ *   n_underflow finite nonzero inputs whose final result is +-0
+ *   n_overflow  finite inputs whose final result is +-inf
+ *   n_nan, n_inf_in  NaN / infinite inputs
+ * The record lives in device memory.
+ */
+typedef struct {
+    uint64_t hist[256];
+    uint64_t n_total, n_zero_in, n_denormal, n_underflow, n_overflow, n_nan, n_inf_in, reserved;
+} qfmt_stats_t;
+
+/*
+ * Round n fp32 elements to format *fmt (Section IV-A, the roundfp operation) after
+ * multiplying each by fmt->loss_scale in IEEE single precision (Section II, loss scaling),
+ * and record the range statistics of the result in the same pass.
+ *
+ *   d_in     device, n floats, 4-byte aligned (16-byte alignment of d_in and d_out, or equal
+ *            misalignment of the two, selects the 128-bit path; otherwise a scalar path runs)
+ *   d_out    device, n floats; receives the rounded values in fp32 containers (the low 23-m
+ *            mantissa bits are zero).  May equal d_in (in place) or be NULL (statistics only).
+ *            Partial overlap with d_in is an error the library cannot detect.
+ *   fmt      host pointer, read during the call
+ *   d_stats  device, 8-byte aligned, or NULL for no statistics
+ *   accumulate  0: the record is cleared first; 1: counts are added to what it holds
+ *
+ * Overflow gives +-inf, NaN gives a quiet NaN with the input's sign, zeros and flushed or
+ * underflowed results keep their sign.  n = 0 is valid (with accumulate = 0 it clears the
+ * record).  The result is deterministic (integer counting only).
+ * Errors: QFMT_ERR_BAD_FORMAT, QFMT_ERR_BAD_ARG, QFMT_ERR_UNSUPPORTED_ARCH, QFMT_ERR_CUDA.
+ */
+int qfmt_quantize_stats(const float* d_in, float* d_out, size_t n, const qfmt_format_t* fmt,
+                        qfmt_stats_t* d_stats, int accumulate, void* stream);
+
+/*
+ * The same operation on HOST buffers: copies h_in to the device, runs the kernel, copies the
+ * rounded tensor (if h_out != NULL) and the statistics (if h_stats != NULL) back, and
+ * SYNCHRONISES the stream before returning.  The caller lends device scratch:
+ *   d_work   device, 16-byte aligned, at least qfmt_quantize_stats_host_work_bytes(n) bytes
+ * For full copy speed h_in / h_out should be page-locked.  h_stats is overwritten.
+ */
+int qfmt_quantize_stats_host(const float* h_in, float* h_out, size_t n, const qfmt_format_t* fmt,
+                             qfmt_stats_t* h_stats, void* d_work, size_t work_bytes, void* stream);
+size_t qfmt_quantize_stats_host_work_bytes(size_t n);
+
+/* Last CUDA error code (cudaError_t as int) seen by a call that returned QFMT_ERR_CUDA. */
+int qfmt_last_cuda_error(void);
+/* Static, NUL-terminated description of a status code. */
+const char* qfmt_status_string(int status);
+/* Library version: major * 10000 + minor * 100 + patch. */
+int qfmt_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* QFMT_H_ */

@@ -1,0 +1,139 @@
+"""Python binding of the qfmt C-ABI library (``include/qfmt.h``).
+
+Argument marshalling only: every step of the path runs in the CUDA kernels of ``libqfmt.so``.
+PyTorch is used by callers for device memory and streams; this module accepts torch tensors
+or raw integer addresses.  There is no CPU fallback: if the shared library cannot be loaded,
+the first call raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libqfmt.so")
+
+QFMT_OK = 0
+QFMT_ERR_BAD_FORMAT = -1
+QFMT_ERR_BAD_ARG = -2
+QFMT_ERR_UNSUPPORTED_ARCH = -3
+QFMT_ERR_CUDA = -4
+QFMT_ERR_TIMEOUT = -5
+
+STATS_WORDS = 264  # 256 histogram bins + 8 counters, all uint64
+(ST_TOTAL, ST_ZERO_IN, ST_DENORMAL, ST_UNDERFLOW, ST_OVERFLOW, ST_NAN, ST_INF_IN) = range(256, 263)
+
+
+class QfmtError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        msg = lib().qfmt_status_string(status).decode()
+        if status == QFMT_ERR_CUDA:
+            msg += f" (cudaError {lib().qfmt_last_cuda_error()})"
+        super().__init__(f"{where}: {msg} [{status}]")
+
+
+class qfmt_format_t(ctypes.Structure):
+    _fields_ = [("e", ctypes.c_int32), ("m", ctypes.c_int32), ("denormals", ctypes.c_int32),
+                ("rounding", ctypes.c_int32), ("loss_scale", ctypes.c_float)]
+
+
+class qfmt_stats_t(ctypes.Structure):
+    _fields_ = [("hist", ctypes.c_uint64 * 256), ("n_total", ctypes.c_uint64),
+                ("n_zero_in", ctypes.c_uint64), ("n_denormal", ctypes.c_uint64),
+                ("n_underflow", ctypes.c_uint64), ("n_overflow", ctypes.c_uint64),
+                ("n_nan", ctypes.c_uint64), ("n_inf_in", ctypes.c_uint64), ("reserved", ctypes.c_uint64)]
+
+
+_lib: Optional[ctypes.CDLL] = None
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded C-ABI library; raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} is missing: build it with "
+                              "`python -m paper_2103_15940_b200.build` (there is no CPU fallback)")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, sz, ci = ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int
+        fmtp = ctypes.POINTER(qfmt_format_t)
+        L.qfmt_quantize_stats.argtypes = [vp, vp, sz, fmtp, vp, ci, vp]
+        L.qfmt_quantize_stats.restype = ci
+        L.qfmt_quantize_stats_host.argtypes = [vp, vp, sz, fmtp, vp, vp, sz, vp]
+        L.qfmt_quantize_stats_host.restype = ci
+        L.qfmt_quantize_stats_host_work_bytes.argtypes = [sz]
+        L.qfmt_quantize_stats_host_work_bytes.restype = sz
+        L.qfmt_last_cuda_error.argtypes = []
+        L.qfmt_last_cuda_error.restype = ci
+        L.qfmt_status_string.argtypes = [ci]
+        L.qfmt_status_string.restype = ctypes.c_char_p
+        L.qfmt_version.argtypes = []
+        L.qfmt_version.restype = ci
+        _bind_optional(L)
+        _lib = L
+    return _lib
+
+
+def _bind_optional(L: ctypes.CDLL) -> None:
+    """Signatures of entry points added after the first two; see include/qfmt.h."""
+    return None
+
+
+def _ptr(x) -> Optional[int]:
+    """Address of a torch tensor / numpy array / int / None."""
+    if x is None:
+        return None
+    if isinstance(x, int):
+        return x
+    if hasattr(x, "data_ptr"):
+        return x.data_ptr()
+    if hasattr(x, "ctypes"):
+        return x.ctypes.data
+    raise TypeError(type(x))
+
+
+def _stream_handle(stream) -> Optional[int]:
+    if stream is None:
+        import torch
+        return torch.cuda.current_stream().cuda_stream
+    if isinstance(stream, int):
+        return stream
+    return stream.cuda_stream
+
+
+def make_format(e: int, m: int, denormals: int = 1, loss_scale: float = 1.0, rounding: int = 0) -> qfmt_format_t:
+    return qfmt_format_t(int(e), int(m), int(denormals), int(rounding), float(loss_scale))
+
+
+def _check(status: int, where: str) -> None:
+    if status != QFMT_OK:
+        raise QfmtError(status, where)
+
+
+def qfmt_quantize_stats(d_in, d_out, n: int, fmt: qfmt_format_t, d_stats=None, accumulate: int = 0,
+                        stream=None) -> None:
+    """Device buffers in, device buffers out; see qfmt_quantize_stats in include/qfmt.h."""
+    _check(lib().qfmt_quantize_stats(_ptr(d_in), _ptr(d_out), int(n), ctypes.byref(fmt), _ptr(d_stats),
+                                     int(accumulate), _stream_handle(stream)), "qfmt_quantize_stats")
+
+
+def qfmt_quantize_stats_host_work_bytes(n: int) -> int:
+    return int(lib().qfmt_quantize_stats_host_work_bytes(int(n)))
+
+
+def qfmt_quantize_stats_host(h_in, h_out, n: int, fmt: qfmt_format_t, h_stats, d_work, work_bytes: int,
+                             stream=None) -> None:
+    """Host buffers in and out (copies inside the call); see include/qfmt.h."""
+    _check(lib().qfmt_quantize_stats_host(_ptr(h_in), _ptr(h_out), int(n), ctypes.byref(fmt), _ptr(h_stats),
+                                          _ptr(d_work), int(work_bytes), _stream_handle(stream)),
+           "qfmt_quantize_stats_host")
+
+
+def qfmt_version() -> int:
+    return int(lib().qfmt_version())
+
+
+def qfmt_status_string(status: int) -> str:
+    return lib().qfmt_status_string(int(status)).decode()
