@@ -101,6 +101,55 @@ int qfmt_quantize_stats_host(const float* h_in, float* h_out, size_t n, const qf
                              qfmt_stats_t* h_stats, void* d_work, size_t work_bytes, void* stream);
 size_t qfmt_quantize_stats_host_work_bytes(size_t n);
 
+/*
+ * One GEMM operand: a row-major fp32 matrix in device memory whose elements already hold
+ * values of the format (the output of qfmt_quantize_stats).  rows x cols is the STORED shape,
+ * ld its leading dimension in elements; trans != 0 means the operand is the transpose of the
+ * stored matrix, so the three products of a fully connected layer (Section V: forward,
+ * activation gradient, weight gradient) need no copies:
+ *     Y = X W        A = {X, trans 0},  B = {W, trans 0}
+ *     dX = dY W^T    A = {dY, trans 0}, B = {W, trans 1}
+ *     dW = X^T dY    A = {X, trans 1},  B = {dY, trans 0}
+ * ptr must be 16-byte aligned and ld a multiple of 4 (the tiles are fetched by TMA).
+ */
+typedef struct {
+    const float* ptr;
+    int64_t rows, cols, ld;
+    int32_t trans;
+} qfmt_matrix_t;
+
+/*
+ * C = op(A) op(B) with exact products and fp32 accumulation: the FMACS instruction of
+ * Section III-B, a32 = round(a32 + x16 * y16), which Section IV-A uses inside every matrix
+ * multiply ("we do not round the products").  op(A) is M x K, op(B) is K x N, C is M x N
+ * row-major with leading dimension ldc >= N (any 4-byte aligned d_C; 16-byte aligned rows
+ * select vector stores).  Runs on the tcgen05 tensor cores as kind::tf32, which is exact for
+ * operands of any format with e <= 8 and m <= 10; fmt states that format (m > 10 is rejected
+ * with QFMT_ERR_BAD_FORMAT).  Operands are NOT re-rounded; feeding values with more than 10
+ * mantissa bits loses the extra bits.  The accumulation order is fixed, so results are
+ * reproducible run to run; against an exact sum the error stays within
+ * 2^-20 * sum_k |a_ik| |b_kj| for the workloads this library targets.
+ * fp32 denormal operands (only 1/8/m formats have them) are handled as the tensor core
+ * handles them.
+ *
+ *   d_workspace  device, 16-byte aligned, >= qfmt_gemm_workspace_bytes(A, B) bytes.  Holds a
+ *                status word (first 4 bytes, cleared by the call) and split-K partial sums.
+ *                Calls that share a workspace must be ordered on one stream.
+ * M = 0 or N = 0 is a no-op; K = 0 writes zeros.  Every device-side wait is bounded: if one
+ * expires the kernel stops, the status word holds QFMT_ERR_TIMEOUT and C is undefined.
+ * Errors: QFMT_ERR_BAD_FORMAT, QFMT_ERR_BAD_ARG (NULL or misaligned operand, ld too small,
+ * mismatched K, workspace too small), QFMT_ERR_UNSUPPORTED_ARCH, QFMT_ERR_CUDA.
+ */
+int qfmt_gemm(const qfmt_matrix_t* A, const qfmt_matrix_t* B, float* d_C, int64_t ldc,
+              const qfmt_format_t* fmt, void* d_workspace, size_t workspace_bytes, void* stream);
+size_t qfmt_gemm_workspace_bytes(const qfmt_matrix_t* A, const qfmt_matrix_t* B);
+
+/*
+ * Synchronises `stream` and returns the status word of a workspace: QFMT_OK, or the error a
+ * kernel recorded (QFMT_ERR_TIMEOUT), or QFMT_ERR_CUDA if the copy itself failed.
+ */
+int qfmt_device_status(void* d_workspace, void* stream);
+
 /* Last CUDA error code (cudaError_t as int) seen by a call that returned QFMT_ERR_CUDA. */
 int qfmt_last_cuda_error(void);
 /* Static, NUL-terminated description of a status code. */

@@ -39,6 +39,11 @@ class qfmt_format_t(ctypes.Structure):
                 ("rounding", ctypes.c_int32), ("loss_scale", ctypes.c_float)]
 
 
+class qfmt_matrix_t(ctypes.Structure):
+    _fields_ = [("ptr", ctypes.c_void_p), ("rows", ctypes.c_int64), ("cols", ctypes.c_int64),
+                ("ld", ctypes.c_int64), ("trans", ctypes.c_int32)]
+
+
 class qfmt_stats_t(ctypes.Structure):
     _fields_ = [("hist", ctypes.c_uint64 * 256), ("n_total", ctypes.c_uint64),
                 ("n_zero_in", ctypes.c_uint64), ("n_denormal", ctypes.c_uint64),
@@ -77,8 +82,15 @@ def lib() -> ctypes.CDLL:
 
 
 def _bind_optional(L: ctypes.CDLL) -> None:
-    """Signatures of entry points added after the first two; see include/qfmt.h."""
-    return None
+    """Signatures of the contraction entry points; see include/qfmt.h."""
+    vp, sz, ci = ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int
+    matp = ctypes.POINTER(qfmt_matrix_t)
+    L.qfmt_gemm.argtypes = [matp, matp, vp, ctypes.c_int64, ctypes.POINTER(qfmt_format_t), vp, sz, vp]
+    L.qfmt_gemm.restype = ci
+    L.qfmt_gemm_workspace_bytes.argtypes = [matp, matp]
+    L.qfmt_gemm_workspace_bytes.restype = sz
+    L.qfmt_device_status.argtypes = [vp, vp]
+    L.qfmt_device_status.restype = ci
 
 
 def _ptr(x) -> Optional[int]:
@@ -137,3 +149,27 @@ def qfmt_version() -> int:
 
 def qfmt_status_string(status: int) -> str:
     return lib().qfmt_status_string(int(status)).decode()
+
+
+def make_matrix(t, trans: bool = False, rows: Optional[int] = None, cols: Optional[int] = None,
+                ld: Optional[int] = None) -> qfmt_matrix_t:
+    """Operand descriptor of a 2-D row-major torch tensor (or of a raw address with rows/cols/ld)."""
+    if hasattr(t, "shape") and rows is None:
+        assert t.dim() == 2 and t.stride(1) == 1
+        rows, cols, ld = t.shape[0], t.shape[1], t.stride(0)
+    return qfmt_matrix_t(_ptr(t), int(rows), int(cols), int(ld if ld is not None else cols), 1 if trans else 0)
+
+
+def qfmt_gemm_workspace_bytes(A: qfmt_matrix_t, B: qfmt_matrix_t) -> int:
+    return int(lib().qfmt_gemm_workspace_bytes(ctypes.byref(A), ctypes.byref(B)))
+
+
+def qfmt_gemm(A: qfmt_matrix_t, B: qfmt_matrix_t, d_C, ldc: int, fmt: qfmt_format_t, d_workspace,
+              workspace_bytes: int, stream=None) -> None:
+    """C = op(A) op(B), exact products, fp32 accumulation; see qfmt_gemm in include/qfmt.h."""
+    _check(lib().qfmt_gemm(ctypes.byref(A), ctypes.byref(B), _ptr(d_C), int(ldc), ctypes.byref(fmt),
+                           _ptr(d_workspace), int(workspace_bytes), _stream_handle(stream)), "qfmt_gemm")
+
+
+def qfmt_device_status(d_workspace, stream=None) -> int:
+    return int(lib().qfmt_device_status(_ptr(d_workspace), _stream_handle(stream)))

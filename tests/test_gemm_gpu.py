@@ -1,0 +1,282 @@
+"""GPU parity of qfmt_gemm against the fp64 oracle.
+
+Bar: |c_gpu - c_exact| <= 2^-20 * sum_k |a_ik||b_kj| per element; bit-exact where every
+accumulation order is exact (small integers, powers of two); identical bits run to run."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2103_15940_b200 as qf
+from paper_2103_15940_b200 import workloads
+
+pytestmark = pytest.mark.gpu
+
+TOL = 2.0 ** -20
+DEV = "cuda:0"
+
+
+def gpu_gemm(A_np, B_np, transA=False, transB=False, fmt=(6, 9), ldc_pad=0, check_status=True):
+    """A_np/B_np are the STORED matrices.  Returns C as numpy float32 [M, N]."""
+    dA = torch.from_numpy(np.ascontiguousarray(A_np)).to(DEV)
+    dB = torch.from_numpy(np.ascontiguousarray(B_np)).to(DEV)
+    M = A_np.shape[1] if transA else A_np.shape[0]
+    N = B_np.shape[0] if transB else B_np.shape[1]
+    ldc = N + ldc_pad
+    dC = torch.full((M, ldc), float("nan"), dtype=torch.float32, device=DEV)
+    a, b = qf.make_matrix(dA, transA), qf.make_matrix(dB, transB)
+    wb = qf.qfmt_gemm_workspace_bytes(a, b)
+    ws = torch.zeros(max(wb, 256), dtype=torch.uint8, device=DEV)
+    qf.qfmt_gemm(a, b, dC, ldc, qf.make_format(*fmt), ws, ws.numel())
+    if check_status:
+        assert qf.qfmt_device_status(ws) == qf.QFMT_OK
+    torch.cuda.synchronize()
+    out = dC.cpu().numpy()
+    if ldc_pad:
+        assert np.all(np.isnan(out[:, N:]))  # padding columns untouched
+    return out[:, :N]
+
+
+def stored(shape_mk, trans, gen):
+    """Stored matrix for a logical (rows, cols) operand."""
+    r, c = shape_mk
+    return gen((c, r)) if trans else gen((r, c))
+
+
+def quantized(rng, shape, e, m, mu=-3.0, sigma=2.0, p_zero=0.0):
+    x = workloads.lognormal_tensor(rng, shape, mu, sigma, p_zero=p_zero)
+    q, _ = oracle.quantize_stats(x, e, m, 1, 1.0, want_stats=False)
+    return q
+
+
+def within_bound(c_gpu, ref, T):
+    """Finite exact results: |c - ref| <= 2^-20 T.  Where an operand was inf/NaN the exact result
+    is inf or NaN (T is not finite) and the GPU result must be of the same class and sign."""
+    c = c_gpu.astype(np.float64)
+    fin = np.isfinite(T)
+    ok = np.abs(c - ref) <= TOL * T
+    ok[~fin] = np.where(np.isnan(ref[~fin]), np.isnan(c[~fin]), c[~fin] == ref[~fin])
+    worst = float(np.max(np.abs(c - ref)[fin] / np.maximum(T[fin], 1e-300))) / TOL if fin.any() else 0.0
+    return bool(np.all(ok)), worst
+
+
+def check(C, A, B, transA, transB, sample=None, seed=0):
+    if sample is None:
+        ref, T = oracle.gemm(A, B, transA, transB)
+        ok, worst = within_bound(C, ref, T)
+    else:
+        rng = np.random.default_rng(seed)
+        M, N = C.shape
+        ii = np.concatenate([rng.integers(0, M, size=sample), [0, M - 1, 0, M - 1]])
+        jj = np.concatenate([rng.integers(0, N, size=sample), [0, N - 1, N - 1, 0]])
+        ref, T = oracle.gemm_sampled(A, B, ii, jj, transA, transB)
+        ok, worst = within_bound(C[ii, jj], ref, T)
+    assert ok, f"worst error {worst:.3f} x tolerance"
+    return worst
+
+
+@pytest.mark.parametrize("transA", [False, True])
+@pytest.mark.parametrize("transB", [False, True])
+def test_small_integers_are_bit_exact(transA, transB):
+    """Entries in -8..8 and K = 64: every partial sum is an integer below 2^24, so any order of
+    fp32 accumulation gives the exact result; a wrong descriptor, swizzle or transpose cannot."""
+    rng = np.random.default_rng(1)
+    M, N, K = 128, 256, 64
+    A = stored((M, K), transA, lambda s: rng.integers(-8, 9, size=s).astype(np.float32))
+    B = stored((K, N), transB, lambda s: rng.integers(-8, 9, size=s).astype(np.float32))
+    C = gpu_gemm(A, B, transA, transB)
+    ref, _ = oracle.gemm(A, B, transA, transB)
+    assert np.array_equal(C.astype(np.float64), ref)
+
+
+@pytest.mark.parametrize("transA,transB", [(False, False), (False, True), (True, False), (True, True)])
+@pytest.mark.parametrize("M,N,K", [(1, 1, 1), (5, 7, 3), (128, 256, 32), (129, 257, 33), (200, 300, 100),
+                                    (256, 512, 96), (127, 255, 31), (64, 16, 8), (300, 40, 260), (1000, 520, 72)])
+def test_ragged_shapes_small_integers(transA, transB, M, N, K):
+    """Small-integer operands (exact in any order) in buffers whose rows are longer than the
+    matrices: the padding holds huge values, so reading a column past the logical width, a
+    wrong transpose or a mis-swizzled tile all show up as wrong integers."""
+    rng = np.random.default_rng(M * 7 + N * 3 + K)
+
+    def padded(shape):
+        r, c = shape
+        ld = (c + 3) // 4 * 4 + 4
+        buf = np.full((r, ld), 1.0e30, dtype=np.float32)
+        buf[:, :c] = rng.integers(-4, 5, size=(r, c)).astype(np.float32)
+        return buf, c
+
+    A_buf, a_cols = padded((K, M) if transA else (M, K))
+    B_buf, b_cols = padded((N, K) if transB else (K, N))
+    dA = torch.from_numpy(A_buf).to(DEV)
+    dB = torch.from_numpy(B_buf).to(DEV)
+    a = qf.qfmt_matrix_t(dA.data_ptr(), A_buf.shape[0], a_cols, A_buf.shape[1], int(transA))
+    b = qf.qfmt_matrix_t(dB.data_ptr(), B_buf.shape[0], b_cols, B_buf.shape[1], int(transB))
+    dC = torch.full((M, N + 3), -777.0, dtype=torch.float32, device=DEV)
+    ws = torch.zeros(qf.qfmt_gemm_workspace_bytes(a, b), dtype=torch.uint8, device=DEV)
+    qf.qfmt_gemm(a, b, dC, N + 3, qf.make_format(6, 9), ws, ws.numel())
+    assert qf.qfmt_device_status(ws) == qf.QFMT_OK
+    out = dC.cpu().numpy()
+    ref, _ = oracle.gemm(np.ascontiguousarray(A_buf[:, :a_cols]), np.ascontiguousarray(B_buf[:, :b_cols]),
+                         transA, transB)
+    assert np.array_equal(out[:, :N].astype(np.float64), ref)
+    assert np.all(out[:, N:] == -777.0)
+
+
+@pytest.mark.parametrize("e,m", [(6, 9), (5, 10), (8, 7)])
+@pytest.mark.parametrize("transA,transB", [(False, False), (False, True), (True, False)])
+def test_format_values_within_bound(e, m, transA, transB):
+    rng = workloads.rng_for(60 + e)
+    M, N, K = 384, 512, 448
+    A = stored((M, K), transA, lambda s: quantized(rng, s, e, m, -6.0, 5.0, 0.01))
+    B = stored((K, N), transB, lambda s: quantized(rng, s, e, m, -6.0, 5.0, 0.01))
+    C = gpu_gemm(A, B, transA, transB, fmt=(e, m))
+    check(C, A, B, transA, transB)
+    C2 = gpu_gemm(A, B, transA, transB, fmt=(e, m))
+    assert np.array_equal(C.view(np.uint32), C2.view(np.uint32))  # run-to-run identical
+
+
+def test_powers_of_two_and_wide_exponent_range():
+    """One nonzero product per output, magnitudes from 2^-60 to 2^60: exact in any order."""
+    K = 64
+    M, N = 128, 256
+    A = np.zeros((M, K), dtype=np.float32)
+    B = np.zeros((K, N), dtype=np.float32)
+    for i in range(M):
+        A[i, i % K] = np.float32(2.0 ** ((i % 61) - 30)) * (1 + (i % 3) * 0.5)
+    for j in range(N):
+        for k in range(K):
+            B[k, j] = np.float32(2.0 ** (((j + k) % 61) - 30)) * (-1 if (j + k) % 2 else 1)
+    C = gpu_gemm(A, B)
+    ref, _ = oracle.gemm(A, B)
+    assert np.array_equal(C.astype(np.float64), ref)
+
+
+def test_same_sign_long_k_stays_within_bound():
+    """All-positive operands, K = 8192: the accumulation error grows with K; the bound must hold."""
+    rng = workloads.rng_for(61)
+    M, N, K = 128, 256, 8192
+    A = np.abs(quantized(rng, (M, K), 6, 9, -2.0, 1.0))
+    B = np.abs(quantized(rng, (K, N), 6, 9, -2.0, 1.0))
+    C = gpu_gemm(A, B)
+    check(C, A, B, False, False)
+
+
+def test_inf_and_nan_propagate():
+    rng = workloads.rng_for(62)
+    M, N, K = 128, 256, 64
+    A = quantized(rng, (M, K), 6, 9)
+    B = quantized(rng, (K, N), 6, 9)
+    A[3, 5] = np.inf      # row 3: +-inf (or NaN where B[5, j] = 0)
+    A[7, 1] = np.nan      # row 7: NaN
+    B[9, 11] = -np.inf    # column 11: +-inf
+    C = gpu_gemm(A, B)
+    check(C, A, B, False, False)
+    assert np.all(np.isnan(C[7, :]))
+    assert np.all(~np.isfinite(C[3, :])) and np.all(~np.isfinite(C[:, 11]))
+    rest = np.ones((M, N), bool)
+    rest[3, :] = rest[7, :] = rest[:, 11] = False
+    assert np.all(np.isfinite(C[rest]))
+
+
+def test_config1_end_to_end():
+    """Quantize A and B on the GPU, multiply on the GPU; compare with the oracle's pipeline."""
+    cfg = workloads.config1()
+    e, m = cfg["fmt"]
+    fmt = qf.make_format(e, m, cfg["denormals"], cfg["loss_scale"])
+    dA = torch.from_numpy(cfg["A"]).to(DEV)
+    dB = torch.from_numpy(cfg["B"]).to(DEV)
+    st = torch.zeros(2, qf.STATS_WORDS, dtype=torch.int64, device=DEV)
+    qf.qfmt_quantize_stats(dA, dA, dA.numel(), fmt, st[0])
+    qf.qfmt_quantize_stats(dB, dB, dB.numel(), fmt, st[1])
+    dC = torch.empty(256, 256, dtype=torch.float32, device=DEV)
+    a, b = qf.make_matrix(dA), qf.make_matrix(dB)
+    ws = torch.zeros(qf.qfmt_gemm_workspace_bytes(a, b), dtype=torch.uint8, device=DEV)
+    qf.qfmt_gemm(a, b, dC, 256, fmt, ws, ws.numel())
+    assert qf.qfmt_device_status(ws) == qf.QFMT_OK
+    qA, sA = oracle.quantize_stats(cfg["A"], e, m, 1, 1.0)
+    qB, sB = oracle.quantize_stats(cfg["B"], e, m, 1, 1.0)
+    assert np.array_equal(dA.cpu().numpy().view(np.uint32), qA.view(np.uint32))
+    assert np.array_equal(st.cpu().numpy().view(np.uint64), np.stack([sA, sB]))
+    check(dC.cpu().numpy(), qA, qB, False, False)
+
+
+def test_k_zero_and_empty():
+    dA = torch.zeros(8, 4, dtype=torch.float32, device=DEV)
+    dC = torch.full((8, 8), 5.0, dtype=torch.float32, device=DEV)
+    ws = torch.zeros(256, dtype=torch.uint8, device=DEV)
+    a = qf.qfmt_matrix_t(dA.data_ptr(), 8, 0, 4, 0)
+    b = qf.qfmt_matrix_t(dA.data_ptr(), 0, 8, 8, 0)
+    qf.qfmt_gemm(a, b, dC, 8, qf.make_format(6, 9), ws, 256)
+    torch.cuda.synchronize()
+    assert torch.all(dC == 0)
+
+
+def test_argument_errors():
+    d = torch.zeros(64, 64, dtype=torch.float32, device=DEV)
+    ws = torch.zeros(256, dtype=torch.uint8, device=DEV)
+    a, b = qf.make_matrix(d), qf.make_matrix(d)
+    for bad_fmt in (qf.make_format(6, 11), qf.make_format(8, 23)):
+        with pytest.raises(qf.QfmtError) as ei:
+            qf.qfmt_gemm(a, b, d, 64, bad_fmt, ws, 256)
+        assert ei.value.status == qf.QFMT_ERR_BAD_FORMAT
+    with pytest.raises(qf.QfmtError):
+        qf.qfmt_gemm(a, qf.qfmt_matrix_t(d.data_ptr(), 32, 64, 64, 0), d, 64, qf.make_format(6, 9), ws, 256)
+    with pytest.raises(qf.QfmtError):
+        qf.qfmt_gemm(a, b, d, 32, qf.make_format(6, 9), ws, 256)  # ldc < N
+    with pytest.raises(qf.QfmtError):
+        qf.qfmt_gemm(a, b, d, 64, qf.make_format(6, 9), None, 0)
+    with pytest.raises(qf.QfmtError):
+        qf.qfmt_gemm(qf.qfmt_matrix_t(d.data_ptr() + 4, 64, 60, 64, 0), qf.qfmt_matrix_t(d.data_ptr(), 60, 64, 64, 0),
+                     d, 64, qf.make_format(6, 9), ws, 256)
+
+
+# ---------------------------------------------------------------------------------------------
+# The benchmark workloads at full size, in the launch configuration bench.py times, checked on
+# sampled outputs (each a full-K dot product in fp64).
+# ---------------------------------------------------------------------------------------------
+def quantize_on_gpu(x_np, e, m, den, scale):
+    d = torch.from_numpy(np.ascontiguousarray(x_np)).to(DEV)
+    qf.qfmt_quantize_stats(d, d, d.numel(), qf.make_format(e, m, den, scale))
+    return d
+
+
+def fc_layer_parity(X, W, dY, e, m, den, grad_scale, samples, seed):
+    """fwd Y = X W, dgrad dX = dY W^T, wgrad dW = X^T dY on GPU-quantized operands."""
+    dX_, dW_, dG_ = (quantize_on_gpu(X, e, m, den, 1.0), quantize_on_gpu(W, e, m, den, 1.0),
+                     quantize_on_gpu(dY, e, m, den, grad_scale))
+    qX, _ = oracle.quantize_stats(X, e, m, den, 1.0, want_stats=False)
+    qW, _ = oracle.quantize_stats(W, e, m, den, 1.0, want_stats=False)
+    qG, _ = oracle.quantize_stats(dY, e, m, den, grad_scale, want_stats=False)
+    assert np.array_equal(dG_.cpu().numpy().view(np.uint32), qG.view(np.uint32))
+    fmt = qf.make_format(e, m, den)
+    ws = torch.zeros(1 << 20, dtype=torch.uint8, device=DEV)
+    worst = {}
+    for name, (ta, A_d, A_h), (tb, B_d, B_h) in (
+            ("fwd", (False, dX_, qX), (False, dW_, qW)),
+            ("dgrad", (False, dG_, qG), (True, dW_, qW)),
+            ("wgrad", (True, dX_, qX), (False, dG_, qG))):
+        M = A_h.shape[1] if ta else A_h.shape[0]
+        N = B_h.shape[0] if tb else B_h.shape[1]
+        C = torch.empty(M, N, dtype=torch.float32, device=DEV)
+        a, b = qf.make_matrix(A_d, ta), qf.make_matrix(B_d, tb)
+        assert qf.qfmt_gemm_workspace_bytes(a, b) <= ws.numel()
+        qf.qfmt_gemm(a, b, C, N, fmt, ws, ws.numel())
+        assert qf.qfmt_device_status(ws) == qf.QFMT_OK
+        worst[name] = check(C.cpu().numpy(), A_h, B_h, ta, tb, sample=samples, seed=seed)
+    return worst
+
+
+@pytest.mark.parametrize("variant", [0, 1, 2, 3])
+def test_config3_bert_base_fc(variant):
+    cfg = workloads.config3()
+    (e, m), den = cfg["variants"][variant]
+    worst = fc_layer_parity(cfg["X"], cfg["W"], cfg["dY"], e, m, den, cfg["grad_scale"], 65536, 30 + variant)
+    print("config3", (e, m, den), worst)
+
+
+@pytest.mark.parametrize("layer", [0, 1, 2, 3])
+def test_config5_bert_large_fc_stack_step0(layer):
+    c = workloads.config5_layer(layer, step=0)
+    e, m = c["fmt"]
+    worst = fc_layer_parity(c["X"], c["W"], c["dY"], e, m, c["denormals"], c["grad_scale"], 65536, 50 + layer)
+    print("config5", c["name"], worst)
