@@ -1,0 +1,360 @@
+#!/usr/bin/env python
+"""Benchmark of the emulated 16-bit-format hot path on B200.
+
+One step = one pass of the format sweep (workload "config2"): the 64 Mi-element fp32 tensor is
+rounded, with range statistics, to 1/5/10, 1/8/7 and 1/6/9, each with denormals kept and
+flushed, at loss scales 2^0, 2^8 and 2^15 (18 kernel launches, 8 bytes of algorithmic traffic
+per element and launch).  `value` is the whole-job GB/s with inputs resident in HBM; `e2e` is
+the same metric through the host-buffer entry point (copies inside the timed region).  The
+contraction half of the path is timed in the same run on the BERT-large FC stack (workload
+"config5", one step: 4 layers x fwd/dgrad/wgrad) and reported under `gemm`.
+
+    python bench.py --gpus N --steps K --warmup W          # this library
+    python bench.py --impl reference ...                    # the CPU oracle on a bounded sample
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2103_15940_b200 import workloads  # noqa: E402
+
+METRIC = "quantize+stats GB/s"
+UNIT = "GB/s"
+BYTES_PER_ELEMENT = 8  # 4 read + 4 written
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d["bf16_tflops"]),
+                "bf16_tflops_sustained": float(d.get("bf16_tflops_sustained", d["bf16_tflops"])),
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML (read-only) while a region is timed."""
+
+    def __init__(self, index: int):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            self._h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self._nv = None
+
+    def _run(self):
+        nv = self._nv
+        names = {nv.nvmlClocksThrottleReasonSwPowerCap: "sw_power_cap",
+                 nv.nvmlClocksThrottleReasonHwSlowdown: "hw_slowdown",
+                 nv.nvmlClocksThrottleReasonSwThermalSlowdown: "sw_thermal_slowdown",
+                 nv.nvmlClocksThrottleReasonHwThermalSlowdown: "hw_thermal_slowdown",
+                 nv.nvmlClocksThrottleReasonHwPowerBrakeSlowdown: "hw_power_brake"}
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM))
+                mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h)
+                for bit, name in names.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(0.004)
+
+    def __enter__(self):
+        if self._nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self):
+        return {"sm_mhz": statistics.median(self.samples) if self.samples else None,
+                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def nvml_index(local_rank: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_rank])
+        except Exception:
+            return local_rank
+    return local_rank
+
+
+# ------------------------------------------------------------------------------------------------
+# reference arm: the CPU oracle, as it stands, on a bounded sample of the same workload
+# ------------------------------------------------------------------------------------------------
+def oracle_sweep(x: np.ndarray) -> float:
+    """Runs the 18 sweep configurations on x with the oracle; returns seconds."""
+    import oracle
+    t0 = time.perf_counter()
+    for _, e, m, den, scale in workloads.config2_runs():
+        oracle.quantize_stats(x, e, m, den, scale)
+    return time.perf_counter() - t0
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    n_sample = 1 << 20
+    x = workloads.config2_tensor(n=n_sample)
+    for _ in range(args.warmup):
+        oracle_sweep(x[: 1 << 16])
+    secs = [oracle_sweep(x) for _ in range(args.steps)]
+    total = sum(secs)
+    value = args.steps * 18 * n_sample * BYTES_PER_ELEMENT / total / 1e9
+    sample = f"18 sweep runs on the first {n_sample} elements of the config2 tensor per step"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u32", "data": "synthetic",
+            "config": {"workload": "config2 format sweep (bounded sample)", "elements": n_sample, "runs_per_step": 18},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------------------
+# this library
+# ------------------------------------------------------------------------------------------------
+def time_events(torch, fn, iters):
+    """Per-call device times (ms) of fn(), CUDA events on the current stream."""
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(iters)]
+    for a, b in evs:
+        a.record()
+        fn()
+        b.record()
+    torch.cuda.synchronize()
+    return [a.elapsed_time(b) for a, b in evs]
+
+
+def gemm_section(torch, qf, dev, peaks, reps=5):
+    """One step of the BERT-large FC stack: 12 GEMMs on operands quantized to 1/6/9 on the GPU."""
+    fmt = qf.make_format(6, 9, 1)
+    ws = torch.zeros(1 << 20, dtype=torch.uint8, device=dev)
+    jobs, flops = [], 0.0
+    for layer in range(len(workloads.CONFIG5_LAYERS)):
+        c = workloads.config5_layer(layer, step=0)
+        t = {}
+        for name, scale in (("X", 1.0), ("W", 1.0), ("dY", c["grad_scale"])):
+            d = torch.from_numpy(c[name]).to(dev)
+            qf.qfmt_quantize_stats(d, d, d.numel(), qf.make_format(6, 9, 1, scale))
+            t[name] = d
+        tokens, d_in = c["X"].shape
+        d_out = c["W"].shape[1]
+        for A, ta, B, tb, M, N, K in ((t["X"], False, t["W"], False, tokens, d_out, d_in),
+                                      (t["dY"], False, t["W"], True, tokens, d_in, d_out),
+                                      (t["X"], True, t["dY"], False, d_in, d_out, tokens)):
+            C = torch.empty(M, N, dtype=torch.float32, device=dev)
+            jobs.append((qf.make_matrix(A, ta), qf.make_matrix(B, tb), C, N, (A, B)))
+            flops += 2.0 * M * N * K
+
+    def step():
+        for a, b, C, N, _ in jobs:
+            qf.qfmt_gemm(a, b, C, N, fmt, ws, ws.numel())
+
+    for _ in range(3):
+        step()
+    assert qf.qfmt_device_status(ws) == qf.QFMT_OK
+    ms = statistics.median(time_events(torch, step, reps))
+    # library TF32 GEMM on the same box, same run: the measured tensor-pipe denominator
+    torch.backends.cuda.matmul.allow_tf32 = True
+    a = torch.randn(8192, 8192, device=dev)
+    b = torch.randn(8192, 8192, device=dev)
+    c = torch.empty(8192, 8192, device=dev)
+    for _ in range(3):
+        torch.matmul(a, b, out=c)
+    lib_ms = min(time_events(torch, lambda: torch.matmul(a, b, out=c), 5))
+    lib_tf32 = 2.0 * 8192 ** 3 / lib_ms / 1e9
+    del a, b, c
+    achieved = flops / ms / 1e9
+    peak = peaks["bf16_tflops"] * (1.1 / 2.25)  # TF32 dense is nominally 1.1/2.25 of bf16 dense
+    return {"metric": "emulated GEMM TFLOP/s", "value": achieved, "unit": "TFLOP/s",
+            "workload": "config5 BERT-large FC stack, one step: 4 layers x fwd/dgrad/wgrad, 1/6/9",
+            "ms_per_step": ms, "gemms_per_step": len(jobs), "gpu_launches_per_step": len(jobs),
+            "roofline": {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                         "frac": achieved / peak, "traffic": None,
+                         "peak_source": f"bf16 {peaks['source']} burst x 1.1/2.25 (nominal TF32:bf16 ratio)",
+                         "library_tf32_same_run": lib_tf32, "frac_of_library_tf32": achieved / lib_tf32,
+                         "nominal_tf32_dense": 1100.0, "frac_of_nominal": achieved / 1100.0}}
+
+
+def run_library(args):
+    import torch
+    import paper_2103_15940_b200 as qf
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    qf.lib()  # fail loudly if the CUDA library has not been built
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group(backend="nccl", device_id=dev)
+
+    peaks = measured_peaks()
+    n = workloads.CONFIG2_N
+    runs = workloads.config2_runs()
+    x_host = workloads.config2_tensor()
+    d_in = torch.from_numpy(x_host).to(dev)
+    d_out = torch.empty_like(d_in)
+    d_stats = torch.zeros(len(runs), qf.STATS_WORDS, dtype=torch.int64, device=dev)
+    fmts = [qf.make_format(e, m, den, s) for _, e, m, den, s in runs]
+
+    def step():
+        for i, f in enumerate(fmts):
+            qf.qfmt_quantize_stats(d_in, d_out, n, f, d_stats[i], 0)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    launch_ms = []
+    barrier()
+    with ClockSampler(nvml_index(local_rank)) as clocks:
+        t_begin = torch.cuda.Event(enable_timing=True)
+        t_end = torch.cuda.Event(enable_timing=True)
+        pairs = []
+        t_begin.record()
+        for _ in range(args.steps):
+            for i, f in enumerate(fmts):
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record()
+                qf.qfmt_quantize_stats(d_in, d_out, n, f, d_stats[i], 0)
+                b.record()
+                pairs.append((a, b))
+        t_end.record()
+        barrier()
+    total_ms = t_begin.elapsed_time(t_end)
+    launch_ms = [a.elapsed_time(b) for a, b in pairs]
+    if dist is not None:
+        t = torch.tensor([total_ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    step_bytes = len(runs) * n * BYTES_PER_ELEMENT
+    value = world * args.steps * step_bytes / total_ms / 1e6  # GB/s over all ranks
+
+    # sanity: the timed kernels did the work (denormal counts of the last step are plausible)
+    st = d_stats.cpu().numpy().view(np.uint64)
+    assert int(st[0, 256]) == n and int(st[:, 258].max()) > 0
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant kernel (quantize+stats): algorithmic bytes / mean launch time
+    mean_launch_ms = statistics.mean(launch_ms)
+    achieved = n * BYTES_PER_ELEMENT / mean_launch_ms / 1e6
+    roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": achieved / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH,
+                "peak_source": f"copy bandwidth, {peaks['source']}", "algorithmic_bytes_per_launch": n * BYTES_PER_ELEMENT,
+                "mean_launch_us": 1e3 * mean_launch_ms, "nominal_hbm_gbs": 7700.0, "frac_of_nominal": achieved / 7700.0}
+
+    sections = set(args.sections.split(","))
+    e2e = gemm = cpu = None
+    if "e2e" in sections:
+        e2e = e2e_section(torch, qf, dev, x_host, fmts, n, step_bytes, args)
+    if "gemm" in sections:
+        gemm = gemm_section(torch, qf, dev, peaks)
+    if "cpu" in sections:
+        # the CPU oracle on this machine's host cores, bounded sample
+        n_cpu = 1 << 24
+        cpu_secs = oracle_sweep(x_host[:n_cpu])
+        cpu_value = len(runs) * n_cpu * BYTES_PER_ELEMENT / cpu_secs / 1e9
+        cpu = {"value": cpu_value, "unit": UNIT, "cores": 1, "kind": "oracle", "seconds": cpu_secs,
+               "host_cores_available": os.cpu_count(),
+               "sample": f"the 18 sweep runs on the first {n_cpu} of {n} elements"}
+    return finish(args, world, value, total_ms, n, runs, clocks, e2e, roofline, cpu, gemm, dist)
+
+
+def e2e_section(torch, qf, dev, x_host, fmts, n, step_bytes, args):
+    """End to end through the host-buffer entry point (pinned host memory, copies timed)."""
+    runs = fmts
+    h_in = torch.from_numpy(x_host).pin_memory()
+    h_out = torch.empty(n, dtype=torch.float32).pin_memory()
+    h_stats = torch.zeros(qf.STATS_WORDS, dtype=torch.int64).pin_memory()
+    wb = qf.qfmt_quantize_stats_host_work_bytes(n)
+    d_work = torch.empty(wb, dtype=torch.uint8, device=dev)
+    e2e_steps = max(1, min(args.steps, 2))
+    qf.qfmt_quantize_stats_host(h_in, h_out, n, fmts[0], h_stats, d_work, wb)
+    e2e_ms = time_events(torch, lambda: [qf.qfmt_quantize_stats_host(h_in, h_out, n, f, h_stats, d_work, wb)
+                                         for f in fmts], e2e_steps)
+    e2e_value = step_bytes / statistics.mean(e2e_ms) / 1e6
+    e2e = {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": len(runs) * n * 4,
+           "d2h_bytes_per_step": len(runs) * (n * 4 + qf.STATS_WORDS * 8), "steps": e2e_steps}
+    del d_work, h_in, h_out
+    return e2e
+
+
+def finish(args, world, value, total_ms, n, runs, clocks, e2e, roofline, cpu, gemm, dist):
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "u32", "data": "synthetic",
+            "config": {"workload": "config2 format sweep: 64 Mi fp32 elements x 18 (format, denormal mode, loss scale) runs",
+                       "elements": n, "runs_per_step": len(runs), "l2": "inputs larger than L2 (256 MiB in, 256 MiB out)",
+                       "multi_gpu": "replicas only: every rank runs the whole sweep on its own copy"},
+            "clocks": clocks.summary(), "e2e": e2e, "gpu_launches": args.steps * len(runs),
+            "roofline": roofline, "cpu_baseline": cpu, "gemm": gemm}
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the quantize+stats kernel, from the
+# ncu capture summarised in profiles/quantize_stats_kernel_config2.md (set to None when the kernel changes).
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 268464640 + 218681088
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="library", choices=["library", "reference"])
+    ap.add_argument("--sections", default="quantize,e2e,gemm,cpu",
+                    help="comma list of what to measure besides the timed sweep (quantize is always timed): "
+                         "e2e, gemm, cpu; profiling captures use a subset")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_library(args)
+
+
+if __name__ == "__main__":
+    main()
