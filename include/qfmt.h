@@ -30,7 +30,8 @@ typedef enum {
     QFMT_ERR_BAD_ARG = -2,     /* NULL/misaligned pointer, bad dimension, workspace too small  */
     QFMT_ERR_UNSUPPORTED_ARCH = -3, /* current device is not compute capability 10.x           */
     QFMT_ERR_CUDA = -4,        /* a CUDA runtime/driver call failed (see qfmt_last_cuda_error)  */
-    QFMT_ERR_TIMEOUT = -5      /* a bounded device-side wait expired (reported via status word) */
+    QFMT_ERR_TIMEOUT = -5,     /* a bounded device-side wait expired (reported via status word) */
+    QFMT_ERR_SCRATCH_LIMIT = -6 /* qfmt_gemm_builtin_scratch: the problem needs more than 16 MiB   */
 } qfmt_status_t;
 
 /*
@@ -143,6 +144,37 @@ typedef struct {
 int qfmt_gemm(const qfmt_matrix_t* A, const qfmt_matrix_t* B, float* d_C, int64_t ldc,
               const qfmt_format_t* fmt, void* d_workspace, size_t workspace_bytes, void* stream);
 size_t qfmt_gemm_workspace_bytes(const qfmt_matrix_t* A, const qfmt_matrix_t* B);
+
+/*
+ * qfmt_gemm for callers that cannot allocate device memory.  (The paper has no counterpart of
+ * this call; it exists for the way the library gets embedded.)
+ *
+ * qfmt_gemm needs a workspace that the caller allocates.  Some callers have no way to do that at
+ * the point where they need the product: code that runs inside another framework's memory plan
+ * and is handed only its input and output buffers; a real-time or safety-certified loop that is
+ * forbidden to allocate once it has started; a process whose device memory has been given out
+ * completely to a pool it does not own.  For them this variant keeps the workspace inside the
+ * library: a fixed 16 MiB array that is part of the loaded GPU module, so every GPU that loads
+ * libqfmt holds those 16 MiB from the first use of the library on that GPU until the process
+ * ends.  The call itself performs no cudaMalloc / cudaFree and uses no allocating library routine.
+ *
+ * Arguments A, B, d_C, ldc, fmt, stream: exactly as for qfmt_gemm, same results bit for bit.
+ *   d_status_out  device, 4-byte aligned, or NULL.  If given, the kernel's status word
+ *                 (QFMT_OK or QFMT_ERR_TIMEOUT) is copied there on `stream` after the product;
+ *                 read it with qfmt_device_status(d_status_out, stream) or your own copy.
+ * Limits and rules
+ *   - A problem for which qfmt_gemm_workspace_bytes(A, B) exceeds 16 MiB is refused with
+ *     QFMT_ERR_SCRATCH_LIMIT and nothing is enqueued; use qfmt_gemm with your own workspace.
+ *   - The first call on each GPU looks up the array's device address (a query, not an
+ *     allocation).  Make that first call during set-up, before any stream capture begins.
+ *   - All calls on one GPU share the one array and it keeps whatever the previous call left.
+ *     The library clears what has to start at zero, but two calls whose GPU work can overlap
+ *     (different streams without an ordering between them, or several host threads) race on it:
+ *     keep every call on a GPU on one stream, or order them with events.
+ * Errors: as qfmt_gemm, plus QFMT_ERR_SCRATCH_LIMIT.
+ */
+int qfmt_gemm_builtin_scratch(const qfmt_matrix_t* A, const qfmt_matrix_t* B, float* d_C, int64_t ldc,
+                              const qfmt_format_t* fmt, int32_t* d_status_out, void* stream);
 
 /*
  * Synchronises `stream` and returns the status word of a workspace: QFMT_OK, or the error a

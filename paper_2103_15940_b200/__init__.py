@@ -20,6 +20,7 @@ QFMT_ERR_BAD_ARG = -2
 QFMT_ERR_UNSUPPORTED_ARCH = -3
 QFMT_ERR_CUDA = -4
 QFMT_ERR_TIMEOUT = -5
+QFMT_ERR_SCRATCH_LIMIT = -6
 
 STATS_WORDS = 264  # 256 histogram bins + 8 counters, all uint64
 (ST_TOTAL, ST_ZERO_IN, ST_DENORMAL, ST_UNDERFLOW, ST_OVERFLOW, ST_NAN, ST_INF_IN) = range(256, 263)
@@ -91,6 +92,8 @@ def _bind_optional(L: ctypes.CDLL) -> None:
     L.qfmt_gemm_workspace_bytes.restype = sz
     L.qfmt_device_status.argtypes = [vp, vp]
     L.qfmt_device_status.restype = ci
+    L.qfmt_gemm_builtin_scratch.argtypes = [matp, matp, vp, ctypes.c_int64, ctypes.POINTER(qfmt_format_t), vp, vp]
+    L.qfmt_gemm_builtin_scratch.restype = ci
 
 
 def _ptr(x) -> Optional[int]:
@@ -173,3 +176,11 @@ def qfmt_gemm(A: qfmt_matrix_t, B: qfmt_matrix_t, d_C, ldc: int, fmt: qfmt_forma
 
 def qfmt_device_status(d_workspace, stream=None) -> int:
     return int(lib().qfmt_device_status(_ptr(d_workspace), _stream_handle(stream)))
+
+
+def qfmt_gemm_builtin_scratch(A: qfmt_matrix_t, B: qfmt_matrix_t, d_C, ldc: int, fmt: qfmt_format_t,
+                              d_status_out=None, stream=None) -> None:
+    """qfmt_gemm for callers that cannot allocate: the workspace is a fixed 16 MiB array inside the
+    library (shared by all calls on a GPU; keep them on one stream).  See include/qfmt.h."""
+    _check(lib().qfmt_gemm_builtin_scratch(ctypes.byref(A), ctypes.byref(B), _ptr(d_C), int(ldc), ctypes.byref(fmt),
+                                           _ptr(d_status_out), _stream_handle(stream)), "qfmt_gemm_builtin_scratch")

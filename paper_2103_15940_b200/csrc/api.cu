@@ -56,6 +56,7 @@ extern "C" const char* qfmt_status_string(int status) {
         case QFMT_ERR_UNSUPPORTED_ARCH: return "device is not compute capability 10.x";
         case QFMT_ERR_CUDA: return "CUDA call failed";
         case QFMT_ERR_TIMEOUT: return "bounded device-side wait expired";
+        case QFMT_ERR_SCRATCH_LIMIT: return "problem needs more scratch memory than the library's built-in 16 MiB";
         default: return "unknown status";
     }
 }

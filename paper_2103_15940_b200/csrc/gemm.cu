@@ -34,6 +34,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "common.cuh"
 #include "ptx.cuh"
 
@@ -498,4 +500,56 @@ extern "C" int qfmt_device_status(void* d_workspace, void* stream) {
     QFMT_CUDA_TRY(cudaMemcpyAsync(&st, d_workspace, sizeof(int), cudaMemcpyDeviceToHost, (cudaStream_t)stream));
     QFMT_CUDA_TRY(cudaStreamSynchronize((cudaStream_t)stream));
     return st;
+}
+
+
+// ------------------------------------------------------------------------------------------------
+// Variant with built-in scratch memory (no counterpart in the paper; see include/qfmt.h).
+// ------------------------------------------------------------------------------------------------
+namespace qfmt {
+namespace {
+
+constexpr size_t kBuiltinScratchBytes = (size_t)16 << 20;  // 16 MiB per GPU that loads the library
+
+// Lives in every device's copy of the module.  In host code this name is only a handle for
+// cudaGetSymbolAddress: it is not a device address and must never be handed to a kernel.
+static __device__ __align__(256) unsigned char g_builtin_scratch[kBuiltinScratchBytes];
+
+// Device address of g_builtin_scratch on the current device, looked up once per device.
+int builtin_scratch_address(void** out) {
+    constexpr int kMaxDevices = 64;
+    static std::atomic<void*> cached[kMaxDevices];
+    int dev = 0;
+    QFMT_CUDA_TRY(cudaGetDevice(&dev));
+    void* p = (dev >= 0 && dev < kMaxDevices) ? cached[dev].load() : nullptr;
+    if (p == nullptr) {
+        QFMT_CUDA_TRY(cudaGetSymbolAddress(&p, g_builtin_scratch));  // with `dev` current
+        if (p == nullptr) { set_last_cuda_error((int)cudaErrorInvalidSymbol); return QFMT_ERR_CUDA; }
+        if (dev >= 0 && dev < kMaxDevices) cached[dev].store(p);
+    }
+    *out = p;
+    return QFMT_OK;
+}
+
+}  // namespace
+}  // namespace qfmt
+
+extern "C" int qfmt_gemm_builtin_scratch(const qfmt_matrix_t* A, const qfmt_matrix_t* B, float* d_C, int64_t ldc,
+                                         const qfmt_format_t* fmt, int32_t* d_status_out, void* stream) {
+    if (A == nullptr || B == nullptr) return QFMT_ERR_BAD_ARG;
+    if (reinterpret_cast<uintptr_t>(d_status_out) & 3u) return QFMT_ERR_BAD_ARG;
+    if (qfmt_gemm_workspace_bytes(A, B) > qfmt::kBuiltinScratchBytes) return QFMT_ERR_SCRATCH_LIMIT;
+    void* scratch = nullptr;
+    int rc = qfmt::builtin_scratch_address(&scratch);
+    if (rc != QFMT_OK) return rc;
+    // The array still holds what the previous call left.  Only the status word at its head has
+    // to start at zero; clear it here as well so that a call that enqueues no kernel (M or N zero)
+    // does not report an older call's status.
+    QFMT_CUDA_TRY(cudaMemsetAsync(scratch, 0, 16, (cudaStream_t)stream));
+    rc = qfmt::gemm_device(A, B, d_C, ldc, fmt, scratch, qfmt::kBuiltinScratchBytes, (cudaStream_t)stream);
+    if (rc != QFMT_OK) return rc;
+    if (d_status_out != nullptr)
+        QFMT_CUDA_TRY(cudaMemcpyAsync(d_status_out, scratch, sizeof(int32_t), cudaMemcpyDeviceToDevice,
+                                      (cudaStream_t)stream));
+    return QFMT_OK;
 }
