@@ -92,6 +92,20 @@ int qfmt_quantize_stats(const float* d_in, float* d_out, size_t n, const qfmt_fo
                         qfmt_stats_t* d_stats, int accumulate, void* stream);
 
 /*
+ * qfmt_quantize_stats with a batched transpose folded into the same pass: d_in is
+ * [batch][rows][cols], d_out is [batch][cols][rows], both dense fp32; rounding, loss scale and
+ * statistics exactly as above (the statistics do not depend on the element order).
+ * This is how convolution operands reach the channels-last layouts qfmt_conv reads, without an
+ * extra trip through memory: the rounding pass of Section IV-A touches every element anyway.
+ *     activations NCHW -> NHWC:  batch = N, rows = C, cols = H*W
+ *     filters     KCRS -> KRSC:  batch = K, rows = C, cols = R*S
+ * d_out must not overlap d_in.  Each of batch, rows, cols < 2^31.
+ */
+int qfmt_quantize_stats_transpose(const float* d_in, float* d_out, int64_t batch, int64_t rows, int64_t cols,
+                                  const qfmt_format_t* fmt, qfmt_stats_t* d_stats, int accumulate,
+                                  void* stream);
+
+/*
  * The same operation on HOST buffers: copies h_in to the device, runs the kernel, copies the
  * rounded tensor (if h_out != NULL) and the statistics (if h_stats != NULL) back, and
  * SYNCHRONISES the stream before returning.  The caller lends device scratch:
@@ -144,6 +158,38 @@ typedef struct {
 int qfmt_gemm(const qfmt_matrix_t* A, const qfmt_matrix_t* B, float* d_C, int64_t ldc,
               const qfmt_format_t* fmt, void* d_workspace, size_t workspace_bytes, void* stream);
 size_t qfmt_gemm_workspace_bytes(const qfmt_matrix_t* A, const qfmt_matrix_t* B);
+
+/*
+ * Convolution layers (Section V: "matrix multiplications, at the core of fully connected and
+ * convolution layers"): the three products of a unit-stride, zero-padded 2-D convolution,
+ * computed as implicit GEMMs with the FMACS semantics of qfmt_gemm (exact products, fp32
+ * accumulation, same error bound).  Nothing is unfolded in memory: tiles of the activation tensor
+ * are fetched by TMA at each filter tap's offset and the padding is the copy engine's zero fill.
+ *
+ * All tensors are dense, channels-last, 16-byte aligned, and already hold format values (produce
+ * them with qfmt_quantize_stats_transpose from NCHW / KCRS data, or qfmt_quantize_stats if they
+ * are channels-last already):
+ *     X  [n][h][w][c_in]      activations           Y, dY [n][oh][ow][c_out]
+ *     W  [c_out][r][s][c_in]  filters               oh = h + 2 pad_h - r + 1, ow likewise
+ *   op = QFMT_CONV_FWD    d_p = X,  d_q = W   d_out = Y   Y[n,oh,ow,co] = sum X[n,oh+r-pad_h,ow+s-pad_w,ci] W[co,r,s,ci]
+ *   op = QFMT_CONV_DGRAD  d_p = dY, d_q = W   d_out = dX  dX[n,h,w,ci] = sum dY[n,h-r+pad_h,w-s+pad_w,co] W[co,r,s,ci]
+ *   op = QFMT_CONV_WGRAD  d_p = dY, d_q = X   d_out = dW  dW[co,r,s,ci] = sum dY[n,oh,ow,co] X[n,oh+r-pad_h,ow+s-pad_w,ci]
+ * Limits: c_in and c_out multiples of 32; output row length (ow; w for the data gradient) at
+ * most 128, and at most 32 for the filter gradient; every tensor below 2^30 elements per
+ * dimension product used as a GEMM extent.  Violations return QFMT_ERR_BAD_ARG.
+ *   d_workspace  device, 16-byte aligned, >= qfmt_conv_workspace_bytes(op, geom) bytes: status
+ *                word, and for the filter gradient the split-K partial sums (the long pixel
+ *                dimension is split over CTAs and the parts are added in a fixed pairwise order,
+ *                so results are reproducible).
+ * Errors and the bounded-wait status word: as qfmt_gemm.
+ */
+typedef struct {
+    int32_t n, c_in, h, w, c_out, r, s, pad_h, pad_w;
+} qfmt_conv_t;
+enum { QFMT_CONV_FWD = 0, QFMT_CONV_DGRAD = 1, QFMT_CONV_WGRAD = 2 };
+int qfmt_conv(int32_t op, const qfmt_conv_t* geom, const float* d_p, const float* d_q, float* d_out,
+              const qfmt_format_t* fmt, void* d_workspace, size_t workspace_bytes, void* stream);
+size_t qfmt_conv_workspace_bytes(int32_t op, const qfmt_conv_t* geom);  /* 0 if geom is unsupported */
 
 /*
  * qfmt_gemm for callers that cannot allocate device memory.  (The paper has no counterpart of

@@ -45,6 +45,13 @@ class qfmt_matrix_t(ctypes.Structure):
                 ("ld", ctypes.c_int64), ("trans", ctypes.c_int32)]
 
 
+class qfmt_conv_t(ctypes.Structure):
+    _fields_ = [(k, ctypes.c_int32) for k in ("n", "c_in", "h", "w", "c_out", "r", "s", "pad_h", "pad_w")]
+
+
+QFMT_CONV_FWD, QFMT_CONV_DGRAD, QFMT_CONV_WGRAD = 0, 1, 2
+
+
 class qfmt_stats_t(ctypes.Structure):
     _fields_ = [("hist", ctypes.c_uint64 * 256), ("n_total", ctypes.c_uint64),
                 ("n_zero_in", ctypes.c_uint64), ("n_denormal", ctypes.c_uint64),
@@ -67,6 +74,8 @@ def lib() -> ctypes.CDLL:
         fmtp = ctypes.POINTER(qfmt_format_t)
         L.qfmt_quantize_stats.argtypes = [vp, vp, sz, fmtp, vp, ci, vp]
         L.qfmt_quantize_stats.restype = ci
+        L.qfmt_quantize_stats_transpose.argtypes = [vp, vp, ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, fmtp, vp, ci, vp]
+        L.qfmt_quantize_stats_transpose.restype = ci
         L.qfmt_quantize_stats_host.argtypes = [vp, vp, sz, fmtp, vp, vp, sz, vp]
         L.qfmt_quantize_stats_host.restype = ci
         L.qfmt_quantize_stats_host_work_bytes.argtypes = [sz]
@@ -92,6 +101,11 @@ def _bind_optional(L: ctypes.CDLL) -> None:
     L.qfmt_gemm_workspace_bytes.restype = sz
     L.qfmt_device_status.argtypes = [vp, vp]
     L.qfmt_device_status.restype = ci
+    convp = ctypes.POINTER(qfmt_conv_t)
+    L.qfmt_conv.argtypes = [ctypes.c_int32, convp, vp, vp, vp, ctypes.POINTER(qfmt_format_t), vp, sz, vp]
+    L.qfmt_conv.restype = ci
+    L.qfmt_conv_workspace_bytes.argtypes = [ctypes.c_int32, convp]
+    L.qfmt_conv_workspace_bytes.restype = sz
     L.qfmt_gemm_builtin_scratch.argtypes = [matp, matp, vp, ctypes.c_int64, ctypes.POINTER(qfmt_format_t), vp, vp]
     L.qfmt_gemm_builtin_scratch.restype = ci
 
@@ -132,6 +146,14 @@ def qfmt_quantize_stats(d_in, d_out, n: int, fmt: qfmt_format_t, d_stats=None, a
     """Device buffers in, device buffers out; see qfmt_quantize_stats in include/qfmt.h."""
     _check(lib().qfmt_quantize_stats(_ptr(d_in), _ptr(d_out), int(n), ctypes.byref(fmt), _ptr(d_stats),
                                      int(accumulate), _stream_handle(stream)), "qfmt_quantize_stats")
+
+
+def qfmt_quantize_stats_transpose(d_in, d_out, batch: int, rows: int, cols: int, fmt: qfmt_format_t, d_stats=None,
+                                  accumulate: int = 0, stream=None) -> None:
+    """[batch][rows][cols] -> rounded [batch][cols][rows]; see include/qfmt.h."""
+    _check(lib().qfmt_quantize_stats_transpose(_ptr(d_in), _ptr(d_out), int(batch), int(rows), int(cols),
+                                               ctypes.byref(fmt), _ptr(d_stats), int(accumulate),
+                                               _stream_handle(stream)), "qfmt_quantize_stats_transpose")
 
 
 def qfmt_quantize_stats_host_work_bytes(n: int) -> int:
@@ -184,3 +206,15 @@ def qfmt_gemm_builtin_scratch(A: qfmt_matrix_t, B: qfmt_matrix_t, d_C, ldc: int,
     library (shared by all calls on a GPU; keep them on one stream).  See include/qfmt.h."""
     _check(lib().qfmt_gemm_builtin_scratch(ctypes.byref(A), ctypes.byref(B), _ptr(d_C), int(ldc), ctypes.byref(fmt),
                                            _ptr(d_status_out), _stream_handle(stream)), "qfmt_gemm_builtin_scratch")
+
+
+def qfmt_conv_workspace_bytes(op: int, geom: qfmt_conv_t) -> int:
+    return int(lib().qfmt_conv_workspace_bytes(int(op), ctypes.byref(geom)))
+
+
+def qfmt_conv(op: int, geom: qfmt_conv_t, d_p, d_q, d_out, fmt: qfmt_format_t, d_workspace, workspace_bytes: int,
+              stream=None) -> None:
+    """Forward / data-gradient / filter-gradient product of a convolution on channels-last tensors;
+    see qfmt_conv in include/qfmt.h."""
+    _check(lib().qfmt_conv(int(op), ctypes.byref(geom), _ptr(d_p), _ptr(d_q), _ptr(d_out), ctypes.byref(fmt),
+                           _ptr(d_workspace), int(workspace_bytes), _stream_handle(stream)), "qfmt_conv")

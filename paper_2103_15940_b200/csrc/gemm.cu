@@ -76,7 +76,43 @@ struct GemmParams {
     int b_mn_major;  // op(B) stored with N contiguous
     int tiles_m, tiles_n;
     int tma_store;   // C base, row pitch and row length are multiples of 16 bytes: C is written by TMA
+    // ---- work decomposition
+    int tile_rows;         // rows of C owned by one M-tile (128, or whole image rows in mode 1)
+    int kb_total;          // stages (k-blocks) in the whole contraction
+    int kb_per_split;      // stages handled by one work item
+    int splits;            // split-K factor; the partial result of split s goes to C + s * split_stride
+    long long split_stride;
+    uint32_t a_bytes, b_bytes;  // bytes TMA delivers per stage
+    // ---- convolution modes (see conv_device): 0 dense, 1 pixels are the M dimension (forward and
+    // data gradient), 2 pixels are the K dimension (filter gradient)
+    int mode;
+    int img_rows, img_w;   // rows per image and pixels per row of the pixel space that is tiled
+    int total_q;           // batch * img_rows
+    int rows_per_blk;      // image rows per M-tile (mode 1) or per stage (mode 2)
+    int taps, taps_s;      // R*S and S
+    int cblocks, ck;       // mode 1: 32-channel blocks per tap and contraction channels; mode 2: ck = C_in
+    int tap_sign, off_h, off_w;  // activation row read for tap (r, s): h + tap_sign * r + off_h
+    int full_tiles_m;      // mode 1: M-tiles that are complete (the C tensor map covers exactly these)
 };
+
+// Position of work item t: tile coordinates, split, and the range of stages it sums.
+struct WorkItem {
+    int tile_m, tile_n, split, m0, n0, kb_begin, num_kb;
+};
+__device__ __forceinline__ WorkItem decode_work(const GemmParams& p, int t) {
+    WorkItem w;
+    const int num_tiles = p.tiles_m * p.tiles_n;
+    const int tile = t % num_tiles;
+    w.split = t / num_tiles;
+    w.tile_m = tile % p.tiles_m;
+    w.tile_n = tile / p.tiles_m;
+    w.m0 = w.tile_m * p.tile_rows;
+    w.n0 = w.tile_n * kBN;
+    w.kb_begin = w.split * p.kb_per_split;
+    const int kb_end = w.kb_begin + p.kb_per_split < p.kb_total ? w.kb_begin + p.kb_per_split : p.kb_total;
+    w.num_kb = kb_end - w.kb_begin;
+    return w;
+}
 
 // Shared-memory matrix descriptor.  Addresses and offsets are stored in 16-byte units.
 //   K-major tile (layout 2, 128-byte swizzle of 16-byte chunks): rows of 128 bytes (32 K
@@ -130,6 +166,13 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
 
+    if (p.mode == 2) {
+        // Filter gradient: a stage holds fewer than 32 pixel rows of K; the rows TMA never writes
+        // must read as zero in both operands.
+        float4* z = reinterpret_cast<float4*>(smem_raw + (tiles - raw));
+        for (uint32_t i = threadIdx.x; i < kStages * kStageBytes / 16; i += kThreads) z[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        ptx::fence_proxy_async();
+    }
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
             ptx::mbar_init(full_bar(s), 1);
@@ -154,8 +197,7 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
 
-    const int num_tiles = p.tiles_m * p.tiles_n;
-    const int num_kb = (p.K + kBK - 1) / kBK;
+    const int num_work = p.tiles_m * p.tiles_n * p.splits;
 
     // Registers are allocated per group of four warps: the producer/MMA group keeps 64 per thread,
     // the accumulate groups take 224 (128 running sums + 32 freshly loaded values + addressing).
@@ -166,10 +208,10 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
         if (lane == 0) {
             int stage = 0;
             uint32_t phase = 0;
-            for (int t = blockIdx.x; t < num_tiles && !*abort_flag; t += gridDim.x) {
-                const int m0 = (t % p.tiles_m) * kBM;
-                const int n0 = (t / p.tiles_m) * kBN;
-                for (int kb = 0; kb < num_kb; ++kb) {
+            for (int t = blockIdx.x; t < num_work && !*abort_flag; t += gridDim.x) {
+                const WorkItem w = decode_work(p, t);
+                const int m0 = w.m0, n0 = w.n0;
+                for (int kb = w.kb_begin; kb < w.kb_begin + w.num_kb; ++kb) {
                     if (!ptx::mbar_wait_bounded(empty_bar(stage), phase ^ 1u, kWaitLimit)) {
                         raise_timeout(p, abort_flag);
                         break;
@@ -177,19 +219,55 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                     if (*abort_flag) break;
                     const uint32_t sa = tiles + stage * kStageBytes;
                     const uint32_t sb = sa + kABytes;
-                    const int k0 = kb * kBK;
-                    ptx::mbar_expect_tx(full_bar(stage), kStageBytes);
-                    if (p.a_mn_major) {
-                        for (int c = 0; c < kBM / 32; ++c)
-                            ptx::tma_load_2d(sa + c * 4096u, &tmap_a, full_bar(stage), m0 + c * 32, k0);
+                    const uint32_t bar = full_bar(stage);
+                    ptx::mbar_expect_tx(bar, p.a_bytes + p.b_bytes);
+                    if (p.mode == 0) {
+                        const int k0 = kb * kBK;
+                        if (p.a_mn_major) {
+                            for (int c = 0; c < kBM / 32; ++c)
+                                ptx::tma_load_2d(sa + c * 4096u, &tmap_a, bar, m0 + c * 32, k0);
+                        } else {
+                            ptx::tma_load_2d(sa, &tmap_a, bar, k0, m0);
+                        }
+                        if (p.b_mn_major) {
+                            for (int c = 0; c < kBN / 32; ++c)
+                                ptx::tma_load_2d(sb + c * 4096u, &tmap_b, bar, n0 + c * 32, k0);
+                        } else {
+                            ptx::tma_load_2d(sb, &tmap_b, bar, k0, n0);
+                        }
+                    } else if (p.mode == 1) {
+                        // A: one box of img_w pixels x 32 channels per image row of the tile, read at
+                        // the tap's offset (rows and columns outside the image read as zero: padding).
+                        const int tap = kb / p.cblocks, cb = kb % p.cblocks;
+                        const int dh = p.tap_sign * (tap / p.taps_s) + p.off_h;
+                        const int dw = p.tap_sign * (tap % p.taps_s) + p.off_w;
+                        for (int j = 0; j < p.rows_per_blk; ++j) {
+                            const int q = w.tile_m * p.rows_per_blk + j;
+                            ptx::tma_load_4d(sa + (uint32_t)(j * p.img_w) * 128u, &tmap_a, bar, cb * 32, dw,
+                                             q % p.img_rows + dh, q / p.img_rows);
+                        }
+                        if (p.b_mn_major) {  // data gradient: filters [C_out][tap][C_in], C_in is N
+                            for (int c = 0; c < kBN / 32; ++c)
+                                ptx::tma_load_3d(sb + c * 4096u, &tmap_b, bar, n0 + c * 32, tap, cb * 32);
+                        } else {             // forward: filters [C_out][tap * C_in], K contiguous
+                            ptx::tma_load_2d(sb, &tmap_b, bar, tap * p.ck + cb * 32, n0);
+                        }
                     } else {
-                        ptx::tma_load_2d(sa, &tmap_a, full_bar(stage), k0, m0);
-                    }
-                    if (p.b_mn_major) {
-                        for (int c = 0; c < kBN / 32; ++c)
-                            ptx::tma_load_2d(sb + c * 4096u, &tmap_b, full_bar(stage), n0 + c * 32, k0);
-                    } else {
-                        ptx::tma_load_2d(sb, &tmap_b, full_bar(stage), k0, n0);
+                        // Filter gradient: K = pixels.  A = output gradient (C_out is M), B = activations
+                        // read at the tap that the N column block belongs to (C_in within a tap is N).
+                        for (int j = 0; j < p.rows_per_blk; ++j) {
+                            const int q = kb * p.rows_per_blk + j;
+                            const int oh = q % p.img_rows, img = q / p.img_rows;
+                            const uint32_t row_off = (uint32_t)(j * p.img_w) * 128u;
+                            for (int c = 0; c < kBM / 32; ++c)
+                                ptx::tma_load_4d(sa + c * 4096u + row_off, &tmap_a, bar, m0 + c * 32, 0, oh, img);
+                            for (int c = 0; c < kBN / 32; ++c) {
+                                const int col = n0 + c * 32;
+                                const int tap = col / p.ck, ci = col % p.ck;
+                                ptx::tma_load_4d(sb + c * 4096u + row_off, &tmap_b, bar, ci, tap % p.taps_s + p.off_w,
+                                                 oh + tap / p.taps_s + p.off_h, img);
+                            }
+                        }
                     }
                     if (++stage == kStages) { stage = 0; phase ^= 1u; }
                 }
@@ -211,7 +289,8 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
             uint32_t phase = 0;
             uint32_t acc_iter = 0;  // chunks issued so far: buffer = acc_iter & 1, phase = (acc_iter >> 1) & 1
             bool dead = false;
-            for (int t = blockIdx.x; t < num_tiles && !dead; t += gridDim.x) {
+            for (int t = blockIdx.x; t < num_work && !dead; t += gridDim.x) {
+                const int num_kb = decode_work(p, t).num_kb;
                 for (int kb0 = 0; kb0 < num_kb && !dead; kb0 += kChunkKB) {
                     const uint32_t acc = acc_iter & 1u, acc_phase = (acc_iter >> 1) & 1u;
                     if (!ptx::mbar_wait_bounded(acc_empty_bar(acc), acc_phase ^ 1u, kWaitLimit)) {
@@ -256,9 +335,15 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
         const int half = (warp - 4) >> 2;      // columns [128*half, 128*half+128) of the tile
         uint32_t acc_iter = 0;
         bool dead = false;
-        for (int t = blockIdx.x; t < num_tiles && !dead; t += gridDim.x) {
-            const int m0 = (t % p.tiles_m) * kBM;
-            const int n0 = (t / p.tiles_m) * kBN;
+        for (int t = blockIdx.x; t < num_work && !dead; t += gridDim.x) {
+            const WorkItem w = decode_work(p, t);
+            const int m0 = w.m0, n0 = w.n0, num_kb = w.num_kb;
+            // rows of C this tile may write, and where split results go
+            const int m_end = m0 + p.tile_rows < p.M ? m0 + p.tile_rows : p.M;
+            float* const c_base = p.C + (long long)w.split * p.split_stride;
+            // In mode 1 the C tensor map is [complete tiles][tile_rows][N]; an incomplete last tile
+            // takes the scalar path.
+            const bool use_tma = p.tma_store && (p.mode != 1 || w.tile_m < p.full_tiles_m);
             float sum[128];  // level-1 running sums; 0 + x is exact, so a group's first chunk needs no special case
 #pragma unroll
             for (int j = 0; j < 128; ++j) sum[j] = 0.0f;
@@ -304,7 +389,7 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                 if (!last && ++in_group < kFlushChunks) continue;
                 // ---- move the level-1 sums to C (level 2): registers -> swizzled shared boxes -> TMA.
                 // The first group of a tile is stored, later groups are added at the destination.
-                if (p.tma_store && flushed) {
+                if (use_tma && flushed) {
                     if (lane == 0) ptx::bulk_wait_all();  // the earlier store/add to these addresses is complete
                 }
 #pragma unroll
@@ -320,14 +405,16 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                         *reinterpret_cast<float4*>(box + lane * 32 + ((c ^ (lane & 7)) << 2)) =
                             make_float4(sum[j], sum[j + 1], sum[j + 2], sum[j + 3]);
                     }
-                    if (p.tma_store) {
+                    if (use_tma) {
                         ptx::fence_proxy_async();
                         __syncwarp();
                         if (lane == 0) {
-                            if (row0 < p.M && col0 < p.N) {
+                            if (row0 < m_end && col0 < p.N) {
                                 const uint32_t src = my_stage_addr + (pass & 1) * kOutBoxBytes;
-                                if (flushed) ptx::tma_reduce_add_2d(&tmap_c, src, col0, row0);
-                                else ptx::tma_store_2d(&tmap_c, src, col0, row0);
+                                const int y = p.mode == 1 ? quad * 32 : row0;
+                                const int z = p.mode == 1 ? w.tile_m : w.split;
+                                if (flushed) ptx::tma_reduce_add_3d(&tmap_c, src, col0, y, z);
+                                else ptx::tma_store_3d(&tmap_c, src, col0, y, z);
                             }
                             ptx::bulk_commit();  // committed even when empty: the wait above counts groups
                         }
@@ -335,10 +422,10 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                         __syncwarp();
                         for (int r = 0; r < 32; ++r) {
                             const int row = row0 + r;
-                            if (row >= p.M) break;
+                            if (row >= m_end) break;
                             const int c = lane;
                             if (col0 + c < p.N) {
-                                float* g = p.C + (long long)row * p.ldc + col0 + c;
+                                float* g = c_base + (long long)row * p.ldc + col0 + c;
                                 const float v = box[r * 32 + (((c >> 2) ^ (r & 7)) << 2) + (c & 3)];
                                 *g = flushed ? __fadd_rn(*g, v) : v;
                             }
@@ -391,24 +478,87 @@ EncodeTiledFn encode_tiled_fn() {
     return fn;
 }
 
-// 2-D fp32 tensor map with dim0 contiguous; box (box0, box1); zero fill out of bounds.
-// Swizzle: 16-byte chunks within 128 bytes for K-major tiles and for C, 32-byte chunks for
-// MN-major operand tiles.
-int make_map_2d(CUtensorMap* map, const float* base, uint64_t dim0, uint64_t dim1, uint64_t ld_elems,
-                uint32_t box0, uint32_t box1, bool mn_major) {
+// fp32 tensor map of rank 2..4 with dim0 contiguous; strides in elements for dims 1..rank-1; zero
+// fill out of bounds.  Swizzle: 16-byte chunks within 128 bytes for K-major operand tiles and for
+// C, 32-byte chunks for MN-major operand tiles.
+int make_map(CUtensorMap* map, const float* base, int rank, const uint64_t* dims, const uint64_t* strides_elems,
+             const uint32_t* box, bool mn_major) {
     EncodeTiledFn fn = encode_tiled_fn();
     if (fn == nullptr) { set_last_cuda_error((int)cudaErrorSymbolNotFound); return QFMT_ERR_CUDA; }
-    cuuint64_t dims[2] = {dim0, dim1};
-    cuuint64_t strides[1] = {ld_elems * sizeof(float)};
-    cuuint32_t box[2] = {box0, box1};
-    cuuint32_t estr[2] = {1, 1};
-    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(base), dims, strides, box, estr,
+    cuuint64_t d[4], st[3];
+    cuuint32_t bx[4], estr[4] = {1, 1, 1, 1};
+    for (int i = 0; i < rank; ++i) { d[i] = dims[i]; bx[i] = box[i]; }
+    for (int i = 0; i + 1 < rank; ++i) st[i] = strides_elems[i] * sizeof(float);
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, (cuuint32_t)rank, const_cast<float*>(base), d, st, bx, estr,
                     CU_TENSOR_MAP_INTERLEAVE_NONE,
                     mn_major ? CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B : CU_TENSOR_MAP_SWIZZLE_128B,
-                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) { set_last_cuda_error(100000 + (int)r); return QFMT_ERR_CUDA; }
     return QFMT_OK;
+}
+
+int make_map_2d(CUtensorMap* map, const float* base, uint64_t dim0, uint64_t dim1, uint64_t ld_elems,
+                uint32_t box0, uint32_t box1, bool mn_major) {
+    const uint64_t dims[2] = {dim0, dim1}, strides[1] = {ld_elems};
+    const uint32_t box[2] = {box0, box1};
+    return make_map(map, base, 2, dims, strides, box, mn_major);
+}
+
+// C (or the split-K partials) as a rank-3 map: [z][rows][N] with 32 x 32 x 1 boxes.
+int make_map_c(CUtensorMap* map, float* base, uint64_t n, uint64_t rows, uint64_t zdim, uint64_t ld, uint64_t zstride) {
+    const uint64_t dims[3] = {n, rows, zdim}, strides[2] = {ld, zstride};
+    const uint32_t box[3] = {32, 32, 1};
+    return make_map(map, base, 3, dims, strides, box, false);
+}
+
+// Sums the split-K partials [splits][rows][cols] (dense) into C in a fixed pairwise order.
+__global__ void __launch_bounds__(256)
+splitk_reduce_kernel(const float* __restrict__ part, float* __restrict__ C, long long rows, long long cols,
+                     long long ldc, int splits) {
+    const long long total = rows * cols;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total;
+         i += (long long)gridDim.x * blockDim.x) {
+        float v[32];
+        for (int s = 0; s < splits; ++s) v[s] = part[(long long)s * total + i];
+        int n = splits;
+        while (n > 1) {  // pairwise tree, the same order on every run
+            const int h = n / 2;
+            for (int s = 0; s < h; ++s) v[s] = __fadd_rn(v[2 * s], v[2 * s + 1]);
+            if (n & 1) { v[h] = v[n - 1]; n = h + 1; } else { n = h; }
+        }
+        C[(i / cols) * ldc + (i % cols)] = v[0];
+    }
+}
+
+constexpr size_t kWorkspaceHeader = 256;  // status word and padding ahead of the partial sums
+constexpr int kMaxSplits = 32;
+
+int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc, const GemmParams& p,
+                const DeviceInfo& dev, cudaStream_t stream) {
+    static bool attr_set[64] = {};
+    if (dev.ordinal < 0 || dev.ordinal >= 64 || !attr_set[dev.ordinal]) {
+        QFMT_CUDA_TRY(cudaFuncSetAttribute(gemm_tf32_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes));
+        if (dev.ordinal >= 0 && dev.ordinal < 64) attr_set[dev.ordinal] = true;
+    }
+    const long long work = (long long)p.tiles_m * p.tiles_n * p.splits;
+    const int grid = work < dev.sm_count ? (int)work : dev.sm_count;
+    gemm_tf32_kernel<<<grid, kThreads, kSmemBytes, stream>>>(ma, mb, mc, p);
+    QFMT_CUDA_TRY(cudaGetLastError());
+    return QFMT_OK;
+}
+
+void dense_defaults(GemmParams* p) {
+    p->mode = 0;
+    p->tile_rows = kBM;
+    p->splits = 1;
+    p->split_stride = 0;
+    p->a_bytes = kABytes;
+    p->b_bytes = kBBytes;
+    p->img_rows = p->img_w = p->total_q = p->rows_per_blk = 1;
+    p->taps = p->taps_s = p->cblocks = p->ck = 1;
+    p->tap_sign = 1;
+    p->off_h = p->off_w = 0;
+    p->full_tiles_m = 0;
 }
 
 }  // namespace
@@ -447,6 +597,7 @@ int gemm_device(const qfmt_matrix_t* A, const qfmt_matrix_t* B, float* d_C, int6
     }
 
     GemmParams p;
+    dense_defaults(&p);
     p.M = (int)M; p.N = (int)N; p.K = (int)K;
     p.ldc = ldc;
     p.C = d_C;
@@ -455,6 +606,8 @@ int gemm_device(const qfmt_matrix_t* A, const qfmt_matrix_t* B, float* d_C, int6
     p.b_mn_major = B->trans ? 0 : 1;
     p.tiles_m = (int)((M + kBM - 1) / kBM);
     p.tiles_n = (int)((N + kBN - 1) / kBN);
+    p.kb_total = (int)((K + kBK - 1) / kBK);
+    p.kb_per_split = p.kb_total;
     // TMA stores clip at 16-byte granularity along the row, so N must be a multiple of 4 as well.
     p.tma_store = ((reinterpret_cast<uintptr_t>(d_C) & 15u) == 0 && (ldc & 3) == 0 && (N & 3) == 0) ? 1 : 0;
 
@@ -465,20 +618,187 @@ int gemm_device(const qfmt_matrix_t* A, const qfmt_matrix_t* B, float* d_C, int6
     if (p.b_mn_major) rc = make_map_2d(&mb, B->ptr, (uint64_t)N, (uint64_t)K, (uint64_t)B->ld, 32, kBK, true);
     else rc = make_map_2d(&mb, B->ptr, (uint64_t)K, (uint64_t)N, (uint64_t)B->ld, kBK, kBN, false);
     if (rc != QFMT_OK) return rc;
-
-    if (p.tma_store) rc = make_map_2d(&mc, d_C, (uint64_t)N, (uint64_t)M, (uint64_t)ldc, 32, 32, false);
+    if (p.tma_store) rc = make_map_c(&mc, d_C, (uint64_t)N, (uint64_t)M, 1, (uint64_t)ldc, (uint64_t)M * (uint64_t)ldc);
     else mc = ma;  // unused by the kernel
     if (rc != QFMT_OK) return rc;
+    return launch_gemm(ma, mb, mc, p, dev, stream);
+}
 
-    static bool attr_set[64] = {};
-    if (dev.ordinal < 0 || dev.ordinal >= 64 || !attr_set[dev.ordinal]) {
-        QFMT_CUDA_TRY(cudaFuncSetAttribute(gemm_tf32_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes));
-        if (dev.ordinal >= 0 && dev.ordinal < 64) attr_set[dev.ordinal] = true;
+// ------------------------------------------------------------------------------------------------
+// Convolution layers as implicit GEMMs on channels-last tensors (unit stride, zero padding).
+// ------------------------------------------------------------------------------------------------
+namespace {
+struct ConvPlan {
+    int64_t oh, ow;
+    int splits;
+    size_t workspace;
+};
+constexpr int kPlanSms = 148;  // B200; the split factor is planned for it so that it does not vary
+int plan_conv(int op, const qfmt_conv_t* g, ConvPlan* plan) {
+    if (g == nullptr || op < QFMT_CONV_FWD || op > QFMT_CONV_WGRAD) return QFMT_ERR_BAD_ARG;
+    if (g->n <= 0 || g->c_in <= 0 || g->h <= 0 || g->w <= 0 || g->c_out <= 0 || g->r <= 0 || g->s <= 0 ||
+        g->pad_h < 0 || g->pad_w < 0)
+        return QFMT_ERR_BAD_ARG;
+    if ((g->c_in & 31) || (g->c_out & 31)) return QFMT_ERR_BAD_ARG;  // 32-channel blocks must not straddle taps
+    plan->oh = (int64_t)g->h + 2 * g->pad_h - g->r + 1;
+    plan->ow = (int64_t)g->w + 2 * g->pad_w - g->s + 1;
+    if (plan->oh <= 0 || plan->ow <= 0) return QFMT_ERR_BAD_ARG;
+    if ((int64_t)g->n * g->h * g->w > (1 << 30) || (int64_t)g->n * plan->oh * plan->ow > (1 << 30) ||
+        (int64_t)g->r * g->s * g->c_in > (1 << 30))
+        return QFMT_ERR_BAD_ARG;
+    plan->splits = 1;
+    plan->workspace = kWorkspaceHeader;
+    if (op == QFMT_CONV_FWD && plan->ow > kBM) return QFMT_ERR_BAD_ARG;   // an M-tile is made of whole output rows
+    if (op == QFMT_CONV_DGRAD && g->w > kBM) return QFMT_ERR_BAD_ARG;
+    if (op == QFMT_CONV_WGRAD) {
+        if (plan->ow > kBK) return QFMT_ERR_BAD_ARG;                      // a stage is made of whole output rows
+        const int rows_per_blk = kBK / (int)plan->ow;
+        const int64_t kb_total = ((int64_t)g->n * plan->oh + rows_per_blk - 1) / rows_per_blk;
+        const int64_t tiles = (((int64_t)g->c_out + kBM - 1) / kBM) * (((int64_t)g->r * g->s * g->c_in + kBN - 1) / kBN);
+        int64_t splits = kPlanSms / tiles;
+        if (splits > kMaxSplits) splits = kMaxSplits;
+        if (splits > kb_total / 8) splits = kb_total / 8;   // at least eight stages per split
+        if (splits < 1) splits = 1;
+        const int64_t per = (kb_total + splits - 1) / splits;
+        plan->splits = (int)((kb_total + per - 1) / per);
+        if (plan->splits > 1)
+            plan->workspace += (size_t)plan->splits * (size_t)g->c_out * (size_t)g->r * g->s * g->c_in * sizeof(float);
     }
-    const int num_tiles = p.tiles_m * p.tiles_n;
-    const int grid = num_tiles < dev.sm_count ? num_tiles : dev.sm_count;
-    gemm_tf32_kernel<<<grid, kThreads, kSmemBytes, stream>>>(ma, mb, mc, p);
-    QFMT_CUDA_TRY(cudaGetLastError());
+    return QFMT_OK;
+}
+}  // namespace
+
+int conv_device(int op, const qfmt_conv_t* g, const float* d_p, const float* d_q, float* d_out,
+                const qfmt_format_t* fmt, void* d_workspace, size_t workspace_bytes, cudaStream_t stream) {
+    int rc = validate_format(fmt);
+    if (rc != QFMT_OK) return rc;
+    if (fmt->m > 10) return QFMT_ERR_BAD_FORMAT;
+    DeviceInfo dev;
+    rc = current_device(&dev);
+    if (rc != QFMT_OK) return rc;
+    ConvPlan plan;
+    rc = plan_conv(op, g, &plan);
+    if (rc != QFMT_OK) return rc;
+    if (d_p == nullptr || d_q == nullptr || d_out == nullptr) return QFMT_ERR_BAD_ARG;
+    if ((reinterpret_cast<uintptr_t>(d_p) & 15u) || (reinterpret_cast<uintptr_t>(d_q) & 15u) ||
+        (reinterpret_cast<uintptr_t>(d_out) & 15u))
+        return QFMT_ERR_BAD_ARG;
+    if (d_workspace == nullptr || workspace_bytes < plan.workspace || (reinterpret_cast<uintptr_t>(d_workspace) & 15u))
+        return QFMT_ERR_BAD_ARG;
+    int* status = reinterpret_cast<int*>(d_workspace);
+    QFMT_CUDA_TRY(cudaMemsetAsync(status, 0, 16, stream));
+
+    const uint64_t N = g->n, CI = g->c_in, H = g->h, W = g->w, CO = g->c_out, R = g->r, S = g->s;
+    const uint64_t OH = plan.oh, OW = plan.ow, TAPS = R * S;
+    GemmParams p;
+    dense_defaults(&p);
+    p.status = status;
+    p.taps = (int)TAPS;
+    p.taps_s = (int)S;
+    p.tma_store = 1;  // channel counts are multiples of 32 and the bases 16-byte aligned
+    CUtensorMap ma, mb, mc;
+
+    if (op == QFMT_CONV_FWD || op == QFMT_CONV_DGRAD) {
+        const bool fwd = op == QFMT_CONV_FWD;
+        // pixel space that is tiled: the output of the product
+        const uint64_t rows = fwd ? OH : H, width = fwd ? OW : W;
+        // activation-like operand that is read: X [N][H][W][CI] forward, dY [N][OH][OW][CO] data gradient
+        const uint64_t src_h = fwd ? H : OH, src_w = fwd ? W : OW, src_c = fwd ? CI : CO;
+        const uint64_t n_cols = fwd ? CO : CI;
+        p.mode = 1;
+        p.img_rows = (int)rows;
+        p.img_w = (int)width;
+        p.total_q = (int)(N * rows);
+        p.rows_per_blk = kBM / (int)width;
+        p.tile_rows = p.rows_per_blk * (int)width;
+        p.M = (int)(N * rows * width);
+        p.N = (int)n_cols;
+        p.K = (int)(TAPS * src_c);
+        p.ldc = (long long)n_cols;
+        p.C = d_out;
+        p.ck = (int)src_c;
+        p.cblocks = (int)(src_c / 32);
+        p.kb_total = (int)TAPS * p.cblocks;
+        p.kb_per_split = p.kb_total;
+        p.tap_sign = fwd ? 1 : -1;
+        p.off_h = fwd ? -g->pad_h : g->pad_h;
+        p.off_w = fwd ? -g->pad_w : g->pad_w;
+        p.tiles_m = (p.total_q + p.rows_per_blk - 1) / p.rows_per_blk;
+        p.tiles_n = (int)((n_cols + kBN - 1) / kBN);
+        p.full_tiles_m = p.total_q / p.rows_per_blk;
+        p.a_mn_major = 0;
+        p.b_mn_major = fwd ? 0 : 1;
+        p.a_bytes = (uint32_t)(p.tile_rows * 128);
+        p.b_bytes = kBBytes;
+        {
+            const uint64_t dims[4] = {src_c, src_w, src_h, N}, st[3] = {src_c, src_w * src_c, src_h * src_w * src_c};
+            const uint32_t box[4] = {32, (uint32_t)width, 1, 1};
+            rc = make_map(&ma, d_p, 4, dims, st, box, false);
+            if (rc != QFMT_OK) return rc;
+        }
+        if (fwd) {  // filters [CO][TAPS*CI], K contiguous
+            rc = make_map_2d(&mb, d_q, TAPS * CI, CO, TAPS * CI, kBK, kBN, false);
+        } else {    // filters [CO][TAPS][CI]: N = CI contiguous, K = CO rows
+            const uint64_t dims[3] = {CI, TAPS, CO}, st[2] = {CI, TAPS * CI};
+            const uint32_t box[3] = {32, 1, kBK};
+            rc = make_map(&mb, d_q, 3, dims, st, box, true);
+        }
+        if (rc != QFMT_OK) return rc;
+        if (p.full_tiles_m > 0)
+            rc = make_map_c(&mc, d_out, n_cols, (uint64_t)p.tile_rows, (uint64_t)p.full_tiles_m, n_cols,
+                            (uint64_t)p.tile_rows * n_cols);
+        else { mc = ma; p.tma_store = 0; }
+        if (rc != QFMT_OK) return rc;
+        return launch_gemm(ma, mb, mc, p, dev, stream);
+    }
+
+    // ---- filter gradient: dW [CO][TAPS*CI] = sum over pixels of dY^T (CO x pixels) * X_tap (pixels x CI)
+    p.mode = 2;
+    p.img_rows = (int)OH;
+    p.img_w = (int)OW;
+    p.total_q = (int)(N * OH);
+    p.rows_per_blk = kBK / (int)OW;
+    p.M = (int)CO;
+    p.N = (int)(TAPS * CI);
+    p.K = (int)(N * OH * OW);
+    p.ck = (int)CI;
+    p.off_h = -g->pad_h;
+    p.off_w = -g->pad_w;
+    p.tiles_m = (int)((CO + kBM - 1) / kBM);
+    p.tiles_n = (p.N + kBN - 1) / kBN;
+    p.kb_total = (p.total_q + p.rows_per_blk - 1) / p.rows_per_blk;
+    p.splits = plan.splits;
+    p.kb_per_split = (p.kb_total + p.splits - 1) / p.splits;
+    p.a_mn_major = 1;
+    p.b_mn_major = 1;
+    p.a_bytes = (uint32_t)((kBM / 32) * p.rows_per_blk * (int)OW * 128);
+    p.b_bytes = (uint32_t)((kBN / 32) * p.rows_per_blk * (int)OW * 128);
+    float* partials = reinterpret_cast<float*>(reinterpret_cast<char*>(d_workspace) + kWorkspaceHeader);
+    p.ldc = (long long)p.N;
+    p.C = p.splits > 1 ? partials : d_out;
+    p.split_stride = (long long)p.M * p.N;
+    {
+        const uint64_t dims[4] = {CO, OW, OH, N}, st[3] = {CO, OW * CO, OH * OW * CO};
+        const uint32_t box[4] = {32, (uint32_t)OW, 1, 1};
+        rc = make_map(&ma, d_p, 4, dims, st, box, true);
+        if (rc != QFMT_OK) return rc;
+    }
+    {
+        const uint64_t dims[4] = {CI, W, H, N}, st[3] = {CI, W * CI, H * W * CI};
+        const uint32_t box[4] = {32, (uint32_t)OW, 1, 1};
+        rc = make_map(&mb, d_q, 4, dims, st, box, true);
+        if (rc != QFMT_OK) return rc;
+    }
+    rc = make_map_c(&mc, p.C, (uint64_t)p.N, (uint64_t)p.M, (uint64_t)p.splits, (uint64_t)p.N, (uint64_t)p.M * p.N);
+    if (rc != QFMT_OK) return rc;
+    rc = launch_gemm(ma, mb, mc, p, dev, stream);
+    if (rc != QFMT_OK) return rc;
+    if (p.splits > 1) {
+        const long long total = (long long)p.M * p.N;
+        const int blocks = (int)((total + 255) / 256 < (long long)dev.sm_count * 8 ? (total + 255) / 256 : dev.sm_count * 8);
+        splitk_reduce_kernel<<<blocks, 256, 0, stream>>>(partials, d_out, p.M, p.N, p.N, p.splits);
+        QFMT_CUDA_TRY(cudaGetLastError());
+    }
     return QFMT_OK;
 }
 
@@ -487,6 +807,17 @@ int gemm_device(const qfmt_matrix_t* A, const qfmt_matrix_t* B, float* d_C, int6
 extern "C" int qfmt_gemm(const qfmt_matrix_t* A, const qfmt_matrix_t* B, float* d_C, int64_t ldc,
                          const qfmt_format_t* fmt, void* d_workspace, size_t workspace_bytes, void* stream) {
     return qfmt::gemm_device(A, B, d_C, ldc, fmt, d_workspace, workspace_bytes, (cudaStream_t)stream);
+}
+
+extern "C" int qfmt_conv(int32_t op, const qfmt_conv_t* geom, const float* d_p, const float* d_q, float* d_out,
+                         const qfmt_format_t* fmt, void* d_workspace, size_t workspace_bytes, void* stream) {
+    return qfmt::conv_device(op, geom, d_p, d_q, d_out, fmt, d_workspace, workspace_bytes, (cudaStream_t)stream);
+}
+
+extern "C" size_t qfmt_conv_workspace_bytes(int32_t op, const qfmt_conv_t* geom) {
+    qfmt::ConvPlan plan;
+    if (qfmt::plan_conv(op, geom, &plan) != QFMT_OK) return 0;
+    return plan.workspace;
 }
 
 extern "C" size_t qfmt_gemm_workspace_bytes(const qfmt_matrix_t* A, const qfmt_matrix_t* B) {

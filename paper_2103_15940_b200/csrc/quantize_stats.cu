@@ -223,6 +223,58 @@ quantize_stats_scalar_kernel(const uint32_t* in, uint32_t* out, unsigned long lo
     }
 }
 
+// Rounding with a batched transpose: in is [batch][rows][cols], out is [batch][cols][rows].
+// 32 x 32 tiles go through shared memory so that both the reads (along cols) and the writes
+// (along rows) are 128-byte segments; statistics as in the flat kernel.
+constexpr int kTThreads = 256;
+template <bool kStats, bool kScale>
+__global__ void __launch_bounds__(kTThreads)
+quantize_stats_transpose_kernel(const uint32_t* __restrict__ in, uint32_t* __restrict__ out, unsigned batch,
+                                unsigned rows, unsigned cols, QuantParams p, qfmt_stats_t* __restrict__ stats,
+                                unsigned long long n_total) {
+    extern __shared__ uint32_t lane_hist[];  // [(top + kExtraBins)][32]
+    __shared__ uint32_t tile[32][33];
+    const int nbins = p.top + kExtraBins;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (kStats) {
+        for (int i = threadIdx.x; i < nbins * 32; i += kTThreads) lane_hist[i] = 0u;
+    }
+    const unsigned tr = (rows + 31) / 32, tc = (cols + 31) / 32;
+    const unsigned long long tiles = (unsigned long long)batch * tr * tc;
+    for (unsigned long long t = blockIdx.x; t < tiles; t += gridDim.x) {
+        const unsigned b = (unsigned)(t / ((unsigned long long)tr * tc));
+        const unsigned rem = (unsigned)(t % ((unsigned long long)tr * tc));
+        const unsigned r0 = (rem / tc) * 32, c0 = (rem % tc) * 32;
+        const unsigned long long base = (unsigned long long)b * rows * cols;
+        __syncthreads();  // previous tile fully written out (and the histogram cleared)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const unsigned r = r0 + warp + 8 * i, c = c0 + lane;
+            if (r < rows && c < cols) {
+                int bin;
+                const uint32_t q = quantize_one<kScale>(in[base + (unsigned long long)r * cols + c], p, bin);
+                tile[warp + 8 * i][lane] = q;
+                if (kStats) atomicAdd(&lane_hist[bin * 32 + lane], 1u);
+            }
+        }
+        __syncthreads();
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const unsigned c = c0 + warp + 8 * i, r = r0 + lane;
+            if (r < rows && c < cols) out[base + (unsigned long long)c * rows + r] = tile[lane][warp + 8 * i];
+        }
+    }
+    if (kStats) {
+        __syncthreads();
+        for (int b = warp + 1; b < nbins; b += kTThreads / 32) {
+            const uint32_t c = __reduce_add_sync(0xFFFFFFFFu, lane_hist[b * 32 + lane]);
+            if (lane == 0 && c != 0u) merge_bin(stats, p, b, c);
+        }
+        if (blockIdx.x == 0 && threadIdx.x == 0 && n_total != 0ull)
+            atomicAdd((unsigned long long*)&stats->n_total, n_total);
+    }
+}
+
 QuantParams make_params(const qfmt_format_t& f) {
     QuantParams p;
     const int bias = (1 << (f.e - 1)) - 1;
@@ -308,11 +360,55 @@ int quantize_stats_device(const float* d_in, float* d_out, size_t n, const qfmt_
     return QFMT_OK;
 }
 
+
+int quantize_stats_transpose_device(const float* d_in, float* d_out, int64_t batch, int64_t rows, int64_t cols,
+                                    const qfmt_format_t* fmt, qfmt_stats_t* d_stats, int accumulate,
+                                    cudaStream_t stream) {
+    int rc = validate_format(fmt);
+    if (rc != QFMT_OK) return rc;
+    if (accumulate != 0 && accumulate != 1) return QFMT_ERR_BAD_ARG;
+    if (batch < 0 || rows < 0 || cols < 0 || batch > 0x7FFFFFFF || rows > 0x7FFFFFFF || cols > 0x7FFFFFFF)
+        return QFMT_ERR_BAD_ARG;
+    const unsigned long long n = (unsigned long long)batch * (unsigned long long)rows * (unsigned long long)cols;
+    if (n > (1ull << 40)) return QFMT_ERR_BAD_ARG;
+    if (n != 0 && (d_in == nullptr || d_out == nullptr || d_in == d_out)) return QFMT_ERR_BAD_ARG;
+    if ((reinterpret_cast<uintptr_t>(d_in) & 3u) || (reinterpret_cast<uintptr_t>(d_out) & 3u) ||
+        (reinterpret_cast<uintptr_t>(d_stats) & 7u))
+        return QFMT_ERR_BAD_ARG;
+    DeviceInfo dev;
+    rc = current_device(&dev);
+    if (rc != QFMT_OK) return rc;
+    if (d_stats != nullptr && accumulate == 0) QFMT_CUDA_TRY(cudaMemsetAsync(d_stats, 0, sizeof(qfmt_stats_t), stream));
+    if (n == 0) return QFMT_OK;
+    const QuantParams p = make_params(*fmt);
+    const uint32_t* in = reinterpret_cast<const uint32_t*>(d_in);
+    uint32_t* out = reinterpret_cast<uint32_t*>(d_out);
+    const bool has_stats = d_stats != nullptr, has_scale = fmt->loss_scale != 1.0f;
+    const size_t smem = has_stats ? (size_t)(p.top + kExtraBins) * 32 * sizeof(uint32_t) : 0;
+    const unsigned long long tiles = (unsigned long long)batch * ((rows + 31) / 32) * ((cols + 31) / 32);
+    unsigned long long want = tiles < (unsigned long long)dev.sm_count * 8 ? tiles : (unsigned long long)dev.sm_count * 8;
+#define QFMT_TLAUNCH(S, C)                                                                                       \
+    quantize_stats_transpose_kernel<S, C><<<(unsigned)want, kTThreads, smem, stream>>>(                          \
+        in, out, (unsigned)batch, (unsigned)rows, (unsigned)cols, p, d_stats, n)
+    if (has_stats) { if (has_scale) QFMT_TLAUNCH(true, true); else QFMT_TLAUNCH(true, false); }
+    else { if (has_scale) QFMT_TLAUNCH(false, true); else QFMT_TLAUNCH(false, false); }
+#undef QFMT_TLAUNCH
+    QFMT_CUDA_TRY(cudaGetLastError());
+    return QFMT_OK;
+}
+
 }  // namespace qfmt
 
 extern "C" int qfmt_quantize_stats(const float* d_in, float* d_out, size_t n, const qfmt_format_t* fmt,
                                    qfmt_stats_t* d_stats, int accumulate, void* stream) {
     return qfmt::quantize_stats_device(d_in, d_out, n, fmt, d_stats, accumulate, (cudaStream_t)stream);
+}
+
+extern "C" int qfmt_quantize_stats_transpose(const float* d_in, float* d_out, int64_t batch, int64_t rows, int64_t cols,
+                                             const qfmt_format_t* fmt, qfmt_stats_t* d_stats, int accumulate,
+                                             void* stream) {
+    return qfmt::quantize_stats_transpose_device(d_in, d_out, batch, rows, cols, fmt, d_stats, accumulate,
+                                                 (cudaStream_t)stream);
 }
 
 extern "C" size_t qfmt_quantize_stats_host_work_bytes(size_t n) {

@@ -180,3 +180,22 @@ def test_errors_leave_outputs_untouched():
     assert ei.value.status == qf.QFMT_ERR_BAD_ARG
     torch.cuda.synchronize()
     assert torch.all(d == 1.0)
+
+
+@pytest.mark.parametrize("batch,rows,cols", [(1, 1, 1), (2, 3, 5), (3, 32, 32), (2, 33, 65), (4, 64, 196),
+                                             (5, 256, 9), (1, 100, 1), (7, 1, 50)])
+@pytest.mark.parametrize("e,m,den,scale", [(6, 9, 1, 1.0), (5, 10, 0, 2.0 ** 10), (8, 7, 1, 1.0)])
+def test_transposing_variant(batch, rows, cols, e, m, den, scale):
+    """[batch][rows][cols] -> [batch][cols][rows]: same bits as the oracle's values, permuted; same counts."""
+    x = workloads.lognormal_tensor(workloads.rng_for(70, batch * rows + cols), (batch, rows, cols), -15.0, 7.0, 0.02)
+    q_ref, st_ref = oracle.quantize_stats(x, e, m, den, scale)
+    d_in = torch.from_numpy(x).to("cuda:0")
+    d_out = torch.full((batch * rows * cols + 8,), 7.0, dtype=torch.float32, device="cuda:0")
+    st = torch.full((qf.STATS_WORDS,), 5, dtype=torch.int64, device="cuda:0")
+    qf.qfmt_quantize_stats_transpose(d_in, d_out, batch, rows, cols, qf.make_format(e, m, den, scale), st, 0)
+    torch.cuda.synchronize()
+    got = d_out.cpu().numpy()
+    assert np.all(got[batch * rows * cols:] == 7.0)
+    want = np.ascontiguousarray(q_ref.transpose(0, 2, 1))
+    assert np.array_equal(got[:batch * rows * cols].view(np.uint32), want.reshape(-1).view(np.uint32))
+    assert np.array_equal(st.cpu().numpy().view(np.uint64), st_ref)
