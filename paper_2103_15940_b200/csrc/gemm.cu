@@ -95,6 +95,14 @@ struct GemmParams {
     int full_tiles_m;      // mode 1: M-tiles that are complete (the C tensor map covers exactly these)
 };
 
+// Mode 1 reads the pixel operand through maps whose boxes hold 1 .. kMaxRowMaps whole image rows
+// (32 channels x img_w pixels x cnt rows), so that a tile's rows are fetched with one box per
+// image they touch instead of one box per row.
+constexpr int kMaxRowMaps = 16;
+struct RowMaps {
+    CUtensorMap m[kMaxRowMaps];
+};
+
 // Position of work item t: tile coordinates, split, and the range of stages it sums.
 struct WorkItem {
     int tile_m, tile_n, split, m0, n0, kb_begin, num_kb;
@@ -147,7 +155,8 @@ __device__ __forceinline__ void raise_timeout(const GemmParams& p, volatile int*
 
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tf32_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
-                 const __grid_constant__ CUtensorMap tmap_c, const GemmParams p) {
+                 const __grid_constant__ CUtensorMap tmap_c, const __grid_constant__ RowMaps row_maps,
+                 const GemmParams p) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = ptx::smem_addr(smem_raw);
     const uint32_t tiles = (raw + 1023u) & ~1023u;  // swizzled tiles need 1024-byte alignment
@@ -205,73 +214,116 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     ptx::setmaxnreg_dec<80>();
     if (warp == 0) {
         // ------------------------------ TMA producer ------------------------------
-        if (lane == 0) {
+        if (p.mode != 2) {
+            // Dense operands and the forward / data-gradient convolutions need one to twelve boxes per
+            // stage: a single thread issues them.
+            if (lane == 0) {
+                int stage = 0;
+                uint32_t phase = 0;
+                for (int t = blockIdx.x; t < num_work && !*abort_flag; t += gridDim.x) {
+                    const WorkItem w = decode_work(p, t);
+                    for (int kb = w.kb_begin; kb < w.kb_begin + w.num_kb; ++kb) {
+                        if (!ptx::mbar_wait_bounded(empty_bar(stage), phase ^ 1u, kWaitLimit)) {
+                            raise_timeout(p, abort_flag);
+                            break;
+                        }
+                        if (*abort_flag) break;
+                        const uint32_t sa = tiles + stage * kStageBytes;
+                        const uint32_t sb = sa + kABytes;
+                        const uint32_t bar = full_bar(stage);
+                        ptx::mbar_expect_tx(bar, p.a_bytes + p.b_bytes);
+                        if (p.mode == 0) {
+                            const int k0 = kb * kBK;
+                            if (p.a_mn_major) {
+                                for (int c = 0; c < kBM / 32; ++c)
+                                    ptx::tma_load_2d(sa + c * 4096u, &tmap_a, bar, w.m0 + c * 32, k0);
+                            } else {
+                                ptx::tma_load_2d(sa, &tmap_a, bar, k0, w.m0);
+                            }
+                            if (p.b_mn_major) {
+                                for (int c = 0; c < kBN / 32; ++c)
+                                    ptx::tma_load_2d(sb + c * 4096u, &tmap_b, bar, w.n0 + c * 32, k0);
+                            } else {
+                                ptx::tma_load_2d(sb, &tmap_b, bar, k0, w.n0);
+                            }
+                        } else {
+                            // A: the tile's image rows at this tap's offset, one box per image touched
+                            // (rows and columns outside the image read as zero: that is the padding).
+                            const int tap = kb / p.cblocks, cb = kb % p.cblocks;
+                            const int dh = p.tap_sign * (tap / p.taps_s) + p.off_h;
+                            const int dw = p.tap_sign * (tap % p.taps_s) + p.off_w;
+                            int j = 0;
+                            while (j < p.rows_per_blk) {
+                                const int q = w.tile_m * p.rows_per_blk + j;
+                                const int h = q % p.img_rows, img = q / p.img_rows;
+                                int cnt = p.rows_per_blk - j;
+                                if (cnt > p.img_rows - h) cnt = p.img_rows - h;
+                                if (cnt > kMaxRowMaps) cnt = kMaxRowMaps;
+                                ptx::tma_load_4d(sa + (uint32_t)(j * p.img_w) * 128u, &row_maps.m[cnt - 1], bar, cb * 32, dw,
+                                                 h + dh, img);
+                                j += cnt;
+                            }
+                            if (p.b_mn_major) {  // data gradient: filters [C_out][tap][C_in], C_in is N
+                                for (int c = 0; c < kBN / 32; ++c)
+                                    ptx::tma_load_3d(sb + c * 4096u, &tmap_b, bar, w.n0 + c * 32, tap, cb * 32);
+                            } else {             // forward: filters [C_out][tap * C_in], K contiguous
+                                ptx::tma_load_2d(sb, &tmap_b, bar, tap * p.ck + cb * 32, w.n0);
+                            }
+                        }
+                        if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                    }
+                }
+            }
+        } else {
+        // The filter gradient needs 24 or more small boxes per stage: lane 0 waits for the stage and
+        // arms its barrier, then the lanes issue the boxes in parallel.
+        {
             int stage = 0;
             uint32_t phase = 0;
-            for (int t = blockIdx.x; t < num_work && !*abort_flag; t += gridDim.x) {
+            bool dead = false;
+            for (int t = blockIdx.x; t < num_work && !dead; t += gridDim.x) {
                 const WorkItem w = decode_work(p, t);
                 const int m0 = w.m0, n0 = w.n0;
                 for (int kb = w.kb_begin; kb < w.kb_begin + w.num_kb; ++kb) {
-                    if (!ptx::mbar_wait_bounded(empty_bar(stage), phase ^ 1u, kWaitLimit)) {
-                        raise_timeout(p, abort_flag);
-                        break;
+                    const uint32_t bar = full_bar(stage);
+                    int ok = 1;
+                    if (lane == 0) {
+                        if (!ptx::mbar_wait_bounded(empty_bar(stage), phase ^ 1u, kWaitLimit)) {
+                            raise_timeout(p, abort_flag);
+                            ok = 0;
+                        } else if (*abort_flag) {
+                            ok = 0;
+                        } else {
+                            ptx::mbar_expect_tx(bar, p.a_bytes + p.b_bytes);
+                        }
                     }
-                    if (*abort_flag) break;
+                    ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
+                    if (!ok) { dead = true; break; }
                     const uint32_t sa = tiles + stage * kStageBytes;
                     const uint32_t sb = sa + kABytes;
-                    const uint32_t bar = full_bar(stage);
-                    ptx::mbar_expect_tx(bar, p.a_bytes + p.b_bytes);
-                    if (p.mode == 0) {
-                        const int k0 = kb * kBK;
-                        if (p.a_mn_major) {
-                            for (int c = 0; c < kBM / 32; ++c)
-                                ptx::tma_load_2d(sa + c * 4096u, &tmap_a, bar, m0 + c * 32, k0);
-                        } else {
-                            ptx::tma_load_2d(sa, &tmap_a, bar, k0, m0);
-                        }
-                        if (p.b_mn_major) {
-                            for (int c = 0; c < kBN / 32; ++c)
-                                ptx::tma_load_2d(sb + c * 4096u, &tmap_b, bar, n0 + c * 32, k0);
-                        } else {
-                            ptx::tma_load_2d(sb, &tmap_b, bar, k0, n0);
-                        }
-                    } else if (p.mode == 1) {
-                        // A: one box of img_w pixels x 32 channels per image row of the tile, read at
-                        // the tap's offset (rows and columns outside the image read as zero: padding).
-                        const int tap = kb / p.cblocks, cb = kb % p.cblocks;
-                        const int dh = p.tap_sign * (tap / p.taps_s) + p.off_h;
-                        const int dw = p.tap_sign * (tap % p.taps_s) + p.off_w;
-                        for (int j = 0; j < p.rows_per_blk; ++j) {
-                            const int q = w.tile_m * p.rows_per_blk + j;
-                            ptx::tma_load_4d(sa + (uint32_t)(j * p.img_w) * 128u, &tmap_a, bar, cb * 32, dw,
-                                             q % p.img_rows + dh, q / p.img_rows);
-                        }
-                        if (p.b_mn_major) {  // data gradient: filters [C_out][tap][C_in], C_in is N
-                            for (int c = 0; c < kBN / 32; ++c)
-                                ptx::tma_load_3d(sb + c * 4096u, &tmap_b, bar, n0 + c * 32, tap, cb * 32);
-                        } else {             // forward: filters [C_out][tap * C_in], K contiguous
-                            ptx::tma_load_2d(sb, &tmap_b, bar, tap * p.ck + cb * 32, n0);
-                        }
-                    } else {
+                    {
                         // Filter gradient: K = pixels.  A = output gradient (C_out is M), B = activations
                         // read at the tap that the N column block belongs to (C_in within a tap is N).
-                        for (int j = 0; j < p.rows_per_blk; ++j) {
+                        const int per_row = kBM / 32 + kBN / 32;
+                        for (int i = lane; i < p.rows_per_blk * per_row; i += 32) {
+                            const int j = i / per_row, c = i % per_row;
                             const int q = kb * p.rows_per_blk + j;
                             const int oh = q % p.img_rows, img = q / p.img_rows;
                             const uint32_t row_off = (uint32_t)(j * p.img_w) * 128u;
-                            for (int c = 0; c < kBM / 32; ++c)
+                            if (c < kBM / 32) {
                                 ptx::tma_load_4d(sa + c * 4096u + row_off, &tmap_a, bar, m0 + c * 32, 0, oh, img);
-                            for (int c = 0; c < kBN / 32; ++c) {
-                                const int col = n0 + c * 32;
+                            } else {
+                                const int col = n0 + (c - kBM / 32) * 32;
                                 const int tap = col / p.ck, ci = col % p.ck;
-                                ptx::tma_load_4d(sb + c * 4096u + row_off, &tmap_b, bar, ci, tap % p.taps_s + p.off_w,
-                                                 oh + tap / p.taps_s + p.off_h, img);
+                                ptx::tma_load_4d(sb + (c - kBM / 32) * 4096u + row_off, &tmap_b, bar, ci,
+                                                 tap % p.taps_s + p.off_w, oh + tap / p.taps_s + p.off_h, img);
                             }
                         }
                     }
                     if (++stage == kStages) { stage = 0; phase ^= 1u; }
                 }
             }
+        }
         }
         __syncwarp();
     } else if (warp == 1) {
@@ -533,8 +585,8 @@ splitk_reduce_kernel(const float* __restrict__ part, float* __restrict__ C, long
 constexpr size_t kWorkspaceHeader = 256;  // status word and padding ahead of the partial sums
 constexpr int kMaxSplits = 32;
 
-int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc, const GemmParams& p,
-                const DeviceInfo& dev, cudaStream_t stream) {
+int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc, const RowMaps& rows,
+                const GemmParams& p, const DeviceInfo& dev, cudaStream_t stream) {
     static bool attr_set[64] = {};
     if (dev.ordinal < 0 || dev.ordinal >= 64 || !attr_set[dev.ordinal]) {
         QFMT_CUDA_TRY(cudaFuncSetAttribute(gemm_tf32_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes));
@@ -542,7 +594,7 @@ int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap&
     }
     const long long work = (long long)p.tiles_m * p.tiles_n * p.splits;
     const int grid = work < dev.sm_count ? (int)work : dev.sm_count;
-    gemm_tf32_kernel<<<grid, kThreads, kSmemBytes, stream>>>(ma, mb, mc, p);
+    gemm_tf32_kernel<<<grid, kThreads, kSmemBytes, stream>>>(ma, mb, mc, rows, p);
     QFMT_CUDA_TRY(cudaGetLastError());
     return QFMT_OK;
 }
@@ -621,7 +673,9 @@ int gemm_device(const qfmt_matrix_t* A, const qfmt_matrix_t* B, float* d_C, int6
     if (p.tma_store) rc = make_map_c(&mc, d_C, (uint64_t)N, (uint64_t)M, 1, (uint64_t)ldc, (uint64_t)M * (uint64_t)ldc);
     else mc = ma;  // unused by the kernel
     if (rc != QFMT_OK) return rc;
-    return launch_gemm(ma, mb, mc, p, dev, stream);
+    RowMaps rows;
+    for (int i = 0; i < kMaxRowMaps; ++i) rows.m[i] = ma;  // unused in dense mode
+    return launch_gemm(ma, mb, mc, rows, p, dev, stream);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -730,12 +784,15 @@ int conv_device(int op, const qfmt_conv_t* g, const float* d_p, const float* d_q
         p.b_mn_major = fwd ? 0 : 1;
         p.a_bytes = (uint32_t)(p.tile_rows * 128);
         p.b_bytes = kBBytes;
-        {
+        RowMaps rmaps;
+        for (int cnt = 1; cnt <= kMaxRowMaps; ++cnt) {
             const uint64_t dims[4] = {src_c, src_w, src_h, N}, st[3] = {src_c, src_w * src_c, src_h * src_w * src_c};
-            const uint32_t box[4] = {32, (uint32_t)width, 1, 1};
-            rc = make_map(&ma, d_p, 4, dims, st, box, false);
+            const uint32_t rows_in_box = cnt <= p.rows_per_blk ? (uint32_t)cnt : 1u;  // larger counts are never used
+            const uint32_t box[4] = {32, (uint32_t)width, rows_in_box, 1};
+            rc = make_map(&rmaps.m[cnt - 1], d_p, 4, dims, st, box, false);
             if (rc != QFMT_OK) return rc;
         }
+        ma = rmaps.m[0];
         if (fwd) {  // filters [CO][TAPS*CI], K contiguous
             rc = make_map_2d(&mb, d_q, TAPS * CI, CO, TAPS * CI, kBK, kBN, false);
         } else {    // filters [CO][TAPS][CI]: N = CI contiguous, K = CO rows
@@ -749,7 +806,7 @@ int conv_device(int op, const qfmt_conv_t* g, const float* d_p, const float* d_q
                             (uint64_t)p.tile_rows * n_cols);
         else { mc = ma; p.tma_store = 0; }
         if (rc != QFMT_OK) return rc;
-        return launch_gemm(ma, mb, mc, p, dev, stream);
+        return launch_gemm(ma, mb, mc, rmaps, p, dev, stream);
     }
 
     // ---- filter gradient: dW [CO][TAPS*CI] = sum over pixels of dY^T (CO x pixels) * X_tap (pixels x CI)
@@ -791,7 +848,9 @@ int conv_device(int op, const qfmt_conv_t* g, const float* d_p, const float* d_q
     }
     rc = make_map_c(&mc, p.C, (uint64_t)p.N, (uint64_t)p.M, (uint64_t)p.splits, (uint64_t)p.N, (uint64_t)p.M * p.N);
     if (rc != QFMT_OK) return rc;
-    rc = launch_gemm(ma, mb, mc, p, dev, stream);
+    RowMaps rows;
+    for (int i = 0; i < kMaxRowMaps; ++i) rows.m[i] = ma;  // unused by the filter gradient
+    rc = launch_gemm(ma, mb, mc, rows, p, dev, stream);
     if (rc != QFMT_OK) return rc;
     if (p.splits > 1) {
         const long long total = (long long)p.M * p.N;

@@ -280,3 +280,43 @@ def test_config5_bert_large_fc_stack_step0(layer):
     e, m = c["fmt"]
     worst = fc_layer_parity(c["X"], c["W"], c["dY"], e, m, c["denormals"], c["grad_scale"], 65536, 50 + layer)
     print("config5", c["name"], worst)
+
+
+# ---------------------------------------------------------------------------------------------
+# bfloat16-family denormals are fp32 denormals: does the tensor pipe keep them?
+# ---------------------------------------------------------------------------------------------
+def test_fp32_denormal_operands_and_results_are_not_flushed():
+    """1/8/7 values m * 2^-133 (m < 128) are fp32 denormals.  Every case below has an exactly
+    representable result, so any flush-to-zero of operands, products or sums shows as a mismatch."""
+    K, M, N = 32, 128, 256
+    A = np.zeros((M, K), dtype=np.float32)
+    B = np.zeros((K, N), dtype=np.float32)
+    den = lambda mant: np.float32(mant) * np.float32(2.0 ** -133)   # 1/8/7 denormal
+    # rows 0..15: denormal operand times large normal -> normal product
+    for i in range(16):
+        A[i, 0] = den(2 * i + 1)
+    B[0, :] = np.float32(2.0 ** 100)
+    # rows 16..31: two normals whose product is an fp32 denormal
+    for i in range(16, 32):
+        A[i, 1] = np.float32(2.0 ** -70) * np.float32(1 + (i % 4) * 0.25)
+    B[1, :] = np.float32(2.0 ** -72)
+    # rows 32..47: a sum of denormal products (denormal operand x 1, 2, 4) stays denormal
+    for i in range(32, 48):
+        A[i, 2], A[i, 3], A[i, 4] = den(i), den(3), -den(1)
+    B[2, :], B[3, :], B[4, :] = 1.0, 2.0, 4.0
+    # rows 48..63: denormal operand on the B side
+    for i in range(48, 64):
+        A[i, 5] = np.float32(2.0 ** 90) * np.float32(i - 40)
+    B[5, :] = den(5)
+    # the oracle agrees these are values of 1/8/7 (denormals kept)
+    for X in (A, B):
+        q, _ = oracle.quantize_stats(X, 8, 7, 1, 1.0, want_stats=False)
+        assert np.array_equal(q.view(np.uint32), X.view(np.uint32))
+    ref, _ = oracle.gemm(A, B)
+    assert np.array_equal(ref.astype(np.float32).astype(np.float64), ref)  # exactly representable
+    assert np.count_nonzero(ref[:64]) == 64 * N
+    for transA, transB in ((False, False), (True, True)):
+        As = np.ascontiguousarray(A.T) if transA else A
+        Bs = np.ascontiguousarray(B.T) if transB else B
+        C = gpu_gemm(As, Bs, transA, transB, fmt=(8, 7))
+        assert np.array_equal(C.astype(np.float64), ref), (transA, transB)
