@@ -156,8 +156,7 @@ def time_events(torch, fn, iters):
 def gemm_section(torch, qf, dev, peaks, reps=5):
     """One step of the BERT-large FC stack: 12 GEMMs on operands quantized to 1/6/9 on the GPU."""
     fmt = qf.make_format(6, 9, 1)
-    ws = torch.zeros(1 << 20, dtype=torch.uint8, device=dev)
-    jobs, flops = [], 0.0
+    jobs, flops, ws_bytes = [], 0.0, 256
     for layer in range(len(workloads.CONFIG5_LAYERS)):
         c = workloads.config5_layer(layer, step=0)
         t = {}
@@ -172,7 +171,10 @@ def gemm_section(torch, qf, dev, peaks, reps=5):
                                       (t["X"], True, t["dY"], False, d_in, d_out, tokens)):
             C = torch.empty(M, N, dtype=torch.float32, device=dev)
             jobs.append((qf.make_matrix(A, ta), qf.make_matrix(B, tb), C, N, (A, B)))
+            ws_bytes = max(ws_bytes, qf.qfmt_gemm_workspace_bytes(jobs[-1][0], jobs[-1][1]))
             flops += 2.0 * M * N * K
+
+    ws = torch.zeros(ws_bytes, dtype=torch.uint8, device=dev)  # the recommended size (split-K partials)
 
     def step():
         for a, b, C, N, _ in jobs:
@@ -202,6 +204,52 @@ def gemm_section(torch, qf, dev, peaks, reps=5):
                          "peak_source": f"bf16 {peaks['source']} burst x 1.1/2.25 (nominal TF32:bf16 ratio)",
                          "library_tf32_same_run": lib_tf32, "frac_of_library_tf32": achieved / lib_tf32,
                          "nominal_tf32_dense": 1100.0, "frac_of_nominal": achieved / 1100.0}}
+
+
+def conv_section(torch, qf, dev, peaks, reps=5):
+    """The two ResNet-50-shaped layers of config4 (batch 128, 14x14): NCHW tensors are rounded to
+    1/6/9 into channels-last by the transposing pass, then fwd, dgrad and wgrad run as implicit GEMMs."""
+    out = {"metric": "emulated conv TFLOP/s", "unit": "TFLOP/s", "layers": {}}
+    total_flops, total_ms, launches = 0.0, 0.0, 0
+    for tag, sh in (("3x3", workloads.CONV3X3), ("1x1", workloads.CONV1X1)):
+        cfg = workloads.config4(sh)
+        n, ci, h, w, co, r, s_, pad = sh.n, sh.c_in, sh.h, sh.w, sh.c_out, sh.r, sh.s, sh.pad
+        g = qf.qfmt_conv_t(n, ci, h, w, co, r, s_, pad, pad)
+        fmt = qf.make_format(6, 9, 1)
+
+        def cl(x, scale=1.0):
+            b, c, hh, ww = x.shape
+            d_in = torch.from_numpy(x).to(dev)
+            d_out = torch.empty(b * hh * ww * c, dtype=torch.float32, device=dev)
+            qf.qfmt_quantize_stats_transpose(d_in, d_out, b, c, hh * ww, qf.make_format(6, 9, 1, scale))
+            return d_out
+        X, Wt, dY = cl(cfg["X"]), cl(cfg["W"]), cl(cfg["dY"], cfg["grad_scale"])
+        jobs = []
+        for op, P, Q, numel in ((qf.QFMT_CONV_FWD, X, Wt, n * h * w * co), (qf.QFMT_CONV_DGRAD, dY, Wt, n * h * w * ci),
+                                (qf.QFMT_CONV_WGRAD, dY, X, co * r * s_ * ci)):
+            wb = qf.qfmt_conv_workspace_bytes(op, g)
+            jobs.append((op, P, Q, torch.empty(numel, dtype=torch.float32, device=dev),
+                         torch.zeros(wb, dtype=torch.uint8, device=dev), wb))
+
+        def step():
+            for op, P, Q, O, ws, wb in jobs:
+                qf.qfmt_conv(op, g, P, Q, O, fmt, ws, wb)
+        for _ in range(3):
+            step()
+        for j in jobs:
+            assert qf.qfmt_device_status(j[4]) == qf.QFMT_OK
+        ms = statistics.median(time_events(torch, step, reps))
+        flops = 3 * 2.0 * n * h * w * co * ci * r * s_
+        out["layers"][tag] = {"ms_per_step": ms, "tflops": flops / ms / 1e9}
+        total_flops += flops
+        total_ms += ms
+        launches += 4  # three products + the split-K reduction of the filter gradient
+    peak = peaks["bf16_tflops"] * (1.1 / 2.25)
+    out.update({"value": total_flops / total_ms / 1e9, "ms_per_step": total_ms, "gpu_launches_per_step": launches,
+                "workload": "config4: 3x3 (256->256) and 1x1 (1024->256) layers, fwd+dgrad+wgrad, 1/6/9, channels-last",
+                "roofline": {"bound": "tensor", "achieved": total_flops / total_ms / 1e9, "peak": peak, "unit": "TFLOP/s",
+                             "frac": total_flops / total_ms / 1e9 / peak, "traffic": None}})
+    return out
 
 
 def run_library(args):
@@ -286,11 +334,13 @@ def run_library(args):
                 "mean_launch_us": 1e3 * mean_launch_ms, "nominal_hbm_gbs": 7700.0, "frac_of_nominal": achieved / 7700.0}
 
     sections = set(args.sections.split(","))
-    e2e = gemm = cpu = None
+    e2e = gemm = cpu = conv = None
     if "e2e" in sections:
         e2e = e2e_section(torch, qf, dev, x_host, fmts, n, step_bytes, args)
     if "gemm" in sections:
         gemm = gemm_section(torch, qf, dev, peaks)
+    if "conv" in sections:
+        conv = conv_section(torch, qf, dev, peaks)
     if "cpu" in sections:
         # the CPU oracle on this machine's host cores, bounded sample
         n_cpu = 1 << 24
@@ -299,7 +349,7 @@ def run_library(args):
         cpu = {"value": cpu_value, "unit": UNIT, "cores": 1, "kind": "oracle", "seconds": cpu_secs,
                "host_cores_available": os.cpu_count(),
                "sample": f"the 18 sweep runs on the first {n_cpu} of {n} elements"}
-    return finish(args, world, value, total_ms, n, runs, clocks, e2e, roofline, cpu, gemm, dist)
+    return finish(args, world, value, total_ms, n, runs, clocks, e2e, roofline, cpu, gemm, conv, dist)
 
 
 def e2e_section(torch, qf, dev, x_host, fmts, n, step_bytes, args):
@@ -321,7 +371,7 @@ def e2e_section(torch, qf, dev, x_host, fmts, n, step_bytes, args):
     return e2e
 
 
-def finish(args, world, value, total_ms, n, runs, clocks, e2e, roofline, cpu, gemm, dist):
+def finish(args, world, value, total_ms, n, runs, clocks, e2e, roofline, cpu, gemm, conv, dist):
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "u32", "data": "synthetic",
@@ -329,7 +379,7 @@ def finish(args, world, value, total_ms, n, runs, clocks, e2e, roofline, cpu, ge
                        "elements": n, "runs_per_step": len(runs), "l2": "inputs larger than L2 (256 MiB in, 256 MiB out)",
                        "multi_gpu": "replicas only: every rank runs the whole sweep on its own copy"},
             "clocks": clocks.summary(), "e2e": e2e, "gpu_launches": args.steps * len(runs),
-            "roofline": roofline, "cpu_baseline": cpu, "gemm": gemm}
+            "roofline": roofline, "cpu_baseline": cpu, "gemm": gemm, "conv": conv}
     print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
@@ -346,9 +396,9 @@ def main():
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="library", choices=["library", "reference"])
-    ap.add_argument("--sections", default="quantize,e2e,gemm,cpu",
+    ap.add_argument("--sections", default="quantize,e2e,gemm,conv,cpu",
                     help="comma list of what to measure besides the timed sweep (quantize is always timed): "
-                         "e2e, gemm, cpu; profiling captures use a subset")
+                         "e2e, gemm, conv, cpu; profiling captures use a subset")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

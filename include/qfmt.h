@@ -147,9 +147,13 @@ typedef struct {
  * fp32 denormal operands (only 1/8/m formats have them) are handled as the tensor core
  * handles them.
  *
- *   d_workspace  device, 16-byte aligned, >= qfmt_gemm_workspace_bytes(A, B) bytes.  Holds a
- *                status word (first 4 bytes, cleared by the call) and split-K partial sums.
- *                Calls that share a workspace must be ordered on one stream.
+ *   d_workspace  device, 16-byte aligned, at least 16 bytes; qfmt_gemm_workspace_bytes(A, B) is
+ *                the size that lets the library run at full speed.  Holds a status word (first
+ *                4 bytes, cleared by the call) and, for products with few output tiles and a
+ *                long K, split-K partial sums (K is shared among CTAs and the parts are added
+ *                in a fixed pairwise order).  A smaller workspace gets fewer or no splits: still
+ *                correct and reproducible, but the last bits can differ from a run with the
+ *                recommended size.  Calls that share a workspace must be ordered on one stream.
  * M = 0 or N = 0 is a no-op; K = 0 writes zeros.  Every device-side wait is bounded: if one
  * expires the kernel stops, the status word holds QFMT_ERR_TIMEOUT and C is undefined.
  * Errors: QFMT_ERR_BAD_FORMAT, QFMT_ERR_BAD_ARG (NULL or misaligned operand, ld too small,

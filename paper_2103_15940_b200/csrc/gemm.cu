@@ -615,6 +615,20 @@ void dense_defaults(GemmParams* p) {
 
 }  // namespace
 
+// Split-K factor for a dense product: used when the output has too few tiles to occupy the GPU and
+// K is long enough to share.  Planned for kPlanSms SMs so that it depends on the problem only.
+int plan_dense_splits(int64_t M, int64_t N, int64_t K) {
+    const int64_t tiles = ((M + kBM - 1) / kBM) * ((N + kBN - 1) / kBN);
+    const int64_t kb_total = (K + kBK - 1) / kBK;
+    if (tiles * 5 >= 148 * 3) return 1;  // at least 60 % of the SMs have a tile already
+    int64_t splits = 148 / tiles;
+    if (splits > kMaxSplits) splits = kMaxSplits;
+    if (splits > kb_total / 16) splits = kb_total / 16;  // at least 512 K elements per split
+    if (splits < 1) splits = 1;
+    const int64_t per = (kb_total + splits - 1) / splits;
+    return (int)((kb_total + per - 1) / per);
+}
+
 int gemm_device(const qfmt_matrix_t* A, const qfmt_matrix_t* B, float* d_C, int64_t ldc, const qfmt_format_t* fmt,
                 void* d_workspace, size_t workspace_bytes, cudaStream_t stream) {
     int rc = validate_format(fmt);
@@ -663,6 +677,20 @@ int gemm_device(const qfmt_matrix_t* A, const qfmt_matrix_t* B, float* d_C, int6
     // TMA stores clip at 16-byte granularity along the row, so N must be a multiple of 4 as well.
     p.tma_store = ((reinterpret_cast<uintptr_t>(d_C) & 15u) == 0 && (ldc & 3) == 0 && (N & 3) == 0) ? 1 : 0;
 
+    // Split K when the workspace the caller lent has room for the partial sums (the recommended size
+    // from qfmt_gemm_workspace_bytes always has); a smaller workspace gets fewer splits.
+    int splits = plan_dense_splits(M, N, K);
+    while (splits > 1 && kWorkspaceHeader + (size_t)splits * (size_t)M * (size_t)N * sizeof(float) > workspace_bytes) --splits;
+    float* partials = reinterpret_cast<float*>(reinterpret_cast<char*>(d_workspace) + kWorkspaceHeader);
+    if (splits > 1) {
+        p.kb_per_split = (p.kb_total + splits - 1) / splits;
+        p.splits = (p.kb_total + p.kb_per_split - 1) / p.kb_per_split;
+        p.split_stride = (long long)M * N;
+        p.C = partials;
+        p.ldc = N;
+        p.tma_store = (N & 3) == 0 ? 1 : 0;
+    }
+
     CUtensorMap ma, mb, mc;
     if (p.a_mn_major) rc = make_map_2d(&ma, A->ptr, (uint64_t)M, (uint64_t)K, (uint64_t)A->ld, 32, kBK, true);
     else rc = make_map_2d(&ma, A->ptr, (uint64_t)K, (uint64_t)M, (uint64_t)A->ld, kBK, kBM, false);
@@ -670,12 +698,21 @@ int gemm_device(const qfmt_matrix_t* A, const qfmt_matrix_t* B, float* d_C, int6
     if (p.b_mn_major) rc = make_map_2d(&mb, B->ptr, (uint64_t)N, (uint64_t)K, (uint64_t)B->ld, 32, kBK, true);
     else rc = make_map_2d(&mb, B->ptr, (uint64_t)K, (uint64_t)N, (uint64_t)B->ld, kBK, kBN, false);
     if (rc != QFMT_OK) return rc;
-    if (p.tma_store) rc = make_map_c(&mc, d_C, (uint64_t)N, (uint64_t)M, 1, (uint64_t)ldc, (uint64_t)M * (uint64_t)ldc);
+    if (p.tma_store)
+        rc = make_map_c(&mc, p.C, (uint64_t)N, (uint64_t)M, (uint64_t)p.splits, (uint64_t)p.ldc, (uint64_t)M * (uint64_t)p.ldc);
     else mc = ma;  // unused by the kernel
     if (rc != QFMT_OK) return rc;
     RowMaps rows;
     for (int i = 0; i < kMaxRowMaps; ++i) rows.m[i] = ma;  // unused in dense mode
-    return launch_gemm(ma, mb, mc, rows, p, dev, stream);
+    rc = launch_gemm(ma, mb, mc, rows, p, dev, stream);
+    if (rc != QFMT_OK) return rc;
+    if (p.splits > 1) {
+        const long long total = (long long)M * N;
+        const long long want = (total + 255) / 256, cap = (long long)dev.sm_count * 8;
+        splitk_reduce_kernel<<<(int)(want < cap ? want : cap), 256, 0, stream>>>(partials, d_C, M, N, ldc, p.splits);
+        QFMT_CUDA_TRY(cudaGetLastError());
+    }
+    return QFMT_OK;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -880,8 +917,13 @@ extern "C" size_t qfmt_conv_workspace_bytes(int32_t op, const qfmt_conv_t* geom)
 }
 
 extern "C" size_t qfmt_gemm_workspace_bytes(const qfmt_matrix_t* A, const qfmt_matrix_t* B) {
-    (void)A; (void)B;
-    return 256;
+    if (A == nullptr || B == nullptr || A->rows < 0 || A->cols < 0 || B->rows < 0 || B->cols < 0)
+        return qfmt::kWorkspaceHeader;
+    const int64_t M = A->trans ? A->cols : A->rows, K = A->trans ? A->rows : A->cols;
+    const int64_t N = B->trans ? B->rows : B->cols;
+    if (M <= 0 || N <= 0 || K <= 0 || M > (1 << 30) || N > (1 << 30) || K > (1 << 30)) return qfmt::kWorkspaceHeader;
+    const int splits = qfmt::plan_dense_splits(M, N, K);
+    return qfmt::kWorkspaceHeader + (splits > 1 ? (size_t)splits * (size_t)M * (size_t)N * sizeof(float) : 0);
 }
 
 extern "C" int qfmt_device_status(void* d_workspace, void* stream) {

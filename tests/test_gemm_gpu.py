@@ -249,7 +249,6 @@ def fc_layer_parity(X, W, dY, e, m, den, grad_scale, samples, seed):
     qG, _ = oracle.quantize_stats(dY, e, m, den, grad_scale, want_stats=False)
     assert np.array_equal(dG_.cpu().numpy().view(np.uint32), qG.view(np.uint32))
     fmt = qf.make_format(e, m, den)
-    ws = torch.zeros(1 << 20, dtype=torch.uint8, device=DEV)
     worst = {}
     for name, (ta, A_d, A_h), (tb, B_d, B_h) in (
             ("fwd", (False, dX_, qX), (False, dW_, qW)),
@@ -259,7 +258,7 @@ def fc_layer_parity(X, W, dY, e, m, den, grad_scale, samples, seed):
         N = B_h.shape[0] if tb else B_h.shape[1]
         C = torch.empty(M, N, dtype=torch.float32, device=DEV)
         a, b = qf.make_matrix(A_d, ta), qf.make_matrix(B_d, tb)
-        assert qf.qfmt_gemm_workspace_bytes(a, b) <= ws.numel()
+        ws = torch.zeros(qf.qfmt_gemm_workspace_bytes(a, b), dtype=torch.uint8, device=DEV)  # as bench.py does
         qf.qfmt_gemm(a, b, C, N, fmt, ws, ws.numel())
         assert qf.qfmt_device_status(ws) == qf.QFMT_OK
         worst[name] = check(C.cpu().numpy(), A_h, B_h, ta, tb, sample=samples, seed=seed)
@@ -320,3 +319,34 @@ def test_fp32_denormal_operands_and_results_are_not_flushed():
         Bs = np.ascontiguousarray(B.T) if transB else B
         C = gpu_gemm(As, Bs, transA, transB, fmt=(8, 7))
         assert np.array_equal(C.astype(np.float64), ref), (transA, transB)
+
+
+@pytest.mark.parametrize("transA,transB", [(False, False), (True, False), (False, True)])
+def test_split_k_few_tiles_long_k(transA, transB):
+    """One or two output tiles and K = 4096: K is split over CTAs and the parts are added in a fixed
+    tree.  Integer operands make every order exact; the result must not depend on how much
+    workspace (hence how many splits) the caller lends, and must repeat bit for bit."""
+    rng = np.random.default_rng(5)
+    M, N, K = 200, 260, 4096
+    A = stored((M, K), transA, lambda s: rng.integers(-2, 3, size=s).astype(np.float32))
+    B = stored((K, N), transB, lambda s: rng.integers(-2, 3, size=s).astype(np.float32))
+    dA, dB = torch.from_numpy(A).to(DEV), torch.from_numpy(B).to(DEV)
+    a, b = qf.make_matrix(dA, transA), qf.make_matrix(dB, transB)
+    full = qf.qfmt_gemm_workspace_bytes(a, b)
+    assert full > 256 + 2 * M * N * 4  # several splits are planned
+    ref, _ = oracle.gemm(A, B, transA, transB)
+    for wb in (full, 256 + 2 * M * N * 4, 256):
+        ws = torch.zeros(wb, dtype=torch.uint8, device=DEV)
+        dC = torch.full((M, N + 4), -777.0, dtype=torch.float32, device=DEV)
+        qf.qfmt_gemm(a, b, dC, N + 4, qf.make_format(6, 9), ws, wb)
+        assert qf.qfmt_device_status(ws) == qf.QFMT_OK
+        out = dC.cpu().numpy()
+        assert np.array_equal(out[:, :N].astype(np.float64), ref), wb
+        assert np.all(out[:, N:] == -777.0)
+    # real-valued data: within the bound and identical on a second run
+    Aq = stored((M, K), transA, lambda s: quantized(workloads.rng_for(66), s, 6, 9, -6.0, 4.0))
+    Bq = stored((K, N), transB, lambda s: quantized(workloads.rng_for(67), s, 6, 9, -6.0, 4.0))
+    C1 = gpu_gemm(Aq, Bq, transA, transB)
+    check(C1, Aq, Bq, transA, transB)
+    C2 = gpu_gemm(Aq, Bq, transA, transB)
+    assert np.array_equal(C1.view(np.uint32), C2.view(np.uint32))
