@@ -164,6 +164,17 @@ int qfmt_gemm(const qfmt_matrix_t* A, const qfmt_matrix_t* B, float* d_C, int64_
 size_t qfmt_gemm_workspace_bytes(const qfmt_matrix_t* A, const qfmt_matrix_t* B);
 
 /*
+ * Tuning and test control (no counterpart in the paper): which kernel dense products run on.
+ *   0  automatic (default)
+ *   1  single-CTA 128 x 256 tiles
+ *   2  CTA-pair 256 x 256 tiles (tcgen05 cta_group::2; each SM stages half of the B operand)
+ * Process-wide and not synchronised with calls in flight; results stay within the same bound under
+ * every policy but their last bits may differ between policies.  Ask qfmt_gemm_workspace_bytes
+ * again after changing it.  Returns QFMT_ERR_BAD_ARG for other values.
+ */
+int qfmt_gemm_tile_policy(int policy);
+
+/*
  * Convolution layers (Section V: "matrix multiplications, at the core of fully connected and
  * convolution layers"): the three products of a unit-stride, zero-padded 2-D convolution,
  * computed as implicit GEMMs with the FMACS semantics of qfmt_gemm (exact products, fp32

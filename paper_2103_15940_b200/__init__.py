@@ -99,6 +99,8 @@ def _bind_optional(L: ctypes.CDLL) -> None:
     L.qfmt_gemm.restype = ci
     L.qfmt_gemm_workspace_bytes.argtypes = [matp, matp]
     L.qfmt_gemm_workspace_bytes.restype = sz
+    L.qfmt_gemm_tile_policy.argtypes = [ci]
+    L.qfmt_gemm_tile_policy.restype = ci
     L.qfmt_device_status.argtypes = [vp, vp]
     L.qfmt_device_status.restype = ci
     convp = ctypes.POINTER(qfmt_conv_t)
@@ -218,3 +220,8 @@ def qfmt_conv(op: int, geom: qfmt_conv_t, d_p, d_q, d_out, fmt: qfmt_format_t, d
     see qfmt_conv in include/qfmt.h."""
     _check(lib().qfmt_conv(int(op), ctypes.byref(geom), _ptr(d_p), _ptr(d_q), _ptr(d_out), ctypes.byref(fmt),
                            _ptr(d_workspace), int(workspace_bytes), _stream_handle(stream)), "qfmt_conv")
+
+
+def qfmt_gemm_tile_policy(policy: int) -> None:
+    """0 automatic, 1 single-CTA tiles, 2 CTA-pair tiles; see include/qfmt.h."""
+    _check(lib().qfmt_gemm_tile_policy(int(policy)), "qfmt_gemm_tile_policy")

@@ -130,15 +130,18 @@ __device__ __forceinline__ WorkItem decode_work(const GemmParams& p, int t) {
 //       bytes = 32 M/N elements]; leading offset = distance between blocks, stride offset =
 //       distance between groups of 4 K-rows (512 bytes).
 constexpr uint32_t kLayoutSw128 = 2, kLayoutSw128Base32 = 1;
-__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes,
-                                              uint32_t layout) {
-    uint64_t d = 0;
-    d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
-    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
-    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
-    d |= (uint64_t)1 << 46;  // descriptor version for sm_100
-    d |= (uint64_t)layout << 61;
-    return d;
+// Field positions: start address bits 0-13, leading offset bits 16-29, stride offset bits 32-45,
+// descriptor version (1 on sm_100) bits 46-47, layout bits 61-63.  The descriptor is kept as a
+// constant high word and a low word to which the tile's offset (in 16-byte units) is added, so
+// that the MMA thread spends one add per operand per MMA.
+__device__ __forceinline__ uint32_t desc_hi(uint32_t sbo_bytes, uint32_t layout) {
+    return ((sbo_bytes >> 4) & 0x3FFFu) | (1u << 14) | (layout << 29);
+}
+__device__ __forceinline__ uint32_t desc_lo(uint32_t saddr, uint32_t lbo_bytes) {
+    return ((saddr & 0x3FFFFu) >> 4) | (((lbo_bytes >> 4) & 0x3FFFu) << 16);
+}
+__device__ __forceinline__ uint64_t desc_join(uint32_t hi, uint32_t lo) {
+    return ((uint64_t)hi << 32) | lo;
 }
 
 __device__ __forceinline__ uint32_t make_idesc(int a_mn, int b_mn) {
@@ -227,7 +230,6 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                             raise_timeout(p, abort_flag);
                             break;
                         }
-                        if (*abort_flag) break;
                         const uint32_t sa = tiles + stage * kStageBytes;
                         const uint32_t sb = sa + kABytes;
                         const uint32_t bar = full_bar(stage);
@@ -330,13 +332,15 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
         // ------------------------------ MMA issuer ------------------------------
         if (lane == 0) {
             const uint32_t idesc = make_idesc(p.a_mn_major, p.b_mn_major);
-            // per-MMA advance of the descriptor start address, in bytes
-            const uint32_t a_step = p.a_mn_major ? 1024u : (uint32_t)kMmaK * 4u;
-            const uint32_t b_step = p.b_mn_major ? 1024u : (uint32_t)kMmaK * 4u;
+            // per-MMA advance of the descriptor start address, in 16-byte units
+            const uint32_t a_step16 = (p.a_mn_major ? 1024u : (uint32_t)kMmaK * 4u) >> 4;
+            const uint32_t b_step16 = (p.b_mn_major ? 1024u : (uint32_t)kMmaK * 4u) >> 4;
             const uint32_t a_lbo = p.a_mn_major ? 4096u : 16u, a_sbo = p.a_mn_major ? 512u : 1024u;
             const uint32_t b_lbo = p.b_mn_major ? 4096u : 16u, b_sbo = p.b_mn_major ? 512u : 1024u;
             const uint32_t a_lay = p.a_mn_major ? kLayoutSw128Base32 : kLayoutSw128;
             const uint32_t b_lay = p.b_mn_major ? kLayoutSw128Base32 : kLayoutSw128;
+            const uint32_t a_hi = desc_hi(a_sbo, a_lay), b_hi = desc_hi(b_sbo, b_lay);
+            const uint32_t a_lo0 = desc_lo(tiles, a_lbo), b_lo0 = desc_lo(tiles + kABytes, b_lbo);
             int stage = 0;
             uint32_t phase = 0;
             uint32_t acc_iter = 0;  // chunks issued so far: buffer = acc_iter & 1, phase = (acc_iter >> 1) & 1
@@ -359,16 +363,12 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                             dead = true;
                             break;
                         }
-                        if (*abort_flag) { dead = true; break; }
                         ptx::tc_fence_after_sync();
-                        const uint32_t sa = tiles + stage * kStageBytes;
-                        const uint32_t sb = sa + kABytes;
+                        const uint32_t off = (uint32_t)stage * (kStageBytes >> 4);
 #pragma unroll
-                        for (int k = 0; k < kBK / kMmaK; ++k) {
-                            const uint64_t da = make_desc(sa + k * a_step, a_lbo, a_sbo, a_lay);
-                            const uint64_t db = make_desc(sb + k * b_step, b_lbo, b_sbo, b_lay);
-                            ptx::mma_tf32(d_tmem, da, db, idesc, (kb != kb0 || k != 0) ? 1u : 0u);
-                        }
+                        for (int k = 0; k < kBK / kMmaK; ++k)
+                            ptx::mma_tf32(d_tmem, desc_join(a_hi, a_lo0 + off + k * a_step16), desc_join(b_hi, b_lo0 + off + k * b_step16),
+                                          idesc, (kb != kb0 || k != 0) ? 1u : 0u);
                         ptx::mma_commit(empty_bar(stage));  // stage reusable once these MMAs have read it
                         if (++stage == kStages) { stage = 0; phase ^= 1u; }
                     }
@@ -512,6 +512,289 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     }
 }
 
+// ------------------------------------------------------------------------------------------------
+// CTA-pair variant (dense products): two CTAs of a cluster share one 256 x 256 tile.
+//
+// Each CTA stages its own 128 rows of op(A) and its own 128 columns of op(B) (32 KB per stage
+// instead of 48), the leader CTA's MMA thread issues tcgen05.mma.cta_group::2 with M = 256, and
+// each CTA's tensor memory receives its 128 x 256 half of the accumulator.  Per MMA a CTA feeds
+// 8 KB of operands from shared memory instead of 12 KB, which is what limits the single-CTA
+// kernel.  Nothing is copied between the CTAs; they only signal each other's barriers:
+//   full[s]      (leader's) two arrivals, one per CTA's producer with that CTA's byte count;
+//                both CTAs' TMA loads credit their bytes to it
+//   empty[s]     (each CTA's own) one arrival from the MMA commit, sent to both CTAs
+//   acc_full[b]  (each CTA's own) one arrival from the MMA commit, sent to both CTAs
+//   acc_empty[b] (leader's) sixteen arrivals: the eight accumulate warps of both CTAs
+// The three-level summation and the output path are those of the single-CTA kernel.
+// ------------------------------------------------------------------------------------------------
+constexpr int kPStages = 5;
+constexpr uint32_t kPABytes = kBM * kBK * 4;          // 128 rows of A
+constexpr uint32_t kPBBytes = (kBN / 2) * kBK * 4;    // 128 of the tile's 256 columns of B
+constexpr uint32_t kPStageBytes = kPABytes + kPBBytes;
+constexpr uint32_t kPairSmemBytes = kPStages * kPStageBytes + kOutBytes + 1024 + 256;
+
+__device__ __forceinline__ uint32_t make_idesc_pair(int a_mn, int b_mn) {
+    return (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)a_mn << 15) | ((uint32_t)b_mn << 16)
+           | ((uint32_t)(kBN >> 3) << 17) | ((uint32_t)((2 * kBM) >> 4) << 24);
+}
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+gemm_tf32_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+                      const __grid_constant__ CUtensorMap tmap_c, const GemmParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = ptx::smem_addr(smem_raw);
+    const uint32_t tiles = (raw + 1023u) & ~1023u;
+    const uint32_t out_stage = tiles + kPStages * kPStageBytes;
+    const uint32_t bars = out_stage + kOutBytes;
+    auto full_bar = [&](int s) { return bars + 8u * s; };
+    auto empty_bar = [&](int s) { return bars + 8u * (kPStages + s); };
+    auto acc_full_bar = [&](int a) { return bars + 8u * (2 * kPStages + a); };
+    auto acc_empty_bar = [&](int a) { return bars + 8u * (2 * kPStages + 2 + a); };
+    uint8_t* gen_bars = smem_raw + (bars - raw);
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen_bars + 8 * (2 * kPStages + 4));
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(gen_bars + 8 * (2 * kPStages + 4) + 8);
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const uint32_t rank = ptx::cluster_ctarank();  // 0 = leader
+    const int cluster_id = blockIdx.x >> 1, num_clusters = gridDim.x >> 1;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kPStages; ++s) {
+            ptx::mbar_init(full_bar(s), 2);
+            ptx::mbar_init(empty_bar(s), 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            ptx::mbar_init(acc_full_bar(a), 1);
+            ptx::mbar_init(acc_empty_bar(a), 2 * kAccWarps);
+        }
+        *abort_flag = 0;
+        ptx::fence_mbar_init();
+        ptx::prefetch_tensormap(&tmap_a);
+        ptx::prefetch_tensormap(&tmap_b);
+        if (p.tma_store) ptx::prefetch_tensormap(&tmap_c);
+    }
+    if (warp == 1) {
+        ptx::tmem_alloc_pair(ptx::smem_addr(const_cast<uint32_t*>(tmem_slot)), kTmemCols);
+        ptx::tmem_relinquish_pair();
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::cluster_sync();  // the peer's barriers exist before anything is signalled to them
+    ptx::tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+    const int num_work = p.tiles_m * p.tiles_n * p.splits;
+
+    if (warp < 4) {
+    ptx::setmaxnreg_dec<80>();
+    if (warp == 0) {
+        // ------------------------------ TMA producer (both CTAs) ------------------------------
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            for (int t = cluster_id; t < num_work && !*abort_flag; t += num_clusters) {
+                const WorkItem w = decode_work(p, t);
+                const int m0 = w.m0 + (int)rank * kBM, n0 = w.n0 + (int)rank * (kBN / 2);
+                for (int kb = w.kb_begin; kb < w.kb_begin + w.num_kb; ++kb) {
+                    if (!ptx::mbar_wait_bounded(empty_bar(stage), phase ^ 1u, kWaitLimit)) {
+                        raise_timeout(p, abort_flag);
+                        break;
+                    }
+                    const uint32_t sa = tiles + stage * kPStageBytes;
+                    const uint32_t sb = sa + kPABytes;
+                    const uint32_t bar = ptx::map_to_cta(full_bar(stage), 0);  // the leader's barrier
+                    const int k0 = kb * kBK;
+                    ptx::mbar_expect_tx_cluster(bar, kPStageBytes);
+                    if (p.a_mn_major) {
+                        for (int c = 0; c < kBM / 32; ++c)
+                            ptx::tma_load_2d_pair(sa + c * 4096u, &tmap_a, bar, m0 + c * 32, k0);
+                    } else {
+                        ptx::tma_load_2d_pair(sa, &tmap_a, bar, k0, m0);
+                    }
+                    if (p.b_mn_major) {
+                        for (int c = 0; c < kBN / 64; ++c)
+                            ptx::tma_load_2d_pair(sb + c * 4096u, &tmap_b, bar, n0 + c * 32, k0);
+                    } else {
+                        ptx::tma_load_2d_pair(sb, &tmap_b, bar, k0, n0);
+                    }
+                    if (++stage == kPStages) { stage = 0; phase ^= 1u; }
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        // ------------------------------ MMA issuer (leader CTA only) ------------------------------
+        if (lane == 0 && rank == 0) {
+            const uint32_t idesc = make_idesc_pair(p.a_mn_major, p.b_mn_major);
+            // per-MMA advance of the descriptor start address, in 16-byte units
+            const uint32_t a_step16 = (p.a_mn_major ? 1024u : (uint32_t)kMmaK * 4u) >> 4;
+            const uint32_t b_step16 = (p.b_mn_major ? 1024u : (uint32_t)kMmaK * 4u) >> 4;
+            const uint32_t a_lbo = p.a_mn_major ? 4096u : 16u, a_sbo = p.a_mn_major ? 512u : 1024u;
+            const uint32_t b_lbo = p.b_mn_major ? 4096u : 16u, b_sbo = p.b_mn_major ? 512u : 1024u;
+            const uint32_t a_lay = p.a_mn_major ? kLayoutSw128Base32 : kLayoutSw128;
+            const uint32_t b_lay = p.b_mn_major ? kLayoutSw128Base32 : kLayoutSw128;
+            const uint32_t a_hi = desc_hi(a_sbo, a_lay), b_hi = desc_hi(b_sbo, b_lay);
+            const uint32_t a_lo0 = desc_lo(tiles, a_lbo), b_lo0 = desc_lo(tiles + kPABytes, b_lbo);
+            int stage = 0;
+            uint32_t phase = 0;
+            uint32_t acc_iter = 0;
+            bool dead = false;
+            for (int t = cluster_id; t < num_work && !dead; t += num_clusters) {
+                const int num_kb = decode_work(p, t).num_kb;
+                for (int kb0 = 0; kb0 < num_kb && !dead; kb0 += kChunkKB) {
+                    const uint32_t acc = acc_iter & 1u, acc_phase = (acc_iter >> 1) & 1u;
+                    if (!ptx::mbar_wait_bounded(acc_empty_bar(acc), acc_phase ^ 1u, kWaitLimit)) {
+                        raise_timeout(p, abort_flag);
+                        dead = true;
+                        break;
+                    }
+                    ptx::tc_fence_after_sync();
+                    const uint32_t d_tmem = tmem_base + acc * kAccCols;
+                    const int kb1 = kb0 + kChunkKB < num_kb ? kb0 + kChunkKB : num_kb;
+                    for (int kb = kb0; kb < kb1; ++kb) {
+                        if (!ptx::mbar_wait_bounded(full_bar(stage), phase, kWaitLimit)) {
+                            raise_timeout(p, abort_flag);
+                            dead = true;
+                            break;
+                        }
+                        ptx::tc_fence_after_sync();
+                        const uint32_t off = (uint32_t)stage * (kPStageBytes >> 4);
+#pragma unroll
+                        for (int k = 0; k < kBK / kMmaK; ++k)
+                            ptx::mma_tf32_pair(d_tmem, desc_join(a_hi, a_lo0 + off + k * a_step16), desc_join(b_hi, b_lo0 + off + k * b_step16),
+                                          idesc, (kb != kb0 || k != 0) ? 1u : 0u);
+                        ptx::mma_commit_pair(empty_bar(stage), 3);  // both CTAs may refill this stage
+                        if (++stage == kPStages) { stage = 0; phase ^= 1u; }
+                    }
+                    if (dead) break;
+                    ptx::mma_commit_pair(acc_full_bar(acc), 3);      // chunk sum complete in both CTAs
+                    ++acc_iter;
+                }
+            }
+        }
+        __syncwarp();
+    }
+    } else {
+        ptx::setmaxnreg_inc<208>();
+        // ------------------------------ accumulate + epilogue (both CTAs) ------------------------------
+        const int quad = warp & 3;
+        const int half = (warp - 4) >> 2;
+        uint32_t acc_iter = 0;
+        bool dead = false;
+        for (int t = cluster_id; t < num_work && !dead; t += num_clusters) {
+            const WorkItem w = decode_work(p, t);
+            const int m0 = w.m0 + (int)rank * kBM, n0 = w.n0, num_kb = w.num_kb;
+            const int m_end = m0 + kBM < p.M ? m0 + kBM : p.M;
+            float* const c_base = p.C + (long long)w.split * p.split_stride;
+            const bool use_tma = p.tma_store != 0;
+            float sum[128];
+#pragma unroll
+            for (int j = 0; j < 128; ++j) sum[j] = 0.0f;
+            const uint32_t my_stage_addr = out_stage + (uint32_t)(warp - 4) * kOutWarpBytes;
+            float* my_stage = reinterpret_cast<float*>(smem_raw + (my_stage_addr - raw));
+            const int row0 = m0 + quad * 32;
+            int in_group = 0;
+            bool flushed = false;
+            for (int kb0 = 0; kb0 < num_kb; kb0 += kChunkKB) {
+                const uint32_t acc = acc_iter & 1u, acc_phase = (acc_iter >> 1) & 1u;
+                bool ok = true;
+                if (lane == 0) ok = ptx::mbar_wait_bounded(acc_full_bar(acc), acc_phase, kWaitLimit);
+                ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0;
+                if (!ok) {
+                    if (lane == 0) raise_timeout(p, abort_flag);
+                    dead = true;
+                    break;
+                }
+                if (*abort_flag) { dead = true; break; }
+                ptx::tc_fence_after_sync();
+                const uint32_t tbase = tmem_base + ((uint32_t)(quad * 32) << 16) + acc * kAccCols + (uint32_t)half * 128u;
+#pragma unroll
+                for (int pair = 0; pair < 2; ++pair) {
+                    uint32_t ra[32], rb[32];
+                    ptx::tmem_load_32cols(tbase + pair * 64, ra);
+                    ptx::tmem_load_32cols(tbase + pair * 64 + 32, rb);
+                    ptx::tmem_load_wait();
+                    if (pair == 1) {
+                        ptx::tc_fence_before_sync();
+                        __syncwarp();
+                        if (lane == 0) ptx::mbar_arrive_cluster(ptx::map_to_cta(acc_empty_bar(acc), 0));
+                    }
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        sum[pair * 64 + j] = __fadd_rn(sum[pair * 64 + j], __uint_as_float(ra[j]));
+                        sum[pair * 64 + 32 + j] = __fadd_rn(sum[pair * 64 + 32 + j], __uint_as_float(rb[j]));
+                    }
+                }
+                ++acc_iter;
+                const bool last = kb0 + kChunkKB >= num_kb;
+                if (!last && ++in_group < kFlushChunks) continue;
+                if (use_tma && flushed) {
+                    if (lane == 0) ptx::bulk_wait_all();
+                }
+#pragma unroll
+                for (int pass = 0; pass < 4; ++pass) {
+                    const int col0 = n0 + half * 128 + pass * kOutCols;
+                    float* box = my_stage + (pass & 1) * 1024;
+                    if (lane == 0) ptx::bulk_wait_read_1();
+                    __syncwarp();
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) {
+                        const int j = pass * kOutCols + c * 4;
+                        *reinterpret_cast<float4*>(box + lane * 32 + ((c ^ (lane & 7)) << 2)) =
+                            make_float4(sum[j], sum[j + 1], sum[j + 2], sum[j + 3]);
+                    }
+                    if (use_tma) {
+                        ptx::fence_proxy_async();
+                        __syncwarp();
+                        if (lane == 0) {
+                            if (row0 < m_end && col0 < p.N) {
+                                const uint32_t src = my_stage_addr + (pass & 1) * kOutBoxBytes;
+                                if (flushed) ptx::tma_reduce_add_3d(&tmap_c, src, col0, row0, w.split);
+                                else ptx::tma_store_3d(&tmap_c, src, col0, row0, w.split);
+                            }
+                            ptx::bulk_commit();
+                        }
+                    } else {
+                        __syncwarp();
+                        for (int r = 0; r < 32; ++r) {
+                            const int row = row0 + r;
+                            if (row >= m_end) break;
+                            const int c = lane;
+                            if (col0 + c < p.N) {
+                                float* g = c_base + (long long)row * p.ldc + col0 + c;
+                                const float v = box[r * 32 + (((c >> 2) ^ (r & 7)) << 2) + (c & 3)];
+                                *g = flushed ? __fadd_rn(*g, v) : v;
+                            }
+                        }
+                        __syncwarp();
+                    }
+                }
+                flushed = true;
+                in_group = 0;
+                if (!last) {
+#pragma unroll
+                    for (int j = 0; j < 128; ++j) sum[j] = 0.0f;
+                }
+            }
+            if (dead) break;
+        }
+        if (lane == 0) ptx::bulk_wait_all();
+        __syncwarp();
+    }
+
+    // ------------------------------ common exit ------------------------------
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    if (*abort_flag) {
+        for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+    }
+    ptx::cluster_sync();  // neither CTA leaves while the other may still signal it
+    if (warp == 1) {
+        ptx::tc_fence_after_sync();
+        ptx::tmem_dealloc_pair(tmem_base, kTmemCols);
+    }
+}
+
 // ---- host side ----------------------------------------------------------------------------------
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -615,18 +898,46 @@ void dense_defaults(GemmParams* p) {
 
 }  // namespace
 
+// Which kernel a dense product runs on: 0 automatic, 1 single-CTA tiles (128 x 256), 2 CTA-pair
+// tiles (256 x 256).  Process-wide; see qfmt_gemm_tile_policy.
+static std::atomic<int> g_tile_policy{0};
+
+bool dense_uses_pair(int64_t M, int64_t N, int64_t K) {
+    (void)N; (void)K;
+    const int policy = g_tile_policy.load();
+    if (policy == 1) return false;
+    if (policy == 2) return true;
+    return M > kBM;  // with a single row of tiles the second CTA of a pair would idle
+}
+
 // Split-K factor for a dense product: used when the output has too few tiles to occupy the GPU and
-// K is long enough to share.  Planned for kPlanSms SMs so that it depends on the problem only.
-int plan_dense_splits(int64_t M, int64_t N, int64_t K) {
-    const int64_t tiles = ((M + kBM - 1) / kBM) * ((N + kBN - 1) / kBN);
+// K is long enough to share.  Planned for a 148-SM part so that it depends on the problem only.
+int plan_dense_splits(int64_t M, int64_t N, int64_t K, bool pair) {
+    const int64_t tile_rows = pair ? 2 * kBM : kBM, units = pair ? 74 : 148;
+    const int64_t tiles = ((M + tile_rows - 1) / tile_rows) * ((N + kBN - 1) / kBN);
     const int64_t kb_total = (K + kBK - 1) / kBK;
-    if (tiles * 5 >= 148 * 3) return 1;  // at least 60 % of the SMs have a tile already
-    int64_t splits = 148 / tiles;
+    if (tiles * 5 >= units * 3) return 1;  // at least 60 % of the SMs have work already
+    int64_t splits = units / tiles;
     if (splits > kMaxSplits) splits = kMaxSplits;
     if (splits > kb_total / 16) splits = kb_total / 16;  // at least 512 K elements per split
     if (splits < 1) splits = 1;
     const int64_t per = (kb_total + splits - 1) / splits;
     return (int)((kb_total + per - 1) / per);
+}
+
+int launch_pair(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc, const GemmParams& p,
+                const DeviceInfo& dev, cudaStream_t stream) {
+    static bool attr_set[64] = {};
+    if (dev.ordinal < 0 || dev.ordinal >= 64 || !attr_set[dev.ordinal]) {
+        QFMT_CUDA_TRY(cudaFuncSetAttribute(gemm_tf32_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           (int)kPairSmemBytes));
+        if (dev.ordinal >= 0 && dev.ordinal < 64) attr_set[dev.ordinal] = true;
+    }
+    const long long work = (long long)p.tiles_m * p.tiles_n * p.splits;
+    const long long clusters = work < dev.sm_count / 2 ? work : dev.sm_count / 2;
+    gemm_tf32_pair_kernel<<<(unsigned)(2 * clusters), kThreads, kPairSmemBytes, stream>>>(ma, mb, mc, p);
+    QFMT_CUDA_TRY(cudaGetLastError());
+    return QFMT_OK;
 }
 
 int gemm_device(const qfmt_matrix_t* A, const qfmt_matrix_t* B, float* d_C, int64_t ldc, const qfmt_format_t* fmt,
@@ -670,7 +981,9 @@ int gemm_device(const qfmt_matrix_t* A, const qfmt_matrix_t* B, float* d_C, int6
     p.status = status;
     p.a_mn_major = A->trans ? 1 : 0;
     p.b_mn_major = B->trans ? 0 : 1;
-    p.tiles_m = (int)((M + kBM - 1) / kBM);
+    const bool pair = dense_uses_pair(M, N, K);
+    p.tile_rows = pair ? 2 * kBM : kBM;
+    p.tiles_m = (int)((M + p.tile_rows - 1) / p.tile_rows);
     p.tiles_n = (int)((N + kBN - 1) / kBN);
     p.kb_total = (int)((K + kBK - 1) / kBK);
     p.kb_per_split = p.kb_total;
@@ -679,7 +992,7 @@ int gemm_device(const qfmt_matrix_t* A, const qfmt_matrix_t* B, float* d_C, int6
 
     // Split K when the workspace the caller lent has room for the partial sums (the recommended size
     // from qfmt_gemm_workspace_bytes always has); a smaller workspace gets fewer splits.
-    int splits = plan_dense_splits(M, N, K);
+    int splits = plan_dense_splits(M, N, K, pair);
     while (splits > 1 && kWorkspaceHeader + (size_t)splits * (size_t)M * (size_t)N * sizeof(float) > workspace_bytes) --splits;
     float* partials = reinterpret_cast<float*>(reinterpret_cast<char*>(d_workspace) + kWorkspaceHeader);
     if (splits > 1) {
@@ -696,15 +1009,19 @@ int gemm_device(const qfmt_matrix_t* A, const qfmt_matrix_t* B, float* d_C, int6
     else rc = make_map_2d(&ma, A->ptr, (uint64_t)K, (uint64_t)M, (uint64_t)A->ld, kBK, kBM, false);
     if (rc != QFMT_OK) return rc;
     if (p.b_mn_major) rc = make_map_2d(&mb, B->ptr, (uint64_t)N, (uint64_t)K, (uint64_t)B->ld, 32, kBK, true);
-    else rc = make_map_2d(&mb, B->ptr, (uint64_t)K, (uint64_t)N, (uint64_t)B->ld, kBK, kBN, false);
+    else rc = make_map_2d(&mb, B->ptr, (uint64_t)K, (uint64_t)N, (uint64_t)B->ld, kBK, pair ? kBN / 2 : kBN, false);
     if (rc != QFMT_OK) return rc;
     if (p.tma_store)
         rc = make_map_c(&mc, p.C, (uint64_t)N, (uint64_t)M, (uint64_t)p.splits, (uint64_t)p.ldc, (uint64_t)M * (uint64_t)p.ldc);
     else mc = ma;  // unused by the kernel
     if (rc != QFMT_OK) return rc;
-    RowMaps rows;
-    for (int i = 0; i < kMaxRowMaps; ++i) rows.m[i] = ma;  // unused in dense mode
-    rc = launch_gemm(ma, mb, mc, rows, p, dev, stream);
+    if (pair) {
+        rc = launch_pair(ma, mb, mc, p, dev, stream);
+    } else {
+        RowMaps rows;
+        for (int i = 0; i < kMaxRowMaps; ++i) rows.m[i] = ma;  // unused in dense mode
+        rc = launch_gemm(ma, mb, mc, rows, p, dev, stream);
+    }
     if (rc != QFMT_OK) return rc;
     if (p.splits > 1) {
         const long long total = (long long)M * N;
@@ -916,13 +1233,19 @@ extern "C" size_t qfmt_conv_workspace_bytes(int32_t op, const qfmt_conv_t* geom)
     return plan.workspace;
 }
 
+extern "C" int qfmt_gemm_tile_policy(int policy) {
+    if (policy < 0 || policy > 2) return QFMT_ERR_BAD_ARG;
+    qfmt::g_tile_policy.store(policy);
+    return QFMT_OK;
+}
+
 extern "C" size_t qfmt_gemm_workspace_bytes(const qfmt_matrix_t* A, const qfmt_matrix_t* B) {
     if (A == nullptr || B == nullptr || A->rows < 0 || A->cols < 0 || B->rows < 0 || B->cols < 0)
         return qfmt::kWorkspaceHeader;
     const int64_t M = A->trans ? A->cols : A->rows, K = A->trans ? A->rows : A->cols;
     const int64_t N = B->trans ? B->rows : B->cols;
     if (M <= 0 || N <= 0 || K <= 0 || M > (1 << 30) || N > (1 << 30) || K > (1 << 30)) return qfmt::kWorkspaceHeader;
-    const int splits = qfmt::plan_dense_splits(M, N, K);
+    const int splits = qfmt::plan_dense_splits(M, N, K, qfmt::dense_uses_pair(M, N, K));
     return qfmt::kWorkspaceHeader + (splits > 1 ? (size_t)splits * (size_t)M * (size_t)N * sizeof(float) : 0);
 }
 
