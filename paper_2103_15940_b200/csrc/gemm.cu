@@ -396,9 +396,11 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
             // In mode 1 the C tensor map is [complete tiles][tile_rows][N]; an incomplete last tile
             // takes the scalar path.
             const bool use_tma = p.tma_store && (p.mode != 1 || w.tile_m < p.full_tiles_m);
-            float sum[128];  // level-1 running sums; 0 + x is exact, so a group's first chunk needs no special case
+            // level-1 running sums, two per 64-bit register (packed adds); 0 + x is exact, so a group's
+            // first chunk needs no special case
+            unsigned long long sum2[64];
 #pragma unroll
-            for (int j = 0; j < 128; ++j) sum[j] = 0.0f;
+            for (int j = 0; j < 64; ++j) sum2[j] = 0ull;
             const uint32_t my_stage_addr = out_stage + (uint32_t)(warp - 4) * kOutWarpBytes;
             float* my_stage = reinterpret_cast<float*>(smem_raw + (my_stage_addr - raw));
             const int row0 = m0 + quad * 32;
@@ -431,9 +433,9 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                         if (lane == 0) ptx::mbar_arrive(acc_empty_bar(acc));
                     }
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        sum[pair * 64 + j] = __fadd_rn(sum[pair * 64 + j], __uint_as_float(ra[j]));
-                        sum[pair * 64 + 32 + j] = __fadd_rn(sum[pair * 64 + 32 + j], __uint_as_float(rb[j]));
+                    for (int j = 0; j < 32; j += 2) {
+                        ptx::add2_rn(sum2[pair * 32 + j / 2], ra[j], ra[j + 1]);
+                        ptx::add2_rn(sum2[pair * 32 + 16 + j / 2], rb[j], rb[j + 1]);
                     }
                 }
                 ++acc_iter;
@@ -454,8 +456,9 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
 #pragma unroll
                     for (int c = 0; c < 8; ++c) {
                         const int j = pass * kOutCols + c * 4;
+                        const float2 v0 = ptx::unpack2(sum2[j / 2]), v1 = ptx::unpack2(sum2[j / 2 + 1]);
                         *reinterpret_cast<float4*>(box + lane * 32 + ((c ^ (lane & 7)) << 2)) =
-                            make_float4(sum[j], sum[j + 1], sum[j + 2], sum[j + 3]);
+                            make_float4(v0.x, v0.y, v1.x, v1.y);
                     }
                     if (use_tma) {
                         ptx::fence_proxy_async();
@@ -489,7 +492,7 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                 in_group = 0;
                 if (!last) {
 #pragma unroll
-                    for (int j = 0; j < 128; ++j) sum[j] = 0.0f;
+                    for (int j = 0; j < 64; ++j) sum2[j] = 0ull;
                 }
             }
             if (dead) break;
@@ -687,9 +690,11 @@ gemm_tf32_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
             const int m_end = m0 + kBM < p.M ? m0 + kBM : p.M;
             float* const c_base = p.C + (long long)w.split * p.split_stride;
             const bool use_tma = p.tma_store != 0;
-            float sum[128];
+            // level-1 running sums, two per 64-bit register (packed adds); 0 + x is exact, so a group's
+            // first chunk needs no special case
+            unsigned long long sum2[64];
 #pragma unroll
-            for (int j = 0; j < 128; ++j) sum[j] = 0.0f;
+            for (int j = 0; j < 64; ++j) sum2[j] = 0ull;
             const uint32_t my_stage_addr = out_stage + (uint32_t)(warp - 4) * kOutWarpBytes;
             float* my_stage = reinterpret_cast<float*>(smem_raw + (my_stage_addr - raw));
             const int row0 = m0 + quad * 32;
@@ -720,9 +725,9 @@ gemm_tf32_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
                         if (lane == 0) ptx::mbar_arrive_cluster(ptx::map_to_cta(acc_empty_bar(acc), 0));
                     }
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        sum[pair * 64 + j] = __fadd_rn(sum[pair * 64 + j], __uint_as_float(ra[j]));
-                        sum[pair * 64 + 32 + j] = __fadd_rn(sum[pair * 64 + 32 + j], __uint_as_float(rb[j]));
+                    for (int j = 0; j < 32; j += 2) {
+                        ptx::add2_rn(sum2[pair * 32 + j / 2], ra[j], ra[j + 1]);
+                        ptx::add2_rn(sum2[pair * 32 + 16 + j / 2], rb[j], rb[j + 1]);
                     }
                 }
                 ++acc_iter;
@@ -740,8 +745,9 @@ gemm_tf32_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
 #pragma unroll
                     for (int c = 0; c < 8; ++c) {
                         const int j = pass * kOutCols + c * 4;
+                        const float2 v0 = ptx::unpack2(sum2[j / 2]), v1 = ptx::unpack2(sum2[j / 2 + 1]);
                         *reinterpret_cast<float4*>(box + lane * 32 + ((c ^ (lane & 7)) << 2)) =
-                            make_float4(sum[j], sum[j + 1], sum[j + 2], sum[j + 3]);
+                            make_float4(v0.x, v0.y, v1.x, v1.y);
                     }
                     if (use_tma) {
                         ptx::fence_proxy_async();
@@ -773,7 +779,7 @@ gemm_tf32_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
                 in_group = 0;
                 if (!last) {
 #pragma unroll
-                    for (int j = 0; j < 128; ++j) sum[j] = 0.0f;
+                    for (int j = 0; j < 64; ++j) sum2[j] = 0ull;
                 }
             }
             if (dead) break;

@@ -230,6 +230,15 @@ __device__ __forceinline__ void tmem_load_16cols(uint32_t taddr, uint32_t (&r)[1
         : "r"(taddr)
         : "memory");
 }
+// acc (two packed fp32) += {lo, hi}: one instruction for two round-to-nearest-even adds.
+__device__ __forceinline__ void add2_rn(unsigned long long& acc, uint32_t lo, uint32_t hi) {
+    asm("{\n\t.reg .b64 t;\n\tmov.b64 t, {%1, %2};\n\tadd.rn.f32x2 %0, %0, t;\n\t}" : "+l"(acc) : "r"(lo), "r"(hi));
+}
+__device__ __forceinline__ float2 unpack2(unsigned long long v) {
+    float2 r;
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(r.x), "=f"(r.y) : "l"(v));
+    return r;
+}
 __device__ __forceinline__ void tmem_load_wait() {
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
