@@ -519,10 +519,10 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
 // CTA-pair variant (dense products): two CTAs of a cluster share one 256 x 256 tile.
 //
 // Each CTA stages its own 128 rows of op(A) and its own 128 columns of op(B) (32 KB per stage
-// instead of 48), the leader CTA's MMA thread issues tcgen05.mma.cta_group::2 with M = 256, and
-// each CTA's tensor memory receives its 128 x 256 half of the accumulator.  Per MMA a CTA feeds
-// 8 KB of operands from shared memory instead of 12 KB, which is what limits the single-CTA
-// kernel.  Nothing is copied between the CTAs; they only signal each other's barriers:
+// instead of 48), the leader CTA's two MMA threads issue tcgen05.mma.cta_group::2 with M = 256,
+// and each CTA's tensor memory receives its 128 x 256 half of the accumulator.  Per MMA a CTA
+// feeds 8 KB of operands from shared memory instead of 12 KB.  Nothing is copied between the
+// CTAs; they only signal each other's barriers:
 //   full[s]      (leader's) two arrivals, one per CTA's producer with that CTA's byte count;
 //                both CTAs' TMA loads credit their bytes to it
 //   empty[s]     (each CTA's own) one arrival from the MMA commit, sent to both CTAs
@@ -625,9 +625,16 @@ gemm_tf32_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
             }
         }
         __syncwarp();
-    } else if (warp == 1) {
-        // ------------------------------ MMA issuer (leader CTA only) ------------------------------
+    } else if (warp == 1 || warp == 2) {
+        // ------------------------------ MMA issuers (leader CTA only) ------------------------------
+        // One thread can hand the tensor pipe an MMA every ~100-150 cycles, and every barrier wait
+        // costs it as much again, so a single issuer with three waits per chunk leaves the pipe idle
+        // a third of the time.  Two threads in different warps share the work: warp 1 issues the even
+        // chunks (accumulator 0), warp 2 the odd ones (accumulator 1).  A chunk's MMAs depend on no
+        // other chunk's, so the two streams need no ordering between them; each thread walks the
+        // whole stage ring and acts on its own chunks only.
         if (lane == 0 && rank == 0) {
+            const uint32_t who = (uint32_t)(warp - 1);
             const uint32_t idesc = make_idesc_pair(p.a_mn_major, p.b_mn_major);
             // per-MMA advance of the descriptor start address, in 16-byte units
             const uint32_t a_step16 = (p.a_mn_major ? 1024u : (uint32_t)kMmaK * 4u) >> 4;
@@ -644,8 +651,13 @@ gemm_tf32_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
             bool dead = false;
             for (int t = cluster_id; t < num_work && !dead; t += num_clusters) {
                 const int num_kb = decode_work(p, t).num_kb;
-                for (int kb0 = 0; kb0 < num_kb && !dead; kb0 += kChunkKB) {
+                for (int kb0 = 0; kb0 < num_kb && !dead; kb0 += kChunkKB, ++acc_iter) {
                     const uint32_t acc = acc_iter & 1u, acc_phase = (acc_iter >> 1) & 1u;
+                    if (acc != who) {  // the other issuer's chunk: step over its stages
+                        stage += kb0 + kChunkKB < num_kb ? kChunkKB : num_kb - kb0;
+                        if (stage >= kPStages) { stage -= kPStages; phase ^= 1u; }
+                        continue;
+                    }
                     if (!ptx::mbar_wait_bounded(acc_empty_bar(acc), acc_phase ^ 1u, kWaitLimit)) {
                         raise_timeout(p, abort_flag);
                         dead = true;
@@ -671,7 +683,6 @@ gemm_tf32_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
                     }
                     if (dead) break;
                     ptx::mma_commit_pair(acc_full_bar(acc), 3);      // chunk sum complete in both CTAs
-                    ++acc_iter;
                 }
             }
         }
