@@ -65,7 +65,7 @@ constexpr uint32_t kOutBoxBytes = 32 * 32 * 4;
 constexpr uint32_t kOutWarpBytes = 2 * kOutBoxBytes;
 constexpr uint32_t kOutBytes = kAccWarps * kOutWarpBytes;
 constexpr uint32_t kSmemBytes = kStages * kStageBytes + kOutBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
-constexpr uint32_t kWaitLimit = 1u << 22;  // polls (with backoff) before a wait is declared dead
+constexpr uint32_t kWaitLimit = 1u << 31;  // SM cycles (about a second) before a wait is declared dead
 
 struct GemmParams {
     int M, N, K;
@@ -174,6 +174,8 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     uint8_t* gen_bars = smem_raw + (bars - raw);
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen_bars + 8 * (2 * kStages + 4));
     volatile int* abort_flag = reinterpret_cast<volatile int*>(gen_bars + 8 * (2 * kStages + 4) + 8);
+    // issue_progress[i]: chunks (counted over the whole kernel) up to which MMA issuer i has seen its operands arrive
+    volatile uint32_t* issue_progress = reinterpret_cast<volatile uint32_t*>(gen_bars + 8 * (2 * kStages + 4) + 16);
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -195,6 +197,8 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
             ptx::mbar_init(acc_empty_bar(a), kAccWarps);  // one arrival per accumulate warp
         }
         *abort_flag = 0;
+        issue_progress[0] = 0;
+        issue_progress[1] = 0;
         ptx::fence_mbar_init();
         ptx::prefetch_tensormap(&tmap_a);
         ptx::prefetch_tensormap(&tmap_b);
@@ -328,9 +332,22 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
         }
         }
         __syncwarp();
-    } else if (warp == 1) {
-        // ------------------------------ MMA issuer ------------------------------
+    } else if (warp == 1 || warp == 2) {
+        // ------------------------------ MMA issuers ------------------------------
+        // One thread can hand the tensor pipe an MMA every ~100-150 cycles, and every barrier wait
+        // costs it as much again, so a single issuer with three waits per chunk leaves the pipe idle
+        // a third of the time.  Two threads in different warps share the work: warp 1 issues the even
+        // chunks (accumulator 0), warp 2 the odd ones (accumulator 1).  A chunk's MMAs depend on no
+        // other chunk's, so the two streams need no ordering between them; each thread walks the
+        // whole stage ring and acts on its own chunks only.
+        //
+        // A parity wait tells "phase k is over" from "phase k has not begun" only while the waiter is
+        // at most one phase ahead of the barrier.  With three stages and two-stage chunks, the
+        // second stage of chunk c+1 is the first stage of chunk c one phase on, so the issuer of
+        // chunk c+1 must not look at the stage barriers until the issuer of chunk c has seen that
+        // chunk's operands arrive: issue_progress carries that fact from one thread to the other.
         if (lane == 0) {
+            const uint32_t who = (uint32_t)(warp - 1);
             const uint32_t idesc = make_idesc(p.a_mn_major, p.b_mn_major);
             // per-MMA advance of the descriptor start address, in 16-byte units
             const uint32_t a_step16 = (p.a_mn_major ? 1024u : (uint32_t)kMmaK * 4u) >> 4;
@@ -347,14 +364,29 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
             bool dead = false;
             for (int t = blockIdx.x; t < num_work && !dead; t += gridDim.x) {
                 const int num_kb = decode_work(p, t).num_kb;
-                for (int kb0 = 0; kb0 < num_kb && !dead; kb0 += kChunkKB) {
+                for (int kb0 = 0; kb0 < num_kb && !dead; kb0 += kChunkKB, ++acc_iter) {
                     const uint32_t acc = acc_iter & 1u, acc_phase = (acc_iter >> 1) & 1u;
+                    if (acc != who) {  // the other issuer's chunk: step over its stages
+                        stage += kb0 + kChunkKB < num_kb ? kChunkKB : num_kb - kb0;
+                        if (stage >= kStages) { stage -= kStages; phase ^= 1u; }
+                        continue;
+                    }
                     if (!ptx::mbar_wait_bounded(acc_empty_bar(acc), acc_phase ^ 1u, kWaitLimit)) {
                         raise_timeout(p, abort_flag);
                         dead = true;
                         break;
                     }
                     ptx::tc_fence_after_sync();
+                    {   // wait (bounded) until the other issuer is past the stage waits of chunk acc_iter - 1
+                        const long long t_begin = clock64();
+                        while (issue_progress[who ^ 1u] < acc_iter) {
+                            if (clock64() - t_begin > (long long)kWaitLimit) { dead = true; break; }
+                        }
+                        if (dead) {
+                            raise_timeout(p, abort_flag);
+                            break;
+                        }
+                    }
                     const uint32_t d_tmem = tmem_base + acc * kAccCols;
                     const int kb1 = kb0 + kChunkKB < num_kb ? kb0 + kChunkKB : num_kb;
                     for (int kb = kb0; kb < kb1; ++kb) {
@@ -362,6 +394,10 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                             raise_timeout(p, abort_flag);
                             dead = true;
                             break;
+                        }
+                        if (kb + 1 == kb1) {  // all of this chunk's operands have arrived
+                            __threadfence_block();
+                            issue_progress[who] = acc_iter + 1u;
                         }
                         ptx::tc_fence_after_sync();
                         const uint32_t off = (uint32_t)stage * (kStageBytes >> 4);
@@ -374,7 +410,6 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                     }
                     if (dead) break;
                     ptx::mma_commit(acc_full_bar(acc));      // chunk sum complete
-                    ++acc_iter;
                 }
             }
         }
@@ -627,12 +662,10 @@ gemm_tf32_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
         __syncwarp();
     } else if (warp == 1 || warp == 2) {
         // ------------------------------ MMA issuers (leader CTA only) ------------------------------
-        // One thread can hand the tensor pipe an MMA every ~100-150 cycles, and every barrier wait
-        // costs it as much again, so a single issuer with three waits per chunk leaves the pipe idle
-        // a third of the time.  Two threads in different warps share the work: warp 1 issues the even
-        // chunks (accumulator 0), warp 2 the odd ones (accumulator 1).  A chunk's MMAs depend on no
-        // other chunk's, so the two streams need no ordering between them; each thread walks the
-        // whole stage ring and acts on its own chunks only.
+        // Two issuers on alternating chunks, as in the single-CTA kernel.  No progress word is needed
+        // here: an issuer reaches chunk c+1 only after the accumulate warps have drained chunk c-1,
+        // hence after chunk c-2 was issued in full, and with a ring of five stages the previous
+        // phase of the stages of chunk c+1 belongs to chunks c-2 and c-1.
         if (lane == 0 && rank == 0) {
             const uint32_t who = (uint32_t)(warp - 1);
             const uint32_t idesc = make_idesc_pair(p.a_mn_major, p.b_mn_major);
@@ -689,6 +722,8 @@ gemm_tf32_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
         __syncwarp();
     }
     } else {
+        // 128 x 80 + 256 x 208 registers fit the 384 x 168 the CTA was launched with; the increase
+        // blocks until that many are free in the CTA's own pool, so a larger request would never return
         ptx::setmaxnreg_inc<208>();
         // ------------------------------ accumulate + epilogue (both CTAs) ------------------------------
         const int quad = warp & 3;

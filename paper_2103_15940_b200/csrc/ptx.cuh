@@ -48,14 +48,17 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
-// Bounded wait: gives up after `limit` polls and returns false (the caller records the error).
+// Bounded wait: gives up once `limit` SM clock cycles have passed and returns false (the caller
+// records the error).  The limit is in cycles, not polls, because a failed try_wait may itself
+// have slept for an unspecified time.
 __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, uint32_t limit) {
     if (mbar_test_wait(bar, parity)) return true;
-    for (uint32_t i = 0; i < limit; ++i) {
+    const long long start = clock64();
+    for (uint32_t i = 0;; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
+        if (clock64() - start > (long long)limit) return false;
         if (i > 64) __nanosleep(32);
     }
-    return false;
 }
 
 // ---- TMA --------------------------------------------------------------------------------------
@@ -243,7 +246,8 @@ __device__ __forceinline__ void tmem_load_16cols(uint32_t taddr, uint32_t (&r)[1
 }
 // acc (two packed fp32) += {lo, hi}: one instruction for two round-to-nearest-even adds.
 __device__ __forceinline__ void add2_rn(unsigned long long& acc, uint32_t lo, uint32_t hi) {
-    asm("{\n\t.reg .b64 t;\n\tmov.b64 t, {%1, %2};\n\tadd.rn.f32x2 %0, %0, t;\n\t}" : "+l"(acc) : "r"(lo), "r"(hi));
+    // volatile: keeps the add behind the tcgen05.wait::ld that makes lo and hi valid
+    asm volatile("{\n\t.reg .b64 t;\n\tmov.b64 t, {%1, %2};\n\tadd.rn.f32x2 %0, %0, t;\n\t}" : "+l"(acc) : "r"(lo), "r"(hi));
 }
 __device__ __forceinline__ float2 unpack2(unsigned long long v) {
     float2 r;
