@@ -76,6 +76,8 @@ struct GemmParams {
     int b_mn_major;  // op(B) stored with N contiguous
     int tiles_m, tiles_n;
     int tma_store;   // C base, row pitch and row length are multiples of 16 bytes: C is written by TMA
+    int a_blocked, b_blocked;  // dense MN-major operand whose extent is a multiple of 32: its map is
+                               // rank 3, {32, K, extent / 32}, and one copy fetches a stage's 32-wide blocks
     // ---- work decomposition
     int tile_rows;         // rows of C owned by one M-tile (128, or whole image rows in mode 1)
     int kb_total;          // stages (k-blocks) in the whole contraction
@@ -240,13 +242,17 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                         ptx::mbar_expect_tx(bar, p.a_bytes + p.b_bytes);
                         if (p.mode == 0) {
                             const int k0 = kb * kBK;
-                            if (p.a_mn_major) {
+                            if (p.a_blocked) {
+                                ptx::tma_load_3d(sa, &tmap_a, bar, 0, k0, w.m0 >> 5);
+                            } else if (p.a_mn_major) {
                                 for (int c = 0; c < kBM / 32; ++c)
                                     ptx::tma_load_2d(sa + c * 4096u, &tmap_a, bar, w.m0 + c * 32, k0);
                             } else {
                                 ptx::tma_load_2d(sa, &tmap_a, bar, k0, w.m0);
                             }
-                            if (p.b_mn_major) {
+                            if (p.b_blocked) {
+                                ptx::tma_load_3d(sb, &tmap_b, bar, 0, k0, w.n0 >> 5);
+                            } else if (p.b_mn_major) {
                                 for (int c = 0; c < kBN / 32; ++c)
                                     ptx::tma_load_2d(sb + c * 4096u, &tmap_b, bar, w.n0 + c * 32, k0);
                             } else {
@@ -643,13 +649,17 @@ gemm_tf32_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
                     const uint32_t bar = ptx::map_to_cta(full_bar(stage), 0);  // the leader's barrier
                     const int k0 = kb * kBK;
                     ptx::mbar_expect_tx_cluster(bar, kPStageBytes);
-                    if (p.a_mn_major) {
+                    if (p.a_blocked) {
+                        ptx::tma_load_3d_pair(sa, &tmap_a, bar, 0, k0, m0 >> 5);
+                    } else if (p.a_mn_major) {
                         for (int c = 0; c < kBM / 32; ++c)
                             ptx::tma_load_2d_pair(sa + c * 4096u, &tmap_a, bar, m0 + c * 32, k0);
                     } else {
                         ptx::tma_load_2d_pair(sa, &tmap_a, bar, k0, m0);
                     }
-                    if (p.b_mn_major) {
+                    if (p.b_blocked) {
+                        ptx::tma_load_3d_pair(sb, &tmap_b, bar, 0, k0, n0 >> 5);
+                    } else if (p.b_mn_major) {
                         for (int c = 0; c < kBN / 64; ++c)
                             ptx::tma_load_2d_pair(sb + c * 4096u, &tmap_b, bar, n0 + c * 32, k0);
                     } else {
@@ -946,6 +956,7 @@ void dense_defaults(GemmParams* p) {
     p->tap_sign = 1;
     p->off_h = p->off_w = 0;
     p->full_tiles_m = 0;
+    p->a_blocked = p->b_blocked = 0;
 }
 
 }  // namespace
@@ -954,27 +965,45 @@ void dense_defaults(GemmParams* p) {
 // tiles (256 x 256).  Process-wide; see qfmt_gemm_tile_policy.
 static std::atomic<int> g_tile_policy{0};
 
-bool dense_uses_pair(int64_t M, int64_t N, int64_t K) {
-    (void)N; (void)K;
-    const int policy = g_tile_policy.load();
-    if (policy == 1) return false;
-    if (policy == 2) return true;
-    return M > kBM;  // with a single row of tiles the second CTA of a pair would idle
-}
+// How a dense product is laid over the GPU: tile shape and split-K factor.
+struct DensePlan {
+    bool pair;
+    int splits;
+};
 
-// Split-K factor for a dense product: used when the output has too few tiles to occupy the GPU and
-// K is long enough to share.  Planned for a 148-SM part so that it depends on the problem only.
-int plan_dense_splits(int64_t M, int64_t N, int64_t K, bool pair) {
-    const int64_t tile_rows = pair ? 2 * kBM : kBM, units = pair ? 74 : 148;
-    const int64_t tiles = ((M + tile_rows - 1) / tile_rows) * ((N + kBN - 1) / kBN);
+// Picks the plan with the least estimated time.  The unit is the time one CTA pair needs for one
+// 64-element K chunk of a 256 x 256 tile, about a microsecond; a single CTA needs 1.07 of it for
+// half the area.  A tile costs its chunks plus three units of exposed epilogue; split K adds a
+// reduction pass over (splits + 1) x M x N floats at about 4 TB/s plus a launch.  The wave count
+// is taken for a 148-SM part whatever the device, so that the plan, and with it the summation
+// order, depends on the problem alone.
+DensePlan plan_dense(int64_t M, int64_t N, int64_t K) {
+    const int policy = g_tile_policy.load();
     const int64_t kb_total = (K + kBK - 1) / kBK;
-    if (tiles * 5 >= units * 3) return 1;  // at least 60 % of the SMs have work already
-    int64_t splits = units / tiles;
-    if (splits > kMaxSplits) splits = kMaxSplits;
-    if (splits > kb_total / 16) splits = kb_total / 16;  // at least 512 K elements per split
-    if (splits < 1) splits = 1;
-    const int64_t per = (kb_total + splits - 1) / splits;
-    return (int)((kb_total + per - 1) / per);
+    DensePlan best = {policy == 2, 1};
+    double best_cost = -1.0;
+    for (int pair = 0; pair < 2; ++pair) {
+        if (policy == 1 && pair) continue;
+        if (policy == 2 && !pair) continue;
+        if (policy == 0 && pair && M <= kBM) continue;  // with one row of tiles the second CTA of a pair would idle
+        const int64_t tile_rows = pair ? 2 * kBM : kBM, units = pair ? 74 : 148;
+        const int64_t tiles = ((M + tile_rows - 1) / tile_rows) * ((N + kBN - 1) / kBN);
+        const double per_chunk = pair ? 1.0 : 1.07;
+        for (int64_t want = 1; want <= kMaxSplits; ++want) {
+            const int64_t per = (kb_total + want - 1) / want;           // K blocks per split
+            if (want > 1 && per < 16) break;                            // at least 512 K elements per split
+            const int64_t splits = per > 0 ? (kb_total + per - 1) / per : 1;
+            if (splits != want) continue;                               // same plan as a smaller request
+            const int64_t waves = (tiles * splits + units - 1) / units;
+            double cost = (double)waves * ((double)((per + kChunkKB - 1) / kChunkKB) * per_chunk + 3.0);
+            if (splits > 1) cost += 3.0 + (double)(splits + 1) * (double)M * (double)N * 4.0 / 4.0e6;
+            if (best_cost < 0.0 || cost < best_cost * 0.97) {  // more splits only for a clear gain
+                best_cost = cost;
+                best = {pair != 0, (int)splits};
+            }
+        }
+    }
+    return best;
 }
 
 int launch_pair(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc, const GemmParams& p,
@@ -1033,7 +1062,8 @@ int gemm_device(const qfmt_matrix_t* A, const qfmt_matrix_t* B, float* d_C, int6
     p.status = status;
     p.a_mn_major = A->trans ? 1 : 0;
     p.b_mn_major = B->trans ? 0 : 1;
-    const bool pair = dense_uses_pair(M, N, K);
+    const DensePlan plan = plan_dense(M, N, K);
+    const bool pair = plan.pair;
     p.tile_rows = pair ? 2 * kBM : kBM;
     p.tiles_m = (int)((M + p.tile_rows - 1) / p.tile_rows);
     p.tiles_n = (int)((N + kBN - 1) / kBN);
@@ -1044,7 +1074,7 @@ int gemm_device(const qfmt_matrix_t* A, const qfmt_matrix_t* B, float* d_C, int6
 
     // Split K when the workspace the caller lent has room for the partial sums (the recommended size
     // from qfmt_gemm_workspace_bytes always has); a smaller workspace gets fewer splits.
-    int splits = plan_dense_splits(M, N, K, pair);
+    int splits = plan.splits;
     while (splits > 1 && kWorkspaceHeader + (size_t)splits * (size_t)M * (size_t)N * sizeof(float) > workspace_bytes) --splits;
     float* partials = reinterpret_cast<float*>(reinterpret_cast<char*>(d_workspace) + kWorkspaceHeader);
     if (splits > 1) {
@@ -1057,10 +1087,24 @@ int gemm_device(const qfmt_matrix_t* A, const qfmt_matrix_t* B, float* d_C, int6
     }
 
     CUtensorMap ma, mb, mc;
-    if (p.a_mn_major) rc = make_map_2d(&ma, A->ptr, (uint64_t)M, (uint64_t)K, (uint64_t)A->ld, 32, kBK, true);
+    // An MN-major operand is staged as 32-wide column blocks of 4 KB.  When its extent is a multiple
+    // of 32 the matrix is described as {32, K, extent / 32} and one copy brings all of a stage's
+    // blocks; otherwise the last block would reach past the row's end, and each block is copied by
+    // itself from the plain rank-2 map, which zero-fills beyond the extent.
+    p.a_blocked = (p.a_mn_major && (M & 31) == 0) ? 1 : 0;
+    p.b_blocked = (p.b_mn_major && (N & 31) == 0) ? 1 : 0;
+    if (p.a_blocked) {
+        const uint64_t dims[3] = {32, (uint64_t)K, (uint64_t)M / 32}, strides[2] = {(uint64_t)A->ld, 32};
+        const uint32_t box[3] = {32, kBK, kBM / 32};
+        rc = make_map(&ma, A->ptr, 3, dims, strides, box, true);
+    } else if (p.a_mn_major) rc = make_map_2d(&ma, A->ptr, (uint64_t)M, (uint64_t)K, (uint64_t)A->ld, 32, kBK, true);
     else rc = make_map_2d(&ma, A->ptr, (uint64_t)K, (uint64_t)M, (uint64_t)A->ld, kBK, kBM, false);
     if (rc != QFMT_OK) return rc;
-    if (p.b_mn_major) rc = make_map_2d(&mb, B->ptr, (uint64_t)N, (uint64_t)K, (uint64_t)B->ld, 32, kBK, true);
+    if (p.b_blocked) {
+        const uint64_t dims[3] = {32, (uint64_t)K, (uint64_t)N / 32}, strides[2] = {(uint64_t)B->ld, 32};
+        const uint32_t box[3] = {32, kBK, (uint32_t)((pair ? kBN / 2 : kBN) / 32)};
+        rc = make_map(&mb, B->ptr, 3, dims, strides, box, true);
+    } else if (p.b_mn_major) rc = make_map_2d(&mb, B->ptr, (uint64_t)N, (uint64_t)K, (uint64_t)B->ld, 32, kBK, true);
     else rc = make_map_2d(&mb, B->ptr, (uint64_t)K, (uint64_t)N, (uint64_t)B->ld, kBK, pair ? kBN / 2 : kBN, false);
     if (rc != QFMT_OK) return rc;
     if (p.tma_store)
@@ -1297,7 +1341,7 @@ extern "C" size_t qfmt_gemm_workspace_bytes(const qfmt_matrix_t* A, const qfmt_m
     const int64_t M = A->trans ? A->cols : A->rows, K = A->trans ? A->rows : A->cols;
     const int64_t N = B->trans ? B->rows : B->cols;
     if (M <= 0 || N <= 0 || K <= 0 || M > (1 << 30) || N > (1 << 30) || K > (1 << 30)) return qfmt::kWorkspaceHeader;
-    const int splits = qfmt::plan_dense_splits(M, N, K, qfmt::dense_uses_pair(M, N, K));
+    const int splits = qfmt::plan_dense(M, N, K).splits;
     return qfmt::kWorkspaceHeader + (splits > 1 ? (size_t)splits * (size_t)M * (size_t)N * sizeof(float) : 0);
 }
 
