@@ -76,6 +76,7 @@ struct GemmParams {
     int b_mn_major;  // op(B) stored with N contiguous
     int tiles_m, tiles_n;
     int tma_store;   // C base, row pitch and row length are multiples of 16 bytes: C is written by TMA
+    int rows_box;    // filter gradient: image rows fetched by one copy (rows_per_blk when it divides the image height, else 1)
     int a_blocked, b_blocked;  // dense MN-major operand whose extent is a multiple of 32: its map is
                                // rank 3, {32, K, extent / 32}, and one copy fetches a stage's 32-wide blocks
     // ---- work decomposition
@@ -317,8 +318,8 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                         // Filter gradient: K = pixels.  A = output gradient (C_out is M), B = activations
                         // read at the tap that the N column block belongs to (C_in within a tap is N).
                         const int per_row = kBM / 32 + kBN / 32;
-                        for (int i = lane; i < p.rows_per_blk * per_row; i += 32) {
-                            const int j = i / per_row, c = i % per_row;
+                        for (int i = lane; i < (p.rows_per_blk / p.rows_box) * per_row; i += 32) {
+                            const int j = (i / per_row) * p.rows_box, c = i % per_row;
                             const int q = kb * p.rows_per_blk + j;
                             const int oh = q % p.img_rows, img = q / p.img_rows;
                             const uint32_t row_off = (uint32_t)(j * p.img_w) * 128u;
@@ -957,6 +958,7 @@ void dense_defaults(GemmParams* p) {
     p->off_h = p->off_w = 0;
     p->full_tiles_m = 0;
     p->a_blocked = p->b_blocked = 0;
+    p->rows_box = 1;
 }
 
 }  // namespace
@@ -1284,15 +1286,18 @@ int conv_device(int op, const qfmt_conv_t* g, const float* d_p, const float* d_q
     p.ldc = (long long)p.N;
     p.C = p.splits > 1 ? partials : d_out;
     p.split_stride = (long long)p.M * p.N;
+    // a stage's image rows never straddle two images when their count divides the image height: one
+    // copy then brings all of them for a channel block, else each row is copied by itself
+    p.rows_box = (OH % p.rows_per_blk == 0) ? p.rows_per_blk : 1;
     {
         const uint64_t dims[4] = {CO, OW, OH, N}, st[3] = {CO, OW * CO, OH * OW * CO};
-        const uint32_t box[4] = {32, (uint32_t)OW, 1, 1};
+        const uint32_t box[4] = {32, (uint32_t)OW, (uint32_t)p.rows_box, 1};
         rc = make_map(&ma, d_p, 4, dims, st, box, true);
         if (rc != QFMT_OK) return rc;
     }
     {
         const uint64_t dims[4] = {CI, W, H, N}, st[3] = {CI, W * CI, H * W * CI};
-        const uint32_t box[4] = {32, (uint32_t)OW, 1, 1};
+        const uint32_t box[4] = {32, (uint32_t)OW, (uint32_t)p.rows_box, 1};
         rc = make_map(&mb, d_q, 4, dims, st, box, true);
         if (rc != QFMT_OK) return rc;
     }
