@@ -276,9 +276,9 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                                                  h + dh, img);
                                 j += cnt;
                             }
-                            if (p.b_mn_major) {  // data gradient: filters [C_out][tap][C_in], C_in is N
-                                for (int c = 0; c < kBN / 32; ++c)
-                                    ptx::tma_load_3d(sb + c * 4096u, &tmap_b, bar, w.n0 + c * 32, tap, cb * 32);
+                            if (p.b_mn_major) {  // data gradient: filters [C_out][tap][C_in] seen as
+                                                 // {32, tap, C_out, C_in / 32}: one copy brings the eight column blocks
+                                ptx::tma_load_4d(sb, &tmap_b, bar, 0, tap, cb * 32, w.n0 >> 5);
                             } else {             // forward: filters [C_out][tap * C_in], K contiguous
                                 ptx::tma_load_2d(sb, &tmap_b, bar, tap * p.ck + cb * 32, w.n0);
                             }
@@ -1248,9 +1248,9 @@ int conv_device(int op, const qfmt_conv_t* g, const float* d_p, const float* d_q
         if (fwd) {  // filters [CO][TAPS*CI], K contiguous
             rc = make_map_2d(&mb, d_q, TAPS * CI, CO, TAPS * CI, kBK, kBN, false);
         } else {    // filters [CO][TAPS][CI]: N = CI contiguous, K = CO rows
-            const uint64_t dims[3] = {CI, TAPS, CO}, st[2] = {CI, TAPS * CI};
-            const uint32_t box[3] = {32, 1, kBK};
-            rc = make_map(&mb, d_q, 3, dims, st, box, true);
+            const uint64_t dims[4] = {32, TAPS, CO, CI / 32}, st[3] = {CI, TAPS * CI, 32};
+            const uint32_t box[4] = {32, 1, kBK, kBN / 32};
+            rc = make_map(&mb, d_q, 4, dims, st, box, true);
         }
         if (rc != QFMT_OK) return rc;
         if (p.full_tiles_m > 0)
