@@ -76,6 +76,14 @@ struct GemmParams {
     int b_mn_major;  // op(B) stored with N contiguous
     int tiles_m, tiles_n;
     int tma_store;   // C base, row pitch and row length are multiples of 16 bytes: C is written by TMA
+    // Balanced schedule (mode 1 only, sk_cpt > 0).  The tiles' 64-element K chunks form one sequence,
+    // tile after tile, and CTA b works on the b-th of gridDim.x equal ranges of it: up to sk_pieces
+    // consecutive tiles, the first and the last possibly in part.  A piece that begins inside a tile
+    // writes to the CTA's slot in sk_partials ([gridDim.x][tile_rows][N]) instead of C; a later
+    // kernel adds the slot to C.  Ranges are at least a tile long, so no tile has two such pieces.
+    int sk_cpt;              // chunks per tile, 0 = schedule off
+    int sk_pieces;           // pieces a CTA may have
+    float* sk_partials;
     int rows_box;    // filter gradient: image rows fetched by one copy (rows_per_blk when it divides the image height, else 1)
     int a_blocked, b_blocked;  // dense MN-major operand whose extent is a multiple of 32: its map is
                                // rank 3, {32, K, extent / 32}, and one copy fetches a stage's 32-wide blocks
@@ -109,10 +117,39 @@ struct RowMaps {
 // Position of work item t: tile coordinates, split, and the range of stages it sums.
 struct WorkItem {
     int tile_m, tile_n, split, m0, n0, kb_begin, num_kb;
+    int partial;  // balanced schedule: the piece begins inside its tile and goes to the CTA's slot
 };
+// Chunk range [lo, hi) of CTA b under the balanced schedule.
+__host__ __device__ __forceinline__ void sk_range(long long total, int ctas, int b, long long* lo, long long* hi) {
+    *lo = total * b / ctas;
+    *hi = total * (b + 1) / ctas;
+}
 __device__ __forceinline__ WorkItem decode_work(const GemmParams& p, int t) {
     WorkItem w;
     const int num_tiles = p.tiles_m * p.tiles_n;
+    w.partial = 0;
+    if (p.sk_cpt > 0) {
+        // t = b + piece * gridDim.x for CTA b
+        const int ctas = (int)gridDim.x, b = t % ctas, piece = t / ctas;
+        long long lo, hi;
+        sk_range((long long)num_tiles * p.sk_cpt, ctas, b, &lo, &hi);
+        const long long tile = lo / p.sk_cpt + piece, first = tile * p.sk_cpt;
+        const long long s = lo > first ? lo : first, e = hi < first + p.sk_cpt ? hi : first + p.sk_cpt;
+        w.split = 0;
+        if (s >= e) {  // no such piece
+            w.tile_m = w.tile_n = w.m0 = w.n0 = w.kb_begin = w.num_kb = 0;
+            return w;
+        }
+        w.tile_m = (int)(tile % p.tiles_m);
+        w.tile_n = (int)(tile / p.tiles_m);
+        w.m0 = w.tile_m * p.tile_rows;
+        w.n0 = w.tile_n * kBN;
+        w.kb_begin = (int)(s - first) * kChunkKB;
+        const int kb_end = (int)(e - first) * kChunkKB < p.kb_total ? (int)(e - first) * kChunkKB : p.kb_total;
+        w.num_kb = kb_end - w.kb_begin;
+        w.partial = s > first ? 1 : 0;
+        return w;
+    }
     const int tile = t % num_tiles;
     w.split = t / num_tiles;
     w.tile_m = tile % p.tiles_m;
@@ -161,8 +198,8 @@ __device__ __forceinline__ void raise_timeout(const GemmParams& p, volatile int*
 
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tf32_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
-                 const __grid_constant__ CUtensorMap tmap_c, const __grid_constant__ RowMaps row_maps,
-                 const GemmParams p) {
+                 const __grid_constant__ CUtensorMap tmap_c, const __grid_constant__ CUtensorMap tmap_p,
+                 const __grid_constant__ RowMaps row_maps, const GemmParams p) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = ptx::smem_addr(smem_raw);
     const uint32_t tiles = (raw + 1023u) & ~1023u;  // swizzled tiles need 1024-byte alignment
@@ -206,6 +243,7 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
         ptx::prefetch_tensormap(&tmap_a);
         ptx::prefetch_tensormap(&tmap_b);
         if (p.tma_store) ptx::prefetch_tensormap(&tmap_c);
+        if (p.sk_cpt > 0) ptx::prefetch_tensormap(&tmap_p);
     }
     if (warp == 1) {
         ptx::tmem_alloc(ptx::smem_addr(const_cast<uint32_t*>(tmem_slot)), kTmemCols);
@@ -216,7 +254,7 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
 
-    const int num_work = p.tiles_m * p.tiles_n * p.splits;
+    const int num_work = p.sk_cpt > 0 ? p.sk_pieces * (int)gridDim.x : p.tiles_m * p.tiles_n * p.splits;
 
     // Registers are allocated per group of four warps: the producer/MMA group keeps 64 per thread,
     // the accumulate groups take 224 (128 running sums + 32 freshly loaded values + addressing).
@@ -434,7 +472,9 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
             const int m0 = w.m0, n0 = w.n0, num_kb = w.num_kb;
             // rows of C this tile may write, and where split results go
             const int m_end = m0 + p.tile_rows < p.M ? m0 + p.tile_rows : p.M;
-            float* const c_base = p.C + (long long)w.split * p.split_stride;
+            // a piece for the CTA's slot addresses it as if the slot were the tile's place in C
+            float* const c_base = w.partial ? p.sk_partials + ((long long)blockIdx.x * p.tile_rows - m0) * p.ldc
+                                            : p.C + (long long)w.split * p.split_stride;
             // In mode 1 the C tensor map is [complete tiles][tile_rows][N]; an incomplete last tile
             // takes the scalar path.
             const bool use_tma = p.tma_store && (p.mode != 1 || w.tile_m < p.full_tiles_m);
@@ -509,9 +549,10 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                             if (row0 < m_end && col0 < p.N) {
                                 const uint32_t src = my_stage_addr + (pass & 1) * kOutBoxBytes;
                                 const int y = p.mode == 1 ? quad * 32 : row0;
-                                const int z = p.mode == 1 ? w.tile_m : w.split;
-                                if (flushed) ptx::tma_reduce_add_3d(&tmap_c, src, col0, y, z);
-                                else ptx::tma_store_3d(&tmap_c, src, col0, y, z);
+                                const int z = w.partial ? (int)blockIdx.x : (p.mode == 1 ? w.tile_m : w.split);
+                                const CUtensorMap* cm = w.partial ? &tmap_p : &tmap_c;
+                                if (flushed) ptx::tma_reduce_add_3d(cm, src, col0, y, z);
+                                else ptx::tma_store_3d(cm, src, col0, y, z);
                             }
                             ptx::bulk_commit();  // committed even when empty: the wait above counts groups
                         }
@@ -931,8 +972,34 @@ splitk_reduce_kernel(const float* __restrict__ part, float* __restrict__ C, long
 constexpr size_t kWorkspaceHeader = 256;  // status word and padding ahead of the partial sums
 constexpr int kMaxSplits = 32;
 
-int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc, const RowMaps& rows,
-                const GemmParams& p, const DeviceInfo& dev, cudaStream_t stream) {
+// Balanced schedule, second pass: CTA b's first piece began inside a tile and sits in slot b; add it
+// to the tile's place in C, which the CTA before wrote.  kFixupParts blocks per slot, each taking
+// every kFixupParts-th row; N is a multiple of 32 here, so rows are moved as float4.
+constexpr int kFixupParts = 16;
+__global__ void __launch_bounds__(256)
+streamk_fixup_kernel(const float* __restrict__ partials, float* __restrict__ C, int ctas, int num_tiles, int tiles_m,
+                     int cpt, int tile_rows, long long M, long long N) {
+    const int b = blockIdx.x / kFixupParts, part = blockIdx.x % kFixupParts;
+    long long lo, hi;
+    sk_range((long long)num_tiles * cpt, ctas, b, &lo, &hi);
+    const long long tile = lo / cpt;
+    if (lo >= hi || lo == tile * cpt) return;  // nothing, or the first piece began with its tile
+    const long long tile_m = tile % tiles_m, tile_n = tile / tiles_m;
+    const long long row0 = tile_m * tile_rows, col0 = tile_n * kBN;
+    const long long rows = row0 + tile_rows < M ? tile_rows : M - row0;
+    const long long cols4 = (col0 + kBN < N ? kBN : N - col0) / 4;
+    const float* src = partials + (long long)b * tile_rows * N;  // the slot is addressed like [tile_rows][N]
+    for (long long r = part; r < rows; r += kFixupParts) {
+        for (long long c4 = threadIdx.x; c4 < cols4; c4 += blockDim.x) {
+            float4* g = reinterpret_cast<float4*>(C + (row0 + r) * N + col0) + c4;
+            const float4 a = *g, v = *(reinterpret_cast<const float4*>(src + r * N + col0) + c4);
+            *g = make_float4(__fadd_rn(a.x, v.x), __fadd_rn(a.y, v.y), __fadd_rn(a.z, v.z), __fadd_rn(a.w, v.w));
+        }
+    }
+}
+
+int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc, const CUtensorMap& mp,
+                const RowMaps& rows, const GemmParams& p, const DeviceInfo& dev, cudaStream_t stream) {
     static bool attr_set[64] = {};
     if (dev.ordinal < 0 || dev.ordinal >= 64 || !attr_set[dev.ordinal]) {
         QFMT_CUDA_TRY(cudaFuncSetAttribute(gemm_tf32_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes));
@@ -940,8 +1007,13 @@ int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap&
     }
     const long long work = (long long)p.tiles_m * p.tiles_n * p.splits;
     const int grid = work < dev.sm_count ? (int)work : dev.sm_count;
-    gemm_tf32_kernel<<<grid, kThreads, kSmemBytes, stream>>>(ma, mb, mc, rows, p);
+    gemm_tf32_kernel<<<grid, kThreads, kSmemBytes, stream>>>(ma, mb, mc, mp, rows, p);
     QFMT_CUDA_TRY(cudaGetLastError());
+    if (p.sk_cpt > 0) {
+        streamk_fixup_kernel<<<grid * kFixupParts, 64, 0, stream>>>(p.sk_partials, p.C, grid, p.tiles_m * p.tiles_n, p.tiles_m,
+                                                       p.sk_cpt, p.tile_rows, (long long)p.M, (long long)p.N);
+        QFMT_CUDA_TRY(cudaGetLastError());
+    }
     return QFMT_OK;
 }
 
@@ -959,6 +1031,9 @@ void dense_defaults(GemmParams* p) {
     p->full_tiles_m = 0;
     p->a_blocked = p->b_blocked = 0;
     p->rows_box = 1;
+    p->sk_cpt = 0;
+    p->sk_pieces = 1;
+    p->sk_partials = nullptr;
 }
 
 }  // namespace
@@ -1118,7 +1193,7 @@ int gemm_device(const qfmt_matrix_t* A, const qfmt_matrix_t* B, float* d_C, int6
     } else {
         RowMaps rows;
         for (int i = 0; i < kMaxRowMaps; ++i) rows.m[i] = ma;  // unused in dense mode
-        rc = launch_gemm(ma, mb, mc, rows, p, dev, stream);
+        rc = launch_gemm(ma, mb, mc, mc, rows, p, dev, stream);
     }
     if (rc != QFMT_OK) return rc;
     if (p.splits > 1) {
@@ -1137,6 +1212,8 @@ namespace {
 struct ConvPlan {
     int64_t oh, ow;
     int splits;
+    int sk_cpt;      // forward / data gradient: chunks per tile when the balanced schedule is used, else 0
+    int sk_pieces;
     size_t workspace;
 };
 constexpr int kPlanSms = 148;  // B200; the split factor is planned for it so that it does not vary
@@ -1153,9 +1230,29 @@ int plan_conv(int op, const qfmt_conv_t* g, ConvPlan* plan) {
         (int64_t)g->r * g->s * g->c_in > (1 << 30))
         return QFMT_ERR_BAD_ARG;
     plan->splits = 1;
+    plan->sk_cpt = 0;
+    plan->sk_pieces = 1;
     plan->workspace = kWorkspaceHeader;
     if (op == QFMT_CONV_FWD && plan->ow > kBM) return QFMT_ERR_BAD_ARG;   // an M-tile is made of whole output rows
     if (op == QFMT_CONV_DGRAD && g->w > kBM) return QFMT_ERR_BAD_ARG;
+    if (op != QFMT_CONV_WGRAD) {
+        // With more tiles than SMs and a last wave that leaves many SMs idle, the K chunks of all
+        // tiles are dealt out in equal ranges instead (see GemmParams::sk_cpt).
+        const bool fwd = op == QFMT_CONV_FWD;
+        const int64_t rows = fwd ? plan->oh : g->h, width = fwd ? plan->ow : g->w;
+        const int64_t rows_per_blk = kBM / width, n_cols = fwd ? g->c_out : g->c_in, src_c = fwd ? g->c_in : g->c_out;
+        const int64_t tiles = (((int64_t)g->n * rows + rows_per_blk - 1) / rows_per_blk) * ((n_cols + kBN - 1) / kBN);
+        const int64_t kb_total = (int64_t)g->r * g->s * (src_c / 32), cpt = (kb_total + kChunkKB - 1) / kChunkKB;
+        const int64_t waves = (tiles + kPlanSms - 1) / kPlanSms;
+        // It pays when the last of a few waves is poorly filled and tiles are long: every piece ends
+        // with an output flush of its own, and pieces that begin inside a tile are added to C later.
+        if (tiles >= kPlanSms && waves <= 3 && waves * kPlanSms * 100 >= tiles * 115 && cpt >= 24) {
+            const int64_t range = (tiles * cpt + kPlanSms - 1) / kPlanSms;
+            plan->sk_cpt = (int)cpt;
+            plan->sk_pieces = (int)((range + cpt - 1) / cpt + 1);
+            plan->workspace += (size_t)kPlanSms * (size_t)(rows_per_blk * width) * (size_t)n_cols * sizeof(float);
+        }
+    }
     if (op == QFMT_CONV_WGRAD) {
         if (plan->ow > kBK) return QFMT_ERR_BAD_ARG;                      // a stage is made of whole output rows
         const int rows_per_blk = kBK / (int)plan->ow;
@@ -1258,7 +1355,16 @@ int conv_device(int op, const qfmt_conv_t* g, const float* d_p, const float* d_q
                             (uint64_t)p.tile_rows * n_cols);
         else { mc = ma; p.tma_store = 0; }
         if (rc != QFMT_OK) return rc;
-        return launch_gemm(ma, mb, mc, rmaps, p, dev, stream);
+        CUtensorMap mp = mc;
+        if (plan.sk_cpt > 0 && dev.sm_count == kPlanSms && p.tma_store) {  // the slots were sized for this many CTAs
+            p.sk_cpt = plan.sk_cpt;
+            p.sk_pieces = plan.sk_pieces;
+            p.sk_partials = reinterpret_cast<float*>(reinterpret_cast<char*>(d_workspace) + kWorkspaceHeader);
+            rc = make_map_c(&mp, p.sk_partials, n_cols, (uint64_t)p.tile_rows, (uint64_t)kPlanSms, n_cols,
+                            (uint64_t)p.tile_rows * n_cols);
+            if (rc != QFMT_OK) return rc;
+        }
+        return launch_gemm(ma, mb, mc, mp, rmaps, p, dev, stream);
     }
 
     // ---- filter gradient: dW [CO][TAPS*CI] = sum over pixels of dY^T (CO x pixels) * X_tap (pixels x CI)
@@ -1305,7 +1411,7 @@ int conv_device(int op, const qfmt_conv_t* g, const float* d_p, const float* d_q
     if (rc != QFMT_OK) return rc;
     RowMaps rows;
     for (int i = 0; i < kMaxRowMaps; ++i) rows.m[i] = ma;  // unused by the filter gradient
-    rc = launch_gemm(ma, mb, mc, rows, p, dev, stream);
+    rc = launch_gemm(ma, mb, mc, mc, rows, p, dev, stream);
     if (rc != QFMT_OK) return rc;
     if (p.splits > 1) {
         const long long total = (long long)p.M * p.N;
