@@ -84,6 +84,9 @@ struct GemmParams {
     int sk_cpt;              // chunks per tile, 0 = schedule off
     int sk_pieces;           // pieces a CTA may have
     float* sk_partials;
+    int wg_padded;   // filter gradient, padded stages: an image row takes a power-of-two number of K rows
+                     // (the copy engine zero-fills the columns past the image), a stage is 32 K rows
+                     // exactly, and one rank-5 copy per operand brings all of its channel blocks
     int rows_box;    // filter gradient: image rows fetched by one copy (rows_per_blk when it divides the image height, else 1)
     int a_blocked, b_blocked;  // dense MN-major operand whose extent is a multiple of 32: its map is
                                // rank 3, {32, K, extent / 32}, and one copy fetches a stage's 32-wide blocks
@@ -352,7 +355,18 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                     if (!ok) { dead = true; break; }
                     const uint32_t sa = tiles + stage * kStageBytes;
                     const uint32_t sb = sa + kABytes;
-                    {
+                    if (p.wg_padded) {
+                        // Both operands as {32 channels, padded row, rows, image, channel block}: the
+                        // tile's 256 columns lie within one tap here, so B is one box at that tap's offset.
+                        if (lane == 0) {
+                            const int q = kb * p.rows_per_blk;
+                            const int oh = q % p.img_rows, img = q / p.img_rows;
+                            const int tap = n0 / p.ck, ci = n0 % p.ck;
+                            ptx::tma_load_5d(sa, &tmap_a, bar, 0, 0, oh, img, m0 >> 5);
+                            ptx::tma_load_5d(sb, &tmap_b, bar, 0, tap % p.taps_s + p.off_w, oh + tap / p.taps_s + p.off_h,
+                                             img, ci >> 5);
+                        }
+                    } else {
                         // Filter gradient: K = pixels.  A = output gradient (C_out is M), B = activations
                         // read at the tap that the N column block belongs to (C_in within a tap is N).
                         const int per_row = kBM / 32 + kBN / 32;
@@ -917,15 +931,15 @@ EncodeTiledFn encode_tiled_fn() {
     return fn;
 }
 
-// fp32 tensor map of rank 2..4 with dim0 contiguous; strides in elements for dims 1..rank-1; zero
+// fp32 tensor map of rank 2..5 with dim0 contiguous; strides in elements for dims 1..rank-1; zero
 // fill out of bounds.  Swizzle: 16-byte chunks within 128 bytes for K-major operand tiles and for
 // C, 32-byte chunks for MN-major operand tiles.
 int make_map(CUtensorMap* map, const float* base, int rank, const uint64_t* dims, const uint64_t* strides_elems,
              const uint32_t* box, bool mn_major) {
     EncodeTiledFn fn = encode_tiled_fn();
     if (fn == nullptr) { set_last_cuda_error((int)cudaErrorSymbolNotFound); return QFMT_ERR_CUDA; }
-    cuuint64_t d[4], st[3];
-    cuuint32_t bx[4], estr[4] = {1, 1, 1, 1};
+    cuuint64_t d[5], st[4];
+    cuuint32_t bx[5], estr[5] = {1, 1, 1, 1, 1};
     for (int i = 0; i < rank; ++i) { d[i] = dims[i]; bx[i] = box[i]; }
     for (int i = 0; i + 1 < rank; ++i) st[i] = strides_elems[i] * sizeof(float);
     CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, (cuuint32_t)rank, const_cast<float*>(base), d, st, bx, estr,
@@ -1031,6 +1045,7 @@ void dense_defaults(GemmParams* p) {
     p->full_tiles_m = 0;
     p->a_blocked = p->b_blocked = 0;
     p->rows_box = 1;
+    p->wg_padded = 0;
     p->sk_cpt = 0;
     p->sk_pieces = 1;
     p->sk_partials = nullptr;
@@ -1216,6 +1231,15 @@ struct ConvPlan {
     int sk_pieces;
     size_t workspace;
 };
+// Output rows per K stage of the filter gradient, and whether stages are padded (GemmParams::wg_padded):
+// padded when every stage then stays inside one image and a tile's 256 columns inside one tap.
+int wgrad_rows_per_stage(int64_t oh, int64_t ow, int64_t c_in, int* padded_row) {
+    int wpad = 1;
+    while (wpad < ow) wpad *= 2;
+    const bool padded = wpad <= kBK && oh % (kBK / wpad) == 0 && c_in % kBN == 0;
+    if (padded_row != nullptr) *padded_row = padded ? wpad : 0;
+    return padded ? kBK / wpad : kBK / (int)ow;
+}
 constexpr int kPlanSms = 148;  // B200; the split factor is planned for it so that it does not vary
 int plan_conv(int op, const qfmt_conv_t* g, ConvPlan* plan) {
     if (g == nullptr || op < QFMT_CONV_FWD || op > QFMT_CONV_WGRAD) return QFMT_ERR_BAD_ARG;
@@ -1255,7 +1279,7 @@ int plan_conv(int op, const qfmt_conv_t* g, ConvPlan* plan) {
     }
     if (op == QFMT_CONV_WGRAD) {
         if (plan->ow > kBK) return QFMT_ERR_BAD_ARG;                      // a stage is made of whole output rows
-        const int rows_per_blk = kBK / (int)plan->ow;
+        const int rows_per_blk = wgrad_rows_per_stage(plan->oh, plan->ow, g->c_in, nullptr);
         const int64_t kb_total = ((int64_t)g->n * plan->oh + rows_per_blk - 1) / rows_per_blk;
         const int64_t tiles = (((int64_t)g->c_out + kBM - 1) / kBM) * (((int64_t)g->r * g->s * g->c_in + kBN - 1) / kBN);
         int64_t splits = kPlanSms / tiles;
@@ -1372,7 +1396,10 @@ int conv_device(int op, const qfmt_conv_t* g, const float* d_p, const float* d_q
     p.img_rows = (int)OH;
     p.img_w = (int)OW;
     p.total_q = (int)(N * OH);
-    p.rows_per_blk = kBK / (int)OW;
+    int padded_row = 0;
+    p.rows_per_blk = wgrad_rows_per_stage((int64_t)OH, (int64_t)OW, (int64_t)CI, &padded_row);
+    p.wg_padded = padded_row > 0 ? 1 : 0;
+    const uint32_t wpad = (uint32_t)padded_row;
     p.M = (int)CO;
     p.N = (int)(TAPS * CI);
     p.K = (int)(N * OH * OW);
@@ -1386,8 +1413,8 @@ int conv_device(int op, const qfmt_conv_t* g, const float* d_p, const float* d_q
     p.kb_per_split = (p.kb_total + p.splits - 1) / p.splits;
     p.a_mn_major = 1;
     p.b_mn_major = 1;
-    p.a_bytes = (uint32_t)((kBM / 32) * p.rows_per_blk * (int)OW * 128);
-    p.b_bytes = (uint32_t)((kBN / 32) * p.rows_per_blk * (int)OW * 128);
+    p.a_bytes = p.wg_padded ? kABytes : (uint32_t)((kBM / 32) * p.rows_per_blk * (int)OW * 128);
+    p.b_bytes = p.wg_padded ? kBBytes : (uint32_t)((kBN / 32) * p.rows_per_blk * (int)OW * 128);
     float* partials = reinterpret_cast<float*>(reinterpret_cast<char*>(d_workspace) + kWorkspaceHeader);
     p.ldc = (long long)p.N;
     p.C = p.splits > 1 ? partials : d_out;
@@ -1395,6 +1422,16 @@ int conv_device(int op, const qfmt_conv_t* g, const float* d_p, const float* d_q
     // a stage's image rows never straddle two images when their count divides the image height: one
     // copy then brings all of them for a channel block, else each row is copied by itself
     p.rows_box = (OH % p.rows_per_blk == 0) ? p.rows_per_blk : 1;
+    if (p.wg_padded) {
+        const uint64_t da[5] = {32, OW, OH, N, CO / 32}, sa_[4] = {CO, OW * CO, OH * OW * CO, 32};
+        const uint32_t ba[5] = {32, wpad, (uint32_t)p.rows_per_blk, 1, kBM / 32};
+        rc = make_map(&ma, d_p, 5, da, sa_, ba, true);
+        if (rc != QFMT_OK) return rc;
+        const uint64_t db[5] = {32, W, H, N, CI / 32}, sb_[4] = {CI, W * CI, H * W * CI, 32};
+        const uint32_t bb[5] = {32, wpad, (uint32_t)p.rows_per_blk, 1, kBN / 32};
+        rc = make_map(&mb, d_q, 5, db, sb_, bb, true);
+        if (rc != QFMT_OK) return rc;
+    } else {
     {
         const uint64_t dims[4] = {CO, OW, OH, N}, st[3] = {CO, OW * CO, OH * OW * CO};
         const uint32_t box[4] = {32, (uint32_t)OW, (uint32_t)p.rows_box, 1};
@@ -1406,6 +1443,7 @@ int conv_device(int op, const qfmt_conv_t* g, const float* d_p, const float* d_q
         const uint32_t box[4] = {32, (uint32_t)OW, (uint32_t)p.rows_box, 1};
         rc = make_map(&mb, d_q, 4, dims, st, box, true);
         if (rc != QFMT_OK) return rc;
+    }
     }
     rc = make_map_c(&mc, p.C, (uint64_t)p.N, (uint64_t)p.M, (uint64_t)p.splits, (uint64_t)p.N, (uint64_t)p.M * p.N);
     if (rc != QFMT_OK) return rc;

@@ -78,6 +78,9 @@ SMALL = [
     (9, 32, 14, 14, 32, 3, 3, 1, 1),      # 126 image rows: split-K in the filter gradient
     (2, 96, 6, 5, 32, 5, 5, 2, 2),        # 25 taps
     (1, 32, 3, 3, 32, 3, 3, 0, 0),        # single output pixel
+    (3, 256, 8, 7, 64, 3, 3, 1, 1),       # filter gradient with padded stages: 7-pixel rows take 8 K rows
+    (2, 256, 10, 9, 32, 3, 3, 0, 0),      # the same without zero padding: the pad rows of B hold real pixels
+    (2, 512, 4, 14, 32, 1, 1, 0, 0),      # padded stages, two 256-column tiles per tap
 ]
 
 
