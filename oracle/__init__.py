@@ -61,6 +61,17 @@ def _L() -> ctypes.CDLL:
         lib.oracle_gemm_sampled.restype = None
         lib.oracle_conv.argtypes = [i32, vp, vp, vp, vp, i64, vp, vp]
         lib.oracle_conv.restype = None
+        lib.oracle_add_round_bits.argtypes = [u32, u32, i32, i32, i32]
+        lib.oracle_add_round_bits.restype = u32
+        lib.oracle_fmac_bits.argtypes = [u32, u32, u32, i32, i32, i32]
+        lib.oracle_fmac_bits.restype = u32
+        lib.oracle_bias_quantize_stats.argtypes = [vp, i64, i64, i64, vp, vp, i64, i32, i32, i32, u32, vp]
+        lib.oracle_bias_quantize_stats.restype = None
+        lib.oracle_fmac8_gemm.argtypes = [vp, i64, i32, vp, i64, i32, i64, i64, i64, i32, i32, i32, i32, vp]
+        lib.oracle_fmac8_gemm.restype = None
+        lib.oracle_fmac8_gemm_sampled.argtypes = [vp, i64, i32, vp, i64, i32, i64, i32, i32, i32, i32, vp, vp,
+                                                  i64, vp]
+        lib.oracle_fmac8_gemm_sampled.restype = None
         _lib = lib
     return _lib
 
@@ -109,6 +120,16 @@ def encode_code(qbits: int, e: int, m: int) -> int:
     return _L().oracle_encode_code(qbits, e, m)
 
 
+def add_round_bits(abits: int, bbits: int, e: int, m: int, denormals: int = 1) -> int:
+    """round(a + b) to (e, m): the exact sum of two fp32 words, rounded once."""
+    return _L().oracle_add_round_bits(abits, bbits, e, m, denormals)
+
+
+def fmac_bits(abits: int, xbits: int, ybits: int, e: int, m: int, denormals: int = 1) -> int:
+    """FMAC: round(a + x*y) to (e, m), one rounding of the exact value."""
+    return _L().oracle_fmac_bits(abits, xbits, ybits, e, m, denormals)
+
+
 # ---- tensors ----------------------------------------------------------------------------------
 def quantize_stats(x: np.ndarray, e: int, m: int, denormals: int = 1, loss_scale: float = 1.0,
                    want_q: bool = True, want_stats: bool = True):
@@ -154,6 +175,60 @@ def gemm_sampled(A: np.ndarray, B: np.ndarray, ii: np.ndarray, jj: np.ndarray,
                              int(transB), K, ii.ctypes.data, jj.ctypes.data, ii.size, c.ctypes.data,
                              t.ctypes.data)
     return c, t
+
+
+def bias_quantize_stats(acc: np.ndarray, bias: Optional[np.ndarray], e: int, m: int, denormals: int = 1,
+                        loss_scale: float = 1.0):
+    """Y = R(R(S acc) + R(S bias)) with statistics of Y; acc is rows x cols, bias has cols entries."""
+    a = _mat(acc)
+    rows, cols = a.shape
+    out = np.empty((rows, cols), dtype=np.uint32)
+    st = np.zeros(STATS_WORDS, dtype=np.uint64)
+    b = None
+    if bias is not None:
+        b = np.ascontiguousarray(bias, dtype=np.float32).reshape(-1)
+        assert b.size == cols
+    _L().oracle_bias_quantize_stats(a.ctypes.data, rows, cols, cols, b.ctypes.data if b is not None else None,
+                                    out.ctypes.data, cols, e, m, int(denormals), _f32_bits(loss_scale),
+                                    st.ctypes.data)
+    return out.view(np.float32), st
+
+
+def _check_narrow(a: np.ndarray) -> None:
+    # the FMAC routines take operands with at most 12 significant bits (formats with m <= 11)
+    if np.any(a.view(np.uint32) & np.uint32(0xFFF)):
+        raise ValueError("FMAC operands must hold values of a format with m <= 11")
+
+
+def fmac8_gemm(A: np.ndarray, B: np.ndarray, e: int, m: int, denormals: int = 1, transA: bool = False,
+               transB: bool = False, group: int = 8) -> np.ndarray:
+    """Algorithm 1 for every output of op(A) op(B); returns the rounded results as float32."""
+    A, B = _mat(A), _mat(B)
+    _check_narrow(A)
+    _check_narrow(B)
+    M, K = (A.shape[1], A.shape[0]) if transA else A.shape
+    K2, N = (B.shape[1], B.shape[0]) if transB else B.shape
+    assert K == K2
+    C = np.empty((M, N), dtype=np.uint32)
+    _L().oracle_fmac8_gemm(A.ctypes.data, A.shape[1], int(transA), B.ctypes.data, B.shape[1], int(transB),
+                           M, N, K, e, m, int(denormals), group, C.ctypes.data)
+    return C.view(np.float32)
+
+
+def fmac8_gemm_sampled(A: np.ndarray, B: np.ndarray, ii: np.ndarray, jj: np.ndarray, e: int, m: int,
+                       denormals: int = 1, transA: bool = False, transB: bool = False,
+                       group: int = 8) -> np.ndarray:
+    A, B = _mat(A), _mat(B)
+    _check_narrow(A)
+    _check_narrow(B)
+    K = A.shape[0] if transA else A.shape[1]
+    ii = np.ascontiguousarray(ii, dtype=np.int64)
+    jj = np.ascontiguousarray(jj, dtype=np.int64)
+    c = np.empty(ii.size, dtype=np.uint32)
+    _L().oracle_fmac8_gemm_sampled(A.ctypes.data, A.shape[1], int(transA), B.ctypes.data, B.shape[1],
+                                   int(transB), K, e, m, int(denormals), group, ii.ctypes.data,
+                                   jj.ctypes.data, ii.size, c.ctypes.data)
+    return c.view(np.float32)
 
 
 CONV_FWD, CONV_DGRAD, CONV_WGRAD = 0, 1, 2

@@ -21,6 +21,10 @@
  *   - Section III-B: FMACS, a32 = round(a32 + x16*y16): exact products, wide accumulation.
  *     The contraction is order dependent in fp32, so the oracle gives the exact result
  *     (fp64 accumulation of exact products) together with sum |a||b| for the error bound.
+ *   - Section III-B, FMAC, a16 = round(a16 + x16*y16), and Algorithm 1 (FMAC-8): the exact value
+ *     of a + x*y is formed in integers and rounded once; the master accumulator adds in fp32.
+ *   - Section IV-A's layer formula Y = R(R(W^T X) + R(B)): exact sum of the two rounded
+ *     terms, rounded once more.
  *   - Section V: "denormal fraction" of each tensor is the logged statistic.
  *
  * Every number here is handled as an integer significand times a power of two.
@@ -269,6 +273,221 @@ void oracle_quantize_stats(const uint32_t *x, uint32_t *q, size_t n, int e, int 
 }
 
 /* ------------------------------------------------------------------------------------------ */
+/* Exact signed sums, rounded once.                                                             */
+/*                                                                                              */
+/* Both FMAC (Section III-B: a16 = round(a16 + x16*y16), one rounding of the exact value) and   */
+/* the layer formula of Section IV-A, Y = R(R(W^T X) + R(B)), need the exact sum of two finite  */
+/* numbers rounded once to a format.  A number is sign, sig * 2^exp2.                           */
+/* ------------------------------------------------------------------------------------------ */
+typedef struct {
+    int cls;  /* CLS_ZERO, CLS_FINITE, CLS_INF, CLS_NAN */
+    int sign; /* 1 = negative */
+    mag_t mg; /* for CLS_FINITE */
+} num_t;
+
+static num_t num_from_f32(uint32_t u) {
+    num_t r;
+    r.cls = decode_f32(u, &r.sign, &r.mg);
+    return r;
+}
+
+static mag_t strip_zeros(mag_t v) {
+    while (v.sig != 0 && (v.sig & 1u) == 0) {
+        v.sig >>= 1;
+        v.exp2 += 1;
+    }
+    return v;
+}
+
+/*
+ * Exact a + b for finite nonzero a, b whose significands, trailing zeros removed, are at most
+ * 24 bits wide.  The result is returned as sign and magnitude such that ROUNDING it to any
+ * format with m <= 23 (or comparing it with zero) gives what the exact sum would give:
+ * when the two numbers are within 38 binary places of each other the sum is formed exactly in
+ * 64-bit integers; when they are further apart the smaller one lies more than 14 places below
+ * the last bit of the larger, it cannot reach any grid point or halfway point of the result's
+ * neighbourhood, and it is replaced by one unit 38 places below the larger one's last bit,
+ * which lies strictly on the same side of all those points.
+ * Returns CLS_ZERO for an exact cancellation.
+ */
+static int exact_sum(int sa, mag_t a, int sb, mag_t b, int *sign, mag_t *out) {
+    a = strip_zeros(a);
+    b = strip_zeros(b);
+    int ta = floor_log2_u64(a.sig) + a.exp2, tb = floor_log2_u64(b.sig) + b.exp2;
+    if (tb > ta) { /* make a the one that reaches higher */
+        mag_t tm = a; a = b; b = tm;
+        int ts = sa; sa = sb; sb = ts;
+        int tt = ta; ta = tb; tb = tt;
+    }
+    int lo = a.exp2 < b.exp2 ? a.exp2 : b.exp2;
+    uint64_t A, B;
+    if (ta - lo <= 61) {
+        A = a.sig << (a.exp2 - lo);
+        B = b.sig << (b.exp2 - lo);
+    } else { /* b far below a: only its presence and sign matter */
+        A = a.sig << 38;
+        B = 1;
+        lo = a.exp2 - 38;
+    }
+    out->exp2 = lo;
+    if (sa == sb) {
+        out->sig = A + B;
+        *sign = sa;
+        return CLS_FINITE;
+    }
+    if (A == B) {
+        out->sig = 0;
+        *sign = 0;
+        return CLS_ZERO;
+    }
+    if (A > B) {
+        out->sig = A - B;
+        *sign = sa;
+    } else {
+        out->sig = B - A;
+        *sign = sb;
+    }
+    return CLS_FINITE;
+}
+
+/* IEEE rules for a sum whose operands are not both finite and nonzero; returns 1 if *r is set. */
+static int special_sum(num_t a, num_t b, num_t *r) {
+    r->mg.sig = 0;
+    r->mg.exp2 = 0;
+    if (a.cls == CLS_NAN || b.cls == CLS_NAN || (a.cls == CLS_INF && b.cls == CLS_INF && a.sign != b.sign)) {
+        r->cls = CLS_NAN; /* the positive quiet NaN stands for every invalid or propagated NaN */
+        r->sign = 0;
+        return 1;
+    }
+    if (a.cls == CLS_INF) { *r = a; return 1; }
+    if (b.cls == CLS_INF) { *r = b; return 1; }
+    if (a.cls == CLS_ZERO && b.cls == CLS_ZERO) {
+        r->cls = CLS_ZERO;
+        r->sign = a.sign & b.sign; /* -0 only when both are -0 (round to nearest) */
+        return 1;
+    }
+    if (a.cls == CLS_ZERO) { *r = b; return 1; }
+    if (b.cls == CLS_ZERO) { *r = a; return 1; }
+    return 0;
+}
+
+/* a + b, exact in the sense of exact_sum */
+static num_t num_add(num_t a, num_t b) {
+    num_t r;
+    if (special_sum(a, b, &r)) return r;
+    r.cls = exact_sum(a.sign, a.mg, b.sign, b.mg, &r.sign, &r.mg);
+    return r;
+}
+
+/* exact product */
+static num_t num_mul(num_t x, num_t y) {
+    num_t r;
+    r.sign = x.sign ^ y.sign;
+    r.mg.sig = 0;
+    r.mg.exp2 = 0;
+    if (x.cls == CLS_NAN || y.cls == CLS_NAN || (x.cls == CLS_INF && y.cls == CLS_ZERO) ||
+        (x.cls == CLS_ZERO && y.cls == CLS_INF)) {
+        r.cls = CLS_NAN;
+        r.sign = 0;
+    } else if (x.cls == CLS_INF || y.cls == CLS_INF) {
+        r.cls = CLS_INF;
+    } else if (x.cls == CLS_ZERO || y.cls == CLS_ZERO) {
+        r.cls = CLS_ZERO;
+    } else {
+        r.cls = CLS_FINITE;
+        r.mg.sig = x.mg.sig * y.mg.sig; /* < 2^48 */
+        r.mg.exp2 = x.mg.exp2 + y.mg.exp2;
+    }
+    return r;
+}
+
+/*
+ * Round a number to format (e, m): fp32 container bits.  Same rules as oracle_quantize_bits
+ * (overflow to inf, sign kept on zeros, flush after rounding when denormals are off).
+ */
+static uint32_t num_round_bits(num_t v, int e, int m, int keep_denormals, int *was_denormal) {
+    uint32_t sign = (uint32_t)v.sign << 31;
+    if (was_denormal) *was_denormal = 0;
+    if (v.cls == CLS_NAN) return sign | 0x7FC00000u;
+    if (v.cls == CLS_INF) return sign | 0x7F800000u;
+    if (v.cls == CLS_ZERO) return sign;
+    int inf;
+    mag_t q = round_to_format(v.mg, e, m, &inf);
+    if (inf) return sign | 0x7F800000u;
+    if (q.sig == 0) return sign;
+    int is_den = (floor_log2_u64(q.sig) + q.exp2) < oracle_emin(e);
+    if (was_denormal) *was_denormal = is_den;
+    if (is_den && !keep_denormals) return sign;
+    return sign | encode_f32_mag(q);
+}
+
+/* round(a + b) to (e, m) for two fp32 words (their trailing-zero-free significands fit 24 bits). */
+uint32_t oracle_add_round_bits(uint32_t abits, uint32_t bbits, int e, int m, int keep_denormals) {
+    return num_round_bits(num_add(num_from_f32(abits), num_from_f32(bbits)), e, m, keep_denormals, NULL);
+}
+
+/*
+ * FMAC (Section III-B): round(a + x*y) to (e, m) with ONE rounding of the exact value.
+ * x and y must hold values with at most 12 significant bits each (any format with m <= 11),
+ * so that the product's significand fits 24 bits.
+ */
+uint32_t oracle_fmac_bits(uint32_t abits, uint32_t xbits, uint32_t ybits, int e, int m, int keep_denormals) {
+    num_t p = num_mul(num_from_f32(xbits), num_from_f32(ybits));
+    if (p.cls == CLS_FINITE) p.mg = strip_zeros(p.mg);
+    return num_round_bits(num_add(num_from_f32(abits), p), e, m, keep_denormals, NULL);
+}
+
+/*
+ * Layer output of Section IV-A's worked example, Y = R(R(acc) + R(B)): acc is the matrix
+ * product (rows x cols, leading dimension ld_acc), bias has one entry per column.  Both are
+ * multiplied by the loss scale and rounded as oracle_quantize_stats does, added exactly and
+ * rounded once more.  Statistics describe the OUTPUT tensor, with the exact sum in the role of
+ * the input: n_zero_in counts sums that are zero, n_underflow nonzero sums that end as zero,
+ * n_overflow finite sums that end as inf, n_inf_in / n_nan infinite / NaN sums.
+ * bias may be NULL (then Y = R(acc), statistics as in oracle_quantize_stats).
+ * stats[] is ADDED to; out may be NULL.
+ */
+void oracle_bias_quantize_stats(const uint32_t *acc, int64_t rows, int64_t cols, int64_t ld_acc,
+                                const uint32_t *bias, uint32_t *out, int64_t ld_out, int e, int m,
+                                int keep_denormals, uint32_t scale_bits, uint64_t *stats) {
+    for (int64_t i = 0; i < rows; ++i)
+        for (int64_t j = 0; j < cols; ++j) {
+            uint32_t xb = acc[i * ld_acc + j];
+            uint32_t yb = (scale_bits == 0x3F800000u) ? xb : oracle_scale_bits(xb, scale_bits);
+            num_t s;
+            if (bias) {
+                uint32_t ra = oracle_quantize_bits(yb, e, m, keep_denormals, NULL);
+                uint32_t bb = (scale_bits == 0x3F800000u) ? bias[j] : oracle_scale_bits(bias[j], scale_bits);
+                uint32_t rb = oracle_quantize_bits(bb, e, m, keep_denormals, NULL);
+                s = num_add(num_from_f32(ra), num_from_f32(rb));
+            } else {
+                s = num_from_f32(yb);
+                if (s.cls == CLS_NAN) s.sign = (int)(xb >> 31);
+            }
+            int was_den;
+            uint32_t qb = num_round_bits(s, e, m, keep_denormals, &was_den);
+            if (out) out[i * ld_out + j] = qb;
+            if (!stats) continue;
+            int q_zero = (qb & 0x7FFFFFFFu) == 0;
+            int q_inf = (qb & 0x7FFFFFFFu) == 0x7F800000u;
+            int in_cls = s.cls;
+            if (!bias) { /* as oracle_quantize_stats: classes of the unscaled input */
+                int sx;
+                mag_t mx;
+                in_cls = decode_f32(xb, &sx, &mx);
+            }
+            stats[exponent_code(qb, e)] += 1;
+            stats[ST_TOTAL] += 1;
+            if (in_cls == CLS_ZERO) stats[ST_ZERO_IN] += 1;
+            if (in_cls == CLS_NAN) stats[ST_NAN] += 1;
+            if (in_cls == CLS_INF) stats[ST_INF_IN] += 1;
+            if (was_den) stats[ST_DENORMAL] += 1;
+            if (in_cls == CLS_FINITE && q_zero) stats[ST_UNDERFLOW] += 1;
+            if ((in_cls == CLS_FINITE || in_cls == CLS_ZERO) && q_inf) stats[ST_OVERFLOW] += 1;
+        }
+}
+
+/* ------------------------------------------------------------------------------------------ */
 /* Contractions (Section III-B, FMACS): exact products summed in fp64 in plain k order, with    */
 /* t = sum |a||b| beside each output for the accumulation-error bound.                          */
 /* Matrices are fp32, row-major with a leading dimension; trans != 0 reads the stored matrix    */
@@ -309,6 +528,51 @@ void oracle_gemm_sampled(const float *A, int64_t lda, int transA, const float *B
 #pragma omp parallel for schedule(static)
     for (int64_t s = 0; s < nsamp; ++s)
         dot_ab(A, lda, transA, B, ldb, transB, K, ii[s], jj[s], &c[s], t ? &t[s] : NULL);
+}
+
+/* ------------------------------------------------------------------------------------------ */
+/* FMAC-8 (Algorithm 1): dot product with a format-precision accumulator that is emptied into   */
+/* a single-precision master accumulator before every eighth FMAC, and once more at the end;    */
+/* the result is rounded to the format.  "+" on the master accumulator is fp32 addition.        */
+/* ------------------------------------------------------------------------------------------ */
+static uint32_t f32_add_bits(uint32_t a, uint32_t b) { return oracle_add_round_bits(a, b, 8, 23, 1); }
+
+static uint32_t fmac8_dot(const float *A, int64_t lda, int transA, const float *B, int64_t ldb, int transB,
+                          int64_t K, int64_t i, int64_t j, int e, int m, int keep_denormals, int group) {
+    uint32_t master = 0, small = 0; /* A^(32) = 0, a^(16) = 0 */
+    for (int64_t k = 0; k < K; ++k) {
+        if (k % group == 0) {
+            master = f32_add_bits(master, small);
+            small = 0;
+        }
+        float x = transA ? A[k * lda + i] : A[i * lda + k];
+        float y = transB ? B[j * ldb + k] : B[k * ldb + j];
+        uint32_t xb, yb;
+        memcpy(&xb, &x, 4);
+        memcpy(&yb, &y, 4);
+        small = oracle_fmac_bits(small, xb, yb, e, m, keep_denormals);
+    }
+    master = f32_add_bits(master, small);
+    return oracle_quantize_bits(master, e, m, keep_denormals, NULL);
+}
+
+/* C (M x N, dense row-major fp32 words) = FMAC-8 product of op(A) (M x K) and op(B) (K x N).   */
+/* group is the number of consecutive FMACs (8 in the paper).                                   */
+void oracle_fmac8_gemm(const float *A, int64_t lda, int transA, const float *B, int64_t ldb, int transB,
+                       int64_t M, int64_t N, int64_t K, int e, int m, int keep_denormals, int group,
+                       uint32_t *C) {
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < M; ++i)
+        for (int64_t j = 0; j < N; ++j)
+            C[i * N + j] = fmac8_dot(A, lda, transA, B, ldb, transB, K, i, j, e, m, keep_denormals, group);
+}
+
+void oracle_fmac8_gemm_sampled(const float *A, int64_t lda, int transA, const float *B, int64_t ldb, int transB,
+                               int64_t K, int e, int m, int keep_denormals, int group, const int64_t *ii,
+                               const int64_t *jj, int64_t nsamp, uint32_t *c) {
+#pragma omp parallel for schedule(static)
+    for (int64_t s = 0; s < nsamp; ++s)
+        c[s] = fmac8_dot(A, lda, transA, B, ldb, transB, K, ii[s], jj[s], e, m, keep_denormals, group);
 }
 
 /* ------------------------------------------------------------------------------------------ */
