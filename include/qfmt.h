@@ -106,6 +106,35 @@ int qfmt_quantize_stats_transpose(const float* d_in, float* d_out, int64_t batch
                                   void* stream);
 
 /*
+ * Output of a layer as Section IV-A's worked example computes it, Y = R(R(acc) + R(B)): `acc` is
+ * the matrix product of the layer (what qfmt_gemm or qfmt_conv wrote: rows x cols, row-major,
+ * leading dimension ld_acc), `bias` has one entry per column.  Each acc element and each bias
+ * entry is multiplied by fmt->loss_scale and rounded to the format exactly as
+ * qfmt_quantize_stats does; the two rounded terms are added without error and the sum is rounded
+ * once more.  One pass over memory instead of three (round, add, round).
+ *
+ *   d_acc    device, 4-byte aligned; rows x cols floats with leading dimension ld_acc >= cols
+ *   d_bias   device, cols floats (the raw fp32 bias; it is rounded inside the call)
+ *   d_out    device, rows x cols with leading dimension ld_out >= cols; may equal d_acc when
+ *            ld_out == ld_acc (in place); other overlap is an error the library cannot detect.
+ *            16-byte aligned pointers with cols, ld_acc, ld_out multiples of 4 select the
+ *            128-bit path, anything else a scalar path.
+ *   d_stats  device or NULL: statistics of the OUTPUT tensor Y, in which the exact sum
+ *            R(acc) + R(B) plays the part the input plays in qfmt_quantize_stats: n_zero_in
+ *            counts sums that are exactly zero, n_underflow nonzero sums that end as zero (only
+ *            possible with denormals flushed), n_overflow finite sums that end as +-inf,
+ *            n_inf_in / n_nan sums that are infinite / NaN (inf - inf included).
+ *   accumulate  as in qfmt_quantize_stats
+ * A zero sum is -0 only if both terms are -0; any NaN comes out as the positive quiet NaN.
+ * Requires m <= 10 (QFMT_ERR_BAD_FORMAT otherwise): the sum is formed by one fp32 addition, which
+ * for such formats is exact or harmless to the final rounding.  rows = 0 or cols = 0 is valid.
+ * Errors: QFMT_ERR_BAD_FORMAT, QFMT_ERR_BAD_ARG, QFMT_ERR_UNSUPPORTED_ARCH, QFMT_ERR_CUDA.
+ */
+int qfmt_bias_quantize_stats(const float* d_acc, int64_t ld_acc, const float* d_bias, float* d_out, int64_t ld_out,
+                             int64_t rows, int64_t cols, const qfmt_format_t* fmt, qfmt_stats_t* d_stats,
+                             int accumulate, void* stream);
+
+/*
  * The same operation on HOST buffers: copies h_in to the device, runs the kernel, copies the
  * rounded tensor (if h_out != NULL) and the statistics (if h_stats != NULL) back, and
  * SYNCHRONISES the stream before returning.  The caller lends device scratch:
@@ -162,6 +191,34 @@ typedef struct {
 int qfmt_gemm(const qfmt_matrix_t* A, const qfmt_matrix_t* B, float* d_C, int64_t ldc,
               const qfmt_format_t* fmt, void* d_workspace, size_t workspace_bytes, void* stream);
 size_t qfmt_gemm_workspace_bytes(const qfmt_matrix_t* A, const qfmt_matrix_t* B);
+
+/*
+ * C = op(A) op(B) with FMAC-8 accumulation (Algorithm 1), for hardware that only offers the FMAC
+ * instruction of Section III-B, a16 = round(a16 + x16 * y16) (one rounding, to the 16-bit format).
+ * Every output is computed as the algorithm states: a format-precision accumulator takes eight
+ * consecutive FMACs (k = 0..7, 8..15, ...), is added to a single-precision master accumulator
+ * with an fp32 addition and restarts from zero; after the last (possibly shorter) group the master
+ * accumulator is rounded to the format.  So, unlike qfmt_gemm, the result is fully specified:
+ * C holds format values and is bit-exact against the definition.
+ *
+ *   A, B     as for qfmt_gemm (operands already hold values of the format; not re-rounded), but
+ *            only 4-byte alignment is needed and any leading dimension >= the stored row length
+ *   d_C      device, M x N floats, leading dimension ldc >= N, 4-byte aligned
+ *   fmt      e <= 7 and m <= 10 (QFMT_ERR_BAD_FORMAT otherwise: the product of two values must be
+ *            exact and finite in fp32); fmt->denormals selects whether the small accumulator and
+ *            the result keep denormals or flush them; fmt->loss_scale is ignored
+ *   d_stats  device or NULL: statistics of the OUTPUT tensor (Table II of the paper reports the
+ *            denormal fraction of tensors produced this way), with the master accumulator in the
+ *            role of the input of qfmt_quantize_stats; accumulate as there
+ *   path     0 automatic; 1 the general kernel (integer/fp32 emulation of the FMAC on the ALUs);
+ *            2 the binary16 kernel (1/5/10 only, else QFMT_ERR_BAD_FORMAT), where the FMAC is the
+ *            GPU's own half-precision fused multiply-add.  Both give the same bits.
+ * Plain-ALU work: no tensor-core instruction rounds its accumulator to 11 bits per product.
+ * M = 0 or N = 0 is a no-op; K = 0 writes +0.  NaN results are the positive quiet NaN.
+ * Errors: QFMT_ERR_BAD_FORMAT, QFMT_ERR_BAD_ARG, QFMT_ERR_UNSUPPORTED_ARCH, QFMT_ERR_CUDA.
+ */
+int qfmt_gemm_fmac8(const qfmt_matrix_t* A, const qfmt_matrix_t* B, float* d_C, int64_t ldc,
+                    const qfmt_format_t* fmt, qfmt_stats_t* d_stats, int accumulate, int path, void* stream);
 
 /*
  * Tuning and test control (no counterpart in the paper): which kernel dense products run on.

@@ -76,6 +76,9 @@ def lib() -> ctypes.CDLL:
         L.qfmt_quantize_stats.restype = ci
         L.qfmt_quantize_stats_transpose.argtypes = [vp, vp, ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, fmtp, vp, ci, vp]
         L.qfmt_quantize_stats_transpose.restype = ci
+        L.qfmt_bias_quantize_stats.argtypes = [vp, ctypes.c_int64, vp, vp, ctypes.c_int64, ctypes.c_int64,
+                                               ctypes.c_int64, fmtp, vp, ci, vp]
+        L.qfmt_bias_quantize_stats.restype = ci
         L.qfmt_quantize_stats_host.argtypes = [vp, vp, sz, fmtp, vp, vp, sz, vp]
         L.qfmt_quantize_stats_host.restype = ci
         L.qfmt_quantize_stats_host_work_bytes.argtypes = [sz]
@@ -99,6 +102,8 @@ def _bind_optional(L: ctypes.CDLL) -> None:
     L.qfmt_gemm.restype = ci
     L.qfmt_gemm_workspace_bytes.argtypes = [matp, matp]
     L.qfmt_gemm_workspace_bytes.restype = sz
+    L.qfmt_gemm_fmac8.argtypes = [matp, matp, vp, ctypes.c_int64, ctypes.POINTER(qfmt_format_t), vp, ci, ci, vp]
+    L.qfmt_gemm_fmac8.restype = ci
     L.qfmt_gemm_tile_policy.argtypes = [ci]
     L.qfmt_gemm_tile_policy.restype = ci
     L.qfmt_device_status.argtypes = [vp, vp]
@@ -158,6 +163,14 @@ def qfmt_quantize_stats_transpose(d_in, d_out, batch: int, rows: int, cols: int,
                                                _stream_handle(stream)), "qfmt_quantize_stats_transpose")
 
 
+def qfmt_bias_quantize_stats(d_acc, ld_acc: int, d_bias, d_out, ld_out: int, rows: int, cols: int,
+                             fmt: qfmt_format_t, d_stats=None, accumulate: int = 0, stream=None) -> None:
+    """Y = R(R(acc) + R(bias)) with the statistics of Y; see qfmt_bias_quantize_stats in include/qfmt.h."""
+    _check(lib().qfmt_bias_quantize_stats(_ptr(d_acc), int(ld_acc), _ptr(d_bias), _ptr(d_out), int(ld_out),
+                                          int(rows), int(cols), ctypes.byref(fmt), _ptr(d_stats), int(accumulate),
+                                          _stream_handle(stream)), "qfmt_bias_quantize_stats")
+
+
 def qfmt_quantize_stats_host_work_bytes(n: int) -> int:
     return int(lib().qfmt_quantize_stats_host_work_bytes(int(n)))
 
@@ -196,6 +209,13 @@ def qfmt_gemm(A: qfmt_matrix_t, B: qfmt_matrix_t, d_C, ldc: int, fmt: qfmt_forma
     """C = op(A) op(B), exact products, fp32 accumulation; see qfmt_gemm in include/qfmt.h."""
     _check(lib().qfmt_gemm(ctypes.byref(A), ctypes.byref(B), _ptr(d_C), int(ldc), ctypes.byref(fmt),
                            _ptr(d_workspace), int(workspace_bytes), _stream_handle(stream)), "qfmt_gemm")
+
+
+def qfmt_gemm_fmac8(A: qfmt_matrix_t, B: qfmt_matrix_t, d_C, ldc: int, fmt: qfmt_format_t, d_stats=None,
+                    accumulate: int = 0, path: int = 0, stream=None) -> None:
+    """C = op(A) op(B) with FMAC-8 accumulation (Algorithm 1); see qfmt_gemm_fmac8 in include/qfmt.h."""
+    _check(lib().qfmt_gemm_fmac8(ctypes.byref(A), ctypes.byref(B), _ptr(d_C), int(ldc), ctypes.byref(fmt),
+                                 _ptr(d_stats), int(accumulate), int(path), _stream_handle(stream)), "qfmt_gemm_fmac8")
 
 
 def qfmt_device_status(d_workspace, stream=None) -> int:

@@ -26,69 +26,10 @@
 #include <stdint.h>
 
 #include "common.cuh"
+#include "round.cuh"
 
 namespace qfmt {
 namespace {
-
-struct QuantParams {
-    uint32_t drop;         // 23 - m: mantissa bits removed from a normal value
-    uint32_t round_add;    // 2^(drop-1) - 1, or 0 when drop == 0
-    uint32_t lsb_mask;     // 1 when drop > 0 (adds the kept LSB: ties go to even)
-    uint32_t keep_mask;    // ~(2^drop - 1)
-    uint32_t min_normal;   // fp32 bits of 2^E_min
-    uint32_t magic;        // fp32 bits of 2^(E_min - m + 23)
-    int32_t code_off;      // 127 - bias: fp32 exponent field minus this = stored exponent field
-    int32_t top;           // 2^e - 1, the inf/NaN exponent field
-    uint32_t keep_denormals;
-    float scale;
-};
-
-// Extra bins after the regular exponent fields 1 .. top-1.
-enum : int { kBinZeroIn = 1, kBinRoundedToZero, kBinDenormal, kBinOverflow, kBinInfIn, kBinNanIn, kExtraBins };
-
-__device__ __forceinline__ float add_ieee(float a, float b) {
-    float r;
-    asm("add.rn.f32 %0, %1, %2;" : "=f"(r) : "f"(a), "f"(b));  // no .ftz: denormals honoured
-    return r;
-}
-__device__ __forceinline__ float sub_ieee(float a, float b) {
-    float r;
-    asm("sub.rn.f32 %0, %1, %2;" : "=f"(r) : "f"(a), "f"(b));
-    return r;
-}
-__device__ __forceinline__ float mul_ieee(float a, float b) {
-    float r;
-    asm("mul.rn.f32 %0, %1, %2;" : "=f"(r) : "f"(a), "f"(b));
-    return r;
-}
-
-// Rounds one element; returns the fp32 container bits and the element's bin.
-template <bool kScale>
-__device__ __forceinline__ uint32_t quantize_one(uint32_t xb, const QuantParams& p, int& bin) {
-    uint32_t yb = kScale ? __float_as_uint(mul_ieee(__uint_as_float(xb), p.scale)) : xb;
-    const uint32_t sign = xb & 0x80000000u;  // the scale is positive; a NaN's sign does not survive the multiply
-    const uint32_t a = yb & 0x7FFFFFFFu;
-    const uint32_t ax = xb & 0x7FFFFFFFu;
-    // at or above the smallest normal: round the word itself
-    const uint32_t qn = (a + p.round_add + ((a >> p.drop) & p.lsb_mask)) & p.keep_mask;
-    // below it: round onto multiples of 2^(E_min-m); cnt is that multiple
-    const float magic = __uint_as_float(p.magic);
-    const float sum = add_ieee(__uint_as_float(a), magic);
-    const uint32_t cnt = __float_as_uint(sum) - p.magic;
-    const uint32_t qd = __float_as_uint(sub_ieee(sum, magic));
-    uint32_t qa = (a < p.min_normal) ? qd : qn;
-    int code = (int)(qa >> 23) - p.code_off;
-    bin = code;
-    if (code >= p.top) {  // overflow, infinite or NaN
-        const bool is_nan = ax > 0x7F800000u;
-        qa = is_nan ? 0x7FC00000u : 0x7F800000u;
-        bin = p.top + (is_nan ? kBinNanIn : (ax == 0x7F800000u ? kBinInfIn : kBinOverflow));
-    } else if (code <= 0) {  // zero or denormal of the format
-        bin = p.top + (ax == 0u ? kBinZeroIn : (cnt == 0u ? kBinRoundedToZero : kBinDenormal));
-        if (!p.keep_denormals) qa = 0u;
-    }
-    return sign | qa;
-}
 
 __device__ __forceinline__ uint4 load_stream(const uint4* p) {
     uint4 v;
@@ -99,27 +40,6 @@ __device__ __forceinline__ uint4 load_stream(const uint4* p) {
 __device__ __forceinline__ void store_stream(uint4* p, const uint4& v) {
     asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};"
                  :: "l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
-}
-
-// Folds one bin's block total into the device record.
-__device__ __forceinline__ void merge_bin(qfmt_stats_t* st, const QuantParams& p, int bin, unsigned long long c) {
-    auto add = [](uint64_t* dst, unsigned long long v) { atomicAdd((unsigned long long*)dst, v); };
-    if (bin < p.top) {
-        add(&st->hist[bin], c);
-        return;
-    }
-    switch (bin - p.top) {
-        case kBinZeroIn: add(&st->hist[0], c); add(&st->n_zero_in, c); break;
-        case kBinRoundedToZero: add(&st->hist[0], c); add(&st->n_underflow, c); break;
-        case kBinDenormal:
-            add(&st->hist[0], c); add(&st->n_denormal, c);
-            if (!p.keep_denormals) add(&st->n_underflow, c);
-            break;
-        case kBinOverflow: add(&st->hist[p.top], c); add(&st->n_overflow, c); break;
-        case kBinInfIn: add(&st->hist[p.top], c); add(&st->n_inf_in, c); break;
-        case kBinNanIn: add(&st->hist[p.top], c); add(&st->n_nan, c); break;
-        default: break;
-    }
 }
 
 constexpr int kThreads = 512;
@@ -275,21 +195,142 @@ quantize_stats_transpose_kernel(const uint32_t* __restrict__ in, uint32_t* __res
     }
 }
 
-QuantParams make_params(const qfmt_format_t& f) {
-    QuantParams p;
-    const int bias = (1 << (f.e - 1)) - 1;
-    const int emin = 1 - bias;
-    p.drop = 23u - (uint32_t)f.m;
-    p.round_add = p.drop ? ((1u << (p.drop - 1)) - 1u) : 0u;
-    p.lsb_mask = p.drop ? 1u : 0u;
-    p.keep_mask = ~((1u << p.drop) - 1u);
-    p.min_normal = (uint32_t)(emin + 127) << 23;
-    p.magic = (uint32_t)(emin - f.m + 23 + 127) << 23;
-    p.code_off = 127 - bias;
-    p.top = (1 << f.e) - 1;
-    p.keep_denormals = f.denormals ? 1u : 0u;
-    p.scale = f.loss_scale;
-    return p;
+// Layer output of Section IV-A's worked example, Y = R(R(acc) + R(B)): the matrix product is
+// rounded, the (rounded) bias of its column is added, and the sum is rounded again, with the
+// statistics of Y taken in the same pass.  The sum of two format values is formed with one IEEE
+// fp32 add; for m <= 10 that add is either exact or so far from every grid and halfway point of
+// the format that rounding its result equals rounding the exact sum (when the add is inexact the
+// smaller term lies below 2^-12 of the larger one's last place).  The block first rounds the bias
+// vector into shared memory (or, for very wide matrices, each element rounds its own bias entry).
+// Vector kernel: rows of c4 = cols/4 128-bit vectors; each thread walks the flat vector index with
+// a fixed stride and keeps (row, column) per slot by adding the stride's quotient and remainder.
+template <bool kScale>
+__device__ __forceinline__ uint32_t bias_round_one(uint32_t acc, uint32_t rb, const QuantParams& p, int& bin) {
+    int unused;
+    const uint32_t ra = quantize_one<kScale>(acc, p, unused);
+    const uint32_t s = __float_as_uint(add_ieee(__uint_as_float(ra), __uint_as_float(rb)));
+    const uint32_t q = quantize_one<false>(s, p, bin);
+    // 1/8/m only: two finite terms whose fp32 sum is already infinite overflowed, they were not infinite
+    if (bin == p.top + kBinInfIn && (ra & 0x7FFFFFFFu) < 0x7F800000u && (rb & 0x7FFFFFFFu) < 0x7F800000u)
+        bin = p.top + kBinOverflow;
+    return q;
+}
+
+template <bool kStats, bool kScale, bool kSmemBias>
+__global__ void __launch_bounds__(kThreads)
+bias_quantize_stats_kernel(const uint32_t* acc, long long ld_acc, const uint32_t* __restrict__ bias, uint32_t* out,
+                           long long ld_out, unsigned long long rows, uint32_t c4, QuantParams p,
+                           qfmt_stats_t* __restrict__ stats) {
+    extern __shared__ uint32_t lane_hist[];  // [(top + kExtraBins)][32], then the rounded bias
+    const int nbins = p.top + kExtraBins;
+    const int lane = threadIdx.x & 31;
+    uint32_t* sbias = lane_hist + (kStats ? nbins * 32 : 0);
+    if (kStats) {
+        for (int i = threadIdx.x; i < nbins * 32; i += kThreads) lane_hist[i] = 0u;
+    }
+    if (kSmemBias) {
+        for (uint32_t j = threadIdx.x; j < c4 * 4u; j += kThreads) {
+            int unused;
+            sbias[j] = quantize_one<kScale>(bias[j], p, unused);
+        }
+    }
+    __syncthreads();
+    const unsigned long long n4 = rows * c4;
+    const unsigned long long stride = (unsigned long long)gridDim.x * (kThreads * kUnroll);
+    const unsigned long long dq = stride / c4;
+    const uint32_t dr = (uint32_t)(stride % c4);
+    unsigned long long row[kUnroll];
+    uint32_t col[kUnroll];
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+        const unsigned long long idx = (unsigned long long)blockIdx.x * (kThreads * kUnroll) + (unsigned long long)u * kThreads + threadIdx.x;
+        row[u] = idx / c4;
+        col[u] = (uint32_t)(idx % c4);
+    }
+    for (unsigned long long base = (unsigned long long)blockIdx.x * (kThreads * kUnroll); base < n4; base += stride) {
+        uint4 v[kUnroll];
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+            if (row[u] < rows) v[u] = load_stream(reinterpret_cast<const uint4*>(acc + row[u] * ld_acc) + col[u]);
+        }
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+            if (row[u] < rows) {
+                uint4 b;
+                if (kSmemBias) {
+                    b = reinterpret_cast<const uint4*>(sbias)[col[u]];
+                } else {
+                    const uint4 raw = reinterpret_cast<const uint4*>(bias)[col[u]];
+                    int unused;
+                    b.x = quantize_one<kScale>(raw.x, p, unused);
+                    b.y = quantize_one<kScale>(raw.y, p, unused);
+                    b.z = quantize_one<kScale>(raw.z, p, unused);
+                    b.w = quantize_one<kScale>(raw.w, p, unused);
+                }
+                int b0, b1, b2, b3;
+                uint4 q;
+                q.x = bias_round_one<kScale>(v[u].x, b.x, p, b0);
+                q.y = bias_round_one<kScale>(v[u].y, b.y, p, b1);
+                q.z = bias_round_one<kScale>(v[u].z, b.z, p, b2);
+                q.w = bias_round_one<kScale>(v[u].w, b.w, p, b3);
+                store_stream(reinterpret_cast<uint4*>(out + row[u] * ld_out) + col[u], q);
+                if (kStats) {
+                    atomicAdd(&lane_hist[b0 * 32 + lane], 1u);
+                    atomicAdd(&lane_hist[b1 * 32 + lane], 1u);
+                    atomicAdd(&lane_hist[b2 * 32 + lane], 1u);
+                    atomicAdd(&lane_hist[b3 * 32 + lane], 1u);
+                }
+            }
+            row[u] += dq;
+            col[u] += dr;
+            if (col[u] >= c4) {
+                col[u] -= c4;
+                row[u] += 1;
+            }
+        }
+    }
+    if (kStats) {
+        __syncthreads();
+        const int warp = threadIdx.x >> 5;
+        for (int b = warp + 1; b < nbins; b += kThreads / 32) {
+            const uint32_t c = __reduce_add_sync(0xFFFFFFFFu, lane_hist[b * 32 + lane]);
+            if (lane == 0 && c != 0u) merge_bin(stats, p, b, c);
+        }
+        if (blockIdx.x == 0 && threadIdx.x == 0) atomicAdd((unsigned long long*)&stats->n_total, n4 * 4ull);
+    }
+}
+
+// Any alignment and any column count: one element per thread per step, bias rounded per element.
+template <bool kStats, bool kScale>
+__global__ void __launch_bounds__(kThreads)
+bias_quantize_stats_scalar_kernel(const uint32_t* acc, long long ld_acc, const uint32_t* __restrict__ bias,
+                                  uint32_t* out, long long ld_out, unsigned long long rows, unsigned long long cols,
+                                  QuantParams p, qfmt_stats_t* __restrict__ stats) {
+    extern __shared__ uint32_t lane_hist[];
+    const int nbins = p.top + kExtraBins;
+    const int lane = threadIdx.x & 31;
+    if (kStats) {
+        for (int i = threadIdx.x; i < nbins * 32; i += kThreads) lane_hist[i] = 0u;
+        __syncthreads();
+    }
+    const unsigned long long n = rows * cols;
+    const unsigned long long stride = (unsigned long long)gridDim.x * kThreads;
+    for (unsigned long long i = (unsigned long long)blockIdx.x * kThreads + threadIdx.x; i < n; i += stride) {
+        const unsigned long long r = i / cols, c = i % cols;
+        int unused, b;
+        const uint32_t rb = quantize_one<kScale>(bias[c], p, unused);
+        out[r * ld_out + c] = bias_round_one<kScale>(acc[r * ld_acc + c], rb, p, b);
+        if (kStats) atomicAdd(&lane_hist[b * 32 + lane], 1u);
+    }
+    if (kStats) {
+        __syncthreads();
+        const int warp = threadIdx.x >> 5;
+        for (int b = warp + 1; b < nbins; b += kThreads / 32) {
+            const uint32_t c = __reduce_add_sync(0xFFFFFFFFu, lane_hist[b * 32 + lane]);
+            if (lane == 0 && c != 0u) merge_bin(stats, p, b, c);
+        }
+        if (blockIdx.x == 0 && threadIdx.x == 0 && n != 0ull) atomicAdd((unsigned long long*)&stats->n_total, n);
+    }
 }
 
 template <bool kOut, bool kStats, bool kScale>
@@ -397,6 +438,78 @@ int quantize_stats_transpose_device(const float* d_in, float* d_out, int64_t bat
     return QFMT_OK;
 }
 
+
+int bias_quantize_stats_device(const float* d_acc, int64_t ld_acc, const float* d_bias, float* d_out, int64_t ld_out,
+                               int64_t rows, int64_t cols, const qfmt_format_t* fmt, qfmt_stats_t* d_stats,
+                               int accumulate, cudaStream_t stream) {
+    int rc = validate_format(fmt);
+    if (rc != QFMT_OK) return rc;
+    if (fmt->m > 10) return QFMT_ERR_BAD_FORMAT;  // the one-add sum is only then a single rounding
+    if (accumulate != 0 && accumulate != 1) return QFMT_ERR_BAD_ARG;
+    if (rows < 0 || cols < 0 || rows > ((int64_t)1 << 40) || cols > 0x7FFFFFFF) return QFMT_ERR_BAD_ARG;
+    const unsigned long long n = (unsigned long long)rows * (unsigned long long)cols;
+    if (n > (1ull << 40)) return QFMT_ERR_BAD_ARG;
+    if (n != 0 && (d_acc == nullptr || d_bias == nullptr || d_out == nullptr)) return QFMT_ERR_BAD_ARG;
+    if (n != 0 && (ld_acc < cols || ld_out < cols)) return QFMT_ERR_BAD_ARG;
+    if ((reinterpret_cast<uintptr_t>(d_acc) & 3u) || (reinterpret_cast<uintptr_t>(d_out) & 3u) ||
+        (reinterpret_cast<uintptr_t>(d_bias) & 3u) || (reinterpret_cast<uintptr_t>(d_stats) & 7u))
+        return QFMT_ERR_BAD_ARG;
+    DeviceInfo dev;
+    rc = current_device(&dev);
+    if (rc != QFMT_OK) return rc;
+    if (d_stats != nullptr && accumulate == 0) QFMT_CUDA_TRY(cudaMemsetAsync(d_stats, 0, sizeof(qfmt_stats_t), stream));
+    if (n == 0) return QFMT_OK;
+
+    const QuantParams p = make_params(*fmt);
+    const uint32_t* acc = reinterpret_cast<const uint32_t*>(d_acc);
+    const uint32_t* bias = reinterpret_cast<const uint32_t*>(d_bias);
+    uint32_t* out = reinterpret_cast<uint32_t*>(d_out);
+    const bool has_stats = d_stats != nullptr, has_scale = fmt->loss_scale != 1.0f;
+    const size_t hist_bytes = has_stats ? (size_t)(p.top + kExtraBins) * 32 * sizeof(uint32_t) : 0;
+    const bool vec = (cols % 4 == 0) && (ld_acc % 4 == 0) && (ld_out % 4 == 0) &&
+                     !((reinterpret_cast<uintptr_t>(d_acc) | reinterpret_cast<uintptr_t>(d_out) |
+                        reinterpret_cast<uintptr_t>(d_bias)) & 15u);
+    cudaError_t err = cudaSuccess;
+    if (vec) {
+        const uint32_t c4 = (uint32_t)(cols / 4);
+        const bool smem_bias = (size_t)cols * 4 <= 64 * 1024;
+        const size_t smem = hist_bytes + (smem_bias ? (size_t)cols * 4 : 0);
+        const unsigned long long per_block = (unsigned long long)kThreads * kUnroll;
+        unsigned long long want = ((unsigned long long)rows * c4 + per_block - 1) / per_block;
+        const unsigned long long cap = (unsigned long long)dev.sm_count * (smem > 36 * 1024 ? 2 : 3);
+        if (want > cap) want = cap;
+#define QFMT_BLAUNCH(S, C, B)                                                                                     \
+    do {                                                                                                          \
+        auto kern = bias_quantize_stats_kernel<S, C, B>;                                                          \
+        if (smem > 48 * 1024) err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
+        if (err == cudaSuccess)                                                                                   \
+            kern<<<(unsigned)want, kThreads, smem, stream>>>(acc, (long long)ld_acc, bias, out, (long long)ld_out, \
+                                                             (unsigned long long)rows, c4, p, d_stats);           \
+    } while (0)
+        if (has_stats) {
+            if (has_scale) { if (smem_bias) QFMT_BLAUNCH(true, true, true); else QFMT_BLAUNCH(true, true, false); }
+            else { if (smem_bias) QFMT_BLAUNCH(true, false, true); else QFMT_BLAUNCH(true, false, false); }
+        } else {
+            if (has_scale) { if (smem_bias) QFMT_BLAUNCH(false, true, true); else QFMT_BLAUNCH(false, true, false); }
+            else { if (smem_bias) QFMT_BLAUNCH(false, false, true); else QFMT_BLAUNCH(false, false, false); }
+        }
+#undef QFMT_BLAUNCH
+    } else {
+        unsigned long long want = (n + kThreads - 1) / kThreads;
+        const unsigned long long cap = (unsigned long long)dev.sm_count * 4;
+        if (want > cap) want = cap;
+#define QFMT_BSLAUNCH(S, C)                                                                                        \
+    bias_quantize_stats_scalar_kernel<S, C><<<(unsigned)want, kThreads, hist_bytes, stream>>>(                     \
+        acc, (long long)ld_acc, bias, out, (long long)ld_out, (unsigned long long)rows, (unsigned long long)cols, p, d_stats)
+        if (has_stats) { if (has_scale) QFMT_BSLAUNCH(true, true); else QFMT_BSLAUNCH(true, false); }
+        else { if (has_scale) QFMT_BSLAUNCH(false, true); else QFMT_BSLAUNCH(false, false); }
+#undef QFMT_BSLAUNCH
+    }
+    QFMT_CUDA_TRY(err);
+    QFMT_CUDA_TRY(cudaGetLastError());
+    return QFMT_OK;
+}
+
 }  // namespace qfmt
 
 extern "C" int qfmt_quantize_stats(const float* d_in, float* d_out, size_t n, const qfmt_format_t* fmt,
@@ -433,4 +546,11 @@ extern "C" int qfmt_quantize_stats_host(const float* h_in, float* h_out, size_t 
     if (h_stats) QFMT_CUDA_TRY(cudaMemcpyAsync(h_stats, d_stats, sizeof(qfmt_stats_t), cudaMemcpyDeviceToHost, stream));
     QFMT_CUDA_TRY(cudaStreamSynchronize(stream));
     return QFMT_OK;
+}
+
+extern "C" int qfmt_bias_quantize_stats(const float* d_acc, int64_t ld_acc, const float* d_bias, float* d_out,
+                                        int64_t ld_out, int64_t rows, int64_t cols, const qfmt_format_t* fmt,
+                                        qfmt_stats_t* d_stats, int accumulate, void* stream) {
+    return qfmt::bias_quantize_stats_device(d_acc, ld_acc, d_bias, d_out, ld_out, rows, cols, fmt, d_stats, accumulate,
+                                            (cudaStream_t)stream);
 }
