@@ -67,7 +67,7 @@ def _L() -> ctypes.CDLL:
         lib.oracle_fmac_bits.restype = u32
         lib.oracle_bias_quantize_stats.argtypes = [vp, i64, i64, i64, vp, vp, i64, i32, i32, i32, u32, vp]
         lib.oracle_bias_quantize_stats.restype = None
-        lib.oracle_fmac8_gemm.argtypes = [vp, i64, i32, vp, i64, i32, i64, i64, i64, i32, i32, i32, i32, vp]
+        lib.oracle_fmac8_gemm.argtypes = [vp, i64, i32, vp, i64, i32, i64, i64, i64, i32, i32, i32, i32, vp, vp]
         lib.oracle_fmac8_gemm.restype = None
         lib.oracle_fmac8_gemm_sampled.argtypes = [vp, i64, i32, vp, i64, i32, i64, i32, i32, i32, i32, vp, vp,
                                                   i64, vp]
@@ -201,8 +201,9 @@ def _check_narrow(a: np.ndarray) -> None:
 
 
 def fmac8_gemm(A: np.ndarray, B: np.ndarray, e: int, m: int, denormals: int = 1, transA: bool = False,
-               transB: bool = False, group: int = 8) -> np.ndarray:
-    """Algorithm 1 for every output of op(A) op(B); returns the rounded results as float32."""
+               transB: bool = False, group: int = 8, want_master: bool = False):
+    """Algorithm 1 for every output of op(A) op(B); returns the rounded results as float32
+    (and, if asked, the fp32 master accumulators before the final rounding)."""
     A, B = _mat(A), _mat(B)
     _check_narrow(A)
     _check_narrow(B)
@@ -210,9 +211,11 @@ def fmac8_gemm(A: np.ndarray, B: np.ndarray, e: int, m: int, denormals: int = 1,
     K2, N = (B.shape[1], B.shape[0]) if transB else B.shape
     assert K == K2
     C = np.empty((M, N), dtype=np.uint32)
+    master = np.empty((M, N), dtype=np.uint32) if want_master else None
     _L().oracle_fmac8_gemm(A.ctypes.data, A.shape[1], int(transA), B.ctypes.data, B.shape[1], int(transB),
-                           M, N, K, e, m, int(denormals), group, C.ctypes.data)
-    return C.view(np.float32)
+                           M, N, K, e, m, int(denormals), group, C.ctypes.data,
+                           master.ctypes.data if want_master else None)
+    return (C.view(np.float32), master.view(np.float32)) if want_master else C.view(np.float32)
 
 
 def fmac8_gemm_sampled(A: np.ndarray, B: np.ndarray, ii: np.ndarray, jj: np.ndarray, e: int, m: int,

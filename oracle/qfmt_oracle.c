@@ -538,7 +538,8 @@ void oracle_gemm_sampled(const float *A, int64_t lda, int transA, const float *B
 static uint32_t f32_add_bits(uint32_t a, uint32_t b) { return oracle_add_round_bits(a, b, 8, 23, 1); }
 
 static uint32_t fmac8_dot(const float *A, int64_t lda, int transA, const float *B, int64_t ldb, int transB,
-                          int64_t K, int64_t i, int64_t j, int e, int m, int keep_denormals, int group) {
+                          int64_t K, int64_t i, int64_t j, int e, int m, int keep_denormals, int group,
+                          uint32_t *master_out) {
     uint32_t master = 0, small = 0; /* A^(32) = 0, a^(16) = 0 */
     for (int64_t k = 0; k < K; ++k) {
         if (k % group == 0) {
@@ -553,18 +554,21 @@ static uint32_t fmac8_dot(const float *A, int64_t lda, int transA, const float *
         small = oracle_fmac_bits(small, xb, yb, e, m, keep_denormals);
     }
     master = f32_add_bits(master, small);
+    if (master_out) *master_out = master; /* A^(32) before the final rounding */
     return oracle_quantize_bits(master, e, m, keep_denormals, NULL);
 }
 
 /* C (M x N, dense row-major fp32 words) = FMAC-8 product of op(A) (M x K) and op(B) (K x N).   */
-/* group is the number of consecutive FMACs (8 in the paper).                                   */
+/* group is the number of consecutive FMACs (8 in the paper).  master (may be NULL) receives     */
+/* the master accumulators before the final rounding.                                           */
 void oracle_fmac8_gemm(const float *A, int64_t lda, int transA, const float *B, int64_t ldb, int transB,
                        int64_t M, int64_t N, int64_t K, int e, int m, int keep_denormals, int group,
-                       uint32_t *C) {
+                       uint32_t *C, uint32_t *master) {
 #pragma omp parallel for schedule(static)
     for (int64_t i = 0; i < M; ++i)
         for (int64_t j = 0; j < N; ++j)
-            C[i * N + j] = fmac8_dot(A, lda, transA, B, ldb, transB, K, i, j, e, m, keep_denormals, group);
+            C[i * N + j] = fmac8_dot(A, lda, transA, B, ldb, transB, K, i, j, e, m, keep_denormals, group,
+                                     master ? &master[i * N + j] : NULL);
 }
 
 void oracle_fmac8_gemm_sampled(const float *A, int64_t lda, int transA, const float *B, int64_t ldb, int transB,
@@ -572,7 +576,7 @@ void oracle_fmac8_gemm_sampled(const float *A, int64_t lda, int transA, const fl
                                const int64_t *jj, int64_t nsamp, uint32_t *c) {
 #pragma omp parallel for schedule(static)
     for (int64_t s = 0; s < nsamp; ++s)
-        c[s] = fmac8_dot(A, lda, transA, B, ldb, transB, K, ii[s], jj[s], e, m, keep_denormals, group);
+        c[s] = fmac8_dot(A, lda, transA, B, ldb, transB, K, ii[s], jj[s], e, m, keep_denormals, group, NULL);
 }
 
 /* ------------------------------------------------------------------------------------------ */

@@ -1,0 +1,352 @@
+// FMAC-8 matrix product (Algorithm 1): every output is a dot product accumulated with FMAC
+// instructions, a16 = round(a16 + x16 * y16) with ONE rounding to the 16-bit format
+// (Section III-B), in groups of eight; each group's sum is added to a single-precision master
+// accumulator with an fp32 add and the small accumulator restarts from zero; the master
+// accumulator is rounded to the format at the end.  Statistics of the output tensor are taken
+// in the same kernel.
+//
+// No tensor core implements "round the accumulator to 11 bits after every product", so this is
+// plain-ALU work (a few dozen integer/float instructions per multiply-add, or one HFMA2 per two
+// multiply-adds for binary16, which the ALUs implement natively); operand traffic is negligible
+// beside it.  Two kernels:
+//   * fmac8_kernel, any format with e <= 7 and m <= 10.  The product of two format values is
+//     exact in fp32 (at most 22 significant bits, exponent within fp32's range for e <= 7).
+//     The exact sum a + x*y is rounded ONCE by forming it to 24 bits with round-to-odd (the two
+//     directed fp32 additions; when they differ the one with an odd last bit is taken) and then
+//     rounding to m+1 bits to nearest-even: a sticky last bit 13 or more places below the target's
+//     last place cannot create or hide a tie.
+//   * fmac8_f16_kernel, 1/5/10: fma.rn.f16x2 is this very operation for IEEE binary16 with
+//     denormals; flushing formats clear results below 2^-14 afterwards.
+// Both keep a 128 x 64 (resp. 128 x 128) tile of outputs per block in registers and stream
+// 32-deep slices of the operands through shared memory.
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "common.cuh"
+#include "round.cuh"
+
+namespace qfmt {
+namespace {
+
+constexpr int kFmThreads = 256;
+constexpr int kFmBK = 32;    // K elements per shared-memory slice: four groups of eight
+constexpr int kGroup = 8;    // FMACs per group (Algorithm 1)
+
+struct FmacParams {
+    const float* A;
+    const float* B;
+    float* C;
+    long long lda, ldb, ldc;
+    int M, N, K;
+    int transA, transB;
+    int vec_store;  // C rows 16-byte aligned
+};
+
+// a + prod rounded to 24 bits with round-to-odd (exact sums come back unchanged; an exact
+// cancellation gives +0 as round-to-nearest does)
+__device__ __forceinline__ uint32_t add_to_odd(float a, float prod) {
+    float lo, hi;
+    asm("add.rm.f32 %0, %1, %2;" : "=f"(lo) : "f"(a), "f"(prod));
+    asm("add.rp.f32 %0, %1, %2;" : "=f"(hi) : "f"(a), "f"(prod));
+    const uint32_t l = __float_as_uint(lo), h = __float_as_uint(hi);
+    return (lo == hi || (h & 1u)) ? h : l;
+}
+
+// Rounds a 24-bit intermediate to the format (no statistics): the small accumulator's rounding.
+__device__ __forceinline__ float round_small(uint32_t s, const QuantParams& p, uint32_t inf_bits) {
+    const uint32_t sign = s & 0x80000000u, a = s & 0x7FFFFFFFu;
+    const uint32_t qn = (a + p.round_add + ((a >> p.drop) & 1u)) & p.keep_mask;
+    const float magic = __uint_as_float(p.magic);
+    const uint32_t qd = __float_as_uint(sub_ieee(add_ieee(__uint_as_float(a), magic), magic));
+    uint32_t q = a < p.min_normal ? qd : qn;
+    if (q >= inf_bits) q = 0x7F800000u;
+    if (!p.keep_denormals && q < p.min_normal) q = 0u;
+    return __uint_as_float(a > 0x7F800000u ? 0x7FC00000u : (sign | q));
+}
+
+__device__ __forceinline__ float fmac(float acc, float x, float y, const QuantParams& p, uint32_t inf_bits) {
+    return round_small(add_to_odd(acc, mul_ieee(x, y)), p, inf_bits);
+}
+
+// One 32-deep slice of op(A) (rows m0.., kBM of them) into shared memory as [k][m]; elements
+// outside the matrix are zero (a zero product leaves a format-valued accumulator unchanged).
+template <int kRows, int kLd, typename T, typename F>
+__device__ __forceinline__ void load_slice(T (*dst)[kLd], const float* src, long long ld, int trans_k_major,
+                                           int r0, int rmax, int k0, int kmax, F convert) {
+    // trans_k_major != 0: k is the contiguous index of the stored matrix
+    for (int idx = threadIdx.x; idx < kRows * kFmBK; idx += kFmThreads) {
+        int r, k;
+        if (trans_k_major) { k = idx % kFmBK; r = idx / kFmBK; }
+        else { r = idx % kRows; k = idx / kRows; }
+        float v = 0.0f;
+        if (r0 + r < rmax && k0 + k < kmax)
+            v = trans_k_major ? src[(long long)(r0 + r) * ld + (k0 + k)] : src[(long long)(k0 + k) * ld + (r0 + r)];
+        dst[k][r] = convert(v);
+    }
+}
+
+// Rounds the master accumulators of one thread's rows x cols patch, stores them and counts.
+template <bool kStats, int kTM, int kTN>
+__device__ __forceinline__ void store_patch(const FmacParams& g, const QuantParams& p, const float (&master)[kTM][kTN],
+                                            int row0, int col0, uint32_t* lane_hist, int lane) {
+#pragma unroll
+    for (int i = 0; i < kTM; ++i) {
+        const int row = row0 + i;
+        if (row >= g.M) break;
+        uint32_t q[kTN];
+#pragma unroll
+        for (int j = 0; j < kTN; ++j) {
+            int bin;
+            q[j] = quantize_one<false>(__float_as_uint(master[i][j]), p, bin);
+            if (kStats && col0 + j < g.N) atomicAdd(&lane_hist[bin * 32 + lane], 1u);
+        }
+        float* dst = g.C + (long long)row * g.ldc + col0;
+#pragma unroll
+        for (int j = 0; j < kTN; j += 4) {
+            if (g.vec_store && col0 + j + 3 < g.N) {
+                *reinterpret_cast<uint4*>(dst + j) = make_uint4(q[j], q[j + 1], q[j + 2], q[j + 3]);
+            } else {
+#pragma unroll
+                for (int jj = j; jj < j + 4; ++jj)
+                    if (col0 + jj < g.N) dst[jj] = __uint_as_float(q[jj]);
+            }
+        }
+    }
+}
+
+template <bool kStats>
+__device__ __forceinline__ void merge_block_hist(qfmt_stats_t* stats, const QuantParams& p, uint32_t* lane_hist,
+                                                 int nbins, unsigned long long n_total) {
+    if (!kStats) return;
+    __syncthreads();
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int b = warp + 1; b < nbins; b += kFmThreads / 32) {
+        const uint32_t c = __reduce_add_sync(0xFFFFFFFFu, lane_hist[b * 32 + lane]);
+        if (lane == 0 && c != 0u) merge_bin(stats, p, b, c);
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0 && n_total != 0ull)
+        atomicAdd((unsigned long long*)&stats->n_total, n_total);
+}
+
+// ---- any format with e <= 7, m <= 10 --------------------------------------------------------
+constexpr int kFmBM = 128, kFmBN = 64, kFmTM = 8, kFmTN = 4;
+
+template <bool kStats>
+__global__ void __launch_bounds__(kFmThreads, 2)
+fmac8_kernel(FmacParams g, QuantParams p, qfmt_stats_t* __restrict__ stats) {
+    __shared__ __align__(16) float As[kFmBK][kFmBM + 4];
+    __shared__ __align__(16) float Bs[kFmBK][kFmBN + 4];
+    extern __shared__ uint32_t lane_hist[];  // [(top + kExtraBins)][32]
+    const int nbins = p.top + kExtraBins;
+    const int lane = threadIdx.x & 31;
+    if (kStats) {
+        for (int i = threadIdx.x; i < nbins * 32; i += kFmThreads) lane_hist[i] = 0u;
+        __syncthreads();
+    }
+    const uint32_t inf_bits = (uint32_t)(p.top + p.code_off) << 23;  // fp32 bits of 2^(E_max+1)
+    const int tx = threadIdx.x % 16, ty = threadIdx.x / 16;
+    const int tiles_n = (g.N + kFmBN - 1) / kFmBN, tiles_m = (g.M + kFmBM - 1) / kFmBM;
+    auto same = [](float v) { return v; };
+    for (long long tile = blockIdx.x; tile < (long long)tiles_m * tiles_n; tile += gridDim.x) {
+        const int m0 = (int)(tile / tiles_n) * kFmBM, n0 = (int)(tile % tiles_n) * kFmBN;
+        float master[kFmTM][kFmTN], small[kFmTM][kFmTN];
+#pragma unroll
+        for (int i = 0; i < kFmTM; ++i)
+#pragma unroll
+            for (int j = 0; j < kFmTN; ++j) master[i][j] = 0.0f, small[i][j] = 0.0f;
+        for (int k0 = 0; k0 < g.K; k0 += kFmBK) {
+            __syncthreads();  // the previous slice is no longer read
+            load_slice<kFmBM, kFmBM + 4>(As, g.A, g.lda, !g.transA, m0, g.M, k0, g.K, same);
+            load_slice<kFmBN, kFmBN + 4>(Bs, g.B, g.ldb, g.transB, n0, g.N, k0, g.K, same);
+            __syncthreads();
+            const int kmax = g.K - k0 < kFmBK ? g.K - k0 : kFmBK;
+#pragma unroll 1
+            for (int kg = 0; kg < kmax; kg += kGroup) {
+#pragma unroll
+                for (int kk = 0; kk < kGroup; ++kk) {
+                    const float4 a0 = *reinterpret_cast<const float4*>(&As[kg + kk][ty * kFmTM]);
+                    const float4 a1 = *reinterpret_cast<const float4*>(&As[kg + kk][ty * kFmTM + 4]);
+                    const float4 b0 = *reinterpret_cast<const float4*>(&Bs[kg + kk][tx * kFmTN]);
+                    const float a[kFmTM] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+                    const float b[kFmTN] = {b0.x, b0.y, b0.z, b0.w};
+#pragma unroll
+                    for (int i = 0; i < kFmTM; ++i)
+#pragma unroll
+                        for (int j = 0; j < kFmTN; ++j) small[i][j] = fmac(small[i][j], a[i], b[j], p, inf_bits);
+                }
+                // the group's sum moves to the master accumulator (fp32 addition)
+#pragma unroll
+                for (int i = 0; i < kFmTM; ++i)
+#pragma unroll
+                    for (int j = 0; j < kFmTN; ++j) {
+                        master[i][j] = add_ieee(master[i][j], small[i][j]);
+                        small[i][j] = 0.0f;
+                    }
+            }
+        }
+        store_patch<kStats, kFmTM, kFmTN>(g, p, master, m0 + ty * kFmTM, n0 + tx * kFmTN, lane_hist, lane);
+    }
+    merge_block_hist<kStats>(stats, p, lane_hist, nbins, (unsigned long long)g.M * (unsigned long long)g.N);
+}
+
+// ---- 1/5/10: the hardware's own half-precision FMA ------------------------------------------
+constexpr int kHfBM = 128, kHfBN = 128, kHfTM = 8, kHfTN = 8;
+
+__device__ __forceinline__ __half2 hfma2_ieee(__half2 a, __half2 b, __half2 c) {
+    uint32_t r;
+    asm("fma.rn.f16x2 %0, %1, %2, %3;"  // no .ftz: denormals honoured
+        : "=r"(r)
+        : "r"(*reinterpret_cast<uint32_t*>(&a)), "r"(*reinterpret_cast<uint32_t*>(&b)),
+          "r"(*reinterpret_cast<uint32_t*>(&c)));
+    return *reinterpret_cast<__half2*>(&r);
+}
+
+// clears the halves whose magnitude is below 2^-14 (0x0400), keeping their signs
+__device__ __forceinline__ __half2 flush_denormals2(__half2 v) {
+    const uint32_t u = *reinterpret_cast<uint32_t*>(&v);
+    const uint32_t mag = u & 0x7FFF7FFFu;
+    uint32_t keep = 0x80008000u;
+    if ((mag & 0xFFFFu) >= 0x0400u) keep |= 0x00007FFFu;
+    if ((mag >> 16) >= 0x0400u) keep |= 0x7FFF0000u;
+    const uint32_t r = u & keep;
+    return *reinterpret_cast<const __half2*>(&r);
+}
+
+template <bool kStats, bool kFlush>
+__global__ void __launch_bounds__(kFmThreads, 1)
+fmac8_f16_kernel(FmacParams g, QuantParams p, qfmt_stats_t* __restrict__ stats) {
+    __shared__ __align__(16) __half As[kFmBK][kHfBM + 8];
+    __shared__ __align__(16) __half Bs[kFmBK][kHfBN + 8];
+    extern __shared__ uint32_t lane_hist[];
+    const int nbins = p.top + kExtraBins;
+    const int lane = threadIdx.x & 31;
+    if (kStats) {
+        for (int i = threadIdx.x; i < nbins * 32; i += kFmThreads) lane_hist[i] = 0u;
+        __syncthreads();
+    }
+    const int tx = threadIdx.x % 16, ty = threadIdx.x / 16;
+    const int tiles_n = (g.N + kHfBN - 1) / kHfBN, tiles_m = (g.M + kHfBM - 1) / kHfBM;
+    auto to_half = [](float v) { return __float2half_rn(v); };  // exact: operands hold binary16 values
+    for (long long tile = blockIdx.x; tile < (long long)tiles_m * tiles_n; tile += gridDim.x) {
+        const int m0 = (int)(tile / tiles_n) * kHfBM, n0 = (int)(tile % tiles_n) * kHfBN;
+        float master[kHfTM][kHfTN];
+        __half2 small[kHfTM][kHfTN / 2];
+        const __half2 zero2 = __float2half2_rn(0.0f);
+#pragma unroll
+        for (int i = 0; i < kHfTM; ++i) {
+#pragma unroll
+            for (int j = 0; j < kHfTN; ++j) master[i][j] = 0.0f;
+#pragma unroll
+            for (int j = 0; j < kHfTN / 2; ++j) small[i][j] = zero2;
+        }
+        for (int k0 = 0; k0 < g.K; k0 += kFmBK) {
+            __syncthreads();
+            load_slice<kHfBM, kHfBM + 8>(As, g.A, g.lda, !g.transA, m0, g.M, k0, g.K, to_half);
+            load_slice<kHfBN, kHfBN + 8>(Bs, g.B, g.ldb, g.transB, n0, g.N, k0, g.K, to_half);
+            __syncthreads();
+            const int kmax = g.K - k0 < kFmBK ? g.K - k0 : kFmBK;
+#pragma unroll 1
+            for (int kg = 0; kg < kmax; kg += kGroup) {
+#pragma unroll
+                for (int kk = 0; kk < kGroup; ++kk) {
+                    const uint4 av = *reinterpret_cast<const uint4*>(&As[kg + kk][ty * kHfTM]);  // 8 halves
+                    const uint4 bv = *reinterpret_cast<const uint4*>(&Bs[kg + kk][tx * kHfTN]);
+                    const uint32_t aw[4] = {av.x, av.y, av.z, av.w};
+                    const uint32_t bw[4] = {bv.x, bv.y, bv.z, bv.w};
+#pragma unroll
+                    for (int i = 0; i < kHfTM; ++i) {
+                        // both halves = a_i
+                        const uint32_t dup = __byte_perm(aw[i >> 1], 0u, (i & 1) ? 0x3232 : 0x1010);
+                        const __half2 a2 = *reinterpret_cast<const __half2*>(&dup);
+#pragma unroll
+                        for (int j = 0; j < kHfTN / 2; ++j) {
+                            __half2 r = hfma2_ieee(a2, *reinterpret_cast<const __half2*>(&bw[j]), small[i][j]);
+                            small[i][j] = kFlush ? flush_denormals2(r) : r;
+                        }
+                    }
+                }
+#pragma unroll
+                for (int i = 0; i < kHfTM; ++i)
+#pragma unroll
+                    for (int j = 0; j < kHfTN / 2; ++j) {
+                        const float2 s = __half22float2(small[i][j]);
+                        master[i][2 * j] = add_ieee(master[i][2 * j], s.x);
+                        master[i][2 * j + 1] = add_ieee(master[i][2 * j + 1], s.y);
+                        small[i][j] = zero2;
+                    }
+            }
+        }
+        store_patch<kStats, kHfTM, kHfTN>(g, p, master, m0 + ty * kHfTM, n0 + tx * kHfTN, lane_hist, lane);
+    }
+    merge_block_hist<kStats>(stats, p, lane_hist, nbins, (unsigned long long)g.M * (unsigned long long)g.N);
+}
+
+}  // namespace
+
+int gemm_fmac8_device(const qfmt_matrix_t* A, const qfmt_matrix_t* B, float* d_C, int64_t ldc, const qfmt_format_t* fmt,
+                      qfmt_stats_t* d_stats, int accumulate, int path, cudaStream_t stream) {
+    int rc = validate_format(fmt);
+    if (rc != QFMT_OK) return rc;
+    if (fmt->m > 10 || fmt->e > 7) return QFMT_ERR_BAD_FORMAT;  // products must be exact and finite in fp32
+    if (A == nullptr || B == nullptr) return QFMT_ERR_BAD_ARG;
+    if (accumulate != 0 && accumulate != 1) return QFMT_ERR_BAD_ARG;
+    if (path < 0 || path > 2) return QFMT_ERR_BAD_ARG;
+    const int64_t M = A->trans ? A->cols : A->rows, K = A->trans ? A->rows : A->cols;
+    const int64_t Kb = B->trans ? B->cols : B->rows, N = B->trans ? B->rows : B->cols;
+    if (M < 0 || N < 0 || K < 0 || K != Kb || M > 0x7FFFFFFF || N > 0x7FFFFFFF || K > 0x7FFFFFFF) return QFMT_ERR_BAD_ARG;
+    if (A->ld < A->cols || B->ld < B->cols || ldc < N) return QFMT_ERR_BAD_ARG;
+    if ((M != 0 && K != 0 && A->ptr == nullptr) || (N != 0 && K != 0 && B->ptr == nullptr) ||
+        (M != 0 && N != 0 && d_C == nullptr))
+        return QFMT_ERR_BAD_ARG;
+    if ((reinterpret_cast<uintptr_t>(A->ptr) & 3u) || (reinterpret_cast<uintptr_t>(B->ptr) & 3u) ||
+        (reinterpret_cast<uintptr_t>(d_C) & 3u) || (reinterpret_cast<uintptr_t>(d_stats) & 7u))
+        return QFMT_ERR_BAD_ARG;
+    const bool native = fmt->e == 5 && fmt->m == 10;
+    if (path == 2 && !native) return QFMT_ERR_BAD_FORMAT;
+    DeviceInfo dev;
+    rc = current_device(&dev);
+    if (rc != QFMT_OK) return rc;
+    if (d_stats != nullptr && accumulate == 0) QFMT_CUDA_TRY(cudaMemsetAsync(d_stats, 0, sizeof(qfmt_stats_t), stream));
+    if (M == 0 || N == 0) return QFMT_OK;
+
+    qfmt_format_t f = *fmt;
+    f.loss_scale = 1.0f;  // operands are already scaled and rounded; nothing is scaled here
+    const QuantParams p = make_params(f);
+    FmacParams g;
+    g.A = A->ptr; g.B = B->ptr; g.C = d_C;
+    g.lda = A->ld; g.ldb = B->ld; g.ldc = ldc;
+    g.M = (int)M; g.N = (int)N; g.K = (int)K;
+    g.transA = A->trans ? 1 : 0; g.transB = B->trans ? 1 : 0;
+    g.vec_store = (ldc % 4 == 0) && !(reinterpret_cast<uintptr_t>(d_C) & 15u);
+    const bool has_stats = d_stats != nullptr;
+    const size_t smem = has_stats ? (size_t)(p.top + kExtraBins) * 32 * sizeof(uint32_t) : 0;
+    const bool use_native = native && path != 1;
+    if (use_native) {
+        const long long tiles = ((M + kHfBM - 1) / kHfBM) * ((N + kHfBN - 1) / kHfBN);
+        const unsigned grid = (unsigned)(tiles < dev.sm_count ? tiles : dev.sm_count);
+        const bool flush = fmt->denormals == 0;
+        if (has_stats) {
+            if (flush) fmac8_f16_kernel<true, true><<<grid, kFmThreads, smem, stream>>>(g, p, d_stats);
+            else fmac8_f16_kernel<true, false><<<grid, kFmThreads, smem, stream>>>(g, p, d_stats);
+        } else {
+            if (flush) fmac8_f16_kernel<false, true><<<grid, kFmThreads, 0, stream>>>(g, p, d_stats);
+            else fmac8_f16_kernel<false, false><<<grid, kFmThreads, 0, stream>>>(g, p, d_stats);
+        }
+    } else {
+        const long long tiles = ((M + kFmBM - 1) / kFmBM) * ((N + kFmBN - 1) / kFmBN);
+        const long long cap = (long long)dev.sm_count * 2;
+        const unsigned grid = (unsigned)(tiles < cap ? tiles : cap);
+        if (has_stats) fmac8_kernel<true><<<grid, kFmThreads, smem, stream>>>(g, p, d_stats);
+        else fmac8_kernel<false><<<grid, kFmThreads, 0, stream>>>(g, p, d_stats);
+    }
+    QFMT_CUDA_TRY(cudaGetLastError());
+    return QFMT_OK;
+}
+
+}  // namespace qfmt
+
+extern "C" int qfmt_gemm_fmac8(const qfmt_matrix_t* A, const qfmt_matrix_t* B, float* d_C, int64_t ldc,
+                               const qfmt_format_t* fmt, qfmt_stats_t* d_stats, int accumulate, int path, void* stream) {
+    return qfmt::gemm_fmac8_device(A, B, d_C, ldc, fmt, d_stats, accumulate, path, (cudaStream_t)stream);
+}
