@@ -43,30 +43,44 @@ struct FmacParams {
     int vec_store;  // C rows 16-byte aligned
 };
 
-// a + prod rounded to 24 bits with round-to-odd (exact sums come back unchanged; an exact
-// cancellation gives +0 as round-to-nearest does)
+// a + prod rounded to 24 bits with round-to-odd: the two directed sums are equal when the sum is
+// exact and adjacent fp32 numbers otherwise, exactly one of which has an odd last bit.  (An exact
+// cancellation gives -0 and +0; the even-looking -0 loses, so +0 comes out as in round-to-nearest.)
 __device__ __forceinline__ uint32_t add_to_odd(float a, float prod) {
     float lo, hi;
     asm("add.rm.f32 %0, %1, %2;" : "=f"(lo) : "f"(a), "f"(prod));
     asm("add.rp.f32 %0, %1, %2;" : "=f"(hi) : "f"(a), "f"(prod));
     const uint32_t l = __float_as_uint(lo), h = __float_as_uint(hi);
-    return (lo == hi || (h & 1u)) ? h : l;
+    return (l & 1u) ? l : h;
 }
 
-// Rounds a 24-bit intermediate to the format (no statistics): the small accumulator's rounding.
-__device__ __forceinline__ float round_small(uint32_t s, const QuantParams& p, uint32_t inf_bits) {
-    const uint32_t sign = s & 0x80000000u, a = s & 0x7FFFFFFFu;
-    const uint32_t qn = (a + p.round_add + ((a >> p.drop) & 1u)) & p.keep_mask;
-    const float magic = __uint_as_float(p.magic);
-    const uint32_t qd = __float_as_uint(sub_ieee(add_ieee(__uint_as_float(a), magic), magic));
-    uint32_t q = a < p.min_normal ? qd : qn;
-    if (q >= inf_bits) q = 0x7F800000u;
-    if (!p.keep_denormals && q < p.min_normal) q = 0u;
-    return __uint_as_float(a > 0x7F800000u ? 0x7FC00000u : (sign | q));
+struct SmallRound {
+    uint32_t min_normal;  // fp32 bits of 2^E_min
+    uint32_t inf_bits;    // fp32 bits of 2^(E_max+1)
+    uint32_t drop_exp;    // (23 - m) << 23
+};
+
+// Rounds a 24-bit intermediate to the format (the small accumulator's rounding; no statistics).
+// With C = +-2^(max(floor(log2|s|), E_min) + 23 - m), the fp32 sum s + C has its last place at the
+// format's quantum for s, so (s + C) - C is s rounded to nearest-even on the format's grid, normal
+// or denormal, sign included.  The exponent is capped at E_max+1 so that C stays finite; values
+// that reach 2^(E_max+1) are made infinite (or the quiet NaN) afterwards.
+template <bool kFlush>
+__device__ __forceinline__ float round_small(uint32_t s, const SmallRound& r) {
+    uint32_t ec = s & 0x7F800000u;
+    ec = ec < r.min_normal ? r.min_normal : ec;
+    ec = ec > r.inf_bits ? r.inf_bits : ec;
+    const float c = __uint_as_float((ec + r.drop_exp) | (s & 0x80000000u));
+    uint32_t q = __float_as_uint(sub_ieee(add_ieee(__uint_as_float(s), c), c));
+    const uint32_t aq = q & 0x7FFFFFFFu;
+    if (aq >= r.inf_bits) q = aq > 0x7F800000u ? 0x7FC00000u : ((q & 0x80000000u) | 0x7F800000u);
+    if (kFlush && aq < r.min_normal) q &= 0x80000000u;
+    return __uint_as_float(q);
 }
 
-__device__ __forceinline__ float fmac(float acc, float x, float y, const QuantParams& p, uint32_t inf_bits) {
-    return round_small(add_to_odd(acc, mul_ieee(x, y)), p, inf_bits);
+template <bool kFlush>
+__device__ __forceinline__ float fmac(float acc, float x, float y, const SmallRound& r) {
+    return round_small<kFlush>(add_to_odd(acc, mul_ieee(x, y)), r);
 }
 
 // One 32-deep slice of op(A) (rows m0.., kBM of them) into shared memory as [k][m]; elements
@@ -132,7 +146,7 @@ __device__ __forceinline__ void merge_block_hist(qfmt_stats_t* stats, const Quan
 // ---- any format with e <= 7, m <= 10 --------------------------------------------------------
 constexpr int kFmBM = 128, kFmBN = 64, kFmTM = 8, kFmTN = 4;
 
-template <bool kStats>
+template <bool kStats, bool kFlush>
 __global__ void __launch_bounds__(kFmThreads, 2)
 fmac8_kernel(FmacParams g, QuantParams p, qfmt_stats_t* __restrict__ stats) {
     __shared__ __align__(16) float As[kFmBK][kFmBM + 4];
@@ -144,7 +158,10 @@ fmac8_kernel(FmacParams g, QuantParams p, qfmt_stats_t* __restrict__ stats) {
         for (int i = threadIdx.x; i < nbins * 32; i += kFmThreads) lane_hist[i] = 0u;
         __syncthreads();
     }
-    const uint32_t inf_bits = (uint32_t)(p.top + p.code_off) << 23;  // fp32 bits of 2^(E_max+1)
+    SmallRound sr;
+    sr.min_normal = p.min_normal;
+    sr.inf_bits = (uint32_t)(p.top + p.code_off) << 23;
+    sr.drop_exp = p.drop << 23;
     const int tx = threadIdx.x % 16, ty = threadIdx.x / 16;
     const int tiles_n = (g.N + kFmBN - 1) / kFmBN, tiles_m = (g.M + kFmBM - 1) / kFmBM;
     auto same = [](float v) { return v; };
@@ -173,7 +190,7 @@ fmac8_kernel(FmacParams g, QuantParams p, qfmt_stats_t* __restrict__ stats) {
 #pragma unroll
                     for (int i = 0; i < kFmTM; ++i)
 #pragma unroll
-                        for (int j = 0; j < kFmTN; ++j) small[i][j] = fmac(small[i][j], a[i], b[j], p, inf_bits);
+                        for (int j = 0; j < kFmTN; ++j) small[i][j] = fmac<kFlush>(small[i][j], a[i], b[j], sr);
                 }
                 // the group's sum moves to the master accumulator (fp32 addition)
 #pragma unroll
@@ -213,10 +230,26 @@ __device__ __forceinline__ __half2 flush_denormals2(__half2 v) {
     return *reinterpret_cast<const __half2*>(&r);
 }
 
+// The slice a thread fetches: kRows * 32 / 256 elements, in the same order load_slice uses.
+template <int kRows>
+__device__ __forceinline__ void fetch_slice(float (&v)[kRows * kFmBK / kFmThreads], const float* src, long long ld,
+                                            int trans_k_major, int r0, int rmax, int k0, int kmax) {
+#pragma unroll
+    for (int t = 0; t < kRows * kFmBK / kFmThreads; ++t) {
+        const int idx = threadIdx.x + t * kFmThreads;
+        int r, k;
+        if (trans_k_major) { k = idx % kFmBK; r = idx / kFmBK; }
+        else { r = idx % kRows; k = idx / kRows; }
+        v[t] = 0.0f;
+        if (r0 + r < rmax && k0 + k < kmax)
+            v[t] = trans_k_major ? src[(long long)(r0 + r) * ld + (k0 + k)] : src[(long long)(k0 + k) * ld + (r0 + r)];
+    }
+}
+
 template <bool kStats, bool kFlush>
 __global__ void __launch_bounds__(kFmThreads, 1)
 fmac8_f16_kernel(FmacParams g, QuantParams p, qfmt_stats_t* __restrict__ stats) {
-    __shared__ __align__(16) __half As[kFmBK][kHfBM + 8];
+    __shared__ __align__(16) uint32_t As2[kFmBK][kHfBM + 4];  // each A value twice: {a, a} as f16x2
     __shared__ __align__(16) __half Bs[kFmBK][kHfBN + 8];
     extern __shared__ uint32_t lane_hist[];
     const int nbins = p.top + kExtraBins;
@@ -227,7 +260,8 @@ fmac8_f16_kernel(FmacParams g, QuantParams p, qfmt_stats_t* __restrict__ stats) 
     }
     const int tx = threadIdx.x % 16, ty = threadIdx.x / 16;
     const int tiles_n = (g.N + kHfBN - 1) / kHfBN, tiles_m = (g.M + kHfBM - 1) / kHfBM;
-    auto to_half = [](float v) { return __float2half_rn(v); };  // exact: operands hold binary16 values
+    constexpr int kPer = kHfBM * kFmBK / kFmThreads;  // elements of each operand a thread moves per slice
+    static_assert(kHfBM == kHfBN, "one fetch count for both operands");
     for (long long tile = blockIdx.x; tile < (long long)tiles_m * tiles_n; tile += gridDim.x) {
         const int m0 = (int)(tile / tiles_n) * kHfBM, n0 = (int)(tile % tiles_n) * kHfBN;
         float master[kHfTM][kHfTN];
@@ -240,39 +274,54 @@ fmac8_f16_kernel(FmacParams g, QuantParams p, qfmt_stats_t* __restrict__ stats) 
 #pragma unroll
             for (int j = 0; j < kHfTN / 2; ++j) small[i][j] = zero2;
         }
+        float fa[kPer], fb[kPer];  // the next slice, on its way from global memory while this one is used
+        fetch_slice<kHfBM>(fa, g.A, g.lda, !g.transA, m0, g.M, 0, g.K);
+        fetch_slice<kHfBN>(fb, g.B, g.ldb, g.transB, n0, g.N, 0, g.K);
         for (int k0 = 0; k0 < g.K; k0 += kFmBK) {
+            __syncthreads();  // the previous slice is no longer read
+#pragma unroll
+            for (int t = 0; t < kPer; ++t) {
+                const int idx = threadIdx.x + t * kFmThreads;
+                // the conversions are exact: operands hold binary16 values
+                const uint32_t ha = __half_as_ushort(__float2half_rn(fa[t]));
+                if (!g.transA) As2[idx % kFmBK][idx / kFmBK] = ha | (ha << 16);
+                else As2[idx / kHfBM][idx % kHfBM] = ha | (ha << 16);
+                if (g.transB) Bs[idx % kFmBK][idx / kFmBK] = __float2half_rn(fb[t]);
+                else Bs[idx / kHfBN][idx % kHfBN] = __float2half_rn(fb[t]);
+            }
             __syncthreads();
-            load_slice<kHfBM, kHfBM + 8>(As, g.A, g.lda, !g.transA, m0, g.M, k0, g.K, to_half);
-            load_slice<kHfBN, kHfBN + 8>(Bs, g.B, g.ldb, g.transB, n0, g.N, k0, g.K, to_half);
-            __syncthreads();
+            if (k0 + kFmBK < g.K) {
+                fetch_slice<kHfBM>(fa, g.A, g.lda, !g.transA, m0, g.M, k0 + kFmBK, g.K);
+                fetch_slice<kHfBN>(fb, g.B, g.ldb, g.transB, n0, g.N, k0 + kFmBK, g.K);
+            }
             const int kmax = g.K - k0 < kFmBK ? g.K - k0 : kFmBK;
 #pragma unroll 1
             for (int kg = 0; kg < kmax; kg += kGroup) {
 #pragma unroll
                 for (int kk = 0; kk < kGroup; ++kk) {
-                    const uint4 av = *reinterpret_cast<const uint4*>(&As[kg + kk][ty * kHfTM]);  // 8 halves
-                    const uint4 bv = *reinterpret_cast<const uint4*>(&Bs[kg + kk][tx * kHfTN]);
-                    const uint32_t aw[4] = {av.x, av.y, av.z, av.w};
-                    const uint32_t bw[4] = {bv.x, bv.y, bv.z, bv.w};
+                    const uint4 a0 = *reinterpret_cast<const uint4*>(&As2[kg + kk][ty * kHfTM]);
+                    const uint4 a1 = *reinterpret_cast<const uint4*>(&As2[kg + kk][ty * kHfTM + 4]);
+                    const uint4 bv = *reinterpret_cast<const uint4*>(&Bs[kg + kk][tx * kHfTN]);  // 8 halves
+                    const uint32_t aw[kHfTM] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+                    const uint32_t bw[kHfTN / 2] = {bv.x, bv.y, bv.z, bv.w};
 #pragma unroll
                     for (int i = 0; i < kHfTM; ++i) {
-                        // both halves = a_i
-                        const uint32_t dup = __byte_perm(aw[i >> 1], 0u, (i & 1) ? 0x3232 : 0x1010);
-                        const __half2 a2 = *reinterpret_cast<const __half2*>(&dup);
+                        const __half2 a2 = *reinterpret_cast<const __half2*>(&aw[i]);
 #pragma unroll
                         for (int j = 0; j < kHfTN / 2; ++j) {
-                            __half2 r = hfma2_ieee(a2, *reinterpret_cast<const __half2*>(&bw[j]), small[i][j]);
+                            const __half2 r = hfma2_ieee(a2, *reinterpret_cast<const __half2*>(&bw[j]), small[i][j]);
                             small[i][j] = kFlush ? flush_denormals2(r) : r;
                         }
                     }
                 }
+                // the group's sums move to the master accumulators (fp32 addition)
 #pragma unroll
                 for (int i = 0; i < kHfTM; ++i)
 #pragma unroll
                     for (int j = 0; j < kHfTN / 2; ++j) {
-                        const float2 s = __half22float2(small[i][j]);
-                        master[i][2 * j] = add_ieee(master[i][2 * j], s.x);
-                        master[i][2 * j + 1] = add_ieee(master[i][2 * j + 1], s.y);
+                        const float2 v = __half22float2(small[i][j]);
+                        master[i][2 * j] = add_ieee(master[i][2 * j], v.x);
+                        master[i][2 * j + 1] = add_ieee(master[i][2 * j + 1], v.y);
                         small[i][j] = zero2;
                     }
             }
@@ -337,8 +386,14 @@ int gemm_fmac8_device(const qfmt_matrix_t* A, const qfmt_matrix_t* B, float* d_C
         const long long tiles = ((M + kFmBM - 1) / kFmBM) * ((N + kFmBN - 1) / kFmBN);
         const long long cap = (long long)dev.sm_count * 2;
         const unsigned grid = (unsigned)(tiles < cap ? tiles : cap);
-        if (has_stats) fmac8_kernel<true><<<grid, kFmThreads, smem, stream>>>(g, p, d_stats);
-        else fmac8_kernel<false><<<grid, kFmThreads, 0, stream>>>(g, p, d_stats);
+        const bool flush = fmt->denormals == 0;
+        if (has_stats) {
+            if (flush) fmac8_kernel<true, true><<<grid, kFmThreads, smem, stream>>>(g, p, d_stats);
+            else fmac8_kernel<true, false><<<grid, kFmThreads, smem, stream>>>(g, p, d_stats);
+        } else {
+            if (flush) fmac8_kernel<false, true><<<grid, kFmThreads, 0, stream>>>(g, p, d_stats);
+            else fmac8_kernel<false, false><<<grid, kFmThreads, 0, stream>>>(g, p, d_stats);
+        }
     }
     QFMT_CUDA_TRY(cudaGetLastError());
     return QFMT_OK;
