@@ -7,7 +7,9 @@ flushed, at loss scales 2^0, 2^8 and 2^15 (18 kernel launches, 8 bytes of algori
 per element and launch).  `value` is the whole-job GB/s with inputs resident in HBM; `e2e` is
 the same metric through the host-buffer entry point (copies inside the timed region).  The
 contraction half of the path is timed in the same run on the BERT-large FC stack (workload
-"config5", one step: 4 layers x fwd/dgrad/wgrad) and reported under `gemm`.
+"config5", one step: 4 layers x fwd/dgrad/wgrad) and reported under `gemm`; the convolution
+layers of config4 under `conv`, the one-pass layer output R(R(acc)+R(B)) under `epilogue` and the
+FMAC-8 product (Algorithm 1) under `fmac8`.
 
     python bench.py --gpus N --steps K --warmup W          # this library
     python bench.py --impl reference ...                    # the CPU oracle on a bounded sample
@@ -252,6 +254,87 @@ def conv_section(torch, qf, dev, peaks, reps=5):
     return out
 
 
+def epilogue_section(torch, qf, dev, peaks, reps=20):
+    """Layer output Y = R(R(acc) + R(B)) with statistics of Y, one pass: the forward output of the
+    config5 FFN-up layer (8192 x 4096, the library's own product as `acc`), 1/6/9."""
+    c = workloads.config5_layer(2, step=0)
+    fmt = qf.make_format(6, 9, 1)
+    X, W = torch.from_numpy(c["X"]).to(dev), torch.from_numpy(c["W"]).to(dev)
+    qf.qfmt_quantize_stats(X, X, X.numel(), fmt)
+    qf.qfmt_quantize_stats(W, W, W.numel(), fmt)
+    rows, cols = X.shape[0], W.shape[1]
+    acc = torch.empty(rows, cols, dtype=torch.float32, device=dev)
+    a, b = qf.make_matrix(X), qf.make_matrix(W)
+    ws = torch.zeros(max(256, qf.qfmt_gemm_workspace_bytes(a, b)), dtype=torch.uint8, device=dev)
+    qf.qfmt_gemm(a, b, acc, cols, fmt, ws, ws.numel())
+    assert qf.qfmt_device_status(ws) == qf.QFMT_OK
+    bias = torch.from_numpy(workloads.normal_tensor(workloads.rng_for(4, 1000), (cols,), 0.02)).to(dev)
+    out = torch.empty_like(acc)
+    st = torch.zeros(qf.STATS_WORDS, dtype=torch.int64, device=dev)
+
+    def step():
+        qf.qfmt_bias_quantize_stats(acc, cols, bias, out, cols, rows, cols, fmt, st)
+    for _ in range(3):
+        step()
+    ms = statistics.median(time_events(torch, step, reps))
+    assert int(st.cpu()[256]) == rows * cols
+    achieved = rows * cols * BYTES_PER_ELEMENT / ms / 1e6
+    return {"metric": "layer output R(R(acc)+R(B)) + stats GB/s", "value": achieved, "unit": "GB/s",
+            "workload": f"config5 FFN-up forward output, {rows} x {cols}, 1/6/9 (268 MB moved per launch, larger than L2)",
+            "ms_per_step": ms, "gpu_launches_per_step": 1,
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                         "frac": achieved / peaks["hbm_gbs"], "traffic": None,
+                         "peak_source": f"copy bandwidth, {peaks['source']}",
+                         "algorithmic_bytes_per_launch": rows * cols * BYTES_PER_ELEMENT}}
+
+
+# FMAC-8 is plain-ALU work.  Peak = SMs x 4 schedulers x 32 lanes x max SM clock / (scheduler cycles one
+# warp-wide multiply-add must cost).  General kernel: per FMAC FMAC8_FLOAT_OPS float-pipe instructions
+# (one per cycle) and FMAC8_INT_OPS integer-pipe instructions (one per two cycles: 16 lanes per
+# scheduler), counted in the kernel's inner loop; the bound is the larger of the issue slots and the
+# integer pipe.  Binary16 kernel: one fma.rn.f16x2 per two FMACs, two cycles each on this part (the
+# float pipe's busy cycles are twice its instruction count for a stream of them).
+SM_COUNT, LANES_PER_SM = 148, 128
+FMAC8_FLOAT_OPS, FMAC8_INT_OPS = 5.0, 6.0
+
+
+def fmac8_section(torch, qf, dev, peaks, clock_mhz, reps=3):
+    """Algorithm 1 (FMAC-8) on the config3 forward product (4096 x 3072 x 768): 1/6/9 on the general
+    ALU kernel and 1/5/10 on the half-precision FMA kernel; output statistics taken in the kernel."""
+    cfg = workloads.config3()
+    M, K = cfg["X"].shape
+    N = cfg["W"].shape[1]
+    out = {"metric": "FMAC-8 product TFMAC/s", "unit": "TFMAC/s",
+           "workload": f"config3 forward product {M} x {N} x {K}, FMAC-8 accumulation, statistics of the output", "runs": {}}
+    clk = clock_mhz * 1e6
+    cyc_general = max(FMAC8_FLOAT_OPS + FMAC8_INT_OPS, 2.0 * FMAC8_INT_OPS)
+    peaks_t = {"general": SM_COUNT * LANES_PER_SM * clk / cyc_general / 1e12,
+               "binary16": SM_COUNT * LANES_PER_SM * clk * 2 / 2.0 / 1e12}
+    for tag, e, m, path, kind in (("1/6/9 general", 6, 9, 0, "general"), ("1/5/10 binary16", 5, 10, 0, "binary16")):
+        fmt = qf.make_format(e, m, 1)
+        X, W = torch.from_numpy(cfg["X"]).to(dev), torch.from_numpy(cfg["W"]).to(dev)
+        qf.qfmt_quantize_stats(X, X, X.numel(), fmt)
+        qf.qfmt_quantize_stats(W, W, W.numel(), fmt)
+        C = torch.empty(M, N, dtype=torch.float32, device=dev)
+        st = torch.zeros(qf.STATS_WORDS, dtype=torch.int64, device=dev)
+        a, b = qf.make_matrix(X), qf.make_matrix(W)
+
+        def step():
+            qf.qfmt_gemm_fmac8(a, b, C, N, fmt, st, 0, path)
+        step()
+        ms = statistics.median(time_events(torch, step, reps))
+        assert int(st.cpu()[256]) == M * N
+        tf = M * N * K / ms / 1e9
+        out["runs"][tag] = {"ms": ms, "tfmac_per_s": tf, "denormal_fraction_of_output": int(st.cpu()[258]) / (M * N),
+                            "roofline": {"bound": "alu", "achieved": tf, "peak": peaks_t[kind], "unit": "TFMAC/s",
+                                         "frac": tf / peaks_t[kind], "traffic": None,
+                                         "peak_source": "derived: SMs x lanes x max SM clock / cycles per FMAC (see comment)"}}
+    first = out["runs"]["1/6/9 general"]
+    out.update({"value": first["tfmac_per_s"], "ms_per_step": first["ms"], "gpu_launches_per_step": 1,
+                "roofline": first["roofline"]})
+    return out
+
+
 def run_library(args):
     import torch
     import paper_2103_15940_b200 as qf
@@ -335,6 +418,11 @@ def run_library(args):
 
     sections = set(args.sections.split(","))
     e2e = gemm = cpu = conv = None
+    extra = {}
+    if "epilogue" in sections:
+        extra["epilogue"] = epilogue_section(torch, qf, dev, peaks)
+    if "fmac8" in sections:
+        extra["fmac8"] = fmac8_section(torch, qf, dev, peaks, clocks.summary()["sm_max_mhz"] or 1965)
     if "e2e" in sections:
         e2e = e2e_section(torch, qf, dev, x_host, fmts, n, step_bytes, args)
     if "gemm" in sections:
@@ -349,7 +437,7 @@ def run_library(args):
         cpu = {"value": cpu_value, "unit": UNIT, "cores": 1, "kind": "oracle", "seconds": cpu_secs,
                "host_cores_available": os.cpu_count(),
                "sample": f"the 18 sweep runs on the first {n_cpu} of {n} elements"}
-    return finish(args, world, value, total_ms, n, runs, clocks, e2e, roofline, cpu, gemm, conv, dist)
+    return finish(args, world, value, total_ms, n, runs, clocks, e2e, roofline, cpu, gemm, conv, dist, extra)
 
 
 def e2e_section(torch, qf, dev, x_host, fmts, n, step_bytes, args):
@@ -371,7 +459,7 @@ def e2e_section(torch, qf, dev, x_host, fmts, n, step_bytes, args):
     return e2e
 
 
-def finish(args, world, value, total_ms, n, runs, clocks, e2e, roofline, cpu, gemm, conv, dist):
+def finish(args, world, value, total_ms, n, runs, clocks, e2e, roofline, cpu, gemm, conv, dist, extra):
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "u32", "data": "synthetic",
@@ -380,6 +468,7 @@ def finish(args, world, value, total_ms, n, runs, clocks, e2e, roofline, cpu, ge
                        "multi_gpu": "replicas only: every rank runs the whole sweep on its own copy"},
             "clocks": clocks.summary(), "e2e": e2e, "gpu_launches": args.steps * len(runs),
             "roofline": roofline, "cpu_baseline": cpu, "gemm": gemm, "conv": conv}
+    line.update(extra)
     print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
@@ -396,9 +485,9 @@ def main():
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="library", choices=["library", "reference"])
-    ap.add_argument("--sections", default="quantize,e2e,gemm,conv,cpu",
+    ap.add_argument("--sections", default="quantize,e2e,gemm,conv,epilogue,fmac8,cpu",
                     help="comma list of what to measure besides the timed sweep (quantize is always timed): "
-                         "e2e, gemm, conv, cpu; profiling captures use a subset")
+                         "e2e, gemm, conv, epilogue, fmac8, cpu; profiling captures use a subset")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -57,30 +57,32 @@ __device__ __forceinline__ uint32_t add_to_odd(float a, float prod) {
 struct SmallRound {
     uint32_t min_normal;  // fp32 bits of 2^E_min
     uint32_t inf_bits;    // fp32 bits of 2^(E_max+1)
-    uint32_t drop_exp;    // (23 - m) << 23
+    uint32_t magic_add;   // ((23 - m) << 23) | 0x400000
 };
 
 // Rounds a 24-bit intermediate to the format (the small accumulator's rounding; no statistics).
-// With C = +-2^(max(floor(log2|s|), E_min) + 23 - m), the fp32 sum s + C has its last place at the
-// format's quantum for s, so (s + C) - C is s rounded to nearest-even on the format's grid, normal
-// or denormal, sign included.  The exponent is capped at E_max+1 so that C stays finite; values
+// With C = 1.5 * 2^(max(floor(log2|s|), E_min) + 23 - m), the fp32 sum s + C stays in C's binade,
+// whose last place is the format's quantum for s, so (s + C) - C is s rounded to nearest-even on
+// the format's grid, normal or denormal, either sign (a zero result may come out as +0 where -0 is
+// meant; nothing downstream can tell: it is only ever added to other numbers).  For e = 7 the sum
+// a + x*y can approach 2^128, so the exponent is capped at E_max+1 to keep C finite (kCap); values
 // that reach 2^(E_max+1) are made infinite (or the quiet NaN) afterwards.
-template <bool kFlush>
+template <bool kFlush, bool kCap>
 __device__ __forceinline__ float round_small(uint32_t s, const SmallRound& r) {
     uint32_t ec = s & 0x7F800000u;
     ec = ec < r.min_normal ? r.min_normal : ec;
-    ec = ec > r.inf_bits ? r.inf_bits : ec;
-    const float c = __uint_as_float((ec + r.drop_exp) | (s & 0x80000000u));
-    uint32_t q = __float_as_uint(sub_ieee(add_ieee(__uint_as_float(s), c), c));
-    const uint32_t aq = q & 0x7FFFFFFFu;
-    if (aq >= r.inf_bits) q = aq > 0x7F800000u ? 0x7FC00000u : ((q & 0x80000000u) | 0x7F800000u);
-    if (kFlush && aq < r.min_normal) q &= 0x80000000u;
-    return __uint_as_float(q);
+    if (kCap) ec = ec > r.inf_bits ? r.inf_bits : ec;
+    const float c = __uint_as_float(ec + r.magic_add);
+    float q = sub_ieee(add_ieee(__uint_as_float(s), c), c);
+    if (!(fabsf(q) < __uint_as_float(r.inf_bits)))
+        q = (q != q) ? __uint_as_float(0x7FC00000u) : copysignf(__uint_as_float(0x7F800000u), q);
+    if (kFlush && fabsf(q) < __uint_as_float(r.min_normal)) q = 0.0f;
+    return q;
 }
 
-template <bool kFlush>
+template <bool kFlush, bool kCap>
 __device__ __forceinline__ float fmac(float acc, float x, float y, const SmallRound& r) {
-    return round_small<kFlush>(add_to_odd(acc, mul_ieee(x, y)), r);
+    return round_small<kFlush, kCap>(add_to_odd(acc, mul_ieee(x, y)), r);
 }
 
 // One 32-deep slice of op(A) (rows m0.., kBM of them) into shared memory as [k][m]; elements
@@ -146,7 +148,7 @@ __device__ __forceinline__ void merge_block_hist(qfmt_stats_t* stats, const Quan
 // ---- any format with e <= 7, m <= 10 --------------------------------------------------------
 constexpr int kFmBM = 128, kFmBN = 64, kFmTM = 8, kFmTN = 4;
 
-template <bool kStats, bool kFlush>
+template <bool kStats, bool kFlush, bool kCap>
 __global__ void __launch_bounds__(kFmThreads, 2)
 fmac8_kernel(FmacParams g, QuantParams p, qfmt_stats_t* __restrict__ stats) {
     __shared__ __align__(16) float As[kFmBK][kFmBM + 4];
@@ -161,7 +163,7 @@ fmac8_kernel(FmacParams g, QuantParams p, qfmt_stats_t* __restrict__ stats) {
     SmallRound sr;
     sr.min_normal = p.min_normal;
     sr.inf_bits = (uint32_t)(p.top + p.code_off) << 23;
-    sr.drop_exp = p.drop << 23;
+    sr.magic_add = p.magic_add;
     const int tx = threadIdx.x % 16, ty = threadIdx.x / 16;
     const int tiles_n = (g.N + kFmBN - 1) / kFmBN, tiles_m = (g.M + kFmBM - 1) / kFmBM;
     auto same = [](float v) { return v; };
@@ -190,7 +192,7 @@ fmac8_kernel(FmacParams g, QuantParams p, qfmt_stats_t* __restrict__ stats) {
 #pragma unroll
                     for (int i = 0; i < kFmTM; ++i)
 #pragma unroll
-                        for (int j = 0; j < kFmTN; ++j) small[i][j] = fmac<kFlush>(small[i][j], a[i], b[j], sr);
+                        for (int j = 0; j < kFmTN; ++j) small[i][j] = fmac<kFlush, kCap>(small[i][j], a[i], b[j], sr);
                 }
                 // the group's sum moves to the master accumulator (fp32 addition)
 #pragma unroll
@@ -386,14 +388,17 @@ int gemm_fmac8_device(const qfmt_matrix_t* A, const qfmt_matrix_t* B, float* d_C
         const long long tiles = ((M + kFmBM - 1) / kFmBM) * ((N + kFmBN - 1) / kFmBN);
         const long long cap = (long long)dev.sm_count * 2;
         const unsigned grid = (unsigned)(tiles < cap ? tiles : cap);
-        const bool flush = fmt->denormals == 0;
+        const bool flush = fmt->denormals == 0, cap_exp = fmt->e == 7;
+        const size_t sm = has_stats ? smem : 0;
+#define QFMT_FLAUNCH(S, F, C) fmac8_kernel<S, F, C><<<grid, kFmThreads, sm, stream>>>(g, p, d_stats)
         if (has_stats) {
-            if (flush) fmac8_kernel<true, true><<<grid, kFmThreads, smem, stream>>>(g, p, d_stats);
-            else fmac8_kernel<true, false><<<grid, kFmThreads, smem, stream>>>(g, p, d_stats);
+            if (flush) { if (cap_exp) QFMT_FLAUNCH(true, true, true); else QFMT_FLAUNCH(true, true, false); }
+            else { if (cap_exp) QFMT_FLAUNCH(true, false, true); else QFMT_FLAUNCH(true, false, false); }
         } else {
-            if (flush) fmac8_kernel<false, true><<<grid, kFmThreads, 0, stream>>>(g, p, d_stats);
-            else fmac8_kernel<false, false><<<grid, kFmThreads, 0, stream>>>(g, p, d_stats);
+            if (flush) { if (cap_exp) QFMT_FLAUNCH(false, true, true); else QFMT_FLAUNCH(false, true, false); }
+            else { if (cap_exp) QFMT_FLAUNCH(false, false, true); else QFMT_FLAUNCH(false, false, false); }
         }
+#undef QFMT_FLAUNCH
     }
     QFMT_CUDA_TRY(cudaGetLastError());
     return QFMT_OK;

@@ -26,6 +26,7 @@ struct QuantParams {
     int32_t top;           // 2^e - 1, the inf/NaN exponent field
     uint32_t keep_denormals;
     float scale;
+    uint32_t magic_add;    // ((23 - m) << 23) | 0x400000: exponent field + this = 1.5 * 2^(exponent + 23 - m)
 };
 
 // Extra bins after the regular exponent fields 1 .. top-1.
@@ -110,6 +111,7 @@ inline QuantParams make_params(const qfmt_format_t& f) {
     p.top = (1 << f.e) - 1;
     p.keep_denormals = f.denormals ? 1u : 0u;
     p.scale = f.loss_scale;
+    p.magic_add = (p.drop << 23) | 0x00400000u;
     return p;
 }
 
