@@ -200,92 +200,129 @@ quantize_stats_transpose_kernel(const uint32_t* __restrict__ in, uint32_t* __res
 // statistics of Y taken in the same pass.  The sum of two format values is formed with one IEEE
 // fp32 add; for m <= 10 that add is either exact or so far from every grid and halfway point of
 // the format that rounding its result equals rounding the exact sum (when the add is inexact the
-// smaller term lies below 2^-12 of the larger one's last place).  The block first rounds the bias
-// vector into shared memory (or, for very wide matrices, each element rounds its own bias entry).
-// Vector kernel: rows of c4 = cols/4 128-bit vectors; each thread walks the flat vector index with
-// a fixed stride and keeps (row, column) per slot by adding the stride's quotient and remainder.
+// smaller term lies below 2^-12 of the larger one's last place).
+// Vector kernel: rows of c4 = cols/4 128-bit vectors; each thread owns a column of vectors (its
+// rounded bias entries stay in registers) and walks down the rows, four loads in flight.
+// R(S * x) without statistics, for formats with e <= 7: the first rounding of the layer formula.
+// The integer pipe runs at half the float pipe's rate, so the rounding is two float operations:
+// with C = 1.5 * 2^(max(floor(log2|y|), E_min) + 23 - m) the sum y + C lies in C's binade, whose
+// last place is the format's quantum for y; the IEEE addition rounds there to nearest-even (C is
+// an even multiple of the quantum) and subtracting C is exact.  Normal and denormal results, both
+// signs; a zero result gets y's sign back with an OR.  The exponent is capped at E_max+1 so that C
+// stays finite; whatever reaches 2^(E_max+1) becomes infinite.  (A NaN stays some NaN: the addition
+// that follows makes it the positive quiet NaN whatever its payload.)
 template <bool kScale>
-__device__ __forceinline__ uint32_t bias_round_one(uint32_t acc, uint32_t rb, const QuantParams& p, int& bin) {
+__device__ __forceinline__ uint32_t round_value(uint32_t xb, const QuantParams& p, uint32_t inf_bits) {
+    const uint32_t yb = kScale ? __float_as_uint(mul_ieee(__uint_as_float(xb), p.scale)) : xb;
+    uint32_t ec = yb & 0x7F800000u;
+    ec = ec < p.min_normal ? p.min_normal : ec;
+    ec = ec > inf_bits ? inf_bits : ec;
+    const float c = __uint_as_float(ec + p.magic_add);
+    float q = sub_ieee(add_ieee(__uint_as_float(yb), c), c);
+    if (!(fabsf(q) < __uint_as_float(inf_bits)) && q == q) q = copysignf(__uint_as_float(0x7F800000u), q);
+    if (!p.keep_denormals && fabsf(q) < __uint_as_float(p.min_normal)) q = 0.0f;
+    return __float_as_uint(q) | (yb & 0x80000000u);
+}
+
+// Second rounding of the layer formula, with the bin: s is the fp32 sum of two format values
+// (e <= 7, so |s| < 2^(E_max+2) and the rounding constant cannot overflow), or inf/NaN.
+__device__ __forceinline__ uint32_t round_sum(uint32_t s, const QuantParams& p, int& bin) {
+    uint32_t ec = s & 0x7F800000u;
+    ec = ec < p.min_normal ? p.min_normal : ec;
+    const float c = __uint_as_float(ec + p.magic_add);
+    const uint32_t sign = s & 0x80000000u;
+    uint32_t q = __float_as_uint(sub_ieee(add_ieee(__uint_as_float(s), c), c)) | sign;
+    const uint32_t aq = q & 0x7FFFFFFFu;
+    const int code = (int)(aq >> 23) - p.code_off;
+    bin = code;
+    if ((unsigned)(code - 1) >= (unsigned)(p.top - 1)) {  // not a normal number of the format
+        const uint32_t as = s & 0x7FFFFFFFu;
+        if (code >= p.top) {
+            const bool is_nan = as > 0x7F800000u;
+            q = is_nan ? 0x7FC00000u : (sign | 0x7F800000u);
+            bin = p.top + (is_nan ? kBinNanIn : (as == 0x7F800000u ? kBinInfIn : kBinOverflow));
+        } else {
+            bin = p.top + (as == 0u ? kBinZeroIn : (aq == 0u ? kBinRoundedToZero : kBinDenormal));
+            if (!p.keep_denormals) q = sign;
+        }
+    }
+    return q;
+}
+
+template <bool kScale>
+__device__ __forceinline__ uint32_t bias_round_one(uint32_t acc, uint32_t rb, const QuantParams& p, uint32_t inf_bits,
+                                                   int& bin) {
+    if (inf_bits != 0u) {
+        const uint32_t ra = round_value<kScale>(acc, p, inf_bits);
+        return round_sum(__float_as_uint(add_ieee(__uint_as_float(ra), __uint_as_float(rb))), p, bin);
+    }
+    // 1/8/m: values near fp32's largest would push the rounding constants out of range
     int unused;
     const uint32_t ra = quantize_one<kScale>(acc, p, unused);
     const uint32_t s = __float_as_uint(add_ieee(__uint_as_float(ra), __uint_as_float(rb)));
     const uint32_t q = quantize_one<false>(s, p, bin);
-    // 1/8/m only: two finite terms whose fp32 sum is already infinite overflowed, they were not infinite
+    // two finite terms whose fp32 sum is already infinite overflowed, they were not infinite
     if (bin == p.top + kBinInfIn && (ra & 0x7FFFFFFFu) < 0x7F800000u && (rb & 0x7FFFFFFFu) < 0x7F800000u)
         bin = p.top + kBinOverflow;
     return q;
 }
 
-template <bool kStats, bool kScale, bool kSmemBias>
+template <bool kStats, bool kScale>
 __global__ void __launch_bounds__(kThreads)
 bias_quantize_stats_kernel(const uint32_t* acc, long long ld_acc, const uint32_t* __restrict__ bias, uint32_t* out,
-                           long long ld_out, unsigned long long rows, uint32_t c4, QuantParams p,
-                           qfmt_stats_t* __restrict__ stats) {
-    extern __shared__ uint32_t lane_hist[];  // [(top + kExtraBins)][32], then the rounded bias
+                           long long ld_out, unsigned long long rows, uint32_t c4, uint32_t cw, uint32_t rpp,
+                           QuantParams p, qfmt_stats_t* __restrict__ stats) {
+    extern __shared__ uint32_t lane_hist[];  // [(top + kExtraBins)][32]
     const int nbins = p.top + kExtraBins;
     const int lane = threadIdx.x & 31;
-    uint32_t* sbias = lane_hist + (kStats ? nbins * 32 : 0);
+    const uint32_t inf_bits = p.top < 255 ? (uint32_t)(p.top + p.code_off) << 23 : 0u;  // 2^(E_max+1); 0 = 1/8/m
     if (kStats) {
         for (int i = threadIdx.x; i < nbins * 32; i += kThreads) lane_hist[i] = 0u;
+        __syncthreads();
     }
-    if (kSmemBias) {
-        for (uint32_t j = threadIdx.x; j < c4 * 4u; j += kThreads) {
+    // A pass of the block covers rpp rows x cw vectors; a thread keeps its column, so the rounded
+    // bias of that column stays in registers while it walks down the rows.
+    const uint32_t r_local = threadIdx.x / cw, c_local = threadIdx.x % cw;
+    if (r_local < rpp) {
+        const unsigned long long row_step = (unsigned long long)gridDim.x * rpp;
+        for (uint32_t cc = c_local; cc < c4; cc += cw) {
+            const uint4 raw = reinterpret_cast<const uint4*>(bias)[cc];
             int unused;
-            sbias[j] = quantize_one<kScale>(bias[j], p, unused);
-        }
-    }
-    __syncthreads();
-    const unsigned long long n4 = rows * c4;
-    const unsigned long long stride = (unsigned long long)gridDim.x * (kThreads * kUnroll);
-    const unsigned long long dq = stride / c4;
-    const uint32_t dr = (uint32_t)(stride % c4);
-    unsigned long long row[kUnroll];
-    uint32_t col[kUnroll];
+            uint4 b;
+            b.x = quantize_one<kScale>(raw.x, p, unused);
+            b.y = quantize_one<kScale>(raw.y, p, unused);
+            b.z = quantize_one<kScale>(raw.z, p, unused);
+            b.w = quantize_one<kScale>(raw.w, p, unused);
+            unsigned long long row = (unsigned long long)blockIdx.x * rpp + r_local;
+            const uint4* pa = reinterpret_cast<const uint4*>(acc + row * ld_acc) + cc;
+            uint4* po = reinterpret_cast<uint4*>(out + row * ld_out) + cc;
+            const unsigned long long step_a = row_step * (unsigned long long)ld_acc / 4ull;  // in vectors
+            const unsigned long long step_o = row_step * (unsigned long long)ld_out / 4ull;
+            for (; row < rows; row += row_step * kUnroll) {
+                uint4 v[kUnroll];
 #pragma unroll
-    for (int u = 0; u < kUnroll; ++u) {
-        const unsigned long long idx = (unsigned long long)blockIdx.x * (kThreads * kUnroll) + (unsigned long long)u * kThreads + threadIdx.x;
-        row[u] = idx / c4;
-        col[u] = (uint32_t)(idx % c4);
-    }
-    for (unsigned long long base = (unsigned long long)blockIdx.x * (kThreads * kUnroll); base < n4; base += stride) {
-        uint4 v[kUnroll];
+                for (int u = 0; u < kUnroll; ++u)
+                    if (row + u * row_step < rows) v[u] = load_stream(pa + u * step_a);
 #pragma unroll
-        for (int u = 0; u < kUnroll; ++u) {
-            if (row[u] < rows) v[u] = load_stream(reinterpret_cast<const uint4*>(acc + row[u] * ld_acc) + col[u]);
-        }
-#pragma unroll
-        for (int u = 0; u < kUnroll; ++u) {
-            if (row[u] < rows) {
-                uint4 b;
-                if (kSmemBias) {
-                    b = reinterpret_cast<const uint4*>(sbias)[col[u]];
-                } else {
-                    const uint4 raw = reinterpret_cast<const uint4*>(bias)[col[u]];
-                    int unused;
-                    b.x = quantize_one<kScale>(raw.x, p, unused);
-                    b.y = quantize_one<kScale>(raw.y, p, unused);
-                    b.z = quantize_one<kScale>(raw.z, p, unused);
-                    b.w = quantize_one<kScale>(raw.w, p, unused);
+                for (int u = 0; u < kUnroll; ++u) {
+                    if (row + u * row_step < rows) {
+                        int b0, b1, b2, b3;
+                        uint4 q;
+                        q.x = bias_round_one<kScale>(v[u].x, b.x, p, inf_bits, b0);
+                        q.y = bias_round_one<kScale>(v[u].y, b.y, p, inf_bits, b1);
+                        q.z = bias_round_one<kScale>(v[u].z, b.z, p, inf_bits, b2);
+                        q.w = bias_round_one<kScale>(v[u].w, b.w, p, inf_bits, b3);
+                        store_stream(po + u * step_o, q);
+                        if (kStats) {
+                            atomicAdd(&lane_hist[b0 * 32 + lane], 1u);
+                            atomicAdd(&lane_hist[b1 * 32 + lane], 1u);
+                            atomicAdd(&lane_hist[b2 * 32 + lane], 1u);
+                            atomicAdd(&lane_hist[b3 * 32 + lane], 1u);
+                        }
+                    }
                 }
-                int b0, b1, b2, b3;
-                uint4 q;
-                q.x = bias_round_one<kScale>(v[u].x, b.x, p, b0);
-                q.y = bias_round_one<kScale>(v[u].y, b.y, p, b1);
-                q.z = bias_round_one<kScale>(v[u].z, b.z, p, b2);
-                q.w = bias_round_one<kScale>(v[u].w, b.w, p, b3);
-                store_stream(reinterpret_cast<uint4*>(out + row[u] * ld_out) + col[u], q);
-                if (kStats) {
-                    atomicAdd(&lane_hist[b0 * 32 + lane], 1u);
-                    atomicAdd(&lane_hist[b1 * 32 + lane], 1u);
-                    atomicAdd(&lane_hist[b2 * 32 + lane], 1u);
-                    atomicAdd(&lane_hist[b3 * 32 + lane], 1u);
-                }
-            }
-            row[u] += dq;
-            col[u] += dr;
-            if (col[u] >= c4) {
-                col[u] -= c4;
-                row[u] += 1;
+                pa += kUnroll * step_a;
+                po += kUnroll * step_o;
             }
         }
     }
@@ -296,7 +333,8 @@ bias_quantize_stats_kernel(const uint32_t* acc, long long ld_acc, const uint32_t
             const uint32_t c = __reduce_add_sync(0xFFFFFFFFu, lane_hist[b * 32 + lane]);
             if (lane == 0 && c != 0u) merge_bin(stats, p, b, c);
         }
-        if (blockIdx.x == 0 && threadIdx.x == 0) atomicAdd((unsigned long long*)&stats->n_total, n4 * 4ull);
+        if (blockIdx.x == 0 && threadIdx.x == 0)
+            atomicAdd((unsigned long long*)&stats->n_total, rows * (unsigned long long)c4 * 4ull);
     }
 }
 
@@ -315,11 +353,12 @@ bias_quantize_stats_scalar_kernel(const uint32_t* acc, long long ld_acc, const u
     }
     const unsigned long long n = rows * cols;
     const unsigned long long stride = (unsigned long long)gridDim.x * kThreads;
+    const uint32_t inf_bits = p.top < 255 ? (uint32_t)(p.top + p.code_off) << 23 : 0u;
     for (unsigned long long i = (unsigned long long)blockIdx.x * kThreads + threadIdx.x; i < n; i += stride) {
         const unsigned long long r = i / cols, c = i % cols;
         int unused, b;
         const uint32_t rb = quantize_one<kScale>(bias[c], p, unused);
-        out[r * ld_out + c] = bias_round_one<kScale>(acc[r * ld_acc + c], rb, p, b);
+        out[r * ld_out + c] = bias_round_one<kScale>(acc[r * ld_acc + c], rb, p, inf_bits, b);
         if (kStats) atomicAdd(&lane_hist[b * 32 + lane], 1u);
     }
     if (kStats) {
@@ -472,27 +511,18 @@ int bias_quantize_stats_device(const float* d_acc, int64_t ld_acc, const float* 
     cudaError_t err = cudaSuccess;
     if (vec) {
         const uint32_t c4 = (uint32_t)(cols / 4);
-        const bool smem_bias = (size_t)cols * 4 <= 64 * 1024;
-        const size_t smem = hist_bytes + (smem_bias ? (size_t)cols * 4 : 0);
-        const unsigned long long per_block = (unsigned long long)kThreads * kUnroll;
-        unsigned long long want = ((unsigned long long)rows * c4 + per_block - 1) / per_block;
-        const unsigned long long cap = (unsigned long long)dev.sm_count * (smem > 36 * 1024 ? 2 : 3);
+        const uint32_t cw = c4 < (uint32_t)kThreads ? c4 : (uint32_t)kThreads;  // vectors of a row per pass
+        const uint32_t rpp = (uint32_t)kThreads / cw;                           // rows per pass
+        const size_t smem = hist_bytes;
+        unsigned long long want = ((unsigned long long)rows + (unsigned long long)rpp * kUnroll - 1) /
+                                  ((unsigned long long)rpp * kUnroll);
+        const unsigned long long cap = (unsigned long long)dev.sm_count * 2;  // 64 registers: two blocks per SM
         if (want > cap) want = cap;
-#define QFMT_BLAUNCH(S, C, B)                                                                                     \
-    do {                                                                                                          \
-        auto kern = bias_quantize_stats_kernel<S, C, B>;                                                          \
-        if (smem > 48 * 1024) err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
-        if (err == cudaSuccess)                                                                                   \
-            kern<<<(unsigned)want, kThreads, smem, stream>>>(acc, (long long)ld_acc, bias, out, (long long)ld_out, \
-                                                             (unsigned long long)rows, c4, p, d_stats);           \
-    } while (0)
-        if (has_stats) {
-            if (has_scale) { if (smem_bias) QFMT_BLAUNCH(true, true, true); else QFMT_BLAUNCH(true, true, false); }
-            else { if (smem_bias) QFMT_BLAUNCH(true, false, true); else QFMT_BLAUNCH(true, false, false); }
-        } else {
-            if (has_scale) { if (smem_bias) QFMT_BLAUNCH(false, true, true); else QFMT_BLAUNCH(false, true, false); }
-            else { if (smem_bias) QFMT_BLAUNCH(false, false, true); else QFMT_BLAUNCH(false, false, false); }
-        }
+#define QFMT_BLAUNCH(S, C)                                                                                        \
+    bias_quantize_stats_kernel<S, C><<<(unsigned)want, kThreads, smem, stream>>>(                                 \
+        acc, (long long)ld_acc, bias, out, (long long)ld_out, (unsigned long long)rows, c4, cw, rpp, p, d_stats)
+        if (has_stats) { if (has_scale) QFMT_BLAUNCH(true, true); else QFMT_BLAUNCH(true, false); }
+        else { if (has_scale) QFMT_BLAUNCH(false, true); else QFMT_BLAUNCH(false, false); }
 #undef QFMT_BLAUNCH
     } else {
         unsigned long long want = (n + kThreads - 1) / kThreads;
