@@ -135,6 +135,45 @@ int qfmt_bias_quantize_stats(const float* d_acc, int64_t ld_acc, const float* d_
                              int accumulate, void* stream);
 
 /*
+ * Dynamic loss scaling with the scale kept in device memory.  Section II describes loss scaling
+ * and Section V trains every format "with DLS" and without; the paper cites the technique and
+ * states no rule, so the usual one is taken: a step whose gradient tensors held any overflow,
+ * infinity or NaN is skipped and the scale is multiplied by `backoff` (not below min_scale);
+ * after `growth_interval` consecutive clean steps it is multiplied by `growth` (not above
+ * max_scale).  The record lives in DEVICE memory; the caller initialises it (scale, growth,
+ * backoff, limits, growth_interval; the rest zero) and may read `skip` back, or pass the record
+ * to its own update kernel, to leave out the weight update of a skipped step.
+ */
+typedef struct {
+    float scale;              /* current loss scale                                              */
+    float growth, backoff;    /* e.g. 2 and 0.5                                                  */
+    float min_scale, max_scale;
+    int32_t growth_interval;  /* clean steps before the scale grows, >= 1                        */
+    int32_t clean_steps;      /* clean steps since the scale last changed                        */
+    int32_t skip;             /* written by qfmt_dls_update: 1 = the step just checked is skipped */
+    int32_t reserved;
+    uint64_t n_steps, n_skipped;
+} qfmt_dls_t;
+
+/*
+ * One controller step: sums n_overflow + n_nan + n_inf_in over the n_records consecutive
+ * statistics records at d_stats (those of the step's gradient tensors, as written by the
+ * rounding pass) and updates *d_state by the rule above.  Everything happens on `stream`; nothing
+ * is copied to the host.  n_records = 0 counts as a clean step.
+ * Errors: QFMT_ERR_BAD_ARG (NULL or misaligned pointer, negative count), QFMT_ERR_UNSUPPORTED_ARCH,
+ * QFMT_ERR_CUDA.
+ */
+int qfmt_dls_update(qfmt_dls_t* d_state, const qfmt_stats_t* d_stats, int64_t n_records, void* stream);
+
+/*
+ * qfmt_quantize_stats with the loss scale read on the device from d_state->scale when the kernel
+ * runs (fmt->loss_scale is ignored, though still validated).  A kernel enqueued after
+ * qfmt_dls_update on the same stream sees the updated scale.
+ */
+int qfmt_quantize_stats_dls(const float* d_in, float* d_out, size_t n, const qfmt_format_t* fmt,
+                            const qfmt_dls_t* d_state, qfmt_stats_t* d_stats, int accumulate, void* stream);
+
+/*
  * The same operation on HOST buffers: copies h_in to the device, runs the kernel, copies the
  * rounded tensor (if h_out != NULL) and the statistics (if h_stats != NULL) back, and
  * SYNCHRONISES the stream before returning.  The caller lends device scratch:

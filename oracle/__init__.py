@@ -72,6 +72,8 @@ def _L() -> ctypes.CDLL:
         lib.oracle_fmac8_gemm_sampled.argtypes = [vp, i64, i32, vp, i64, i32, i64, i32, i32, i32, i32, vp, vp,
                                                   i64, vp]
         lib.oracle_fmac8_gemm_sampled.restype = None
+        lib.oracle_dls_update.argtypes = [vp, vp, i64]
+        lib.oracle_dls_update.restype = None
         _lib = lib
     return _lib
 
@@ -232,6 +234,20 @@ def fmac8_gemm_sampled(A: np.ndarray, B: np.ndarray, ii: np.ndarray, jj: np.ndar
                                    int(transB), K, e, m, int(denormals), group, ii.ctypes.data,
                                    jj.ctypes.data, ii.size, c.ctypes.data)
     return c.view(np.float32)
+
+
+class DlsState(ctypes.Structure):
+    """Dynamic-loss-scale controller state (same field order as the C struct in qfmt_oracle.c)."""
+    _fields_ = [("scale", ctypes.c_float), ("growth", ctypes.c_float), ("backoff", ctypes.c_float),
+                ("min_scale", ctypes.c_float), ("max_scale", ctypes.c_float),
+                ("growth_interval", ctypes.c_int32), ("clean_steps", ctypes.c_int32), ("skip", ctypes.c_int32),
+                ("reserved", ctypes.c_int32), ("n_steps", ctypes.c_uint64), ("n_skipped", ctypes.c_uint64)]
+
+
+def dls_update(state: DlsState, stats: np.ndarray) -> None:
+    """One controller step on the statistics records (uint64[n][264]) of a step's gradient tensors."""
+    st = np.ascontiguousarray(stats, dtype=np.uint64).reshape(-1, STATS_WORDS)
+    _L().oracle_dls_update(ctypes.byref(state), st.ctypes.data, st.shape[0])
 
 
 CONV_FWD, CONV_DGRAD, CONV_WGRAD = 0, 1, 2

@@ -488,6 +488,44 @@ void oracle_bias_quantize_stats(const uint32_t *acc, int64_t rows, int64_t cols,
 }
 
 /* ------------------------------------------------------------------------------------------ */
+/* Dynamic loss scaling (Sections II and V use it; the paper cites the method and gives no        */
+/* algorithm).  Rule taken: after a step whose gradient tensors held any overflow, infinity or    */
+/* NaN the step is skipped, the scale is multiplied by `backoff` (not below min_scale) and the    */
+/* count of clean steps restarts; otherwise the count grows, and when it reaches growth_interval   */
+/* the scale is multiplied by `growth` (not above max_scale) and the count restarts.               */
+/* The products are fp32 multiplications.                                                          */
+/* ------------------------------------------------------------------------------------------ */
+typedef struct {
+    float scale, growth, backoff, min_scale, max_scale;
+    int32_t growth_interval, clean_steps, skip, reserved;
+    uint64_t n_steps, n_skipped;
+} dls_t;
+
+void oracle_dls_update(dls_t *st, const uint64_t *stats, int64_t n_records) {
+    uint64_t bad = 0;
+    for (int64_t r = 0; r < n_records; ++r) {
+        const uint64_t *rec = stats + r * ST_WORDS;
+        bad += rec[ST_OVERFLOW] + rec[ST_NAN] + rec[ST_INF_IN];
+    }
+    st->n_steps += 1;
+    if (bad != 0) {
+        float s = st->scale * st->backoff;
+        st->scale = s < st->min_scale ? st->min_scale : s;
+        st->clean_steps = 0;
+        st->skip = 1;
+        st->n_skipped += 1;
+    } else {
+        st->skip = 0;
+        st->clean_steps += 1;
+        if (st->clean_steps >= st->growth_interval) {
+            float s = st->scale * st->growth;
+            st->scale = s > st->max_scale ? st->max_scale : s;
+            st->clean_steps = 0;
+        }
+    }
+}
+
+/* ------------------------------------------------------------------------------------------ */
 /* Contractions (Section III-B, FMACS): exact products summed in fp64 in plain k order, with    */
 /* t = sum |a||b| beside each output for the accumulation-error bound.                          */
 /* Matrices are fp32, row-major with a leading dimension; trans != 0 reads the stored matrix    */

@@ -59,6 +59,13 @@ class qfmt_stats_t(ctypes.Structure):
                 ("n_nan", ctypes.c_uint64), ("n_inf_in", ctypes.c_uint64), ("reserved", ctypes.c_uint64)]
 
 
+class qfmt_dls_t(ctypes.Structure):
+    _fields_ = [("scale", ctypes.c_float), ("growth", ctypes.c_float), ("backoff", ctypes.c_float),
+                ("min_scale", ctypes.c_float), ("max_scale", ctypes.c_float),
+                ("growth_interval", ctypes.c_int32), ("clean_steps", ctypes.c_int32), ("skip", ctypes.c_int32),
+                ("reserved", ctypes.c_int32), ("n_steps", ctypes.c_uint64), ("n_skipped", ctypes.c_uint64)]
+
+
 _lib: Optional[ctypes.CDLL] = None
 
 
@@ -104,6 +111,10 @@ def _bind_optional(L: ctypes.CDLL) -> None:
     L.qfmt_gemm_workspace_bytes.restype = sz
     L.qfmt_gemm_fmac8.argtypes = [matp, matp, vp, ctypes.c_int64, ctypes.POINTER(qfmt_format_t), vp, ci, ci, vp]
     L.qfmt_gemm_fmac8.restype = ci
+    L.qfmt_dls_update.argtypes = [vp, vp, ctypes.c_int64, vp]
+    L.qfmt_dls_update.restype = ci
+    L.qfmt_quantize_stats_dls.argtypes = [vp, vp, sz, ctypes.POINTER(qfmt_format_t), vp, vp, ci, vp]
+    L.qfmt_quantize_stats_dls.restype = ci
     L.qfmt_gemm_tile_policy.argtypes = [ci]
     L.qfmt_gemm_tile_policy.restype = ci
     L.qfmt_device_status.argtypes = [vp, vp]
@@ -216,6 +227,19 @@ def qfmt_gemm_fmac8(A: qfmt_matrix_t, B: qfmt_matrix_t, d_C, ldc: int, fmt: qfmt
     """C = op(A) op(B) with FMAC-8 accumulation (Algorithm 1); see qfmt_gemm_fmac8 in include/qfmt.h."""
     _check(lib().qfmt_gemm_fmac8(ctypes.byref(A), ctypes.byref(B), _ptr(d_C), int(ldc), ctypes.byref(fmt),
                                  _ptr(d_stats), int(accumulate), int(path), _stream_handle(stream)), "qfmt_gemm_fmac8")
+
+
+def qfmt_dls_update(d_state, d_stats, n_records: int, stream=None) -> None:
+    """One dynamic-loss-scale controller step on device records; see qfmt_dls_update in include/qfmt.h."""
+    _check(lib().qfmt_dls_update(_ptr(d_state), _ptr(d_stats), int(n_records), _stream_handle(stream)), "qfmt_dls_update")
+
+
+def qfmt_quantize_stats_dls(d_in, d_out, n: int, fmt: qfmt_format_t, d_state, d_stats=None, accumulate: int = 0,
+                            stream=None) -> None:
+    """qfmt_quantize_stats with the loss scale read from a device-resident qfmt_dls_t; see include/qfmt.h."""
+    _check(lib().qfmt_quantize_stats_dls(_ptr(d_in), _ptr(d_out), int(n), ctypes.byref(fmt), _ptr(d_state),
+                                         _ptr(d_stats), int(accumulate), _stream_handle(stream)),
+           "qfmt_quantize_stats_dls")
 
 
 def qfmt_device_status(d_workspace, stream=None) -> int:

@@ -51,8 +51,9 @@ template <bool kOut, bool kStats, bool kScale>
 __global__ void __launch_bounds__(kThreads)
 quantize_stats_kernel(const uint32_t* in, uint32_t* out, uint32_t head,
                       unsigned long long n4, uint32_t tail, QuantParams p, qfmt_stats_t* __restrict__ stats,
-                      unsigned long long n_total) {
+                      unsigned long long n_total, const float* __restrict__ d_scale) {
     extern __shared__ uint32_t lane_hist[];  // [(top + kExtraBins)][32]
+    if (kScale && d_scale != nullptr) p.scale = *d_scale;  // loss scale kept on the device (dynamic loss scaling)
     const int nbins = p.top + kExtraBins;
     const int lane = threadIdx.x & 31;
     if (kStats) {
@@ -116,8 +117,9 @@ quantize_stats_kernel(const uint32_t* in, uint32_t* out, uint32_t head,
 template <bool kOut, bool kStats, bool kScale>
 __global__ void __launch_bounds__(kThreads)
 quantize_stats_scalar_kernel(const uint32_t* in, uint32_t* out, unsigned long long n,
-                             QuantParams p, qfmt_stats_t* __restrict__ stats) {
+                             QuantParams p, qfmt_stats_t* __restrict__ stats, const float* __restrict__ d_scale) {
     extern __shared__ uint32_t lane_hist[];
+    if (kScale && d_scale != nullptr) p.scale = *d_scale;
     const int nbins = p.top + kExtraBins;
     const int lane = threadIdx.x & 31;
     if (kStats) {
@@ -374,7 +376,7 @@ bias_quantize_stats_scalar_kernel(const uint32_t* acc, long long ld_acc, const u
 
 template <bool kOut, bool kStats, bool kScale>
 cudaError_t launch(const uint32_t* in, uint32_t* out, size_t n, const QuantParams& p, qfmt_stats_t* stats,
-                   int sm_count, cudaStream_t stream) {
+                   int sm_count, cudaStream_t stream, const float* d_scale) {
     const size_t smem = kStats ? (size_t)(p.top + kExtraBins) * 32 * sizeof(uint32_t) : 0;
     const uintptr_t ai = reinterpret_cast<uintptr_t>(in), ao = reinterpret_cast<uintptr_t>(out);
     const bool same_phase = !kOut || ((ai & 15u) == (ao & 15u));
@@ -396,14 +398,14 @@ cudaError_t launch(const uint32_t* in, uint32_t* out, size_t n, const QuantParam
         if (want > cap) want = cap;
         if (want == 0) want = 1;
         kern<<<(unsigned)want, kThreads, smem, stream>>>(in, out, (uint32_t)head, n4, tail, p, stats,
-                                                         (unsigned long long)n);
+                                                         (unsigned long long)n, d_scale);
     } else {
         auto kern = quantize_stats_scalar_kernel<kOut, kStats, kScale>;
         unsigned long long want = (n + kThreads - 1) / kThreads;
         const unsigned long long cap = (unsigned long long)sm_count * 4;
         if (want > cap) want = cap;
         if (want == 0) want = 1;
-        kern<<<(unsigned)want, kThreads, smem, stream>>>(in, out, (unsigned long long)n, p, stats);
+        kern<<<(unsigned)want, kThreads, smem, stream>>>(in, out, (unsigned long long)n, p, stats, d_scale);
     }
     return cudaGetLastError();
 }
@@ -411,7 +413,7 @@ cudaError_t launch(const uint32_t* in, uint32_t* out, size_t n, const QuantParam
 }  // namespace
 
 int quantize_stats_device(const float* d_in, float* d_out, size_t n, const qfmt_format_t* fmt,
-                          qfmt_stats_t* d_stats, int accumulate, cudaStream_t stream) {
+                          qfmt_stats_t* d_stats, int accumulate, cudaStream_t stream, const float* d_scale) {
     int rc = validate_format(fmt);
     if (rc != QFMT_OK) return rc;
     if (accumulate != 0 && accumulate != 1) return QFMT_ERR_BAD_ARG;
@@ -429,9 +431,10 @@ int quantize_stats_device(const float* d_in, float* d_out, size_t n, const qfmt_
     const QuantParams p = make_params(*fmt);
     const uint32_t* in = reinterpret_cast<const uint32_t*>(d_in);
     uint32_t* out = reinterpret_cast<uint32_t*>(d_out);
-    const bool has_out = d_out != nullptr, has_stats = d_stats != nullptr, has_scale = fmt->loss_scale != 1.0f;
+    const bool has_out = d_out != nullptr, has_stats = d_stats != nullptr;
+    const bool has_scale = fmt->loss_scale != 1.0f || d_scale != nullptr;
     cudaError_t err;
-#define QFMT_DISPATCH(O, S, C) err = launch<O, S, C>(in, out, n, p, d_stats, dev.sm_count, stream)
+#define QFMT_DISPATCH(O, S, C) err = launch<O, S, C>(in, out, n, p, d_stats, dev.sm_count, stream, d_scale)
     if (has_out && has_stats) { if (has_scale) QFMT_DISPATCH(true, true, true); else QFMT_DISPATCH(true, true, false); }
     else if (has_out) { if (has_scale) QFMT_DISPATCH(true, false, true); else QFMT_DISPATCH(true, false, false); }
     else { if (has_scale) QFMT_DISPATCH(false, true, true); else QFMT_DISPATCH(false, true, false); }
@@ -544,7 +547,7 @@ int bias_quantize_stats_device(const float* d_acc, int64_t ld_acc, const float* 
 
 extern "C" int qfmt_quantize_stats(const float* d_in, float* d_out, size_t n, const qfmt_format_t* fmt,
                                    qfmt_stats_t* d_stats, int accumulate, void* stream) {
-    return qfmt::quantize_stats_device(d_in, d_out, n, fmt, d_stats, accumulate, (cudaStream_t)stream);
+    return qfmt::quantize_stats_device(d_in, d_out, n, fmt, d_stats, accumulate, (cudaStream_t)stream, nullptr);
 }
 
 extern "C" int qfmt_quantize_stats_transpose(const float* d_in, float* d_out, int64_t batch, int64_t rows, int64_t cols,
@@ -570,7 +573,8 @@ extern "C" int qfmt_quantize_stats_host(const float* h_in, float* h_out, size_t 
     qfmt_stats_t* d_stats = reinterpret_cast<qfmt_stats_t*>(reinterpret_cast<char*>(d_work) +
                                                             ((n * sizeof(float) + 255u) & ~(size_t)255u));
     if (n) QFMT_CUDA_TRY(cudaMemcpyAsync(d_buf, h_in, n * sizeof(float), cudaMemcpyHostToDevice, stream));
-    rc = qfmt::quantize_stats_device(d_buf, h_out ? d_buf : nullptr, n, fmt, h_stats ? d_stats : nullptr, 0, stream);
+    rc = qfmt::quantize_stats_device(d_buf, h_out ? d_buf : nullptr, n, fmt, h_stats ? d_stats : nullptr, 0, stream,
+                                     nullptr);
     if (rc != QFMT_OK) return rc;
     if (n && h_out) QFMT_CUDA_TRY(cudaMemcpyAsync(h_out, d_buf, n * sizeof(float), cudaMemcpyDeviceToHost, stream));
     if (h_stats) QFMT_CUDA_TRY(cudaMemcpyAsync(h_stats, d_stats, sizeof(qfmt_stats_t), cudaMemcpyDeviceToHost, stream));
