@@ -17,7 +17,7 @@
 //     last place cannot create or hide a tie.
 //   * fmac8_f16_kernel, 1/5/10: fma.rn.f16x2 is this very operation for IEEE binary16 with
 //     denormals; flushing formats clear results below 2^-14 afterwards.
-// Both keep a 128 x 64 (resp. 128 x 128) tile of outputs per block in registers and stream
+// They keep a 64 x 64 (resp. 64 x 128) tile of outputs per block in registers and stream
 // 32-deep slices of the operands through shared memory.
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
@@ -146,10 +146,13 @@ __device__ __forceinline__ void merge_block_hist(qfmt_stats_t* stats, const Quan
 }
 
 // ---- any format with e <= 7, m <= 10 --------------------------------------------------------
-constexpr int kFmBM = 128, kFmBN = 64, kFmTM = 8, kFmTN = 4;
+// 4 x 4 outputs per thread: the FMAC chain of one output is a dozen dependent instructions, so
+// many resident warps (four blocks per SM) hide more latency than a larger patch per thread would.
+constexpr int kFmBM = 64, kFmBN = 64, kFmTM = 4, kFmTN = 4;
+constexpr int kFmBlocksPerSm = 4;
 
 template <bool kStats, bool kFlush, bool kCap>
-__global__ void __launch_bounds__(kFmThreads, 2)
+__global__ void __launch_bounds__(kFmThreads, kFmBlocksPerSm)
 fmac8_kernel(FmacParams g, QuantParams p, qfmt_stats_t* __restrict__ stats) {
     __shared__ __align__(16) float As[kFmBK][kFmBM + 4];
     __shared__ __align__(16) float Bs[kFmBK][kFmBN + 4];
@@ -185,9 +188,8 @@ fmac8_kernel(FmacParams g, QuantParams p, qfmt_stats_t* __restrict__ stats) {
 #pragma unroll
                 for (int kk = 0; kk < kGroup; ++kk) {
                     const float4 a0 = *reinterpret_cast<const float4*>(&As[kg + kk][ty * kFmTM]);
-                    const float4 a1 = *reinterpret_cast<const float4*>(&As[kg + kk][ty * kFmTM + 4]);
                     const float4 b0 = *reinterpret_cast<const float4*>(&Bs[kg + kk][tx * kFmTN]);
-                    const float a[kFmTM] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+                    const float a[kFmTM] = {a0.x, a0.y, a0.z, a0.w};
                     const float b[kFmTN] = {b0.x, b0.y, b0.z, b0.w};
 #pragma unroll
                     for (int i = 0; i < kFmTM; ++i)
@@ -210,7 +212,8 @@ fmac8_kernel(FmacParams g, QuantParams p, qfmt_stats_t* __restrict__ stats) {
 }
 
 // ---- 1/5/10: the hardware's own half-precision FMA ------------------------------------------
-constexpr int kHfBM = 128, kHfBN = 128, kHfTM = 8, kHfTN = 8;
+constexpr int kHfBM = 64, kHfBN = 128, kHfTM = 4, kHfTN = 8;
+constexpr int kHfBlocksPerSm = 2;
 
 __device__ __forceinline__ __half2 hfma2_ieee(__half2 a, __half2 b, __half2 c) {
     uint32_t r;
@@ -249,7 +252,7 @@ __device__ __forceinline__ void fetch_slice(float (&v)[kRows * kFmBK / kFmThread
 }
 
 template <bool kStats, bool kFlush>
-__global__ void __launch_bounds__(kFmThreads, 1)
+__global__ void __launch_bounds__(kFmThreads, kHfBlocksPerSm)
 fmac8_f16_kernel(FmacParams g, QuantParams p, qfmt_stats_t* __restrict__ stats) {
     __shared__ __align__(16) uint32_t As2[kFmBK][kHfBM + 4];  // each A value twice: {a, a} as f16x2
     __shared__ __align__(16) __half Bs[kFmBK][kHfBN + 8];
@@ -262,8 +265,7 @@ fmac8_f16_kernel(FmacParams g, QuantParams p, qfmt_stats_t* __restrict__ stats) 
     }
     const int tx = threadIdx.x % 16, ty = threadIdx.x / 16;
     const int tiles_n = (g.N + kHfBN - 1) / kHfBN, tiles_m = (g.M + kHfBM - 1) / kHfBM;
-    constexpr int kPer = kHfBM * kFmBK / kFmThreads;  // elements of each operand a thread moves per slice
-    static_assert(kHfBM == kHfBN, "one fetch count for both operands");
+    constexpr int kPerA = kHfBM * kFmBK / kFmThreads, kPerB = kHfBN * kFmBK / kFmThreads;  // elements a thread moves
     for (long long tile = blockIdx.x; tile < (long long)tiles_m * tiles_n; tile += gridDim.x) {
         const int m0 = (int)(tile / tiles_n) * kHfBM, n0 = (int)(tile % tiles_n) * kHfBN;
         float master[kHfTM][kHfTN];
@@ -276,18 +278,22 @@ fmac8_f16_kernel(FmacParams g, QuantParams p, qfmt_stats_t* __restrict__ stats) 
 #pragma unroll
             for (int j = 0; j < kHfTN / 2; ++j) small[i][j] = zero2;
         }
-        float fa[kPer], fb[kPer];  // the next slice, on its way from global memory while this one is used
+        float fa[kPerA], fb[kPerB];  // the next slice, on its way from global memory while this one is used
         fetch_slice<kHfBM>(fa, g.A, g.lda, !g.transA, m0, g.M, 0, g.K);
         fetch_slice<kHfBN>(fb, g.B, g.ldb, g.transB, n0, g.N, 0, g.K);
         for (int k0 = 0; k0 < g.K; k0 += kFmBK) {
             __syncthreads();  // the previous slice is no longer read
+            // the conversions are exact: operands hold binary16 values
 #pragma unroll
-            for (int t = 0; t < kPer; ++t) {
+            for (int t = 0; t < kPerA; ++t) {
                 const int idx = threadIdx.x + t * kFmThreads;
-                // the conversions are exact: operands hold binary16 values
                 const uint32_t ha = __half_as_ushort(__float2half_rn(fa[t]));
                 if (!g.transA) As2[idx % kFmBK][idx / kFmBK] = ha | (ha << 16);
                 else As2[idx / kHfBM][idx % kHfBM] = ha | (ha << 16);
+            }
+#pragma unroll
+            for (int t = 0; t < kPerB; ++t) {
+                const int idx = threadIdx.x + t * kFmThreads;
                 if (g.transB) Bs[idx % kFmBK][idx / kFmBK] = __float2half_rn(fb[t]);
                 else Bs[idx / kHfBN][idx % kHfBN] = __float2half_rn(fb[t]);
             }
@@ -302,9 +308,8 @@ fmac8_f16_kernel(FmacParams g, QuantParams p, qfmt_stats_t* __restrict__ stats) 
 #pragma unroll
                 for (int kk = 0; kk < kGroup; ++kk) {
                     const uint4 a0 = *reinterpret_cast<const uint4*>(&As2[kg + kk][ty * kHfTM]);
-                    const uint4 a1 = *reinterpret_cast<const uint4*>(&As2[kg + kk][ty * kHfTM + 4]);
                     const uint4 bv = *reinterpret_cast<const uint4*>(&Bs[kg + kk][tx * kHfTN]);  // 8 halves
-                    const uint32_t aw[kHfTM] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+                    const uint32_t aw[kHfTM] = {a0.x, a0.y, a0.z, a0.w};
                     const uint32_t bw[kHfTN / 2] = {bv.x, bv.y, bv.z, bv.w};
 #pragma unroll
                     for (int i = 0; i < kHfTM; ++i) {
@@ -375,7 +380,8 @@ int gemm_fmac8_device(const qfmt_matrix_t* A, const qfmt_matrix_t* B, float* d_C
     const bool use_native = native && path != 1;
     if (use_native) {
         const long long tiles = ((M + kHfBM - 1) / kHfBM) * ((N + kHfBN - 1) / kHfBN);
-        const unsigned grid = (unsigned)(tiles < dev.sm_count ? tiles : dev.sm_count);
+        const long long slots = (long long)dev.sm_count * kHfBlocksPerSm;
+        const unsigned grid = (unsigned)(tiles < slots ? tiles : slots);
         const bool flush = fmt->denormals == 0;
         if (has_stats) {
             if (flush) fmac8_f16_kernel<true, true><<<grid, kFmThreads, smem, stream>>>(g, p, d_stats);
@@ -386,7 +392,7 @@ int gemm_fmac8_device(const qfmt_matrix_t* A, const qfmt_matrix_t* B, float* d_C
         }
     } else {
         const long long tiles = ((M + kFmBM - 1) / kFmBM) * ((N + kFmBN - 1) / kFmBN);
-        const long long cap = (long long)dev.sm_count * 2;
+        const long long cap = (long long)dev.sm_count * kFmBlocksPerSm;
         const unsigned grid = (unsigned)(tiles < cap ? tiles : cap);
         const bool flush = fmt->denormals == 0, cap_exp = fmt->e == 7;
         const size_t sm = has_stats ? smem : 0;
