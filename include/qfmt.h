@@ -232,6 +232,33 @@ int qfmt_gemm(const qfmt_matrix_t* A, const qfmt_matrix_t* B, float* d_C, int64_
 size_t qfmt_gemm_workspace_bytes(const qfmt_matrix_t* A, const qfmt_matrix_t* B);
 
 /*
+ * Forward pass of a fully connected layer as Section IV-A's worked example states it,
+ *     Y = R( R( op(A) op(B) ) + R(bias) ),
+ * with the FMACS contraction of qfmt_gemm inside and the statistics of Y recorded: qfmt_gemm
+ * followed by qfmt_bias_quantize_stats, in one call.  When the contraction length K is at most
+ * 1024 and e <= 7, both roundings, the bias addition and the counting happen in the GEMM kernel
+ * itself, on the sums while they are still in registers: the fp32 product never goes to memory
+ * and the layer output is written once.  Otherwise the two kernels run one after the other, in
+ * place on d_Y.  The fused kernel sums K in one piece; its result has the bits of the two entry
+ * points called in turn whenever qfmt_gemm does not split K for the problem (it may for products
+ * with few output tiles, and then the two results agree within qfmt_gemm's error bound before the
+ * final roundings).
+ *
+ *   A, B, fmt        as for qfmt_gemm (operands hold format values); fmt->loss_scale must be 1
+ *   d_bias           device, N floats (raw fp32; rounded inside the call)
+ *   d_Y, ldy         device, M x N, leading dimension ldy >= N; receives Y (format values)
+ *   d_stats, accumulate   as for qfmt_bias_quantize_stats (d_stats may be NULL)
+ *   d_workspace      device, 16-byte aligned, at least qfmt_linear_forward_workspace_bytes(A, B)
+ *                    bytes: status word as for qfmt_gemm (qfmt_device_status reads it), split-K
+ *                    partial sums when the kernels run separately, and the rounded bias
+ * Errors: as qfmt_gemm and qfmt_bias_quantize_stats; QFMT_ERR_BAD_FORMAT also for loss_scale != 1.
+ */
+int qfmt_linear_forward(const qfmt_matrix_t* A, const qfmt_matrix_t* B, const float* d_bias, float* d_Y, int64_t ldy,
+                        const qfmt_format_t* fmt, qfmt_stats_t* d_stats, int accumulate, void* d_workspace,
+                        size_t workspace_bytes, void* stream);
+size_t qfmt_linear_forward_workspace_bytes(const qfmt_matrix_t* A, const qfmt_matrix_t* B);
+
+/*
  * C = op(A) op(B) with FMAC-8 accumulation (Algorithm 1), for hardware that only offers the FMAC
  * instruction of Section III-B, a16 = round(a16 + x16 * y16) (one rounding, to the 16-bit format).
  * Every output is computed as the algorithm states: a format-precision accumulator takes eight

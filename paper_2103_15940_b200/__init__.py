@@ -115,6 +115,10 @@ def _bind_optional(L: ctypes.CDLL) -> None:
     L.qfmt_dls_update.restype = ci
     L.qfmt_quantize_stats_dls.argtypes = [vp, vp, sz, ctypes.POINTER(qfmt_format_t), vp, vp, ci, vp]
     L.qfmt_quantize_stats_dls.restype = ci
+    L.qfmt_linear_forward.argtypes = [matp, matp, vp, vp, ctypes.c_int64, ctypes.POINTER(qfmt_format_t), vp, ci, vp, sz, vp]
+    L.qfmt_linear_forward.restype = ci
+    L.qfmt_linear_forward_workspace_bytes.argtypes = [matp, matp]
+    L.qfmt_linear_forward_workspace_bytes.restype = sz
     L.qfmt_gemm_tile_policy.argtypes = [ci]
     L.qfmt_gemm_tile_policy.restype = ci
     L.qfmt_device_status.argtypes = [vp, vp]
@@ -240,6 +244,18 @@ def qfmt_quantize_stats_dls(d_in, d_out, n: int, fmt: qfmt_format_t, d_state, d_
     _check(lib().qfmt_quantize_stats_dls(_ptr(d_in), _ptr(d_out), int(n), ctypes.byref(fmt), _ptr(d_state),
                                          _ptr(d_stats), int(accumulate), _stream_handle(stream)),
            "qfmt_quantize_stats_dls")
+
+
+def qfmt_linear_forward_workspace_bytes(A: qfmt_matrix_t, B: qfmt_matrix_t) -> int:
+    return int(lib().qfmt_linear_forward_workspace_bytes(ctypes.byref(A), ctypes.byref(B)))
+
+
+def qfmt_linear_forward(A: qfmt_matrix_t, B: qfmt_matrix_t, d_bias, d_Y, ldy: int, fmt: qfmt_format_t, d_stats,
+                        accumulate: int, d_workspace, workspace_bytes: int, stream=None) -> None:
+    """Y = R(R(op(A) op(B)) + R(bias)) with the statistics of Y; see qfmt_linear_forward in include/qfmt.h."""
+    _check(lib().qfmt_linear_forward(ctypes.byref(A), ctypes.byref(B), _ptr(d_bias), _ptr(d_Y), int(ldy),
+                                     ctypes.byref(fmt), _ptr(d_stats), int(accumulate), _ptr(d_workspace),
+                                     int(workspace_bytes), _stream_handle(stream)), "qfmt_linear_forward")
 
 
 def qfmt_device_status(d_workspace, stream=None) -> int:

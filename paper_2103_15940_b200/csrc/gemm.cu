@@ -38,6 +38,7 @@
 
 #include "common.cuh"
 #include "ptx.cuh"
+#include "round.cuh"
 
 namespace qfmt {
 namespace {
@@ -64,7 +65,10 @@ constexpr int kOutCols = 32;
 constexpr uint32_t kOutBoxBytes = 32 * 32 * 4;
 constexpr uint32_t kOutWarpBytes = 2 * kOutBoxBytes;
 constexpr uint32_t kOutBytes = kAccWarps * kOutWarpBytes;
-constexpr uint32_t kSmemBytes = kStages * kStageBytes + kOutBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+// Layer-output epilogue (Y = R(R(acc) + R(B)) with statistics): one counter per bin for the CTA.
+constexpr int kEpiBins = 160;  // 2^7 - 1 + the split bins, rounded up (formats with e <= 7)
+constexpr uint32_t kEpiHistBytes = kEpiBins * 4;
+constexpr uint32_t kSmemBytes = kStages * kStageBytes + kOutBytes + 1024 /*alignment slack*/ + 256 /*barriers*/ + kEpiHistBytes;
 constexpr uint32_t kWaitLimit = 1u << 31;  // SM cycles (about a second) before a wait is declared dead
 
 struct GemmParams {
@@ -107,6 +111,13 @@ struct GemmParams {
     int cblocks, ck;       // mode 1: 32-channel blocks per tap and contraction channels; mode 2: ck = C_in
     int tap_sign, off_h, off_w;  // activation row read for tap (r, s): h + tap_sign * r + off_h
     int full_tiles_m;      // mode 1: M-tiles that are complete (the C tensor map covers exactly these)
+    // ---- layer-output epilogue (dense mode, one summation group, no split K): the sums are rounded,
+    // the rounded bias of their column is added, the result is rounded again and counted, all in the
+    // accumulate warps' registers before the tile is stored
+    int epi;                  // 0 = off
+    const float* epi_rbias;   // rounded bias, padded with zeros to tiles_n * kBN entries
+    qfmt_stats_t* epi_stats;  // may be null
+    QuantParams epi_q;
 };
 
 // Mode 1 reads the pixel operand through maps whose boxes hold 1 .. kMaxRowMaps whole image rows
@@ -199,6 +210,53 @@ __device__ __forceinline__ void raise_timeout(const GemmParams& p, volatile int*
     atomicCAS(p.status, 0, (int)QFMT_ERR_TIMEOUT);
 }
 
+// Layer-output epilogue on one thread's 128 sums of a row (columns col_base + 0..127; sum2[i] holds
+// columns 2i and 2i+1): Y = R(R(acc) + R(B)) of Section IV-A's worked example, then one count per
+// element in the CTA's histogram.  Lanes of a warp hold different rows of the same column, so equal
+// bins are common: the lanes that share a bin elect one of them to add their number.
+__device__ __forceinline__ void epi_transform(unsigned long long (&sum2)[64], const GemmParams& p, bool row_ok,
+                                              int col_base, uint32_t* hist, int lane) {
+    const uint32_t inf_bits = (uint32_t)(p.epi_q.top + p.epi_q.code_off) << 23;
+    const bool count = p.epi_stats != nullptr;
+#pragma unroll  // fully: sum2 must stay in registers
+    for (int i = 0; i < 64; ++i) {
+        const int col = col_base + 2 * i;
+        const float2 rb = *reinterpret_cast<const float2*>(p.epi_rbias + col);  // same address for the whole warp
+        const float2 v = ptx::unpack2(sum2[i]);
+        int b0, b1;
+        const uint32_t r0 = round_value<false>(__float_as_uint(v.x), p.epi_q, inf_bits);
+        const uint32_t r1 = round_value<false>(__float_as_uint(v.y), p.epi_q, inf_bits);
+        const uint32_t q0 = round_sum(__float_as_uint(add_ieee(__uint_as_float(r0), rb.x)), p.epi_q, b0);
+        const uint32_t q1 = round_sum(__float_as_uint(add_ieee(__uint_as_float(r1), rb.y)), p.epi_q, b1);
+        sum2[i] = ptx::pack2(__uint_as_float(q0), __uint_as_float(q1));
+        if (count) {
+            const bool ok0 = row_ok && col < p.N, ok1 = row_ok && col + 1 < p.N;
+            const unsigned m0 = __ballot_sync(0xFFFFFFFFu, ok0);
+            if (ok0) {
+                const unsigned same = __match_any_sync(m0, b0);
+                if (lane == __ffs(same) - 1) atomicAdd(&hist[b0], (uint32_t)__popc(same));
+            }
+            const unsigned m1 = __ballot_sync(0xFFFFFFFFu, ok1);
+            if (ok1) {
+                const unsigned same = __match_any_sync(m1, b1);
+                if (lane == __ffs(same) - 1) atomicAdd(&hist[b1], (uint32_t)__popc(same));
+            }
+        }
+    }
+}
+
+// Folds the CTA's epilogue histogram into the device record (all threads of the CTA call it).
+__device__ __forceinline__ void epi_merge(const GemmParams& p, const uint32_t* hist) {
+    if (!p.epi || p.epi_stats == nullptr) return;
+    const int nbins = p.epi_q.top + kExtraBins;
+    for (int b = 1 + (int)threadIdx.x; b < nbins; b += kThreads) {
+        const uint32_t c = hist[b];
+        if (c != 0u) merge_bin(p.epi_stats, p.epi_q, b, c);
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0)
+        atomicAdd((unsigned long long*)&p.epi_stats->n_total, (unsigned long long)p.M * (unsigned long long)p.N);
+}
+
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tf32_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                  const __grid_constant__ CUtensorMap tmap_c, const __grid_constant__ CUtensorMap tmap_p,
@@ -219,9 +277,13 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     volatile int* abort_flag = reinterpret_cast<volatile int*>(gen_bars + 8 * (2 * kStages + 4) + 8);
     // issue_progress[i]: chunks (counted over the whole kernel) up to which MMA issuer i has seen its operands arrive
     volatile uint32_t* issue_progress = reinterpret_cast<volatile uint32_t*>(gen_bars + 8 * (2 * kStages + 4) + 16);
+    uint32_t* epi_hist = reinterpret_cast<uint32_t*>(gen_bars + 256);
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
+    if (p.epi) {
+        for (int i = threadIdx.x; i < kEpiBins; i += kThreads) epi_hist[i] = 0u;
+    }
 
     if (p.mode == 2) {
         // Filter gradient: a stage holds fewer than 32 pixel rows of K; the rows TMA never writes
@@ -539,6 +601,7 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                 if (!last && ++in_group < kFlushChunks) continue;
                 // ---- move the level-1 sums to C (level 2): registers -> swizzled shared boxes -> TMA.
                 // The first group of a tile is stored, later groups are added at the destination.
+                if (p.epi) epi_transform(sum2, p, row0 + lane < m_end, n0 + half * 128, epi_hist, lane);
                 if (use_tma && flushed) {
                     if (lane == 0) ptx::bulk_wait_all();  // the earlier store/add to these addresses is complete
                 }
@@ -601,6 +664,7 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     // ------------------------------ common exit ------------------------------
     ptx::tc_fence_before_sync();
     __syncthreads();
+    epi_merge(p, epi_hist);
     if (*abort_flag) {
         // give TMA copies that may still be in flight time to land before the CTA's shared
         // memory is handed to another CTA
@@ -631,7 +695,7 @@ constexpr int kPStages = 5;
 constexpr uint32_t kPABytes = kBM * kBK * 4;          // 128 rows of A
 constexpr uint32_t kPBBytes = (kBN / 2) * kBK * 4;    // 128 of the tile's 256 columns of B
 constexpr uint32_t kPStageBytes = kPABytes + kPBBytes;
-constexpr uint32_t kPairSmemBytes = kPStages * kPStageBytes + kOutBytes + 1024 + 256;
+constexpr uint32_t kPairSmemBytes = kPStages * kPStageBytes + kOutBytes + 1024 + 256 + kEpiHistBytes;
 
 __device__ __forceinline__ uint32_t make_idesc_pair(int a_mn, int b_mn) {
     return (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)a_mn << 15) | ((uint32_t)b_mn << 16)
@@ -653,10 +717,14 @@ gemm_tf32_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
     uint8_t* gen_bars = smem_raw + (bars - raw);
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen_bars + 8 * (2 * kPStages + 4));
     volatile int* abort_flag = reinterpret_cast<volatile int*>(gen_bars + 8 * (2 * kPStages + 4) + 8);
+    uint32_t* epi_hist = reinterpret_cast<uint32_t*>(gen_bars + 256);
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     const uint32_t rank = ptx::cluster_ctarank();  // 0 = leader
+    if (p.epi) {
+        for (int i = threadIdx.x; i < kEpiBins; i += kThreads) epi_hist[i] = 0u;
+    }
     const int cluster_id = blockIdx.x >> 1, num_clusters = gridDim.x >> 1;
 
     if (threadIdx.x == 0) {
@@ -845,6 +913,7 @@ gemm_tf32_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
                 ++acc_iter;
                 const bool last = kb0 + kChunkKB >= num_kb;
                 if (!last && ++in_group < kFlushChunks) continue;
+                if (p.epi) epi_transform(sum2, p, row0 + lane < m_end, n0 + half * 128, epi_hist, lane);
                 if (use_tma && flushed) {
                     if (lane == 0) ptx::bulk_wait_all();
                 }
@@ -903,6 +972,7 @@ gemm_tf32_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
     // ------------------------------ common exit ------------------------------
     ptx::tc_fence_before_sync();
     __syncthreads();
+    epi_merge(p, epi_hist);
     if (*abort_flag) {
         for (int i = 0; i < 2000; ++i) __nanosleep(1000);
     }
@@ -1049,6 +1119,9 @@ void dense_defaults(GemmParams* p) {
     p->sk_cpt = 0;
     p->sk_pieces = 1;
     p->sk_partials = nullptr;
+    p->epi = 0;
+    p->epi_rbias = nullptr;
+    p->epi_stats = nullptr;
 }
 
 }  // namespace
@@ -1113,8 +1186,16 @@ int launch_pair(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap&
     return QFMT_OK;
 }
 
+// Layer-output epilogue request for gemm_device: the rounded, zero-padded bias and the record.
+struct EpiArgs {
+    const float* rbias;
+    qfmt_stats_t* stats;
+};
+// The epilogue runs on the sums of one group held in registers: at most this many K elements.
+constexpr int64_t kEpiMaxK = (int64_t)kFlushChunks * kChunkKB * kBK;
+
 int gemm_device(const qfmt_matrix_t* A, const qfmt_matrix_t* B, float* d_C, int64_t ldc, const qfmt_format_t* fmt,
-                void* d_workspace, size_t workspace_bytes, cudaStream_t stream) {
+                void* d_workspace, size_t workspace_bytes, cudaStream_t stream, const EpiArgs* epi = nullptr) {
     int rc = validate_format(fmt);
     if (rc != QFMT_OK) return rc;
     if (fmt->m > 10) return QFMT_ERR_BAD_FORMAT;  // beyond TF32's mantissa: products would not be exact
@@ -1166,7 +1247,16 @@ int gemm_device(const qfmt_matrix_t* A, const qfmt_matrix_t* B, float* d_C, int6
 
     // Split K when the workspace the caller lent has room for the partial sums (the recommended size
     // from qfmt_gemm_workspace_bytes always has); a smaller workspace gets fewer splits.
-    int splits = plan.splits;
+    int splits = epi != nullptr ? 1 : plan.splits;
+    if (epi != nullptr) {
+        if (K > kEpiMaxK || fmt->e > 7) return QFMT_ERR_BAD_ARG;  // callers check before asking
+        qfmt_format_t f = *fmt;
+        f.loss_scale = 1.0f;
+        p.epi = 1;
+        p.epi_rbias = epi->rbias;
+        p.epi_stats = epi->stats;
+        p.epi_q = make_params(f);
+    }
     while (splits > 1 && kWorkspaceHeader + (size_t)splits * (size_t)M * (size_t)N * sizeof(float) > workspace_bytes) --splits;
     float* partials = reinterpret_cast<float*>(reinterpret_cast<char*>(d_workspace) + kWorkspaceHeader);
     if (splits > 1) {
@@ -1476,6 +1566,79 @@ extern "C" size_t qfmt_conv_workspace_bytes(int32_t op, const qfmt_conv_t* geom)
     qfmt::ConvPlan plan;
     if (qfmt::plan_conv(op, geom, &plan) != QFMT_OK) return 0;
     return plan.workspace;
+}
+
+namespace qfmt {
+int bias_quantize_stats_device(const float* d_acc, int64_t ld_acc, const float* d_bias, float* d_out, int64_t ld_out,
+                               int64_t rows, int64_t cols, const qfmt_format_t* fmt, qfmt_stats_t* d_stats,
+                               int accumulate, cudaStream_t stream);
+namespace {
+
+// Rounds the bias vector for the fused epilogue; entries n .. padded-1 become zero.
+__global__ void __launch_bounds__(256)
+round_bias_kernel(const float* __restrict__ bias, float* __restrict__ out, int n, int padded, QuantParams q) {
+    const uint32_t inf_bits = (uint32_t)(q.top + q.code_off) << 23;
+    for (int i = blockIdx.x * 256 + threadIdx.x; i < padded; i += gridDim.x * 256)
+        out[i] = i < n ? __uint_as_float(round_value<false>(__float_as_uint(bias[i]), q, inf_bits)) : 0.0f;
+}
+
+size_t linear_bias_bytes(int64_t N) {  // rounded bias, padded with zeros to whole tiles
+    return (size_t)((N + kBN - 1) / kBN) * kBN * sizeof(float);
+}
+
+}  // namespace
+
+int linear_forward_device(const qfmt_matrix_t* A, const qfmt_matrix_t* B, const float* d_bias, float* d_Y, int64_t ldy,
+                          const qfmt_format_t* fmt, qfmt_stats_t* d_stats, int accumulate, void* d_workspace,
+                          size_t workspace_bytes, cudaStream_t stream) {
+    int rc = validate_format(fmt);
+    if (rc != QFMT_OK) return rc;
+    if (fmt->m > 10 || fmt->loss_scale != 1.0f) return QFMT_ERR_BAD_FORMAT;
+    if (A == nullptr || B == nullptr || d_bias == nullptr) return QFMT_ERR_BAD_ARG;
+    if (accumulate != 0 && accumulate != 1) return QFMT_ERR_BAD_ARG;
+    if ((reinterpret_cast<uintptr_t>(d_bias) & 3u) || (reinterpret_cast<uintptr_t>(d_stats) & 7u)) return QFMT_ERR_BAD_ARG;
+    if (A->rows < 0 || A->cols < 0 || B->rows < 0 || B->cols < 0) return QFMT_ERR_BAD_ARG;
+    const int64_t M = A->trans ? A->cols : A->rows, K = A->trans ? A->rows : A->cols;
+    const int64_t N = B->trans ? B->rows : B->cols;
+    if (M > (1 << 30) || N > (1 << 30) || K > (1 << 30)) return QFMT_ERR_BAD_ARG;
+    if (d_workspace == nullptr || (reinterpret_cast<uintptr_t>(d_workspace) & 15u)) return QFMT_ERR_BAD_ARG;
+    const size_t bias_bytes = linear_bias_bytes(N);
+    if (workspace_bytes < kWorkspaceHeader + bias_bytes + 256) return QFMT_ERR_BAD_ARG;
+    // layout: [status word and padding | GEMM partial sums (unfused path) ... | rounded bias at the end,
+    // on a 256-byte boundary]
+    const size_t gemm_bytes = (workspace_bytes - bias_bytes) & ~(size_t)255u;
+    float* rbias = reinterpret_cast<float*>(reinterpret_cast<char*>(d_workspace) + gemm_bytes);
+    const bool fused = fmt->e <= 7 && K >= 1 && K <= kEpiMaxK && M > 0 && N > 0;
+    if (!fused) {
+        rc = gemm_device(A, B, d_Y, ldy, fmt, d_workspace, gemm_bytes, stream);
+        if (rc != QFMT_OK) return rc;
+        return bias_quantize_stats_device(d_Y, ldy, d_bias, d_Y, ldy, M, N, fmt, d_stats, accumulate, stream);
+    }
+    DeviceInfo dev;
+    rc = current_device(&dev);
+    if (rc != QFMT_OK) return rc;
+    if (d_stats != nullptr && accumulate == 0) QFMT_CUDA_TRY(cudaMemsetAsync(d_stats, 0, sizeof(qfmt_stats_t), stream));
+    const int padded = (int)(((N + kBN - 1) / kBN) * kBN);
+    round_bias_kernel<<<(padded + 255) / 256, 256, 0, stream>>>(d_bias, rbias, (int)N, padded, make_params(*fmt));
+    QFMT_CUDA_TRY(cudaGetLastError());
+    const EpiArgs epi = {rbias, d_stats};
+    return gemm_device(A, B, d_Y, ldy, fmt, d_workspace, gemm_bytes, stream, &epi);
+}
+
+}  // namespace qfmt
+
+extern "C" int qfmt_linear_forward(const qfmt_matrix_t* A, const qfmt_matrix_t* B, const float* d_bias, float* d_Y,
+                                   int64_t ldy, const qfmt_format_t* fmt, qfmt_stats_t* d_stats, int accumulate,
+                                   void* d_workspace, size_t workspace_bytes, void* stream) {
+    return qfmt::linear_forward_device(A, B, d_bias, d_Y, ldy, fmt, d_stats, accumulate, d_workspace, workspace_bytes,
+                                       (cudaStream_t)stream);
+}
+
+extern "C" size_t qfmt_linear_forward_workspace_bytes(const qfmt_matrix_t* A, const qfmt_matrix_t* B) {
+    if (A == nullptr || B == nullptr) return 0;
+    const int64_t N = B->trans ? B->rows : B->cols;
+    if (N < 0 || N > (1 << 30)) return 0;
+    return qfmt_gemm_workspace_bytes(A, B) + qfmt::linear_bias_bytes(N) + 256;
 }
 
 extern "C" int qfmt_gemm_tile_policy(int policy) {

@@ -76,6 +76,52 @@ __device__ __forceinline__ uint32_t quantize_one(uint32_t xb, const QuantParams&
     return sign | qa;
 }
 
+// R(S * x) without statistics, for formats with e <= 7: the first rounding of the layer formula.
+// The integer pipe runs at half the float pipe's rate, so the rounding is two float operations:
+// with C = 1.5 * 2^(max(floor(log2|y|), E_min) + 23 - m) the sum y + C lies in C's binade, whose
+// last place is the format's quantum for y; the IEEE addition rounds there to nearest-even (C is
+// an even multiple of the quantum) and subtracting C is exact.  Normal and denormal results, both
+// signs; a zero result gets y's sign back with an OR.  The exponent is capped at E_max+1 so that C
+// stays finite; whatever reaches 2^(E_max+1) becomes infinite.  (A NaN stays some NaN: the addition
+// that follows makes it the positive quiet NaN whatever its payload.)
+template <bool kScale>
+__device__ __forceinline__ uint32_t round_value(uint32_t xb, const QuantParams& p, uint32_t inf_bits) {
+    const uint32_t yb = kScale ? __float_as_uint(mul_ieee(__uint_as_float(xb), p.scale)) : xb;
+    uint32_t ec = yb & 0x7F800000u;
+    ec = ec < p.min_normal ? p.min_normal : ec;
+    ec = ec > inf_bits ? inf_bits : ec;
+    const float c = __uint_as_float(ec + p.magic_add);
+    float q = sub_ieee(add_ieee(__uint_as_float(yb), c), c);
+    if (!(fabsf(q) < __uint_as_float(inf_bits)) && q == q) q = copysignf(__uint_as_float(0x7F800000u), q);
+    if (!p.keep_denormals && fabsf(q) < __uint_as_float(p.min_normal)) q = 0.0f;
+    return __float_as_uint(q) | (yb & 0x80000000u);
+}
+
+// Second rounding of the layer formula, with the bin: s is the fp32 sum of two format values
+// (e <= 7, so |s| < 2^(E_max+2) and the rounding constant cannot overflow), or inf/NaN.
+__device__ __forceinline__ uint32_t round_sum(uint32_t s, const QuantParams& p, int& bin) {
+    uint32_t ec = s & 0x7F800000u;
+    ec = ec < p.min_normal ? p.min_normal : ec;
+    const float c = __uint_as_float(ec + p.magic_add);
+    const uint32_t sign = s & 0x80000000u;
+    uint32_t q = __float_as_uint(sub_ieee(add_ieee(__uint_as_float(s), c), c)) | sign;
+    const uint32_t aq = q & 0x7FFFFFFFu;
+    const int code = (int)(aq >> 23) - p.code_off;
+    bin = code;
+    if ((unsigned)(code - 1) >= (unsigned)(p.top - 1)) {  // not a normal number of the format
+        const uint32_t as = s & 0x7FFFFFFFu;
+        if (code >= p.top) {
+            const bool is_nan = as > 0x7F800000u;
+            q = is_nan ? 0x7FC00000u : (sign | 0x7F800000u);
+            bin = p.top + (is_nan ? kBinNanIn : (as == 0x7F800000u ? kBinInfIn : kBinOverflow));
+        } else {
+            bin = p.top + (as == 0u ? kBinZeroIn : (aq == 0u ? kBinRoundedToZero : kBinDenormal));
+            if (!p.keep_denormals) q = sign;
+        }
+    }
+    return q;
+}
+
 // Folds one bin's block total into the device record.
 __device__ __forceinline__ void merge_bin(qfmt_stats_t* st, const QuantParams& p, int bin, unsigned long long c) {
     auto add = [](uint64_t* dst, unsigned long long v) { atomicAdd((unsigned long long*)dst, v); };
