@@ -279,7 +279,32 @@ def epilogue_section(torch, qf, dev, peaks, reps=20):
     ms = statistics.median(time_events(torch, step, reps))
     assert int(st.cpu()[256]) == rows * cols
     achieved = rows * cols * BYTES_PER_ELEMENT / ms / 1e6
-    return {"metric": "layer output R(R(acc)+R(B)) + stats GB/s", "value": achieved, "unit": "GB/s",
+    # the whole forward layer through qfmt_linear_forward: default plan (GEMM, then the pass above in place)
+    # and with the epilogue inside the GEMM kernel (K = 1024)
+    wb = qf.qfmt_linear_forward_workspace_bytes(a, b)
+    ws2 = torch.zeros(wb, dtype=torch.uint8, device=dev)
+
+    def layer():
+        qf.qfmt_linear_forward(a, b, bias, out, cols, fmt, st, 0, ws2, wb)
+
+    def gemm_only():
+        qf.qfmt_gemm(a, b, acc, cols, fmt, ws, ws.numel())
+    timings = {}
+    for name, policy in (("two_kernels", 0), ("in_kernel", 1)):
+        qf.qfmt_linear_fusion_policy(policy)
+        for _ in range(3):
+            layer()
+        assert qf.qfmt_device_status(ws2) == qf.QFMT_OK
+        timings[name] = statistics.median(time_events(torch, layer, reps))
+    qf.qfmt_linear_fusion_policy(0)
+    for _ in range(3):
+        gemm_only()
+    gemm_ms = statistics.median(time_events(torch, gemm_only, reps))
+    flops = 2.0 * rows * cols * X.shape[1]
+    linear = {"workload": f"config5 FFN-up forward layer, {rows} x {cols} x {X.shape[1]}, Y = R(R(XW) + R(B)) with statistics",
+              "ms": timings["two_kernels"], "tflops": flops / timings["two_kernels"] / 1e9, "gemm_alone_ms": gemm_ms,
+              "epilogue_in_gemm_kernel_ms": timings["in_kernel"]}
+    return {"metric": "layer output R(R(acc)+R(B)) + stats GB/s", "value": achieved, "unit": "GB/s", "linear_forward": linear,
             "workload": f"config5 FFN-up forward output, {rows} x {cols}, 1/6/9 (268 MB moved per launch, larger than L2)",
             "ms_per_step": ms, "gpu_launches_per_step": 1,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",

@@ -235,14 +235,14 @@ size_t qfmt_gemm_workspace_bytes(const qfmt_matrix_t* A, const qfmt_matrix_t* B)
  * Forward pass of a fully connected layer as Section IV-A's worked example states it,
  *     Y = R( R( op(A) op(B) ) + R(bias) ),
  * with the FMACS contraction of qfmt_gemm inside and the statistics of Y recorded: qfmt_gemm
- * followed by qfmt_bias_quantize_stats, in one call.  When the contraction length K is at most
- * 1024 and e <= 7, both roundings, the bias addition and the counting happen in the GEMM kernel
- * itself, on the sums while they are still in registers: the fp32 product never goes to memory
- * and the layer output is written once.  Otherwise the two kernels run one after the other, in
- * place on d_Y.  The fused kernel sums K in one piece; its result has the bits of the two entry
- * points called in turn whenever qfmt_gemm does not split K for the problem (it may for products
- * with few output tiles, and then the two results agree within qfmt_gemm's error bound before the
- * final roundings).
+ * followed by qfmt_bias_quantize_stats, in one call and in place on d_Y.
+ *
+ * The library can also run both roundings, the bias addition and the counting inside the GEMM
+ * kernel, on the sums while they are still in registers (contraction length K at most 1024 and
+ * e <= 6), so that the fp32 product never goes to memory: see qfmt_linear_fusion_policy.  That
+ * kernel sums K in one piece; its result has the bits of the two entry points called in turn
+ * whenever qfmt_gemm does not split K for the problem (it may for products with few output tiles,
+ * and then the two results agree within qfmt_gemm's error bound before the final roundings).
  *
  *   A, B, fmt        as for qfmt_gemm (operands hold format values); fmt->loss_scale must be 1
  *   d_bias           device, N floats (raw fp32; rounded inside the call)
@@ -257,6 +257,17 @@ int qfmt_linear_forward(const qfmt_matrix_t* A, const qfmt_matrix_t* B, const fl
                         const qfmt_format_t* fmt, qfmt_stats_t* d_stats, int accumulate, void* d_workspace,
                         size_t workspace_bytes, void* stream);
 size_t qfmt_linear_forward_workspace_bytes(const qfmt_matrix_t* A, const qfmt_matrix_t* B);
+
+/*
+ * Tuning and test control (no counterpart in the paper): how qfmt_linear_forward runs.
+ *   0  automatic (default; currently two kernels, which measures faster: the epilogue's integer
+ *      work in the GEMM kernel's few epilogue warps keeps the tensor cores waiting longer than
+ *      the separate full-occupancy pass takes)
+ *   1  epilogue inside the GEMM kernel whenever K <= 1024 and e <= 6
+ *   2  always two kernels
+ * Process-wide and not synchronised with calls in flight.  QFMT_ERR_BAD_ARG for other values.
+ */
+int qfmt_linear_fusion_policy(int policy);
 
 /*
  * C = op(A) op(B) with FMAC-8 accumulation (Algorithm 1), for hardware that only offers the FMAC

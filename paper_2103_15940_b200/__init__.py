@@ -117,6 +117,8 @@ def _bind_optional(L: ctypes.CDLL) -> None:
     L.qfmt_quantize_stats_dls.restype = ci
     L.qfmt_linear_forward.argtypes = [matp, matp, vp, vp, ctypes.c_int64, ctypes.POINTER(qfmt_format_t), vp, ci, vp, sz, vp]
     L.qfmt_linear_forward.restype = ci
+    L.qfmt_linear_fusion_policy.argtypes = [ci]
+    L.qfmt_linear_fusion_policy.restype = ci
     L.qfmt_linear_forward_workspace_bytes.argtypes = [matp, matp]
     L.qfmt_linear_forward_workspace_bytes.restype = sz
     L.qfmt_gemm_tile_policy.argtypes = [ci]
@@ -244,6 +246,11 @@ def qfmt_quantize_stats_dls(d_in, d_out, n: int, fmt: qfmt_format_t, d_state, d_
     _check(lib().qfmt_quantize_stats_dls(_ptr(d_in), _ptr(d_out), int(n), ctypes.byref(fmt), _ptr(d_state),
                                          _ptr(d_stats), int(accumulate), _stream_handle(stream)),
            "qfmt_quantize_stats_dls")
+
+
+def qfmt_linear_fusion_policy(policy: int) -> None:
+    """0 automatic, 1 epilogue inside the GEMM kernel when it applies, 2 two kernels; see include/qfmt.h."""
+    _check(lib().qfmt_linear_fusion_policy(int(policy)), "qfmt_linear_fusion_policy")
 
 
 def qfmt_linear_forward_workspace_bytes(A: qfmt_matrix_t, B: qfmt_matrix_t) -> int:

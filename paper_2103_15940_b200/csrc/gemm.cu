@@ -66,7 +66,7 @@ constexpr uint32_t kOutBoxBytes = 32 * 32 * 4;
 constexpr uint32_t kOutWarpBytes = 2 * kOutBoxBytes;
 constexpr uint32_t kOutBytes = kAccWarps * kOutWarpBytes;
 // Layer-output epilogue (Y = R(R(acc) + R(B)) with statistics): one counter per bin for the CTA.
-constexpr int kEpiBins = 160;  // 2^7 - 1 + the split bins, rounded up (formats with e <= 7)
+constexpr int kEpiBins = 128;  // 2^6 - 1 + the split bins, rounded up (formats with e <= 6)
 constexpr uint32_t kEpiHistBytes = kEpiBins * 4;
 constexpr uint32_t kSmemBytes = kStages * kStageBytes + kOutBytes + 1024 /*alignment slack*/ + 256 /*barriers*/ + kEpiHistBytes;
 constexpr uint32_t kWaitLimit = 1u << 31;  // SM cycles (about a second) before a wait is declared dead
@@ -212,12 +212,22 @@ __device__ __forceinline__ void raise_timeout(const GemmParams& p, volatile int*
 
 // Layer-output epilogue on one thread's 128 sums of a row (columns col_base + 0..127; sum2[i] holds
 // columns 2i and 2i+1): Y = R(R(acc) + R(B)) of Section IV-A's worked example, then one count per
-// element in the CTA's histogram.  Lanes of a warp hold different rows of the same column, so equal
-// bins are common: the lanes that share a bin elect one of them to add their number.
+// element.  The warp counts in its own output staging boxes, idle at this point, used as a
+// histogram of [128 bins][16 slots] (a lane adds to slot lane mod 16, so at most two lanes share a
+// counter); afterwards the slots are summed into the CTA's histogram.  Needs at most 128 bins
+// (e <= 6).
 __device__ __forceinline__ void epi_transform(unsigned long long (&sum2)[64], const GemmParams& p, bool row_ok,
-                                              int col_base, uint32_t* hist, int lane) {
+                                              int col_base, uint32_t* warp_hist, uint32_t* hist, int lane) {
     const uint32_t inf_bits = (uint32_t)(p.epi_q.top + p.epi_q.code_off) << 23;
     const bool count = p.epi_stats != nullptr;
+    if (count) {
+        if (lane == 0) ptx::bulk_wait_read_all();  // copies of the previous tile no longer read the boxes
+        __syncwarp();
+#pragma unroll
+        for (int i = 0; i < 64; ++i) warp_hist[i * 32 + lane] = 0u;
+        __syncwarp();
+    }
+    const int slot = lane & 15;
 #pragma unroll  // fully: sum2 must stay in registers
     for (int i = 0; i < 64; ++i) {
         const int col = col_base + 2 * i;
@@ -229,19 +239,21 @@ __device__ __forceinline__ void epi_transform(unsigned long long (&sum2)[64], co
         const uint32_t q0 = round_sum(__float_as_uint(add_ieee(__uint_as_float(r0), rb.x)), p.epi_q, b0);
         const uint32_t q1 = round_sum(__float_as_uint(add_ieee(__uint_as_float(r1), rb.y)), p.epi_q, b1);
         sum2[i] = ptx::pack2(__uint_as_float(q0), __uint_as_float(q1));
-        if (count) {
-            const bool ok0 = row_ok && col < p.N, ok1 = row_ok && col + 1 < p.N;
-            const unsigned m0 = __ballot_sync(0xFFFFFFFFu, ok0);
-            if (ok0) {
-                const unsigned same = __match_any_sync(m0, b0);
-                if (lane == __ffs(same) - 1) atomicAdd(&hist[b0], (uint32_t)__popc(same));
-            }
-            const unsigned m1 = __ballot_sync(0xFFFFFFFFu, ok1);
-            if (ok1) {
-                const unsigned same = __match_any_sync(m1, b1);
-                if (lane == __ffs(same) - 1) atomicAdd(&hist[b1], (uint32_t)__popc(same));
-            }
+        if (count && row_ok) {
+            if (col < p.N) atomicAdd(&warp_hist[b0 * 16 + slot], 1u);
+            if (col + 1 < p.N) atomicAdd(&warp_hist[b1 * 16 + slot], 1u);
         }
+    }
+    if (count) {
+        __syncwarp();
+        const int nbins = p.epi_q.top + kExtraBins;
+        for (int b = lane; b < nbins; b += 32) {
+            uint32_t c = 0u;
+#pragma unroll
+            for (int s = 0; s < 16; ++s) c += warp_hist[b * 16 + ((s + lane) & 15)];
+            if (c != 0u) atomicAdd(&hist[b], c);
+        }
+        __syncwarp();  // the boxes are about to be refilled with the tile's values
     }
 }
 
@@ -257,6 +269,9 @@ __device__ __forceinline__ void epi_merge(const GemmParams& p, const uint32_t* h
         atomicAdd((unsigned long long*)&p.epi_stats->n_total, (unsigned long long)p.M * (unsigned long long)p.N);
 }
 
+// kEpi: the layer-output epilogue is compiled in (its own instantiation, so that plain products
+// carry none of its code)
+template <bool kEpi>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tf32_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                  const __grid_constant__ CUtensorMap tmap_c, const __grid_constant__ CUtensorMap tmap_p,
@@ -281,7 +296,7 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
-    if (p.epi) {
+    if (kEpi) {
         for (int i = threadIdx.x; i < kEpiBins; i += kThreads) epi_hist[i] = 0u;
     }
 
@@ -601,7 +616,8 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                 if (!last && ++in_group < kFlushChunks) continue;
                 // ---- move the level-1 sums to C (level 2): registers -> swizzled shared boxes -> TMA.
                 // The first group of a tile is stored, later groups are added at the destination.
-                if (p.epi) epi_transform(sum2, p, row0 + lane < m_end, n0 + half * 128, epi_hist, lane);
+                if (kEpi)
+                    epi_transform(sum2, p, row0 + lane < m_end, n0 + half * 128, reinterpret_cast<uint32_t*>(my_stage), epi_hist, lane);
                 if (use_tma && flushed) {
                     if (lane == 0) ptx::bulk_wait_all();  // the earlier store/add to these addresses is complete
                 }
@@ -664,7 +680,7 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     // ------------------------------ common exit ------------------------------
     ptx::tc_fence_before_sync();
     __syncthreads();
-    epi_merge(p, epi_hist);
+    if (kEpi) epi_merge(p, epi_hist);
     if (*abort_flag) {
         // give TMA copies that may still be in flight time to land before the CTA's shared
         // memory is handed to another CTA
@@ -702,6 +718,7 @@ __device__ __forceinline__ uint32_t make_idesc_pair(int a_mn, int b_mn) {
            | ((uint32_t)(kBN >> 3) << 17) | ((uint32_t)((2 * kBM) >> 4) << 24);
 }
 
+template <bool kEpi>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 gemm_tf32_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                       const __grid_constant__ CUtensorMap tmap_c, const GemmParams p) {
@@ -722,7 +739,7 @@ gemm_tf32_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     const uint32_t rank = ptx::cluster_ctarank();  // 0 = leader
-    if (p.epi) {
+    if (kEpi) {
         for (int i = threadIdx.x; i < kEpiBins; i += kThreads) epi_hist[i] = 0u;
     }
     const int cluster_id = blockIdx.x >> 1, num_clusters = gridDim.x >> 1;
@@ -913,7 +930,8 @@ gemm_tf32_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
                 ++acc_iter;
                 const bool last = kb0 + kChunkKB >= num_kb;
                 if (!last && ++in_group < kFlushChunks) continue;
-                if (p.epi) epi_transform(sum2, p, row0 + lane < m_end, n0 + half * 128, epi_hist, lane);
+                if (kEpi)
+                    epi_transform(sum2, p, row0 + lane < m_end, n0 + half * 128, reinterpret_cast<uint32_t*>(my_stage), epi_hist, lane);
                 if (use_tma && flushed) {
                     if (lane == 0) ptx::bulk_wait_all();
                 }
@@ -972,7 +990,7 @@ gemm_tf32_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
     // ------------------------------ common exit ------------------------------
     ptx::tc_fence_before_sync();
     __syncthreads();
-    epi_merge(p, epi_hist);
+    if (kEpi) epi_merge(p, epi_hist);
     if (*abort_flag) {
         for (int i = 0; i < 2000; ++i) __nanosleep(1000);
     }
@@ -1086,12 +1104,14 @@ int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap&
                 const RowMaps& rows, const GemmParams& p, const DeviceInfo& dev, cudaStream_t stream) {
     static bool attr_set[64] = {};
     if (dev.ordinal < 0 || dev.ordinal >= 64 || !attr_set[dev.ordinal]) {
-        QFMT_CUDA_TRY(cudaFuncSetAttribute(gemm_tf32_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes));
+        QFMT_CUDA_TRY(cudaFuncSetAttribute(gemm_tf32_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes));
+        QFMT_CUDA_TRY(cudaFuncSetAttribute(gemm_tf32_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes));
         if (dev.ordinal >= 0 && dev.ordinal < 64) attr_set[dev.ordinal] = true;
     }
     const long long work = (long long)p.tiles_m * p.tiles_n * p.splits;
     const int grid = work < dev.sm_count ? (int)work : dev.sm_count;
-    gemm_tf32_kernel<<<grid, kThreads, kSmemBytes, stream>>>(ma, mb, mc, mp, rows, p);
+    if (p.epi) gemm_tf32_kernel<true><<<grid, kThreads, kSmemBytes, stream>>>(ma, mb, mc, mp, rows, p);
+    else gemm_tf32_kernel<false><<<grid, kThreads, kSmemBytes, stream>>>(ma, mb, mc, mp, rows, p);
     QFMT_CUDA_TRY(cudaGetLastError());
     if (p.sk_cpt > 0) {
         streamk_fixup_kernel<<<grid * kFixupParts, 64, 0, stream>>>(p.sk_partials, p.C, grid, p.tiles_m * p.tiles_n, p.tiles_m,
@@ -1175,13 +1195,16 @@ int launch_pair(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap&
                 const DeviceInfo& dev, cudaStream_t stream) {
     static bool attr_set[64] = {};
     if (dev.ordinal < 0 || dev.ordinal >= 64 || !attr_set[dev.ordinal]) {
-        QFMT_CUDA_TRY(cudaFuncSetAttribute(gemm_tf32_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        QFMT_CUDA_TRY(cudaFuncSetAttribute(gemm_tf32_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           (int)kPairSmemBytes));
+        QFMT_CUDA_TRY(cudaFuncSetAttribute(gemm_tf32_pair_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                            (int)kPairSmemBytes));
         if (dev.ordinal >= 0 && dev.ordinal < 64) attr_set[dev.ordinal] = true;
     }
     const long long work = (long long)p.tiles_m * p.tiles_n * p.splits;
     const long long clusters = work < dev.sm_count / 2 ? work : dev.sm_count / 2;
-    gemm_tf32_pair_kernel<<<(unsigned)(2 * clusters), kThreads, kPairSmemBytes, stream>>>(ma, mb, mc, p);
+    if (p.epi) gemm_tf32_pair_kernel<true><<<(unsigned)(2 * clusters), kThreads, kPairSmemBytes, stream>>>(ma, mb, mc, p);
+    else gemm_tf32_pair_kernel<false><<<(unsigned)(2 * clusters), kThreads, kPairSmemBytes, stream>>>(ma, mb, mc, p);
     QFMT_CUDA_TRY(cudaGetLastError());
     return QFMT_OK;
 }
@@ -1249,7 +1272,7 @@ int gemm_device(const qfmt_matrix_t* A, const qfmt_matrix_t* B, float* d_C, int6
     // from qfmt_gemm_workspace_bytes always has); a smaller workspace gets fewer splits.
     int splits = epi != nullptr ? 1 : plan.splits;
     if (epi != nullptr) {
-        if (K > kEpiMaxK || fmt->e > 7) return QFMT_ERR_BAD_ARG;  // callers check before asking
+        if (K > kEpiMaxK || fmt->e > 6) return QFMT_ERR_BAD_ARG;  // callers check before asking
         qfmt_format_t f = *fmt;
         f.loss_scale = 1.0f;
         p.epi = 1;
@@ -1588,6 +1611,10 @@ size_t linear_bias_bytes(int64_t N) {  // rounded bias, padded with zeros to who
 
 }  // namespace
 
+// 0 automatic, 1 epilogue inside the GEMM kernel whenever it applies, 2 always two kernels; see
+// qfmt_linear_fusion_policy.
+static std::atomic<int> g_fusion_policy{0};
+
 int linear_forward_device(const qfmt_matrix_t* A, const qfmt_matrix_t* B, const float* d_bias, float* d_Y, int64_t ldy,
                           const qfmt_format_t* fmt, qfmt_stats_t* d_stats, int accumulate, void* d_workspace,
                           size_t workspace_bytes, cudaStream_t stream) {
@@ -1608,7 +1635,9 @@ int linear_forward_device(const qfmt_matrix_t* A, const qfmt_matrix_t* B, const 
     // on a 256-byte boundary]
     const size_t gemm_bytes = (workspace_bytes - bias_bytes) & ~(size_t)255u;
     float* rbias = reinterpret_cast<float*>(reinterpret_cast<char*>(d_workspace) + gemm_bytes);
-    const bool fused = fmt->e <= 7 && K >= 1 && K <= kEpiMaxK && M > 0 && N > 0;
+    // e <= 6: at most 128 bins.  Automatic means two kernels: measured on B200, the epilogue's ALU work
+    // in the eight accumulate warps holds a tile longer than the separate full-occupancy pass costs.
+    const bool fused = g_fusion_policy.load() == 1 && fmt->e <= 6 && K >= 1 && K <= kEpiMaxK && M > 0 && N > 0;
     if (!fused) {
         rc = gemm_device(A, B, d_Y, ldy, fmt, d_workspace, gemm_bytes, stream);
         if (rc != QFMT_OK) return rc;
@@ -1632,6 +1661,12 @@ extern "C" int qfmt_linear_forward(const qfmt_matrix_t* A, const qfmt_matrix_t* 
                                    void* d_workspace, size_t workspace_bytes, void* stream) {
     return qfmt::linear_forward_device(A, B, d_bias, d_Y, ldy, fmt, d_stats, accumulate, d_workspace, workspace_bytes,
                                        (cudaStream_t)stream);
+}
+
+extern "C" int qfmt_linear_fusion_policy(int policy) {
+    if (policy < 0 || policy > 2) return QFMT_ERR_BAD_ARG;
+    qfmt::g_fusion_policy.store(policy);
+    return QFMT_OK;
 }
 
 extern "C" size_t qfmt_linear_forward_workspace_bytes(const qfmt_matrix_t* A, const qfmt_matrix_t* B) {

@@ -1,7 +1,7 @@
 """GPU tests of qfmt_linear_forward, Y = R(R(op(A) op(B)) + R(bias)) with the statistics of Y
 (Section IV-A's worked example).  The call must give the bits of its two parts, qfmt_gemm followed
 by qfmt_bias_quantize_stats (with the same K-summation plan), whether the epilogue runs inside
-the GEMM kernel (K <= 1024, e <= 7) or after it; the parts are checked against the oracle in their own tests, and once more here."""
+the GEMM kernel (K <= 1024, e <= 6) or after it; the parts are checked against the oracle in their own tests, and once more here."""
 import numpy as np
 import pytest
 import torch
@@ -15,10 +15,19 @@ pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
 
 
-@pytest.fixture(autouse=True)
-def _reset_policy():
-    yield
+@pytest.fixture(autouse=True, params=[1, 0], ids=["in-kernel", "default"])
+def fusion(request):
+    """Every test runs with the epilogue inside the GEMM kernel (where it applies) and with the
+    default plan."""
+    qf.qfmt_linear_fusion_policy(request.param)
+    yield request.param
+    qf.qfmt_linear_fusion_policy(0)
     qf.qfmt_gemm_tile_policy(0)
+
+
+def in_kernel(K, e):
+    """True when qfmt_linear_forward runs the epilogue inside the GEMM kernel under policy 1."""
+    return K <= 1024 and e <= 6
 
 
 def two_step(a, b, d_bias, M, N, fmt, fused=True):
@@ -36,7 +45,7 @@ def two_step(a, b, d_bias, M, N, fmt, fused=True):
     return acc, y, st
 
 
-def run_case(A, B, bias, e, m, den, transA=False, transB=False, ldy=None, check_oracle=False):
+def run_case(fusion, A, B, bias, e, m, den, transA=False, transB=False, ldy=None, check_oracle=False):
     """A, B: STORED matrices (numpy), already holding format values."""
     fmt = qf.make_format(e, m, den)
     dA, dB = torch.from_numpy(A).to(DEV), torch.from_numpy(B).to(DEV)
@@ -45,7 +54,7 @@ def run_case(A, B, bias, e, m, den, transA=False, transB=False, ldy=None, check_
     M = A.shape[1] if transA else A.shape[0]
     N = B.shape[0] if transB else B.shape[1]
     K = A.shape[0] if transA else A.shape[1]
-    acc, y_ref, st_ref = two_step(a, b, d_bias, M, N, fmt, fused=(K <= 1024 and e <= 7))
+    acc, y_ref, st_ref = two_step(a, b, d_bias, M, N, fmt, fused=(fusion == 1 and in_kernel(K, e)))
     ldy = ldy or N
     buf = torch.full((M * ldy + 8,), 7.0, dtype=torch.float32, device=DEV)
     y = buf[:M * ldy].view(M, ldy)
@@ -78,7 +87,7 @@ def operands(seed, shape_a, shape_b, e, m, den, mu=-3.0, sigma=2.0):
 
 @pytest.mark.parametrize("policy", [1, 2])
 @pytest.mark.parametrize("M,N,K", [(256, 256, 64), (300, 260, 200), (129, 516, 1024), (512, 1024, 96), (77, 30, 17)])
-def test_fused_matches_two_step(policy, M, N, K):
+def test_fused_matches_two_step(fusion, policy, M, N, K):
     """K <= 1024: the epilogue runs inside the GEMM kernel (both tile shapes, ragged tiles, and an N
     that is not a multiple of 4, which takes the scalar store path).  Operands sit in buffers whose
     leading dimensions are padded to a multiple of 4, as the TMA loads need."""
@@ -92,7 +101,7 @@ def test_fused_matches_two_step(policy, M, N, K):
     b = qf.make_matrix(dB.data_ptr(), False, K, N, N4)
     bias = workloads.normal_tensor(workloads.rng_for(601, N), (N,), 0.05)
     d_bias = torch.from_numpy(bias).to(DEV)
-    acc, y_ref, st_ref = two_step(a, b, d_bias, M, N, fmt)
+    acc, y_ref, st_ref = two_step(a, b, d_bias, M, N, fmt, fused=(fusion == 1))
     y = torch.empty(M, N, dtype=torch.float32, device=DEV)
     st = torch.full((qf.STATS_WORDS,), 99, dtype=torch.int64, device=DEV)
     wb = qf.qfmt_linear_forward_workspace_bytes(a, b)
@@ -108,39 +117,39 @@ def test_fused_matches_two_step(policy, M, N, K):
 
 
 @pytest.mark.parametrize("e,m,den", [(5, 10, 1), (5, 10, 0), (6, 9, 0), (7, 8, 1)])
-def test_formats_and_flushing(e, m, den):
+def test_formats_and_flushing(fusion, e, m, den):
     A, B = operands(610 + e, (260, 128), (128, 264), e, m, den, mu=-8.0, sigma=3.0)   # small sums: denormals
     bias = workloads.lognormal_tensor(workloads.rng_for(611), (264,), -12.0, 3.0)
-    st = run_case(A, B, bias, e, m, den, check_oracle=True)
+    st = run_case(fusion, A, B, bias, e, m, den, check_oracle=True)
     assert int(st[oracle.ST_DENORMAL]) > 0 or (e, m) != (5, 10)
 
 
-def test_transposed_operands_and_leading_dimension():
+def test_transposed_operands_and_leading_dimension(fusion):
     A, B = operands(620, (96, 260), (264, 96), 6, 9, 1)        # stored K x M and N x K
     bias = workloads.normal_tensor(workloads.rng_for(621), (264,), 0.05)
-    run_case(A, B, bias, 6, 9, 1, transA=True, transB=True, ldy=272)
+    run_case(fusion, A, B, bias, 6, 9, 1, transA=True, transB=True, ldy=272)
 
 
-def test_long_contraction_and_bfloat16_family_run_the_two_kernels():
+def test_long_contraction_and_bfloat16_family_run_the_two_kernels(fusion):
     """K > 1024 (sums leave the registers between groups) and e = 8 take the unfused path."""
     A, B = operands(630, (200, 1100), (1100, 256), 6, 9, 1)
     bias = workloads.normal_tensor(workloads.rng_for(631), (256,), 0.05)
-    run_case(A, B, bias, 6, 9, 1)
+    run_case(fusion, A, B, bias, 6, 9, 1)
     A, B = operands(632, (130, 64), (64, 256), 8, 7, 1)
-    run_case(A, B, bias, 8, 7, 1, check_oracle=True)
+    run_case(fusion, A, B, bias, 8, 7, 1, check_oracle=True)
 
 
-def test_special_values_pass_through_the_epilogue():
+def test_special_values_pass_through_the_epilogue(fusion):
     A, B = operands(640, (128, 64), (64, 256), 6, 9, 1)
     A[0, 0], A[1, 1], A[2, 2] = np.inf, -np.inf, np.nan
     B[:, 7] = 0.0
     bias = workloads.normal_tensor(workloads.rng_for(641), (256,), 0.05)
     bias[7], bias[8], bias[9] = -0.0, np.inf, np.nan
-    run_case(A, B, bias, 6, 9, 1, check_oracle=True)
+    run_case(fusion, A, B, bias, 6, 9, 1, check_oracle=True)
 
 
 @pytest.mark.parametrize("layer", [0, 1, 2])
-def test_config5_forward_layers_full_size(layer):
+def test_config5_forward_layers_full_size(fusion, layer):
     """BERT-large forward products with K = 1024 at full size, in the benchmark's launch
     configuration: fused output and statistics equal the two-step result bit for bit."""
     c = workloads.config5_layer(layer, 0)
@@ -153,7 +162,7 @@ def test_config5_forward_layers_full_size(layer):
     bias = workloads.normal_tensor(workloads.rng_for(650, layer), (N,), 0.02)
     d_bias = torch.from_numpy(bias).to(DEV)
     a, b = qf.make_matrix(dX), qf.make_matrix(dW)
-    acc, y_ref, st_ref = two_step(a, b, d_bias, M, N, fmt)
+    acc, y_ref, st_ref = two_step(a, b, d_bias, M, N, fmt, fused=(fusion == 1))
     y = torch.empty(M, N, dtype=torch.float32, device=DEV)
     st = torch.zeros(qf.STATS_WORDS, dtype=torch.int64, device=DEV)
     wb = qf.qfmt_linear_forward_workspace_bytes(a, b)
