@@ -1370,6 +1370,16 @@ int plan_conv(int op, const qfmt_conv_t* g, ConvPlan* plan) {
     plan->sk_cpt = 0;
     plan->sk_pieces = 1;
     plan->workspace = kWorkspaceHeader;
+    if (g->r == 1 && g->s == 1 && g->pad_h == 0 && g->pad_w == 0) {
+        // runs as a dense product (see conv_device): the dense planner's workspace, no row-length limits
+        const int64_t pixels = (int64_t)g->n * g->h * g->w;
+        const int64_t M = op == QFMT_CONV_WGRAD ? g->c_out : pixels;
+        const int64_t N = op == QFMT_CONV_FWD ? g->c_out : g->c_in;
+        const int64_t K = op == QFMT_CONV_FWD ? g->c_in : (op == QFMT_CONV_DGRAD ? g->c_out : pixels);
+        const int splits = plan_dense(M, N, K).splits;
+        if (splits > 1) plan->workspace += (size_t)splits * (size_t)M * (size_t)N * sizeof(float);
+        return QFMT_OK;
+    }
     if (op == QFMT_CONV_FWD && plan->ow > kBM) return QFMT_ERR_BAD_ARG;   // an M-tile is made of whole output rows
     if (op == QFMT_CONV_DGRAD && g->w > kBM) return QFMT_ERR_BAD_ARG;
     if (op != QFMT_CONV_WGRAD) {
@@ -1408,6 +1418,32 @@ int plan_conv(int op, const qfmt_conv_t* g, ConvPlan* plan) {
 }
 }  // namespace
 
+namespace {
+// A 1 x 1 filter without padding is a plain matrix product on channels-last tensors:
+//   forward  Y[pixels][c_out]  = X[pixels][c_in] . W[c_out][c_in]^T
+//   dgrad    dX[pixels][c_in]  = dY[pixels][c_out] . W[c_out][c_in]
+//   wgrad    dW[c_out][c_in]   = dY[pixels][c_out]^T . X[pixels][c_in]
+// so it runs on the dense kernels (CTA pairs, split K) instead of the implicit-GEMM modes.
+bool conv_is_pointwise(const qfmt_conv_t* g) { return g->r == 1 && g->s == 1 && g->pad_h == 0 && g->pad_w == 0; }
+void pointwise_operands(int op, const qfmt_conv_t* g, const float* d_p, const float* d_q, qfmt_matrix_t* A,
+                        qfmt_matrix_t* B, int64_t* ldc) {
+    const int64_t pixels = (int64_t)g->n * g->h * g->w;
+    if (op == QFMT_CONV_FWD) {
+        *A = {d_p, pixels, g->c_in, g->c_in, 0};
+        *B = {d_q, g->c_out, g->c_in, g->c_in, 1};
+        *ldc = g->c_out;
+    } else if (op == QFMT_CONV_DGRAD) {
+        *A = {d_p, pixels, g->c_out, g->c_out, 0};
+        *B = {d_q, g->c_out, g->c_in, g->c_in, 0};
+        *ldc = g->c_in;
+    } else {
+        *A = {d_p, pixels, g->c_out, g->c_out, 1};
+        *B = {d_q, pixels, g->c_in, g->c_in, 0};
+        *ldc = g->c_in;
+    }
+}
+}  // namespace
+
 int conv_device(int op, const qfmt_conv_t* g, const float* d_p, const float* d_q, float* d_out,
                 const qfmt_format_t* fmt, void* d_workspace, size_t workspace_bytes, cudaStream_t stream) {
     int rc = validate_format(fmt);
@@ -1425,6 +1461,12 @@ int conv_device(int op, const qfmt_conv_t* g, const float* d_p, const float* d_q
         return QFMT_ERR_BAD_ARG;
     if (d_workspace == nullptr || workspace_bytes < plan.workspace || (reinterpret_cast<uintptr_t>(d_workspace) & 15u))
         return QFMT_ERR_BAD_ARG;
+    if (conv_is_pointwise(g)) {
+        qfmt_matrix_t A, B;
+        int64_t ldc;
+        pointwise_operands(op, g, d_p, d_q, &A, &B, &ldc);
+        return gemm_device(&A, &B, d_out, ldc, fmt, d_workspace, workspace_bytes, stream);
+    }
     int* status = reinterpret_cast<int*>(d_workspace);
     QFMT_CUDA_TRY(cudaMemsetAsync(status, 0, 16, stream));
 
