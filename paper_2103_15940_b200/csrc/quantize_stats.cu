@@ -205,6 +205,85 @@ quantize_stats_transpose_kernel(const uint32_t* __restrict__ in, uint32_t* __res
 // smaller term lies below 2^-12 of the larger one's last place).
 // Vector kernel: rows of c4 = cols/4 128-bit vectors; each thread owns a column of vectors (its
 // rounded bias entries stay in registers) and walks down the rows, four loads in flight.
+// The same with 128-bit accesses on both sides, for rows and cols that are multiples of 4 and
+// 16-byte aligned tensors: tiles of 64 rows x 32 columns; a thread loads four consecutive columns of
+// a row (eight threads cover a 128-byte segment) and, after the exchange through shared memory,
+// stores four consecutive rows of a column (sixteen threads cover the tile's 256 bytes of that
+// output row).
+constexpr int kTvRows = 64, kTvCols = 32;
+template <bool kStats, bool kScale>
+__global__ void __launch_bounds__(kTThreads)
+quantize_stats_transpose_vec_kernel(const uint32_t* __restrict__ in, uint32_t* __restrict__ out, unsigned batch,
+                                    unsigned rows, unsigned cols, QuantParams p, qfmt_stats_t* __restrict__ stats,
+                                    unsigned long long n_total) {
+    extern __shared__ uint32_t lane_hist[];  // [(top + kExtraBins)][32]
+    __shared__ uint32_t tile[kTvRows][kTvCols + 1];
+    const int nbins = p.top + kExtraBins;
+    const int lane = threadIdx.x & 31;
+    if (kStats) {
+        for (int i = threadIdx.x; i < nbins * 32; i += kTThreads) lane_hist[i] = 0u;
+    }
+    const unsigned tr = (rows + kTvRows - 1) / kTvRows, tc = (cols + kTvCols - 1) / kTvCols;
+    const unsigned long long tiles = (unsigned long long)batch * tr * tc;
+    const unsigned lr = threadIdx.x / 8, lc4 = threadIdx.x % 8;    // load: row within a 32-row pass, column quad
+    const unsigned sc = threadIdx.x / 16, sr4 = threadIdx.x % 16;  // store: column within a 16-column pass, row quad
+    for (unsigned long long t = blockIdx.x; t < tiles; t += gridDim.x) {
+        const unsigned b = (unsigned)(t / ((unsigned long long)tr * tc));
+        const unsigned rem = (unsigned)(t % ((unsigned long long)tr * tc));
+        const unsigned r0 = (rem / tc) * kTvRows, c0 = (rem % tc) * kTvCols;
+        const unsigned long long base = (unsigned long long)b * rows * cols;
+        uint4 v[2];
+        bool ok[2];
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            const unsigned r = r0 + lr + 32 * i, c = c0 + 4 * lc4;
+            ok[i] = r < rows && c < cols;
+            if (ok[i]) v[i] = load_stream(reinterpret_cast<const uint4*>(in + base + (unsigned long long)r * cols + c));
+        }
+        __syncthreads();  // previous tile fully written out (and the histogram cleared)
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            if (ok[i]) {
+                int b0, b1, b2, b3;
+                uint32_t* dst = &tile[lr + 32 * i][4 * lc4];
+                dst[0] = quantize_one<kScale>(v[i].x, p, b0);
+                dst[1] = quantize_one<kScale>(v[i].y, p, b1);
+                dst[2] = quantize_one<kScale>(v[i].z, p, b2);
+                dst[3] = quantize_one<kScale>(v[i].w, p, b3);
+                if (kStats) {
+                    atomicAdd(&lane_hist[b0 * 32 + lane], 1u);
+                    atomicAdd(&lane_hist[b1 * 32 + lane], 1u);
+                    atomicAdd(&lane_hist[b2 * 32 + lane], 1u);
+                    atomicAdd(&lane_hist[b3 * 32 + lane], 1u);
+                }
+            }
+        }
+        __syncthreads();
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            const unsigned c = c0 + sc + 16 * i, r = r0 + 4 * sr4;
+            if (c < cols && r < rows) {
+                uint4 q;
+                q.x = tile[4 * sr4 + 0][sc + 16 * i];
+                q.y = tile[4 * sr4 + 1][sc + 16 * i];
+                q.z = tile[4 * sr4 + 2][sc + 16 * i];
+                q.w = tile[4 * sr4 + 3][sc + 16 * i];
+                store_stream(reinterpret_cast<uint4*>(out + base + (unsigned long long)c * rows + r), q);
+            }
+        }
+    }
+    if (kStats) {
+        __syncthreads();
+        const int warp = threadIdx.x >> 5;
+        for (int b = warp + 1; b < nbins; b += kTThreads / 32) {
+            const uint32_t c = __reduce_add_sync(0xFFFFFFFFu, lane_hist[b * 32 + lane]);
+            if (lane == 0 && c != 0u) merge_bin(stats, p, b, c);
+        }
+        if (blockIdx.x == 0 && threadIdx.x == 0 && n_total != 0ull)
+            atomicAdd((unsigned long long*)&stats->n_total, n_total);
+    }
+}
+
 template <bool kScale>
 __device__ __forceinline__ uint32_t bias_round_one(uint32_t acc, uint32_t rb, const QuantParams& p, uint32_t inf_bits,
                                                    int& bin) {
@@ -422,11 +501,21 @@ int quantize_stats_transpose_device(const float* d_in, float* d_out, int64_t bat
     uint32_t* out = reinterpret_cast<uint32_t*>(d_out);
     const bool has_stats = d_stats != nullptr, has_scale = fmt->loss_scale != 1.0f;
     const size_t smem = has_stats ? (size_t)(p.top + kExtraBins) * 32 * sizeof(uint32_t) : 0;
-    const unsigned long long tiles = (unsigned long long)batch * ((rows + 31) / 32) * ((cols + 31) / 32);
+    const bool vec = (rows % 4 == 0) && (cols % 4 == 0) &&
+                     !((reinterpret_cast<uintptr_t>(d_in) | reinterpret_cast<uintptr_t>(d_out)) & 15u);
+    const unsigned long long tiles =
+        vec ? (unsigned long long)batch * ((rows + kTvRows - 1) / kTvRows) * ((cols + kTvCols - 1) / kTvCols)
+            : (unsigned long long)batch * ((rows + 31) / 32) * ((cols + 31) / 32);
     unsigned long long want = tiles < (unsigned long long)dev.sm_count * 8 ? tiles : (unsigned long long)dev.sm_count * 8;
 #define QFMT_TLAUNCH(S, C)                                                                                       \
-    quantize_stats_transpose_kernel<S, C><<<(unsigned)want, kTThreads, smem, stream>>>(                          \
-        in, out, (unsigned)batch, (unsigned)rows, (unsigned)cols, p, d_stats, n)
+    do {                                                                                                         \
+        if (vec)                                                                                                 \
+            quantize_stats_transpose_vec_kernel<S, C><<<(unsigned)want, kTThreads, smem, stream>>>(              \
+                in, out, (unsigned)batch, (unsigned)rows, (unsigned)cols, p, d_stats, n);                        \
+        else                                                                                                     \
+            quantize_stats_transpose_kernel<S, C><<<(unsigned)want, kTThreads, smem, stream>>>(                  \
+                in, out, (unsigned)batch, (unsigned)rows, (unsigned)cols, p, d_stats, n);                        \
+    } while (0)
     if (has_stats) { if (has_scale) QFMT_TLAUNCH(true, true); else QFMT_TLAUNCH(true, false); }
     else { if (has_scale) QFMT_TLAUNCH(false, true); else QFMT_TLAUNCH(false, false); }
 #undef QFMT_TLAUNCH

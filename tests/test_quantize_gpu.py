@@ -183,7 +183,9 @@ def test_errors_leave_outputs_untouched():
 
 
 @pytest.mark.parametrize("batch,rows,cols", [(1, 1, 1), (2, 3, 5), (3, 32, 32), (2, 33, 65), (4, 64, 196),
-                                             (5, 256, 9), (1, 100, 1), (7, 1, 50)])
+                                             (5, 256, 9), (1, 100, 1), (7, 1, 50),
+                                             # rows and cols multiples of 4: the 128-bit kernel, ragged tiles
+                                             (1, 4, 4), (2, 68, 36), (3, 128, 100), (5, 256, 12), (2, 60, 200)])
 @pytest.mark.parametrize("e,m,den,scale", [(6, 9, 1, 1.0), (5, 10, 0, 2.0 ** 10), (8, 7, 1, 1.0)])
 def test_transposing_variant(batch, rows, cols, e, m, den, scale):
     """[batch][rows][cols] -> [batch][cols][rows]: same bits as the oracle's values, permuted; same counts."""
