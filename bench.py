@@ -144,6 +144,20 @@ def run_reference(args):
 # ------------------------------------------------------------------------------------------------
 # this library
 # ------------------------------------------------------------------------------------------------
+def max_over_ranks(torch, dist, value: float, device) -> float:
+    """The slowest rank's time: what a multi-GPU number is computed from (dist is None for one rank)."""
+    if dist is None:
+        return value
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(world: int, steps: int, step_bytes: int, total_ms: float) -> float:
+    """GB/s over all ranks: every rank ran `steps` sweeps of `step_bytes` on its own replica."""
+    return world * steps * step_bytes / total_ms / 1e6
+
+
 def time_events(torch, fn, iters):
     """Per-call device times (ms) of fn(), CUDA events on the current stream."""
     evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(iters)]
@@ -417,12 +431,9 @@ def run_library(args):
         barrier()
     total_ms = t_begin.elapsed_time(t_end)
     launch_ms = [a.elapsed_time(b) for a, b in pairs]
-    if dist is not None:
-        t = torch.tensor([total_ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(torch, dist, total_ms, dev)
     step_bytes = len(runs) * n * BYTES_PER_ELEMENT
-    value = world * args.steps * step_bytes / total_ms / 1e6  # GB/s over all ranks
+    value = whole_job_value(world, args.steps, step_bytes, total_ms)
 
     # sanity: the timed kernels did the work (denormal counts of the last step are plausible)
     st = d_stats.cpu().numpy().view(np.uint64)
