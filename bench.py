@@ -322,7 +322,7 @@ def epilogue_section(torch, qf, dev, peaks, reps=20):
             "workload": f"config5 FFN-up forward output, {rows} x {cols}, 1/6/9 (268 MB moved per launch, larger than L2)",
             "ms_per_step": ms, "gpu_launches_per_step": 1,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                         "frac": achieved / peaks["hbm_gbs"], "traffic": None,
+                         "frac": achieved / peaks["hbm_gbs"], "traffic": NCU_EPILOGUE_TRAFFIC_BYTES_PER_LAUNCH,
                          "peak_source": f"copy bandwidth, {peaks['source']}",
                          "algorithmic_bytes_per_launch": rows * cols * BYTES_PER_ELEMENT}}
 
@@ -513,6 +513,8 @@ def finish(args, world, value, total_ms, n, runs, clocks, e2e, roofline, cpu, ge
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the quantize+stats kernel, from the
 # ncu capture summarised in profiles/quantize_stats_kernel_config2.md (set to None when the kernel changes).
 NCU_TRAFFIC_BYTES_PER_LAUNCH = 268464640 + 218681088
+# the same for the layer-output kernel on the 8192 x 4096 product (profiles/bias_quantize_stats_kernel_config5.md)
+NCU_EPILOGUE_TRAFFIC_BYTES_PER_LAUNCH = 134290688 + 85444352
 
 
 def main():
