@@ -72,6 +72,10 @@ def _L() -> ctypes.CDLL:
         lib.oracle_fmac8_gemm_sampled.argtypes = [vp, i64, i32, vp, i64, i32, i64, i32, i32, i32, i32, vp, vp,
                                                   i64, vp]
         lib.oracle_fmac8_gemm_sampled.restype = None
+        lib.oracle_quantize_stats_pack16.argtypes = [vp, vp, sz, i32, i32, i32, u32, vp]
+        lib.oracle_quantize_stats_pack16.restype = None
+        lib.oracle_unpack16.argtypes = [vp, vp, sz, i32, i32]
+        lib.oracle_unpack16.restype = None
         lib.oracle_dls_update.argtypes = [vp, vp, i64]
         lib.oracle_dls_update.restype = None
         _lib = lib
@@ -144,6 +148,25 @@ def quantize_stats(x: np.ndarray, e: int, m: int, denormals: int = 1, loss_scale
                                int(denormals), _f32_bits(loss_scale),
                                st.ctypes.data if want_stats else None)
     return (q.view(np.float32).reshape(xf.shape) if want_q else None), st
+
+
+def quantize_stats_pack16(x: np.ndarray, e: int, m: int, denormals: int = 1, loss_scale: float = 1.0):
+    """Rounded tensor as packed 16-bit codes (uint16, shaped like x) and its statistics."""
+    xf = np.ascontiguousarray(x, dtype=np.float32)
+    xb = xf.view(np.uint32).reshape(-1)
+    codes = np.empty(xb.size, dtype=np.uint16)
+    st = np.zeros(STATS_WORDS, dtype=np.uint64)
+    _L().oracle_quantize_stats_pack16(xb.ctypes.data, codes.ctypes.data, xb.size, e, m, int(denormals),
+                                      _f32_bits(loss_scale), st.ctypes.data)
+    return codes.reshape(xf.shape), st
+
+
+def unpack16(codes: np.ndarray, e: int, m: int) -> np.ndarray:
+    """fp32 containers of packed 16-bit codes."""
+    c = np.ascontiguousarray(codes, dtype=np.uint16)
+    q = np.empty(c.size, dtype=np.uint32)
+    _L().oracle_unpack16(c.ctypes.data, q.ctypes.data, c.size, e, m)
+    return q.view(np.float32).reshape(c.shape)
 
 
 def _mat(a: np.ndarray) -> np.ndarray:

@@ -273,6 +273,25 @@ void oracle_quantize_stats(const uint32_t *x, uint32_t *q, size_t n, int e, int 
 }
 
 /* ------------------------------------------------------------------------------------------ */
+/* 16-bit storage (Section II: activations and gradients are kept in half precision, halving     */
+/* storage and bandwidth): a tensor is rounded as oracle_quantize_stats does and each value is    */
+/* stored as its packed code, sign | stored exponent | mantissa (1 + e + m <= 16 bits, in the     */
+/* low bits of a 16-bit word); unpacking returns the fp32 containers.                             */
+/* ------------------------------------------------------------------------------------------ */
+void oracle_quantize_stats_pack16(const uint32_t *x, uint16_t *codes, size_t n, int e, int m, int keep_denormals,
+                                  uint32_t scale_bits, uint64_t *stats) {
+    for (size_t i = 0; i < n; ++i) {
+        uint32_t q;
+        oracle_quantize_stats(&x[i], &q, 1, e, m, keep_denormals, scale_bits, stats);
+        codes[i] = (uint16_t)oracle_encode_code(q, e, m);
+    }
+}
+
+void oracle_unpack16(const uint16_t *codes, uint32_t *q, size_t n, int e, int m) {
+    for (size_t i = 0; i < n; ++i) q[i] = oracle_decode_code(codes[i], e, m);
+}
+
+/* ------------------------------------------------------------------------------------------ */
 /* Exact signed sums, rounded once.                                                             */
 /*                                                                                              */
 /* Both FMAC (Section III-B: a16 = round(a16 + x16*y16), one rounding of the exact value) and   */
