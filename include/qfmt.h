@@ -106,6 +106,24 @@ int qfmt_quantize_stats_transpose(const float* d_in, float* d_out, int64_t batch
                                   void* stream);
 
 /*
+ * 16-bit storage.  Section II: in mixed-precision training "activations and gradients are kept in
+ * half-precision, halving the required storage and bandwidth".  qfmt_quantize_stats_pack16 is
+ * qfmt_quantize_stats writing, instead of fp32 containers, the packed code of every rounded value:
+ * sign | stored exponent field | mantissa in the low 1 + e + m bits of a 16-bit word (Definition
+ * III.1 with Section III's special encodings: all-ones exponent = inf, or NaN with the top mantissa
+ * bit set; all-zero exponent = zero / denormal).  For 1/5/10 and 1/8/7 these are the bits of IEEE
+ * binary16 and of bfloat16.  6 bytes of traffic per element instead of 8.  qfmt_unpack16 expands
+ * codes to the fp32 containers the contractions read.
+ *   d_codes   device, n 16-bit words, 2-byte aligned (16-byte alignment of both pointers selects
+ *             the 128-bit path)
+ * Requires e + m <= 15 (QFMT_ERR_BAD_FORMAT otherwise).  Statistics, loss scale, accumulate, n = 0
+ * and errors as for qfmt_quantize_stats.
+ */
+int qfmt_quantize_stats_pack16(const float* d_in, uint16_t* d_codes, size_t n, const qfmt_format_t* fmt,
+                               qfmt_stats_t* d_stats, int accumulate, void* stream);
+int qfmt_unpack16(const uint16_t* d_codes, float* d_out, size_t n, const qfmt_format_t* fmt, void* stream);
+
+/*
  * Output of a layer as Section IV-A's worked example computes it, Y = R(R(acc) + R(B)): `acc` is
  * the matrix product of the layer (what qfmt_gemm or qfmt_conv wrote: rows x cols, row-major,
  * leading dimension ld_acc), `bias` has one entry per column.  Each acc element and each bias

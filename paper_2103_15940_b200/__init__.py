@@ -86,6 +86,10 @@ def lib() -> ctypes.CDLL:
         L.qfmt_bias_quantize_stats.argtypes = [vp, ctypes.c_int64, vp, vp, ctypes.c_int64, ctypes.c_int64,
                                                ctypes.c_int64, fmtp, vp, ci, vp]
         L.qfmt_bias_quantize_stats.restype = ci
+        L.qfmt_quantize_stats_pack16.argtypes = [vp, vp, sz, fmtp, vp, ci, vp]
+        L.qfmt_quantize_stats_pack16.restype = ci
+        L.qfmt_unpack16.argtypes = [vp, vp, sz, fmtp, vp]
+        L.qfmt_unpack16.restype = ci
         L.qfmt_quantize_stats_host.argtypes = [vp, vp, sz, fmtp, vp, vp, sz, vp]
         L.qfmt_quantize_stats_host.restype = ci
         L.qfmt_quantize_stats_host_work_bytes.argtypes = [sz]
@@ -186,6 +190,19 @@ def qfmt_bias_quantize_stats(d_acc, ld_acc: int, d_bias, d_out, ld_out: int, row
     _check(lib().qfmt_bias_quantize_stats(_ptr(d_acc), int(ld_acc), _ptr(d_bias), _ptr(d_out), int(ld_out),
                                           int(rows), int(cols), ctypes.byref(fmt), _ptr(d_stats), int(accumulate),
                                           _stream_handle(stream)), "qfmt_bias_quantize_stats")
+
+
+def qfmt_quantize_stats_pack16(d_in, d_codes, n: int, fmt: qfmt_format_t, d_stats=None, accumulate: int = 0,
+                               stream=None) -> None:
+    """Rounding pass that stores packed 16-bit codes; see qfmt_quantize_stats_pack16 in include/qfmt.h."""
+    _check(lib().qfmt_quantize_stats_pack16(_ptr(d_in), _ptr(d_codes), int(n), ctypes.byref(fmt), _ptr(d_stats),
+                                            int(accumulate), _stream_handle(stream)), "qfmt_quantize_stats_pack16")
+
+
+def qfmt_unpack16(d_codes, d_out, n: int, fmt: qfmt_format_t, stream=None) -> None:
+    """Packed 16-bit codes to fp32 containers; see qfmt_unpack16 in include/qfmt.h."""
+    _check(lib().qfmt_unpack16(_ptr(d_codes), _ptr(d_out), int(n), ctypes.byref(fmt), _stream_handle(stream)),
+           "qfmt_unpack16")
 
 
 def qfmt_quantize_stats_host_work_bytes(n: int) -> int:

@@ -197,6 +197,90 @@ quantize_stats_transpose_kernel(const uint32_t* __restrict__ in, uint32_t* __res
     }
 }
 
+// 16-bit storage (Section II: activations and gradients are kept in 16 bits, halving storage and
+// bandwidth): the rounding pass writing packed codes instead of fp32 containers, 4 bytes read and
+// 2 written per element, and the pass that expands codes back to containers for the contraction.
+// A thread takes eight consecutive elements: two 128-bit loads, one 128-bit store.
+template <bool kStats, bool kScale>
+__global__ void __launch_bounds__(kThreads)
+quantize_stats_pack16_kernel(const uint32_t* __restrict__ in, uint16_t* __restrict__ codes, unsigned long long n,
+                             int vec, QuantParams p, int sign_shift, qfmt_stats_t* __restrict__ stats) {
+    extern __shared__ uint32_t lane_hist[];
+    const int nbins = p.top + kExtraBins;
+    const int lane = threadIdx.x & 31;
+    if (kStats) {
+        for (int i = threadIdx.x; i < nbins * 32; i += kThreads) lane_hist[i] = 0u;
+        __syncthreads();
+    }
+    const unsigned long long n8 = vec ? n / 8 : 0ull;
+    const unsigned long long stride = (unsigned long long)gridDim.x * (kThreads * 2);
+    for (unsigned long long base = (unsigned long long)blockIdx.x * (kThreads * 2); base < n8; base += stride) {
+        uint4 v[2][2];
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            const unsigned long long idx = base + (unsigned long long)u * kThreads + threadIdx.x;
+            if (idx < n8) {
+                v[u][0] = load_stream(reinterpret_cast<const uint4*>(in) + 2 * idx);
+                v[u][1] = load_stream(reinterpret_cast<const uint4*>(in) + 2 * idx + 1);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            const unsigned long long idx = base + (unsigned long long)u * kThreads + threadIdx.x;
+            if (idx < n8) {
+                const uint32_t w[8] = {v[u][0].x, v[u][0].y, v[u][0].z, v[u][0].w, v[u][1].x, v[u][1].y, v[u][1].z, v[u][1].w};
+                uint32_t c[8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    int b;
+                    c[j] = quantize_pack_one<kScale>(w[j], p, sign_shift, b);
+                    if (kStats) atomicAdd(&lane_hist[b * 32 + lane], 1u);
+                }
+                store_stream(reinterpret_cast<uint4*>(codes) + idx,
+                             make_uint4(c[0] | (c[1] << 16), c[2] | (c[3] << 16), c[4] | (c[5] << 16), c[6] | (c[7] << 16)));
+            }
+        }
+    }
+    // what the vector body leaves (everything when the pointers are not 16-byte aligned)
+    const unsigned long long done = n8 * 8;
+    for (unsigned long long i = done + (unsigned long long)blockIdx.x * kThreads + threadIdx.x; i < n;
+         i += (unsigned long long)gridDim.x * kThreads) {
+        int b;
+        codes[i] = (uint16_t)quantize_pack_one<kScale>(in[i], p, sign_shift, b);
+        if (kStats) atomicAdd(&lane_hist[b * 32 + lane], 1u);
+    }
+    if (kStats) {
+        __syncthreads();
+        const int warp = threadIdx.x >> 5;
+        for (int b = warp + 1; b < nbins; b += kThreads / 32) {
+            const uint32_t c = __reduce_add_sync(0xFFFFFFFFu, lane_hist[b * 32 + lane]);
+            if (lane == 0 && c != 0u) merge_bin(stats, p, b, c);
+        }
+        if (blockIdx.x == 0 && threadIdx.x == 0 && n != 0ull) atomicAdd((unsigned long long*)&stats->n_total, n);
+    }
+}
+
+__global__ void __launch_bounds__(kThreads)
+unpack16_kernel(const uint16_t* __restrict__ codes, uint32_t* __restrict__ out, unsigned long long n, int vec,
+                QuantParams p, int sign_shift) {
+    const unsigned long long n8 = vec ? n / 8 : 0ull;
+    const unsigned long long stride = (unsigned long long)gridDim.x * kThreads;
+    for (unsigned long long idx = (unsigned long long)blockIdx.x * kThreads + threadIdx.x; idx < n8; idx += stride) {
+        const uint4 c = load_stream(reinterpret_cast<const uint4*>(codes) + idx);
+        const uint32_t w[4] = {c.x, c.y, c.z, c.w};
+        uint32_t q[8];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            q[2 * j] = unpack_one(w[j] & 0xFFFFu, p, sign_shift);
+            q[2 * j + 1] = unpack_one(w[j] >> 16, p, sign_shift);
+        }
+        store_stream(reinterpret_cast<uint4*>(out) + 2 * idx, make_uint4(q[0], q[1], q[2], q[3]));
+        store_stream(reinterpret_cast<uint4*>(out) + 2 * idx + 1, make_uint4(q[4], q[5], q[6], q[7]));
+    }
+    for (unsigned long long i = n8 * 8 + (unsigned long long)blockIdx.x * kThreads + threadIdx.x; i < n; i += stride)
+        out[i] = unpack_one(codes[i], p, sign_shift);
+}
+
 // Layer output of Section IV-A's worked example, Y = R(R(acc) + R(B)): the matrix product is
 // rounded, the (rounded) bias of its column is added, and the sum is rounded again, with the
 // statistics of Y taken in the same pass.  The sum of two format values is formed with one IEEE
@@ -586,6 +670,65 @@ int bias_quantize_stats_device(const float* d_acc, int64_t ld_acc, const float* 
     return QFMT_OK;
 }
 
+
+int quantize_stats_pack16_device(const float* d_in, uint16_t* d_codes, size_t n, const qfmt_format_t* fmt,
+                                 qfmt_stats_t* d_stats, int accumulate, cudaStream_t stream) {
+    int rc = validate_format(fmt);
+    if (rc != QFMT_OK) return rc;
+    if (fmt->e + fmt->m > 15) return QFMT_ERR_BAD_FORMAT;  // sign, exponent and mantissa must fit 16 bits
+    if (accumulate != 0 && accumulate != 1) return QFMT_ERR_BAD_ARG;
+    if (n > ((size_t)1 << 40)) return QFMT_ERR_BAD_ARG;
+    if (n != 0 && (d_in == nullptr || d_codes == nullptr)) return QFMT_ERR_BAD_ARG;
+    if ((reinterpret_cast<uintptr_t>(d_in) & 3u) || (reinterpret_cast<uintptr_t>(d_codes) & 1u) ||
+        (reinterpret_cast<uintptr_t>(d_stats) & 7u))
+        return QFMT_ERR_BAD_ARG;
+    DeviceInfo dev;
+    rc = current_device(&dev);
+    if (rc != QFMT_OK) return rc;
+    if (d_stats != nullptr && accumulate == 0) QFMT_CUDA_TRY(cudaMemsetAsync(d_stats, 0, sizeof(qfmt_stats_t), stream));
+    if (n == 0) return QFMT_OK;
+    const QuantParams p = make_params(*fmt);
+    const bool has_stats = d_stats != nullptr, has_scale = fmt->loss_scale != 1.0f;
+    const size_t smem = has_stats ? (size_t)(p.top + kExtraBins) * 32 * sizeof(uint32_t) : 0;
+    const int vec = !((reinterpret_cast<uintptr_t>(d_in) | reinterpret_cast<uintptr_t>(d_codes)) & 15u);
+    const unsigned long long per_block = (unsigned long long)kThreads * 16;  // elements per block and sweep
+    unsigned long long want = (n + per_block - 1) / per_block;
+    const unsigned long long cap = (unsigned long long)dev.sm_count * 2;  // 56 registers x 512 threads: two per SM
+    if (want > cap) want = cap;
+    const uint32_t* in = reinterpret_cast<const uint32_t*>(d_in);
+    const int sign_shift = fmt->e + fmt->m;
+#define QFMT_PLAUNCH(S, C)                                                                                  \
+    quantize_stats_pack16_kernel<S, C><<<(unsigned)want, kThreads, smem, stream>>>(in, d_codes, n, vec, p,  \
+                                                                                    sign_shift, d_stats)
+    if (has_stats) { if (has_scale) QFMT_PLAUNCH(true, true); else QFMT_PLAUNCH(true, false); }
+    else { if (has_scale) QFMT_PLAUNCH(false, true); else QFMT_PLAUNCH(false, false); }
+#undef QFMT_PLAUNCH
+    QFMT_CUDA_TRY(cudaGetLastError());
+    return QFMT_OK;
+}
+
+int unpack16_device(const uint16_t* d_codes, float* d_out, size_t n, const qfmt_format_t* fmt, cudaStream_t stream) {
+    int rc = validate_format(fmt);
+    if (rc != QFMT_OK) return rc;
+    if (fmt->e + fmt->m > 15) return QFMT_ERR_BAD_FORMAT;
+    if (n > ((size_t)1 << 40)) return QFMT_ERR_BAD_ARG;
+    if (n != 0 && (d_codes == nullptr || d_out == nullptr)) return QFMT_ERR_BAD_ARG;
+    if ((reinterpret_cast<uintptr_t>(d_codes) & 1u) || (reinterpret_cast<uintptr_t>(d_out) & 3u)) return QFMT_ERR_BAD_ARG;
+    DeviceInfo dev;
+    rc = current_device(&dev);
+    if (rc != QFMT_OK) return rc;
+    if (n == 0) return QFMT_OK;
+    const QuantParams p = make_params(*fmt);
+    const int vec = !((reinterpret_cast<uintptr_t>(d_codes) | reinterpret_cast<uintptr_t>(d_out)) & 15u);
+    unsigned long long want = (n / 8 + kThreads) / kThreads;
+    const unsigned long long cap = (unsigned long long)dev.sm_count * 4;
+    if (want > cap) want = cap;
+    unpack16_kernel<<<(unsigned)want, kThreads, 0, stream>>>(d_codes, reinterpret_cast<uint32_t*>(d_out), n, vec, p,
+                                                             fmt->e + fmt->m);
+    QFMT_CUDA_TRY(cudaGetLastError());
+    return QFMT_OK;
+}
+
 }  // namespace qfmt
 
 extern "C" int qfmt_quantize_stats(const float* d_in, float* d_out, size_t n, const qfmt_format_t* fmt,
@@ -630,4 +773,13 @@ extern "C" int qfmt_bias_quantize_stats(const float* d_acc, int64_t ld_acc, cons
                                         qfmt_stats_t* d_stats, int accumulate, void* stream) {
     return qfmt::bias_quantize_stats_device(d_acc, ld_acc, d_bias, d_out, ld_out, rows, cols, fmt, d_stats, accumulate,
                                             (cudaStream_t)stream);
+}
+
+extern "C" int qfmt_quantize_stats_pack16(const float* d_in, uint16_t* d_codes, size_t n, const qfmt_format_t* fmt,
+                                          qfmt_stats_t* d_stats, int accumulate, void* stream) {
+    return qfmt::quantize_stats_pack16_device(d_in, d_codes, n, fmt, d_stats, accumulate, (cudaStream_t)stream);
+}
+
+extern "C" int qfmt_unpack16(const uint16_t* d_codes, float* d_out, size_t n, const qfmt_format_t* fmt, void* stream) {
+    return qfmt::unpack16_device(d_codes, d_out, n, fmt, (cudaStream_t)stream);
 }

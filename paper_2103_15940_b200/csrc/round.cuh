@@ -122,6 +122,51 @@ __device__ __forceinline__ uint32_t round_sum(uint32_t s, const QuantParams& p, 
     return q;
 }
 
+// Rounds one element and returns its packed code, sign | stored exponent | mantissa in the low
+// 1 + e + m bits (Definition III.1 with the special encodings of Section III), and the bin.
+// For normal results exponent and mantissa fields are the fp32 word's own, re-biased and shifted;
+// for denormal results the mantissa is the integer multiple of the smallest denormal that the
+// rounding addition leaves in its sum's mantissa field.
+template <bool kScale>
+__device__ __forceinline__ uint32_t quantize_pack_one(uint32_t xb, const QuantParams& p, int sign_shift, int& bin) {
+    uint32_t yb = kScale ? __float_as_uint(mul_ieee(__uint_as_float(xb), p.scale)) : xb;
+    const uint32_t sign = (xb >> 31) << sign_shift;
+    const uint32_t a = yb & 0x7FFFFFFFu;
+    const uint32_t ax = xb & 0x7FFFFFFFu;
+    const uint32_t qn = (a + p.round_add + ((a >> p.drop) & p.lsb_mask)) & p.keep_mask;
+    const float magic = __uint_as_float(p.magic);
+    const float sum = add_ieee(__uint_as_float(a), magic);
+    const uint32_t cnt = __float_as_uint(sum) - p.magic;
+    const uint32_t qd = __float_as_uint(sub_ieee(sum, magic));
+    const uint32_t qa = (a < p.min_normal) ? qd : qn;
+    const int code = (int)(qa >> 23) - p.code_off;
+    const int m = 23 - (int)p.drop;
+    uint32_t packed = (qa - ((uint32_t)p.code_off << 23)) >> p.drop;
+    bin = code;
+    if (code >= p.top) {  // overflow, infinite or NaN
+        const bool is_nan = ax > 0x7F800000u;
+        packed = ((uint32_t)p.top << m) | (is_nan ? (1u << (m - 1)) : 0u);
+        bin = p.top + (is_nan ? kBinNanIn : (ax == 0x7F800000u ? kBinInfIn : kBinOverflow));
+    } else if (code <= 0) {  // zero or denormal of the format
+        bin = p.top + (ax == 0u ? kBinZeroIn : (cnt == 0u ? kBinRoundedToZero : kBinDenormal));
+        packed = p.keep_denormals ? cnt : 0u;
+    }
+    return sign | packed;
+}
+
+// fp32 container of a packed code.
+__device__ __forceinline__ uint32_t unpack_one(uint32_t code, const QuantParams& p, int sign_shift) {
+    const int m = 23 - (int)p.drop;
+    const uint32_t sign = ((code >> sign_shift) & 1u) << 31;
+    const uint32_t E = (code >> m) & (uint32_t)p.top, f = code & ((1u << m) - 1u);
+    if (E == (uint32_t)p.top) return sign | (f ? 0x7FC00000u : 0x7F800000u);
+    if (E == 0u) {  // f multiples of the smallest denormal 2^(E_min - m): exact, also when that is an fp32 denormal
+        const float quantum = mul_ieee(__uint_as_float(p.magic), 1.1920928955078125e-07f);  // magic = 2^(E_min - m + 23)
+        return sign | __float_as_uint(mul_ieee((float)f, quantum));
+    }
+    return sign | ((E + (uint32_t)p.code_off) << 23) | (f << p.drop);
+}
+
 // Folds one bin's block total into the device record.
 __device__ __forceinline__ void merge_bin(qfmt_stats_t* st, const QuantParams& p, int bin, unsigned long long c) {
     auto add = [](uint64_t* dst, unsigned long long v) { atomicAdd((unsigned long long*)dst, v); };
