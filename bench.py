@@ -327,6 +327,30 @@ def epilogue_section(torch, qf, dev, peaks, reps=20):
                          "algorithmic_bytes_per_launch": rows * cols * BYTES_PER_ELEMENT}}
 
 
+def pack16_section(torch, qf, dev, peaks, d_in, n, reps=20):
+    """16-bit storage on the config2 tensor: the rounding pass writing packed codes (4 B read + 2 B
+    written per element) and the expansion back to fp32 containers (2 B read + 4 B written)."""
+    codes = torch.empty(n, dtype=torch.int16, device=dev)
+    out = torch.empty(n, dtype=torch.float32, device=dev)
+    st = torch.zeros(qf.STATS_WORDS, dtype=torch.int64, device=dev)
+    fmt = qf.make_format(6, 9, 1, 2.0 ** 8)
+    res = {}
+    for name, fn in (("pack", lambda: qf.qfmt_quantize_stats_pack16(d_in, codes, n, fmt, st)),
+                     ("unpack", lambda: qf.qfmt_unpack16(codes, out, n, fmt))):
+        for _ in range(3):
+            fn()
+        ms = statistics.median(time_events(torch, fn, reps))
+        gbs = n * 6 / ms / 1e6
+        res[name] = {"ms": ms, "value": gbs, "unit": "GB/s",
+                     "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                                  "frac": gbs / peaks["hbm_gbs"], "traffic": None,
+                                  "algorithmic_bytes_per_launch": n * 6}}
+    assert int(st.cpu()[256]) == n
+    return {"metric": "quantize+stats to packed 16-bit codes GB/s", "value": res["pack"]["value"], "unit": "GB/s",
+            "workload": f"config2 tensor, {n} elements, 1/6/9 with loss scale 2^8 (6 B per element)",
+            "gpu_launches_per_step": 2, "roofline": res["pack"]["roofline"], "runs": res}
+
+
 # FMAC-8 is plain-ALU work.  Peak = SMs x 4 schedulers x 32 lanes x max SM clock / (scheduler cycles one
 # warp-wide multiply-add must cost).  General kernel: per FMAC FMAC8_FLOAT_OPS float-pipe instructions
 # (one per cycle) and FMAC8_INT_OPS integer-pipe instructions (one per two cycles: 16 lanes per
@@ -457,6 +481,8 @@ def run_library(args):
     extra = {}
     if "epilogue" in sections:
         extra["epilogue"] = epilogue_section(torch, qf, dev, peaks)
+    if "pack16" in sections:
+        extra["pack16"] = pack16_section(torch, qf, dev, peaks, d_in, n)
     if "fmac8" in sections:
         extra["fmac8"] = fmac8_section(torch, qf, dev, peaks, clocks.summary()["sm_max_mhz"] or 1965)
     if "e2e" in sections:
@@ -523,9 +549,9 @@ def main():
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="library", choices=["library", "reference"])
-    ap.add_argument("--sections", default="quantize,e2e,gemm,conv,epilogue,fmac8,cpu",
+    ap.add_argument("--sections", default="quantize,e2e,gemm,conv,epilogue,pack16,fmac8,cpu",
                     help="comma list of what to measure besides the timed sweep (quantize is always timed): "
-                         "e2e, gemm, conv, epilogue, fmac8, cpu; profiling captures use a subset")
+                         "e2e, gemm, conv, epilogue, pack16, fmac8, cpu; profiling captures use a subset")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
