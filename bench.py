@@ -327,6 +327,62 @@ def epilogue_section(torch, qf, dev, peaks, reps=20):
                          "algorithmic_bytes_per_launch": rows * cols * BYTES_PER_ELEMENT}}
 
 
+def step5_section(torch, qf, dev, peaks, reps=5):
+    """One training step of the config5 BERT-large FC stack with everything the path does per step:
+    for each of the four layers the operands are rounded to 1/6/9 with per-tensor statistics (X, W, and
+    dY with the device-resident loss scale), the forward layer output is Y = R(R(XW) + R(B)) with
+    statistics, the two gradient products follow, and the loss-scale controller reads the gradients'
+    overflow counts -- all enqueued on one stream, nothing returns to the host."""
+    fmt = qf.make_format(6, 9, 1)
+    state = qf.qfmt_dls_t(2.0 ** 16, 2.0, 0.5, 1.0, 2.0 ** 24, 2000, 0, 0, 0, 0, 0)
+    d_state = torch.from_numpy(np.frombuffer(bytes(state), dtype=np.uint8).copy()).to(dev)
+    layers, flops, bytes_rounded = [], 0.0, 0
+    for li in range(len(workloads.CONFIG5_LAYERS)):
+        c = workloads.config5_layer(li, step=0)
+        raw = {k: torch.from_numpy(c[k]).to(dev) for k in ("X", "W", "dY")}
+        q = {k: torch.empty_like(v) for k, v in raw.items()}
+        tokens, d_in = c["X"].shape
+        d_out = c["W"].shape[1]
+        bias = torch.from_numpy(workloads.normal_tensor(workloads.rng_for(4, 2000 + li), (d_out,), 0.02)).to(dev)
+        Y = torch.empty(tokens, d_out, dtype=torch.float32, device=dev)
+        dX = torch.empty(tokens, d_in, dtype=torch.float32, device=dev)
+        dW = torch.empty(d_in, d_out, dtype=torch.float32, device=dev)
+        fwd = (qf.make_matrix(q["X"]), qf.make_matrix(q["W"]))
+        dg = (qf.make_matrix(q["dY"]), qf.make_matrix(q["W"], True))
+        wg = (qf.make_matrix(q["X"], True), qf.make_matrix(q["dY"]))
+        wb = max(qf.qfmt_linear_forward_workspace_bytes(*fwd), qf.qfmt_gemm_workspace_bytes(*dg),
+                 qf.qfmt_gemm_workspace_bytes(*wg), 256)
+        layers.append((raw, q, bias, Y, dX, dW, fwd, dg, wg, torch.zeros(wb, dtype=torch.uint8, device=dev), wb,
+                       d_out, d_in))
+        flops += 3 * 2.0 * tokens * d_in * d_out
+        bytes_rounded += BYTES_PER_ELEMENT * (sum(v.numel() for v in raw.values()) + tokens * d_out)
+    stats = torch.zeros(len(layers), 4, qf.STATS_WORDS, dtype=torch.int64, device=dev)   # X, W, -, Y per layer
+    grad_stats = torch.zeros(len(layers), qf.STATS_WORDS, dtype=torch.int64, device=dev)
+
+    def step():
+        for li, (raw, q, bias, Y, dX, dW, fwd, dg, wg, ws, wb, d_out, d_in) in enumerate(layers):
+            qf.qfmt_quantize_stats(raw["X"], q["X"], raw["X"].numel(), fmt, stats[li, 0])
+            qf.qfmt_quantize_stats(raw["W"], q["W"], raw["W"].numel(), fmt, stats[li, 1])
+            qf.qfmt_quantize_stats_dls(raw["dY"], q["dY"], raw["dY"].numel(), fmt, d_state, grad_stats[li])
+            qf.qfmt_linear_forward(fwd[0], fwd[1], bias, Y, d_out, fmt, stats[li, 3], 0, ws, wb)
+            qf.qfmt_gemm(dg[0], dg[1], dX, d_in, fmt, ws, wb)
+            qf.qfmt_gemm(wg[0], wg[1], dW, d_out, fmt, ws, wb)
+        qf.qfmt_dls_update(d_state, grad_stats, len(layers))
+    for _ in range(3):
+        step()
+    for l in layers:
+        assert qf.qfmt_device_status(l[9]) == qf.QFMT_OK
+    ms = statistics.median(time_events(torch, step, reps))
+    final = qf.qfmt_dls_t.from_buffer_copy(d_state.cpu().numpy().tobytes())
+    return {"metric": "config5 training step, ms", "value": ms, "unit": "ms", "higher_is_better": False,
+            "workload": "config5 step: 4 layers x (round X, W, dY with statistics; Y = R(R(XW)+R(B)) with statistics; "
+                        "dgrad; wgrad) + loss-scale controller, 1/6/9, loss scale 2^16 kept on the device",
+            "ms_per_step": ms, "gemm_tflops_over_whole_step": flops / ms / 1e9,
+            "rounded_bytes_per_step": bytes_rounded, "gpu_launches_per_step": 7 * len(layers) + 1,
+            "steps_seen_by_controller": int(final.n_steps), "steps_skipped": int(final.n_skipped),
+            "loss_scale": float(final.scale)}
+
+
 def pack16_section(torch, qf, dev, peaks, d_in, n, reps=20):
     """16-bit storage on the config2 tensor: the rounding pass writing packed codes (4 B read + 2 B
     written per element) and the expansion back to fp32 containers (2 B read + 4 B written)."""
@@ -481,6 +537,8 @@ def run_library(args):
     extra = {}
     if "epilogue" in sections:
         extra["epilogue"] = epilogue_section(torch, qf, dev, peaks)
+    if "step5" in sections:
+        extra["step5"] = step5_section(torch, qf, dev, peaks)
     if "pack16" in sections:
         extra["pack16"] = pack16_section(torch, qf, dev, peaks, d_in, n)
     if "fmac8" in sections:
@@ -549,9 +607,9 @@ def main():
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="library", choices=["library", "reference"])
-    ap.add_argument("--sections", default="quantize,e2e,gemm,conv,epilogue,pack16,fmac8,cpu",
+    ap.add_argument("--sections", default="quantize,e2e,gemm,conv,epilogue,step5,pack16,fmac8,cpu",
                     help="comma list of what to measure besides the timed sweep (quantize is always timed): "
-                         "e2e, gemm, conv, epilogue, pack16, fmac8, cpu; profiling captures use a subset")
+                         "e2e, gemm, conv, epilogue, step5, pack16, fmac8, cpu; profiling captures use a subset")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
