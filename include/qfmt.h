@@ -197,6 +197,9 @@ int qfmt_quantize_stats_dls(const float* d_in, float* d_out, size_t n, const qfm
  * SYNCHRONISES the stream before returning.  The caller lends device scratch:
  *   d_work   device, 16-byte aligned, at least qfmt_quantize_stats_host_work_bytes(n) bytes
  * For full copy speed h_in / h_out should be page-locked.  h_stats is overwritten.
+ * Tensors of more than 2 Mi elements are moved in pieces on two internal streams (created once
+ * per GPU, on first use), so that the copy to the device, the rounding and the copy back overlap;
+ * the call still starts after the work already on `stream` and returns when everything is done.
  */
 int qfmt_quantize_stats_host(const float* h_in, float* h_out, size_t n, const qfmt_format_t* fmt,
                              qfmt_stats_t* h_stats, void* d_work, size_t work_bytes, void* stream);

@@ -25,6 +25,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <mutex>
+
 #include "common.cuh"
 #include "round.cuh"
 
@@ -747,6 +749,34 @@ extern "C" size_t qfmt_quantize_stats_host_work_bytes(size_t n) {
     return ((n * sizeof(float) + 255u) & ~(size_t)255u) + sizeof(qfmt_stats_t);
 }
 
+namespace qfmt {
+namespace {
+
+// Two helper streams per device for the host-buffer entry point: the copy to the device, the
+// kernel and the copy back run on three streams so that the two directions of the link work at the
+// same time.  Created on first use and kept until the process ends.
+constexpr size_t kHostChunk = (size_t)2 << 20;  // elements per pipeline step (8 MiB)
+struct HostPipe {
+    cudaStream_t in = nullptr, out = nullptr;
+};
+int host_pipe(int ordinal, HostPipe* pipe) {
+    static std::mutex mu;
+    static HostPipe pipes[64];
+    if (ordinal < 0 || ordinal >= 64) return QFMT_ERR_BAD_ARG;
+    std::lock_guard<std::mutex> lock(mu);
+    if (pipes[ordinal].in == nullptr) {
+        HostPipe hp;
+        QFMT_CUDA_TRY(cudaStreamCreateWithFlags(&hp.in, cudaStreamNonBlocking));
+        QFMT_CUDA_TRY(cudaStreamCreateWithFlags(&hp.out, cudaStreamNonBlocking));
+        pipes[ordinal] = hp;
+    }
+    *pipe = pipes[ordinal];
+    return QFMT_OK;
+}
+
+}  // namespace
+}  // namespace qfmt
+
 extern "C" int qfmt_quantize_stats_host(const float* h_in, float* h_out, size_t n, const qfmt_format_t* fmt,
                                         qfmt_stats_t* h_stats, void* d_work, size_t work_bytes, void* stream_) {
     cudaStream_t stream = (cudaStream_t)stream_;
@@ -758,13 +788,58 @@ extern "C" int qfmt_quantize_stats_host(const float* h_in, float* h_out, size_t 
     float* d_buf = reinterpret_cast<float*>(d_work);
     qfmt_stats_t* d_stats = reinterpret_cast<qfmt_stats_t*>(reinterpret_cast<char*>(d_work) +
                                                             ((n * sizeof(float) + 255u) & ~(size_t)255u));
-    if (n) QFMT_CUDA_TRY(cudaMemcpyAsync(d_buf, h_in, n * sizeof(float), cudaMemcpyHostToDevice, stream));
-    rc = qfmt::quantize_stats_device(d_buf, h_out ? d_buf : nullptr, n, fmt, h_stats ? d_stats : nullptr, 0, stream,
-                                     nullptr);
+    if (n <= qfmt::kHostChunk) {  // one piece: everything in order on the caller's stream
+        if (n) QFMT_CUDA_TRY(cudaMemcpyAsync(d_buf, h_in, n * sizeof(float), cudaMemcpyHostToDevice, stream));
+        rc = qfmt::quantize_stats_device(d_buf, h_out ? d_buf : nullptr, n, fmt, h_stats ? d_stats : nullptr, 0, stream,
+                                         nullptr);
+        if (rc != QFMT_OK) return rc;
+        if (n && h_out) QFMT_CUDA_TRY(cudaMemcpyAsync(h_out, d_buf, n * sizeof(float), cudaMemcpyDeviceToHost, stream));
+        if (h_stats) QFMT_CUDA_TRY(cudaMemcpyAsync(h_stats, d_stats, sizeof(qfmt_stats_t), cudaMemcpyDeviceToHost, stream));
+        QFMT_CUDA_TRY(cudaStreamSynchronize(stream));
+        return QFMT_OK;
+    }
+    // Pipeline over pieces of the tensor: piece i+1 travels to the device while piece i is rounded and
+    // piece i-1 travels back.  Each piece has its own place in d_work, so nothing is overwritten.
+    qfmt::DeviceInfo dev;
+    rc = qfmt::current_device(&dev);
     if (rc != QFMT_OK) return rc;
-    if (n && h_out) QFMT_CUDA_TRY(cudaMemcpyAsync(h_out, d_buf, n * sizeof(float), cudaMemcpyDeviceToHost, stream));
-    if (h_stats) QFMT_CUDA_TRY(cudaMemcpyAsync(h_stats, d_stats, sizeof(qfmt_stats_t), cudaMemcpyDeviceToHost, stream));
-    QFMT_CUDA_TRY(cudaStreamSynchronize(stream));
+    qfmt::HostPipe pipe;
+    rc = qfmt::host_pipe(dev.ordinal, &pipe);
+    if (rc != QFMT_OK) return rc;
+    cudaEvent_t ev_in = nullptr, ev_k = nullptr;
+    QFMT_CUDA_TRY(cudaEventCreateWithFlags(&ev_in, cudaEventDisableTiming));
+    if (cudaEventCreateWithFlags(&ev_k, cudaEventDisableTiming) != cudaSuccess) {
+        cudaEventDestroy(ev_in);
+        return QFMT_ERR_CUDA;
+    }
+    cudaError_t err = cudaEventRecord(ev_k, stream);  // work already on the caller's stream comes first
+    if (err == cudaSuccess) err = cudaStreamWaitEvent(pipe.in, ev_k, 0);
+    if (err == cudaSuccess) err = cudaStreamWaitEvent(pipe.out, ev_k, 0);
+    for (size_t off = 0, piece = 0; off < n && err == cudaSuccess && rc == QFMT_OK; off += qfmt::kHostChunk, ++piece) {
+        const size_t len = n - off < qfmt::kHostChunk ? n - off : qfmt::kHostChunk;
+        err = cudaMemcpyAsync(d_buf + off, h_in + off, len * sizeof(float), cudaMemcpyHostToDevice, pipe.in);
+        if (err == cudaSuccess) err = cudaEventRecord(ev_in, pipe.in);
+        if (err == cudaSuccess) err = cudaStreamWaitEvent(stream, ev_in, 0);
+        if (err != cudaSuccess) break;
+        rc = qfmt::quantize_stats_device(d_buf + off, h_out ? d_buf + off : nullptr, len, fmt, h_stats ? d_stats : nullptr,
+                                         piece == 0 ? 0 : 1, stream, nullptr);
+        if (rc != QFMT_OK) break;
+        if (h_out) {
+            err = cudaEventRecord(ev_k, stream);
+            if (err == cudaSuccess) err = cudaStreamWaitEvent(pipe.out, ev_k, 0);
+            if (err == cudaSuccess)
+                err = cudaMemcpyAsync(h_out + off, d_buf + off, len * sizeof(float), cudaMemcpyDeviceToHost, pipe.out);
+        }
+    }
+    if (err == cudaSuccess && rc == QFMT_OK && h_stats)
+        err = cudaMemcpyAsync(h_stats, d_stats, sizeof(qfmt_stats_t), cudaMemcpyDeviceToHost, stream);
+    // everything that was enqueued is waited for, also after an error, before the events go
+    cudaError_t e1 = cudaStreamSynchronize(pipe.in), e2 = cudaStreamSynchronize(stream), e3 = cudaStreamSynchronize(pipe.out);
+    cudaEventDestroy(ev_in);
+    cudaEventDestroy(ev_k);
+    if (rc != QFMT_OK) return rc;
+    if (err == cudaSuccess) err = e1 != cudaSuccess ? e1 : (e2 != cudaSuccess ? e2 : e3);
+    QFMT_CUDA_TRY(err);
     return QFMT_OK;
 }
 

@@ -170,6 +170,35 @@ def test_host_buffer_entry_point():
     assert np.array_equal(h_st.numpy().view(np.uint64), st_ref)
 
 
+def test_host_buffer_entry_point_pipelined_pieces():
+    """More than 2 Mi elements: the tensor crosses the link in pieces on the library's own streams
+    while earlier pieces are rounded and returned; values and the accumulated statistics are those
+    of one pass.  Also without an output tensor (statistics only) and twice in a row."""
+    n = (20 << 20) + 3
+    x = workloads.lognormal_tensor(workloads.rng_for(55), (n,), -18.0, 8.0, p_zero=0.005)
+    q_ref, st_ref = oracle.quantize_stats(x, 5, 10, 0, 2.0 ** 8)
+    h_in = torch.from_numpy(x).pin_memory()
+    h_out = torch.empty(n, dtype=torch.float32).pin_memory()
+    h_st = torch.zeros(qf.STATS_WORDS, dtype=torch.int64).pin_memory()
+    wb = qf.qfmt_quantize_stats_host_work_bytes(n)
+    d_work = torch.empty(wb, dtype=torch.uint8, device="cuda:0")
+    fmt = qf.make_format(5, 10, 0, 2.0 ** 8)
+    for _ in range(2):
+        h_out.zero_()
+        qf.qfmt_quantize_stats_host(h_in, h_out, n, fmt, h_st, d_work, wb)
+        assert np.array_equal(h_out.numpy().view(np.uint32), q_ref.view(np.uint32))
+        assert np.array_equal(h_st.numpy().view(np.uint64), st_ref)
+    h_st.zero_()
+    qf.qfmt_quantize_stats_host(h_in, None, n, fmt, h_st, d_work, wb)
+    assert np.array_equal(h_st.numpy().view(np.uint64), st_ref)
+    # on a side stream, after work that is already queued there
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        h_out.zero_()
+        qf.qfmt_quantize_stats_host(h_in, h_out, n, fmt, None, d_work, wb, stream=side)
+    assert np.array_equal(h_out.numpy().view(np.uint32), q_ref.view(np.uint32))
+
+
 def test_errors_leave_outputs_untouched():
     d = torch.ones(16, dtype=torch.float32, device="cuda:0")
     with pytest.raises(qf.QfmtError) as ei:
