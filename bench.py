@@ -596,7 +596,7 @@ def finish(args, world, value, total_ms, n, runs, clocks, e2e, roofline, cpu, ge
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the quantize+stats kernel, from the
 # ncu capture summarised in profiles/quantize_stats_kernel_config2.md (set to None when the kernel changes).
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 268464640 + 218681088
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 268463872 + 218315520
 # the same for the layer-output kernel on the 8192 x 4096 product (profiles/bias_quantize_stats_kernel_config5.md)
 NCU_EPILOGUE_TRAFFIC_BYTES_PER_LAUNCH = 134290688 + 85444352
 
