@@ -212,7 +212,19 @@ def gemm_section(torch, qf, dev, peaks, reps=5):
     del a, b, c
     achieved = flops / ms / 1e9
     peak = peaks["bf16_tflops"] * (1.1 / 2.25)  # TF32 dense is nominally 1.1/2.25 of bf16 dense
-    return {"metric": "emulated GEMM TFLOP/s", "value": achieved, "unit": "TFLOP/s",
+    # the fp64 oracle on this machine's host cores (OpenMP over outputs): 2^18 sampled outputs of the first product
+    import oracle
+    a0, b0, _, n0, (A0, B0) = jobs[0]
+    hA, hB = A0.cpu().numpy(), B0.cpu().numpy()
+    rng = np.random.default_rng(0)
+    ii, jj = rng.integers(0, hA.shape[0], size=1 << 18), rng.integers(0, hB.shape[1], size=1 << 18)
+    t0 = time.perf_counter()
+    oracle.gemm_sampled(hA, hB, ii, jj)
+    cpu_s = time.perf_counter() - t0
+    cpu = {"value": 2.0 * ii.size * hA.shape[1] / cpu_s / 1e12, "unit": "TFLOP/s", "cores": os.cpu_count(),
+           "kind": "oracle", "seconds": cpu_s,
+           "sample": f"{ii.size} sampled outputs of the {hA.shape[0]} x {hB.shape[1]} x {hA.shape[1]} forward product"}
+    return {"metric": "emulated GEMM TFLOP/s", "value": achieved, "unit": "TFLOP/s", "cpu_baseline": cpu,
             "workload": "config5 BERT-large FC stack, one step: 4 layers x fwd/dgrad/wgrad, 1/6/9",
             "ms_per_step": ms, "gemms_per_step": len(jobs), "gpu_launches_per_step": len(jobs),
             "roofline": {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
