@@ -420,13 +420,14 @@ def pack16_section(torch, qf, dev, peaks, d_in, n, reps=20):
 
 
 # FMAC-8 is plain-ALU work.  Peak = SMs x 4 schedulers x 32 lanes x max SM clock / (scheduler cycles one
-# warp-wide multiply-add must cost).  General kernel: per FMAC FMAC8_FLOAT_OPS float-pipe instructions
+# warp-wide multiply-add must cost).  General kernel: per FMAC FMAC8_FLOAT_OPS float-pipe instructions (two
+# directed fused multiply-adds, add and subtract of the rounding constant)
 # (one per cycle) and FMAC8_INT_OPS integer-pipe instructions (one per two cycles: 16 lanes per
 # scheduler), counted in the kernel's inner loop; the bound is the larger of the issue slots and the
 # integer pipe.  Binary16 kernel: one fma.rn.f16x2 per two FMACs, two cycles each on this part (the
 # float pipe's busy cycles are twice its instruction count for a stream of them).
 SM_COUNT, LANES_PER_SM = 148, 128
-FMAC8_FLOAT_OPS, FMAC8_INT_OPS = 5.0, 6.0
+FMAC8_FLOAT_OPS, FMAC8_INT_OPS = 4.0, 6.0
 
 
 def fmac8_section(torch, qf, dev, peaks, clock_mhz, reps=3):

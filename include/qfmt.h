@@ -302,9 +302,8 @@ int qfmt_linear_fusion_policy(int policy);
  *   A, B     as for qfmt_gemm (operands already hold values of the format; not re-rounded), but
  *            only 4-byte alignment is needed and any leading dimension >= the stored row length
  *   d_C      device, M x N floats, leading dimension ldc >= N, 4-byte aligned
- *   fmt      e <= 7 and m <= 10 (QFMT_ERR_BAD_FORMAT otherwise: the product of two values must be
- *            exact and finite in fp32); fmt->denormals selects whether the small accumulator and
- *            the result keep denormals or flush them; fmt->loss_scale is ignored
+ *   fmt      m <= 10 (QFMT_ERR_BAD_FORMAT otherwise); fmt->denormals selects whether the small
+ *            accumulator and the result keep denormals or flush them; fmt->loss_scale is ignored
  *   d_stats  device or NULL: statistics of the OUTPUT tensor (Table II of the paper reports the
  *            denormal fraction of tensors produced this way), with the master accumulator in the
  *            role of the input of qfmt_quantize_stats; accumulate as there

@@ -9,12 +9,10 @@
 // plain-ALU work (a few dozen integer/float instructions per multiply-add, or one HFMA2 per two
 // multiply-adds for binary16, which the ALUs implement natively); operand traffic is negligible
 // beside it.  Two kernels:
-//   * fmac8_kernel, any format with e <= 7 and m <= 10.  The product of two format values is
-//     exact in fp32 (at most 22 significant bits, exponent within fp32's range for e <= 7).
-//     The exact sum a + x*y is rounded ONCE by forming it to 24 bits with round-to-odd (the two
-//     directed fp32 additions; when they differ the one with an odd last bit is taken) and then
-//     rounding to m+1 bits to nearest-even: a sticky last bit 13 or more places below the target's
-//     last place cannot create or hide a tie.
+//   * fmac8_kernel, any format with m <= 10.  The exact value a + x*y is rounded ONCE by forming
+//     it to 24 bits with round-to-odd (the two directed fp32 fused multiply-adds; when they differ
+//     the one with an odd last bit is taken) and then rounding to m+1 bits to nearest-even: a
+//     sticky last bit 13 or more places below the target's last place cannot create or hide a tie.
 //   * fmac8_f16_kernel, 1/5/10: fma.rn.f16x2 is this very operation for IEEE binary16 with
 //     denormals; flushing formats clear results below 2^-14 afterwards.
 // They keep a 64 x 64 (resp. 64 x 128) tile of outputs per block in registers and stream
@@ -43,46 +41,61 @@ struct FmacParams {
     int vec_store;  // C rows 16-byte aligned
 };
 
-// a + prod rounded to 24 bits with round-to-odd: the two directed sums are equal when the sum is
-// exact and adjacent fp32 numbers otherwise, exactly one of which has an odd last bit.  (An exact
-// cancellation gives -0 and +0; the even-looking -0 loses, so +0 comes out as in round-to-nearest.)
-__device__ __forceinline__ uint32_t add_to_odd(float a, float prod) {
+// a + x*y rounded to 24 bits with round-to-odd.  The two directed fused multiply-adds (exact
+// product, one rounding) are equal when the value is exact and adjacent fp32 numbers otherwise,
+// exactly one of which has an odd last bit.  (An exact cancellation gives -0 and +0; the
+// even-looking -0 loses, so +0 comes out as in round-to-nearest.)  Nothing is required of the
+// product's range: beyond fp32's largest the pair is (largest, inf) and the odd "largest" rounds
+// to the format's infinity afterwards; below its smallest denormal the pair is (0, 2^-149) and the
+// odd 2^-149 is a sticky bit far below every format's quantum.
+__device__ __forceinline__ uint32_t fma_to_odd(float a, float x, float y) {
     float lo, hi;
-    asm("add.rm.f32 %0, %1, %2;" : "=f"(lo) : "f"(a), "f"(prod));
-    asm("add.rp.f32 %0, %1, %2;" : "=f"(hi) : "f"(a), "f"(prod));
+    asm("fma.rm.f32 %0, %1, %2, %3;" : "=f"(lo) : "f"(x), "f"(y), "f"(a));
+    asm("fma.rp.f32 %0, %1, %2, %3;" : "=f"(hi) : "f"(x), "f"(y), "f"(a));
     const uint32_t l = __float_as_uint(lo), h = __float_as_uint(hi);
     return (l & 1u) ? l : h;
 }
 
 struct SmallRound {
     uint32_t min_normal;  // fp32 bits of 2^E_min
-    uint32_t inf_bits;    // fp32 bits of 2^(E_max+1)
+    uint32_t inf_bits;    // fp32 bits of 2^(E_max+1) (of +inf for e = 8)
     uint32_t magic_add;   // ((23 - m) << 23) | 0x400000
+    uint32_t big_exp;     // e = 8: exponent fields above this one take the integer rounding
+    uint32_t drop, round_add, keep_mask;
 };
 
 // Rounds a 24-bit intermediate to the format (the small accumulator's rounding; no statistics).
 // With C = 1.5 * 2^(max(floor(log2|s|), E_min) + 23 - m), the fp32 sum s + C stays in C's binade,
 // whose last place is the format's quantum for s, so (s + C) - C is s rounded to nearest-even on
 // the format's grid, normal or denormal, either sign (a zero result may come out as +0 where -0 is
-// meant; nothing downstream can tell: it is only ever added to other numbers).  For e = 7 the sum
-// a + x*y can approach 2^128, so the exponent is capped at E_max+1 to keep C finite (kCap); values
-// that reach 2^(E_max+1) are made infinite (or the quiet NaN) afterwards.
-template <bool kFlush, bool kCap>
+// meant; nothing downstream can tell: it is only ever added to other numbers).  kWide = 1 (e = 7):
+// a + x*y can approach 2^128, so the exponent is capped at E_max+1 to keep C finite; whatever
+// reaches 2^(E_max+1) is made infinite afterwards.  kWide = 2 (e = 8): values up to fp32's largest
+// are values of the format, and near the top C would leave fp32's range; those few take the
+// integer rounding of the fp32 word instead.
+template <bool kFlush, int kWide>
 __device__ __forceinline__ float round_small(uint32_t s, const SmallRound& r) {
     uint32_t ec = s & 0x7F800000u;
-    ec = ec < r.min_normal ? r.min_normal : ec;
-    if (kCap) ec = ec > r.inf_bits ? r.inf_bits : ec;
-    const float c = __uint_as_float(ec + r.magic_add);
-    float q = sub_ieee(add_ieee(__uint_as_float(s), c), c);
+    float q;
+    if (kWide == 2 && ec > r.big_exp) {
+        const uint32_t a = s & 0x7FFFFFFFu;
+        const uint32_t qa = a > 0x7F800000u ? 0x7FC00000u : ((a + r.round_add + ((a >> r.drop) & 1u)) & r.keep_mask);
+        q = __uint_as_float((s & 0x80000000u) | qa);
+    } else {
+        ec = ec < r.min_normal ? r.min_normal : ec;
+        if (kWide == 1) ec = ec > r.inf_bits ? r.inf_bits : ec;
+        const float c = __uint_as_float(ec + r.magic_add);
+        q = sub_ieee(add_ieee(__uint_as_float(s), c), c);
+    }
     if (!(fabsf(q) < __uint_as_float(r.inf_bits)))
         q = (q != q) ? __uint_as_float(0x7FC00000u) : copysignf(__uint_as_float(0x7F800000u), q);
     if (kFlush && fabsf(q) < __uint_as_float(r.min_normal)) q = 0.0f;
     return q;
 }
 
-template <bool kFlush, bool kCap>
+template <bool kFlush, int kWide>
 __device__ __forceinline__ float fmac(float acc, float x, float y, const SmallRound& r) {
-    return round_small<kFlush, kCap>(add_to_odd(acc, mul_ieee(x, y)), r);
+    return round_small<kFlush, kWide>(fma_to_odd(acc, x, y), r);
 }
 
 // One 32-deep slice of op(A) (rows m0.., kBM of them) into shared memory as [k][m]; elements
@@ -145,13 +158,13 @@ __device__ __forceinline__ void merge_block_hist(qfmt_stats_t* stats, const Quan
         atomicAdd((unsigned long long*)&stats->n_total, n_total);
 }
 
-// ---- any format with e <= 7, m <= 10 --------------------------------------------------------
+// ---- any format with m <= 10 ----------------------------------------------------------------
 // 4 x 4 outputs per thread: the FMAC chain of one output is a dozen dependent instructions, so
 // many resident warps (four blocks per SM) hide more latency than a larger patch per thread would.
 constexpr int kFmBM = 64, kFmBN = 64, kFmTM = 4, kFmTN = 4;
 constexpr int kFmBlocksPerSm = 4;
 
-template <bool kStats, bool kFlush, bool kCap>
+template <bool kStats, bool kFlush, int kWide>
 __global__ void __launch_bounds__(kFmThreads, kFmBlocksPerSm)
 fmac8_kernel(FmacParams g, QuantParams p, qfmt_stats_t* __restrict__ stats) {
     __shared__ __align__(16) float As[kFmBK][kFmBM + 4];
@@ -167,6 +180,10 @@ fmac8_kernel(FmacParams g, QuantParams p, qfmt_stats_t* __restrict__ stats) {
     sr.min_normal = p.min_normal;
     sr.inf_bits = (uint32_t)(p.top + p.code_off) << 23;
     sr.magic_add = p.magic_add;
+    sr.big_exp = (254u - p.drop) << 23;
+    sr.drop = p.drop;
+    sr.round_add = p.round_add;
+    sr.keep_mask = p.keep_mask;
     const int tx = threadIdx.x % 16, ty = threadIdx.x / 16;
     const int tiles_n = (g.N + kFmBN - 1) / kFmBN, tiles_m = (g.M + kFmBM - 1) / kFmBM;
     auto same = [](float v) { return v; };
@@ -194,7 +211,7 @@ fmac8_kernel(FmacParams g, QuantParams p, qfmt_stats_t* __restrict__ stats) {
 #pragma unroll
                     for (int i = 0; i < kFmTM; ++i)
 #pragma unroll
-                        for (int j = 0; j < kFmTN; ++j) small[i][j] = fmac<kFlush, kCap>(small[i][j], a[i], b[j], sr);
+                        for (int j = 0; j < kFmTN; ++j) small[i][j] = fmac<kFlush, kWide>(small[i][j], a[i], b[j], sr);
                 }
                 // the group's sum moves to the master accumulator (fp32 addition)
 #pragma unroll
@@ -344,7 +361,7 @@ int gemm_fmac8_device(const qfmt_matrix_t* A, const qfmt_matrix_t* B, float* d_C
                       qfmt_stats_t* d_stats, int accumulate, int path, cudaStream_t stream) {
     int rc = validate_format(fmt);
     if (rc != QFMT_OK) return rc;
-    if (fmt->m > 10 || fmt->e > 7) return QFMT_ERR_BAD_FORMAT;  // products must be exact and finite in fp32
+    if (fmt->m > 10) return QFMT_ERR_BAD_FORMAT;  // operands of at most 11 significant bits
     if (A == nullptr || B == nullptr) return QFMT_ERR_BAD_ARG;
     if (accumulate != 0 && accumulate != 1) return QFMT_ERR_BAD_ARG;
     if (path < 0 || path > 2) return QFMT_ERR_BAD_ARG;
@@ -394,16 +411,23 @@ int gemm_fmac8_device(const qfmt_matrix_t* A, const qfmt_matrix_t* B, float* d_C
         const long long tiles = ((M + kFmBM - 1) / kFmBM) * ((N + kFmBN - 1) / kFmBN);
         const long long cap = (long long)dev.sm_count * kFmBlocksPerSm;
         const unsigned grid = (unsigned)(tiles < cap ? tiles : cap);
-        const bool flush = fmt->denormals == 0, cap_exp = fmt->e == 7;
+        const bool flush = fmt->denormals == 0;
+        const int wide = fmt->e == 8 ? 2 : (fmt->e == 7 ? 1 : 0);
         const size_t sm = has_stats ? smem : 0;
-#define QFMT_FLAUNCH(S, F, C) fmac8_kernel<S, F, C><<<grid, kFmThreads, sm, stream>>>(g, p, d_stats)
-        if (has_stats) {
-            if (flush) { if (cap_exp) QFMT_FLAUNCH(true, true, true); else QFMT_FLAUNCH(true, true, false); }
-            else { if (cap_exp) QFMT_FLAUNCH(true, false, true); else QFMT_FLAUNCH(true, false, false); }
-        } else {
-            if (flush) { if (cap_exp) QFMT_FLAUNCH(false, true, true); else QFMT_FLAUNCH(false, true, false); }
-            else { if (cap_exp) QFMT_FLAUNCH(false, false, true); else QFMT_FLAUNCH(false, false, false); }
-        }
+        // 256-bin histograms (e = 8) put static + dynamic shared memory past the 48 KB that need no opt-in
+#define QFMT_FLAUNCH(S, F, W)                                                                              \
+    do {                                                                                                   \
+        if (sm > 24 * 1024)                                                                                \
+            QFMT_CUDA_TRY(cudaFuncSetAttribute(fmac8_kernel<S, F, W>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm)); \
+        fmac8_kernel<S, F, W><<<grid, kFmThreads, sm, stream>>>(g, p, d_stats);                             \
+    } while (0)
+#define QFMT_FWIDE(S, F)                                                                                   \
+    do {                                                                                                   \
+        if (wide == 2) QFMT_FLAUNCH(S, F, 2); else if (wide == 1) QFMT_FLAUNCH(S, F, 1); else QFMT_FLAUNCH(S, F, 0); \
+    } while (0)
+        if (has_stats) { if (flush) QFMT_FWIDE(true, true); else QFMT_FWIDE(true, false); }
+        else { if (flush) QFMT_FWIDE(false, true); else QFMT_FWIDE(false, false); }
+#undef QFMT_FWIDE
 #undef QFMT_FLAUNCH
     }
     QFMT_CUDA_TRY(cudaGetLastError());

@@ -55,7 +55,7 @@ def paths_for(e, m):
     return (0, 1, 2) if (e, m) == (5, 10) else (0, 1)
 
 
-@pytest.mark.parametrize("e,m", [(5, 10), (6, 9), (7, 8), (4, 3)])
+@pytest.mark.parametrize("e,m", [(5, 10), (6, 9), (7, 8), (4, 3), (8, 7)])
 @pytest.mark.parametrize("den", [1, 0])
 @pytest.mark.parametrize("mu", [-2.0, -9.0])
 def test_random_operands_all_transposes(e, m, den, mu):
@@ -85,7 +85,7 @@ def test_small_integers_force_ties(e, m):
     assert np.any(c_ref != exact)   # the small accumulator really lost something
 
 
-@pytest.mark.parametrize("e,m", [(5, 10), (6, 9)])
+@pytest.mark.parametrize("e,m", [(5, 10), (6, 9), (7, 8), (8, 7)])
 @pytest.mark.parametrize("den", [1, 0])
 def test_overflow_infinities_nans_and_zeros(e, m, den):
     rng = workloads.rng_for(420 + e, den)
@@ -113,6 +113,22 @@ def test_shapes(M, N, K):
             assert c.shape == (M, N) and int(st.sum()) == 0
             continue
         check(A, B, e, m, 1, paths=paths_for(e, m))
+
+
+@pytest.mark.parametrize("den", [1, 0])
+def test_bfloat16_family_extreme_exponents(den):
+    """1/8/7: products far outside fp32's range in both directions (2^-250 .. 2^250), sums that
+    overflow fp32 before they are rounded, fp32-denormal accumulator values."""
+    rng = workloads.rng_for(445, den)
+    M, N, K = 70, 66, 50
+    e, m = 8, 7
+    A = quantized(workloads.lognormal_tensor(rng, (M, K), 0.0, 40.0, p_zero=0.05), e, m, den)
+    B = quantized(workloads.lognormal_tensor(rng, (K, N), 0.0, 40.0, p_zero=0.05), e, m, den)
+    A[:, :10] = quantized(workloads.lognormal_tensor(rng, (M, 10), -70.0, 3.0), e, m, den)   # tiny x tiny
+    B[:10, :] = quantized(workloads.lognormal_tensor(rng, (10, N), -66.0, 3.0), e, m, den)
+    A[:, 10:14] = quantized(workloads.lognormal_tensor(rng, (M, 4), 63.0, 1.0), e, m, den)   # near the top
+    B[10:14, :] = quantized(workloads.lognormal_tensor(rng, (4, N), 63.5, 1.0), e, m, den)
+    check(A, B, e, m, den)
 
 
 def test_unaligned_output_and_leading_dimension():
@@ -182,8 +198,8 @@ def test_errors():
     d = torch.ones(64, dtype=torch.float32, device=DEV)
     a = qf.make_matrix(d.data_ptr(), False, 8, 8, 8)
     with pytest.raises(qf.QfmtError) as ei:
-        qf.qfmt_gemm_fmac8(a, a, d, 8, qf.make_format(8, 7))
-    assert ei.value.status == qf.QFMT_ERR_BAD_FORMAT       # products of 1/8/m values leave the fp32 range
+        qf.qfmt_gemm_fmac8(a, a, d, 8, qf.make_format(8, 11))
+    assert ei.value.status == qf.QFMT_ERR_BAD_FORMAT       # operands of more than 11 significant bits
     with pytest.raises(qf.QfmtError) as ei:
         qf.qfmt_gemm_fmac8(a, a, d, 8, qf.make_format(6, 9), None, 0, 2)
     assert ei.value.status == qf.QFMT_ERR_BAD_FORMAT       # the binary16 kernel is for 1/5/10 only

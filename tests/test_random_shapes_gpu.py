@@ -100,7 +100,7 @@ def test_layer_output(seed):
 def test_fmac8_product(seed):
     rng = np.random.default_rng(9200 + seed)
     for _ in range(3):
-        e, m = [(5, 10), (6, 9), (7, 10), (4, 3), (6, 5)][int(rng.integers(5))]
+        e, m = [(5, 10), (6, 9), (7, 10), (4, 3), (6, 5), (8, 7)][int(rng.integers(6))]
         den = int(rng.integers(2))
         M, N, K = int(rng.integers(1, 150)), int(rng.integers(1, 150)), int(rng.integers(0, 90))
         tA, tB = bool(rng.integers(2)), bool(rng.integers(2))
