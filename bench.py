@@ -424,7 +424,7 @@ def pack16_section(torch, qf, dev, peaks, d_in, n, reps=20):
 # directed fused multiply-adds, add and subtract of the rounding constant)
 # (one per cycle) and FMAC8_INT_OPS integer-pipe instructions (one per two cycles: 16 lanes per
 # scheduler), counted in the kernel's inner loop; the bound is the larger of the issue slots and the
-# integer pipe.  Binary16 kernel: one fma.rn.f16x2 per two FMACs, two cycles each on this part (the
+# integer pipe.  Native kernel (binary16, bfloat16): one fma.rn.f16x2 / fma.rn.bf16x2 per two FMACs, two cycles each on this part (the
 # float pipe's busy cycles are twice its instruction count for a stream of them).
 SM_COUNT, LANES_PER_SM = 148, 128
 FMAC8_FLOAT_OPS, FMAC8_INT_OPS = 4.0, 6.0
@@ -432,7 +432,7 @@ FMAC8_FLOAT_OPS, FMAC8_INT_OPS = 4.0, 6.0
 
 def fmac8_section(torch, qf, dev, peaks, clock_mhz, reps=3):
     """Algorithm 1 (FMAC-8) on the config3 forward product (4096 x 3072 x 768): 1/6/9 on the general
-    ALU kernel and 1/5/10 on the half-precision FMA kernel; output statistics taken in the kernel."""
+    ALU kernel, 1/5/10 and 1/8/7 on the native 16-bit FMA kernel; output statistics taken in the kernel."""
     cfg = workloads.config3()
     M, K = cfg["X"].shape
     N = cfg["W"].shape[1]
@@ -442,7 +442,8 @@ def fmac8_section(torch, qf, dev, peaks, clock_mhz, reps=3):
     cyc_general = max(FMAC8_FLOAT_OPS + FMAC8_INT_OPS, 2.0 * FMAC8_INT_OPS)
     peaks_t = {"general": SM_COUNT * LANES_PER_SM * clk / cyc_general / 1e12,
                "binary16": SM_COUNT * LANES_PER_SM * clk * 2 / 2.0 / 1e12}
-    for tag, e, m, path, kind in (("1/6/9 general", 6, 9, 0, "general"), ("1/5/10 binary16", 5, 10, 0, "binary16")):
+    for tag, e, m, path, kind in (("1/6/9 general", 6, 9, 0, "general"), ("1/5/10 binary16", 5, 10, 0, "binary16"),
+                                  ("1/8/7 bfloat16", 8, 7, 0, "binary16")):
         fmt = qf.make_format(e, m, 1)
         X, W = torch.from_numpy(cfg["X"]).to(dev), torch.from_numpy(cfg["W"]).to(dev)
         qf.qfmt_quantize_stats(X, X, X.numel(), fmt)

@@ -308,8 +308,8 @@ int qfmt_linear_fusion_policy(int policy);
  *            denormal fraction of tensors produced this way), with the master accumulator in the
  *            role of the input of qfmt_quantize_stats; accumulate as there
  *   path     0 automatic; 1 the general kernel (integer/fp32 emulation of the FMAC on the ALUs);
- *            2 the binary16 kernel (1/5/10 only, else QFMT_ERR_BAD_FORMAT), where the FMAC is the
- *            GPU's own half-precision fused multiply-add.  Both give the same bits.
+ *            2 the native kernel (1/5/10 and 1/8/7 only, else QFMT_ERR_BAD_FORMAT), where the FMAC
+ *            is the GPU's own binary16 / bfloat16 fused multiply-add.  Both give the same bits.
  * Plain-ALU work: no tensor-core instruction rounds its accumulator to 11 bits per product.
  * M = 0 or N = 0 is a no-op; K = 0 writes +0.  NaN results are the positive quiet NaN.
  * Errors: QFMT_ERR_BAD_FORMAT, QFMT_ERR_BAD_ARG, QFMT_ERR_UNSUPPORTED_ARCH, QFMT_ERR_CUDA.

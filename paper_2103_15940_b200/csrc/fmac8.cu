@@ -13,8 +13,9 @@
 //     it to 24 bits with round-to-odd (the two directed fp32 fused multiply-adds; when they differ
 //     the one with an odd last bit is taken) and then rounding to m+1 bits to nearest-even: a
 //     sticky last bit 13 or more places below the target's last place cannot create or hide a tie.
-//   * fmac8_f16_kernel, 1/5/10: fma.rn.f16x2 is this very operation for IEEE binary16 with
-//     denormals; flushing formats clear results below 2^-14 afterwards.
+//   * fmac8_f16_kernel, 1/5/10 and 1/8/7: fma.rn.f16x2 and fma.rn.bf16x2 are this very operation
+//     for IEEE binary16 and for bfloat16 with denormals; flushing formats clear results below the
+//     smallest normal afterwards.
 // They keep a 64 x 64 (resp. 64 x 128) tile of outputs per block in registers and stream
 // 32-deep slices of the operands through shared memory.
 #include <cuda_fp16.h>
@@ -228,28 +229,41 @@ fmac8_kernel(FmacParams g, QuantParams p, qfmt_stats_t* __restrict__ stats) {
     merge_block_hist<kStats>(stats, p, lane_hist, nbins, (unsigned long long)g.M * (unsigned long long)g.N);
 }
 
-// ---- 1/5/10: the hardware's own half-precision FMA ------------------------------------------
+// ---- 1/5/10 and 1/8/7: the hardware's own 16-bit fused multiply-adds --------------------------
 constexpr int kHfBM = 64, kHfBN = 128, kHfTM = 4, kHfTN = 8;
 constexpr int kHfBlocksPerSm = 2;
 
-__device__ __forceinline__ __half2 hfma2_ieee(__half2 a, __half2 b, __half2 c) {
+// two FMACs: {a.lo * b.lo + c.lo, a.hi * b.hi + c.hi}, each rounded once to the 16-bit type
+template <bool kBf16>
+__device__ __forceinline__ uint32_t fma2_16(uint32_t a, uint32_t b, uint32_t c) {
     uint32_t r;
-    asm("fma.rn.f16x2 %0, %1, %2, %3;"  // no .ftz: denormals honoured
-        : "=r"(r)
-        : "r"(*reinterpret_cast<uint32_t*>(&a)), "r"(*reinterpret_cast<uint32_t*>(&b)),
-          "r"(*reinterpret_cast<uint32_t*>(&c)));
-    return *reinterpret_cast<__half2*>(&r);
+    if (kBf16) asm("fma.rn.bf16x2 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(c));
+    else asm("fma.rn.f16x2 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(c));  // no .ftz: denormals honoured
+    return r;
 }
 
-// clears the halves whose magnitude is below 2^-14 (0x0400), keeping their signs
-__device__ __forceinline__ __half2 flush_denormals2(__half2 v) {
-    const uint32_t u = *reinterpret_cast<uint32_t*>(&v);
+// clears the 16-bit halves whose magnitude is below the smallest normal (0x0400 = 2^-14 for
+// binary16, 0x0080 = 2^-126 for bfloat16), keeping their signs
+template <bool kBf16>
+__device__ __forceinline__ uint32_t flush_denormals2(uint32_t u) {
+    constexpr uint32_t kMinNormal = kBf16 ? 0x0080u : 0x0400u;
     const uint32_t mag = u & 0x7FFF7FFFu;
     uint32_t keep = 0x80008000u;
-    if ((mag & 0xFFFFu) >= 0x0400u) keep |= 0x00007FFFu;
-    if ((mag >> 16) >= 0x0400u) keep |= 0x7FFF0000u;
-    const uint32_t r = u & keep;
-    return *reinterpret_cast<const __half2*>(&r);
+    if ((mag & 0xFFFFu) >= kMinNormal) keep |= 0x00007FFFu;
+    if ((mag >> 16) >= kMinNormal) keep |= 0x7FFF0000u;
+    return u & keep;
+}
+
+// the 16-bit code of an fp32 container that holds a value of the type (exact)
+template <bool kBf16>
+__device__ __forceinline__ uint32_t to_16(float v) {
+    return kBf16 ? (__float_as_uint(v) >> 16) : (uint32_t)__half_as_ushort(__float2half_rn(v));
+}
+
+template <bool kBf16>
+__device__ __forceinline__ float2 pair_to_float2(uint32_t u) {
+    if (kBf16) return make_float2(__uint_as_float(u << 16), __uint_as_float(u & 0xFFFF0000u));
+    return __half22float2(*reinterpret_cast<const __half2*>(&u));
 }
 
 // The slice a thread fetches: kRows * 32 / 256 elements, in the same order load_slice uses.
@@ -268,11 +282,11 @@ __device__ __forceinline__ void fetch_slice(float (&v)[kRows * kFmBK / kFmThread
     }
 }
 
-template <bool kStats, bool kFlush>
+template <bool kStats, bool kFlush, bool kBf16>
 __global__ void __launch_bounds__(kFmThreads, kHfBlocksPerSm)
 fmac8_f16_kernel(FmacParams g, QuantParams p, qfmt_stats_t* __restrict__ stats) {
     __shared__ __align__(16) uint32_t As2[kFmBK][kHfBM + 4];  // each A value twice: {a, a} as f16x2
-    __shared__ __align__(16) __half Bs[kFmBK][kHfBN + 8];
+    __shared__ __align__(16) uint16_t Bs[kFmBK][kHfBN + 8];
     extern __shared__ uint32_t lane_hist[];
     const int nbins = p.top + kExtraBins;
     const int lane = threadIdx.x & 31;
@@ -286,8 +300,8 @@ fmac8_f16_kernel(FmacParams g, QuantParams p, qfmt_stats_t* __restrict__ stats) 
     for (long long tile = blockIdx.x; tile < (long long)tiles_m * tiles_n; tile += gridDim.x) {
         const int m0 = (int)(tile / tiles_n) * kHfBM, n0 = (int)(tile % tiles_n) * kHfBN;
         float master[kHfTM][kHfTN];
-        __half2 small[kHfTM][kHfTN / 2];
-        const __half2 zero2 = __float2half2_rn(0.0f);
+        uint32_t small[kHfTM][kHfTN / 2];  // pairs of 16-bit accumulators
+        const uint32_t zero2 = 0u;
 #pragma unroll
         for (int i = 0; i < kHfTM; ++i) {
 #pragma unroll
@@ -300,19 +314,19 @@ fmac8_f16_kernel(FmacParams g, QuantParams p, qfmt_stats_t* __restrict__ stats) 
         fetch_slice<kHfBN>(fb, g.B, g.ldb, g.transB, n0, g.N, 0, g.K);
         for (int k0 = 0; k0 < g.K; k0 += kFmBK) {
             __syncthreads();  // the previous slice is no longer read
-            // the conversions are exact: operands hold binary16 values
+            // the conversions are exact: operands hold values of the 16-bit type
 #pragma unroll
             for (int t = 0; t < kPerA; ++t) {
                 const int idx = threadIdx.x + t * kFmThreads;
-                const uint32_t ha = __half_as_ushort(__float2half_rn(fa[t]));
+                const uint32_t ha = to_16<kBf16>(fa[t]);
                 if (!g.transA) As2[idx % kFmBK][idx / kFmBK] = ha | (ha << 16);
                 else As2[idx / kHfBM][idx % kHfBM] = ha | (ha << 16);
             }
 #pragma unroll
             for (int t = 0; t < kPerB; ++t) {
                 const int idx = threadIdx.x + t * kFmThreads;
-                if (g.transB) Bs[idx % kFmBK][idx / kFmBK] = __float2half_rn(fb[t]);
-                else Bs[idx / kHfBN][idx % kHfBN] = __float2half_rn(fb[t]);
+                if (g.transB) Bs[idx % kFmBK][idx / kFmBK] = (uint16_t)to_16<kBf16>(fb[t]);
+                else Bs[idx / kHfBN][idx % kHfBN] = (uint16_t)to_16<kBf16>(fb[t]);
             }
             __syncthreads();
             if (k0 + kFmBK < g.K) {
@@ -330,11 +344,10 @@ fmac8_f16_kernel(FmacParams g, QuantParams p, qfmt_stats_t* __restrict__ stats) 
                     const uint32_t bw[kHfTN / 2] = {bv.x, bv.y, bv.z, bv.w};
 #pragma unroll
                     for (int i = 0; i < kHfTM; ++i) {
-                        const __half2 a2 = *reinterpret_cast<const __half2*>(&aw[i]);
 #pragma unroll
                         for (int j = 0; j < kHfTN / 2; ++j) {
-                            const __half2 r = hfma2_ieee(a2, *reinterpret_cast<const __half2*>(&bw[j]), small[i][j]);
-                            small[i][j] = kFlush ? flush_denormals2(r) : r;
+                            const uint32_t r = fma2_16<kBf16>(aw[i], bw[j], small[i][j]);
+                            small[i][j] = kFlush ? flush_denormals2<kBf16>(r) : r;
                         }
                     }
                 }
@@ -343,7 +356,7 @@ fmac8_f16_kernel(FmacParams g, QuantParams p, qfmt_stats_t* __restrict__ stats) 
                 for (int i = 0; i < kHfTM; ++i)
 #pragma unroll
                     for (int j = 0; j < kHfTN / 2; ++j) {
-                        const float2 v = __half22float2(small[i][j]);
+                        const float2 v = pair_to_float2<kBf16>(small[i][j]);
                         master[i][2 * j] = add_ieee(master[i][2 * j], v.x);
                         master[i][2 * j + 1] = add_ieee(master[i][2 * j + 1], v.y);
                         small[i][j] = zero2;
@@ -375,7 +388,8 @@ int gemm_fmac8_device(const qfmt_matrix_t* A, const qfmt_matrix_t* B, float* d_C
     if ((reinterpret_cast<uintptr_t>(A->ptr) & 3u) || (reinterpret_cast<uintptr_t>(B->ptr) & 3u) ||
         (reinterpret_cast<uintptr_t>(d_C) & 3u) || (reinterpret_cast<uintptr_t>(d_stats) & 7u))
         return QFMT_ERR_BAD_ARG;
-    const bool native = fmt->e == 5 && fmt->m == 10;
+    const bool bf16 = fmt->e == 8 && fmt->m == 7;
+    const bool native = (fmt->e == 5 && fmt->m == 10) || bf16;
     if (path == 2 && !native) return QFMT_ERR_BAD_FORMAT;
     DeviceInfo dev;
     rc = current_device(&dev);
@@ -400,13 +414,22 @@ int gemm_fmac8_device(const qfmt_matrix_t* A, const qfmt_matrix_t* B, float* d_C
         const long long slots = (long long)dev.sm_count * kHfBlocksPerSm;
         const unsigned grid = (unsigned)(tiles < slots ? tiles : slots);
         const bool flush = fmt->denormals == 0;
-        if (has_stats) {
-            if (flush) fmac8_f16_kernel<true, true><<<grid, kFmThreads, smem, stream>>>(g, p, d_stats);
-            else fmac8_f16_kernel<true, false><<<grid, kFmThreads, smem, stream>>>(g, p, d_stats);
-        } else {
-            if (flush) fmac8_f16_kernel<false, true><<<grid, kFmThreads, 0, stream>>>(g, p, d_stats);
-            else fmac8_f16_kernel<false, false><<<grid, kFmThreads, 0, stream>>>(g, p, d_stats);
-        }
+        const size_t sm = has_stats ? smem : 0;
+        // 256-bin histograms (bfloat16) put static + dynamic shared memory past the 48 KB that need no opt-in
+#define QFMT_HLAUNCH(S, F, B)                                                                               \
+    do {                                                                                                   \
+        if (sm > 24 * 1024)                                                                                \
+            QFMT_CUDA_TRY(cudaFuncSetAttribute(fmac8_f16_kernel<S, F, B>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm)); \
+        fmac8_f16_kernel<S, F, B><<<grid, kFmThreads, sm, stream>>>(g, p, d_stats);                         \
+    } while (0)
+#define QFMT_HTYPE(S, F)                                                                                   \
+    do {                                                                                                   \
+        if (bf16) QFMT_HLAUNCH(S, F, true); else QFMT_HLAUNCH(S, F, false);                                \
+    } while (0)
+        if (has_stats) { if (flush) QFMT_HTYPE(true, true); else QFMT_HTYPE(true, false); }
+        else { if (flush) QFMT_HTYPE(false, true); else QFMT_HTYPE(false, false); }
+#undef QFMT_HTYPE
+#undef QFMT_HLAUNCH
     } else {
         const long long tiles = ((M + kFmBM - 1) / kFmBM) * ((N + kFmBN - 1) / kFmBN);
         const long long cap = (long long)dev.sm_count * kFmBlocksPerSm;
