@@ -40,6 +40,7 @@ struct FmacParams {
     int M, N, K;
     int transA, transB;
     int vec_store;  // C rows 16-byte aligned
+    int vec_a, vec_b;  // operand base and leading dimension allow 128-bit loads
 };
 
 // a + x*y rounded to 24 bits with round-to-odd.  The two directed fused multiply-adds (exact
@@ -266,19 +267,38 @@ __device__ __forceinline__ float2 pair_to_float2(uint32_t u) {
     return __half22float2(*reinterpret_cast<const __half2*>(&u));
 }
 
-// The slice a thread fetches: kRows * 32 / 256 elements, in the same order load_slice uses.
+// The part of a 32-deep slice of an operand tile (kRows rows of op(A), or columns of op(B)) that a
+// thread fetches: kRows * 32 / 1024 groups of four elements that are consecutive in memory (four k
+// of a row when k is the contiguous index, four rows of a k otherwise).  A group inside the matrix
+// of a 16-byte aligned operand is one 128-bit load; at the edges, and for other operands, its
+// elements are loaded one by one, zero outside the matrix.
 template <int kRows>
-__device__ __forceinline__ void fetch_slice(float (&v)[kRows * kFmBK / kFmThreads], const float* src, long long ld,
-                                            int trans_k_major, int r0, int rmax, int k0, int kmax) {
+__device__ __forceinline__ void group_position(int f, int k_major, int& r, int& k) {
+    if (k_major) { r = f / (kFmBK / 4); k = 4 * (f % (kFmBK / 4)); }
+    else { k = f / (kRows / 4); r = 4 * (f % (kRows / 4)); }
+}
+template <int kRows>
+__device__ __forceinline__ void fetch_slice(float4 (&v)[kRows * kFmBK / (4 * kFmThreads)], const float* src, long long ld,
+                                            int k_major, int vec_ok, int r0, int rmax, int k0, int kmax) {
 #pragma unroll
-    for (int t = 0; t < kRows * kFmBK / kFmThreads; ++t) {
-        const int idx = threadIdx.x + t * kFmThreads;
+    for (int t = 0; t < kRows * kFmBK / (4 * kFmThreads); ++t) {
         int r, k;
-        if (trans_k_major) { k = idx % kFmBK; r = idx / kFmBK; }
-        else { r = idx % kRows; k = idx / kRows; }
-        v[t] = 0.0f;
-        if (r0 + r < rmax && k0 + k < kmax)
-            v[t] = trans_k_major ? src[(long long)(r0 + r) * ld + (k0 + k)] : src[(long long)(k0 + k) * ld + (r0 + r)];
+        group_position<kRows>(threadIdx.x + t * kFmThreads, k_major, r, k);
+        r += r0;
+        k += k0;
+        const float* ptr = k_major ? src + (long long)r * ld + k : src + (long long)k * ld + r;
+        const bool full = k_major ? (r < rmax && k + 3 < kmax) : (k < kmax && r + 3 < rmax);
+        if (vec_ok && full) {
+            v[t] = *reinterpret_cast<const float4*>(ptr);
+        } else {
+            float e[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int rr = k_major ? r : r + j, kk = k_major ? k + j : k;
+                e[j] = (rr < rmax && kk < kmax) ? (k_major ? ptr[j] : ptr[j]) : 0.0f;
+            }
+            v[t] = make_float4(e[0], e[1], e[2], e[3]);
+        }
     }
 }
 
@@ -296,7 +316,7 @@ fmac8_f16_kernel(FmacParams g, QuantParams p, qfmt_stats_t* __restrict__ stats) 
     }
     const int tx = threadIdx.x % 16, ty = threadIdx.x / 16;
     const int tiles_n = (g.N + kHfBN - 1) / kHfBN, tiles_m = (g.M + kHfBM - 1) / kHfBM;
-    constexpr int kPerA = kHfBM * kFmBK / kFmThreads, kPerB = kHfBN * kFmBK / kFmThreads;  // elements a thread moves
+    constexpr int kPerA = kHfBM * kFmBK / (4 * kFmThreads), kPerB = kHfBN * kFmBK / (4 * kFmThreads);  // groups of four a thread moves
     for (long long tile = blockIdx.x; tile < (long long)tiles_m * tiles_n; tile += gridDim.x) {
         const int m0 = (int)(tile / tiles_n) * kHfBM, n0 = (int)(tile % tiles_n) * kHfBN;
         float master[kHfTM][kHfTN];
@@ -309,29 +329,47 @@ fmac8_f16_kernel(FmacParams g, QuantParams p, qfmt_stats_t* __restrict__ stats) 
 #pragma unroll
             for (int j = 0; j < kHfTN / 2; ++j) small[i][j] = zero2;
         }
-        float fa[kPerA], fb[kPerB];  // the next slice, on its way from global memory while this one is used
-        fetch_slice<kHfBM>(fa, g.A, g.lda, !g.transA, m0, g.M, 0, g.K);
-        fetch_slice<kHfBN>(fb, g.B, g.ldb, g.transB, n0, g.N, 0, g.K);
+        float4 fa[kPerA], fb[kPerB];  // the next slice, on its way from global memory while this one is used
+        fetch_slice<kHfBM>(fa, g.A, g.lda, !g.transA, g.vec_a, m0, g.M, 0, g.K);
+        fetch_slice<kHfBN>(fb, g.B, g.ldb, g.transB, g.vec_b, n0, g.N, 0, g.K);
         for (int k0 = 0; k0 < g.K; k0 += kFmBK) {
             __syncthreads();  // the previous slice is no longer read
             // the conversions are exact: operands hold values of the 16-bit type
 #pragma unroll
             for (int t = 0; t < kPerA; ++t) {
-                const int idx = threadIdx.x + t * kFmThreads;
-                const uint32_t ha = to_16<kBf16>(fa[t]);
-                if (!g.transA) As2[idx % kFmBK][idx / kFmBK] = ha | (ha << 16);
-                else As2[idx / kHfBM][idx % kHfBM] = ha | (ha << 16);
+                int r, k;
+                group_position<kHfBM>(threadIdx.x + t * kFmThreads, !g.transA, r, k);
+                const uint32_t h0 = to_16<kBf16>(fa[t].x), h1 = to_16<kBf16>(fa[t].y), h2 = to_16<kBf16>(fa[t].z),
+                               h3 = to_16<kBf16>(fa[t].w);
+                if (!g.transA) {  // four k of one row
+                    As2[k][r] = h0 | (h0 << 16);
+                    As2[k + 1][r] = h1 | (h1 << 16);
+                    As2[k + 2][r] = h2 | (h2 << 16);
+                    As2[k + 3][r] = h3 | (h3 << 16);
+                } else {          // four rows of one k
+                    *reinterpret_cast<uint4*>(&As2[k][r]) =
+                        make_uint4(h0 | (h0 << 16), h1 | (h1 << 16), h2 | (h2 << 16), h3 | (h3 << 16));
+                }
             }
 #pragma unroll
             for (int t = 0; t < kPerB; ++t) {
-                const int idx = threadIdx.x + t * kFmThreads;
-                if (g.transB) Bs[idx % kFmBK][idx / kFmBK] = (uint16_t)to_16<kBf16>(fb[t]);
-                else Bs[idx / kHfBN][idx % kHfBN] = (uint16_t)to_16<kBf16>(fb[t]);
+                int r, k;
+                group_position<kHfBN>(threadIdx.x + t * kFmThreads, g.transB, r, k);
+                const uint32_t h0 = to_16<kBf16>(fb[t].x), h1 = to_16<kBf16>(fb[t].y), h2 = to_16<kBf16>(fb[t].z),
+                               h3 = to_16<kBf16>(fb[t].w);
+                if (g.transB) {   // four k of one column
+                    Bs[k][r] = (uint16_t)h0;
+                    Bs[k + 1][r] = (uint16_t)h1;
+                    Bs[k + 2][r] = (uint16_t)h2;
+                    Bs[k + 3][r] = (uint16_t)h3;
+                } else {          // four columns of one k
+                    *reinterpret_cast<uint2*>(&Bs[k][r]) = make_uint2(h0 | (h1 << 16), h2 | (h3 << 16));
+                }
             }
             __syncthreads();
             if (k0 + kFmBK < g.K) {
-                fetch_slice<kHfBM>(fa, g.A, g.lda, !g.transA, m0, g.M, k0 + kFmBK, g.K);
-                fetch_slice<kHfBN>(fb, g.B, g.ldb, g.transB, n0, g.N, k0 + kFmBK, g.K);
+                fetch_slice<kHfBM>(fa, g.A, g.lda, !g.transA, g.vec_a, m0, g.M, k0 + kFmBK, g.K);
+                fetch_slice<kHfBN>(fb, g.B, g.ldb, g.transB, g.vec_b, n0, g.N, k0 + kFmBK, g.K);
             }
             const int kmax = g.K - k0 < kFmBK ? g.K - k0 : kFmBK;
 #pragma unroll 1
@@ -406,6 +444,8 @@ int gemm_fmac8_device(const qfmt_matrix_t* A, const qfmt_matrix_t* B, float* d_C
     g.M = (int)M; g.N = (int)N; g.K = (int)K;
     g.transA = A->trans ? 1 : 0; g.transB = B->trans ? 1 : 0;
     g.vec_store = (ldc % 4 == 0) && !(reinterpret_cast<uintptr_t>(d_C) & 15u);
+    g.vec_a = (A->ld % 4 == 0) && !(reinterpret_cast<uintptr_t>(A->ptr) & 15u);
+    g.vec_b = (B->ld % 4 == 0) && !(reinterpret_cast<uintptr_t>(B->ptr) & 15u);
     const bool has_stats = d_stats != nullptr;
     const size_t smem = has_stats ? (size_t)(p.top + kExtraBins) * 32 * sizeof(uint32_t) : 0;
     const bool use_native = native && path != 1;
