@@ -395,6 +395,98 @@ def step5_section(torch, qf, dev, peaks, reps=5):
             "loss_scale": float(final.scale)}
 
 
+def config13_section(torch, qf, dev, peaks, reps=5):
+    """The two remaining workloads.  config1: the small reference case (A 256x512, B 512x256 rounded to
+    1/6/9 with statistics, C = A B), latency-bound: time per pass.  config3: the BERT-base FC layer in four
+    variants (1/6/9 and 1/5/10, denormals kept and flushed): X, W and dY (loss scale 2^10) rounded with
+    statistics, then forward, data-gradient and weight-gradient products."""
+    out = {}
+    c1 = workloads.config1()
+    e, m = c1["fmt"]
+    fmt = qf.make_format(e, m, c1["denormals"], c1["loss_scale"])
+    rA, rB = torch.from_numpy(c1["A"]).to(dev), torch.from_numpy(c1["B"]).to(dev)
+    qA, qB = torch.empty_like(rA), torch.empty_like(rB)
+    st = torch.zeros(2, qf.STATS_WORDS, dtype=torch.int64, device=dev)
+    C = torch.empty(256, 256, dtype=torch.float32, device=dev)
+    a, b = qf.make_matrix(qA), qf.make_matrix(qB)
+    ws = torch.zeros(max(256, qf.qfmt_gemm_workspace_bytes(a, b)), dtype=torch.uint8, device=dev)
+
+    def pass1():
+        qf.qfmt_quantize_stats(rA, qA, rA.numel(), fmt, st[0])
+        qf.qfmt_quantize_stats(rB, qB, rB.numel(), fmt, st[1])
+        qf.qfmt_gemm(a, b, C, 256, fmt, ws, ws.numel())
+    for _ in range(3):
+        pass1()
+    assert qf.qfmt_device_status(ws) == qf.QFMT_OK
+    ms = statistics.median(time_events(torch, pass1, 20))
+    # the same pass replayed from a CUDA graph: what remains once the host-side launch cost is gone
+    graph_ms = None
+    try:
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            pass1()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            pass1()
+        for _ in range(3):
+            graph.replay()
+        graph_ms = statistics.median(time_events(torch, graph.replay, 20))
+        torch.cuda.synchronize()
+    except Exception as exc:  # capture is an extra, not part of the path
+        graph_ms = None
+        out["config1_graph_error"] = str(exc)[:200]
+    out["config1"] = {"workload": "config1: round A 256x512 and B 512x256 to 1/6/9 with statistics, C = A B",
+                      "ms_per_pass": ms, "ms_per_pass_cuda_graph": graph_ms, "gpu_launches_per_pass": 3,
+                      "gemm_gflop": 2.0 * 256 * 256 * 512 / 1e9,
+                      "note": "latency-bound (three small launches): time only, no roofline fraction"}
+
+    c3 = workloads.config3()
+    raw = {k: torch.from_numpy(c3[k]).to(dev) for k in ("X", "W", "dY")}
+    q = {k: torch.empty_like(v) for k, v in raw.items()}
+    tokens, d_in = c3["X"].shape
+    d_out = c3["W"].shape[1]
+    Y = torch.empty(tokens, d_out, dtype=torch.float32, device=dev)
+    dX = torch.empty(tokens, d_in, dtype=torch.float32, device=dev)
+    dW = torch.empty(d_in, d_out, dtype=torch.float32, device=dev)
+    prods = ((qf.make_matrix(q["X"]), qf.make_matrix(q["W"]), Y, d_out),
+             (qf.make_matrix(q["dY"]), qf.make_matrix(q["W"], True), dX, d_in),
+             (qf.make_matrix(q["X"], True), qf.make_matrix(q["dY"]), dW, d_out))
+    wb = max([256] + [qf.qfmt_gemm_workspace_bytes(pa, pb) for pa, pb, _, _ in prods])
+    ws3 = torch.zeros(wb, dtype=torch.uint8, device=dev)
+    st3 = torch.zeros(3, qf.STATS_WORDS, dtype=torch.int64, device=dev)
+    variants = c3["variants"]
+
+    def rounding():
+        for (e_, m_), den in variants:
+            for i, (name, scale) in enumerate((("X", 1.0), ("W", 1.0), ("dY", c3["grad_scale"]))):
+                qf.qfmt_quantize_stats(raw[name], q[name], raw[name].numel(), qf.make_format(e_, m_, den, scale), st3[i])
+
+    def products():
+        for (e_, m_), den in variants:
+            f = qf.make_format(e_, m_, den)
+            for pa, pb, Cc, ldc in prods:
+                qf.qfmt_gemm(pa, pb, Cc, ldc, f, ws3, wb)
+    for _ in range(3):
+        rounding()
+        products()
+    assert qf.qfmt_device_status(ws3) == qf.QFMT_OK
+    r_ms = statistics.median(time_events(torch, rounding, reps))
+    p_ms = statistics.median(time_events(torch, products, reps))
+    r_bytes = len(variants) * BYTES_PER_ELEMENT * sum(v.numel() for v in raw.values())
+    flops = len(variants) * 3 * 2.0 * tokens * d_in * d_out
+    tf = flops / p_ms / 1e9
+    peak = peaks["bf16_tflops"] * (1.1 / 2.25)
+    out["config3"] = {"workload": f"config3 BERT-base FC layer ({tokens} x {d_in} x {d_out}), 4 variants: 12 rounding passes with "
+                                  "statistics, 12 products",
+                      "rounding_ms": r_ms, "rounding_gbs": r_bytes / r_ms / 1e6,
+                      "rounding_note": "tensors of 9-50 MB, smaller than L2: not an HBM figure",
+                      "products_ms": p_ms, "gemm_tflops": tf, "gpu_launches_per_step": 24,
+                      "roofline": {"bound": "tensor", "achieved": tf, "peak": peak, "unit": "TFLOP/s", "frac": tf / peak,
+                                   "traffic": None}}
+    return out
+
+
 def pack16_section(torch, qf, dev, peaks, d_in, n, reps=20):
     """16-bit storage on the config2 tensor: the rounding pass writing packed codes (4 B read + 2 B
     written per element) and the expansion back to fp32 containers (2 B read + 4 B written)."""
@@ -551,6 +643,8 @@ def run_library(args):
     extra = {}
     if "epilogue" in sections:
         extra["epilogue"] = epilogue_section(torch, qf, dev, peaks)
+    if "config13" in sections:
+        extra.update(config13_section(torch, qf, dev, peaks))
     if "step5" in sections:
         extra["step5"] = step5_section(torch, qf, dev, peaks)
     if "pack16" in sections:
@@ -621,9 +715,9 @@ def main():
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="library", choices=["library", "reference"])
-    ap.add_argument("--sections", default="quantize,e2e,gemm,conv,epilogue,step5,pack16,fmac8,cpu",
+    ap.add_argument("--sections", default="quantize,e2e,gemm,conv,config13,epilogue,step5,pack16,fmac8,cpu",
                     help="comma list of what to measure besides the timed sweep (quantize is always timed): "
-                         "e2e, gemm, conv, epilogue, step5, pack16, fmac8, cpu; profiling captures use a subset")
+                         "e2e, gemm, conv, config13, epilogue, step5, pack16, fmac8, cpu; profiling captures use a subset")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
