@@ -1052,23 +1052,59 @@ int make_map_c(CUtensorMap* map, float* base, uint64_t n, uint64_t rows, uint64_
     return make_map(map, base, 3, dims, strides, box, false);
 }
 
-// Sums the split-K partials [splits][rows][cols] (dense) into C in a fixed pairwise order.
+// Sums the split-K partials [splits][rows][cols] (dense) into C in a fixed pairwise order: adjacent
+// pairs level by level, an odd one out joining the next level as it is.  The tree is taken over
+// kMax (a power of two >= splits) register slots with the absent ones holding -0, the value that
+// changes no sum, so that every slot index is a compile-time constant.  T is float4 when rows can
+// be moved 16 bytes at a time (cols then counts groups of four), else float.
+__device__ __forceinline__ float tree_add(float a, float b) { return __fadd_rn(a, b); }
+__device__ __forceinline__ float4 tree_add(float4 a, float4 b) {
+    return make_float4(__fadd_rn(a.x, b.x), __fadd_rn(a.y, b.y), __fadd_rn(a.z, b.z), __fadd_rn(a.w, b.w));
+}
+__device__ __forceinline__ void tree_identity(float& v) { v = -0.0f; }
+__device__ __forceinline__ void tree_identity(float4& v) { v = make_float4(-0.0f, -0.0f, -0.0f, -0.0f); }
+template <typename T, int kMax>
 __global__ void __launch_bounds__(256)
-splitk_reduce_kernel(const float* __restrict__ part, float* __restrict__ C, long long rows, long long cols,
+splitk_reduce_kernel(const T* __restrict__ part, T* __restrict__ C, long long rows, long long cols,
                      long long ldc, int splits) {
     const long long total = rows * cols;
     for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total;
          i += (long long)gridDim.x * blockDim.x) {
-        float v[32];
-        for (int s = 0; s < splits; ++s) v[s] = part[(long long)s * total + i];
-        int n = splits;
-        while (n > 1) {  // pairwise tree, the same order on every run
-            const int h = n / 2;
-            for (int s = 0; s < h; ++s) v[s] = __fadd_rn(v[2 * s], v[2 * s + 1]);
-            if (n & 1) { v[h] = v[n - 1]; n = h + 1; } else { n = h; }
+        T v[kMax];
+#pragma unroll
+        for (int s = 0; s < kMax; ++s) {
+            if (s < splits) v[s] = part[(long long)s * total + i];
+            else tree_identity(v[s]);
+        }
+#pragma unroll
+        for (int n = kMax; n > 1; n /= 2) {
+#pragma unroll
+            for (int s = 0; s < n / 2; ++s) v[s] = tree_add(v[2 * s], v[2 * s + 1]);
         }
         C[(i / cols) * ldc + (i % cols)] = v[0];
     }
+}
+template <typename T>
+void launch_splitk_reduce_as(const float* part, float* C, long long rows, long long cols, long long ldc, int splits,
+                             int sm_count, cudaStream_t stream) {
+    const long long total = rows * cols, want = (total + 255) / 256, cap = (long long)sm_count * 16;
+    const int blocks = (int)(want < cap ? want : cap);
+    const T* p = reinterpret_cast<const T*>(part);
+    T* c = reinterpret_cast<T*>(C);
+    if (splits <= 2) splitk_reduce_kernel<T, 2><<<blocks, 256, 0, stream>>>(p, c, rows, cols, ldc, splits);
+    else if (splits <= 4) splitk_reduce_kernel<T, 4><<<blocks, 256, 0, stream>>>(p, c, rows, cols, ldc, splits);
+    else if (splits <= 8) splitk_reduce_kernel<T, 8><<<blocks, 256, 0, stream>>>(p, c, rows, cols, ldc, splits);
+    else if (splits <= 16) splitk_reduce_kernel<T, 16><<<blocks, 256, 0, stream>>>(p, c, rows, cols, ldc, splits);
+    else splitk_reduce_kernel<T, 32><<<blocks, 256, 0, stream>>>(p, c, rows, cols, ldc, splits);
+}
+// splits <= 32 (kMaxSplits).  The partials are dense, so groups of four stay inside a row when cols % 4 == 0.
+void launch_splitk_reduce(const float* part, float* C, long long rows, long long cols, long long ldc, int splits,
+                          int sm_count, cudaStream_t stream) {
+    if (rows <= 0 || cols <= 0) return;
+    const bool vec = cols % 4 == 0 && ldc % 4 == 0 && (reinterpret_cast<uintptr_t>(part) & 15) == 0 &&
+                     (reinterpret_cast<uintptr_t>(C) & 15) == 0;
+    if (vec) launch_splitk_reduce_as<float4>(part, C, rows, cols / 4, ldc / 4, splits, sm_count, stream);
+    else launch_splitk_reduce_as<float>(part, C, rows, cols, ldc, splits, sm_count, stream);
 }
 
 constexpr size_t kWorkspaceHeader = 256;  // status word and padding ahead of the partial sums
@@ -1325,9 +1361,7 @@ int gemm_device(const qfmt_matrix_t* A, const qfmt_matrix_t* B, float* d_C, int6
     }
     if (rc != QFMT_OK) return rc;
     if (p.splits > 1) {
-        const long long total = (long long)M * N;
-        const long long want = (total + 255) / 256, cap = (long long)dev.sm_count * 8;
-        splitk_reduce_kernel<<<(int)(want < cap ? want : cap), 256, 0, stream>>>(partials, d_C, M, N, ldc, p.splits);
+        launch_splitk_reduce(partials, d_C, M, N, ldc, p.splits, dev.sm_count, stream);
         QFMT_CUDA_TRY(cudaGetLastError());
     }
     return QFMT_OK;
@@ -1607,9 +1641,7 @@ int conv_device(int op, const qfmt_conv_t* g, const float* d_p, const float* d_q
     rc = launch_gemm(ma, mb, mc, mc, rows, p, dev, stream);
     if (rc != QFMT_OK) return rc;
     if (p.splits > 1) {
-        const long long total = (long long)p.M * p.N;
-        const int blocks = (int)((total + 255) / 256 < (long long)dev.sm_count * 8 ? (total + 255) / 256 : dev.sm_count * 8);
-        splitk_reduce_kernel<<<blocks, 256, 0, stream>>>(partials, d_out, p.M, p.N, p.N, p.splits);
+        launch_splitk_reduce(partials, d_out, p.M, p.N, p.N, p.splits, dev.sm_count, stream);
         QFMT_CUDA_TRY(cudaGetLastError());
     }
     return QFMT_OK;
