@@ -713,12 +713,17 @@ constexpr uint32_t kPBBytes = (kBN / 2) * kBK * 4;    // 128 of the tile's 256 c
 constexpr uint32_t kPStageBytes = kPABytes + kPBBytes;
 constexpr uint32_t kPairSmemBytes = kPStages * kPStageBytes + kOutBytes + 1024 + 256 + kEpiHistBytes;
 
-__device__ __forceinline__ uint32_t make_idesc_pair(int a_mn, int b_mn) {
-    return (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)a_mn << 15) | ((uint32_t)b_mn << 16)
+// Operand kinds of the pair kernel: fp32 containers read as TF32, or packed 16-bit codes that are
+// binary16 (1/5/10) or bfloat16 (1/8/7) words.  A stage is one 128-byte swizzle row per operand row
+// in every kind: 32 TF32 or 64 16-bit K elements, four MMAs.
+enum : int { kKindTf32 = 0, kKindF16 = 1, kKindBf16 = 2 };
+__device__ __forceinline__ uint32_t make_idesc_pair(int a_mn, int b_mn, int kind) {
+    const uint32_t ab = kind == kKindTf32 ? 2u : (kind == kKindF16 ? 0u : 1u);  // A, B format field
+    return (1u << 4) | (ab << 7) | (ab << 10) | ((uint32_t)a_mn << 15) | ((uint32_t)b_mn << 16)
            | ((uint32_t)(kBN >> 3) << 17) | ((uint32_t)((2 * kBM) >> 4) << 24);
 }
 
-template <bool kEpi>
+template <bool kEpi, int kKind>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 gemm_tf32_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                       const __grid_constant__ CUtensorMap tmap_c, const GemmParams p) {
@@ -788,7 +793,7 @@ gemm_tf32_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
                     const uint32_t sa = tiles + stage * kPStageBytes;
                     const uint32_t sb = sa + kPABytes;
                     const uint32_t bar = ptx::map_to_cta(full_bar(stage), 0);  // the leader's barrier
-                    const int k0 = kb * kBK;
+                    const int k0 = kb * (kKind == kKindTf32 ? kBK : 2 * kBK);
                     ptx::mbar_expect_tx_cluster(bar, kPStageBytes);
                     if (p.a_blocked) {
                         ptx::tma_load_3d_pair(sa, &tmap_a, bar, 0, k0, m0 >> 5);
@@ -819,7 +824,7 @@ gemm_tf32_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
         // phase of the stages of chunk c+1 belongs to chunks c-2 and c-1.
         if (lane == 0 && rank == 0) {
             const uint32_t who = (uint32_t)(warp - 1);
-            const uint32_t idesc = make_idesc_pair(p.a_mn_major, p.b_mn_major);
+            const uint32_t idesc = make_idesc_pair(p.a_mn_major, p.b_mn_major, kKind);
             // per-MMA advance of the descriptor start address, in 16-byte units
             const uint32_t a_step16 = (p.a_mn_major ? 1024u : (uint32_t)kMmaK * 4u) >> 4;
             const uint32_t b_step16 = (p.b_mn_major ? 1024u : (uint32_t)kMmaK * 4u) >> 4;
@@ -859,9 +864,12 @@ gemm_tf32_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
                         ptx::tc_fence_after_sync();
                         const uint32_t off = (uint32_t)stage * (kPStageBytes >> 4);
 #pragma unroll
-                        for (int k = 0; k < kBK / kMmaK; ++k)
-                            ptx::mma_tf32_pair(d_tmem, desc_join(a_hi, a_lo0 + off + k * a_step16), desc_join(b_hi, b_lo0 + off + k * b_step16),
-                                          idesc, (kb != kb0 || k != 0) ? 1u : 0u);
+                        for (int k = 0; k < kBK / kMmaK; ++k) {
+                            const uint64_t da = desc_join(a_hi, a_lo0 + off + k * a_step16);
+                            const uint64_t db = desc_join(b_hi, b_lo0 + off + k * b_step16);
+                            if (kKind == kKindTf32) ptx::mma_tf32_pair(d_tmem, da, db, idesc, (kb != kb0 || k != 0) ? 1u : 0u);
+                            else ptx::mma_f16_pair(d_tmem, da, db, idesc, (kb != kb0 || k != 0) ? 1u : 0u);
+                        }
                         ptx::mma_commit_pair(empty_bar(stage), 3);  // both CTAs may refill this stage
                         if (++stage == kPStages) { stage = 0; phase ^= 1u; }
                     }
@@ -1045,6 +1053,19 @@ int make_map_2d(CUtensorMap* map, const float* base, uint64_t dim0, uint64_t dim
     return make_map(map, base, 2, dims, strides, box, mn_major);
 }
 
+// K-major matrix of packed 16-bit codes: dim0 = K (contiguous), boxes of 64 x box1 (128-byte rows).
+int make_map16_2d(CUtensorMap* map, const uint16_t* base, uint64_t k, uint64_t rows, uint64_t ld_elems, uint32_t box1) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (fn == nullptr) { set_last_cuda_error((int)cudaErrorSymbolNotFound); return QFMT_ERR_CUDA; }
+    cuuint64_t d[2] = {k, rows}, st[1] = {ld_elems * sizeof(uint16_t)};
+    cuuint32_t bx[2] = {2 * kBK, box1}, estr[2] = {1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT16, 2, const_cast<uint16_t*>(base), d, st, bx, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) { set_last_cuda_error(100000 + (int)r); return QFMT_ERR_CUDA; }
+    return QFMT_OK;
+}
+
 // C (or the split-K partials) as a rank-3 map: [z][rows][N] with 32 x 32 x 1 boxes.
 int make_map_c(CUtensorMap* map, float* base, uint64_t n, uint64_t rows, uint64_t zdim, uint64_t ld, uint64_t zstride) {
     const uint64_t dims[3] = {n, rows, zdim}, strides[2] = {ld, zstride};
@@ -1198,8 +1219,8 @@ struct DensePlan {
 // reduction pass over (splits + 1) x M x N floats at about 4 TB/s plus a launch.  The wave count
 // is taken for a 148-SM part whatever the device, so that the plan, and with it the summation
 // order, depends on the problem alone.
-DensePlan plan_dense(int64_t M, int64_t N, int64_t K) {
-    const int policy = g_tile_policy.load();
+DensePlan plan_dense(int64_t M, int64_t N, int64_t K, int policy_override = -1) {
+    const int policy = policy_override >= 0 ? policy_override : g_tile_policy.load();
     const int64_t kb_total = (K + kBK - 1) / kBK;
     DensePlan best = {policy == 2, 1};
     double best_cost = -1.0;
@@ -1228,19 +1249,26 @@ DensePlan plan_dense(int64_t M, int64_t N, int64_t K) {
 }
 
 int launch_pair(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc, const GemmParams& p,
-                const DeviceInfo& dev, cudaStream_t stream) {
+                const DeviceInfo& dev, cudaStream_t stream, int kind = kKindTf32) {
     static bool attr_set[64] = {};
     if (dev.ordinal < 0 || dev.ordinal >= 64 || !attr_set[dev.ordinal]) {
-        QFMT_CUDA_TRY(cudaFuncSetAttribute(gemm_tf32_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                           (int)kPairSmemBytes));
-        QFMT_CUDA_TRY(cudaFuncSetAttribute(gemm_tf32_pair_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                           (int)kPairSmemBytes));
+        QFMT_CUDA_TRY(cudaFuncSetAttribute(gemm_tf32_pair_kernel<false, kKindTf32>,
+                                           cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPairSmemBytes));
+        QFMT_CUDA_TRY(cudaFuncSetAttribute(gemm_tf32_pair_kernel<true, kKindTf32>,
+                                           cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPairSmemBytes));
+        QFMT_CUDA_TRY(cudaFuncSetAttribute(gemm_tf32_pair_kernel<false, kKindF16>,
+                                           cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPairSmemBytes));
+        QFMT_CUDA_TRY(cudaFuncSetAttribute(gemm_tf32_pair_kernel<false, kKindBf16>,
+                                           cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPairSmemBytes));
         if (dev.ordinal >= 0 && dev.ordinal < 64) attr_set[dev.ordinal] = true;
     }
     const long long work = (long long)p.tiles_m * p.tiles_n * p.splits;
     const long long clusters = work < dev.sm_count / 2 ? work : dev.sm_count / 2;
-    if (p.epi) gemm_tf32_pair_kernel<true><<<(unsigned)(2 * clusters), kThreads, kPairSmemBytes, stream>>>(ma, mb, mc, p);
-    else gemm_tf32_pair_kernel<false><<<(unsigned)(2 * clusters), kThreads, kPairSmemBytes, stream>>>(ma, mb, mc, p);
+    const unsigned grid = (unsigned)(2 * clusters);
+    if (kind == kKindF16) gemm_tf32_pair_kernel<false, kKindF16><<<grid, kThreads, kPairSmemBytes, stream>>>(ma, mb, mc, p);
+    else if (kind == kKindBf16) gemm_tf32_pair_kernel<false, kKindBf16><<<grid, kThreads, kPairSmemBytes, stream>>>(ma, mb, mc, p);
+    else if (p.epi) gemm_tf32_pair_kernel<true, kKindTf32><<<grid, kThreads, kPairSmemBytes, stream>>>(ma, mb, mc, p);
+    else gemm_tf32_pair_kernel<false, kKindTf32><<<grid, kThreads, kPairSmemBytes, stream>>>(ma, mb, mc, p);
     QFMT_CUDA_TRY(cudaGetLastError());
     return QFMT_OK;
 }
@@ -1359,6 +1387,77 @@ int gemm_device(const qfmt_matrix_t* A, const qfmt_matrix_t* B, float* d_C, int6
         for (int i = 0; i < kMaxRowMaps; ++i) rows.m[i] = ma;  // unused in dense mode
         rc = launch_gemm(ma, mb, mc, mc, rows, p, dev, stream);
     }
+    if (rc != QFMT_OK) return rc;
+    if (p.splits > 1) {
+        launch_splitk_reduce(partials, d_C, M, N, ldc, p.splits, dev.sm_count, stream);
+        QFMT_CUDA_TRY(cudaGetLastError());
+    }
+    return QFMT_OK;
+}
+
+// C = A B^T on packed 16-bit codes of 1/5/10 (binary16 words) or 1/8/7 (bfloat16 words): the pair
+// kernel with kind::f16 MMAs.  A is M x K and B is N x K, both with K contiguous, so a stage is 64
+// K elements per 128-byte row and a TMEM chunk 128 (eight MMAs, as for TF32); the plan is the one
+// of a TF32 product of half the length, which costs the same number of MMAs.
+int gemm16_device(const uint16_t* d_A, int64_t lda, const uint16_t* d_B, int64_t ldb, int64_t M, int64_t N, int64_t K,
+                  float* d_C, int64_t ldc, const qfmt_format_t* fmt, void* d_workspace, size_t workspace_bytes,
+                  cudaStream_t stream) {
+    int rc = validate_format(fmt);
+    if (rc != QFMT_OK) return rc;
+    const bool f16 = fmt->e == 5 && fmt->m == 10, bf16 = fmt->e == 8 && fmt->m == 7;
+    if (!f16 && !bf16) return QFMT_ERR_BAD_FORMAT;
+    if (M < 0 || N < 0 || K < 0 || M > (1 << 30) || N > (1 << 30) || K > (1 << 30)) return QFMT_ERR_BAD_ARG;
+    if (lda < K || ldb < K || ldc < N) return QFMT_ERR_BAD_ARG;
+    if (d_workspace == nullptr || workspace_bytes < 16 || (reinterpret_cast<uintptr_t>(d_workspace) & 15u))
+        return QFMT_ERR_BAD_ARG;
+    if (M == 0 || N == 0) return QFMT_OK;
+    if ((d_A == nullptr || d_B == nullptr) && K != 0) return QFMT_ERR_BAD_ARG;
+    if (d_C == nullptr || (reinterpret_cast<uintptr_t>(d_C) & 3u)) return QFMT_ERR_BAD_ARG;
+    if ((reinterpret_cast<uintptr_t>(d_A) & 15u) || (reinterpret_cast<uintptr_t>(d_B) & 15u) || (lda & 7) || (ldb & 7))
+        return QFMT_ERR_BAD_ARG;  // TMA: 16-byte aligned bases and row pitches
+    DeviceInfo dev;
+    rc = current_device(&dev);
+    if (rc != QFMT_OK) return rc;
+    int* status = reinterpret_cast<int*>(d_workspace);
+    QFMT_CUDA_TRY(cudaMemsetAsync(status, 0, 16, stream));
+    if (K == 0) {
+        QFMT_CUDA_TRY(cudaMemset2DAsync(d_C, (size_t)ldc * sizeof(float), 0, (size_t)N * sizeof(float), (size_t)M, stream));
+        return QFMT_OK;
+    }
+    GemmParams p;
+    dense_defaults(&p);
+    p.M = (int)M; p.N = (int)N; p.K = (int)K;
+    p.ldc = ldc;
+    p.C = d_C;
+    p.status = status;
+    p.a_mn_major = p.b_mn_major = 0;
+    p.tile_rows = 2 * kBM;
+    p.tiles_m = (int)((M + p.tile_rows - 1) / p.tile_rows);
+    p.tiles_n = (int)((N + kBN - 1) / kBN);
+    p.kb_total = (int)((K + 2 * kBK - 1) / (2 * kBK));
+    p.kb_per_split = p.kb_total;
+    p.tma_store = ((reinterpret_cast<uintptr_t>(d_C) & 15u) == 0 && (ldc & 3) == 0 && (N & 3) == 0) ? 1 : 0;
+    int splits = plan_dense(M, N, (K + 1) / 2, 2).splits;
+    while (splits > 1 && kWorkspaceHeader + (size_t)splits * (size_t)M * (size_t)N * sizeof(float) > workspace_bytes) --splits;
+    float* partials = reinterpret_cast<float*>(reinterpret_cast<char*>(d_workspace) + kWorkspaceHeader);
+    if (splits > 1) {
+        p.kb_per_split = (p.kb_total + splits - 1) / splits;
+        p.splits = (p.kb_total + p.kb_per_split - 1) / p.kb_per_split;
+        p.split_stride = (long long)M * N;
+        p.C = partials;
+        p.ldc = N;
+        p.tma_store = (N & 3) == 0 ? 1 : 0;
+    }
+    CUtensorMap ma, mb, mc;
+    rc = make_map16_2d(&ma, d_A, (uint64_t)K, (uint64_t)M, (uint64_t)lda, kBM);
+    if (rc != QFMT_OK) return rc;
+    rc = make_map16_2d(&mb, d_B, (uint64_t)K, (uint64_t)N, (uint64_t)ldb, kBN / 2);
+    if (rc != QFMT_OK) return rc;
+    if (p.tma_store)
+        rc = make_map_c(&mc, p.C, (uint64_t)N, (uint64_t)M, (uint64_t)p.splits, (uint64_t)p.ldc, (uint64_t)M * (uint64_t)p.ldc);
+    else mc = ma;  // unused by the kernel
+    if (rc != QFMT_OK) return rc;
+    rc = launch_pair(ma, mb, mc, p, dev, stream, f16 ? kKindF16 : kKindBf16);
     if (rc != QFMT_OK) return rc;
     if (p.splits > 1) {
         launch_splitk_reduce(partials, d_C, M, N, ldc, p.splits, dev.sm_count, stream);
@@ -1654,6 +1753,13 @@ extern "C" int qfmt_gemm(const qfmt_matrix_t* A, const qfmt_matrix_t* B, float* 
     return qfmt::gemm_device(A, B, d_C, ldc, fmt, d_workspace, workspace_bytes, (cudaStream_t)stream);
 }
 
+extern "C" int qfmt_gemm_packed16(const uint16_t* d_A, int64_t lda, const uint16_t* d_B, int64_t ldb, int64_t M,
+                                  int64_t N, int64_t K, float* d_C, int64_t ldc, const qfmt_format_t* fmt,
+                                  void* d_workspace, size_t workspace_bytes, void* stream) {
+    return qfmt::gemm16_device(d_A, lda, d_B, ldb, M, N, K, d_C, ldc, fmt, d_workspace, workspace_bytes,
+                               (cudaStream_t)stream);
+}
+
 extern "C" int qfmt_conv(int32_t op, const qfmt_conv_t* geom, const float* d_p, const float* d_q, float* d_out,
                          const qfmt_format_t* fmt, void* d_workspace, size_t workspace_bytes, void* stream) {
     return qfmt::conv_device(op, geom, d_p, d_q, d_out, fmt, d_workspace, workspace_bytes, (cudaStream_t)stream);
@@ -1763,6 +1869,12 @@ extern "C" size_t qfmt_gemm_workspace_bytes(const qfmt_matrix_t* A, const qfmt_m
     const int64_t N = B->trans ? B->rows : B->cols;
     if (M <= 0 || N <= 0 || K <= 0 || M > (1 << 30) || N > (1 << 30) || K > (1 << 30)) return qfmt::kWorkspaceHeader;
     const int splits = qfmt::plan_dense(M, N, K).splits;
+    return qfmt::kWorkspaceHeader + (splits > 1 ? (size_t)splits * (size_t)M * (size_t)N * sizeof(float) : 0);
+}
+
+extern "C" size_t qfmt_gemm_packed16_workspace_bytes(int64_t M, int64_t N, int64_t K) {
+    if (M <= 0 || N <= 0 || K <= 0 || M > (1 << 30) || N > (1 << 30) || K > (1 << 30)) return qfmt::kWorkspaceHeader;
+    const int splits = qfmt::plan_dense(M, N, (K + 1) / 2, 2).splits;
     return qfmt::kWorkspaceHeader + (splits > 1 ? (size_t)splits * (size_t)M * (size_t)N * sizeof(float) : 0);
 }
 
