@@ -511,6 +511,53 @@ def pack16_section(torch, qf, dev, peaks, d_in, n, reps=20):
             "gpu_launches_per_step": 2, "roofline": res["pack"]["roofline"], "runs": res}
 
 
+def gemm16_section(torch, qf, dev, peaks, reps=5):
+    """The four forward products of the BERT-large FC stack on packed 16-bit operands (1/5/10 as
+    binary16 words, 1/8/7 as bfloat16 words): the rounding pass writes the codes of X [tokens, d_in]
+    and of the weight stored output-major [d_out, d_in]; qfmt_gemm_packed16 contracts them."""
+    out = {"metric": "emulated GEMM on packed 16-bit operands TFLOP/s", "unit": "TFLOP/s", "runs": {},
+           "workload": "config5 BERT-large FC stack, forward products of the 4 layers (8192 tokens), packed codes"}
+    for tag, e, m in (("1/5/10 binary16", 5, 10), ("1/8/7 bfloat16", 8, 7)):
+        fmt = qf.make_format(e, m, 1)
+        jobs, flops, ws_bytes, pack_ms = [], 0.0, 256, 0.0
+        for layer in range(len(workloads.CONFIG5_LAYERS)):
+            c = workloads.config5_layer(layer, step=0)
+            X = torch.from_numpy(c["X"]).to(dev)
+            Wt = torch.from_numpy(np.ascontiguousarray(c["W"].T)).to(dev)
+            cX = torch.empty(X.shape, dtype=torch.int16, device=dev)
+            cW = torch.empty(Wt.shape, dtype=torch.int16, device=dev)
+            st = torch.zeros(qf.STATS_WORDS, dtype=torch.int64, device=dev)
+
+            def pack():
+                qf.qfmt_quantize_stats_pack16(X, cX, X.numel(), fmt, st)
+                qf.qfmt_quantize_stats_pack16(Wt, cW, Wt.numel(), fmt, st)
+            pack()
+            pack_ms += statistics.median(time_events(torch, pack, 3))
+            M, K = X.shape
+            N = Wt.shape[0]
+            jobs.append((cX, cW, M, N, K, torch.empty(M, N, dtype=torch.float32, device=dev)))
+            ws_bytes = max(ws_bytes, qf.qfmt_gemm_packed16_workspace_bytes(M, N, K))
+            flops += 2.0 * M * N * K
+        ws = torch.zeros(ws_bytes, dtype=torch.uint8, device=dev)
+
+        def step():
+            for cX, cW, M, N, K, C in jobs:
+                qf.qfmt_gemm_packed16(cX, K, cW, K, M, N, K, C, N, fmt, ws, ws.numel())
+        for _ in range(3):
+            step()
+        assert qf.qfmt_device_status(ws) == qf.QFMT_OK
+        ms = statistics.median(time_events(torch, step, reps))
+        tf = flops / ms / 1e9
+        out["runs"][tag] = {"ms_per_step": ms, "tflops": tf, "rounding_to_codes_ms": pack_ms, "gpu_launches_per_step": len(jobs),
+                            "roofline": {"bound": "tensor", "achieved": tf, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                                         "frac": tf / peaks["bf16_tflops"], "traffic": None,
+                                         "peak_source": f"bf16 {peaks['source']} burst"}}
+        del jobs, ws
+    first = out["runs"]["1/5/10 binary16"]
+    out.update({"value": first["tflops"], "ms_per_step": first["ms_per_step"], "roofline": first["roofline"]})
+    return out
+
+
 # FMAC-8 is plain-ALU work.  Peak = SMs x 4 schedulers x 32 lanes x max SM clock / (scheduler cycles one
 # warp-wide multiply-add must cost).  General kernel: per FMAC FMAC8_FLOAT_OPS float-pipe instructions (two
 # directed fused multiply-adds, add and subtract of the rounding constant)
@@ -649,6 +696,8 @@ def run_library(args):
         extra["step5"] = step5_section(torch, qf, dev, peaks)
     if "pack16" in sections:
         extra["pack16"] = pack16_section(torch, qf, dev, peaks, d_in, n)
+    if "gemm16" in sections:
+        extra["gemm16"] = gemm16_section(torch, qf, dev, peaks)
     if "fmac8" in sections:
         extra["fmac8"] = fmac8_section(torch, qf, dev, peaks, clocks.summary()["sm_max_mhz"] or 1965)
     if "e2e" in sections:
@@ -715,7 +764,7 @@ def main():
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="library", choices=["library", "reference"])
-    ap.add_argument("--sections", default="quantize,e2e,gemm,conv,config13,epilogue,step5,pack16,fmac8,cpu",
+    ap.add_argument("--sections", default="quantize,e2e,gemm,conv,config13,epilogue,step5,pack16,gemm16,fmac8,cpu",
                     help="comma list of what to measure besides the timed sweep (quantize is always timed): "
                          "e2e, gemm, conv, config13, epilogue, step5, pack16, fmac8, cpu; profiling captures use a subset")
     args = ap.parse_args()
