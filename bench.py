@@ -535,14 +535,15 @@ def gemm16_section(torch, qf, dev, peaks, reps=5):
             pack_ms += statistics.median(time_events(torch, pack, 3))
             M, K = X.shape
             N = Wt.shape[0]
-            jobs.append((cX, cW, M, N, K, torch.empty(M, N, dtype=torch.float32, device=dev)))
-            ws_bytes = max(ws_bytes, qf.qfmt_gemm_packed16_workspace_bytes(M, N, K))
+            jobs.append((qf.make_matrix(cX), qf.make_matrix(cW, True), N, torch.empty(M, N, dtype=torch.float32, device=dev),
+                         (cX, cW)))
+            ws_bytes = max(ws_bytes, qf.qfmt_gemm_packed16_workspace_bytes(jobs[-1][0], jobs[-1][1]))
             flops += 2.0 * M * N * K
         ws = torch.zeros(ws_bytes, dtype=torch.uint8, device=dev)
 
         def step():
-            for cX, cW, M, N, K, C in jobs:
-                qf.qfmt_gemm_packed16(cX, K, cW, K, M, N, K, C, N, fmt, ws, ws.numel())
+            for a, b, N, C, _ in jobs:
+                qf.qfmt_gemm_packed16(a, b, C, N, fmt, ws, ws.numel())
         for _ in range(3):
             step()
         assert qf.qfmt_device_status(ws) == qf.QFMT_OK

@@ -318,31 +318,37 @@ int qfmt_gemm_fmac8(const qfmt_matrix_t* A, const qfmt_matrix_t* B, float* d_C, 
                     const qfmt_format_t* fmt, qfmt_stats_t* d_stats, int accumulate, int path, void* stream);
 
 /*
- * C = A B^T on operands stored as packed 16-bit codes (the output of qfmt_quantize_stats_pack16),
- * for the two formats whose codes are words the tensor cores read directly: 1/5/10 (IEEE binary16)
- * and 1/8/7 (bfloat16).  The same FMACS contraction as qfmt_gemm (Section III-B: exact products,
- * fp32 accumulation), run as tcgen05 kind::f16 at twice the TF32 rate and with half the operand
- * traffic; the summation is taken in the same three levels with chunks of 128 K elements, and
- * results stay within 2^-20 * sum_k |a_ik| |b_jk| of the exact sum for the workloads this library
- * targets.  Denormal codes are honoured; inf and NaN codes propagate as in IEEE arithmetic.
+ * One operand of qfmt_gemm_packed16: a row-major matrix of packed 16-bit codes (the output of
+ * qfmt_quantize_stats_pack16) in device memory; rows, cols, ld and trans as in qfmt_matrix_t.
+ * ptr must be 16-byte aligned and ld a multiple of 8 (the tiles are fetched by TMA).
+ */
+typedef struct {
+    const uint16_t* ptr;
+    int64_t rows, cols, ld;
+    int32_t trans;
+} qfmt_matrix16_t;
+
+/*
+ * C = op(A) op(B) on operands stored as packed 16-bit codes, for the two formats whose codes are
+ * words the tensor cores read directly: 1/5/10 (IEEE binary16) and 1/8/7 (bfloat16).  The same
+ * FMACS contraction as qfmt_gemm (Section III-B: exact products, fp32 accumulation) with the same
+ * operand conventions (the three products of a layer need no copies), run as tcgen05 kind::f16 at
+ * twice the TF32 rate and with half the operand traffic; the summation is taken in the same three
+ * levels with chunks of 128 K elements, and results stay within 2^-20 * sum_k |a_ik| |b_kj| of the
+ * exact sum for the workloads this library targets.  Denormal codes are honoured; inf and NaN
+ * codes propagate as in IEEE arithmetic.
  *
- *   d_A   device, M x K codes, row-major with leading dimension lda >= K (elements)
- *   d_B   device, N x K codes, row-major with leading dimension ldb >= K: a fully connected layer's
- *         weight stored output-major, or the transposed copy of any other operand (both operands
- *         have K contiguous; other layouts are not offered)
- *         d_A, d_B 16-byte aligned, lda and ldb multiples of 8 (the tiles are fetched by TMA)
  *   d_C   device, M x N floats, leading dimension ldc >= N, 4-byte aligned
  *   fmt   {5, 10} or {8, 7}, QFMT_ERR_BAD_FORMAT otherwise (1/6/9 codes fit neither word: expand
  *         them with qfmt_unpack16 and use qfmt_gemm); denormals and loss_scale are ignored
- *   d_workspace, workspace_bytes   as for qfmt_gemm; qfmt_gemm_packed16_workspace_bytes(M, N, K)
- *         is the size that allows split K.  Status word and timeouts as for qfmt_gemm.
+ *   d_workspace, workspace_bytes   as for qfmt_gemm; qfmt_gemm_packed16_workspace_bytes(A, B) is
+ *         the size that allows split K.  Status word and timeouts as for qfmt_gemm.
  * M = 0 or N = 0 is a no-op; K = 0 writes zeros.
  * Errors: QFMT_ERR_BAD_FORMAT, QFMT_ERR_BAD_ARG, QFMT_ERR_UNSUPPORTED_ARCH, QFMT_ERR_CUDA.
  */
-int qfmt_gemm_packed16(const uint16_t* d_A, int64_t lda, const uint16_t* d_B, int64_t ldb, int64_t M, int64_t N,
-                       int64_t K, float* d_C, int64_t ldc, const qfmt_format_t* fmt, void* d_workspace,
-                       size_t workspace_bytes, void* stream);
-size_t qfmt_gemm_packed16_workspace_bytes(int64_t M, int64_t N, int64_t K);
+int qfmt_gemm_packed16(const qfmt_matrix16_t* A, const qfmt_matrix16_t* B, float* d_C, int64_t ldc,
+                       const qfmt_format_t* fmt, void* d_workspace, size_t workspace_bytes, void* stream);
+size_t qfmt_gemm_packed16_workspace_bytes(const qfmt_matrix16_t* A, const qfmt_matrix16_t* B);
 
 /*
  * Tuning and test control (no counterpart in the paper): which kernel dense products run on.

@@ -114,9 +114,9 @@ def _bind_optional(L: ctypes.CDLL) -> None:
     L.qfmt_gemm_workspace_bytes.argtypes = [matp, matp]
     L.qfmt_gemm_workspace_bytes.restype = sz
     i64 = ctypes.c_int64
-    L.qfmt_gemm_packed16.argtypes = [vp, i64, vp, i64, i64, i64, i64, vp, i64, ctypes.POINTER(qfmt_format_t), vp, sz, vp]
+    L.qfmt_gemm_packed16.argtypes = [matp, matp, vp, i64, ctypes.POINTER(qfmt_format_t), vp, sz, vp]
     L.qfmt_gemm_packed16.restype = ci
-    L.qfmt_gemm_packed16_workspace_bytes.argtypes = [i64, i64, i64]
+    L.qfmt_gemm_packed16_workspace_bytes.argtypes = [matp, matp]
     L.qfmt_gemm_packed16_workspace_bytes.restype = sz
     L.qfmt_gemm_fmac8.argtypes = [matp, matp, vp, ctypes.c_int64, ctypes.POINTER(qfmt_format_t), vp, ci, ci, vp]
     L.qfmt_gemm_fmac8.restype = ci
@@ -250,16 +250,19 @@ def qfmt_gemm(A: qfmt_matrix_t, B: qfmt_matrix_t, d_C, ldc: int, fmt: qfmt_forma
                            _ptr(d_workspace), int(workspace_bytes), _stream_handle(stream)), "qfmt_gemm")
 
 
-def qfmt_gemm_packed16_workspace_bytes(M: int, N: int, K: int) -> int:
-    return int(lib().qfmt_gemm_packed16_workspace_bytes(int(M), int(N), int(K)))
+qfmt_matrix16_t = qfmt_matrix_t  # the same record with a pointer to 16-bit codes; make_matrix builds both
 
 
-def qfmt_gemm_packed16(d_A, lda: int, d_B, ldb: int, M: int, N: int, K: int, d_C, ldc: int, fmt: qfmt_format_t,
-                       d_workspace, workspace_bytes: int, stream=None) -> None:
-    """C = A B^T on packed binary16 / bfloat16 codes; see qfmt_gemm_packed16 in include/qfmt.h."""
-    _check(lib().qfmt_gemm_packed16(_ptr(d_A), int(lda), _ptr(d_B), int(ldb), int(M), int(N), int(K), _ptr(d_C),
-                                    int(ldc), ctypes.byref(fmt), _ptr(d_workspace), int(workspace_bytes),
-                                    _stream_handle(stream)), "qfmt_gemm_packed16")
+def qfmt_gemm_packed16_workspace_bytes(A: qfmt_matrix_t, B: qfmt_matrix_t) -> int:
+    return int(lib().qfmt_gemm_packed16_workspace_bytes(ctypes.byref(A), ctypes.byref(B)))
+
+
+def qfmt_gemm_packed16(A: qfmt_matrix_t, B: qfmt_matrix_t, d_C, ldc: int, fmt: qfmt_format_t, d_workspace,
+                       workspace_bytes: int, stream=None) -> None:
+    """C = op(A) op(B) on packed binary16 / bfloat16 codes; see qfmt_gemm_packed16 in include/qfmt.h."""
+    _check(lib().qfmt_gemm_packed16(ctypes.byref(A), ctypes.byref(B), _ptr(d_C), int(ldc), ctypes.byref(fmt),
+                                    _ptr(d_workspace), int(workspace_bytes), _stream_handle(stream)),
+           "qfmt_gemm_packed16")
 
 
 def qfmt_gemm_fmac8(A: qfmt_matrix_t, B: qfmt_matrix_t, d_C, ldc: int, fmt: qfmt_format_t, d_stats=None,

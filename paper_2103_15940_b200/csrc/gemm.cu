@@ -795,19 +795,23 @@ gemm_tf32_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
                     const uint32_t bar = ptx::map_to_cta(full_bar(stage), 0);  // the leader's barrier
                     const int k0 = kb * (kKind == kKindTf32 ? kBK : 2 * kBK);
                     ptx::mbar_expect_tx_cluster(bar, kPStageBytes);
+                    // an MN-major operand arrives as column blocks of one 128-byte row per K element:
+                    // 32 columns x 32 K rows (TF32) or 64 columns x 64 K rows (16-bit codes)
+                    constexpr int kBlkShift = kKind == kKindTf32 ? 5 : 6, kBlk = 1 << kBlkShift;
+                    constexpr uint32_t kBlkBytes = kKind == kKindTf32 ? 4096u : 8192u;
                     if (p.a_blocked) {
-                        ptx::tma_load_3d_pair(sa, &tmap_a, bar, 0, k0, m0 >> 5);
+                        ptx::tma_load_3d_pair(sa, &tmap_a, bar, 0, k0, m0 >> kBlkShift);
                     } else if (p.a_mn_major) {
-                        for (int c = 0; c < kBM / 32; ++c)
-                            ptx::tma_load_2d_pair(sa + c * 4096u, &tmap_a, bar, m0 + c * 32, k0);
+                        for (int c = 0; c < kBM / kBlk; ++c)
+                            ptx::tma_load_2d_pair(sa + c * kBlkBytes, &tmap_a, bar, m0 + c * kBlk, k0);
                     } else {
                         ptx::tma_load_2d_pair(sa, &tmap_a, bar, k0, m0);
                     }
                     if (p.b_blocked) {
-                        ptx::tma_load_3d_pair(sb, &tmap_b, bar, 0, k0, n0 >> 5);
+                        ptx::tma_load_3d_pair(sb, &tmap_b, bar, 0, k0, n0 >> kBlkShift);
                     } else if (p.b_mn_major) {
-                        for (int c = 0; c < kBN / 64; ++c)
-                            ptx::tma_load_2d_pair(sb + c * 4096u, &tmap_b, bar, n0 + c * 32, k0);
+                        for (int c = 0; c < (kBN / 2) / kBlk; ++c)
+                            ptx::tma_load_2d_pair(sb + c * kBlkBytes, &tmap_b, bar, n0 + c * kBlk, k0);
                     } else {
                         ptx::tma_load_2d_pair(sb, &tmap_b, bar, k0, n0);
                     }
@@ -826,12 +830,18 @@ gemm_tf32_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
             const uint32_t who = (uint32_t)(warp - 1);
             const uint32_t idesc = make_idesc_pair(p.a_mn_major, p.b_mn_major, kKind);
             // per-MMA advance of the descriptor start address, in 16-byte units
-            const uint32_t a_step16 = (p.a_mn_major ? 1024u : (uint32_t)kMmaK * 4u) >> 4;
-            const uint32_t b_step16 = (p.b_mn_major ? 1024u : (uint32_t)kMmaK * 4u) >> 4;
-            const uint32_t a_lbo = p.a_mn_major ? 4096u : 16u, a_sbo = p.a_mn_major ? 512u : 1024u;
-            const uint32_t b_lbo = p.b_mn_major ? 4096u : 16u, b_sbo = p.b_mn_major ? 512u : 1024u;
-            const uint32_t a_lay = p.a_mn_major ? kLayoutSw128Base32 : kLayoutSw128;
-            const uint32_t b_lay = p.b_mn_major ? kLayoutSw128Base32 : kLayoutSw128;
+            // MN-major operand: the leading offset is the pitch of its column blocks, the stride offset
+            // that of eight K rows, and one MMA consumes 8 (TF32) or 16 (16-bit) K rows of 128 bytes.
+            // TF32 needs the 32-byte-atom form of the 128-byte swizzle there, 16-bit codes the plain one.
+            constexpr bool k16 = kKind != kKindTf32;
+            constexpr uint32_t mn_step = k16 ? 2048u : 1024u, mn_lbo = k16 ? 8192u : 4096u, mn_sbo = k16 ? 1024u : 512u;
+            constexpr uint32_t mn_lay = k16 ? kLayoutSw128 : kLayoutSw128Base32;
+            const uint32_t a_step16 = (p.a_mn_major ? mn_step : (uint32_t)kMmaK * 4u) >> 4;
+            const uint32_t b_step16 = (p.b_mn_major ? mn_step : (uint32_t)kMmaK * 4u) >> 4;
+            const uint32_t a_lbo = p.a_mn_major ? mn_lbo : 16u, a_sbo = p.a_mn_major ? mn_sbo : 1024u;
+            const uint32_t b_lbo = p.b_mn_major ? mn_lbo : 16u, b_sbo = p.b_mn_major ? mn_sbo : 1024u;
+            const uint32_t a_lay = p.a_mn_major ? mn_lay : kLayoutSw128;
+            const uint32_t b_lay = p.b_mn_major ? mn_lay : kLayoutSw128;
             const uint32_t a_hi = desc_hi(a_sbo, a_lay), b_hi = desc_hi(b_sbo, b_lay);
             const uint32_t a_lo0 = desc_lo(tiles, a_lbo), b_lo0 = desc_lo(tiles + kPABytes, b_lbo);
             int stage = 0;
@@ -1053,17 +1063,42 @@ int make_map_2d(CUtensorMap* map, const float* base, uint64_t dim0, uint64_t dim
     return make_map(map, base, 2, dims, strides, box, mn_major);
 }
 
-// K-major matrix of packed 16-bit codes: dim0 = K (contiguous), boxes of 64 x box1 (128-byte rows).
-int make_map16_2d(CUtensorMap* map, const uint16_t* base, uint64_t k, uint64_t rows, uint64_t ld_elems, uint32_t box1) {
+// Map over packed 16-bit codes (plain 128-byte swizzle): rank 2 or 3, strides in elements.
+int make_map16(CUtensorMap* map, const uint16_t* base, int rank, const uint64_t* dims, const uint64_t* strides_elems,
+               const uint32_t* box) {
     EncodeTiledFn fn = encode_tiled_fn();
     if (fn == nullptr) { set_last_cuda_error((int)cudaErrorSymbolNotFound); return QFMT_ERR_CUDA; }
-    cuuint64_t d[2] = {k, rows}, st[1] = {ld_elems * sizeof(uint16_t)};
-    cuuint32_t bx[2] = {2 * kBK, box1}, estr[2] = {1, 1};
-    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT16, 2, const_cast<uint16_t*>(base), d, st, bx, estr,
+    cuuint64_t d[3], st[2];
+    cuuint32_t bx[3], estr[3] = {1, 1, 1};
+    for (int i = 0; i < rank; ++i) { d[i] = dims[i]; bx[i] = box[i]; }
+    for (int i = 0; i + 1 < rank; ++i) st[i] = strides_elems[i] * sizeof(uint16_t);
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT16, (cuuint32_t)rank, const_cast<uint16_t*>(base), d, st, bx, estr,
                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) { set_last_cuda_error(100000 + (int)r); return QFMT_ERR_CUDA; }
     return QFMT_OK;
+}
+// One operand of the packed contraction.  `extent` is its M (or N) size and `tile` the rows of it a
+// CTA stages (128).  K-major: {K, extent} with 64 x tile boxes.  MN-major: 64-wide column blocks of
+// 64 K rows; {64, K, extent / 64} with one box per stage when the extent is a multiple of 64
+// (*blocked = 1), else the plain {extent, K} map, one 64 x 64 box per block, zero-filled past the end.
+int make_operand_map16(CUtensorMap* map, const uint16_t* base, bool mn_major, uint64_t extent, uint64_t k, uint64_t ld,
+                       uint32_t tile, int* blocked) {
+    *blocked = 0;
+    if (!mn_major) {
+        const uint64_t dims[2] = {k, extent}, strides[1] = {ld};
+        const uint32_t box[2] = {2 * kBK, tile};
+        return make_map16(map, base, 2, dims, strides, box);
+    }
+    if (extent % 64 == 0) {
+        *blocked = 1;
+        const uint64_t dims[3] = {64, k, extent / 64}, strides[2] = {ld, 64};
+        const uint32_t box[3] = {64, 2 * kBK, tile / 64};
+        return make_map16(map, base, 3, dims, strides, box);
+    }
+    const uint64_t dims[2] = {extent, k}, strides[1] = {ld};
+    const uint32_t box[2] = {64, 2 * kBK};
+    return make_map16(map, base, 2, dims, strides, box);
 }
 
 // C (or the split-K partials) as a rank-3 map: [z][rows][N] with 32 x 32 x 1 boxes.
@@ -1395,25 +1430,30 @@ int gemm_device(const qfmt_matrix_t* A, const qfmt_matrix_t* B, float* d_C, int6
     return QFMT_OK;
 }
 
-// C = A B^T on packed 16-bit codes of 1/5/10 (binary16 words) or 1/8/7 (bfloat16 words): the pair
-// kernel with kind::f16 MMAs.  A is M x K and B is N x K, both with K contiguous, so a stage is 64
-// K elements per 128-byte row and a TMEM chunk 128 (eight MMAs, as for TF32); the plan is the one
-// of a TF32 product of half the length, which costs the same number of MMAs.
-int gemm16_device(const uint16_t* d_A, int64_t lda, const uint16_t* d_B, int64_t ldb, int64_t M, int64_t N, int64_t K,
-                  float* d_C, int64_t ldc, const qfmt_format_t* fmt, void* d_workspace, size_t workspace_bytes,
-                  cudaStream_t stream) {
+// C = op(A) op(B) on packed 16-bit codes of 1/5/10 (binary16 words) or 1/8/7 (bfloat16 words): the
+// pair kernel with kind::f16 MMAs.  A stage is 64 K elements per 128-byte row and a TMEM chunk 128
+// (eight MMAs, as for TF32); the plan is the one of a TF32 product of half the length, which costs
+// the same number of MMAs.
+int gemm16_device(const qfmt_matrix16_t* A, const qfmt_matrix16_t* B, float* d_C, int64_t ldc, const qfmt_format_t* fmt,
+                  void* d_workspace, size_t workspace_bytes, cudaStream_t stream) {
     int rc = validate_format(fmt);
     if (rc != QFMT_OK) return rc;
     const bool f16 = fmt->e == 5 && fmt->m == 10, bf16 = fmt->e == 8 && fmt->m == 7;
     if (!f16 && !bf16) return QFMT_ERR_BAD_FORMAT;
-    if (M < 0 || N < 0 || K < 0 || M > (1 << 30) || N > (1 << 30) || K > (1 << 30)) return QFMT_ERR_BAD_ARG;
-    if (lda < K || ldb < K || ldc < N) return QFMT_ERR_BAD_ARG;
+    if (A == nullptr || B == nullptr) return QFMT_ERR_BAD_ARG;
+    if (A->rows < 0 || A->cols < 0 || B->rows < 0 || B->cols < 0) return QFMT_ERR_BAD_ARG;
+    const int64_t M = A->trans ? A->cols : A->rows, K = A->trans ? A->rows : A->cols;
+    const int64_t Kb = B->trans ? B->cols : B->rows, N = B->trans ? B->rows : B->cols;
+    if (K != Kb) return QFMT_ERR_BAD_ARG;
+    if (M > (1 << 30) || N > (1 << 30) || K > (1 << 30)) return QFMT_ERR_BAD_ARG;
+    if (A->ld < A->cols || B->ld < B->cols || ldc < N) return QFMT_ERR_BAD_ARG;
     if (d_workspace == nullptr || workspace_bytes < 16 || (reinterpret_cast<uintptr_t>(d_workspace) & 15u))
         return QFMT_ERR_BAD_ARG;
     if (M == 0 || N == 0) return QFMT_OK;
-    if ((d_A == nullptr || d_B == nullptr) && K != 0) return QFMT_ERR_BAD_ARG;
+    if ((A->ptr == nullptr || B->ptr == nullptr) && K != 0) return QFMT_ERR_BAD_ARG;
     if (d_C == nullptr || (reinterpret_cast<uintptr_t>(d_C) & 3u)) return QFMT_ERR_BAD_ARG;
-    if ((reinterpret_cast<uintptr_t>(d_A) & 15u) || (reinterpret_cast<uintptr_t>(d_B) & 15u) || (lda & 7) || (ldb & 7))
+    if ((reinterpret_cast<uintptr_t>(A->ptr) & 15u) || (reinterpret_cast<uintptr_t>(B->ptr) & 15u) || (A->ld & 7) ||
+        (B->ld & 7))
         return QFMT_ERR_BAD_ARG;  // TMA: 16-byte aligned bases and row pitches
     DeviceInfo dev;
     rc = current_device(&dev);
@@ -1430,7 +1470,8 @@ int gemm16_device(const uint16_t* d_A, int64_t lda, const uint16_t* d_B, int64_t
     p.ldc = ldc;
     p.C = d_C;
     p.status = status;
-    p.a_mn_major = p.b_mn_major = 0;
+    p.a_mn_major = A->trans ? 1 : 0;
+    p.b_mn_major = B->trans ? 0 : 1;
     p.tile_rows = 2 * kBM;
     p.tiles_m = (int)((M + p.tile_rows - 1) / p.tile_rows);
     p.tiles_n = (int)((N + kBN - 1) / kBN);
@@ -1449,9 +1490,9 @@ int gemm16_device(const uint16_t* d_A, int64_t lda, const uint16_t* d_B, int64_t
         p.tma_store = (N & 3) == 0 ? 1 : 0;
     }
     CUtensorMap ma, mb, mc;
-    rc = make_map16_2d(&ma, d_A, (uint64_t)K, (uint64_t)M, (uint64_t)lda, kBM);
+    rc = make_operand_map16(&ma, A->ptr, p.a_mn_major != 0, (uint64_t)M, (uint64_t)K, (uint64_t)A->ld, kBM, &p.a_blocked);
     if (rc != QFMT_OK) return rc;
-    rc = make_map16_2d(&mb, d_B, (uint64_t)K, (uint64_t)N, (uint64_t)ldb, kBN / 2);
+    rc = make_operand_map16(&mb, B->ptr, p.b_mn_major != 0, (uint64_t)N, (uint64_t)K, (uint64_t)B->ld, kBN / 2, &p.b_blocked);
     if (rc != QFMT_OK) return rc;
     if (p.tma_store)
         rc = make_map_c(&mc, p.C, (uint64_t)N, (uint64_t)M, (uint64_t)p.splits, (uint64_t)p.ldc, (uint64_t)M * (uint64_t)p.ldc);
@@ -1753,11 +1794,9 @@ extern "C" int qfmt_gemm(const qfmt_matrix_t* A, const qfmt_matrix_t* B, float* 
     return qfmt::gemm_device(A, B, d_C, ldc, fmt, d_workspace, workspace_bytes, (cudaStream_t)stream);
 }
 
-extern "C" int qfmt_gemm_packed16(const uint16_t* d_A, int64_t lda, const uint16_t* d_B, int64_t ldb, int64_t M,
-                                  int64_t N, int64_t K, float* d_C, int64_t ldc, const qfmt_format_t* fmt,
-                                  void* d_workspace, size_t workspace_bytes, void* stream) {
-    return qfmt::gemm16_device(d_A, lda, d_B, ldb, M, N, K, d_C, ldc, fmt, d_workspace, workspace_bytes,
-                               (cudaStream_t)stream);
+extern "C" int qfmt_gemm_packed16(const qfmt_matrix16_t* A, const qfmt_matrix16_t* B, float* d_C, int64_t ldc,
+                                  const qfmt_format_t* fmt, void* d_workspace, size_t workspace_bytes, void* stream) {
+    return qfmt::gemm16_device(A, B, d_C, ldc, fmt, d_workspace, workspace_bytes, (cudaStream_t)stream);
 }
 
 extern "C" int qfmt_conv(int32_t op, const qfmt_conv_t* geom, const float* d_p, const float* d_q, float* d_out,
@@ -1872,7 +1911,11 @@ extern "C" size_t qfmt_gemm_workspace_bytes(const qfmt_matrix_t* A, const qfmt_m
     return qfmt::kWorkspaceHeader + (splits > 1 ? (size_t)splits * (size_t)M * (size_t)N * sizeof(float) : 0);
 }
 
-extern "C" size_t qfmt_gemm_packed16_workspace_bytes(int64_t M, int64_t N, int64_t K) {
+extern "C" size_t qfmt_gemm_packed16_workspace_bytes(const qfmt_matrix16_t* A, const qfmt_matrix16_t* B) {
+    if (A == nullptr || B == nullptr || A->rows < 0 || A->cols < 0 || B->rows < 0 || B->cols < 0)
+        return qfmt::kWorkspaceHeader;
+    const int64_t M = A->trans ? A->cols : A->rows, K = A->trans ? A->rows : A->cols;
+    const int64_t N = B->trans ? B->rows : B->cols;
     if (M <= 0 || N <= 0 || K <= 0 || M > (1 << 30) || N > (1 << 30) || K > (1 << 30)) return qfmt::kWorkspaceHeader;
     const int splits = qfmt::plan_dense(M, N, (K + 1) / 2, 2).splits;
     return qfmt::kWorkspaceHeader + (splits > 1 ? (size_t)splits * (size_t)M * (size_t)N * sizeof(float) : 0);

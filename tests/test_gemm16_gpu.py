@@ -24,20 +24,24 @@ def codes_of(x, e, m):
     return codes, oracle.unpack16(codes, e, m)
 
 
-def gpu_gemm16(cA, cB, e, m, lda_pad=0, ldb_pad=0, ldc_pad=0, workspace=None):
-    M, K = cA.shape
-    N = cB.shape[0]
-    lda, ldb, ldc = K + lda_pad, K + ldb_pad, N + ldc_pad
-    dA = torch.full((max(M, 1), lda), 0x7E00, dtype=torch.int16, device=DEV)   # padding holds NaN codes
-    dB = torch.full((max(N, 1), ldb), 0x7E00, dtype=torch.int16, device=DEV)
-    if M and K:
-        dA[:M, :K] = torch.from_numpy(cA.view(np.int16)).to(DEV)
-    if N and K:
-        dB[:N, :K] = torch.from_numpy(cB.view(np.int16)).to(DEV)
+def gpu_gemm16(cA, cB, e, m, transA=False, transB=True, lda_pad=0, ldb_pad=0, ldc_pad=0, workspace=None):
+    """cA, cB are the STORED code matrices; C = op(A) op(B) as float32 [M, N].  The default flags are
+    the K-contiguous pair A [M, K], B [N, K]."""
+    def stored(c, pad, trans):
+        r, k = c.shape
+        d = torch.full((max(r, 1), k + pad), 0x7E00, dtype=torch.int16, device=DEV)   # padding holds NaN codes
+        if r and k:
+            d[:r, :k] = torch.from_numpy(np.ascontiguousarray(c).view(np.int16)).to(DEV)
+        return qf.make_matrix(d, trans, rows=r, cols=k, ld=k + pad), d
+    a, dA = stored(cA, lda_pad, transA)
+    b, dB = stored(cB, ldb_pad, transB)
+    M = cA.shape[1] if transA else cA.shape[0]
+    N = cB.shape[0] if transB else cB.shape[1]
+    ldc = N + ldc_pad
     dC = torch.full((max(M, 1), ldc), float("nan"), dtype=torch.float32, device=DEV)
-    wb = qf.qfmt_gemm_packed16_workspace_bytes(M, N, K) if workspace is None else workspace
+    wb = qf.qfmt_gemm_packed16_workspace_bytes(a, b) if workspace is None else workspace
     ws = torch.zeros(max(wb, 256), dtype=torch.uint8, device=DEV)
-    qf.qfmt_gemm_packed16(dA, lda, dB, ldb, M, N, K, dC, ldc, qf.make_format(e, m), ws, max(wb, 256))
+    qf.qfmt_gemm_packed16(a, b, dC, ldc, qf.make_format(e, m), ws, max(wb, 256))
     assert qf.qfmt_device_status(ws) == qf.QFMT_OK
     torch.cuda.synchronize()
     out = dC.cpu().numpy()[:M]
@@ -46,17 +50,17 @@ def gpu_gemm16(cA, cB, e, m, lda_pad=0, ldb_pad=0, ldc_pad=0, workspace=None):
     return out[:, :N]
 
 
-def worst_ratio(C, A, B, sample=None, seed=0):
-    """A [M, K], B [N, K] fp32 containers; returns the worst error as a multiple of the tolerance."""
+def worst_ratio(C, A, B, sample=None, seed=0, transA=False, transB=True):
+    """A, B: stored fp32 containers; returns the worst error as a multiple of the tolerance."""
     if sample is None:
-        ref, T = oracle.gemm(A, B, False, True)
+        ref, T = oracle.gemm(A, B, transA, transB)
         c = C.astype(np.float64)
     else:
         rng = np.random.default_rng(seed)
         M, N = C.shape
         ii = np.concatenate([rng.integers(0, M, size=sample), [0, M - 1, 0, M - 1]])
         jj = np.concatenate([rng.integers(0, N, size=sample), [0, N - 1, N - 1, 0]])
-        ref, T = oracle.gemm_sampled(A, B, ii, jj, False, True)
+        ref, T = oracle.gemm_sampled(A, B, ii, jj, transA, transB)
         c = C[ii, jj].astype(np.float64)
     err = np.abs(c - ref)
     assert np.all(err <= TOL * T), f"worst {float(np.max(err / np.maximum(T, 1e-300))) / TOL:.3f} x tolerance"
@@ -64,22 +68,25 @@ def worst_ratio(C, A, B, sample=None, seed=0):
 
 
 @pytest.mark.parametrize("e,m", FORMATS)
-@pytest.mark.parametrize("M,N,K", [(1, 1, 8), (5, 3, 16), (128, 256, 64), (256, 256, 128), (300, 260, 200),
+@pytest.mark.parametrize("transA", [False, True])
+@pytest.mark.parametrize("transB", [True, False])
+@pytest.mark.parametrize("M,N,K", [(1, 8, 8), (5, 3, 16), (64, 128, 64), (128, 256, 64), (256, 256, 128), (300, 260, 200),
                                    (513, 40, 1000), (64, 700, 72), (70, 50, 203), (257, 513, 4104)])
-def test_small_integers_are_bit_exact(e, m, M, N, K):
+def test_small_integers_are_bit_exact(e, m, M, N, K, transA, transB):
     """Entries in -4..4: every product and partial sum is a small integer, exact in any order, so
-    a wrong tile offset, K range, transpose or split shows up as a wrong integer.  Ragged sizes:
+    a wrong tile offset, K range, transpose or split shows up as a wrong integer.  All four
+    operand layouts (K-contiguous and M- / N-contiguous).  Ragged sizes:
     partial tiles in M and N, K not a multiple of the 64-element stage (the copy engine zero-fills
     past K; the NaN codes in the row padding must never be read as data)."""
     rng = np.random.default_rng(M * 7 + N * 3 + K)
-    A = rng.integers(-4, 5, size=(M, K)).astype(np.float32)
-    B = rng.integers(-4, 5, size=(N, K)).astype(np.float32)
+    A = rng.integers(-4, 5, size=(K, M) if transA else (M, K)).astype(np.float32)
+    B = rng.integers(-4, 5, size=(N, K) if transB else (K, N)).astype(np.float32)
     cA, qA = codes_of(A, e, m)
     cB, qB = codes_of(B, e, m)
     assert np.array_equal(qA, A) and np.array_equal(qB, B)
-    pad = 8 if K % 8 == 0 else 8 - K % 8
-    C = gpu_gemm16(cA, cB, e, m, lda_pad=pad, ldb_pad=pad + 8, ldc_pad=3)
-    ref, _ = oracle.gemm(A, B, False, True)
+    pad = lambda c: 8 if c % 8 == 0 else 8 - c % 8      # leading dimensions must be multiples of 8
+    C = gpu_gemm16(cA, cB, e, m, transA, transB, lda_pad=pad(A.shape[1]), ldb_pad=pad(B.shape[1]) + 8, ldc_pad=3)
+    ref, _ = oracle.gemm(A, B, transA, transB)
     assert np.array_equal(C.astype(np.float64), ref)
 
 
@@ -95,7 +102,10 @@ def test_operand_order_and_layout(e, m):
     B = np.ldexp(1.0, rng.integers(-12, 12, size=(N, K))).astype(np.float32) * rng.choice([-1.0, 1.0], size=(N, K))
     cA, _ = codes_of(A, e, m)
     cB, qB = codes_of(B, e, m)
-    C = gpu_gemm16(cA, cB, e, m, lda_pad=8 - K % 8 if K % 8 else 0)
+    C = gpu_gemm16(cA, cB, e, m)
+    assert np.array_equal(C, 2.0 * qB[:, ks].T)
+    # the same product from the transposed copies of both operands (M and N contiguous)
+    C = gpu_gemm16(np.ascontiguousarray(cA.T), np.ascontiguousarray(cB.T), e, m, True, False, lda_pad=6, ldb_pad=2)
     assert np.array_equal(C, 2.0 * qB[:, ks].T)
 
 
@@ -145,6 +155,9 @@ def test_config5_ffn_up_forward_full_size(e, m):
     cB, qB = codes_of(np.ascontiguousarray(cfg["W"].T), e, m)
     C = gpu_gemm16(cA, cB, e, m)
     print("config5 ffn_up", (e, m), worst_ratio(C, qA, qB, sample=65536, seed=9))
+    cW, qW = codes_of(cfg["W"], e, m)                     # stored [d_in, d_out]: N contiguous
+    C2 = gpu_gemm16(cA, cW, e, m, False, False)
+    assert np.array_equal(C.view(np.uint32), C2.view(np.uint32))
 
 
 @pytest.mark.parametrize("e,m", FORMATS)
@@ -152,37 +165,41 @@ def test_long_k_weight_gradient_shape(e, m):
     """1024 x 1024 x 8192: few tiles and a long K, so K is split among CTAs and the parts are added
     by the reduction pass."""
     rng = workloads.rng_for(701, e)
-    Xt = workloads.lognormal_tensor(rng, (1024, 8192), -3.0, 2.0)
-    Gt = workloads.lognormal_tensor(rng, (1024, 8192), -6.0, 3.0)
-    cA, qA = codes_of(Xt, e, m)
-    cB, qB = codes_of(Gt, e, m)
-    assert qf.qfmt_gemm_packed16_workspace_bytes(1024, 1024, 8192) > 256
-    C = gpu_gemm16(cA, cB, e, m)
-    print("long K", (e, m), worst_ratio(C, qA, qB, sample=32768, seed=3))
+    X = workloads.lognormal_tensor(rng, (8192, 1024), -3.0, 2.0)
+    G = workloads.lognormal_tensor(rng, (8192, 1024), -6.0, 3.0)
+    cA, qA = codes_of(X, e, m)
+    cB, qB = codes_of(G, e, m)
+    C = gpu_gemm16(cA, cB, e, m, True, False)           # dW = X^T dY: tokens are K, both operands MN-major
+    print("wgrad", (e, m), worst_ratio(C, qA, qB, sample=32768, seed=3, transA=True, transB=False))
+    cAt, cBt = np.ascontiguousarray(cA.T), np.ascontiguousarray(cB.T)
+    C2 = gpu_gemm16(cAt, cBt, e, m)                      # the same product from K-contiguous copies
+    assert np.array_equal(C.view(np.uint32), C2.view(np.uint32))
 
 
 def test_empty_and_errors():
     fmt = qf.make_format(5, 10)
-    d16 = torch.zeros(64 * 64, dtype=torch.int16, device=DEV)
+    d16 = torch.zeros(64 * 64 + 8, dtype=torch.int16, device=DEV)
     dC = torch.full((64, 64), 5.0, dtype=torch.float32, device=DEV)
     ws = torch.zeros(256, dtype=torch.uint8, device=DEV)
-    qf.qfmt_gemm_packed16(d16, 64, d16, 64, 0, 64, 64, dC, 64, fmt, ws, 256)       # M = 0: nothing happens
-    qf.qfmt_gemm_packed16(d16, 64, d16, 64, 64, 0, 64, dC, 64, fmt, ws, 256)
+    mat = lambda rows, cols, ld=64, trans=False, t=d16: qf.make_matrix(t, trans, rows=rows, cols=cols, ld=ld)
+    qf.qfmt_gemm_packed16(mat(0, 64), mat(64, 64), dC, 64, fmt, ws, 256)       # M = 0: nothing happens
+    qf.qfmt_gemm_packed16(mat(64, 64), mat(64, 0), dC, 64, fmt, ws, 256)       # N = 0
     torch.cuda.synchronize()
     assert torch.all(dC == 5.0)
-    qf.qfmt_gemm_packed16(d16, 64, d16, 64, 64, 64, 0, dC, 64, fmt, ws, 256)       # K = 0: zeros
+    qf.qfmt_gemm_packed16(mat(64, 0), mat(0, 64), dC, 64, fmt, ws, 256)        # K = 0: zeros
     torch.cuda.synchronize()
     assert torch.all(dC == 0.0)
     for bad_fmt in ((6, 9), (4, 3), (8, 10)):
         with pytest.raises(qf.QfmtError) as ei:
-            qf.qfmt_gemm_packed16(d16, 64, d16, 64, 64, 64, 64, dC, 64, qf.make_format(*bad_fmt), ws, 256)
+            qf.qfmt_gemm_packed16(mat(64, 64), mat(64, 64), dC, 64, qf.make_format(*bad_fmt), ws, 256)
         assert ei.value.status == qf.QFMT_ERR_BAD_FORMAT
-    for args in ((d16, 60, d16, 64, 64, 64, 64, dC, 64),      # lda below K
-                 (d16, 68, d16, 64, 8, 64, 64, dC, 64),       # lda not a multiple of 8
-                 (d16[1:], 64, d16, 64, 8, 64, 64, dC, 64),   # base not 16-byte aligned
-                 (d16, 64, d16, 64, 64, 64, 64, dC, 60),      # ldc below N
-                 (None, 64, d16, 64, 64, 64, 64, dC, 64)):
+    for a, b, ldc in ((mat(64, 64, ld=56), mat(64, 64), 64),          # ld below the row length
+                      (mat(8, 60, ld=60), mat(60, 64), 64),           # ld not a multiple of 8
+                      (mat(8, 64, t=d16[1:]), mat(64, 64), 64),       # base not 16-byte aligned
+                      (mat(64, 64), mat(32, 64), 64),                 # K mismatch
+                      (mat(64, 64), mat(64, 64), 60),                 # ldc below N
+                      (mat(64, 64, t=None), mat(64, 64), 64)):
         with pytest.raises(qf.QfmtError) as ei:
-            qf.qfmt_gemm_packed16(*args, fmt, ws, 256)
+            qf.qfmt_gemm_packed16(a, b, dC, ldc, fmt, ws, 256)
         assert ei.value.status == qf.QFMT_ERR_BAD_ARG
     torch.cuda.synchronize()
