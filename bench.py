@@ -512,44 +512,48 @@ def pack16_section(torch, qf, dev, peaks, d_in, n, reps=20):
 
 
 def gemm16_section(torch, qf, dev, peaks, reps=5):
-    """The four forward products of the BERT-large FC stack on packed 16-bit operands (1/5/10 as
-    binary16 words, 1/8/7 as bfloat16 words): the rounding pass writes the codes of X [tokens, d_in]
-    and of the weight stored output-major [d_out, d_in]; qfmt_gemm_packed16 contracts them."""
+    """One step of the BERT-large FC stack (12 products: forward, activation gradient, weight
+    gradient of 4 layers) on packed 16-bit operands: the rounding pass writes the codes of X, W and
+    dY (1/5/10 as binary16 words, 1/8/7 as bfloat16 words), qfmt_gemm_packed16 contracts them in
+    the layouts they are stored in."""
     out = {"metric": "emulated GEMM on packed 16-bit operands TFLOP/s", "unit": "TFLOP/s", "runs": {},
-           "workload": "config5 BERT-large FC stack, forward products of the 4 layers (8192 tokens), packed codes"}
+           "workload": "config5 BERT-large FC stack, one step: 4 layers x fwd/dgrad/wgrad, operands as packed codes"}
     for tag, e, m in (("1/5/10 binary16", 5, 10), ("1/8/7 bfloat16", 8, 7)):
         fmt = qf.make_format(e, m, 1)
-        jobs, flops, ws_bytes, pack_ms = [], 0.0, 256, 0.0
+        jobs, flops, fwd_flops, ws_bytes, pack_ms = [], 0.0, 0.0, 256, 0.0
+        st = torch.zeros(qf.STATS_WORDS, dtype=torch.int64, device=dev)
         for layer in range(len(workloads.CONFIG5_LAYERS)):
             c = workloads.config5_layer(layer, step=0)
-            X = torch.from_numpy(c["X"]).to(dev)
-            Wt = torch.from_numpy(np.ascontiguousarray(c["W"].T)).to(dev)
-            cX = torch.empty(X.shape, dtype=torch.int16, device=dev)
-            cW = torch.empty(Wt.shape, dtype=torch.int16, device=dev)
-            st = torch.zeros(qf.STATS_WORDS, dtype=torch.int64, device=dev)
-
-            def pack():
-                qf.qfmt_quantize_stats_pack16(X, cX, X.numel(), fmt, st)
-                qf.qfmt_quantize_stats_pack16(Wt, cW, Wt.numel(), fmt, st)
-            pack()
-            pack_ms += statistics.median(time_events(torch, pack, 3))
-            M, K = X.shape
-            N = Wt.shape[0]
-            jobs.append((qf.make_matrix(cX), qf.make_matrix(cW, True), N, torch.empty(M, N, dtype=torch.float32, device=dev),
-                         (cX, cW)))
-            ws_bytes = max(ws_bytes, qf.qfmt_gemm_packed16_workspace_bytes(jobs[-1][0], jobs[-1][1]))
-            flops += 2.0 * M * N * K
+            t = {}
+            for name, scale in (("X", 1.0), ("W", 1.0), ("dY", c["grad_scale"])):
+                src = torch.from_numpy(c[name]).to(dev)
+                codes = torch.empty(src.shape, dtype=torch.int16, device=dev)
+                f = qf.make_format(e, m, 1, scale)
+                qf.qfmt_quantize_stats_pack16(src, codes, src.numel(), f, st)
+                pack_ms += statistics.median(time_events(
+                    torch, lambda: qf.qfmt_quantize_stats_pack16(src, codes, src.numel(), f, st), 3))
+                t[name] = codes
+            tokens, d_in = c["X"].shape
+            d_out = c["W"].shape[1]
+            for A, ta, B, tb, M, N, K in ((t["X"], False, t["W"], False, tokens, d_out, d_in),
+                                          (t["dY"], False, t["W"], True, tokens, d_in, d_out),
+                                          (t["X"], True, t["dY"], False, d_in, d_out, tokens)):
+                C = torch.empty(M, N, dtype=torch.float32, device=dev)
+                jobs.append((qf.make_matrix(A, ta), qf.make_matrix(B, tb), C, N, (A, B)))
+                ws_bytes = max(ws_bytes, qf.qfmt_gemm_packed16_workspace_bytes(jobs[-1][0], jobs[-1][1]))
+                flops += 2.0 * M * N * K
         ws = torch.zeros(ws_bytes, dtype=torch.uint8, device=dev)
 
-        def step():
-            for a, b, N, C, _ in jobs:
+        def step(which=jobs):
+            for a, b, C, N, _ in which:
                 qf.qfmt_gemm_packed16(a, b, C, N, fmt, ws, ws.numel())
         for _ in range(3):
             step()
         assert qf.qfmt_device_status(ws) == qf.QFMT_OK
         ms = statistics.median(time_events(torch, step, reps))
         tf = flops / ms / 1e9
-        out["runs"][tag] = {"ms_per_step": ms, "tflops": tf, "rounding_to_codes_ms": pack_ms, "gpu_launches_per_step": len(jobs),
+        out["runs"][tag] = {"ms_per_step": ms, "tflops": tf, "rounding_to_codes_ms": pack_ms, "gemms_per_step": len(jobs),
+                            "gpu_launches_per_step": len(jobs),
                             "roofline": {"bound": "tensor", "achieved": tf, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
                                          "frac": tf / peaks["bf16_tflops"], "traffic": None,
                                          "peak_source": f"bf16 {peaks['source']} burst"}}
