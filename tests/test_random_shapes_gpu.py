@@ -163,6 +163,39 @@ def test_fmacs_product(seed):
             qf.qfmt_gemm_tile_policy(0)
 
 
+@pytest.mark.parametrize("seed", range(16))
+def test_fmacs_product_on_packed_codes(seed):
+    """qfmt_gemm_packed16 on random shapes (any M, N, K; stored row lengths padded to multiples of
+    8), layouts and the two formats; against the oracle's expansion of the same codes."""
+    rng = np.random.default_rng(9500 + seed)
+    for _ in range(3):
+        e, m = [(5, 10), (8, 7)][int(rng.integers(2))]
+        M, N, K = int(rng.integers(1, 480)), int(rng.integers(1, 640)), int(rng.integers(1, 2800))
+        tA, tB = bool(rng.integers(2)), bool(rng.integers(2))
+        cA, _ = oracle.quantize_stats_pack16(workloads.lognormal_tensor(workloads.rng_for(int(rng.integers(1 << 30))),
+                                                                        (K, M) if tA else (M, K), -3.0, 2.0, p_zero=0.02),
+                                             e, m, 1, 1.0)
+        cB, _ = oracle.quantize_stats_pack16(workloads.normal_tensor(workloads.rng_for(int(rng.integers(1 << 30))),
+                                                                     (N, K) if tB else (K, N), 0.05), e, m, 1, 1.0)
+        A, B = oracle.unpack16(cA, e, m), oracle.unpack16(cB, e, m)
+        mats = []
+        for c, t in ((cA, tA), (cB, tB)):
+            ld = (c.shape[1] + 7) // 8 * 8 + 8 * int(rng.integers(0, 2))
+            d = torch.full((c.shape[0], ld), 0x7C00, dtype=torch.int16, device=DEV)   # padding: binary16 infinity
+            d[:, :c.shape[1]] = torch.from_numpy(c.view(np.int16)).to(DEV)
+            mats.append((qf.make_matrix(d, t, rows=c.shape[0], cols=c.shape[1], ld=ld), d))
+        ldc = N + int(rng.integers(0, 3))
+        dC = torch.full((M, ldc), 7.0, dtype=torch.float32, device=DEV)
+        wb = max(256, qf.qfmt_gemm_packed16_workspace_bytes(mats[0][0], mats[1][0]))
+        ws = torch.zeros(wb, dtype=torch.uint8, device=DEV)
+        qf.qfmt_gemm_packed16(mats[0][0], mats[1][0], dC, ldc, qf.make_format(e, m), ws, wb)
+        assert qf.qfmt_device_status(ws) == qf.QFMT_OK
+        ref, T = oracle.gemm(A, B, tA, tB)
+        err = np.abs(dC[:, :N].cpu().numpy().astype(np.float64) - ref)
+        assert np.all(err <= 2.0 ** -20 * T), (e, m, M, N, K, tA, tB, float(np.max(err / np.maximum(T, 1e-300))) * 2 ** 20)
+        assert torch.all(dC[:, N:] == 7.0)
+
+
 @pytest.mark.parametrize("seed", range(12))
 def test_convolution_products(seed):
     """Random small geometries with small-integer tensors: every order of summation is exact, so the
