@@ -518,23 +518,26 @@ def gemm16_section(torch, qf, dev, peaks, reps=5):
     the layouts they are stored in."""
     out = {"metric": "emulated GEMM on packed 16-bit operands TFLOP/s", "unit": "TFLOP/s", "runs": {},
            "workload": "config5 BERT-large FC stack, one step: 4 layers x fwd/dgrad/wgrad, operands as packed codes"}
+    layers = []
+    for layer in range(len(workloads.CONFIG5_LAYERS)):
+        c = workloads.config5_layer(layer, step=0)
+        layers.append(({k: torch.from_numpy(c[k]).to(dev) for k in ("X", "W", "dY")}, c["grad_scale"]))
     for tag, e, m in (("1/5/10 binary16", 5, 10), ("1/8/7 bfloat16", 8, 7)):
         fmt = qf.make_format(e, m, 1)
-        jobs, flops, fwd_flops, ws_bytes, pack_ms = [], 0.0, 0.0, 256, 0.0
+        jobs, flops, ws_bytes, pack_ms = [], 0.0, 256, 0.0
         st = torch.zeros(qf.STATS_WORDS, dtype=torch.int64, device=dev)
-        for layer in range(len(workloads.CONFIG5_LAYERS)):
-            c = workloads.config5_layer(layer, step=0)
+        for fp32, grad_scale in layers:
             t = {}
-            for name, scale in (("X", 1.0), ("W", 1.0), ("dY", c["grad_scale"])):
-                src = torch.from_numpy(c[name]).to(dev)
+            for name, scale in (("X", 1.0), ("W", 1.0), ("dY", grad_scale)):
+                src = fp32[name]
                 codes = torch.empty(src.shape, dtype=torch.int16, device=dev)
                 f = qf.make_format(e, m, 1, scale)
                 qf.qfmt_quantize_stats_pack16(src, codes, src.numel(), f, st)
                 pack_ms += statistics.median(time_events(
                     torch, lambda: qf.qfmt_quantize_stats_pack16(src, codes, src.numel(), f, st), 3))
                 t[name] = codes
-            tokens, d_in = c["X"].shape
-            d_out = c["W"].shape[1]
+            tokens, d_in = fp32["X"].shape
+            d_out = fp32["W"].shape[1]
             for A, ta, B, tb, M, N, K in ((t["X"], False, t["W"], False, tokens, d_out, d_in),
                                           (t["dY"], False, t["W"], True, tokens, d_in, d_out),
                                           (t["X"], True, t["dY"], False, d_in, d_out, tokens)):
