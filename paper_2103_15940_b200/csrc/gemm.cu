@@ -27,6 +27,13 @@
 // A third level keeps the sequential part short: after kFlushChunks chunk sums (1024 K elements)
 // the register sums are added into the C tile itself and reset, so an output sees at most
 // kFlushChunks + K/1024 rounded additions of large partial sums instead of K/64.
+//
+// Packed 16-bit operands.  1/5/10 codes are IEEE binary16 words and 1/8/7 codes are bfloat16 words,
+// so for these two formats the CTA-pair kernel (gemm_tf32_pair_kernel, despite its name) is also
+// instantiated with kind::f16 MMAs that read the codes as they are stored: a stage is then 64 K
+// elements per 128-byte row, a chunk 128 K elements (still eight MMAs) and a group 2048; the
+// products are as exact as in TF32 and the three levels are the same (gemm16_device).
+//
 // Every mbarrier wait is bounded; on expiry the thread records QFMT_ERR_TIMEOUT in the status
 // word, raises a CTA-wide abort flag and every role drains to the common exit, where TMEM is
 // released.
