@@ -1258,7 +1258,7 @@ struct DensePlan {
 // Picks the plan with the least estimated time.  The unit is the time one CTA pair needs for one
 // 64-element K chunk of a 256 x 256 tile, about a microsecond; a single CTA needs 1.07 of it for
 // half the area.  A tile costs its chunks plus three units of exposed epilogue; split K adds a
-// reduction pass over (splits + 1) x M x N floats at about 4 TB/s plus a launch.  The wave count
+// reduction pass over (splits + 1) x M x N floats at about 6.5 TB/s (measured: the partials are still in L2) plus a launch.  The wave count
 // is taken for a 148-SM part whatever the device, so that the plan, and with it the summation
 // order, depends on the problem alone.
 DensePlan plan_dense(int64_t M, int64_t N, int64_t K, int policy_override = -1) {
@@ -1280,7 +1280,7 @@ DensePlan plan_dense(int64_t M, int64_t N, int64_t K, int policy_override = -1) 
             if (splits != want) continue;                               // same plan as a smaller request
             const int64_t waves = (tiles * splits + units - 1) / units;
             double cost = (double)waves * ((double)((per + kChunkKB - 1) / kChunkKB) * per_chunk + 3.0);
-            if (splits > 1) cost += 3.0 + (double)(splits + 1) * (double)M * (double)N * 4.0 / 4.0e6;
+            if (splits > 1) cost += 3.0 + (double)(splits + 1) * (double)M * (double)N * 4.0 / 6.5e6;
             if (best_cost < 0.0 || cost < best_cost * 0.97) {  // more splits only for a clear gain
                 best_cost = cost;
                 best = {pair != 0, (int)splits};
