@@ -153,6 +153,22 @@ int qfmt_bias_quantize_stats(const float* d_acc, int64_t ld_acc, const float* d_
                              int accumulate, void* stream);
 
 /*
+ * The same layer-output pass with Y written as packed 16-bit codes (the encoding of
+ * qfmt_quantize_stats_pack16) instead of fp32 containers, so that a layer whose operands are codes
+ * (qfmt_gemm_packed16) hands codes to the next one: 6 bytes per element instead of 8, and no
+ * separate packing pass.  Arguments as for qfmt_bias_quantize_stats except
+ *   d_codes   device, 2-byte aligned; rows x cols codes with leading dimension ld_codes >= cols.
+ *             8-byte aligned d_codes with 16-byte aligned d_acc and d_bias and cols, ld_acc,
+ *             ld_codes multiples of 4 select the vector path, anything else a scalar path.
+ * The codes are those of the containers qfmt_bias_quantize_stats would write (NaN: the positive
+ * quiet NaN code).  Requires m <= 10 and e + m <= 15 (QFMT_ERR_BAD_FORMAT otherwise).
+ * Errors: QFMT_ERR_BAD_FORMAT, QFMT_ERR_BAD_ARG, QFMT_ERR_UNSUPPORTED_ARCH, QFMT_ERR_CUDA.
+ */
+int qfmt_bias_quantize_stats_pack16(const float* d_acc, int64_t ld_acc, const float* d_bias, uint16_t* d_codes,
+                                    int64_t ld_codes, int64_t rows, int64_t cols, const qfmt_format_t* fmt,
+                                    qfmt_stats_t* d_stats, int accumulate, void* stream);
+
+/*
  * Dynamic loss scaling with the scale kept in device memory.  Section II describes loss scaling
  * and Section V trains every format "with DLS" and without; the paper cites the technique and
  * states no rule, so the usual one is taken: a step whose gradient tensors held any overflow,

@@ -86,6 +86,8 @@ def lib() -> ctypes.CDLL:
         L.qfmt_bias_quantize_stats.argtypes = [vp, ctypes.c_int64, vp, vp, ctypes.c_int64, ctypes.c_int64,
                                                ctypes.c_int64, fmtp, vp, ci, vp]
         L.qfmt_bias_quantize_stats.restype = ci
+        L.qfmt_bias_quantize_stats_pack16.argtypes = L.qfmt_bias_quantize_stats.argtypes
+        L.qfmt_bias_quantize_stats_pack16.restype = ci
         L.qfmt_quantize_stats_pack16.argtypes = [vp, vp, sz, fmtp, vp, ci, vp]
         L.qfmt_quantize_stats_pack16.restype = ci
         L.qfmt_unpack16.argtypes = [vp, vp, sz, fmtp, vp]
@@ -195,6 +197,15 @@ def qfmt_bias_quantize_stats(d_acc, ld_acc: int, d_bias, d_out, ld_out: int, row
     _check(lib().qfmt_bias_quantize_stats(_ptr(d_acc), int(ld_acc), _ptr(d_bias), _ptr(d_out), int(ld_out),
                                           int(rows), int(cols), ctypes.byref(fmt), _ptr(d_stats), int(accumulate),
                                           _stream_handle(stream)), "qfmt_bias_quantize_stats")
+
+
+def qfmt_bias_quantize_stats_pack16(d_acc, ld_acc: int, d_bias, d_codes, ld_codes: int, rows: int, cols: int,
+                                    fmt: qfmt_format_t, d_stats=None, accumulate: int = 0, stream=None) -> None:
+    """Y = R(R(acc) + R(bias)) as packed 16-bit codes, with the statistics of Y; see include/qfmt.h."""
+    _check(lib().qfmt_bias_quantize_stats_pack16(_ptr(d_acc), int(ld_acc), _ptr(d_bias), _ptr(d_codes), int(ld_codes),
+                                                 int(rows), int(cols), ctypes.byref(fmt), _ptr(d_stats),
+                                                 int(accumulate), _stream_handle(stream)),
+           "qfmt_bias_quantize_stats_pack16")
 
 
 def qfmt_quantize_stats_pack16(d_in, d_codes, n: int, fmt: qfmt_format_t, d_stats=None, accumulate: int = 0,

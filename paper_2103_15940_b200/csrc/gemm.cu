@@ -1818,9 +1818,9 @@ extern "C" size_t qfmt_conv_workspace_bytes(int32_t op, const qfmt_conv_t* geom)
 }
 
 namespace qfmt {
-int bias_quantize_stats_device(const float* d_acc, int64_t ld_acc, const float* d_bias, float* d_out, int64_t ld_out,
+int bias_quantize_stats_device(const float* d_acc, int64_t ld_acc, const float* d_bias, void* d_out, int64_t ld_out,
                                int64_t rows, int64_t cols, const qfmt_format_t* fmt, qfmt_stats_t* d_stats,
-                               int accumulate, cudaStream_t stream);
+                               int accumulate, cudaStream_t stream, bool pack);
 namespace {
 
 // Rounds the bias vector for the fused epilogue; entries n .. padded-1 become zero.
@@ -1867,7 +1867,7 @@ int linear_forward_device(const qfmt_matrix_t* A, const qfmt_matrix_t* B, const 
     if (!fused) {
         rc = gemm_device(A, B, d_Y, ldy, fmt, d_workspace, gemm_bytes, stream);
         if (rc != QFMT_OK) return rc;
-        return bias_quantize_stats_device(d_Y, ldy, d_bias, d_Y, ldy, M, N, fmt, d_stats, accumulate, stream);
+        return bias_quantize_stats_device(d_Y, ldy, d_bias, d_Y, ldy, M, N, fmt, d_stats, accumulate, stream, false);
     }
     DeviceInfo dev;
     rc = current_device(&dev);

@@ -44,6 +44,10 @@ __device__ __forceinline__ void store_stream(uint4* p, const uint4& v) {
                  :: "l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
 
+__device__ __forceinline__ void store_stream(uint2* p, const uint2& v) {
+    asm volatile("st.global.cs.v2.u32 [%0], {%1,%2};" :: "l"(p), "r"(v.x), "r"(v.y) : "memory");
+}
+
 constexpr int kThreads = 512;
 constexpr int kUnroll = 4;  // 128-bit loads in flight per thread
 
@@ -388,11 +392,15 @@ __device__ __forceinline__ uint32_t bias_round_one(uint32_t acc, uint32_t rb, co
     return q;
 }
 
-template <bool kStats, bool kScale>
+// kPack: the output is written as packed 16-bit codes (out_v points at uint16_t, ld_out counts codes;
+// four codes per 8-byte store) instead of fp32 containers.
+template <bool kStats, bool kScale, bool kPack>
 __global__ void __launch_bounds__(kThreads)
-bias_quantize_stats_kernel(const uint32_t* acc, long long ld_acc, const uint32_t* __restrict__ bias, uint32_t* out,
+bias_quantize_stats_kernel(const uint32_t* acc, long long ld_acc, const uint32_t* __restrict__ bias, void* out_v,
                            long long ld_out, unsigned long long rows, uint32_t c4, uint32_t cw, uint32_t rpp,
-                           QuantParams p, qfmt_stats_t* __restrict__ stats) {
+                           QuantParams p, qfmt_stats_t* __restrict__ stats, int sign_shift) {
+    uint32_t* const out = kPack ? nullptr : static_cast<uint32_t*>(out_v);
+    uint16_t* const out16 = kPack ? static_cast<uint16_t*>(out_v) : nullptr;
     extern __shared__ uint32_t lane_hist[];  // [(top + kExtraBins)][32]
     const int nbins = p.top + kExtraBins;
     const int lane = threadIdx.x & 31;
@@ -416,7 +424,8 @@ bias_quantize_stats_kernel(const uint32_t* acc, long long ld_acc, const uint32_t
             b.w = quantize_one<kScale>(raw.w, p, unused);
             unsigned long long row = (unsigned long long)blockIdx.x * rpp + r_local;
             const uint4* pa = reinterpret_cast<const uint4*>(acc + row * ld_acc) + cc;
-            uint4* po = reinterpret_cast<uint4*>(out + row * ld_out) + cc;
+            uint4* po = kPack ? nullptr : reinterpret_cast<uint4*>(out + row * ld_out) + cc;
+            uint2* po16 = kPack ? reinterpret_cast<uint2*>(out16 + row * ld_out) + cc : nullptr;
             const unsigned long long step_a = row_step * (unsigned long long)ld_acc / 4ull;  // in vectors
             const unsigned long long step_o = row_step * (unsigned long long)ld_out / 4ull;
             for (; row < rows; row += row_step * kUnroll) {
@@ -433,7 +442,13 @@ bias_quantize_stats_kernel(const uint32_t* acc, long long ld_acc, const uint32_t
                         q.y = bias_round_one<kScale>(v[u].y, b.y, p, inf_bits, b1);
                         q.z = bias_round_one<kScale>(v[u].z, b.z, p, inf_bits, b2);
                         q.w = bias_round_one<kScale>(v[u].w, b.w, p, inf_bits, b3);
-                        store_stream(po + u * step_o, q);
+                        if (kPack) {
+                            const uint32_t c0 = encode_container(q.x, p, sign_shift), c1 = encode_container(q.y, p, sign_shift);
+                            const uint32_t c2 = encode_container(q.z, p, sign_shift), c3 = encode_container(q.w, p, sign_shift);
+                            store_stream(po16 + u * step_o, make_uint2(c0 | (c1 << 16), c2 | (c3 << 16)));
+                        } else {
+                            store_stream(po + u * step_o, q);
+                        }
                         if (kStats) {
                             atomicAdd(&lane_hist[b0 * 32 + lane], 1u);
                             atomicAdd(&lane_hist[b1 * 32 + lane], 1u);
@@ -443,7 +458,7 @@ bias_quantize_stats_kernel(const uint32_t* acc, long long ld_acc, const uint32_t
                     }
                 }
                 pa += kUnroll * step_a;
-                po += kUnroll * step_o;
+                if (kPack) po16 += kUnroll * step_o; else po += kUnroll * step_o;
             }
         }
     }
@@ -460,11 +475,11 @@ bias_quantize_stats_kernel(const uint32_t* acc, long long ld_acc, const uint32_t
 }
 
 // Any alignment and any column count: one element per thread per step, bias rounded per element.
-template <bool kStats, bool kScale>
+template <bool kStats, bool kScale, bool kPack>
 __global__ void __launch_bounds__(kThreads)
 bias_quantize_stats_scalar_kernel(const uint32_t* acc, long long ld_acc, const uint32_t* __restrict__ bias,
-                                  uint32_t* out, long long ld_out, unsigned long long rows, unsigned long long cols,
-                                  QuantParams p, qfmt_stats_t* __restrict__ stats) {
+                                  void* out_v, long long ld_out, unsigned long long rows, unsigned long long cols,
+                                  QuantParams p, qfmt_stats_t* __restrict__ stats, int sign_shift) {
     extern __shared__ uint32_t lane_hist[];
     const int nbins = p.top + kExtraBins;
     const int lane = threadIdx.x & 31;
@@ -479,7 +494,9 @@ bias_quantize_stats_scalar_kernel(const uint32_t* acc, long long ld_acc, const u
         const unsigned long long r = i / cols, c = i % cols;
         int unused, b;
         const uint32_t rb = quantize_one<kScale>(bias[c], p, unused);
-        out[r * ld_out + c] = bias_round_one<kScale>(acc[r * ld_acc + c], rb, p, inf_bits, b);
+        const uint32_t q = bias_round_one<kScale>(acc[r * ld_acc + c], rb, p, inf_bits, b);
+        if (kPack) static_cast<uint16_t*>(out_v)[r * ld_out + c] = (uint16_t)encode_container(q, p, sign_shift);
+        else static_cast<uint32_t*>(out_v)[r * ld_out + c] = q;
         if (kStats) atomicAdd(&lane_hist[b * 32 + lane], 1u);
     }
     if (kStats) {
@@ -612,19 +629,21 @@ int quantize_stats_transpose_device(const float* d_in, float* d_out, int64_t bat
 }
 
 
-int bias_quantize_stats_device(const float* d_acc, int64_t ld_acc, const float* d_bias, float* d_out, int64_t ld_out,
+// pack: d_out points at 16-bit codes (ld_out counts codes) instead of fp32 containers.
+int bias_quantize_stats_device(const float* d_acc, int64_t ld_acc, const float* d_bias, void* d_out, int64_t ld_out,
                                int64_t rows, int64_t cols, const qfmt_format_t* fmt, qfmt_stats_t* d_stats,
-                               int accumulate, cudaStream_t stream) {
+                               int accumulate, cudaStream_t stream, bool pack = false) {
     int rc = validate_format(fmt);
     if (rc != QFMT_OK) return rc;
     if (fmt->m > 10) return QFMT_ERR_BAD_FORMAT;  // the one-add sum is only then a single rounding
+    if (pack && fmt->e + fmt->m > 15) return QFMT_ERR_BAD_FORMAT;  // sign, exponent and mantissa must fit 16 bits
     if (accumulate != 0 && accumulate != 1) return QFMT_ERR_BAD_ARG;
     if (rows < 0 || cols < 0 || rows > ((int64_t)1 << 40) || cols > 0x7FFFFFFF) return QFMT_ERR_BAD_ARG;
     const unsigned long long n = (unsigned long long)rows * (unsigned long long)cols;
     if (n > (1ull << 40)) return QFMT_ERR_BAD_ARG;
     if (n != 0 && (d_acc == nullptr || d_bias == nullptr || d_out == nullptr)) return QFMT_ERR_BAD_ARG;
     if (n != 0 && (ld_acc < cols || ld_out < cols)) return QFMT_ERR_BAD_ARG;
-    if ((reinterpret_cast<uintptr_t>(d_acc) & 3u) || (reinterpret_cast<uintptr_t>(d_out) & 3u) ||
+    if ((reinterpret_cast<uintptr_t>(d_acc) & 3u) || (reinterpret_cast<uintptr_t>(d_out) & (pack ? 1u : 3u)) ||
         (reinterpret_cast<uintptr_t>(d_bias) & 3u) || (reinterpret_cast<uintptr_t>(d_stats) & 7u))
         return QFMT_ERR_BAD_ARG;
     DeviceInfo dev;
@@ -636,12 +655,14 @@ int bias_quantize_stats_device(const float* d_acc, int64_t ld_acc, const float* 
     const QuantParams p = make_params(*fmt);
     const uint32_t* acc = reinterpret_cast<const uint32_t*>(d_acc);
     const uint32_t* bias = reinterpret_cast<const uint32_t*>(d_bias);
-    uint32_t* out = reinterpret_cast<uint32_t*>(d_out);
+    void* out = d_out;
+    const int sign_shift = fmt->e + fmt->m;
     const bool has_stats = d_stats != nullptr, has_scale = fmt->loss_scale != 1.0f;
     const size_t hist_bytes = has_stats ? (size_t)(p.top + kExtraBins) * 32 * sizeof(uint32_t) : 0;
+    // vector path: four elements per access, 16 bytes of fp32 and 8 bytes of codes
     const bool vec = (cols % 4 == 0) && (ld_acc % 4 == 0) && (ld_out % 4 == 0) &&
-                     !((reinterpret_cast<uintptr_t>(d_acc) | reinterpret_cast<uintptr_t>(d_out) |
-                        reinterpret_cast<uintptr_t>(d_bias)) & 15u);
+                     !((reinterpret_cast<uintptr_t>(d_acc) | reinterpret_cast<uintptr_t>(d_bias)) & 15u) &&
+                     !(reinterpret_cast<uintptr_t>(d_out) & (pack ? 7u : 15u));
     cudaError_t err = cudaSuccess;
     if (vec) {
         const uint32_t c4 = (uint32_t)(cols / 4);
@@ -652,21 +673,25 @@ int bias_quantize_stats_device(const float* d_acc, int64_t ld_acc, const float* 
                                   ((unsigned long long)rpp * kUnroll);
         const unsigned long long cap = (unsigned long long)dev.sm_count * 2;  // 64 registers: two blocks per SM
         if (want > cap) want = cap;
-#define QFMT_BLAUNCH(S, C)                                                                                        \
-    bias_quantize_stats_kernel<S, C><<<(unsigned)want, kThreads, smem, stream>>>(                                 \
-        acc, (long long)ld_acc, bias, out, (long long)ld_out, (unsigned long long)rows, c4, cw, rpp, p, d_stats)
-        if (has_stats) { if (has_scale) QFMT_BLAUNCH(true, true); else QFMT_BLAUNCH(true, false); }
-        else { if (has_scale) QFMT_BLAUNCH(false, true); else QFMT_BLAUNCH(false, false); }
+#define QFMT_BLAUNCH(S, C, P)                                                                                     \
+    bias_quantize_stats_kernel<S, C, P><<<(unsigned)want, kThreads, smem, stream>>>(                              \
+        acc, (long long)ld_acc, bias, out, (long long)ld_out, (unsigned long long)rows, c4, cw, rpp, p, d_stats, sign_shift)
+#define QFMT_BLAUNCH2(S, C) do { if (pack) QFMT_BLAUNCH(S, C, true); else QFMT_BLAUNCH(S, C, false); } while (0)
+        if (has_stats) { if (has_scale) QFMT_BLAUNCH2(true, true); else QFMT_BLAUNCH2(true, false); }
+        else { if (has_scale) QFMT_BLAUNCH2(false, true); else QFMT_BLAUNCH2(false, false); }
+#undef QFMT_BLAUNCH2
 #undef QFMT_BLAUNCH
     } else {
         unsigned long long want = (n + kThreads - 1) / kThreads;
         const unsigned long long cap = (unsigned long long)dev.sm_count * 4;
         if (want > cap) want = cap;
-#define QFMT_BSLAUNCH(S, C)                                                                                        \
-    bias_quantize_stats_scalar_kernel<S, C><<<(unsigned)want, kThreads, hist_bytes, stream>>>(                     \
-        acc, (long long)ld_acc, bias, out, (long long)ld_out, (unsigned long long)rows, (unsigned long long)cols, p, d_stats)
-        if (has_stats) { if (has_scale) QFMT_BSLAUNCH(true, true); else QFMT_BSLAUNCH(true, false); }
-        else { if (has_scale) QFMT_BSLAUNCH(false, true); else QFMT_BSLAUNCH(false, false); }
+#define QFMT_BSLAUNCH(S, C, P)                                                                                     \
+    bias_quantize_stats_scalar_kernel<S, C, P><<<(unsigned)want, kThreads, hist_bytes, stream>>>(                  \
+        acc, (long long)ld_acc, bias, out, (long long)ld_out, (unsigned long long)rows, (unsigned long long)cols, p, d_stats, sign_shift)
+#define QFMT_BSLAUNCH2(S, C) do { if (pack) QFMT_BSLAUNCH(S, C, true); else QFMT_BSLAUNCH(S, C, false); } while (0)
+        if (has_stats) { if (has_scale) QFMT_BSLAUNCH2(true, true); else QFMT_BSLAUNCH2(true, false); }
+        else { if (has_scale) QFMT_BSLAUNCH2(false, true); else QFMT_BSLAUNCH2(false, false); }
+#undef QFMT_BSLAUNCH2
 #undef QFMT_BSLAUNCH
     }
     QFMT_CUDA_TRY(err);
@@ -850,6 +875,13 @@ extern "C" int qfmt_bias_quantize_stats(const float* d_acc, int64_t ld_acc, cons
                                         qfmt_stats_t* d_stats, int accumulate, void* stream) {
     return qfmt::bias_quantize_stats_device(d_acc, ld_acc, d_bias, d_out, ld_out, rows, cols, fmt, d_stats, accumulate,
                                             (cudaStream_t)stream);
+}
+
+extern "C" int qfmt_bias_quantize_stats_pack16(const float* d_acc, int64_t ld_acc, const float* d_bias, uint16_t* d_codes,
+                                               int64_t ld_codes, int64_t rows, int64_t cols, const qfmt_format_t* fmt,
+                                               qfmt_stats_t* d_stats, int accumulate, void* stream) {
+    return qfmt::bias_quantize_stats_device(d_acc, ld_acc, d_bias, d_codes, ld_codes, rows, cols, fmt, d_stats, accumulate,
+                                            (cudaStream_t)stream, true);
 }
 
 extern "C" int qfmt_quantize_stats_pack16(const float* d_in, uint16_t* d_codes, size_t n, const qfmt_format_t* fmt,

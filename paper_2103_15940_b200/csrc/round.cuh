@@ -154,6 +154,18 @@ __device__ __forceinline__ uint32_t quantize_pack_one(uint32_t xb, const QuantPa
     return sign | packed;
 }
 
+// Packed code of a value that already lies on the format's grid (container bits q as the rounding
+// functions return them: finite format values, +-inf, or a NaN).
+__device__ __forceinline__ uint32_t encode_container(uint32_t q, const QuantParams& p, int sign_shift) {
+    const int m = 23 - (int)p.drop;
+    const uint32_t a = q & 0x7FFFFFFFu;
+    uint32_t packed;
+    if (a >= 0x7F800000u) packed = ((uint32_t)p.top << m) | (a > 0x7F800000u ? (1u << (m - 1)) : 0u);
+    else if (a >= p.min_normal) packed = (a - ((uint32_t)p.code_off << 23)) >> p.drop;
+    else packed = __float_as_uint(add_ieee(__uint_as_float(a), __uint_as_float(p.magic))) - p.magic;  // multiple of the quantum
+    return ((q >> 31) << sign_shift) | packed;
+}
+
 // fp32 container of a packed code.
 __device__ __forceinline__ uint32_t unpack_one(uint32_t code, const QuantParams& p, int sign_shift) {
     const int m = 23 - (int)p.drop;

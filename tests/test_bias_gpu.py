@@ -153,6 +153,96 @@ def test_linear_layer_forward_config3_and_config5_shapes():
         assert np.array_equal(st.cpu().numpy().view(np.uint64), st_ref)
 
 
+def run_gpu_pack(acc, bias, e, m, den, scale, *, ld_acc=None, ld_codes=None, off=0, want_stats=True):
+    rows, cols = acc.shape
+    ld_acc, ld_codes = ld_acc or cols, ld_codes or cols
+    buf_a = torch.full((rows * ld_acc + 64,), 3.0, dtype=torch.float32, device=DEV)
+    d_acc = buf_a[off:off + rows * ld_acc]
+    d_acc.view(rows, ld_acc)[:, :cols].copy_(torch.from_numpy(acc))
+    buf_b = torch.zeros(cols + 64, dtype=torch.float32, device=DEV)
+    d_bias = buf_b[off:off + cols]
+    d_bias.copy_(torch.from_numpy(bias))
+    buf_o = torch.full((rows * ld_codes + 64,), 0x1234, dtype=torch.int16, device=DEV)
+    d_codes = buf_o[off:off + rows * ld_codes]
+    stats_t = torch.full((qf.STATS_WORDS,), 99, dtype=torch.int64, device=DEV) if want_stats else None
+    qf.qfmt_bias_quantize_stats_pack16(d_acc, ld_acc, d_bias, d_codes, ld_codes, rows, cols, qf.make_format(e, m, den, scale),
+                                       stats_t)
+    torch.cuda.synchronize()
+    full = d_codes.view(rows, ld_codes).cpu().numpy().view(np.uint16)
+    assert np.all(full[:, cols:] == 0x1234)                     # padding untouched
+    assert torch.all(buf_o[:off] == 0x1234) and torch.all(buf_o[off + rows * ld_codes:] == 0x1234)
+    return np.ascontiguousarray(full[:, :cols]), (stats_t.cpu().numpy().view(np.uint64) if want_stats else None)
+
+
+def check_pack(acc, bias, e, m, den, scale, **kw):
+    """Codes must be the encoding of the containers the oracle's layer formula gives (packing a
+    tensor that is already rounded loses nothing); the statistics are those of the container pass."""
+    y_ref, st_ref = oracle.bias_quantize_stats(acc, bias, e, m, den, scale)
+    codes_ref, _ = oracle.quantize_stats_pack16(y_ref, e, m, 1, 1.0)
+    codes, st = run_gpu_pack(acc, bias, e, m, den, scale, **kw)
+    assert np.array_equal(codes, codes_ref.reshape(codes.shape))
+    if st is not None:
+        assert np.array_equal(st, st_ref)
+
+
+@pytest.mark.parametrize("e,m", [(5, 10), (6, 9), (8, 7), (4, 3), (7, 8)])
+@pytest.mark.parametrize("den", [1, 0])
+@pytest.mark.parametrize("scale", [1.0, 2.0 ** 8])
+def test_pack16_arbitrary_bit_patterns(e, m, den, scale):
+    rng = np.random.default_rng(340 + e * 31 + m)
+    rows, cols = 531, 132
+    acc = rng.integers(0, 1 << 32, size=rows * cols, dtype=np.uint64).astype(np.uint32)
+    edge = workloads.edge_bit_patterns()
+    acc[:edge.size] = edge
+    bias = rng.integers(0, 1 << 32, size=cols, dtype=np.uint64).astype(np.uint32)
+    bias[:40] = edge[:40]
+    check_pack(acc.view(np.float32).reshape(rows, cols), bias.view(np.float32), e, m, den, scale)
+
+
+@pytest.mark.parametrize("e,m", [(5, 10), (6, 9), (8, 7)])
+def test_pack16_all_codes_come_back(e, m):
+    """acc runs over every finite container of the format with a zero bias: the codes written must
+    be the codes the containers came from."""
+    all_codes = np.arange(1 << 16, dtype=np.uint16)
+    vals = oracle.unpack16(all_codes, e, m)
+    keep = np.isfinite(vals)
+    acc = np.zeros(1 << 16, np.float32)
+    acc[keep] = vals[keep]
+    codes, _ = run_gpu_pack(acc.reshape(256, 256), np.zeros(256, np.float32), e, m, 1, 1.0)
+    got = codes.reshape(-1)
+    neg_zero = all_codes == 0x8000            # -0 + (+0) = +0 in round-to-nearest
+    assert np.array_equal(got[keep & ~neg_zero], all_codes[keep & ~neg_zero])
+    assert got[0x8000] == 0
+
+
+@pytest.mark.parametrize("rows,cols,off,ld_acc,ld_codes", [(0, 8, 0, 8, 8), (5, 0, 0, 4, 4), (1, 1, 0, 1, 1), (3, 5, 0, 5, 7),
+                                                          (129, 36, 0, 36, 36), (129, 36, 0, 40, 44), (129, 36, 1, 36, 36),
+                                                          (129, 36, 2, 36, 38), (1000, 1024, 0, 1024, 1024),
+                                                          (2, 20000, 0, 20000, 20000), (64, 3072, 4, 3072, 3072)])
+def test_pack16_shapes_and_alignment(rows, cols, off, ld_acc, ld_codes):
+    rng = workloads.rng_for(341, rows * 7 + cols + off)
+    acc = workloads.lognormal_tensor(rng, (rows, cols), -6.0, 5.0, p_zero=0.02)
+    bias = workloads.lognormal_tensor(rng, (cols,), -7.0, 4.0, p_zero=0.05)
+    check_pack(acc, bias, 6, 9, 1, 1.0, off=off, ld_acc=ld_acc, ld_codes=ld_codes)
+    check_pack(acc, bias, 8, 7, 0, 1.0, off=off, ld_acc=ld_acc, ld_codes=ld_codes, want_stats=False)
+
+
+def test_pack16_errors():
+    d = torch.ones(64, dtype=torch.float32, device=DEV)
+    c = torch.zeros(64, dtype=torch.int16, device=DEV)
+    with pytest.raises(qf.QfmtError) as ei:
+        qf.qfmt_bias_quantize_stats_pack16(d, 8, d, c, 8, 8, 8, qf.make_format(8, 8))
+    assert ei.value.status == qf.QFMT_ERR_BAD_FORMAT          # 1 + 8 + 8 bits do not fit
+    with pytest.raises(qf.QfmtError) as ei:
+        qf.qfmt_bias_quantize_stats_pack16(d, 8, d, c, 4, 8, 8, qf.make_format(6, 9))
+    assert ei.value.status == qf.QFMT_ERR_BAD_ARG
+    with pytest.raises(qf.QfmtError) as ei:
+        qf.qfmt_bias_quantize_stats_pack16(d, 8, d, None, 8, 8, 8, qf.make_format(6, 9))
+    assert ei.value.status == qf.QFMT_ERR_BAD_ARG
+    torch.cuda.synchronize()
+    assert torch.all(c == 0)
+
+
 def test_errors():
     d = torch.ones(64, dtype=torch.float32, device=DEV)
     with pytest.raises(qf.QfmtError) as ei:
