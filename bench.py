@@ -305,6 +305,20 @@ def epilogue_section(torch, qf, dev, peaks, reps=20):
     ms = statistics.median(time_events(torch, step, reps))
     assert int(st.cpu()[256]) == rows * cols
     achieved = rows * cols * BYTES_PER_ELEMENT / ms / 1e6
+    # the same pass writing packed 16-bit codes: 4 B read + 2 B written per element
+    codes = torch.empty(rows, cols, dtype=torch.int16, device=dev)
+
+    def step_codes():
+        qf.qfmt_bias_quantize_stats_pack16(acc, cols, bias, codes, cols, rows, cols, fmt, st)
+    for _ in range(3):
+        step_codes()
+    ms_codes = statistics.median(time_events(torch, step_codes, reps))
+    codes_gbs = rows * cols * 6 / ms_codes / 1e6
+    to_codes = {"ms": ms_codes, "value": codes_gbs, "unit": "GB/s",
+                "roofline": {"bound": "hbm", "achieved": codes_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                             "frac": codes_gbs / peaks["hbm_gbs"], "traffic": None,
+                             "algorithmic_bytes_per_launch": rows * cols * 6}}
+    del codes
     # the whole forward layer through qfmt_linear_forward: default plan (GEMM, then the pass above in place)
     # and with the epilogue inside the GEMM kernel (K = 1024)
     wb = qf.qfmt_linear_forward_workspace_bytes(a, b)
@@ -331,6 +345,7 @@ def epilogue_section(torch, qf, dev, peaks, reps=20):
               "ms": timings["two_kernels"], "tflops": flops / timings["two_kernels"] / 1e9, "gemm_alone_ms": gemm_ms,
               "epilogue_in_gemm_kernel_ms": timings["in_kernel"]}
     return {"metric": "layer output R(R(acc)+R(B)) + stats GB/s", "value": achieved, "unit": "GB/s", "linear_forward": linear,
+            "to_packed_codes": to_codes,
             "workload": f"config5 FFN-up forward output, {rows} x {cols}, 1/6/9 (268 MB moved per launch, larger than L2)",
             "ms_per_step": ms, "gpu_launches_per_step": 1,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
@@ -763,7 +778,7 @@ def finish(args, world, value, total_ms, n, runs, clocks, e2e, roofline, cpu, ge
 # ncu capture summarised in profiles/quantize_stats_kernel_config2.md (set to None when the kernel changes).
 NCU_TRAFFIC_BYTES_PER_LAUNCH = 268463872 + 218315520
 # the same for the layer-output kernel on the 8192 x 4096 product (profiles/bias_quantize_stats_kernel_config5.md)
-NCU_EPILOGUE_TRAFFIC_BYTES_PER_LAUNCH = 134290688 + 85444352
+NCU_EPILOGUE_TRAFFIC_BYTES_PER_LAUNCH = 134286336 + 86052352
 
 
 def main():
