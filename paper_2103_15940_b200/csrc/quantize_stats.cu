@@ -443,8 +443,8 @@ bias_quantize_stats_kernel(const uint32_t* acc, long long ld_acc, const uint32_t
                         q.z = bias_round_one<kScale>(v[u].z, b.z, p, inf_bits, b2);
                         q.w = bias_round_one<kScale>(v[u].w, b.w, p, inf_bits, b3);
                         if (kPack) {
-                            const uint32_t c0 = encode_container(q.x, p, sign_shift), c1 = encode_container(q.y, p, sign_shift);
-                            const uint32_t c2 = encode_container(q.z, p, sign_shift), c3 = encode_container(q.w, p, sign_shift);
+                            const uint32_t c0 = encode_container(q.x, b0, p, sign_shift), c1 = encode_container(q.y, b1, p, sign_shift);
+                            const uint32_t c2 = encode_container(q.z, b2, p, sign_shift), c3 = encode_container(q.w, b3, p, sign_shift);
                             store_stream(po16 + u * step_o, make_uint2(c0 | (c1 << 16), c2 | (c3 << 16)));
                         } else {
                             store_stream(po + u * step_o, q);

@@ -166,6 +166,17 @@ __device__ __forceinline__ uint32_t encode_container(uint32_t q, const QuantPara
     return ((q >> 31) << sign_shift) | packed;
 }
 
+// The same when the value's bin is known: bins 1 .. top-1 are the stored exponent fields of normal
+// results, which need no case distinction; the sign comes in with one arithmetic shift and a
+// bitwise select.
+__device__ __forceinline__ uint32_t encode_container(uint32_t q, int bin, const QuantParams& p, int sign_shift) {
+    if ((unsigned)(bin - 1) < (unsigned)(p.top - 1)) {
+        const uint32_t packed = ((q & 0x7FFFFFFFu) - ((uint32_t)p.code_off << 23)) >> p.drop;
+        return packed | ((uint32_t)((int32_t)q >> 31) & (1u << sign_shift));
+    }
+    return encode_container(q, p, sign_shift);
+}
+
 // fp32 container of a packed code.
 __device__ __forceinline__ uint32_t unpack_one(uint32_t code, const QuantParams& p, int sign_shift) {
     const int m = 23 - (int)p.drop;
