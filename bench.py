@@ -532,7 +532,9 @@ def gemm16_section(torch, qf, dev, peaks, reps=5):
     dY (1/5/10 as binary16 words, 1/8/7 as bfloat16 words), qfmt_gemm_packed16 contracts them in
     the layouts they are stored in."""
     out = {"metric": "emulated GEMM on packed 16-bit operands TFLOP/s", "unit": "TFLOP/s", "runs": {},
-           "workload": "config5 BERT-large FC stack, one step: 4 layers x fwd/dgrad/wgrad, operands as packed codes"}
+           "workload": "config5 BERT-large FC stack, one step: 4 layers x fwd/dgrad/wgrad, operands as packed codes; "
+                       "whole_step_ms adds the rounding of X, W, dY to codes with statistics, the layer output as codes "
+                       "with statistics and the loss-scale controller (gradient scale 2^16 given by the host)"}
     layers = []
     for layer in range(len(workloads.CONFIG5_LAYERS)):
         c = workloads.config5_layer(layer, step=0)
@@ -570,7 +572,41 @@ def gemm16_section(torch, qf, dev, peaks, reps=5):
         assert qf.qfmt_device_status(ws) == qf.QFMT_OK
         ms = statistics.median(time_events(torch, step, reps))
         tf = flops / ms / 1e9
+        # the whole step with codes as the only stored form: per layer X, W and dY are rounded to codes with
+        # statistics, the forward product gets Y = R(R(XW) + R(B)) written as codes with statistics, the two
+        # gradient products follow; the loss-scale controller reads the gradients' records at the end
+        n_layers = len(layers)
+        rec = torch.zeros(n_layers, 4, qf.STATS_WORDS, dtype=torch.int64, device=dev)
+        grad_rec = torch.zeros(n_layers, qf.STATS_WORDS, dtype=torch.int64, device=dev)
+        state = qf.qfmt_dls_t(2.0 ** 16, 2.0, 0.5, 1.0, 2.0 ** 24, 2000, 0, 0, 0, 0, 0)
+        d_state = torch.from_numpy(np.frombuffer(bytes(state), dtype=np.uint8).copy()).to(dev)
+        extras = []
+        for li, (fp32, grad_scale) in enumerate(layers):
+            d_out = fp32["W"].shape[1]
+            bias = torch.from_numpy(workloads.normal_tensor(workloads.rng_for(4, 2000 + li), (d_out,), 0.02)).to(dev)
+            extras.append((bias, torch.empty(fp32["X"].shape[0], d_out, dtype=torch.int16, device=dev),
+                           qf.make_format(e, m, 1, grad_scale)))
+
+        def whole_step():
+            for li, (fp32, _) in enumerate(layers):
+                bias, y_codes, gfmt = extras[li]
+                (a0, b0, C0, N0, (cX, cW)), (a1, b1, C1, N1, (cG, _)), (a2, b2, C2, N2, _) = jobs[3 * li:3 * li + 3]
+                qf.qfmt_quantize_stats_pack16(fp32["X"], cX, cX.numel(), fmt, rec[li, 0])
+                qf.qfmt_quantize_stats_pack16(fp32["W"], cW, cW.numel(), fmt, rec[li, 1])
+                qf.qfmt_quantize_stats_pack16(fp32["dY"], cG, cG.numel(), gfmt, grad_rec[li])
+                qf.qfmt_gemm_packed16(a0, b0, C0, N0, fmt, ws, ws.numel())
+                qf.qfmt_bias_quantize_stats_pack16(C0, N0, bias, y_codes, N0, C0.shape[0], N0, fmt, rec[li, 3])
+                qf.qfmt_gemm_packed16(a1, b1, C1, N1, fmt, ws, ws.numel())
+                qf.qfmt_gemm_packed16(a2, b2, C2, N2, fmt, ws, ws.numel())
+            qf.qfmt_dls_update(d_state, grad_rec, n_layers)
+        for _ in range(3):
+            whole_step()
+        assert qf.qfmt_device_status(ws) == qf.QFMT_OK
+        whole_ms = statistics.median(time_events(torch, whole_step, reps))
+        del extras
         out["runs"][tag] = {"ms_per_step": ms, "tflops": tf, "rounding_to_codes_ms": pack_ms, "gemms_per_step": len(jobs),
+                            "whole_step_ms": whole_ms, "whole_step_gemm_tflops": flops / whole_ms / 1e9,
+                            "whole_step_launches": 7 * n_layers + 1,
                             "gpu_launches_per_step": len(jobs),
                             "roofline": {"bound": "tensor", "achieved": tf, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
                                          "frac": tf / peaks["bf16_tflops"], "traffic": None,
