@@ -7,7 +7,8 @@ flushed, at loss scales 2^0, 2^8 and 2^15 (18 kernel launches, 8 bytes of algori
 per element and launch).  `value` is the whole-job GB/s with inputs resident in HBM; `e2e` is
 the same metric through the host-buffer entry point (copies inside the timed region).  The
 contraction half of the path is timed in the same run on the BERT-large FC stack (workload
-"config5", one step: 4 layers x fwd/dgrad/wgrad) and reported under `gemm`; the convolution
+"config5", its ten seeded steps: 4 layers x fwd/dgrad/wgrad each, fresh tensors and per-tensor
+statistics every step) and reported under `gemm` and again inside `roofline`; the convolution
 layers of config4 under `conv`, the one-pass layer output R(R(acc)+R(B)) under `epilogue` and the
 FMAC-8 product (Algorithm 1) under `fmac8`.
 
@@ -110,12 +111,12 @@ def nvml_index(local_rank: int) -> int:
 # ------------------------------------------------------------------------------------------------
 # reference arm: the CPU oracle, as it stands, on a bounded sample of the same workload
 # ------------------------------------------------------------------------------------------------
-def oracle_sweep(x: np.ndarray) -> float:
+def oracle_sweep(x: np.ndarray, threads: int = 1) -> float:
     """Runs the 18 sweep configurations on x with the oracle; returns seconds."""
     import oracle
     t0 = time.perf_counter()
     for _, e, m, den, scale in workloads.config2_runs():
-        oracle.quantize_stats(x, e, m, den, scale)
+        oracle.quantize_stats(x, e, m, den, scale, threads=threads)
     return time.perf_counter() - t0
 
 
@@ -169,38 +170,73 @@ def time_events(torch, fn, iters):
     return [a.elapsed_time(b) for a, b in evs]
 
 
-def gemm_section(torch, qf, dev, peaks, reps=5):
-    """One step of the BERT-large FC stack: 12 GEMMs on operands quantized to 1/6/9 on the GPU."""
+def gemm_section(torch, qf, dev, peaks, reps=3, steps=workloads.CONFIG5_STEPS):
+    """The BERT-large FC stack over its ten seeded steps.  Every step has fresh tensors; per step and
+    layer X, W and dY (loss scale 2^16) are rounded to 1/6/9 with a statistics record of their own
+    (accumulate = 0), then the forward, data-gradient and weight-gradient products run: 12 rounding
+    passes and 12 products per step, 120 + 120 over the workload.  Timed twice with CUDA events per
+    step: the whole step, and its products alone (the contraction half of the metric)."""
+    from concurrent.futures import ThreadPoolExecutor
     fmt = qf.make_format(6, 9, 1)
-    jobs, flops, ws_bytes = [], 0.0, 256
-    for layer in range(len(workloads.CONFIG5_LAYERS)):
-        c = workloads.config5_layer(layer, step=0)
-        t = {}
-        for name, scale in (("X", 1.0), ("W", 1.0), ("dY", c["grad_scale"])):
-            d = torch.from_numpy(c[name]).to(dev)
-            qf.qfmt_quantize_stats(d, d, d.numel(), qf.make_format(6, 9, 1, scale))
-            t[name] = d
-        tokens, d_in = c["X"].shape
-        d_out = c["W"].shape[1]
-        for A, ta, B, tb, M, N, K in ((t["X"], False, t["W"], False, tokens, d_out, d_in),
-                                      (t["dY"], False, t["W"], True, tokens, d_in, d_out),
-                                      (t["X"], True, t["dY"], False, d_in, d_out, tokens)):
-            C = torch.empty(M, N, dtype=torch.float32, device=dev)
-            jobs.append((qf.make_matrix(A, ta), qf.make_matrix(B, tb), C, N, (A, B)))
-            ws_bytes = max(ws_bytes, qf.qfmt_gemm_workspace_bytes(jobs[-1][0], jobs[-1][1]))
-            flops += 2.0 * M * N * K
-
+    n_layers = len(workloads.CONFIG5_LAYERS)
+    keys = [(s_, l_) for s_ in range(steps) for l_ in range(n_layers)]
+    with ThreadPoolExecutor(max_workers=min(16, os.cpu_count() or 1)) as pool:   # host-side generation only
+        host = dict(zip(keys, pool.map(lambda k: workloads.config5_layer(k[1], step=k[0]), keys)))
+    grad_fmt = qf.make_format(6, 9, 1, host[(0, 0)]["grad_scale"])
+    raw, q, outs, jobs = {}, {}, [], {}
+    flops_per_step, rounded_bytes_per_step, ws_bytes = 0.0, 0, 256
+    for l_ in range(n_layers):
+        tokens, d_in = host[(0, l_)]["X"].shape
+        d_out = host[(0, l_)]["W"].shape[1]
+        outs.append((torch.empty(tokens, d_out, dtype=torch.float32, device=dev),
+                     torch.empty(tokens, d_in, dtype=torch.float32, device=dev),
+                     torch.empty(d_in, d_out, dtype=torch.float32, device=dev)))
+        flops_per_step += 3 * 2.0 * tokens * d_in * d_out
+    for k in keys:
+        raw[k] = {n_: torch.from_numpy(host[k][n_]).to(dev) for n_ in ("X", "W", "dY")}
+        q[k] = {n_: torch.empty_like(v) for n_, v in raw[k].items()}
+        Y, dX, dW = outs[k[1]]
+        jobs[k] = ((qf.make_matrix(q[k]["X"]), qf.make_matrix(q[k]["W"]), Y, Y.shape[1]),
+                   (qf.make_matrix(q[k]["dY"]), qf.make_matrix(q[k]["W"], True), dX, dX.shape[1]),
+                   (qf.make_matrix(q[k]["X"], True), qf.make_matrix(q[k]["dY"]), dW, dW.shape[1]))
+        for a, b, _, _ in jobs[k]:
+            ws_bytes = max(ws_bytes, qf.qfmt_gemm_workspace_bytes(a, b))
+        if k[0] == 0:
+            rounded_bytes_per_step += BYTES_PER_ELEMENT * sum(v.numel() for v in raw[k].values())
+    sample_A, sample_B = host[(0, 0)]["X"], host[(0, 0)]["W"]
+    del host
     ws = torch.zeros(ws_bytes, dtype=torch.uint8, device=dev)  # the recommended size (split-K partials)
+    records = torch.zeros(steps, n_layers, 3, qf.STATS_WORDS, dtype=torch.int64, device=dev)
 
-    def step():
-        for a, b, C, N, _ in jobs:
-            qf.qfmt_gemm(a, b, C, N, fmt, ws, ws.numel())
+    def rounding(s_):
+        for l_ in range(n_layers):
+            k = (s_, l_)
+            for i, (n_, f) in enumerate((("X", fmt), ("W", fmt), ("dY", grad_fmt))):
+                qf.qfmt_quantize_stats(raw[k][n_], q[k][n_], raw[k][n_].numel(), f, records[s_, l_, i], 0)
 
-    for _ in range(3):
-        step()
+    def products(s_):
+        for l_ in range(n_layers):
+            for a, b, C, ldc in jobs[(s_, l_)]:
+                qf.qfmt_gemm(a, b, C, ldc, fmt, ws, ws.numel())
+
+    def whole(s_):
+        rounding(s_)
+        products(s_)
+
+    for _ in range(2):  # warm-up over the whole workload (also fills the rounded operands)
+        for s_ in range(steps):
+            whole(s_)
     assert qf.qfmt_device_status(ws) == qf.QFMT_OK
-    ms = statistics.median(time_events(torch, step, reps))
-    # library TF32 GEMM on the same box, same run: the measured tensor-pipe denominator
+    rec = records.cpu().numpy().view(np.uint64)
+    for (s_, l_) in keys:
+        for i, n_ in enumerate(("X", "W", "dY")):
+            assert int(rec[s_, l_, i, 256]) == raw[(s_, l_)][n_].numel() == int(rec[s_, l_, i, :256].sum())
+    step_ms = [statistics.median(v) for v in zip(*[[time_events(torch, lambda s_=s_: whole(s_), 1)[0]
+                                                     for s_ in range(steps)] for _ in range(reps)])]
+    gemm_ms = [statistics.median(v) for v in zip(*[[time_events(torch, lambda s_=s_: products(s_), 1)[0]
+                                                     for s_ in range(steps)] for _ in range(reps)])]
+    denormal_fraction_dY = [float(rec[s_, :, 2, 258].sum()) / float(rec[s_, :, 2, 256].sum()) for s_ in range(steps)]
+    # library TF32 GEMM on the same box, same run: a second view of the tensor-pipe denominator
     torch.backends.cuda.matmul.allow_tf32 = True
     a = torch.randn(8192, 8192, device=dev)
     b = torch.randn(8192, 8192, device=dev)
@@ -210,12 +246,13 @@ def gemm_section(torch, qf, dev, peaks, reps=5):
     lib_ms = min(time_events(torch, lambda: torch.matmul(a, b, out=c), 5))
     lib_tf32 = 2.0 * 8192 ** 3 / lib_ms / 1e9
     del a, b, c
-    achieved = flops / ms / 1e9
+    total_gemm_ms, total_step_ms = sum(gemm_ms), sum(step_ms)
+    achieved = steps * flops_per_step / total_gemm_ms / 1e9
     peak = peaks["bf16_tflops"] * (1.1 / 2.25)  # TF32 dense is nominally 1.1/2.25 of bf16 dense
     # the fp64 oracle on this machine's host cores (OpenMP over outputs): 2^18 sampled outputs of the first product
     import oracle
-    a0, b0, _, n0, (A0, B0) = jobs[0]
-    hA, hB = A0.cpu().numpy(), B0.cpu().numpy()
+    hA, _ = oracle.quantize_stats(sample_A, 6, 9, 1, 1.0, want_stats=False)
+    hB, _ = oracle.quantize_stats(sample_B, 6, 9, 1, 1.0, want_stats=False)
     rng = np.random.default_rng(0)
     ii, jj = rng.integers(0, hA.shape[0], size=1 << 18), rng.integers(0, hB.shape[1], size=1 << 18)
     t0 = time.perf_counter()
@@ -223,13 +260,21 @@ def gemm_section(torch, qf, dev, peaks, reps=5):
     cpu_s = time.perf_counter() - t0
     cpu = {"value": 2.0 * ii.size * hA.shape[1] / cpu_s / 1e12, "unit": "TFLOP/s", "cores": os.cpu_count(),
            "kind": "oracle", "seconds": cpu_s,
-           "sample": f"{ii.size} sampled outputs of the {hA.shape[0]} x {hB.shape[1]} x {hA.shape[1]} forward product"}
+           "sample": f"{ii.size} sampled outputs of the {hA.shape[0]} x {hB.shape[1]} x {hA.shape[1]} forward product "
+                     "(step 0, QKV layer), full-K fp64 dot products"}
     return {"metric": "emulated GEMM TFLOP/s", "value": achieved, "unit": "TFLOP/s", "cpu_baseline": cpu,
-            "workload": "config5 BERT-large FC stack, one step: 4 layers x fwd/dgrad/wgrad, 1/6/9",
-            "ms_per_step": ms, "gemms_per_step": len(jobs), "gpu_launches_per_step": len(jobs),
+            "workload": f"config5 BERT-large FC stack, {steps} seeded steps x 4 layers x fwd/dgrad/wgrad, 1/6/9, fresh "
+                        "tensors per step (5.6 GB of operands: larger than L2), per-tensor statistics every step",
+            "steps": steps, "ms_per_step": total_gemm_ms / steps, "per_step_gemm_ms": gemm_ms,
+            "per_step_whole_ms": step_ms, "total_gemm_ms": total_gemm_ms, "total_whole_ms": total_step_ms,
+            "whole_step_gemm_tflops": steps * flops_per_step / total_step_ms / 1e9,
+            "rounding_gbs": steps * rounded_bytes_per_step / max(total_step_ms - total_gemm_ms, 1e-9) / 1e6,
+            "denormal_fraction_of_dY_per_step": denormal_fraction_dY,
+            "gemms_per_step": 3 * n_layers, "gpu_launches_per_step": 6 * n_layers,
             "roofline": {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
                          "frac": achieved / peak, "traffic": None,
                          "peak_source": f"bf16 {peaks['source']} burst x 1.1/2.25 (nominal TF32:bf16 ratio)",
+                         "frac_of_sustained": achieved / (peaks["bf16_tflops_sustained"] * (1.1 / 2.25)),
                          "library_tf32_same_run": lib_tf32, "frac_of_library_tf32": achieved / lib_tf32,
                          "nominal_tf32_dense": 1100.0, "frac_of_nominal": achieved / 1100.0}}
 
@@ -766,13 +811,19 @@ def run_library(args):
     if "conv" in sections:
         conv = conv_section(torch, qf, dev, peaks)
     if "cpu" in sections:
-        # the CPU oracle on this machine's host cores, bounded sample
+        # the CPU oracle on this machine's host cores: one thread on a quarter of the tensor, and every core
+        # (pieces in parallel, records summed) on the whole tensor
         n_cpu = 1 << 24
         cpu_secs = oracle_sweep(x_host[:n_cpu])
         cpu_value = len(runs) * n_cpu * BYTES_PER_ELEMENT / cpu_secs / 1e9
+        cores = os.cpu_count() or 1
+        all_secs = oracle_sweep(x_host, threads=cores)
         cpu = {"value": cpu_value, "unit": UNIT, "cores": 1, "kind": "oracle", "seconds": cpu_secs,
-               "host_cores_available": os.cpu_count(),
-               "sample": f"the 18 sweep runs on the first {n_cpu} of {n} elements"}
+               "host_cores_available": cores,
+               "sample": f"the 18 sweep runs on the first {n_cpu} of {n} elements",
+               "all_cores": {"value": len(runs) * n * BYTES_PER_ELEMENT / all_secs / 1e9, "unit": UNIT, "cores": cores,
+                             "kind": "oracle", "seconds": all_secs,
+                             "sample": f"the 18 sweep runs on all {n} elements, {cores} pieces in parallel"}}
     return finish(args, world, value, total_ms, n, runs, clocks, e2e, roofline, cpu, gemm, conv, dist, extra)
 
 
@@ -805,15 +856,32 @@ def finish(args, world, value, total_ms, n, runs, clocks, e2e, roofline, cpu, ge
             "clocks": clocks.summary(), "e2e": e2e, "gpu_launches": args.steps * len(runs),
             "roofline": roofline, "cpu_baseline": cpu, "gemm": gemm, "conv": conv}
     line.update(extra)
+    # The metric has two halves.  The contraction half (and the other tensor-bound workloads) is repeated
+    # inside `roofline` and `cpu_baseline`, next to the rounding pass's own figures.
+    def brief(section):
+        r = section["roofline"]
+        keep = {k: r[k] for k in ("bound", "achieved", "peak", "unit", "frac", "peak_source", "frac_of_sustained",
+                                  "library_tf32_same_run", "frac_of_library_tf32", "frac_of_nominal") if k in r}
+        keep["workload"] = section["workload"]
+        return keep
+    if gemm is not None:
+        roofline["gemm"] = brief(gemm)
+        if cpu is not None:
+            cpu["gemm"] = gemm["cpu_baseline"]
+    if conv is not None:
+        roofline["conv"] = brief(conv)
+    if "config3" in line:
+        roofline["config3"] = brief(line["config3"])
     print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the quantize+stats kernel, from the
-# ncu capture summarised in profiles/quantize_stats_kernel_config2.md (set to None when the kernel changes).
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the quantize+stats kernel on the 64 Mi-element
+# tensor, from one ncu capture of that kernel (read + write).  A figure here belongs to the kernel as it was
+# when the counters were taken: it is set to None as soon as that kernel's code changes, until re-taken.
 NCU_TRAFFIC_BYTES_PER_LAUNCH = 268463872 + 218315520
-# the same for the layer-output kernel on the 8192 x 4096 product (profiles/bias_quantize_stats_kernel_config5.md)
+# the same for the layer-output kernel on the 8192 x 4096 product
 NCU_EPILOGUE_TRAFFIC_BYTES_PER_LAUNCH = 134286336 + 86052352
 
 

@@ -376,6 +376,14 @@ size_t qfmt_gemm_packed16_workspace_bytes(const qfmt_matrix16_t* A, const qfmt_m
  * again after changing it.  Returns QFMT_ERR_BAD_ARG for other values.
  */
 int qfmt_gemm_tile_policy(int policy);
+/*
+ * The same for the forward and data-gradient products of qfmt_conv (filters larger than 1 x 1):
+ *   0  automatic (default): CTA pairs, each CTA one M-tile of whole image rows and half of the filter
+ *      columns, whenever there are two or more M-tiles
+ *   1  always the single-CTA kernel
+ * Ask qfmt_conv_workspace_bytes again after changing it.
+ */
+int qfmt_conv_tile_policy(int policy);
 
 /*
  * Convolution layers (Section V: "matrix multiplications, at the core of fully connected and
@@ -427,8 +435,13 @@ size_t qfmt_conv_workspace_bytes(int32_t op, const qfmt_conv_t* geom);  /* 0 if 
  *                 (QFMT_OK or QFMT_ERR_TIMEOUT) is copied there on `stream` after the product;
  *                 read it with qfmt_device_status(d_status_out, stream) or your own copy.
  * Limits and rules
- *   - A problem for which qfmt_gemm_workspace_bytes(A, B) exceeds 16 MiB is refused with
- *     QFMT_ERR_SCRATCH_LIMIT and nothing is enqueued; use qfmt_gemm with your own workspace.
+ *   - A problem for which qfmt_gemm_workspace_bytes(A, B) exceeds 16 MiB (16 777 216 bytes) is
+ *     refused with QFMT_ERR_SCRATCH_LIMIT and nothing is enqueued; use qfmt_gemm with your own
+ *     workspace.  That figure counts the whole workspace: the 256-byte header that holds the
+ *     status word as well as the partial sums of a product whose K dimension is split, so a
+ *     product whose partial sums take exactly 16 MiB (1024 x 1024 outputs in four splits, say) is
+ *     refused by those 256 bytes.  All argument checks of qfmt_gemm run before anything is
+ *     enqueued, so every error return of this call leaves the stream untouched.
  *   - The first call on each GPU looks up the array's device address (a query, not an
  *     allocation).  Make that first call during set-up, before any stream capture begins.
  *   - All calls on one GPU share the one array and it keeps whatever the previous call left.
@@ -439,6 +452,21 @@ size_t qfmt_conv_workspace_bytes(int32_t op, const qfmt_conv_t* geom);  /* 0 if 
  */
 int qfmt_gemm_builtin_scratch(const qfmt_matrix_t* A, const qfmt_matrix_t* B, float* d_C, int64_t ldc,
                               const qfmt_format_t* fmt, int32_t* d_status_out, void* stream);
+
+/*
+ * Self-test of the error path the contraction kernels take when a device-side wait does not end
+ * (every wait in them is bounded; see QFMT_ERR_TIMEOUT).  Launches one small block that waits, with
+ * the same primitives, on a barrier nothing ever arrives on; the wait gives up after
+ * `limit_cycles` SM cycles (1 .. 2^24, i.e. at most a few milliseconds), the block records
+ * QFMT_ERR_TIMEOUT in *d_status exactly as a contraction kernel would, its other warp notices the
+ * block-wide abort flag, and the kernel returns normally: the context stays usable.
+ *   d_status  device, 4-byte aligned: receives QFMT_ERR_TIMEOUT (cleared first); read it with
+ *             qfmt_device_status(d_status, stream)
+ *   d_trace   device, four int32: [0] = 1 the waiting warp saw its wait expire, [1] = 1 the other warp
+ *             left because of the abort flag, [2] = cycles waited, [3] unused
+ * The paper has no counterpart; this is a diagnostic of the library.
+ */
+int qfmt_selftest_bounded_wait(int32_t* d_status, uint32_t limit_cycles, int32_t* d_trace, void* stream);
 
 /*
  * Synchronises `stream` and returns the status word of a workspace: QFMT_OK, or the error a

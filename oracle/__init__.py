@@ -55,6 +55,8 @@ def _L() -> ctypes.CDLL:
         lib.oracle_encode_code.restype = u32
         lib.oracle_quantize_stats.argtypes = [vp, vp, sz, i32, i32, i32, u32, vp]
         lib.oracle_quantize_stats.restype = None
+        lib.oracle_quantize_stats_threads.argtypes = [vp, vp, sz, i32, i32, i32, u32, vp, i32]
+        lib.oracle_quantize_stats_threads.restype = None
         lib.oracle_gemm.argtypes = [vp, i64, i32, vp, i64, i32, i64, i64, i64, vp, vp]
         lib.oracle_gemm.restype = None
         lib.oracle_gemm_sampled.argtypes = [vp, i64, i32, vp, i64, i32, i64, vp, vp, i64, vp, vp]
@@ -138,15 +140,19 @@ def fmac_bits(abits: int, xbits: int, ybits: int, e: int, m: int, denormals: int
 
 # ---- tensors ----------------------------------------------------------------------------------
 def quantize_stats(x: np.ndarray, e: int, m: int, denormals: int = 1, loss_scale: float = 1.0,
-                   want_q: bool = True, want_stats: bool = True):
-    """Returns (q as float32 array shaped like x or None, stats as uint64[264] or None)."""
+                   want_q: bool = True, want_stats: bool = True, threads: int = 1):
+    """Returns (q as float32 array shaped like x or None, stats as uint64[264] or None).
+    threads > 1 cuts the tensor into that many pieces handled in parallel (records summed)."""
     xf = np.ascontiguousarray(x, dtype=np.float32)
     xb = xf.view(np.uint32).reshape(-1)
     q = np.empty_like(xb) if want_q else None
     st = np.zeros(STATS_WORDS, dtype=np.uint64) if want_stats else None
-    _L().oracle_quantize_stats(xb.ctypes.data, q.ctypes.data if want_q else None, xb.size, e, m,
-                               int(denormals), _f32_bits(loss_scale),
-                               st.ctypes.data if want_stats else None)
+    args = (xb.ctypes.data, q.ctypes.data if want_q else None, xb.size, e, m, int(denormals), _f32_bits(loss_scale),
+            st.ctypes.data if want_stats else None)
+    if threads > 1:
+        _L().oracle_quantize_stats_threads(*args, int(threads))
+    else:
+        _L().oracle_quantize_stats(*args)
     return (q.view(np.float32).reshape(xf.shape) if want_q else None), st
 
 

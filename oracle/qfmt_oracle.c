@@ -272,6 +272,28 @@ void oracle_quantize_stats(const uint32_t *x, uint32_t *q, size_t n, int e, int 
     }
 }
 
+/*
+ * The same over `threads` host threads: the tensor is cut into that many contiguous pieces, each
+ * piece is handled by oracle_quantize_stats with a record of its own, and the records are summed
+ * at the end (elements are independent and counts add).  For timing the oracle on all cores.
+ */
+void oracle_quantize_stats_threads(const uint32_t *x, uint32_t *q, size_t n, int e, int m, int keep_denormals,
+                                   uint32_t scale_bits, uint64_t *stats, int threads) {
+    if (threads < 1) threads = 1;
+#pragma omp parallel for schedule(static) num_threads(threads)
+    for (int t = 0; t < threads; ++t) {
+        size_t lo = n / (size_t)threads * (size_t)t, hi = (t == threads - 1) ? n : n / (size_t)threads * (size_t)(t + 1);
+        uint64_t local[ST_WORDS];
+        memset(local, 0, sizeof local);
+        oracle_quantize_stats(x + lo, q ? q + lo : NULL, hi - lo, e, m, keep_denormals, scale_bits,
+                              stats ? local : NULL);
+        if (stats) {
+#pragma omp critical
+            for (int w = 0; w < ST_WORDS; ++w) stats[w] += local[w];
+        }
+    }
+}
+
 /* ------------------------------------------------------------------------------------------ */
 /* 16-bit storage (Section II: activations and gradients are kept in half precision, halving     */
 /* storage and bandwidth): a tensor is rounded as oracle_quantize_stats does and each value is    */
@@ -588,31 +610,37 @@ void oracle_gemm_sampled(const float *A, int64_t lda, int transA, const float *B
 }
 
 /* ------------------------------------------------------------------------------------------ */
-/* FMAC-8 (Algorithm 1): dot product with a format-precision accumulator that is emptied into   */
-/* a single-precision master accumulator before every eighth FMAC, and once more at the end;    */
-/* the result is rounded to the format.  "+" on the master accumulator is fp32 addition.        */
+/* FMAC-8 (Algorithm 1).  A dot product is cut, from its start, into runs of `group` consecutive  */
+/* terms (8 in the paper; the last run may be shorter).  Each run is summed by fused multiply-    */
+/* accumulates into an accumulator of the 16-bit format that starts at zero, every FMAC rounding   */
+/* its exact a + x*y once to the format; the finished run sum is then added, in fp32 arithmetic,  */
+/* to a single-precision total that also starts at zero.  The total is rounded to the format at   */
+/* the end.  An empty dot product gives R(+0).                                                     */
 /* ------------------------------------------------------------------------------------------ */
 static uint32_t f32_add_bits(uint32_t a, uint32_t b) { return oracle_add_round_bits(a, b, 8, 23, 1); }
 
+static uint32_t word_of(float v) {
+    uint32_t w;
+    memcpy(&w, &v, 4);
+    return w;
+}
+
 static uint32_t fmac8_dot(const float *A, int64_t lda, int transA, const float *B, int64_t ldb, int transB,
                           int64_t K, int64_t i, int64_t j, int e, int m, int keep_denormals, int group,
-                          uint32_t *master_out) {
-    uint32_t master = 0, small = 0; /* A^(32) = 0, a^(16) = 0 */
-    for (int64_t k = 0; k < K; ++k) {
-        if (k % group == 0) {
-            master = f32_add_bits(master, small);
-            small = 0;
+                          uint32_t *total_out) {
+    uint32_t total = 0; /* fp32 word of +0 */
+    for (int64_t first = 0; first < K; first += group) {
+        const int64_t end = first + group < K ? first + group : K;
+        uint32_t run_sum = 0; /* format value +0, kept as its fp32 word */
+        for (int64_t k = first; k < end; ++k) {
+            const float x = transA ? A[k * lda + i] : A[i * lda + k];
+            const float y = transB ? B[j * ldb + k] : B[k * ldb + j];
+            run_sum = oracle_fmac_bits(run_sum, word_of(x), word_of(y), e, m, keep_denormals);
         }
-        float x = transA ? A[k * lda + i] : A[i * lda + k];
-        float y = transB ? B[j * ldb + k] : B[k * ldb + j];
-        uint32_t xb, yb;
-        memcpy(&xb, &x, 4);
-        memcpy(&yb, &y, 4);
-        small = oracle_fmac_bits(small, xb, yb, e, m, keep_denormals);
+        total = f32_add_bits(total, run_sum);
     }
-    master = f32_add_bits(master, small);
-    if (master_out) *master_out = master; /* A^(32) before the final rounding */
-    return oracle_quantize_bits(master, e, m, keep_denormals, NULL);
+    if (total_out) *total_out = total; /* the single-precision total before the final rounding */
+    return oracle_quantize_bits(total, e, m, keep_denormals, NULL);
 }
 
 /* C (M x N, dense row-major fp32 words) = FMAC-8 product of op(A) (M x K) and op(B) (K x N).   */

@@ -134,6 +134,8 @@ def _bind_optional(L: ctypes.CDLL) -> None:
     L.qfmt_linear_forward_workspace_bytes.restype = sz
     L.qfmt_gemm_tile_policy.argtypes = [ci]
     L.qfmt_gemm_tile_policy.restype = ci
+    L.qfmt_conv_tile_policy.argtypes = [ci]
+    L.qfmt_conv_tile_policy.restype = ci
     L.qfmt_device_status.argtypes = [vp, vp]
     L.qfmt_device_status.restype = ci
     convp = ctypes.POINTER(qfmt_conv_t)
@@ -143,6 +145,8 @@ def _bind_optional(L: ctypes.CDLL) -> None:
     L.qfmt_conv_workspace_bytes.restype = sz
     L.qfmt_gemm_builtin_scratch.argtypes = [matp, matp, vp, ctypes.c_int64, ctypes.POINTER(qfmt_format_t), vp, vp]
     L.qfmt_gemm_builtin_scratch.restype = ci
+    L.qfmt_selftest_bounded_wait.argtypes = [vp, ctypes.c_uint32, vp, vp]
+    L.qfmt_selftest_bounded_wait.restype = ci
 
 
 def _ptr(x) -> Optional[int]:
@@ -325,6 +329,12 @@ def qfmt_gemm_builtin_scratch(A: qfmt_matrix_t, B: qfmt_matrix_t, d_C, ldc: int,
                                            _ptr(d_status_out), _stream_handle(stream)), "qfmt_gemm_builtin_scratch")
 
 
+def qfmt_selftest_bounded_wait(d_status, limit_cycles: int, d_trace, stream=None) -> None:
+    """Runs the library's bounded-wait self-test kernel; see qfmt_selftest_bounded_wait in include/qfmt.h."""
+    _check(lib().qfmt_selftest_bounded_wait(_ptr(d_status), int(limit_cycles), _ptr(d_trace), _stream_handle(stream)),
+           "qfmt_selftest_bounded_wait")
+
+
 def qfmt_conv_workspace_bytes(op: int, geom: qfmt_conv_t) -> int:
     return int(lib().qfmt_conv_workspace_bytes(int(op), ctypes.byref(geom)))
 
@@ -335,6 +345,11 @@ def qfmt_conv(op: int, geom: qfmt_conv_t, d_p, d_q, d_out, fmt: qfmt_format_t, d
     see qfmt_conv in include/qfmt.h."""
     _check(lib().qfmt_conv(int(op), ctypes.byref(geom), _ptr(d_p), _ptr(d_q), _ptr(d_out), ctypes.byref(fmt),
                            _ptr(d_workspace), int(workspace_bytes), _stream_handle(stream)), "qfmt_conv")
+
+
+def qfmt_conv_tile_policy(policy: int) -> None:
+    """0 automatic (CTA pairs), 1 single-CTA kernel for conv forward / data gradient; see include/qfmt.h."""
+    _check(lib().qfmt_conv_tile_policy(int(policy)), "qfmt_conv_tile_policy")
 
 
 def qfmt_gemm_tile_policy(policy: int) -> None:

@@ -87,6 +87,7 @@ struct GemmParams {
     int b_mn_major;  // op(B) stored with N contiguous
     int tiles_m, tiles_n;
     int tma_store;   // C base, row pitch and row length are multiples of 16 bytes: C is written by TMA
+    int c_blocked;   // pair kernel: N is a multiple of 32 and the C map is {32, rows, N / 32, splits}
     // Balanced schedule (mode 1 only, sk_cpt > 0).  The tiles' 64-element K chunks form one sequence,
     // tile after tile, and CTA b works on the b-th of gridDim.x equal ranges of it: up to sk_pieces
     // consecutive tiles, the first and the last possibly in part.  A piece that begins inside a tile
@@ -95,6 +96,16 @@ struct GemmParams {
     int sk_cpt;              // chunks per tile, 0 = schedule off
     int sk_pieces;           // pieces a CTA may have
     float* sk_partials;
+    // The same schedule in the pair kernel (sk_flags != nullptr), dealt among the CTA pairs, without the
+    // slots and without the second kernel.  A pair runs the piece that begins inside a tile LAST and adds
+    // it into C at the destination; by then the pair before it, whose range ends inside that tile, has
+    // written the tile's first part as the last-but-one piece of its own range and has said so in
+    // sk_flags ([pair][2 CTAs x 8 accumulate warps] words, zeroed before the launch; a word covers the
+    // 32 x 128 patch of the tile that the same warp of both pairs owns).  A tile has at most two pieces
+    // (ranges are at least a tile long), the first stored and the second added after it in program
+    // order of a flag hand-over, so the sums are the same on every run.
+    int* sk_flags;
+    int sk_q, sk_r;          // quotient and remainder of (tiles * sk_cpt) / pairs
     int wg_padded;   // filter gradient, padded stages: an image row takes a power-of-two number of K rows
                      // (the copy engine zero-fills the columns past the image), a stage is 32 K rows
                      // exactly, and one rank-5 copy per operand brings all of its channel blocks
@@ -118,6 +129,7 @@ struct GemmParams {
     int cblocks, ck;       // mode 1: 32-channel blocks per tap and contraction channels; mode 2: ck = C_in
     int tap_sign, off_h, off_w;  // activation row read for tap (r, s): h + tap_sign * r + off_h
     int full_tiles_m;      // mode 1: M-tiles that are complete (the C tensor map covers exactly these)
+    int conv_rows;         // mode 1 on CTA pairs: pixels (rows of C) in one CTA's M-tile
     // ---- layer-output epilogue (dense mode, one summation group, no split K): the sums are rounded,
     // the rounded bias of their column is added, the result is rounded again and counted, all in the
     // accumulate warps' registers before the tile is stored
@@ -139,16 +151,69 @@ struct RowMaps {
 struct WorkItem {
     int tile_m, tile_n, split, m0, n0, kb_begin, num_kb;
     int partial;  // balanced schedule: the piece begins inside its tile and goes to the CTA's slot
+    int head;     // balanced schedule of the pair kernel: the next pair adds the rest of this tile
 };
+// Piece j (in the order a pair runs them) of pair `unit` under the balanced schedule of the pair
+// kernel: the pieces of the pair's chunk range in their natural order, except that a first piece that
+// begins inside a tile moves to the end.  `head`: the piece begins its tile and ends before the tile
+// does (the next pair finishes it).  `partial`: the piece begins inside its tile.
+struct PairPiece {
+    int tile, kb_begin, num_kb, partial, head;
+};
+// Range boundaries come from the quotient q and remainder r of total / units, so that everything
+// stays in 32 bits: lo(u) = q * u + r * u / units (total < 2^31, units < 2^15).
+__host__ __device__ __forceinline__ PairPiece pair_piece(int q, int r, int cpt, int kb_total, int units, int unit, int j) {
+    PairPiece pc = {0, 0, 0, 0, 0};
+    const int lo = q * unit + r * unit / units, hi = q * (unit + 1) + r * (unit + 1) / units;
+    if (hi <= lo) return pc;
+    const int first_tile = lo / cpt, last_tile = (hi - 1) / cpt;
+    const int n_nat = last_tile - first_tile + 1;
+    const bool first_partial = lo > first_tile * cpt;
+    int nat = j;
+    if (first_partial) nat = j + 1 < n_nat ? j + 1 : (j + 1 == n_nat ? 0 : n_nat);
+    if (nat >= n_nat) return pc;
+    const int tile = first_tile + nat, first = tile * cpt;
+    const int s = lo > first ? lo : first, e = hi < first + cpt ? hi : first + cpt;
+    pc.tile = tile;
+    pc.kb_begin = (s - first) * kChunkKB;
+    const int kb_end = (e - first) * kChunkKB < kb_total ? (e - first) * kChunkKB : kb_total;
+    pc.num_kb = kb_end - pc.kb_begin;
+    pc.partial = s > first ? 1 : 0;
+    pc.head = e < first + cpt ? 1 : 0;
+    return pc;
+}
+
 // Chunk range [lo, hi) of CTA b under the balanced schedule.
 __host__ __device__ __forceinline__ void sk_range(long long total, int ctas, int b, long long* lo, long long* hi) {
     *lo = total * b / ctas;
     *hi = total * (b + 1) / ctas;
 }
+// Balanced schedule of the pair kernel: t = pair + piece * pairs.  Kept out of line: it runs once per
+// piece, and inlined into the producer's, the issuers' and the accumulate warps' loops it cost them
+// registers they need (measured: every product 12 % slower).
+__device__ __noinline__ int4 decode_work_pairs(int q, int r, int cpt, int kb_total, int t) {
+    const int units = (int)(gridDim.x >> 1);
+    const PairPiece pc = pair_piece(q, r, cpt, kb_total, units, t % units, t / units);
+    return make_int4(pc.tile, pc.kb_begin, pc.num_kb, pc.partial | (pc.head << 1));
+}
 __device__ __forceinline__ WorkItem decode_work(const GemmParams& p, int t) {
     WorkItem w;
     const int num_tiles = p.tiles_m * p.tiles_n;
     w.partial = 0;
+    w.head = 0;
+    if (p.sk_flags != nullptr) {
+        const int4 pc = decode_work_pairs(p.sk_q, p.sk_r, p.sk_cpt, p.kb_total, t);
+        w.split = 0;
+        w.tile_m = pc.x % p.tiles_m;
+        w.tile_n = pc.x / p.tiles_m;
+        w.m0 = w.tile_m * p.tile_rows;
+        w.n0 = w.tile_n * kBN;
+        w.kb_begin = pc.y;
+        w.num_kb = pc.z;
+        w.partial = pc.w & 1;
+        w.head = pc.w >> 1;
+        return w;
+    }
     if (p.sk_cpt > 0) {
         // t = b + piece * gridDim.x for CTA b
         const int ctas = (int)gridDim.x, b = t % ctas, piece = t / ctas;
@@ -212,9 +277,60 @@ __device__ __forceinline__ uint32_t make_idesc(int a_mn, int b_mn) {
            | ((uint32_t)(kBN >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
 }
 
-__device__ __forceinline__ void raise_timeout(const GemmParams& p, volatile int* abort_flag) {
+// What a role does when one of its bounded waits runs out: the CTA-wide flag tells the other roles
+// to stop at their next check, the status word (first error wins) tells the host.
+__device__ __forceinline__ void raise_timeout(int* status, volatile int* abort_flag) {
     *abort_flag = 1;
-    atomicCAS(p.status, 0, (int)QFMT_ERR_TIMEOUT);
+    atomicCAS(status, 0, (int)QFMT_ERR_TIMEOUT);
+}
+__device__ __forceinline__ void raise_timeout(const GemmParams& p, volatile int* abort_flag) {
+    raise_timeout(p.status, abort_flag);
+}
+
+// Self-test of the bounded-wait path with the primitives the GEMM kernels use, on a barrier that
+// nothing ever arrives on.  Warp 0 plays a role whose wait runs out after `limit` cycles: it must
+// come back from mbar_wait_bounded with false and raise the timeout.  Warp 1 plays a role that is
+// not itself stuck: it polls the abort flag (itself bounded, at 64 limits) and leaves when the flag
+// is up.  Both meet at the common exit and the kernel returns normally; nothing can spin forever.
+// trace[0] = 1 if warp 0's wait returned false, trace[1] = 1 if warp 1 left because of the flag,
+// trace[2] = cycles warp 0 waited.
+__global__ void __launch_bounds__(64, 1)
+bounded_wait_selftest_kernel(int* status, uint32_t limit, int* trace) {
+    __shared__ __align__(8) unsigned long long bar_storage;
+    __shared__ int abort_word;
+    volatile int* abort_flag = &abort_word;
+    const uint32_t bar = ptx::smem_addr(&bar_storage);
+    if (threadIdx.x == 0) {
+        ptx::mbar_init(bar, 1);
+        *abort_flag = 0;
+        ptx::fence_mbar_init();
+    }
+    __syncthreads();
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (warp == 0) {
+        if (lane == 0) {
+            const long long t0 = clock64();
+            const bool ok = ptx::mbar_wait_bounded(bar, 0u, limit);  // phase 0 never completes
+            trace[2] = (int)(clock64() - t0);
+            if (!ok) {
+                raise_timeout(status, abort_flag);
+                trace[0] = 1;
+            }
+        }
+        __syncwarp();
+    } else {
+        if (lane == 0) {
+            const long long t0 = clock64();
+            int saw = 0;
+            while (clock64() - t0 < 64ll * (long long)limit) {
+                if (*abort_flag) { saw = 1; break; }
+                __nanosleep(64);
+            }
+            trace[1] = saw;
+        }
+        __syncwarp();
+    }
+    __syncthreads();
 }
 
 // Layer-output epilogue on one thread's 128 sums of a row (columns col_base + 0..127; sum2[i] holds
@@ -714,11 +830,32 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
 //   acc_empty[b] (leader's) sixteen arrivals: the eight accumulate warps of both CTAs
 // The three-level summation and the output path are those of the single-CTA kernel.
 // ------------------------------------------------------------------------------------------------
-constexpr int kPStages = 5;
+#ifndef QFMT_PSTAGES
+#define QFMT_PSTAGES 5
+#endif
+#ifndef QFMT_POUT_BLOCKS
+#define QFMT_POUT_BLOCKS 2
+#endif
+constexpr int kPStages = QFMT_PSTAGES;
 constexpr uint32_t kPABytes = kBM * kBK * 4;          // 128 rows of A
 constexpr uint32_t kPBBytes = (kBN / 2) * kBK * 4;    // 128 of the tile's 256 columns of B
 constexpr uint32_t kPStageBytes = kPABytes + kPBBytes;
-constexpr uint32_t kPairSmemBytes = kPStages * kPStageBytes + kOutBytes + 1024 + 256 + kEpiHistBytes;
+// Output staging of the pair kernel.  When N is a multiple of 32, C is described to the copy engine as
+// {32 columns, rows, N / 32 column blocks, splits}, and one copy moves kPOutBlocks 32 x 32 blocks of a
+// warp's 32 x 128 patch: with kPOutBlocks = 4 the whole patch is staged at once (16 KB per warp) and a
+// flush costs the copy engine eight instructions per CTA instead of thirty-two.
+constexpr int kPOutBlocks = QFMT_POUT_BLOCKS;
+constexpr uint32_t kPOutWarpBytes = (kPOutBlocks * kOutBoxBytes > kOutWarpBytes) ? kPOutBlocks * kOutBoxBytes : kOutWarpBytes;
+constexpr uint32_t kPOutBytes = kAccWarps * kPOutWarpBytes;
+constexpr uint32_t kPairSmemBytes = kPStages * kPStageBytes + kPOutBytes + 1024 + 256 + kEpiHistBytes;
+static_assert(kPairSmemBytes <= 232448, "pair kernel: shared memory");
+// The two MMA issuers of the pair kernel tell a stage's phases apart without a progress word only
+// when the ring has at least four stages (see the issuer's comment); three stages gave wrong sums.
+static_assert(kPStages >= 4, "pair kernel: at least four stages");
+// kPOutBlocks = 3: three blocks go through the staging area in one copy and the fourth is written from
+// the registers (the staging area for all four does not fit beside four stages, and waiting for the
+// copy engine to have read a smaller area before refilling it costs ~2 k cycles per flush).
+static_assert(4 % kPOutBlocks == 0 || kPOutBlocks == 3, "pair kernel: a warp's four column blocks");
 
 // Operand kinds of the pair kernel: fp32 containers read as TF32, or packed 16-bit codes that are
 // binary16 (1/5/10) or bfloat16 (1/8/7) words.  A stage is one 128-byte swizzle row per operand row
@@ -730,15 +867,19 @@ __device__ __forceinline__ uint32_t make_idesc_pair(int a_mn, int b_mn, int kind
            | ((uint32_t)(kBN >> 3) << 17) | ((uint32_t)((2 * kBM) >> 4) << 24);
 }
 
-template <bool kEpi, int kKind>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
-gemm_tf32_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
-                      const __grid_constant__ CUtensorMap tmap_c, const GemmParams p) {
+// kMode 0: dense operands.  kMode 1: forward / data gradient of a convolution (see conv_device): each
+// CTA of the pair owns one M-tile of whole image rows (p.rows_per_blk rows, p.conv_rows pixels) and
+// half of the 256 filter columns; its pixel operand arrives as one box per image touched from
+// row_maps, C is written through tmap_c ({32, conv_rows, N / 32, complete tiles}: rows past the tile
+// are clipped) or, for the incomplete last tile, tmap_c2.
+template <bool kEpi, int kKind, int kMode>
+__device__ __forceinline__ void pair_body(const CUtensorMap& tmap_a, const CUtensorMap& tmap_b, const CUtensorMap& tmap_c,
+                                          const CUtensorMap* tmap_c2, const CUtensorMap* row_maps, const GemmParams& p) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = ptx::smem_addr(smem_raw);
     const uint32_t tiles = (raw + 1023u) & ~1023u;
     const uint32_t out_stage = tiles + kPStages * kPStageBytes;
-    const uint32_t bars = out_stage + kOutBytes;
+    const uint32_t bars = out_stage + kPOutBytes;
     auto full_bar = [&](int s) { return bars + 8u * s; };
     auto empty_bar = [&](int s) { return bars + 8u * (kPStages + s); };
     auto acc_full_bar = [&](int a) { return bars + 8u * (2 * kPStages + a); };
@@ -780,10 +921,10 @@ gemm_tf32_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
     ptx::cluster_sync();  // the peer's barriers exist before anything is signalled to them
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
-    const int num_work = p.tiles_m * p.tiles_n * p.splits;
+    const int num_work = p.sk_flags != nullptr ? p.sk_pieces * num_clusters : p.tiles_m * p.tiles_n * p.splits;
 
     if (warp < 4) {
-    ptx::setmaxnreg_dec<80>();
+    ptx::setmaxnreg_dec<56>();
     if (warp == 0) {
         // ------------------------------ TMA producer (both CTAs) ------------------------------
         if (lane == 0) {
@@ -801,6 +942,30 @@ gemm_tf32_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
                     const uint32_t sb = sa + kPABytes;
                     const uint32_t bar = ptx::map_to_cta(full_bar(stage), 0);  // the leader's barrier
                     const int k0 = kb * (kKind == kKindTf32 ? kBK : 2 * kBK);
+                    if (kMode == 1) {
+                        ptx::mbar_expect_tx_cluster(bar, p.a_bytes + kPBBytes);
+                        // A: this CTA's image rows at the tap's offset, one box per image touched (rows and
+                        // columns outside the image, and images past the batch, read as zero)
+                        const int tap = kb / p.cblocks, cb = kb % p.cblocks;
+                        const int dh = p.tap_sign * (tap / p.taps_s) + p.off_h;
+                        const int dw = p.tap_sign * (tap % p.taps_s) + p.off_w;
+                        const int ctile = 2 * w.tile_m + (int)rank;
+                        int j = 0;
+                        while (j < p.rows_per_blk) {
+                            const int q = ctile * p.rows_per_blk + j;
+                            const int h = q % p.img_rows, img = q / p.img_rows;
+                            int cnt = p.rows_per_blk - j;
+                            if (cnt > p.img_rows - h) cnt = p.img_rows - h;
+                            if (cnt > kMaxRowMaps) cnt = kMaxRowMaps;
+                            ptx::tma_load_4d_pair(sa + (uint32_t)(j * p.img_w) * 128u, &row_maps[cnt - 1], bar, cb * 32, dw,
+                                                  h + dh, img);
+                            j += cnt;
+                        }
+                        if (p.b_mn_major) ptx::tma_load_4d_pair(sb, &tmap_b, bar, 0, tap, cb * 32, n0 >> 5);
+                        else ptx::tma_load_2d_pair(sb, &tmap_b, bar, tap * p.ck + cb * 32, n0);
+                        if (++stage == kPStages) { stage = 0; phase ^= 1u; }
+                        continue;
+                    }
                     ptx::mbar_expect_tx_cluster(bar, kPStageBytes);
                     // an MN-major operand arrives as column blocks of one 128-byte row per K element:
                     // 32 columns x 32 K rows (TF32) or 64 columns x 64 K rows (16-bit codes)
@@ -898,9 +1063,11 @@ gemm_tf32_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
         __syncwarp();
     }
     } else {
-        // 128 x 80 + 256 x 208 registers fit the 384 x 168 the CTA was launched with; the increase
-        // blocks until that many are free in the CTA's own pool, so a larger request would never return
-        ptx::setmaxnreg_inc<208>();
+        // 128 x 56 + 256 x 224 registers are exactly the 384 x 168 the CTA was launched with; the increase
+        // blocks until that many are free in the CTA's own pool, so a larger request would never return.
+        // The accumulate warps hold 128 sums and 64 freshly loaded values; with 208 registers a few
+        // more live values in their loop already spilled (measured: 12 % slower products).
+        ptx::setmaxnreg_inc<224>();
         // ------------------------------ accumulate + epilogue (both CTAs) ------------------------------
         const int quad = warp & 3;
         const int half = (warp - 4) >> 2;
@@ -908,8 +1075,10 @@ gemm_tf32_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
         bool dead = false;
         for (int t = cluster_id; t < num_work && !dead; t += num_clusters) {
             const WorkItem w = decode_work(p, t);
-            const int m0 = w.m0 + (int)rank * kBM, n0 = w.n0, num_kb = w.num_kb;
-            const int m_end = m0 + kBM < p.M ? m0 + kBM : p.M;
+            constexpr bool kConv = kMode == 1;
+            const int cta_rows = kConv ? p.conv_rows : kBM;  // rows of C this CTA owns in the tile
+            const int m0 = w.m0 + (int)rank * cta_rows, n0 = w.n0, num_kb = w.num_kb;
+            const int m_end = m0 + cta_rows < p.M ? m0 + cta_rows : p.M;
             float* const c_base = p.C + (long long)w.split * p.split_stride;
             const bool use_tma = p.tma_store != 0;
             // level-1 running sums, two per 64-bit register (packed adds); 0 + x is exact, so a group's
@@ -917,11 +1086,13 @@ gemm_tf32_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
             unsigned long long sum2[64];
 #pragma unroll
             for (int j = 0; j < 64; ++j) sum2[j] = 0ull;
-            const uint32_t my_stage_addr = out_stage + (uint32_t)(warp - 4) * kOutWarpBytes;
+            const uint32_t my_stage_addr = out_stage + (uint32_t)(warp - 4) * kPOutWarpBytes;
             float* my_stage = reinterpret_cast<float*>(smem_raw + (my_stage_addr - raw));
             const int row0 = m0 + quad * 32;
             int in_group = 0;
-            bool flushed = false;
+            // a piece that begins inside its tile adds to what the pair before has stored there
+            bool flushed = w.partial != 0;
+            bool handed_over = w.partial == 0;  // the first part of the tile is known to be in C
             for (int kb0 = 0; kb0 < num_kb; kb0 += kChunkKB) {
                 const uint32_t acc = acc_iter & 1u, acc_phase = (acc_iter >> 1) & 1u;
                 bool ok = true;
@@ -957,9 +1128,107 @@ gemm_tf32_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
                 if (!last && ++in_group < kFlushChunks) continue;
                 if (kEpi)
                     epi_transform(sum2, p, row0 + lane < m_end, n0 + half * 128, reinterpret_cast<uint32_t*>(my_stage), epi_hist, lane);
+                if (!handed_over) {
+                    // wait (bounded) until the same warp of the pair before this one has completed its
+                    // stores to this patch of the tile
+                    int seen = 1;
+                    if (lane == 0) {
+                        volatile int* flag = p.sk_flags + (cluster_id * 16 + (int)rank * 8 + (warp - 4));
+                        const long long t_begin = clock64();
+                        while (*flag == 0) {
+                            if (clock64() - t_begin > (long long)kWaitLimit) { seen = 0; break; }
+                            __nanosleep(64);
+                        }
+                        __threadfence();
+                        ptx::fence_proxy_async_all();
+                    }
+                    seen = __shfl_sync(0xFFFFFFFFu, seen, 0);
+                    if (!seen) {
+                        if (lane == 0) raise_timeout(p, abort_flag);
+                        dead = true;
+                        break;
+                    }
+                    handed_over = true;
+                }
                 if (use_tma && flushed) {
                     if (lane == 0) ptx::bulk_wait_all();
                 }
+                if (kPOutBlocks == 3 && p.c_blocked) {
+                    if (lane == 0) ptx::bulk_wait_read_all();  // the previous flush's copy has read the staging area
+                    __syncwarp();
+#pragma unroll
+                    for (int blk = 0; blk < 3; ++blk) {
+                        float* box = my_stage + blk * 1024;
+#pragma unroll
+                        for (int c = 0; c < 8; ++c) {
+                            const int j = blk * kOutCols + c * 4;
+                            const float2 v0 = ptx::unpack2(sum2[j / 2]), v1 = ptx::unpack2(sum2[j / 2 + 1]);
+                            *reinterpret_cast<float4*>(box + lane * 32 + ((c ^ (lane & 7)) << 2)) =
+                                make_float4(v0.x, v0.y, v1.x, v1.y);
+                        }
+                    }
+                    ptx::fence_proxy_async();
+                    __syncwarp();
+                    if (lane == 0) {
+                        const int cblk = (n0 + half * 128) >> 5;
+                        if (row0 < m_end && cblk * 32 < p.N) {
+                            // convolution: the CTA's own tile of the per-tile map (or the map of the incomplete last tile)
+                            const int ctile = 2 * w.tile_m + (int)rank;
+                            const bool whole = !kConv || ctile < p.full_tiles_m;
+                            const CUtensorMap* cm = whole ? &tmap_c : tmap_c2;
+                            const int ry = kConv ? quad * 32 : row0, rz = kConv ? (whole ? ctile : 0) : w.split;
+                            if (flushed) ptx::tma_reduce_add_4d(cm, my_stage_addr, 0, ry, cblk, rz);
+                            else ptx::tma_store_4d(cm, my_stage_addr, 0, ry, cblk, rz);
+                        }
+                        ptx::bulk_commit();
+                    }
+                    // fourth block: each lane writes its row's 32 columns (128 bytes) itself
+                    const int col3 = n0 + half * 128 + 3 * kOutCols;
+                    if (row0 + lane < m_end && col3 < p.N) {
+                        float* g = c_base + (long long)(row0 + lane) * p.ldc + col3;
+#pragma unroll
+                        for (int c = 0; c < 8; ++c) {
+                            const int j = 3 * kOutCols + c * 4;
+                            const float2 v0 = ptx::unpack2(sum2[j / 2]), v1 = ptx::unpack2(sum2[j / 2 + 1]);
+                            if (flushed) ptx::red_add_v4(g + c * 4, v0.x, v0.y, v1.x, v1.y);
+                            else *reinterpret_cast<float4*>(g + c * 4) = make_float4(v0.x, v0.y, v1.x, v1.y);
+                        }
+                    }
+                } else if (p.c_blocked) {
+                    // Whole copies of kPOutBlocks column blocks: the staging area is filled (each 32 x 32 block
+                    // in the swizzled layout of a one-block box), then ONE copy instruction stores it or adds
+                    // it at the destination.  Blocks past N and rows past M are clipped by the copy engine.
+#pragma unroll
+                    for (int pass = 0; pass < (kPOutBlocks == 3 ? 0 : 4 / kPOutBlocks); ++pass) {
+                        if (lane == 0) ptx::bulk_wait_read_all();  // the previous copy has read the staging area
+                        __syncwarp();
+#pragma unroll
+                        for (int blk = 0; blk < kPOutBlocks; ++blk) {
+                            float* box = my_stage + blk * 1024;
+#pragma unroll
+                            for (int c = 0; c < 8; ++c) {
+                                const int j = (pass * kPOutBlocks + blk) * kOutCols + c * 4;
+                                const float2 v0 = ptx::unpack2(sum2[j / 2]), v1 = ptx::unpack2(sum2[j / 2 + 1]);
+                                *reinterpret_cast<float4*>(box + lane * 32 + ((c ^ (lane & 7)) << 2)) =
+                                    make_float4(v0.x, v0.y, v1.x, v1.y);
+                            }
+                        }
+                        ptx::fence_proxy_async();
+                        __syncwarp();
+                        if (lane == 0) {
+                            const int cblk = ((n0 + half * 128) >> 5) + pass * kPOutBlocks;
+                            if (row0 < m_end && cblk * 32 < p.N) {
+                                const int ctile = 2 * w.tile_m + (int)rank;
+                                const bool whole = !kConv || ctile < p.full_tiles_m;
+                                const CUtensorMap* cm = whole ? &tmap_c : tmap_c2;
+                                const int ry = kConv ? quad * 32 : row0, rz = kConv ? (whole ? ctile : 0) : w.split;
+                                if (flushed) ptx::tma_reduce_add_4d(cm, my_stage_addr, 0, ry, cblk, rz);
+                                else ptx::tma_store_4d(cm, my_stage_addr, 0, ry, cblk, rz);
+                            }
+                            ptx::bulk_commit();
+                        }
+                    }
+                } else
 #pragma unroll
                 for (int pass = 0; pass < 4; ++pass) {
                     const int col0 = n0 + half * 128 + pass * kOutCols;
@@ -1007,6 +1276,16 @@ gemm_tf32_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
                 }
             }
             if (dead) break;
+            if (w.head && num_kb > 0) {
+                // this warp's part of the tile's first piece is in C: tell the pair that adds the rest
+                if (lane == 0) {
+                    ptx::bulk_wait_all();
+                    ptx::fence_proxy_async_all();
+                    __threadfence();
+                    *reinterpret_cast<volatile int*>(p.sk_flags + ((cluster_id + 1) * 16 + (int)rank * 8 + (warp - 4))) = 1;
+                }
+                __syncwarp();
+            }
         }
         if (lane == 0) ptx::bulk_wait_all();
         __syncwarp();
@@ -1024,6 +1303,22 @@ gemm_tf32_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
         ptx::tc_fence_after_sync();
         ptx::tmem_dealloc_pair(tmem_base, kTmemCols);
     }
+}
+
+template <bool kEpi, int kKind>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+gemm_tf32_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+                      const __grid_constant__ CUtensorMap tmap_c, const GemmParams p) {
+    pair_body<kEpi, kKind, 0>(tmap_a, tmap_b, tmap_c, nullptr, nullptr, p);
+}
+
+// Forward / data gradient of a convolution on CTA pairs (its own instantiation, so that the dense
+// products carry none of its code).
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+gemm_conv_pair_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_constant__ CUtensorMap tmap_c,
+                      const __grid_constant__ CUtensorMap tmap_c2, const __grid_constant__ RowMaps row_maps,
+                      const GemmParams p) {
+    pair_body<false, kKindTf32, 1>(row_maps.m[0], tmap_b, tmap_c, &tmap_c2, row_maps.m, p);
 }
 
 // ---- host side ----------------------------------------------------------------------------------
@@ -1113,6 +1408,14 @@ int make_map_c(CUtensorMap* map, float* base, uint64_t n, uint64_t rows, uint64_
     const uint64_t dims[3] = {n, rows, zdim}, strides[2] = {ld, zstride};
     const uint32_t box[3] = {32, 32, 1};
     return make_map(map, base, 3, dims, strides, box, false);
+}
+
+// The same for N a multiple of 32, seen as [z][N / 32][rows][32]: a box takes kPOutBlocks whole 32 x 32
+// blocks that are adjacent along the row, each landing in shared memory as one 4 KB swizzled block.
+int make_map_c_blocked(CUtensorMap* map, float* base, uint64_t n, uint64_t rows, uint64_t zdim, uint64_t ld, uint64_t zstride) {
+    const uint64_t dims[4] = {32, rows, n / 32, zdim}, strides[3] = {ld, 32, zstride};
+    const uint32_t box[4] = {32, 32, (uint32_t)kPOutBlocks, 1};
+    return make_map(map, base, 4, dims, strides, box, false);
 }
 
 // Sums the split-K partials [splits][rows][cols] (dense) into C in a fixed pairwise order: adjacent
@@ -1232,12 +1535,15 @@ void dense_defaults(GemmParams* p) {
     p->tap_sign = 1;
     p->off_h = p->off_w = 0;
     p->full_tiles_m = 0;
+    p->conv_rows = 0;
     p->a_blocked = p->b_blocked = 0;
+    p->c_blocked = 0;
     p->rows_box = 1;
     p->wg_padded = 0;
     p->sk_cpt = 0;
     p->sk_pieces = 1;
     p->sk_partials = nullptr;
+    p->sk_flags = nullptr;
     p->epi = 0;
     p->epi_rbias = nullptr;
     p->epi_stats = nullptr;
@@ -1249,11 +1555,18 @@ void dense_defaults(GemmParams* p) {
 // tiles (256 x 256).  Process-wide; see qfmt_gemm_tile_policy.
 static std::atomic<int> g_tile_policy{0};
 
+// Which kernel the forward / data-gradient products of a convolution run on: 0 automatic (CTA pairs
+// when there are two or more M-tiles), 1 always the single-CTA kernel.  See qfmt_gemm_tile_policy.
+static std::atomic<int> g_conv_pair_policy{0};
+
 // How a dense product is laid over the GPU: tile shape and split-K factor.
 struct DensePlan {
     bool pair;
     int splits;
+    bool sk;  // CTA-pair tiles under the balanced schedule (GemmParams::sk_flags)
 };
+constexpr int kPlanPairs = 74;  // CTA pairs of a 148-SM part: the balanced schedule is dealt among exactly these
+constexpr size_t kSkFlagBytes = ((size_t)(kPlanPairs + 1) * 16 * sizeof(int) + 255) & ~(size_t)255;
 
 // Picks the plan with the least estimated time.  The unit is the time one CTA pair needs for one
 // 64-element K chunk of a 256 x 256 tile, about a microsecond; a single CTA needs 1.07 of it for
@@ -1264,7 +1577,7 @@ struct DensePlan {
 DensePlan plan_dense(int64_t M, int64_t N, int64_t K, int policy_override = -1) {
     const int policy = policy_override >= 0 ? policy_override : g_tile_policy.load();
     const int64_t kb_total = (K + kBK - 1) / kBK;
-    DensePlan best = {policy == 2, 1};
+    DensePlan best = {policy == 2, 1, false};
     double best_cost = -1.0;
     for (int pair = 0; pair < 2; ++pair) {
         if (policy == 1 && pair) continue;
@@ -1283,7 +1596,17 @@ DensePlan plan_dense(int64_t M, int64_t N, int64_t K, int policy_override = -1) 
             if (splits > 1) cost += 3.0 + (double)(splits + 1) * (double)M * (double)N * 4.0 / 6.5e6;
             if (best_cost < 0.0 || cost < best_cost * 0.97) {  // more splits only for a clear gain
                 best_cost = cost;
-                best = {pair != 0, (int)splits};
+                best = {pair != 0, (int)splits, false};
+            }
+        }
+        // Balanced schedule: the tiles' chunks dealt among the 74 pairs in equal ranges.  A pair then runs
+        // tiles / 74 + 1 pieces, each with its own move of sums to C.  Needs ranges of at least a tile.
+        if (pair && tiles >= kPlanPairs) {
+            const double chunks = (double)((kb_total + kChunkKB - 1) / kChunkKB);
+            const double cost = (double)tiles * chunks / kPlanPairs + 3.0 * ((double)tiles / kPlanPairs + 1.0);
+            if (cost < best_cost * 0.97) {
+                best_cost = cost;
+                best = {true, 1, true};
             }
         }
     }
@@ -1305,12 +1628,27 @@ int launch_pair(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap&
         if (dev.ordinal >= 0 && dev.ordinal < 64) attr_set[dev.ordinal] = true;
     }
     const long long work = (long long)p.tiles_m * p.tiles_n * p.splits;
-    const long long clusters = work < dev.sm_count / 2 ? work : dev.sm_count / 2;
+    const long long clusters = p.sk_flags != nullptr ? kPlanPairs : (work < dev.sm_count / 2 ? work : dev.sm_count / 2);
     const unsigned grid = (unsigned)(2 * clusters);
     if (kind == kKindF16) gemm_tf32_pair_kernel<false, kKindF16><<<grid, kThreads, kPairSmemBytes, stream>>>(ma, mb, mc, p);
     else if (kind == kKindBf16) gemm_tf32_pair_kernel<false, kKindBf16><<<grid, kThreads, kPairSmemBytes, stream>>>(ma, mb, mc, p);
     else if (p.epi) gemm_tf32_pair_kernel<true, kKindTf32><<<grid, kThreads, kPairSmemBytes, stream>>>(ma, mb, mc, p);
     else gemm_tf32_pair_kernel<false, kKindTf32><<<grid, kThreads, kPairSmemBytes, stream>>>(ma, mb, mc, p);
+    QFMT_CUDA_TRY(cudaGetLastError());
+    return QFMT_OK;
+}
+
+int launch_conv_pair(const CUtensorMap& mb, const CUtensorMap& mc, const CUtensorMap& mc2, const RowMaps& rows,
+                     const GemmParams& p, const DeviceInfo& dev, cudaStream_t stream) {
+    static bool attr_set[64] = {};
+    if (dev.ordinal < 0 || dev.ordinal >= 64 || !attr_set[dev.ordinal]) {
+        QFMT_CUDA_TRY(cudaFuncSetAttribute(gemm_conv_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           (int)kPairSmemBytes));
+        if (dev.ordinal >= 0 && dev.ordinal < 64) attr_set[dev.ordinal] = true;
+    }
+    const long long work = (long long)p.tiles_m * p.tiles_n;
+    const long long clusters = p.sk_flags != nullptr ? kPlanPairs : (work < dev.sm_count / 2 ? work : dev.sm_count / 2);
+    gemm_conv_pair_kernel<<<(unsigned)(2 * clusters), kThreads, kPairSmemBytes, stream>>>(mb, mc, mc2, rows, p);
     QFMT_CUDA_TRY(cudaGetLastError());
     return QFMT_OK;
 }
@@ -1323,8 +1661,26 @@ struct EpiArgs {
 // The epilogue runs on the sums of one group held in registers: at most this many K elements.
 constexpr int64_t kEpiMaxK = (int64_t)kFlushChunks * kChunkKB * kBK;
 
-int gemm_device(const qfmt_matrix_t* A, const qfmt_matrix_t* B, float* d_C, int64_t ldc, const qfmt_format_t* fmt,
-                void* d_workspace, size_t workspace_bytes, cudaStream_t stream, const EpiArgs* epi = nullptr) {
+// Turns the balanced schedule of the pair kernel on: chunks per tile, the most pieces a pair can have,
+// and the flag words behind the workspace header (cleared on the stream, with the status word).
+int enable_pair_schedule(GemmParams* p, void* d_workspace, cudaStream_t stream) {
+    p->sk_cpt = (p->kb_total + kChunkKB - 1) / kChunkKB;
+    const long long total = (long long)p->tiles_m * p->tiles_n * p->sk_cpt;
+    const long long range = (total + kPlanPairs - 1) / kPlanPairs;
+    p->sk_pieces = (int)((range + p->sk_cpt - 1) / p->sk_cpt + 1);
+    p->sk_q = (int)(total / kPlanPairs);
+    p->sk_r = (int)(total % kPlanPairs);
+    p->sk_flags = reinterpret_cast<int*>(reinterpret_cast<char*>(d_workspace) + kWorkspaceHeader);
+    QFMT_CUDA_TRY(cudaMemsetAsync(p->sk_flags, 0, kSkFlagBytes, stream));
+    return QFMT_OK;
+}
+
+// Host-side checks of a dense product's arguments, in the order the entry points report them: format,
+// descriptors and shapes, workspace, output and operand pointers.  Touches no device state.  On
+// QFMT_OK *M, *N, *K hold the product's dimensions (M or N may be zero: nothing to do).
+int validate_gemm_args(const qfmt_matrix_t* A, const qfmt_matrix_t* B, const float* d_C, int64_t ldc,
+                       const qfmt_format_t* fmt, const void* d_workspace, size_t workspace_bytes, int64_t* M_out,
+                       int64_t* N_out, int64_t* K_out) {
     int rc = validate_format(fmt);
     if (rc != QFMT_OK) return rc;
     if (fmt->m > 10) return QFMT_ERR_BAD_FORMAT;  // beyond TF32's mantissa: products would not be exact
@@ -1337,6 +1693,7 @@ int gemm_device(const qfmt_matrix_t* A, const qfmt_matrix_t* B, float* d_C, int6
     if (A->ld < A->cols || B->ld < B->cols || ldc < N) return QFMT_ERR_BAD_ARG;
     if (d_workspace == nullptr || workspace_bytes < 16 || (reinterpret_cast<uintptr_t>(d_workspace) & 15u))
         return QFMT_ERR_BAD_ARG;
+    *M_out = M; *N_out = N; *K_out = K;
     if (M == 0 || N == 0) return QFMT_OK;
     if (A->ptr == nullptr && K != 0) return QFMT_ERR_BAD_ARG;
     if (B->ptr == nullptr && K != 0) return QFMT_ERR_BAD_ARG;
@@ -1345,6 +1702,15 @@ int gemm_device(const qfmt_matrix_t* A, const qfmt_matrix_t* B, float* d_C, int6
     if ((reinterpret_cast<uintptr_t>(A->ptr) & 15u) || (reinterpret_cast<uintptr_t>(B->ptr) & 15u) ||
         (A->ld & 3) || (B->ld & 3))
         return QFMT_ERR_BAD_ARG;
+    return QFMT_OK;
+}
+
+int gemm_device(const qfmt_matrix_t* A, const qfmt_matrix_t* B, float* d_C, int64_t ldc, const qfmt_format_t* fmt,
+                void* d_workspace, size_t workspace_bytes, cudaStream_t stream, const EpiArgs* epi = nullptr) {
+    int64_t M = 0, N = 0, K = 0;
+    int rc = validate_gemm_args(A, B, d_C, ldc, fmt, d_workspace, workspace_bytes, &M, &N, &K);
+    if (rc != QFMT_OK) return rc;
+    if (M == 0 || N == 0) return QFMT_OK;
     DeviceInfo dev;
     rc = current_device(&dev);
     if (rc != QFMT_OK) return rc;
@@ -1377,6 +1743,11 @@ int gemm_device(const qfmt_matrix_t* A, const qfmt_matrix_t* B, float* d_C, int6
     // Split K when the workspace the caller lent has room for the partial sums (the recommended size
     // from qfmt_gemm_workspace_bytes always has); a smaller workspace gets fewer splits.
     int splits = epi != nullptr ? 1 : plan.splits;
+    // The balanced schedule needs every pair resident at once (148 SMs), room for its flags in the
+    // workspace, and the blocked C map.
+    const bool sk = plan.sk && epi == nullptr && pair && dev.sm_count >= 2 * kPlanPairs && p.tma_store &&
+                    (N & 31) == 0 && workspace_bytes >= kWorkspaceHeader + kSkFlagBytes &&
+                    (long long)p.tiles_m * p.tiles_n * ((p.kb_total + kChunkKB - 1) / kChunkKB) < (1ll << 30);
     if (epi != nullptr) {
         if (K > kEpiMaxK || fmt->e > 6) return QFMT_ERR_BAD_ARG;  // callers check before asking
         qfmt_format_t f = *fmt;
@@ -1388,7 +1759,10 @@ int gemm_device(const qfmt_matrix_t* A, const qfmt_matrix_t* B, float* d_C, int6
     }
     while (splits > 1 && kWorkspaceHeader + (size_t)splits * (size_t)M * (size_t)N * sizeof(float) > workspace_bytes) --splits;
     float* partials = reinterpret_cast<float*>(reinterpret_cast<char*>(d_workspace) + kWorkspaceHeader);
-    if (splits > 1) {
+    if (sk) {
+        rc = enable_pair_schedule(&p, d_workspace, stream);
+        if (rc != QFMT_OK) return rc;
+    } else if (splits > 1) {
         p.kb_per_split = (p.kb_total + splits - 1) / splits;
         p.splits = (p.kb_total + p.kb_per_split - 1) / p.kb_per_split;
         p.split_stride = (long long)M * N;
@@ -1418,7 +1792,10 @@ int gemm_device(const qfmt_matrix_t* A, const qfmt_matrix_t* B, float* d_C, int6
     } else if (p.b_mn_major) rc = make_map_2d(&mb, B->ptr, (uint64_t)N, (uint64_t)K, (uint64_t)B->ld, 32, kBK, true);
     else rc = make_map_2d(&mb, B->ptr, (uint64_t)K, (uint64_t)N, (uint64_t)B->ld, kBK, pair ? kBN / 2 : kBN, false);
     if (rc != QFMT_OK) return rc;
-    if (p.tma_store)
+    p.c_blocked = (pair && p.tma_store && (N & 31) == 0) ? 1 : 0;
+    if (p.c_blocked)
+        rc = make_map_c_blocked(&mc, p.C, (uint64_t)N, (uint64_t)M, (uint64_t)p.splits, (uint64_t)p.ldc, (uint64_t)M * (uint64_t)p.ldc);
+    else if (p.tma_store)
         rc = make_map_c(&mc, p.C, (uint64_t)N, (uint64_t)M, (uint64_t)p.splits, (uint64_t)p.ldc, (uint64_t)M * (uint64_t)p.ldc);
     else mc = ma;  // unused by the kernel
     if (rc != QFMT_OK) return rc;
@@ -1485,10 +1862,17 @@ int gemm16_device(const qfmt_matrix16_t* A, const qfmt_matrix16_t* B, float* d_C
     p.kb_total = (int)((K + 2 * kBK - 1) / (2 * kBK));
     p.kb_per_split = p.kb_total;
     p.tma_store = ((reinterpret_cast<uintptr_t>(d_C) & 15u) == 0 && (ldc & 3) == 0 && (N & 3) == 0) ? 1 : 0;
-    int splits = plan_dense(M, N, (K + 1) / 2, 2).splits;
+    const DensePlan plan = plan_dense(M, N, (K + 1) / 2, 2);
+    int splits = plan.splits;
+    const bool sk = plan.sk && dev.sm_count >= 2 * kPlanPairs && p.tma_store && (N & 31) == 0 &&
+                    workspace_bytes >= kWorkspaceHeader + kSkFlagBytes &&
+                    (long long)p.tiles_m * p.tiles_n * ((p.kb_total + kChunkKB - 1) / kChunkKB) < (1ll << 30);
     while (splits > 1 && kWorkspaceHeader + (size_t)splits * (size_t)M * (size_t)N * sizeof(float) > workspace_bytes) --splits;
     float* partials = reinterpret_cast<float*>(reinterpret_cast<char*>(d_workspace) + kWorkspaceHeader);
-    if (splits > 1) {
+    if (sk) {
+        rc = enable_pair_schedule(&p, d_workspace, stream);
+        if (rc != QFMT_OK) return rc;
+    } else if (splits > 1) {
         p.kb_per_split = (p.kb_total + splits - 1) / splits;
         p.splits = (p.kb_total + p.kb_per_split - 1) / p.kb_per_split;
         p.split_stride = (long long)M * N;
@@ -1501,7 +1885,10 @@ int gemm16_device(const qfmt_matrix16_t* A, const qfmt_matrix16_t* B, float* d_C
     if (rc != QFMT_OK) return rc;
     rc = make_operand_map16(&mb, B->ptr, p.b_mn_major != 0, (uint64_t)N, (uint64_t)K, (uint64_t)B->ld, kBN / 2, &p.b_blocked);
     if (rc != QFMT_OK) return rc;
-    if (p.tma_store)
+    p.c_blocked = (p.tma_store && (N & 31) == 0) ? 1 : 0;
+    if (p.c_blocked)
+        rc = make_map_c_blocked(&mc, p.C, (uint64_t)N, (uint64_t)M, (uint64_t)p.splits, (uint64_t)p.ldc, (uint64_t)M * (uint64_t)p.ldc);
+    else if (p.tma_store)
         rc = make_map_c(&mc, p.C, (uint64_t)N, (uint64_t)M, (uint64_t)p.splits, (uint64_t)p.ldc, (uint64_t)M * (uint64_t)p.ldc);
     else mc = ma;  // unused by the kernel
     if (rc != QFMT_OK) return rc;
@@ -1520,6 +1907,8 @@ int gemm16_device(const qfmt_matrix16_t* A, const qfmt_matrix16_t* B, float* d_C
 namespace {
 struct ConvPlan {
     int64_t oh, ow;
+    bool pair;       // forward / data gradient on CTA pairs (two M-tiles of whole image rows per pair)
+    bool pair_sk;    // ... under the balanced schedule of the pair kernel
     int splits;
     int sk_cpt;      // forward / data gradient: chunks per tile when the balanced schedule is used, else 0
     int sk_pieces;
@@ -1548,6 +1937,8 @@ int plan_conv(int op, const qfmt_conv_t* g, ConvPlan* plan) {
         (int64_t)g->r * g->s * g->c_in > (1 << 30))
         return QFMT_ERR_BAD_ARG;
     plan->splits = 1;
+    plan->pair = false;
+    plan->pair_sk = false;
     plan->sk_cpt = 0;
     plan->sk_pieces = 1;
     plan->workspace = kWorkspaceHeader;
@@ -1557,8 +1948,9 @@ int plan_conv(int op, const qfmt_conv_t* g, ConvPlan* plan) {
         const int64_t M = op == QFMT_CONV_WGRAD ? g->c_out : pixels;
         const int64_t N = op == QFMT_CONV_FWD ? g->c_out : g->c_in;
         const int64_t K = op == QFMT_CONV_FWD ? g->c_in : (op == QFMT_CONV_DGRAD ? g->c_out : pixels);
-        const int splits = plan_dense(M, N, K).splits;
-        if (splits > 1) plan->workspace += (size_t)splits * (size_t)M * (size_t)N * sizeof(float);
+        const DensePlan dense = plan_dense(M, N, K);
+        if (dense.sk) plan->workspace += kSkFlagBytes;
+        else if (dense.splits > 1) plan->workspace += (size_t)dense.splits * (size_t)M * (size_t)N * sizeof(float);
         return QFMT_OK;
     }
     if (op == QFMT_CONV_FWD && plan->ow > kBM) return QFMT_ERR_BAD_ARG;   // an M-tile is made of whole output rows
@@ -1572,6 +1964,21 @@ int plan_conv(int op, const qfmt_conv_t* g, ConvPlan* plan) {
         const int64_t tiles = (((int64_t)g->n * rows + rows_per_blk - 1) / rows_per_blk) * ((n_cols + kBN - 1) / kBN);
         const int64_t kb_total = (int64_t)g->r * g->s * (src_c / 32), cpt = (kb_total + kChunkKB - 1) / kChunkKB;
         const int64_t waves = (tiles + kPlanSms - 1) / kPlanSms;
+        // Two or more M-tiles: CTA pairs, each CTA one M-tile and half of the filter columns (8 KB of
+        // operands per MMA and CTA instead of 12).  The balanced schedule is priced as for dense products.
+        const int64_t conv_tiles_m = ((int64_t)g->n * rows + rows_per_blk - 1) / rows_per_blk;
+        if (conv_tiles_m >= 2 && g_conv_pair_policy.load() != 1) {
+            plan->pair = true;
+            const int64_t ptiles = ((conv_tiles_m + 1) / 2) * ((n_cols + kBN - 1) / kBN);
+            if (ptiles >= kPlanPairs) {
+                const int64_t pwaves = (ptiles + kPlanPairs - 1) / kPlanPairs;
+                const double plain = (double)pwaves * ((double)cpt + 3.0);
+                const double sk = (double)ptiles * (double)cpt / kPlanPairs + 3.0 * ((double)ptiles / kPlanPairs + 1.0);
+                plan->pair_sk = sk < plain * 0.97 && ptiles * cpt < (1ll << 30);
+            }
+            plan->workspace += kSkFlagBytes;
+            return QFMT_OK;
+        }
         // It pays when the last of a few waves is poorly filled and tiles are long: every piece ends
         // with an output flush of its own, and pieces that begin inside a tile are added to C later.
         if (tiles >= kPlanSms && waves <= 3 && waves * kPlanSms * 100 >= tiles * 115 && cpt >= 24) {
@@ -1702,6 +2109,45 @@ int conv_device(int op, const qfmt_conv_t* g, const float* d_p, const float* d_q
             if (rc != QFMT_OK) return rc;
         }
         ma = rmaps.m[0];
+        if (plan.pair) {
+            // CTA pairs: a pair tile is two M-tiles; each CTA stages its own pixels and 128 filter columns
+            const int conv_tiles_m = p.tiles_m;
+            p.conv_rows = p.tile_rows;
+            p.tile_rows = 2 * p.conv_rows;
+            p.tiles_m = (conv_tiles_m + 1) / 2;
+            p.c_blocked = 1;
+            if (fwd) {
+                rc = make_map_2d(&mb, d_q, TAPS * CI, CO, TAPS * CI, kBK, kBN / 2, false);
+            } else {
+                const uint64_t dims[4] = {32, TAPS, CO, CI / 32}, st[3] = {CI, TAPS * CI, 32};
+                const uint32_t box[4] = {32, 1, kBK, (kBN / 2) / 32};
+                rc = make_map(&mb, d_q, 4, dims, st, box, true);
+            }
+            if (rc != QFMT_OK) return rc;
+            // C per M-tile: {32, conv_rows, N / 32, complete tiles}; the incomplete last tile has a map of its own
+            CUtensorMap mc2;
+            const uint64_t full = (uint64_t)p.full_tiles_m, rem = (uint64_t)p.M - full * (uint64_t)p.conv_rows;
+            const uint32_t cbox[4] = {32, 32, (uint32_t)kPOutBlocks, 1};
+            if (rem > 0) {
+                const uint64_t d2[4] = {32, rem, n_cols / 32, 1}, s2[3] = {n_cols, 32, rem * n_cols};
+                rc = make_map(&mc2, d_out + full * (uint64_t)p.conv_rows * n_cols, 4, d2, s2, cbox, false);
+                if (rc != QFMT_OK) return rc;
+            }
+            if (full > 0) {
+                const uint64_t d1[4] = {32, (uint64_t)p.conv_rows, n_cols / 32, full};
+                const uint64_t s1[3] = {n_cols, 32, (uint64_t)p.conv_rows * n_cols};
+                rc = make_map(&mc, d_out, 4, d1, s1, cbox, false);
+                if (rc != QFMT_OK) return rc;
+            } else {
+                mc = mc2;
+            }
+            if (rem == 0) mc2 = mc;
+            if (plan.pair_sk && dev.sm_count >= 2 * kPlanPairs) {
+                rc = enable_pair_schedule(&p, d_workspace, stream);
+                if (rc != QFMT_OK) return rc;
+            }
+            return launch_conv_pair(mb, mc, mc2, rmaps, p, dev, stream);
+        }
         if (fwd) {  // filters [CO][TAPS*CI], K contiguous
             rc = make_map_2d(&mb, d_q, TAPS * CI, CO, TAPS * CI, kBK, kBN, false);
         } else {    // filters [CO][TAPS][CI]: N = CI contiguous, K = CO rows
@@ -1902,6 +2348,12 @@ extern "C" size_t qfmt_linear_forward_workspace_bytes(const qfmt_matrix_t* A, co
     return qfmt_gemm_workspace_bytes(A, B) + qfmt::linear_bias_bytes(N) + 256;
 }
 
+extern "C" int qfmt_conv_tile_policy(int policy) {
+    if (policy < 0 || policy > 1) return QFMT_ERR_BAD_ARG;
+    qfmt::g_conv_pair_policy.store(policy);
+    return QFMT_OK;
+}
+
 extern "C" int qfmt_gemm_tile_policy(int policy) {
     if (policy < 0 || policy > 2) return QFMT_ERR_BAD_ARG;
     qfmt::g_tile_policy.store(policy);
@@ -1914,8 +2366,9 @@ extern "C" size_t qfmt_gemm_workspace_bytes(const qfmt_matrix_t* A, const qfmt_m
     const int64_t M = A->trans ? A->cols : A->rows, K = A->trans ? A->rows : A->cols;
     const int64_t N = B->trans ? B->rows : B->cols;
     if (M <= 0 || N <= 0 || K <= 0 || M > (1 << 30) || N > (1 << 30) || K > (1 << 30)) return qfmt::kWorkspaceHeader;
-    const int splits = qfmt::plan_dense(M, N, K).splits;
-    return qfmt::kWorkspaceHeader + (splits > 1 ? (size_t)splits * (size_t)M * (size_t)N * sizeof(float) : 0);
+    const qfmt::DensePlan plan = qfmt::plan_dense(M, N, K);
+    if (plan.sk) return qfmt::kWorkspaceHeader + qfmt::kSkFlagBytes;
+    return qfmt::kWorkspaceHeader + (plan.splits > 1 ? (size_t)plan.splits * (size_t)M * (size_t)N * sizeof(float) : 0);
 }
 
 extern "C" size_t qfmt_gemm_packed16_workspace_bytes(const qfmt_matrix16_t* A, const qfmt_matrix16_t* B) {
@@ -1924,8 +2377,9 @@ extern "C" size_t qfmt_gemm_packed16_workspace_bytes(const qfmt_matrix16_t* A, c
     const int64_t M = A->trans ? A->cols : A->rows, K = A->trans ? A->rows : A->cols;
     const int64_t N = B->trans ? B->rows : B->cols;
     if (M <= 0 || N <= 0 || K <= 0 || M > (1 << 30) || N > (1 << 30) || K > (1 << 30)) return qfmt::kWorkspaceHeader;
-    const int splits = qfmt::plan_dense(M, N, (K + 1) / 2, 2).splits;
-    return qfmt::kWorkspaceHeader + (splits > 1 ? (size_t)splits * (size_t)M * (size_t)N * sizeof(float) : 0);
+    const qfmt::DensePlan plan = qfmt::plan_dense(M, N, (K + 1) / 2, 2);
+    if (plan.sk) return qfmt::kWorkspaceHeader + qfmt::kSkFlagBytes;
+    return qfmt::kWorkspaceHeader + (plan.splits > 1 ? (size_t)plan.splits * (size_t)M * (size_t)N * sizeof(float) : 0);
 }
 
 extern "C" int qfmt_device_status(void* d_workspace, void* stream) {
@@ -1936,6 +2390,20 @@ extern "C" int qfmt_device_status(void* d_workspace, void* stream) {
     return st;
 }
 
+
+extern "C" int qfmt_selftest_bounded_wait(int32_t* d_status, uint32_t limit_cycles, int32_t* d_trace, void* stream) {
+    if (d_status == nullptr || d_trace == nullptr) return QFMT_ERR_BAD_ARG;
+    if ((reinterpret_cast<uintptr_t>(d_status) & 3u) || (reinterpret_cast<uintptr_t>(d_trace) & 3u)) return QFMT_ERR_BAD_ARG;
+    if (limit_cycles == 0 || limit_cycles > (1u << 24)) return QFMT_ERR_BAD_ARG;  // at most a few milliseconds
+    qfmt::DeviceInfo dev;
+    int rc = qfmt::current_device(&dev);
+    if (rc != QFMT_OK) return rc;
+    QFMT_CUDA_TRY(cudaMemsetAsync(d_status, 0, sizeof(int32_t), (cudaStream_t)stream));
+    QFMT_CUDA_TRY(cudaMemsetAsync(d_trace, 0, 4 * sizeof(int32_t), (cudaStream_t)stream));
+    qfmt::bounded_wait_selftest_kernel<<<1, 64, 0, (cudaStream_t)stream>>>(d_status, limit_cycles, d_trace);
+    QFMT_CUDA_TRY(cudaGetLastError());
+    return QFMT_OK;
+}
 
 // ------------------------------------------------------------------------------------------------
 // Variant with built-in scratch memory (no counterpart in the paper; see include/qfmt.h).
@@ -1970,16 +2438,22 @@ int builtin_scratch_address(void** out) {
 
 extern "C" int qfmt_gemm_builtin_scratch(const qfmt_matrix_t* A, const qfmt_matrix_t* B, float* d_C, int64_t ldc,
                                          const qfmt_format_t* fmt, int32_t* d_status_out, void* stream) {
+    // Everything the host can check comes first, so that an error return has enqueued nothing.  The
+    // checks use a stand-in workspace address; the array's real address is looked up afterwards.
+    int64_t M = 0, N = 0, K = 0;
+    alignas(16) static const char placeholder[16] = {};
     if (A == nullptr || B == nullptr) return QFMT_ERR_BAD_ARG;
+    int rc = qfmt::validate_gemm_args(A, B, d_C, ldc, fmt, placeholder, qfmt::kBuiltinScratchBytes, &M, &N, &K);
+    if (rc != QFMT_OK) return rc;
     if (reinterpret_cast<uintptr_t>(d_status_out) & 3u) return QFMT_ERR_BAD_ARG;
     if (qfmt_gemm_workspace_bytes(A, B) > qfmt::kBuiltinScratchBytes) return QFMT_ERR_SCRATCH_LIMIT;
     void* scratch = nullptr;
-    int rc = qfmt::builtin_scratch_address(&scratch);
+    rc = qfmt::builtin_scratch_address(&scratch);
     if (rc != QFMT_OK) return rc;
-    // The array still holds what the previous call left.  Only the status word at its head has
-    // to start at zero; clear it here as well so that a call that enqueues no kernel (M or N zero)
-    // does not report an older call's status.
-    QFMT_CUDA_TRY(cudaMemsetAsync(scratch, 0, 16, (cudaStream_t)stream));
+    // The array still holds what the previous call left.  Only the status word at its head has to
+    // start at zero; a product with work to do clears it itself, so it is cleared here only for
+    // the call that enqueues no kernel (M or N zero), which must not report an older call's status.
+    if (M == 0 || N == 0) QFMT_CUDA_TRY(cudaMemsetAsync(scratch, 0, 16, (cudaStream_t)stream));
     rc = qfmt::gemm_device(A, B, d_C, ldc, fmt, scratch, qfmt::kBuiltinScratchBytes, (cudaStream_t)stream);
     if (rc != QFMT_OK) return rc;
     if (d_status_out != nullptr)

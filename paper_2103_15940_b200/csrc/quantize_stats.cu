@@ -392,6 +392,25 @@ __device__ __forceinline__ uint32_t bias_round_one(uint32_t acc, uint32_t rb, co
     return q;
 }
 
+// The common case of the layer formula in eleven float/integer operations per element: when the scaled
+// product lies in a normal binade of the format below the top one, and so does the fp32 sum with the
+// bias, neither rounding can overflow, underflow, lose a sign or meet a special value, and the result's
+// bin is its own exponent field.  `ok` is cleared when either condition fails (the caller then takes
+// the general path for the whole vector); lo2 = 2 * 2^E_min as a word shifted left by one (the sign
+// drops out), span2 the width of the admitted exponent range in the same units.
+template <bool kScale>
+__device__ __forceinline__ uint32_t bias_round_fast(uint32_t acc, uint32_t rb, const QuantParams& p, uint32_t lo2,
+                                                    uint32_t span2, bool& ok) {
+    const uint32_t yb = kScale ? __float_as_uint(mul_ieee(__uint_as_float(acc), p.scale)) : acc;
+    ok = ok && (((yb << 1) - lo2) < span2);
+    const float c = __uint_as_float((yb & 0x7F800000u) + p.magic_add);
+    const float ra = sub_ieee(add_ieee(__uint_as_float(yb), c), c);
+    const uint32_t sb = __float_as_uint(add_ieee(ra, __uint_as_float(rb)));
+    ok = ok && (((sb << 1) - lo2) < span2);
+    const float c2 = __uint_as_float((sb & 0x7F800000u) + p.magic_add);
+    return __float_as_uint(sub_ieee(add_ieee(__uint_as_float(sb), c2), c2));
+}
+
 // kPack: the output is written as packed 16-bit codes (out_v points at uint16_t, ld_out counts codes;
 // four codes per 8-byte store) instead of fp32 containers.
 template <bool kStats, bool kScale, bool kPack>
@@ -405,6 +424,8 @@ bias_quantize_stats_kernel(const uint32_t* acc, long long ld_acc, const uint32_t
     const int nbins = p.top + kExtraBins;
     const int lane = threadIdx.x & 31;
     const uint32_t inf_bits = p.top < 255 ? (uint32_t)(p.top + p.code_off) << 23 : 0u;  // 2^(E_max+1); 0 = 1/8/m
+    // fast path: exponent fields from E_min up to E_max - 1 (see bias_round_fast)
+    const uint32_t lo2 = p.min_normal << 1, span2 = (inf_bits - (1u << 23) - p.min_normal) << 1;
     if (kStats) {
         for (int i = threadIdx.x; i < nbins * 32; i += kThreads) lane_hist[i] = 0u;
         __syncthreads();
@@ -438,10 +459,23 @@ bias_quantize_stats_kernel(const uint32_t* acc, long long ld_acc, const uint32_t
                     if (row + u * row_step < rows) {
                         int b0, b1, b2, b3;
                         uint4 q;
-                        q.x = bias_round_one<kScale>(v[u].x, b.x, p, inf_bits, b0);
-                        q.y = bias_round_one<kScale>(v[u].y, b.y, p, inf_bits, b1);
-                        q.z = bias_round_one<kScale>(v[u].z, b.z, p, inf_bits, b2);
-                        q.w = bias_round_one<kScale>(v[u].w, b.w, p, inf_bits, b3);
+                        bool ok = inf_bits != 0u;
+                        if (ok) {
+                            q.x = bias_round_fast<kScale>(v[u].x, b.x, p, lo2, span2, ok);
+                            q.y = bias_round_fast<kScale>(v[u].y, b.y, p, lo2, span2, ok);
+                            q.z = bias_round_fast<kScale>(v[u].z, b.z, p, lo2, span2, ok);
+                            q.w = bias_round_fast<kScale>(v[u].w, b.w, p, lo2, span2, ok);
+                            b0 = (int)((q.x >> 23) & 0xFFu) - p.code_off;
+                            b1 = (int)((q.y >> 23) & 0xFFu) - p.code_off;
+                            b2 = (int)((q.z >> 23) & 0xFFu) - p.code_off;
+                            b3 = (int)((q.w >> 23) & 0xFFu) - p.code_off;
+                        }
+                        if (!ok) {
+                            q.x = bias_round_one<kScale>(v[u].x, b.x, p, inf_bits, b0);
+                            q.y = bias_round_one<kScale>(v[u].y, b.y, p, inf_bits, b1);
+                            q.z = bias_round_one<kScale>(v[u].z, b.z, p, inf_bits, b2);
+                            q.w = bias_round_one<kScale>(v[u].w, b.w, p, inf_bits, b3);
+                        }
                         if (kPack) {
                             const uint32_t c0 = encode_container(q.x, b0, p, sign_shift), c1 = encode_container(q.y, b1, p, sign_shift);
                             const uint32_t c2 = encode_container(q.z, b2, p, sign_shift), c3 = encode_container(q.w, b3, p, sign_shift);

@@ -76,3 +76,35 @@ def test_null_format_and_bad_flags(lib):
         == qf.QFMT_ERR_BAD_ARG
     assert lib.qfmt_quantize_stats_host(None, None, 16, ctypes.byref(fmt), None, None, 0, None) == qf.QFMT_ERR_BAD_ARG
     assert qf.qfmt_quantize_stats_host_work_bytes(100) >= 400 + 264 * 8
+
+
+def test_builtin_scratch_refuses_on_the_host_what_does_not_fit(lib):
+    """qfmt_gemm_builtin_scratch answers QFMT_ERR_SCRATCH_LIMIT from host arithmetic alone (no device
+    call has happened yet, so this runs without a GPU) whenever the product's whole workspace --
+    256-byte header included -- exceeds the built-in 16 MiB.  The BERT-large stack has such a product:
+    the out-projection's weight gradient, 1024 x 1024 outputs over K = 8192 tokens, planned in four
+    K splits of 4 MiB each."""
+    limit = 16 << 20
+    fmt = qf.make_format(6, 9)
+    refused = 0
+    # (M, N, K) as op(A) [M x K] = stored [K x M] transposed, B stored [K x N]
+    for M, N, K in ((1024, 1024, 8192), (1024, 2048, 32768), (2048, 2048, 65536), (512, 512, 1 << 20)):
+        a = qf.qfmt_matrix_t(0x10000, K, M, M, 1)
+        b = qf.qfmt_matrix_t(0x20000, K, N, N, 0)
+        need = qf.qfmt_gemm_workspace_bytes(a, b)
+        if need > limit:
+            rc = lib.qfmt_gemm_builtin_scratch(ctypes.byref(a), ctypes.byref(b), ctypes.c_void_p(0x30000), N,
+                                               ctypes.byref(fmt), None, None)
+            assert rc == qf.QFMT_ERR_SCRATCH_LIMIT, (M, N, K, need)
+            refused += 1
+    assert refused >= 1, "no candidate product needs more than the built-in scratch: pick larger ones"
+    # argument errors are reported before the size check and before any device call
+    a = qf.qfmt_matrix_t(0x10000, 8192, 1024, 1024, 1)
+    b = qf.qfmt_matrix_t(0x20000, 8192, 1024, 1024, 0)
+    bad = qf.make_format(6, 11)
+    assert lib.qfmt_gemm_builtin_scratch(ctypes.byref(a), ctypes.byref(b), ctypes.c_void_p(0x30000), 1024,
+                                         ctypes.byref(bad), None, None) == qf.QFMT_ERR_BAD_FORMAT
+    assert lib.qfmt_gemm_builtin_scratch(ctypes.byref(a), ctypes.byref(b), ctypes.c_void_p(0x30000), 512,
+                                         ctypes.byref(fmt), None, None) == qf.QFMT_ERR_BAD_ARG  # ldc < N
+    assert lib.qfmt_gemm_builtin_scratch(ctypes.byref(a), ctypes.byref(b), ctypes.c_void_p(0x30002), 1024,
+                                         ctypes.byref(fmt), None, None) == qf.QFMT_ERR_BAD_ARG  # misaligned C

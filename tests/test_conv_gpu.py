@@ -84,8 +84,16 @@ SMALL = [
 ]
 
 
+@pytest.fixture(params=[0, 1], ids=["cta_pairs", "single_cta"])
+def conv_kernel(request):
+    """Forward and data gradient on both kernels: CTA pairs (the default) and the single-CTA kernel."""
+    qf.qfmt_conv_tile_policy(request.param)
+    yield request.param
+    qf.qfmt_conv_tile_policy(0)
+
+
 @pytest.mark.parametrize("geom", SMALL)
-def test_small_integer_convolutions_are_exact(geom):
+def test_small_integer_convolutions_are_exact(geom, conv_kernel):
     """Entries in -3..3: all sums are small integers, exact in any accumulation order, so a wrong
     tap offset, padding, channel block, transpose or split shows up as a wrong integer."""
     n, ci, h, w, co, r, s, ph, pw = geom
@@ -97,11 +105,12 @@ def test_small_integer_convolutions_are_exact(geom):
     all_three(geom, X, Wt, dY, exact=True)
 
 
-def test_balanced_schedule_is_exact():
-    """163 four-row tiles (the last one three rows) of 27 chunks each on 148 SMs: forward and data
-    gradient deal the K chunks out in equal ranges, so most CTAs finish one tile and begin another,
-    and the pieces that begin inside a tile reach C through the second pass.  Small integers keep
-    every order of summation exact; outputs are sampled because the oracle is slow at this size."""
+def test_balanced_schedule_is_exact(conv_kernel):
+    """163 four-row tiles (the last one three rows) of 27 chunks each: forward and data gradient deal
+    the K chunks out in equal ranges (among 148 CTAs on the single-CTA kernel, among 74 pairs of two
+    tiles on the pair kernel), so most of them finish one tile and begin another, and the pieces that
+    begin inside a tile are added to what another CTA or pair stored.  Small integers keep every
+    order of summation exact; outputs are sampled because the oracle is slow at this size."""
     geom = (21, 192, 31, 32, 192, 3, 3, 1, 1)
     n, ci, h, w, co, r, s, ph, pw = geom
     rng = np.random.default_rng(11)
@@ -120,6 +129,25 @@ def test_format_values_within_bound(geom):
     Wt = workloads.normal_tensor(rng, (co, ci, r, s), 0.05)
     dY = workloads.lognormal_tensor(rng, (n, co, oh, ow), -20.0, 4.0)
     all_three(geom, X, Wt, dY, grad_scale=2.0 ** 10)
+
+
+def test_pair_schedule_on_config4_shape_is_exact_and_reproducible():
+    """The 3 x 3 layer of the ResNet-50-shaped workload (batch 128, 256 -> 256 channels, 14 x 14): 100
+    pair tiles of 36 chunks on 74 pairs, the last conv tile incomplete.  Integers: exact; then real
+    values twice: identical bits."""
+    sh = workloads.CONV3X3
+    geom = (sh.n, sh.c_in, sh.h, sh.w, sh.c_out, sh.r, sh.s, sh.pad, sh.pad)
+    rng = np.random.default_rng(17)
+    X = rng.integers(-2, 3, size=(sh.n, sh.c_in, sh.h, sh.w)).astype(np.float32)
+    Wt = rng.integers(-2, 3, size=(sh.c_out, sh.c_in, sh.r, sh.s)).astype(np.float32)
+    dY = rng.integers(-2, 3, size=(sh.n, sh.c_out, sh.h, sh.w)).astype(np.float32)
+    all_three(geom, X, Wt, dY, exact=True, sample=30000, seed=6)
+    cfg = workloads.config4(sh)
+    fmt = qf.make_format(6, 9, 1)
+    dX, dW = to_channels_last(cfg["X"], fmt), to_channels_last(cfg["W"], fmt)
+    outs = [run_conv(qf.QFMT_CONV_FWD, geom, dX, dW, (sh.n, sh.h, sh.w, sh.c_out), fmt).cpu().numpy() for _ in range(3)]
+    assert np.array_equal(outs[0].view(np.uint32), outs[1].view(np.uint32))
+    assert np.array_equal(outs[0].view(np.uint32), outs[2].view(np.uint32))
 
 
 @pytest.mark.parametrize("shape", [workloads.CONV3X3, workloads.CONV1X1], ids=["3x3", "1x1"])

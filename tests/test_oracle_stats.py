@@ -138,3 +138,19 @@ def test_empty_and_stats_only():
     x = np.array([1.0, 0.0, -0.0, 2.0 ** -35], dtype=np.float32)
     q, st = oracle.quantize_stats(x, 6, 9, want_q=False)
     assert q is None and int(st[oracle.ST_TOTAL]) == 4 and int(st[oracle.ST_DENORMAL]) == 1
+
+
+@pytest.mark.parametrize("threads", [2, 3, 16])
+def test_pieces_in_parallel_equal_the_single_pass(threads):
+    """The all-cores form used for timing (pieces with records of their own, summed) gives the same
+    tensor and the same record as the one-element-at-a-time pass, ragged piece sizes included."""
+    x = workloads.lognormal_tensor(workloads.rng_for(77), (100003,), -25.0, 8.0, p_zero=0.01)
+    x[::977] = np.inf
+    x[5::1013] = np.nan
+    for e, m, den, scale in ((6, 9, 1, 1.0), (5, 10, 0, 2.0 ** 8), (8, 7, 1, 3.0e-5)):
+        q1, s1 = oracle.quantize_stats(x, e, m, den, scale)
+        qt, stt = oracle.quantize_stats(x, e, m, den, scale, threads=threads)
+        assert np.array_equal(q1.view(np.uint32), qt.view(np.uint32))
+        assert np.array_equal(s1, stt)
+    _, s0 = oracle.quantize_stats(x[:5], 6, 9, threads=threads)  # fewer elements than pieces
+    assert int(s0[oracle.ST_TOTAL]) == 5

@@ -70,3 +70,31 @@ def test_argument_errors_enqueue_nothing():
     assert "16 MiB" in qf.qfmt_status_string(qf.QFMT_ERR_SCRATCH_LIMIT)
     torch.cuda.synchronize()
     assert torch.all(d == 1.0)
+
+
+def test_a_product_beyond_the_limit_is_refused_and_nothing_runs():
+    """The BERT-large out-projection's weight gradient (1024 x 1024 outputs over 8192 tokens) is planned
+    with K splits whose partial sums, plus the 256-byte header, exceed the 16 MiB array: the call must
+    say QFMT_ERR_SCRATCH_LIMIT, leave the output and the status word alone, and qfmt_gemm with a
+    caller's workspace must still do the product."""
+    lib = qf.lib()
+    fmt = qf.make_format(6, 9)
+    M = N = 1024
+    K = 8192
+    X = torch.ones(K, M, dtype=torch.float32, device=DEV)
+    G = torch.ones(K, N, dtype=torch.float32, device=DEV)
+    a, b = qf.make_matrix(X, True), qf.make_matrix(G, False)
+    need = qf.qfmt_gemm_workspace_bytes(a, b)
+    if need <= (16 << 20):
+        pytest.skip("this product fits the built-in scratch under the current plan")
+    C = torch.full((M, N), -5.0, dtype=torch.float32, device=DEV)
+    status = torch.full((4,), 77, dtype=torch.int32, device=DEV)
+    rc = lib.qfmt_gemm_builtin_scratch(ctypes.byref(a), ctypes.byref(b), C.data_ptr(), N, ctypes.byref(fmt),
+                                       status.data_ptr(), torch.cuda.current_stream().cuda_stream)
+    assert rc == qf.QFMT_ERR_SCRATCH_LIMIT
+    torch.cuda.synchronize()
+    assert torch.all(C == -5.0) and torch.all(status == 77)
+    ws = torch.zeros(need, dtype=torch.uint8, device=DEV)
+    qf.qfmt_gemm(a, b, C, N, fmt, ws, need)
+    assert qf.qfmt_device_status(ws) == qf.QFMT_OK
+    assert torch.all(C == float(K))
