@@ -852,10 +852,7 @@ static_assert(kPairSmemBytes <= 232448, "pair kernel: shared memory");
 // The two MMA issuers of the pair kernel tell a stage's phases apart without a progress word only
 // when the ring has at least four stages (see the issuer's comment); three stages gave wrong sums.
 static_assert(kPStages >= 4, "pair kernel: at least four stages");
-// kPOutBlocks = 3: three blocks go through the staging area in one copy and the fourth is written from
-// the registers (the staging area for all four does not fit beside four stages, and waiting for the
-// copy engine to have read a smaller area before refilling it costs ~2 k cycles per flush).
-static_assert(4 % kPOutBlocks == 0 || kPOutBlocks == 3, "pair kernel: a warp's four column blocks");
+static_assert(4 % kPOutBlocks == 0, "pair kernel: a warp's four column blocks in whole copies");
 
 // Operand kinds of the pair kernel: fp32 containers read as TF32, or packed 16-bit codes that are
 // binary16 (1/5/10) or bfloat16 (1/8/7) words.  A stage is one 128-byte swizzle row per operand row
@@ -884,9 +881,12 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmap_a, const CUten
     auto empty_bar = [&](int s) { return bars + 8u * (kPStages + s); };
     auto acc_full_bar = [&](int a) { return bars + 8u * (2 * kPStages + a); };
     auto acc_empty_bar = [&](int a) { return bars + 8u * (2 * kPStages + 2 + a); };
+    // balanced schedule: head_bar collects the accumulate warps whose stores of a tile's first piece
+    // are complete, tail_bar tells them that the pair before has stored the first piece of their tile
+    const uint32_t head_bar = bars + 8u * (2 * kPStages + 4), tail_bar = bars + 8u * (2 * kPStages + 5);
     uint8_t* gen_bars = smem_raw + (bars - raw);
-    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen_bars + 8 * (2 * kPStages + 4));
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(gen_bars + 8 * (2 * kPStages + 4) + 8);
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen_bars + 8 * (2 * kPStages + 6));
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(gen_bars + 8 * (2 * kPStages + 6) + 8);
     uint32_t* epi_hist = reinterpret_cast<uint32_t*>(gen_bars + 256);
 
     const int warp = threadIdx.x >> 5;
@@ -906,6 +906,8 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmap_a, const CUten
             ptx::mbar_init(acc_full_bar(a), 1);
             ptx::mbar_init(acc_empty_bar(a), 2 * kAccWarps);
         }
+        ptx::mbar_init(head_bar, kAccWarps);
+        ptx::mbar_init(tail_bar, 1);
         *abort_flag = 0;
         ptx::fence_mbar_init();
         ptx::prefetch_tensormap(&tmap_a);
@@ -1061,6 +1063,45 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmap_a, const CUten
             }
         }
         __syncwarp();
+    } else if (warp == 3 && p.sk_flags != nullptr) {
+        // ------------------------------ balanced schedule: hand-over between pairs ------------------------------
+        // A tile cut by a range boundary is begun by one pair (its last-but-one piece, "head") and
+        // finished by the next (its last piece, which adds at the destination).  This thread passes
+        // the news: once the eight accumulate warps of this CTA have completed their stores of a head
+        // piece it raises this CTA's flag for the next pair; before this CTA's accumulate warps may
+        // add a piece that begins inside a tile it waits for the flag of the pair before.  One word
+        // per pair and CTA rank (the same rank owns the same rows in both pairs).
+        if (lane == 0) {
+            bool dead = false;
+            for (int t = cluster_id; t < num_work && !dead; t += num_clusters) {
+                const WorkItem w = decode_work(p, t);
+                if (w.num_kb <= 0) continue;
+                if (w.head) {
+                    if (!ptx::mbar_wait_bounded(head_bar, 0u, kWaitLimit)) {
+                        raise_timeout(p, abort_flag);
+                        break;
+                    }
+                    ptx::fence_proxy_async_all();
+                    __threadfence();
+                    *reinterpret_cast<volatile int*>(p.sk_flags + ((cluster_id + 1) * 16 + (int)rank)) = 1;
+                }
+                if (w.partial) {
+                    volatile int* flag = p.sk_flags + (cluster_id * 16 + (int)rank);
+                    const long long t_begin = clock64();
+                    while (*flag == 0 && !*abort_flag) {
+                        if (clock64() - t_begin > (long long)kWaitLimit) { dead = true; break; }
+                        __nanosleep(64);
+                    }
+                    if (dead) {
+                        raise_timeout(p, abort_flag);
+                        break;
+                    }
+                    __threadfence();
+                    ptx::mbar_arrive(tail_bar);
+                }
+            }
+        }
+        __syncwarp();
     }
     } else {
         // 128 x 56 + 256 x 224 registers are exactly the 384 x 168 the CTA was launched with; the increase
@@ -1071,145 +1112,98 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmap_a, const CUten
         // ------------------------------ accumulate + epilogue (both CTAs) ------------------------------
         const int quad = warp & 3;
         const int half = (warp - 4) >> 2;
+        const uint32_t my_stage_addr = out_stage + (uint32_t)(warp - 4) * kPOutWarpBytes;
+        float* const my_stage = reinterpret_cast<float*>(smem_raw + (my_stage_addr - raw));
         uint32_t acc_iter = 0;
         bool dead = false;
         for (int t = cluster_id; t < num_work && !dead; t += num_clusters) {
             const WorkItem w = decode_work(p, t);
             constexpr bool kConv = kMode == 1;
             const int cta_rows = kConv ? p.conv_rows : kBM;  // rows of C this CTA owns in the tile
-            const int m0 = w.m0 + (int)rank * cta_rows, n0 = w.n0, num_kb = w.num_kb;
+            const int m0 = w.m0 + (int)rank * cta_rows, n0 = w.n0;
             const int m_end = m0 + cta_rows < p.M ? m0 + cta_rows : p.M;
             float* const c_base = p.C + (long long)w.split * p.split_stride;
             const bool use_tma = p.tma_store != 0;
-            // level-1 running sums, two per 64-bit register (packed adds); 0 + x is exact, so a group's
-            // first chunk needs no special case
-            unsigned long long sum2[64];
-#pragma unroll
-            for (int j = 0; j < 64; ++j) sum2[j] = 0ull;
-            const uint32_t my_stage_addr = out_stage + (uint32_t)(warp - 4) * kPOutWarpBytes;
-            float* my_stage = reinterpret_cast<float*>(smem_raw + (my_stage_addr - raw));
             const int row0 = m0 + quad * 32;
-            int in_group = 0;
             // a piece that begins inside its tile adds to what the pair before has stored there
             bool flushed = w.partial != 0;
-            bool handed_over = w.partial == 0;  // the first part of the tile is known to be in C
-            for (int kb0 = 0; kb0 < num_kb; kb0 += kChunkKB) {
-                const uint32_t acc = acc_iter & 1u, acc_phase = (acc_iter >> 1) & 1u;
-                bool ok = true;
-                if (lane == 0) ok = ptx::mbar_wait_bounded(acc_full_bar(acc), acc_phase, kWaitLimit);
-                ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0;
-                if (!ok) {
-                    if (lane == 0) raise_timeout(p, abort_flag);
-                    dead = true;
-                    break;
-                }
-                if (*abort_flag) { dead = true; break; }
-                ptx::tc_fence_after_sync();
-                const uint32_t tbase = tmem_base + ((uint32_t)(quad * 32) << 16) + acc * kAccCols + (uint32_t)half * 128u;
+            // The piece's chunks in groups of kFlushChunks: a group's chunk sums are added up in registers
+            // (the inner loop holds nothing else), then the group moves to C.
+            const int chunks = (w.num_kb + kChunkKB - 1) / kChunkKB;
+            for (int c0 = 0; c0 < chunks; c0 += kFlushChunks) {
+                // level-1 running sums, two per 64-bit register (packed adds); 0 + x is exact, so a group's
+                // first chunk needs no special case
+                unsigned long long sum2[64];
 #pragma unroll
-                for (int pair = 0; pair < 2; ++pair) {
-                    uint32_t ra[32], rb[32];
-                    ptx::tmem_load_32cols(tbase + pair * 64, ra);
-                    ptx::tmem_load_32cols(tbase + pair * 64 + 32, rb);
-                    ptx::tmem_load_wait();
-                    if (pair == 1) {
-                        ptx::tc_fence_before_sync();
-                        __syncwarp();
-                        if (lane == 0) ptx::mbar_arrive_cluster(ptx::map_to_cta(acc_empty_bar(acc), 0));
+                for (int j = 0; j < 64; ++j) sum2[j] = 0ull;
+                const int c1 = c0 + kFlushChunks < chunks ? c0 + kFlushChunks : chunks;
+                for (int c = c0; c < c1; ++c) {
+                    const uint32_t acc = acc_iter & 1u, acc_phase = (acc_iter >> 1) & 1u;
+                    bool ok = true;
+                    if (lane == 0) ok = ptx::mbar_wait_bounded(acc_full_bar(acc), acc_phase, kWaitLimit);
+                    ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0;
+                    if (!ok) {
+                        if (lane == 0) raise_timeout(p, abort_flag);
+                        dead = true;
+                        break;
                     }
+                    if (*abort_flag) { dead = true; break; }
+                    ptx::tc_fence_after_sync();
+                    const uint32_t tbase = tmem_base + ((uint32_t)(quad * 32) << 16) + acc * kAccCols + (uint32_t)half * 128u;
 #pragma unroll
-                    for (int j = 0; j < 32; j += 2) {
-                        ptx::add2_rn(sum2[pair * 32 + j / 2], ra[j], ra[j + 1]);
-                        ptx::add2_rn(sum2[pair * 32 + 16 + j / 2], rb[j], rb[j + 1]);
+                    for (int pair = 0; pair < 2; ++pair) {
+                        uint32_t ra[32], rb[32];
+                        ptx::tmem_load_32cols(tbase + pair * 64, ra);
+                        ptx::tmem_load_32cols(tbase + pair * 64 + 32, rb);
+                        ptx::tmem_load_wait();
+                        if (pair == 1) {
+                            ptx::tc_fence_before_sync();
+                            __syncwarp();
+                            if (lane == 0) ptx::mbar_arrive_cluster(ptx::map_to_cta(acc_empty_bar(acc), 0));
+                        }
+#pragma unroll
+                        for (int j = 0; j < 32; j += 2) {
+                            ptx::add2_rn(sum2[pair * 32 + j / 2], ra[j], ra[j + 1]);
+                            ptx::add2_rn(sum2[pair * 32 + 16 + j / 2], rb[j], rb[j + 1]);
+                        }
                     }
+                    ++acc_iter;
                 }
-                ++acc_iter;
-                const bool last = kb0 + kChunkKB >= num_kb;
-                if (!last && ++in_group < kFlushChunks) continue;
+                if (dead) break;
+                // ---- the group's sums move to C: registers -> swizzled staging -> TMA (stored for the
+                // first group of a tile, added at the destination for later ones)
                 if (kEpi)
                     epi_transform(sum2, p, row0 + lane < m_end, n0 + half * 128, reinterpret_cast<uint32_t*>(my_stage), epi_hist, lane);
-                if (!handed_over) {
-                    // wait (bounded) until the same warp of the pair before this one has completed its
-                    // stores to this patch of the tile
-                    int seen = 1;
-                    if (lane == 0) {
-                        volatile int* flag = p.sk_flags + (cluster_id * 16 + (int)rank * 8 + (warp - 4));
-                        const long long t_begin = clock64();
-                        while (*flag == 0) {
-                            if (clock64() - t_begin > (long long)kWaitLimit) { seen = 0; break; }
-                            __nanosleep(64);
-                        }
-                        __threadfence();
-                        ptx::fence_proxy_async_all();
-                    }
-                    seen = __shfl_sync(0xFFFFFFFFu, seen, 0);
+                if (w.partial && c0 == 0) {
+                    // the pair before this one has stored the first piece of this tile (warp 3 watches its flag)
+                    bool seen = true;
+                    if (lane == 0) seen = ptx::mbar_wait_bounded(tail_bar, 0u, kWaitLimit);
+                    seen = __shfl_sync(0xFFFFFFFFu, seen ? 1 : 0, 0) != 0;
                     if (!seen) {
                         if (lane == 0) raise_timeout(p, abort_flag);
                         dead = true;
                         break;
                     }
-                    handed_over = true;
                 }
                 if (use_tma && flushed) {
-                    if (lane == 0) ptx::bulk_wait_all();
+                    if (lane == 0) ptx::bulk_wait_all();  // the earlier store/add to these addresses is complete
                 }
-                if (kPOutBlocks == 3 && p.c_blocked) {
-                    if (lane == 0) ptx::bulk_wait_read_all();  // the previous flush's copy has read the staging area
-                    __syncwarp();
-#pragma unroll
-                    for (int blk = 0; blk < 3; ++blk) {
-                        float* box = my_stage + blk * 1024;
-#pragma unroll
-                        for (int c = 0; c < 8; ++c) {
-                            const int j = blk * kOutCols + c * 4;
-                            const float2 v0 = ptx::unpack2(sum2[j / 2]), v1 = ptx::unpack2(sum2[j / 2 + 1]);
-                            *reinterpret_cast<float4*>(box + lane * 32 + ((c ^ (lane & 7)) << 2)) =
-                                make_float4(v0.x, v0.y, v1.x, v1.y);
-                        }
-                    }
-                    ptx::fence_proxy_async();
-                    __syncwarp();
-                    if (lane == 0) {
-                        const int cblk = (n0 + half * 128) >> 5;
-                        if (row0 < m_end && cblk * 32 < p.N) {
-                            // convolution: the CTA's own tile of the per-tile map (or the map of the incomplete last tile)
-                            const int ctile = 2 * w.tile_m + (int)rank;
-                            const bool whole = !kConv || ctile < p.full_tiles_m;
-                            const CUtensorMap* cm = whole ? &tmap_c : tmap_c2;
-                            const int ry = kConv ? quad * 32 : row0, rz = kConv ? (whole ? ctile : 0) : w.split;
-                            if (flushed) ptx::tma_reduce_add_4d(cm, my_stage_addr, 0, ry, cblk, rz);
-                            else ptx::tma_store_4d(cm, my_stage_addr, 0, ry, cblk, rz);
-                        }
-                        ptx::bulk_commit();
-                    }
-                    // fourth block: each lane writes its row's 32 columns (128 bytes) itself
-                    const int col3 = n0 + half * 128 + 3 * kOutCols;
-                    if (row0 + lane < m_end && col3 < p.N) {
-                        float* g = c_base + (long long)(row0 + lane) * p.ldc + col3;
-#pragma unroll
-                        for (int c = 0; c < 8; ++c) {
-                            const int j = 3 * kOutCols + c * 4;
-                            const float2 v0 = ptx::unpack2(sum2[j / 2]), v1 = ptx::unpack2(sum2[j / 2 + 1]);
-                            if (flushed) ptx::red_add_v4(g + c * 4, v0.x, v0.y, v1.x, v1.y);
-                            else *reinterpret_cast<float4*>(g + c * 4) = make_float4(v0.x, v0.y, v1.x, v1.y);
-                        }
-                    }
-                } else if (p.c_blocked) {
+                if (p.c_blocked) {
                     // Whole copies of kPOutBlocks column blocks: the staging area is filled (each 32 x 32 block
                     // in the swizzled layout of a one-block box), then ONE copy instruction stores it or adds
                     // it at the destination.  Blocks past N and rows past M are clipped by the copy engine.
 #pragma unroll
-                    for (int pass = 0; pass < (kPOutBlocks == 3 ? 0 : 4 / kPOutBlocks); ++pass) {
+                    for (int pass = 0; pass < 4 / kPOutBlocks; ++pass) {
                         if (lane == 0) ptx::bulk_wait_read_all();  // the previous copy has read the staging area
                         __syncwarp();
 #pragma unroll
                         for (int blk = 0; blk < kPOutBlocks; ++blk) {
                             float* box = my_stage + blk * 1024;
 #pragma unroll
-                            for (int c = 0; c < 8; ++c) {
-                                const int j = (pass * kPOutBlocks + blk) * kOutCols + c * 4;
+                            for (int cc = 0; cc < 8; ++cc) {
+                                const int j = (pass * kPOutBlocks + blk) * kOutCols + cc * 4;
                                 const float2 v0 = ptx::unpack2(sum2[j / 2]), v1 = ptx::unpack2(sum2[j / 2 + 1]);
-                                *reinterpret_cast<float4*>(box + lane * 32 + ((c ^ (lane & 7)) << 2)) =
+                                *reinterpret_cast<float4*>(box + lane * 32 + ((cc ^ (lane & 7)) << 2)) =
                                     make_float4(v0.x, v0.y, v1.x, v1.y);
                             }
                         }
@@ -1218,6 +1212,7 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmap_a, const CUten
                         if (lane == 0) {
                             const int cblk = ((n0 + half * 128) >> 5) + pass * kPOutBlocks;
                             if (row0 < m_end && cblk * 32 < p.N) {
+                                // convolution: the CTA's own tile of the per-tile map (or the map of the incomplete last tile)
                                 const int ctile = 2 * w.tile_m + (int)rank;
                                 const bool whole = !kConv || ctile < p.full_tiles_m;
                                 const CUtensorMap* cm = whole ? &tmap_c : tmap_c2;
@@ -1225,64 +1220,57 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmap_a, const CUten
                                 if (flushed) ptx::tma_reduce_add_4d(cm, my_stage_addr, 0, ry, cblk, rz);
                                 else ptx::tma_store_4d(cm, my_stage_addr, 0, ry, cblk, rz);
                             }
-                            ptx::bulk_commit();
+                            ptx::bulk_commit();  // committed even when empty: the waits count groups
                         }
                     }
-                } else
+                } else {
 #pragma unroll
-                for (int pass = 0; pass < 4; ++pass) {
-                    const int col0 = n0 + half * 128 + pass * kOutCols;
-                    float* box = my_stage + (pass & 1) * 1024;
-                    if (lane == 0) ptx::bulk_wait_read_1();
-                    __syncwarp();
+                    for (int pass = 0; pass < 4; ++pass) {
+                        const int col0 = n0 + half * 128 + pass * kOutCols;
+                        float* box = my_stage + (pass & 1) * 1024;
+                        if (lane == 0) ptx::bulk_wait_read_1();  // at most the newest copy (it reads the other box) may still be reading
+                        __syncwarp();
 #pragma unroll
-                    for (int c = 0; c < 8; ++c) {
-                        const int j = pass * kOutCols + c * 4;
-                        const float2 v0 = ptx::unpack2(sum2[j / 2]), v1 = ptx::unpack2(sum2[j / 2 + 1]);
-                        *reinterpret_cast<float4*>(box + lane * 32 + ((c ^ (lane & 7)) << 2)) =
-                            make_float4(v0.x, v0.y, v1.x, v1.y);
-                    }
-                    if (use_tma) {
-                        ptx::fence_proxy_async();
-                        __syncwarp();
-                        if (lane == 0) {
-                            if (row0 < m_end && col0 < p.N) {
-                                const uint32_t src = my_stage_addr + (pass & 1) * kOutBoxBytes;
-                                if (flushed) ptx::tma_reduce_add_3d(&tmap_c, src, col0, row0, w.split);
-                                else ptx::tma_store_3d(&tmap_c, src, col0, row0, w.split);
-                            }
-                            ptx::bulk_commit();
+                        for (int cc = 0; cc < 8; ++cc) {
+                            const int j = pass * kOutCols + cc * 4;
+                            const float2 v0 = ptx::unpack2(sum2[j / 2]), v1 = ptx::unpack2(sum2[j / 2 + 1]);
+                            *reinterpret_cast<float4*>(box + lane * 32 + ((cc ^ (lane & 7)) << 2)) =
+                                make_float4(v0.x, v0.y, v1.x, v1.y);
                         }
-                    } else {
-                        __syncwarp();
-                        for (int r = 0; r < 32; ++r) {
-                            const int row = row0 + r;
-                            if (row >= m_end) break;
-                            const int c = lane;
-                            if (col0 + c < p.N) {
-                                float* g = c_base + (long long)row * p.ldc + col0 + c;
-                                const float v = box[r * 32 + (((c >> 2) ^ (r & 7)) << 2) + (c & 3)];
-                                *g = flushed ? __fadd_rn(*g, v) : v;
+                        if (use_tma) {
+                            ptx::fence_proxy_async();
+                            __syncwarp();
+                            if (lane == 0) {
+                                if (row0 < m_end && col0 < p.N) {
+                                    const uint32_t src = my_stage_addr + (pass & 1) * kOutBoxBytes;
+                                    if (flushed) ptx::tma_reduce_add_3d(&tmap_c, src, col0, row0, w.split);
+                                    else ptx::tma_store_3d(&tmap_c, src, col0, row0, w.split);
+                                }
+                                ptx::bulk_commit();
                             }
+                        } else {
+                            __syncwarp();
+                            for (int r = 0; r < 32; ++r) {
+                                const int row = row0 + r;
+                                if (row >= m_end) break;
+                                if (col0 + lane < p.N) {
+                                    float* g = c_base + (long long)row * p.ldc + col0 + lane;
+                                    const float v = box[r * 32 + (((lane >> 2) ^ (r & 7)) << 2) + (lane & 3)];
+                                    *g = flushed ? __fadd_rn(*g, v) : v;
+                                }
+                            }
+                            __syncwarp();
                         }
-                        __syncwarp();
                     }
                 }
                 flushed = true;
-                in_group = 0;
-                if (!last) {
-#pragma unroll
-                    for (int j = 0; j < 64; ++j) sum2[j] = 0ull;
-                }
             }
             if (dead) break;
-            if (w.head && num_kb > 0) {
-                // this warp's part of the tile's first piece is in C: tell the pair that adds the rest
+            if (w.head && chunks > 0) {
+                // this warp's part of the tile's first piece is in C (its copies have completed)
                 if (lane == 0) {
                     ptx::bulk_wait_all();
-                    ptx::fence_proxy_async_all();
-                    __threadfence();
-                    *reinterpret_cast<volatile int*>(p.sk_flags + ((cluster_id + 1) * 16 + (int)rank * 8 + (warp - 4))) = 1;
+                    ptx::mbar_arrive(head_bar);
                 }
                 __syncwarp();
             }

@@ -294,10 +294,6 @@ __device__ __forceinline__ void add2_rn(unsigned long long& acc, uint32_t lo, ui
     // volatile: keeps the add behind the tcgen05.wait::ld that makes lo and hi valid
     asm volatile("{\n\t.reg .b64 t;\n\tmov.b64 t, {%1, %2};\n\tadd.rn.f32x2 %0, %0, t;\n\t}" : "+l"(acc) : "r"(lo), "r"(hi));
 }
-// Four fp32 additions at the destination (16 bytes, 16-byte aligned), no value returned.
-__device__ __forceinline__ void red_add_v4(float* p, float a, float b, float c, float d) {
-    asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(p), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
-}
 __device__ __forceinline__ float2 unpack2(unsigned long long v) {
     float2 r;
     asm("mov.b64 {%0, %1}, %2;" : "=f"(r.x), "=f"(r.y) : "l"(v));

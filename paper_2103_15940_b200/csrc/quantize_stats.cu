@@ -207,7 +207,9 @@ quantize_stats_transpose_kernel(const uint32_t* __restrict__ in, uint32_t* __res
 // bandwidth): the rounding pass writing packed codes instead of fp32 containers, 4 bytes read and
 // 2 written per element, and the pass that expands codes back to containers for the contraction.
 // A thread takes eight consecutive elements: two 128-bit loads, one 128-bit store.
-template <bool kStats, bool kScale>
+// kRare: results below the smallest normal are expected to be rare (formats with e >= 6): the denormal
+// grid sits behind a branch (quantize_pack_one_rare_denormals).
+template <bool kStats, bool kScale, bool kRare>
 __global__ void __launch_bounds__(kThreads)
 quantize_stats_pack16_kernel(const uint32_t* __restrict__ in, uint16_t* __restrict__ codes, unsigned long long n,
                              int vec, QuantParams p, int sign_shift, qfmt_stats_t* __restrict__ stats) {
@@ -239,7 +241,8 @@ quantize_stats_pack16_kernel(const uint32_t* __restrict__ in, uint16_t* __restri
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
                     int b;
-                    c[j] = quantize_pack_one<kScale>(w[j], p, sign_shift, b);
+                    c[j] = kRare ? quantize_pack_one_rare_denormals<kScale>(w[j], p, sign_shift, b)
+                                 : quantize_pack_one<kScale>(w[j], p, sign_shift, b);
                     if (kStats) atomicAdd(&lane_hist[b * 32 + lane], 1u);
                 }
                 store_stream(reinterpret_cast<uint4*>(codes) + idx,
@@ -252,7 +255,8 @@ quantize_stats_pack16_kernel(const uint32_t* __restrict__ in, uint16_t* __restri
     for (unsigned long long i = done + (unsigned long long)blockIdx.x * kThreads + threadIdx.x; i < n;
          i += (unsigned long long)gridDim.x * kThreads) {
         int b;
-        codes[i] = (uint16_t)quantize_pack_one<kScale>(in[i], p, sign_shift, b);
+        codes[i] = (uint16_t)(kRare ? quantize_pack_one_rare_denormals<kScale>(in[i], p, sign_shift, b)
+                                    : quantize_pack_one<kScale>(in[i], p, sign_shift, b));
         if (kStats) atomicAdd(&lane_hist[b * 32 + lane], 1u);
     }
     if (kStats) {
@@ -477,8 +481,14 @@ bias_quantize_stats_kernel(const uint32_t* acc, long long ld_acc, const uint32_t
                             q.w = bias_round_one<kScale>(v[u].w, b.w, p, inf_bits, b3);
                         }
                         if (kPack) {
-                            const uint32_t c0 = encode_container(q.x, b0, p, sign_shift), c1 = encode_container(q.y, b1, p, sign_shift);
-                            const uint32_t c2 = encode_container(q.z, b2, p, sign_shift), c3 = encode_container(q.w, b3, p, sign_shift);
+                            uint32_t c0, c1, c2, c3;
+                            if (ok) {  // four normal results: re-biased fields shifted down, sign bit moved beside them
+                                c0 = encode_normal(q.x, p, sign_shift); c1 = encode_normal(q.y, p, sign_shift);
+                                c2 = encode_normal(q.z, p, sign_shift); c3 = encode_normal(q.w, p, sign_shift);
+                            } else {
+                                c0 = encode_container(q.x, b0, p, sign_shift); c1 = encode_container(q.y, b1, p, sign_shift);
+                                c2 = encode_container(q.z, b2, p, sign_shift); c3 = encode_container(q.w, b3, p, sign_shift);
+                            }
                             store_stream(po16 + u * step_o, make_uint2(c0 | (c1 << 16), c2 | (c3 << 16)));
                         } else {
                             store_stream(po + u * step_o, q);
@@ -760,9 +770,16 @@ int quantize_stats_pack16_device(const float* d_in, uint16_t* d_codes, size_t n,
     if (want > cap) want = cap;
     const uint32_t* in = reinterpret_cast<const uint32_t*>(d_in);
     const int sign_shift = fmt->e + fmt->m;
-#define QFMT_PLAUNCH(S, C)                                                                                  \
-    quantize_stats_pack16_kernel<S, C><<<(unsigned)want, kThreads, smem, stream>>>(in, d_codes, n, vec, p,  \
-                                                                                    sign_shift, d_stats)
+    // 1/5/m tensors of small gradients are mostly denormal (the paper's observation on binary16), so
+    // only wider exponents take the kernel that branches on results below the smallest normal
+    const bool rare = fmt->e >= 6;
+#define QFMT_PLAUNCH(S, C)                                                                                         \
+    do {                                                                                                           \
+        if (rare) quantize_stats_pack16_kernel<S, C, true><<<(unsigned)want, kThreads, smem, stream>>>(            \
+                      in, d_codes, n, vec, p, sign_shift, d_stats);                                                \
+        else quantize_stats_pack16_kernel<S, C, false><<<(unsigned)want, kThreads, smem, stream>>>(               \
+                      in, d_codes, n, vec, p, sign_shift, d_stats);                                                \
+    } while (0)
     if (has_stats) { if (has_scale) QFMT_PLAUNCH(true, true); else QFMT_PLAUNCH(true, false); }
     else { if (has_scale) QFMT_PLAUNCH(false, true); else QFMT_PLAUNCH(false, false); }
 #undef QFMT_PLAUNCH

@@ -154,6 +154,42 @@ __device__ __forceinline__ uint32_t quantize_pack_one(uint32_t xb, const QuantPa
     return sign | packed;
 }
 
+// The same with the denormal grid behind a branch, for tensors in which results below the smallest
+// normal are rare (what the paper reports for 1/6/9 and what holds for 1/8/7): the common path is the
+// rounding of the word and its re-biased fields only.  If the word's own rounding already reaches a
+// normal binade the result is that rounding (for inputs just below 2^E_min both grids give 2^E_min);
+// otherwise the input is rounded onto multiples of 2^(E_min-m), and that multiple IS the packed code:
+// 2^m, the smallest normal, when the rounding carries.
+template <bool kScale>
+__device__ __forceinline__ uint32_t quantize_pack_one_rare_denormals(uint32_t xb, const QuantParams& p, int sign_shift,
+                                                                     int& bin) {
+    const uint32_t yb = kScale ? __float_as_uint(mul_ieee(__uint_as_float(xb), p.scale)) : xb;
+    const uint32_t a = yb & 0x7FFFFFFFu;
+    const uint32_t qn = (a + p.round_add + ((a >> p.drop) & p.lsb_mask)) & p.keep_mask;
+    const int code = (int)(qn >> 23) - p.code_off;
+    const int m = 23 - (int)p.drop;
+    uint32_t packed = (qn - ((uint32_t)p.code_off << 23)) >> p.drop;
+    bin = code;
+    if ((unsigned)(code - 1) >= (unsigned)(p.top - 1)) {
+        const uint32_t ax = xb & 0x7FFFFFFFu;
+        if (code >= p.top) {  // overflow, infinite or NaN
+            const bool is_nan = ax > 0x7F800000u;
+            packed = ((uint32_t)p.top << m) | (is_nan ? (1u << (m - 1)) : 0u);
+            bin = p.top + (is_nan ? kBinNanIn : (ax == 0x7F800000u ? kBinInfIn : kBinOverflow));
+        } else {              // below the smallest normal: the denormal grid
+            const uint32_t cnt = __float_as_uint(add_ieee(__uint_as_float(a), __uint_as_float(p.magic))) - p.magic;
+            if (cnt >> m) {   // carried to 2^E_min
+                packed = cnt;
+                bin = 1;
+            } else {
+                bin = p.top + (ax == 0u ? kBinZeroIn : (cnt == 0u ? kBinRoundedToZero : kBinDenormal));
+                packed = p.keep_denormals ? cnt : 0u;
+            }
+        }
+    }
+    return ((xb >> 31) << sign_shift) | packed;
+}
+
 // Packed code of a value that already lies on the format's grid (container bits q as the rounding
 // functions return them: finite format values, +-inf, or a NaN).
 __device__ __forceinline__ uint32_t encode_container(uint32_t q, const QuantParams& p, int sign_shift) {
@@ -175,6 +211,15 @@ __device__ __forceinline__ uint32_t encode_container(uint32_t q, int bin, const 
         return packed | ((uint32_t)((int32_t)q >> 31) & (1u << sign_shift));
     }
     return encode_container(q, p, sign_shift);
+}
+
+// Packed code of a normal value of the format (container bits q, sign included): subtracting the
+// exponent re-bias leaves the sign bit alone, the shift brings exponent and mantissa fields down, and
+// the sign is taken from a second shift of the word (bits above the sign position are empty there).
+__device__ __forceinline__ uint32_t encode_normal(uint32_t q, const QuantParams& p, int sign_shift) {
+    const uint32_t low = (1u << sign_shift) - 1u;
+    const uint32_t fields = (q - ((uint32_t)p.code_off << 23)) >> p.drop;
+    return (fields & low) | ((q >> (31 - sign_shift)) & ~low);
 }
 
 // fp32 container of a packed code.
