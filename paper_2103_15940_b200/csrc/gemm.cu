@@ -188,32 +188,11 @@ __host__ __device__ __forceinline__ void sk_range(long long total, int ctas, int
     *lo = total * b / ctas;
     *hi = total * (b + 1) / ctas;
 }
-// Balanced schedule of the pair kernel: t = pair + piece * pairs.  Kept out of line: it runs once per
-// piece, and inlined into the producer's, the issuers' and the accumulate warps' loops it cost them
-// registers they need (measured: every product 12 % slower).
-__device__ __noinline__ int4 decode_work_pairs(int q, int r, int cpt, int kb_total, int t) {
-    const int units = (int)(gridDim.x >> 1);
-    const PairPiece pc = pair_piece(q, r, cpt, kb_total, units, t % units, t / units);
-    return make_int4(pc.tile, pc.kb_begin, pc.num_kb, pc.partial | (pc.head << 1));
-}
 __device__ __forceinline__ WorkItem decode_work(const GemmParams& p, int t) {
     WorkItem w;
     const int num_tiles = p.tiles_m * p.tiles_n;
     w.partial = 0;
     w.head = 0;
-    if (p.sk_flags != nullptr) {
-        const int4 pc = decode_work_pairs(p.sk_q, p.sk_r, p.sk_cpt, p.kb_total, t);
-        w.split = 0;
-        w.tile_m = pc.x % p.tiles_m;
-        w.tile_n = pc.x / p.tiles_m;
-        w.m0 = w.tile_m * p.tile_rows;
-        w.n0 = w.tile_n * kBN;
-        w.kb_begin = pc.y;
-        w.num_kb = pc.z;
-        w.partial = pc.w & 1;
-        w.head = pc.w >> 1;
-        return w;
-    }
     if (p.sk_cpt > 0) {
         // t = b + piece * gridDim.x for CTA b
         const int ctas = (int)gridDim.x, b = t % ctas, piece = t / ctas;
@@ -847,7 +826,11 @@ constexpr uint32_t kPStageBytes = kPABytes + kPBBytes;
 constexpr int kPOutBlocks = QFMT_POUT_BLOCKS;
 constexpr uint32_t kPOutWarpBytes = (kPOutBlocks * kOutBoxBytes > kOutWarpBytes) ? kPOutBlocks * kOutBoxBytes : kOutWarpBytes;
 constexpr uint32_t kPOutBytes = kAccWarps * kPOutWarpBytes;
-constexpr uint32_t kPairSmemBytes = kPStages * kPStageBytes + kPOutBytes + 1024 + 256 + kEpiHistBytes;
+// Balanced schedule: a pair's pieces (at most kMaxSkPieces) are worked out once, by the first threads of
+// each CTA, into a table in shared memory that every role then reads.
+constexpr int kMaxSkPieces = 64;
+constexpr uint32_t kSkTableBytes = kMaxSkPieces * 16;
+constexpr uint32_t kPairSmemBytes = kPStages * kPStageBytes + kPOutBytes + 1024 + 256 + kEpiHistBytes + kSkTableBytes;
 static_assert(kPairSmemBytes <= 232448, "pair kernel: shared memory");
 // The two MMA issuers of the pair kernel tell a stage's phases apart without a progress word only
 // when the ring has at least four stages (see the issuer's comment); three stages gave wrong sums.
@@ -869,7 +852,9 @@ __device__ __forceinline__ uint32_t make_idesc_pair(int a_mn, int b_mn, int kind
 // half of the 256 filter columns; its pixel operand arrives as one box per image touched from
 // row_maps, C is written through tmap_c ({32, conv_rows, N / 32, complete tiles}: rows past the tile
 // are clipped) or, for the incomplete last tile, tmap_c2.
-template <bool kEpi, int kKind, int kMode>
+// kSk: the balanced schedule (GemmParams::sk_flags) is compiled in; products that do not use it run an
+// instantiation without any of its code.
+template <bool kEpi, int kKind, int kMode, bool kSk>
 __device__ __forceinline__ void pair_body(const CUtensorMap& tmap_a, const CUtensorMap& tmap_b, const CUtensorMap& tmap_c,
                                           const CUtensorMap* tmap_c2, const CUtensorMap* row_maps, const GemmParams& p) {
     extern __shared__ uint8_t smem_raw[];
@@ -888,6 +873,7 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmap_a, const CUten
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen_bars + 8 * (2 * kPStages + 6));
     volatile int* abort_flag = reinterpret_cast<volatile int*>(gen_bars + 8 * (2 * kPStages + 6) + 8);
     uint32_t* epi_hist = reinterpret_cast<uint32_t*>(gen_bars + 256);
+    int4* const sk_table = reinterpret_cast<int4*>(gen_bars + 256 + kEpiHistBytes);
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -896,6 +882,13 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmap_a, const CUten
         for (int i = threadIdx.x; i < kEpiBins; i += kThreads) epi_hist[i] = 0u;
     }
     const int cluster_id = blockIdx.x >> 1, num_clusters = gridDim.x >> 1;
+    if (kSk) {
+        // piece j of this pair: {tile, first stage, stages, partial | head << 1}
+        if ((int)threadIdx.x < p.sk_pieces) {
+            const PairPiece pc = pair_piece(p.sk_q, p.sk_r, p.sk_cpt, p.kb_total, num_clusters, cluster_id, (int)threadIdx.x);
+            sk_table[threadIdx.x] = make_int4(pc.tile, pc.kb_begin, pc.num_kb, pc.partial | (pc.head << 1));
+        }
+    }
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kPStages; ++s) {
@@ -923,7 +916,27 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmap_a, const CUten
     ptx::cluster_sync();  // the peer's barriers exist before anything is signalled to them
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
-    const int num_work = p.sk_flags != nullptr ? p.sk_pieces * num_clusters : p.tiles_m * p.tiles_n * p.splits;
+    // work items of this pair: its pieces under the balanced schedule (t = 0, 1, ...), else every
+    // num_clusters-th tile (t = cluster_id, cluster_id + num_clusters, ...)
+    const int t_begin = kSk ? 0 : cluster_id, t_step = kSk ? 1 : num_clusters;
+    const int t_end = kSk ? p.sk_pieces : p.tiles_m * p.tiles_n * p.splits;
+    auto work_item = [&](int j) -> WorkItem {
+        if (kSk) {
+            const int4 e = sk_table[j];
+            WorkItem w;
+            w.split = 0;
+            w.tile_m = e.x % p.tiles_m;
+            w.tile_n = e.x / p.tiles_m;
+            w.m0 = w.tile_m * p.tile_rows;
+            w.n0 = w.tile_n * kBN;
+            w.kb_begin = e.y;
+            w.num_kb = e.z;
+            w.partial = e.w & 1;
+            w.head = e.w >> 1;
+            return w;
+        }
+        return decode_work(p, j);
+    };
 
     if (warp < 4) {
     ptx::setmaxnreg_dec<56>();
@@ -932,8 +945,8 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmap_a, const CUten
         if (lane == 0) {
             int stage = 0;
             uint32_t phase = 0;
-            for (int t = cluster_id; t < num_work && !*abort_flag; t += num_clusters) {
-                const WorkItem w = decode_work(p, t);
+            for (int t = t_begin; t < t_end && !*abort_flag; t += t_step) {
+                const WorkItem w = work_item(t);
                 const int m0 = w.m0 + (int)rank * kBM, n0 = w.n0 + (int)rank * (kBN / 2);
                 for (int kb = w.kb_begin; kb < w.kb_begin + w.num_kb; ++kb) {
                     if (!ptx::mbar_wait_bounded(empty_bar(stage), phase ^ 1u, kWaitLimit)) {
@@ -1022,8 +1035,8 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmap_a, const CUten
             uint32_t phase = 0;
             uint32_t acc_iter = 0;
             bool dead = false;
-            for (int t = cluster_id; t < num_work && !dead; t += num_clusters) {
-                const int num_kb = decode_work(p, t).num_kb;
+            for (int t = t_begin; t < t_end && !dead; t += t_step) {
+                const int num_kb = kSk ? sk_table[t].z : decode_work(p, t).num_kb;
                 for (int kb0 = 0; kb0 < num_kb && !dead; kb0 += kChunkKB, ++acc_iter) {
                     const uint32_t acc = acc_iter & 1u, acc_phase = (acc_iter >> 1) & 1u;
                     if (acc != who) {  // the other issuer's chunk: step over its stages
@@ -1063,7 +1076,7 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmap_a, const CUten
             }
         }
         __syncwarp();
-    } else if (warp == 3 && p.sk_flags != nullptr) {
+    } else if (kSk && warp == 3) {
         // ------------------------------ balanced schedule: hand-over between pairs ------------------------------
         // A tile cut by a range boundary is begun by one pair (its last-but-one piece, "head") and
         // finished by the next (its last piece, which adds at the destination).  This thread passes
@@ -1073,8 +1086,8 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmap_a, const CUten
         // per pair and CTA rank (the same rank owns the same rows in both pairs).
         if (lane == 0) {
             bool dead = false;
-            for (int t = cluster_id; t < num_work && !dead; t += num_clusters) {
-                const WorkItem w = decode_work(p, t);
+            for (int t = t_begin; t < t_end && !dead; t += t_step) {
+                const WorkItem w = work_item(t);
                 if (w.num_kb <= 0) continue;
                 if (w.head) {
                     if (!ptx::mbar_wait_bounded(head_bar, 0u, kWaitLimit)) {
@@ -1116,8 +1129,8 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmap_a, const CUten
         float* const my_stage = reinterpret_cast<float*>(smem_raw + (my_stage_addr - raw));
         uint32_t acc_iter = 0;
         bool dead = false;
-        for (int t = cluster_id; t < num_work && !dead; t += num_clusters) {
-            const WorkItem w = decode_work(p, t);
+        for (int t = t_begin; t < t_end && !dead; t += t_step) {
+            const WorkItem w = work_item(t);
             constexpr bool kConv = kMode == 1;
             const int cta_rows = kConv ? p.conv_rows : kBM;  // rows of C this CTA owns in the tile
             const int m0 = w.m0 + (int)rank * cta_rows, n0 = w.n0;
@@ -1126,7 +1139,7 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmap_a, const CUten
             const bool use_tma = p.tma_store != 0;
             const int row0 = m0 + quad * 32;
             // a piece that begins inside its tile adds to what the pair before has stored there
-            bool flushed = w.partial != 0;
+            bool flushed = kSk && w.partial != 0;
             // The piece's chunks in groups of kFlushChunks: a group's chunk sums are added up in registers
             // (the inner loop holds nothing else), then the group moves to C.
             const int chunks = (w.num_kb + kChunkKB - 1) / kChunkKB;
@@ -1174,7 +1187,7 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmap_a, const CUten
                 // first group of a tile, added at the destination for later ones)
                 if (kEpi)
                     epi_transform(sum2, p, row0 + lane < m_end, n0 + half * 128, reinterpret_cast<uint32_t*>(my_stage), epi_hist, lane);
-                if (w.partial && c0 == 0) {
+                if (kSk && w.partial && c0 == 0) {
                     // the pair before this one has stored the first piece of this tile (warp 3 watches its flag)
                     bool seen = true;
                     if (lane == 0) seen = ptx::mbar_wait_bounded(tail_bar, 0u, kWaitLimit);
@@ -1266,7 +1279,7 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmap_a, const CUten
                 flushed = true;
             }
             if (dead) break;
-            if (w.head && chunks > 0) {
+            if (kSk && w.head && chunks > 0) {
                 // this warp's part of the tile's first piece is in C (its copies have completed)
                 if (lane == 0) {
                     ptx::bulk_wait_all();
@@ -1293,20 +1306,21 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmap_a, const CUten
     }
 }
 
-template <bool kEpi, int kKind>
+template <bool kEpi, int kKind, bool kSk>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 gemm_tf32_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                       const __grid_constant__ CUtensorMap tmap_c, const GemmParams p) {
-    pair_body<kEpi, kKind, 0>(tmap_a, tmap_b, tmap_c, nullptr, nullptr, p);
+    pair_body<kEpi, kKind, 0, kSk>(tmap_a, tmap_b, tmap_c, nullptr, nullptr, p);
 }
 
 // Forward / data gradient of a convolution on CTA pairs (its own instantiation, so that the dense
 // products carry none of its code).
+template <bool kSk>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 gemm_conv_pair_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_constant__ CUtensorMap tmap_c,
                       const __grid_constant__ CUtensorMap tmap_c2, const __grid_constant__ RowMaps row_maps,
                       const GemmParams p) {
-    pair_body<false, kKindTf32, 1>(row_maps.m[0], tmap_b, tmap_c, &tmap_c2, row_maps.m, p);
+    pair_body<false, kKindTf32, 1, kSk>(row_maps.m[0], tmap_b, tmap_c, &tmap_c2, row_maps.m, p);
 }
 
 // ---- host side ----------------------------------------------------------------------------------
@@ -1605,23 +1619,30 @@ int launch_pair(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap&
                 const DeviceInfo& dev, cudaStream_t stream, int kind = kKindTf32) {
     static bool attr_set[64] = {};
     if (dev.ordinal < 0 || dev.ordinal >= 64 || !attr_set[dev.ordinal]) {
-        QFMT_CUDA_TRY(cudaFuncSetAttribute(gemm_tf32_pair_kernel<false, kKindTf32>,
-                                           cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPairSmemBytes));
-        QFMT_CUDA_TRY(cudaFuncSetAttribute(gemm_tf32_pair_kernel<true, kKindTf32>,
-                                           cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPairSmemBytes));
-        QFMT_CUDA_TRY(cudaFuncSetAttribute(gemm_tf32_pair_kernel<false, kKindF16>,
-                                           cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPairSmemBytes));
-        QFMT_CUDA_TRY(cudaFuncSetAttribute(gemm_tf32_pair_kernel<false, kKindBf16>,
-                                           cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPairSmemBytes));
+#define QFMT_PAIR_ATTR(...)                                                                                       \
+    QFMT_CUDA_TRY(cudaFuncSetAttribute(gemm_tf32_pair_kernel<__VA_ARGS__>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
+                                       (int)kPairSmemBytes))
+        QFMT_PAIR_ATTR(false, kKindTf32, false);
+        QFMT_PAIR_ATTR(false, kKindTf32, true);
+        QFMT_PAIR_ATTR(true, kKindTf32, false);
+        QFMT_PAIR_ATTR(false, kKindF16, false);
+        QFMT_PAIR_ATTR(false, kKindF16, true);
+        QFMT_PAIR_ATTR(false, kKindBf16, false);
+        QFMT_PAIR_ATTR(false, kKindBf16, true);
+#undef QFMT_PAIR_ATTR
         if (dev.ordinal >= 0 && dev.ordinal < 64) attr_set[dev.ordinal] = true;
     }
     const long long work = (long long)p.tiles_m * p.tiles_n * p.splits;
     const long long clusters = p.sk_flags != nullptr ? kPlanPairs : (work < dev.sm_count / 2 ? work : dev.sm_count / 2);
     const unsigned grid = (unsigned)(2 * clusters);
-    if (kind == kKindF16) gemm_tf32_pair_kernel<false, kKindF16><<<grid, kThreads, kPairSmemBytes, stream>>>(ma, mb, mc, p);
-    else if (kind == kKindBf16) gemm_tf32_pair_kernel<false, kKindBf16><<<grid, kThreads, kPairSmemBytes, stream>>>(ma, mb, mc, p);
-    else if (p.epi) gemm_tf32_pair_kernel<true, kKindTf32><<<grid, kThreads, kPairSmemBytes, stream>>>(ma, mb, mc, p);
-    else gemm_tf32_pair_kernel<false, kKindTf32><<<grid, kThreads, kPairSmemBytes, stream>>>(ma, mb, mc, p);
+    const bool sk = p.sk_flags != nullptr;
+#define QFMT_PAIR_LAUNCH(...) gemm_tf32_pair_kernel<__VA_ARGS__><<<grid, kThreads, kPairSmemBytes, stream>>>(ma, mb, mc, p)
+    if (kind == kKindF16) { if (sk) QFMT_PAIR_LAUNCH(false, kKindF16, true); else QFMT_PAIR_LAUNCH(false, kKindF16, false); }
+    else if (kind == kKindBf16) { if (sk) QFMT_PAIR_LAUNCH(false, kKindBf16, true); else QFMT_PAIR_LAUNCH(false, kKindBf16, false); }
+    else if (p.epi) QFMT_PAIR_LAUNCH(true, kKindTf32, false);
+    else if (sk) QFMT_PAIR_LAUNCH(false, kKindTf32, true);
+    else QFMT_PAIR_LAUNCH(false, kKindTf32, false);
+#undef QFMT_PAIR_LAUNCH
     QFMT_CUDA_TRY(cudaGetLastError());
     return QFMT_OK;
 }
@@ -1630,13 +1651,18 @@ int launch_conv_pair(const CUtensorMap& mb, const CUtensorMap& mc, const CUtenso
                      const GemmParams& p, const DeviceInfo& dev, cudaStream_t stream) {
     static bool attr_set[64] = {};
     if (dev.ordinal < 0 || dev.ordinal >= 64 || !attr_set[dev.ordinal]) {
-        QFMT_CUDA_TRY(cudaFuncSetAttribute(gemm_conv_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        QFMT_CUDA_TRY(cudaFuncSetAttribute(gemm_conv_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           (int)kPairSmemBytes));
+        QFMT_CUDA_TRY(cudaFuncSetAttribute(gemm_conv_pair_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                            (int)kPairSmemBytes));
         if (dev.ordinal >= 0 && dev.ordinal < 64) attr_set[dev.ordinal] = true;
     }
     const long long work = (long long)p.tiles_m * p.tiles_n;
     const long long clusters = p.sk_flags != nullptr ? kPlanPairs : (work < dev.sm_count / 2 ? work : dev.sm_count / 2);
-    gemm_conv_pair_kernel<<<(unsigned)(2 * clusters), kThreads, kPairSmemBytes, stream>>>(mb, mc, mc2, rows, p);
+    if (p.sk_flags != nullptr)
+        gemm_conv_pair_kernel<true><<<(unsigned)(2 * clusters), kThreads, kPairSmemBytes, stream>>>(mb, mc, mc2, rows, p);
+    else
+        gemm_conv_pair_kernel<false><<<(unsigned)(2 * clusters), kThreads, kPairSmemBytes, stream>>>(mb, mc, mc2, rows, p);
     QFMT_CUDA_TRY(cudaGetLastError());
     return QFMT_OK;
 }
@@ -1648,6 +1674,15 @@ struct EpiArgs {
 };
 // The epilogue runs on the sums of one group held in registers: at most this many K elements.
 constexpr int64_t kEpiMaxK = (int64_t)kFlushChunks * kChunkKB * kBK;
+
+// Whether the balanced schedule can take a product of `tiles` pair tiles of `cpt` chunks: the chunk count
+// stays in 32 bits and a pair's pieces fit the kernel's table.
+bool pair_schedule_fits(long long tiles, long long cpt) {
+    const long long total = tiles * cpt;
+    if (cpt <= 0 || total >= (1ll << 30)) return false;
+    const long long range = (total + kPlanPairs - 1) / kPlanPairs;
+    return (range + cpt - 1) / cpt + 1 <= kMaxSkPieces;
+}
 
 // Turns the balanced schedule of the pair kernel on: chunks per tile, the most pieces a pair can have,
 // and the flag words behind the workspace header (cleared on the stream, with the status word).
@@ -1735,7 +1770,7 @@ int gemm_device(const qfmt_matrix_t* A, const qfmt_matrix_t* B, float* d_C, int6
     // workspace, and the blocked C map.
     const bool sk = plan.sk && epi == nullptr && pair && dev.sm_count >= 2 * kPlanPairs && p.tma_store &&
                     (N & 31) == 0 && workspace_bytes >= kWorkspaceHeader + kSkFlagBytes &&
-                    (long long)p.tiles_m * p.tiles_n * ((p.kb_total + kChunkKB - 1) / kChunkKB) < (1ll << 30);
+                    pair_schedule_fits((long long)p.tiles_m * p.tiles_n, (p.kb_total + kChunkKB - 1) / kChunkKB);
     if (epi != nullptr) {
         if (K > kEpiMaxK || fmt->e > 6) return QFMT_ERR_BAD_ARG;  // callers check before asking
         qfmt_format_t f = *fmt;
@@ -1854,7 +1889,7 @@ int gemm16_device(const qfmt_matrix16_t* A, const qfmt_matrix16_t* B, float* d_C
     int splits = plan.splits;
     const bool sk = plan.sk && dev.sm_count >= 2 * kPlanPairs && p.tma_store && (N & 31) == 0 &&
                     workspace_bytes >= kWorkspaceHeader + kSkFlagBytes &&
-                    (long long)p.tiles_m * p.tiles_n * ((p.kb_total + kChunkKB - 1) / kChunkKB) < (1ll << 30);
+                    pair_schedule_fits((long long)p.tiles_m * p.tiles_n, (p.kb_total + kChunkKB - 1) / kChunkKB);
     while (splits > 1 && kWorkspaceHeader + (size_t)splits * (size_t)M * (size_t)N * sizeof(float) > workspace_bytes) --splits;
     float* partials = reinterpret_cast<float*>(reinterpret_cast<char*>(d_workspace) + kWorkspaceHeader);
     if (sk) {
@@ -2130,7 +2165,8 @@ int conv_device(int op, const qfmt_conv_t* g, const float* d_p, const float* d_q
                 mc = mc2;
             }
             if (rem == 0) mc2 = mc;
-            if (plan.pair_sk && dev.sm_count >= 2 * kPlanPairs) {
+            if (plan.pair_sk && dev.sm_count >= 2 * kPlanPairs &&
+                pair_schedule_fits((long long)p.tiles_m * p.tiles_n, (p.kb_total + kChunkKB - 1) / kChunkKB)) {
                 rc = enable_pair_schedule(&p, d_workspace, stream);
                 if (rc != QFMT_OK) return rc;
             }
