@@ -371,6 +371,11 @@ size_t qfmt_gemm_packed16_workspace_bytes(const qfmt_matrix16_t* A, const qfmt_m
  *   0  automatic (default)
  *   1  single-CTA 128 x 256 tiles
  *   2  CTA-pair 256 x 256 tiles (tcgen05 cta_group::2; each SM stages half of the B operand)
+ *   3  CTA-pair tiles under the balanced schedule wherever it applies (74 or more tiles, room for its
+ *      flag words in the workspace): the tiles' K chunks are dealt among the 74 pairs in equal ranges,
+ *      a tile cut by a range boundary is stored by one pair and completed by the next with an add at
+ *      the destination, in a fixed order.  Never chosen automatically for dense products: measured
+ *      slower than whole tiles on every product of the library's workloads.
  * Process-wide and not synchronised with calls in flight; results stay within the same bound under
  * every policy but their last bits may differ between policies.  Ask qfmt_gemm_workspace_bytes
  * again after changing it.  Returns QFMT_ERR_BAD_ARG for other values.
@@ -381,6 +386,8 @@ int qfmt_gemm_tile_policy(int policy);
  *   0  automatic (default): CTA pairs, each CTA one M-tile of whole image rows and half of the filter
  *      columns, whenever there are two or more M-tiles
  *   1  always the single-CTA kernel
+ *   2  CTA pairs on whole tiles
+ *   3  CTA pairs under the balanced schedule wherever it applies
  * Ask qfmt_conv_workspace_bytes again after changing it.
  */
 int qfmt_conv_tile_policy(int policy);

@@ -100,8 +100,7 @@ struct GemmParams {
     // slots and without the second kernel.  A pair runs the piece that begins inside a tile LAST and adds
     // it into C at the destination; by then the pair before it, whose range ends inside that tile, has
     // written the tile's first part as the last-but-one piece of its own range and has said so in
-    // sk_flags ([pair][2 CTAs x 8 accumulate warps] words, zeroed before the launch; a word covers the
-    // 32 x 128 patch of the tile that the same warp of both pairs owns).  A tile has at most two pieces
+    // sk_flags (one word per pair, 64 bytes apart, zeroed before the launch).  A tile has at most two pieces
     // (ranges are at least a tile long), the first stored and the second added after it in program
     // order of a flag hand-over, so the sums are the same on every run.
     int* sk_flags;
@@ -866,8 +865,9 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmap_a, const CUten
     auto empty_bar = [&](int s) { return bars + 8u * (kPStages + s); };
     auto acc_full_bar = [&](int a) { return bars + 8u * (2 * kPStages + a); };
     auto acc_empty_bar = [&](int a) { return bars + 8u * (2 * kPStages + 2 + a); };
-    // balanced schedule: head_bar collects the accumulate warps whose stores of a tile's first piece
-    // are complete, tail_bar tells them that the pair before has stored the first piece of their tile
+    // balanced schedule: head_bar (the non-leader CTA's) collects the pair's accumulate warps whose stores
+    // of a tile's first piece are complete, tail_bar tells a CTA's accumulate warps that the pair before
+    // has stored the first piece of their tile
     const uint32_t head_bar = bars + 8u * (2 * kPStages + 4), tail_bar = bars + 8u * (2 * kPStages + 5);
     uint8_t* gen_bars = smem_raw + (bars - raw);
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen_bars + 8 * (2 * kPStages + 6));
@@ -899,7 +899,7 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmap_a, const CUten
             ptx::mbar_init(acc_full_bar(a), 1);
             ptx::mbar_init(acc_empty_bar(a), 2 * kAccWarps);
         }
-        ptx::mbar_init(head_bar, kAccWarps);
+        ptx::mbar_init(head_bar, 2 * kAccWarps);  // used in the non-leader CTA: the accumulate warps of both
         ptx::mbar_init(tail_bar, 1);
         *abort_flag = 0;
         ptx::fence_mbar_init();
@@ -940,15 +940,25 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmap_a, const CUten
 
     if (warp < 4) {
     ptx::setmaxnreg_dec<56>();
-    if (warp == 0) {
-        // ------------------------------ TMA producer (both CTAs) ------------------------------
+    if (warp == 0 || warp == 3) {
+        // ------------------------------ TMA producers (both CTAs) ------------------------------
+        // One thread needs ~700 cycles for a dense stage (the wait on its slot, the byte count, two
+        // copies) and over 1000 for a convolution's (tap arithmetic, a copy per image touched), and the
+        // tensor pipe consumes a stage in 512, so two threads fill alternate stages: warp 0 the even
+        // ones of the CTA's stage sequence, warp 3 the odd ones.
         if (lane == 0) {
+            const uint32_t who = warp == 0 ? 0u : 1u;
+            uint32_t seq = 0;
             int stage = 0;
             uint32_t phase = 0;
             for (int t = t_begin; t < t_end && !*abort_flag; t += t_step) {
                 const WorkItem w = work_item(t);
                 const int m0 = w.m0 + (int)rank * kBM, n0 = w.n0 + (int)rank * (kBN / 2);
                 for (int kb = w.kb_begin; kb < w.kb_begin + w.num_kb; ++kb) {
+                    if ((seq++ & 1u) != who) {  // the other producer's stage
+                        if (++stage == kPStages) { stage = 0; phase ^= 1u; }
+                        continue;
+                    }
                     if (!ptx::mbar_wait_bounded(empty_bar(stage), phase ^ 1u, kWaitLimit)) {
                         raise_timeout(p, abort_flag);
                         break;
@@ -1013,6 +1023,44 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmap_a, const CUten
         // here: an issuer reaches chunk c+1 only after the accumulate warps have drained chunk c-1,
         // hence after chunk c-2 was issued in full, and with a ring of five stages the previous
         // phase of the stages of chunk c+1 belongs to chunks c-2 and c-1.
+        if (kSk && lane == 0 && rank == 1 && warp == 1) {
+            // ---- balanced schedule: hand-over between pairs (this warp has no MMAs to issue in the
+            // non-leader CTA).  A tile cut by a range boundary is begun by one pair (its last-but-one
+            // piece, "head") and finished by the next (its last piece, which adds at the destination).
+            // Once the sixteen accumulate warps of this pair have completed their stores of a head
+            // piece this thread raises the next pair's flag; before this pair's accumulate warps may
+            // add a piece that begins inside a tile it waits for this pair's own flag and then lets
+            // both CTAs go on.
+            bool dead = false;
+            for (int t = t_begin; t < t_end && !dead; t += t_step) {
+                const WorkItem w = work_item(t);
+                if (w.num_kb <= 0) continue;
+                if (w.head) {
+                    if (!ptx::mbar_wait_bounded(head_bar, 0u, kWaitLimit)) {
+                        raise_timeout(p, abort_flag);
+                        break;
+                    }
+                    ptx::fence_proxy_async_all();
+                    __threadfence();
+                    *reinterpret_cast<volatile int*>(p.sk_flags + (cluster_id + 1) * 16) = 1;
+                }
+                if (w.partial) {
+                    volatile int* flag = p.sk_flags + cluster_id * 16;
+                    const long long t_begin_wait = clock64();
+                    while (*flag == 0 && !*abort_flag) {
+                        if (clock64() - t_begin_wait > (long long)kWaitLimit) { dead = true; break; }
+                        __nanosleep(64);
+                    }
+                    if (dead) {
+                        raise_timeout(p, abort_flag);
+                        break;
+                    }
+                    __threadfence();
+                    ptx::mbar_arrive(tail_bar);
+                    ptx::mbar_arrive_cluster(ptx::map_to_cta(tail_bar, 0));
+                }
+            }
+        }
         if (lane == 0 && rank == 0) {
             const uint32_t who = (uint32_t)(warp - 1);
             const uint32_t idesc = make_idesc_pair(p.a_mn_major, p.b_mn_major, kKind);
@@ -1072,45 +1120,6 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmap_a, const CUten
                     }
                     if (dead) break;
                     ptx::mma_commit_pair(acc_full_bar(acc), 3);      // chunk sum complete in both CTAs
-                }
-            }
-        }
-        __syncwarp();
-    } else if (kSk && warp == 3) {
-        // ------------------------------ balanced schedule: hand-over between pairs ------------------------------
-        // A tile cut by a range boundary is begun by one pair (its last-but-one piece, "head") and
-        // finished by the next (its last piece, which adds at the destination).  This thread passes
-        // the news: once the eight accumulate warps of this CTA have completed their stores of a head
-        // piece it raises this CTA's flag for the next pair; before this CTA's accumulate warps may
-        // add a piece that begins inside a tile it waits for the flag of the pair before.  One word
-        // per pair and CTA rank (the same rank owns the same rows in both pairs).
-        if (lane == 0) {
-            bool dead = false;
-            for (int t = t_begin; t < t_end && !dead; t += t_step) {
-                const WorkItem w = work_item(t);
-                if (w.num_kb <= 0) continue;
-                if (w.head) {
-                    if (!ptx::mbar_wait_bounded(head_bar, 0u, kWaitLimit)) {
-                        raise_timeout(p, abort_flag);
-                        break;
-                    }
-                    ptx::fence_proxy_async_all();
-                    __threadfence();
-                    *reinterpret_cast<volatile int*>(p.sk_flags + ((cluster_id + 1) * 16 + (int)rank)) = 1;
-                }
-                if (w.partial) {
-                    volatile int* flag = p.sk_flags + (cluster_id * 16 + (int)rank);
-                    const long long t_begin = clock64();
-                    while (*flag == 0 && !*abort_flag) {
-                        if (clock64() - t_begin > (long long)kWaitLimit) { dead = true; break; }
-                        __nanosleep(64);
-                    }
-                    if (dead) {
-                        raise_timeout(p, abort_flag);
-                        break;
-                    }
-                    __threadfence();
-                    ptx::mbar_arrive(tail_bar);
                 }
             }
         }
@@ -1283,7 +1292,8 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmap_a, const CUten
                 // this warp's part of the tile's first piece is in C (its copies have completed)
                 if (lane == 0) {
                     ptx::bulk_wait_all();
-                    ptx::mbar_arrive(head_bar);
+                    __threadfence();
+                    ptx::mbar_arrive_cluster(ptx::map_to_cta(head_bar, 1));
                 }
                 __syncwarp();
             }
@@ -1554,11 +1564,14 @@ void dense_defaults(GemmParams* p) {
 }  // namespace
 
 // Which kernel a dense product runs on: 0 automatic, 1 single-CTA tiles (128 x 256), 2 CTA-pair
-// tiles (256 x 256).  Process-wide; see qfmt_gemm_tile_policy.
+// tiles (256 x 256), 3 CTA-pair tiles under the balanced schedule wherever it applies.  Process-wide;
+// see qfmt_gemm_tile_policy.
 static std::atomic<int> g_tile_policy{0};
 
 // Which kernel the forward / data-gradient products of a convolution run on: 0 automatic (CTA pairs
-// when there are two or more M-tiles), 1 always the single-CTA kernel.  See qfmt_gemm_tile_policy.
+// when there are two or more M-tiles, the balanced schedule by estimated cost), 1 always the single-CTA
+// kernel, 2 CTA pairs on whole tiles, 3 CTA pairs under the balanced schedule wherever it applies.
+// See qfmt_gemm_tile_policy.
 static std::atomic<int> g_conv_pair_policy{0};
 
 // How a dense product is laid over the GPU: tile shape and split-K factor.
@@ -1577,7 +1590,9 @@ constexpr size_t kSkFlagBytes = ((size_t)(kPlanPairs + 1) * 16 * sizeof(int) + 2
 // is taken for a 148-SM part whatever the device, so that the plan, and with it the summation
 // order, depends on the problem alone.
 DensePlan plan_dense(int64_t M, int64_t N, int64_t K, int policy_override = -1) {
-    const int policy = policy_override >= 0 ? policy_override : g_tile_policy.load();
+    const int chosen = g_tile_policy.load();
+    const bool want_sk = chosen == 3;
+    const int policy = policy_override >= 0 ? policy_override : (want_sk ? 2 : chosen);
     const int64_t kb_total = (K + kBK - 1) / kBK;
     DensePlan best = {policy == 2, 1, false};
     double best_cost = -1.0;
@@ -1603,13 +1618,13 @@ DensePlan plan_dense(int64_t M, int64_t N, int64_t K, int policy_override = -1) 
         }
         // Balanced schedule: the tiles' chunks dealt among the 74 pairs in equal ranges.  A pair then runs
         // tiles / 74 + 1 pieces, each with its own move of sums to C.  Needs ranges of at least a tile.
-        if (pair && tiles >= kPlanPairs) {
-            const double chunks = (double)((kb_total + kChunkKB - 1) / kChunkKB);
-            const double cost = (double)tiles * chunks / kPlanPairs + 3.0 * ((double)tiles / kPlanPairs + 1.0);
-            if (cost < best_cost * 0.97) {
-                best_cost = cost;
-                best = {true, 1, true};
-            }
+        // Only on request (policy 3).  Measured on dense products it loses to whole tiles even where a
+        // third of the last wave idles (8192 x 1024 x 1024: 48 against 40 us): pairs that walk through
+        // different tiles at different K offsets share no operand bytes in flight, each pair has one more
+        // move of sums to C, and the planner's automatic choice therefore never takes it.
+        if (pair && want_sk && tiles >= kPlanPairs) {
+            best = {true, 1, true};
+            break;
         }
     }
     return best;
@@ -1997,7 +2012,8 @@ int plan_conv(int op, const qfmt_conv_t* g, ConvPlan* plan) {
                 const int64_t pwaves = (ptiles + kPlanPairs - 1) / kPlanPairs;
                 const double plain = (double)pwaves * ((double)cpt + 3.0);
                 const double sk = (double)ptiles * (double)cpt / kPlanPairs + 3.0 * ((double)ptiles / kPlanPairs + 1.0);
-                plan->pair_sk = sk < plain * 0.97 && ptiles * cpt < (1ll << 30);
+                const int cp = g_conv_pair_policy.load();
+                plan->pair_sk = cp == 3 || (cp == 0 && sk < plain * 0.97 && ptiles * cpt < (1ll << 30));
             }
             plan->workspace += kSkFlagBytes;
             return QFMT_OK;
@@ -2373,13 +2389,13 @@ extern "C" size_t qfmt_linear_forward_workspace_bytes(const qfmt_matrix_t* A, co
 }
 
 extern "C" int qfmt_conv_tile_policy(int policy) {
-    if (policy < 0 || policy > 1) return QFMT_ERR_BAD_ARG;
+    if (policy < 0 || policy > 3) return QFMT_ERR_BAD_ARG;
     qfmt::g_conv_pair_policy.store(policy);
     return QFMT_OK;
 }
 
 extern "C" int qfmt_gemm_tile_policy(int policy) {
-    if (policy < 0 || policy > 2) return QFMT_ERR_BAD_ARG;
+    if (policy < 0 || policy > 3) return QFMT_ERR_BAD_ARG;
     qfmt::g_tile_policy.store(policy);
     return QFMT_OK;
 }

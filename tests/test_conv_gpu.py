@@ -84,9 +84,9 @@ SMALL = [
 ]
 
 
-@pytest.fixture(params=[0, 1], ids=["cta_pairs", "single_cta"])
+@pytest.fixture(params=[0, 1, 2, 3], ids=["automatic", "single_cta", "pairs_whole_tiles", "pairs_balanced"])
 def conv_kernel(request):
-    """Forward and data gradient on both kernels: CTA pairs (the default) and the single-CTA kernel."""
+    """Forward and data gradient on both kernels and both schedules of the pair kernel."""
     qf.qfmt_conv_tile_policy(request.param)
     yield request.param
     qf.qfmt_conv_tile_policy(0)

@@ -398,16 +398,23 @@ def test_split_k_few_tiles_long_k(transA, transB):
 
 
 # ---------------------------------------------------------------------------------------------
-# Balanced schedule of the CTA-pair kernel: with at least 74 tiles whose last wave would leave
-# pairs idle, the tiles' K chunks are dealt among the 74 pairs in equal ranges; a tile cut by a
-# range boundary is stored by one pair and completed by the next with an add at the destination.
+# Balanced schedule of the CTA-pair kernel (tile policy 3): with at least 74 tiles, the tiles' K
+# chunks are dealt among the 74 pairs in equal ranges; a tile cut by a range boundary is stored by
+# one pair and completed by the next with an add at the destination.
 # ---------------------------------------------------------------------------------------------
 SK_WORKSPACE = 256 + 4864  # header + the schedule's flag words: what the planner asks for when it picks the schedule
 
 
+@pytest.fixture
+def balanced_schedule():
+    qf.qfmt_gemm_tile_policy(3)
+    yield
+    qf.qfmt_gemm_tile_policy(0)
+
+
 @pytest.mark.parametrize("transA,transB", [(False, False), (False, True), (True, False), (True, True)])
 @pytest.mark.parametrize("M,N,K", [(2560, 2560, 200), (2304, 2304, 1100), (4096, 3072, 768), (2500, 2336, 96)])
-def test_balanced_schedule_small_integers_are_exact(transA, transB, M, N, K):
+def test_balanced_schedule_small_integers_are_exact(balanced_schedule, transA, transB, M, N, K):
     rng = np.random.default_rng(M + 3 * N + 7 * K)
     A = stored((M, K), transA, lambda s: rng.integers(-3, 4, size=s).astype(np.float32))
     B = stored((K, N), transB, lambda s: rng.integers(-3, 4, size=s).astype(np.float32))
@@ -426,7 +433,7 @@ def test_balanced_schedule_small_integers_are_exact(transA, transB, M, N, K):
 
 
 @pytest.mark.parametrize("M,N,K", [(2304, 2304, 2560), (8192, 1024, 4096)])
-def test_balanced_schedule_real_values_within_bound_and_reproducible(M, N, K):
+def test_balanced_schedule_real_values_within_bound_and_reproducible(balanced_schedule, M, N, K):
     """Pieces longer than one summation group: a cut tile gets store, add, add ... from one pair and then
     add, add ... from the next; the order is fixed, so two runs give the same bits."""
     A = quantized(workloads.rng_for(81), (M, K), 6, 9, -6.0, 4.0)
