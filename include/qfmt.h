@@ -476,6 +476,20 @@ int qfmt_gemm_builtin_scratch(const qfmt_matrix_t* A, const qfmt_matrix_t* B, fl
 int qfmt_selftest_bounded_wait(int32_t* d_status, uint32_t limit_cycles, int32_t* d_trace, void* stream);
 
 /*
+ * Host-only view of the balanced schedule of the CTA-pair kernels (tile policy 3, and the forward /
+ * data-gradient products of qfmt_conv when their plan picks it): piece `j`, in the order pair `pair`
+ * (0 .. 73) runs its pieces, of a product of `tiles` 256 x 256 tiles (>= 74) with `chunks_per_tile`
+ * 64-element K chunks each.  Touches no device.
+ *   out[0] tile index   out[1] first chunk within the tile   out[2] chunks (0: the pair has no piece j)
+ *   out[3] 1 = the piece begins inside its tile and is added to what the pair before stored
+ *   out[4] 1 = the piece ends before its tile does: the next pair finishes the tile
+ *   out[5] the number of pieces the kernel provides for per pair
+ * Returns QFMT_ERR_BAD_ARG for arguments outside these ranges or a product the schedule does not take.
+ * The paper has no counterpart; this is a diagnostic of the library.
+ */
+int qfmt_selftest_pair_schedule(int64_t tiles, int32_t chunks_per_tile, int32_t pair, int32_t j, int32_t* out);
+
+/*
  * Synchronises `stream` and returns the status word of a workspace: QFMT_OK, or the error a
  * kernel recorded (QFMT_ERR_TIMEOUT), or QFMT_ERR_CUDA if the copy itself failed.
  */

@@ -147,6 +147,8 @@ def _bind_optional(L: ctypes.CDLL) -> None:
     L.qfmt_gemm_builtin_scratch.restype = ci
     L.qfmt_selftest_bounded_wait.argtypes = [vp, ctypes.c_uint32, vp, vp]
     L.qfmt_selftest_bounded_wait.restype = ci
+    L.qfmt_selftest_pair_schedule.argtypes = [i64, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, vp]
+    L.qfmt_selftest_pair_schedule.restype = ci
 
 
 def _ptr(x) -> Optional[int]:
@@ -335,6 +337,15 @@ def qfmt_selftest_bounded_wait(d_status, limit_cycles: int, d_trace, stream=None
            "qfmt_selftest_bounded_wait")
 
 
+def qfmt_selftest_pair_schedule(tiles: int, chunks_per_tile: int, pair: int, j: int):
+    """Piece j of a pair under the balanced schedule as (tile, first chunk, chunks, partial, head, pieces per
+    pair); host only.  See qfmt_selftest_pair_schedule in include/qfmt.h."""
+    out = (ctypes.c_int32 * 6)()
+    _check(lib().qfmt_selftest_pair_schedule(int(tiles), int(chunks_per_tile), int(pair), int(j),
+                                             ctypes.cast(out, ctypes.c_void_p)), "qfmt_selftest_pair_schedule")
+    return tuple(int(v) for v in out)
+
+
 def qfmt_conv_workspace_bytes(op: int, geom: qfmt_conv_t) -> int:
     return int(lib().qfmt_conv_workspace_bytes(int(op), ctypes.byref(geom)))
 
@@ -348,10 +359,12 @@ def qfmt_conv(op: int, geom: qfmt_conv_t, d_p, d_q, d_out, fmt: qfmt_format_t, d
 
 
 def qfmt_conv_tile_policy(policy: int) -> None:
-    """0 automatic (CTA pairs), 1 single-CTA kernel for conv forward / data gradient; see include/qfmt.h."""
+    """0 automatic, 1 single-CTA kernel, 2 CTA pairs on whole tiles, 3 CTA pairs under the balanced schedule,
+    for conv forward / data gradient; see include/qfmt.h."""
     _check(lib().qfmt_conv_tile_policy(int(policy)), "qfmt_conv_tile_policy")
 
 
 def qfmt_gemm_tile_policy(policy: int) -> None:
-    """0 automatic, 1 single-CTA tiles, 2 CTA-pair tiles; see include/qfmt.h."""
+    """0 automatic, 1 single-CTA tiles, 2 CTA-pair tiles, 3 CTA-pair tiles under the balanced schedule; see
+    include/qfmt.h."""
     _check(lib().qfmt_gemm_tile_policy(int(policy)), "qfmt_gemm_tile_policy")

@@ -99,7 +99,7 @@ struct GemmParams {
     // The same schedule in the pair kernel (sk_flags != nullptr), dealt among the CTA pairs, without the
     // slots and without the second kernel.  A pair runs the piece that begins inside a tile LAST and adds
     // it into C at the destination; by then the pair before it, whose range ends inside that tile, has
-    // written the tile's first part as the last-but-one piece of its own range and has said so in
+    // written the tile's first part as the FIRST piece of its own range and has said so in
     // sk_flags (one word per pair, 64 bytes apart, zeroed before the launch).  A tile has at most two pieces
     // (ranges are at least a tile long), the first stored and the second added after it in program
     // order of a flag hand-over, so the sums are the same on every run.
@@ -153,9 +153,12 @@ struct WorkItem {
     int head;     // balanced schedule of the pair kernel: the next pair adds the rest of this tile
 };
 // Piece j (in the order a pair runs them) of pair `unit` under the balanced schedule of the pair
-// kernel: the pieces of the pair's chunk range in their natural order, except that a first piece that
-// begins inside a tile moves to the end.  `head`: the piece begins its tile and ends before the tile
-// does (the next pair finishes it).  `partial`: the piece begins inside its tile.
+// kernel: first the range's last piece if it ends before its tile does (`head`: the next pair finishes
+// that tile, and needs it stored early), then the whole tiles in their natural order, last the range's
+// first piece if it begins inside a tile (`partial`: it adds to what the pair before has stored).
+// Every pair starts at the same moment and ranges are at least a tile long, so a head piece (at most a
+// tile) is in C before the pair after it has worked through the rest of its range and the first
+// summation group of its partial piece.
 struct PairPiece {
     int tile, kb_begin, num_kb, partial, head;
 };
@@ -167,10 +170,15 @@ __host__ __device__ __forceinline__ PairPiece pair_piece(int q, int r, int cpt, 
     if (hi <= lo) return pc;
     const int first_tile = lo / cpt, last_tile = (hi - 1) / cpt;
     const int n_nat = last_tile - first_tile + 1;
-    const bool first_partial = lo > first_tile * cpt;
-    int nat = j;
-    if (first_partial) nat = j + 1 < n_nat ? j + 1 : (j + 1 == n_nat ? 0 : n_nat);
-    if (nat >= n_nat) return pc;
+    const bool first_partial = lo > first_tile * cpt, last_head = hi < (last_tile + 1) * cpt;
+    int nat;
+    if (last_head && j == 0) {
+        nat = n_nat - 1;
+    } else {
+        const int idx = last_head ? j - 1 : j, m = last_head ? n_nat - 1 : n_nat;  // the other pieces
+        if (idx >= m) return pc;
+        nat = first_partial ? (idx + 1 < m ? idx + 1 : 0) : idx;
+    }
     const int tile = first_tile + nat, first = tile * cpt;
     const int s = lo > first ? lo : first, e = hi < first + cpt ? hi : first + cpt;
     pc.tile = tile;
@@ -1025,8 +1033,8 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmap_a, const CUten
         // phase of the stages of chunk c+1 belongs to chunks c-2 and c-1.
         if (kSk && lane == 0 && rank == 1 && warp == 1) {
             // ---- balanced schedule: hand-over between pairs (this warp has no MMAs to issue in the
-            // non-leader CTA).  A tile cut by a range boundary is begun by one pair (its last-but-one
-            // piece, "head") and finished by the next (its last piece, which adds at the destination).
+            // non-leader CTA).  A tile cut by a range boundary is begun by one pair (its first piece,
+            // "head") and finished by the next (its last piece, which adds at the destination).
             // Once the sixteen accumulate warps of this pair have completed their stores of a head
             // piece this thread raises the next pair's flag; before this pair's accumulate warps may
             // add a piece that begins inside a tile it waits for this pair's own flag and then lets
@@ -2391,6 +2399,19 @@ extern "C" size_t qfmt_linear_forward_workspace_bytes(const qfmt_matrix_t* A, co
 extern "C" int qfmt_conv_tile_policy(int policy) {
     if (policy < 0 || policy > 3) return QFMT_ERR_BAD_ARG;
     qfmt::g_conv_pair_policy.store(policy);
+    return QFMT_OK;
+}
+
+extern "C" int qfmt_selftest_pair_schedule(int64_t tiles, int32_t chunks_per_tile, int32_t pair, int32_t j, int32_t* out) {
+    if (out == nullptr || tiles < qfmt::kPlanPairs || chunks_per_tile <= 0 || pair < 0 || pair >= qfmt::kPlanPairs || j < 0)
+        return QFMT_ERR_BAD_ARG;
+    if (!qfmt::pair_schedule_fits(tiles, chunks_per_tile)) return QFMT_ERR_BAD_ARG;
+    const long long total = tiles * chunks_per_tile;
+    const qfmt::PairPiece pc = qfmt::pair_piece((int)(total / qfmt::kPlanPairs), (int)(total % qfmt::kPlanPairs), chunks_per_tile,
+                                                chunks_per_tile * qfmt::kChunkKB, qfmt::kPlanPairs, pair, j);
+    out[0] = pc.tile; out[1] = pc.kb_begin / qfmt::kChunkKB; out[2] = pc.num_kb / qfmt::kChunkKB; out[3] = pc.partial; out[4] = pc.head;
+    const long long range = (total + qfmt::kPlanPairs - 1) / qfmt::kPlanPairs;
+    out[5] = (int32_t)((range + chunks_per_tile - 1) / chunks_per_tile + 1);
     return QFMT_OK;
 }
 
