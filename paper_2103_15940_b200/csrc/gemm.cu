@@ -962,7 +962,36 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmap_a, const CUten
             for (int t = t_begin; t < t_end && !*abort_flag; t += t_step) {
                 const WorkItem w = work_item(t);
                 const int m0 = w.m0 + (int)rank * kBM, n0 = w.n0 + (int)rank * (kBN / 2);
+                // convolution: the boxes of this CTA's M-tile (one per image it touches: first row within
+                // the image, image, rows) and the tap / channel block of the piece's first stage; the
+                // stage loop then only counts
+                int box_h[3], box_img[3], box_cnt[3], n_boxes = 0;
+                int tap = 0, cb = 0, tap_r = 0, tap_s = 0;
+                if (kMode == 1) {
+                    const int ctile = 2 * w.tile_m + (int)rank;
+                    int j = 0;
+                    while (j < p.rows_per_blk && n_boxes < 3) {
+                        const int q = ctile * p.rows_per_blk + j;
+                        const int h = q % p.img_rows;
+                        int cnt = p.rows_per_blk - j;
+                        if (cnt > p.img_rows - h) cnt = p.img_rows - h;
+                        if (cnt > kMaxRowMaps) cnt = kMaxRowMaps;
+                        box_h[n_boxes] = h; box_img[n_boxes] = q / p.img_rows; box_cnt[n_boxes] = cnt;
+                        ++n_boxes;
+                        j += cnt;
+                    }
+                    if (j < p.rows_per_blk) n_boxes = -1;  // more than three boxes: worked out per stage below
+                    tap = w.kb_begin / p.cblocks; cb = w.kb_begin % p.cblocks;
+                    tap_r = tap / p.taps_s; tap_s = tap % p.taps_s;
+                }
                 for (int kb = w.kb_begin; kb < w.kb_begin + w.num_kb; ++kb) {
+                    const int my_tap = tap, my_cb = cb, my_r = tap_r, my_s = tap_s;
+                    if (kMode == 1) {  // the next stage's tap and channel block
+                        if (++cb == p.cblocks) {
+                            cb = 0; ++tap;
+                            if (++tap_s == p.taps_s) { tap_s = 0; ++tap_r; }
+                        }
+                    }
                     if ((seq++ & 1u) != who) {  // the other producer's stage
                         if (++stage == kPStages) { stage = 0; phase ^= 1u; }
                         continue;
@@ -979,23 +1008,31 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmap_a, const CUten
                         ptx::mbar_expect_tx_cluster(bar, p.a_bytes + kPBBytes);
                         // A: this CTA's image rows at the tap's offset, one box per image touched (rows and
                         // columns outside the image, and images past the batch, read as zero)
-                        const int tap = kb / p.cblocks, cb = kb % p.cblocks;
-                        const int dh = p.tap_sign * (tap / p.taps_s) + p.off_h;
-                        const int dw = p.tap_sign * (tap % p.taps_s) + p.off_w;
-                        const int ctile = 2 * w.tile_m + (int)rank;
-                        int j = 0;
-                        while (j < p.rows_per_blk) {
-                            const int q = ctile * p.rows_per_blk + j;
-                            const int h = q % p.img_rows, img = q / p.img_rows;
-                            int cnt = p.rows_per_blk - j;
-                            if (cnt > p.img_rows - h) cnt = p.img_rows - h;
-                            if (cnt > kMaxRowMaps) cnt = kMaxRowMaps;
-                            ptx::tma_load_4d_pair(sa + (uint32_t)(j * p.img_w) * 128u, &row_maps[cnt - 1], bar, cb * 32, dw,
-                                                  h + dh, img);
-                            j += cnt;
+                        const int dh = p.tap_sign * my_r + p.off_h, dw = p.tap_sign * my_s + p.off_w;
+                        uint32_t dst = sa;
+#pragma unroll
+                        for (int b = 0; b < 3; ++b) {
+                            if (b < n_boxes) {
+                                ptx::tma_load_4d_pair(dst, &row_maps[box_cnt[b] - 1], bar, my_cb * 32, dw, box_h[b] + dh, box_img[b]);
+                                dst += (uint32_t)(box_cnt[b] * p.img_w) * 128u;
+                            }
                         }
-                        if (p.b_mn_major) ptx::tma_load_4d_pair(sb, &tmap_b, bar, 0, tap, cb * 32, n0 >> 5);
-                        else ptx::tma_load_2d_pair(sb, &tmap_b, bar, tap * p.ck + cb * 32, n0);
+                        if (n_boxes < 0) {
+                            const int ctile = 2 * w.tile_m + (int)rank;
+                            int j = 0;
+                            while (j < p.rows_per_blk) {
+                                const int q = ctile * p.rows_per_blk + j;
+                                const int h = q % p.img_rows, img = q / p.img_rows;
+                                int cnt = p.rows_per_blk - j;
+                                if (cnt > p.img_rows - h) cnt = p.img_rows - h;
+                                if (cnt > kMaxRowMaps) cnt = kMaxRowMaps;
+                                ptx::tma_load_4d_pair(sa + (uint32_t)(j * p.img_w) * 128u, &row_maps[cnt - 1], bar, my_cb * 32, dw,
+                                                      h + dh, img);
+                                j += cnt;
+                            }
+                        }
+                        if (p.b_mn_major) ptx::tma_load_4d_pair(sb, &tmap_b, bar, 0, my_tap, my_cb * 32, n0 >> 5);
+                        else ptx::tma_load_2d_pair(sb, &tmap_b, bar, my_tap * p.ck + my_cb * 32, n0);
                         if (++stage == kPStages) { stage = 0; phase ^= 1u; }
                         continue;
                     }

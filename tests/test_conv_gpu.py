@@ -81,6 +81,7 @@ SMALL = [
     (3, 256, 8, 7, 64, 3, 3, 1, 1),       # filter gradient with padded stages: 7-pixel rows take 8 K rows
     (2, 256, 10, 9, 32, 3, 3, 0, 0),      # the same without zero padding: the pad rows of B hold real pixels
     (2, 512, 4, 14, 32, 1, 1, 0, 0),      # padded stages, two 256-column tiles per tap
+    (64, 32, 3, 3, 64, 3, 3, 1, 1),       # 42 three-pixel rows per M-tile: fourteen images (copies) per tile and stage
 ]
 
 
