@@ -30,7 +30,7 @@ typedef enum {
     QFMT_ERR_BAD_ARG = -2,     /* NULL/misaligned pointer, bad dimension, workspace too small  */
     QFMT_ERR_UNSUPPORTED_ARCH = -3, /* current device is not compute capability 10.x           */
     QFMT_ERR_CUDA = -4,        /* a CUDA runtime/driver call failed (see qfmt_last_cuda_error)  */
-    QFMT_ERR_TIMEOUT = -5,     /* a bounded device-side wait expired (reported via status word) */
+    QFMT_ERR_TIMEOUT = -5,     /* a bounded device-side wait expired (reported via the status area) */
     QFMT_ERR_SCRATCH_LIMIT = -6 /* qfmt_gemm_builtin_scratch: the problem needs more than 16 MiB   */
 } qfmt_status_t;
 
@@ -253,14 +253,17 @@ typedef struct {
  * handles them.
  *
  *   d_workspace  device, 16-byte aligned, at least 16 bytes; qfmt_gemm_workspace_bytes(A, B) is
- *                the size that lets the library run at full speed.  Holds a status word (first
- *                4 bytes, cleared by the call) and, for products with few output tiles and a
+ *                the size that lets the library run at full speed.  Holds a status area (first
+ *                16 bytes: an error entry and the tag of the launch that last used the area; an
+ *                entry counts only under that launch's tag, so the call clears nothing and the
+ *                area's earlier contents never read as an error; read it with
+ *                qfmt_device_status) and, for products with few output tiles and a
  *                long K, split-K partial sums (K is shared among CTAs and the parts are added
  *                in a fixed pairwise order).  A smaller workspace gets fewer or no splits: still
  *                correct and reproducible, but the last bits can differ from a run with the
  *                recommended size.  Calls that share a workspace must be ordered on one stream.
  * M = 0 or N = 0 is a no-op; K = 0 writes zeros.  Every device-side wait is bounded: if one
- * expires the kernel stops, the status word holds QFMT_ERR_TIMEOUT and C is undefined.
+ * expires the kernel stops, the status area reports QFMT_ERR_TIMEOUT and C is undefined.
  * Errors: QFMT_ERR_BAD_FORMAT, QFMT_ERR_BAD_ARG (NULL or misaligned operand, ld too small,
  * mismatched K, workspace too small), QFMT_ERR_UNSUPPORTED_ARCH, QFMT_ERR_CUDA.
  */
@@ -286,7 +289,7 @@ size_t qfmt_gemm_workspace_bytes(const qfmt_matrix_t* A, const qfmt_matrix_t* B)
  *   d_Y, ldy         device, M x N, leading dimension ldy >= N; receives Y (format values)
  *   d_stats, accumulate   as for qfmt_bias_quantize_stats (d_stats may be NULL)
  *   d_workspace      device, 16-byte aligned, at least qfmt_linear_forward_workspace_bytes(A, B)
- *                    bytes: status word as for qfmt_gemm (qfmt_device_status reads it), split-K
+ *                    bytes: status area as for qfmt_gemm (qfmt_device_status reads it), split-K
  *                    partial sums when the kernels run separately, and the rounded bias
  * Errors: as qfmt_gemm and qfmt_bias_quantize_stats; QFMT_ERR_BAD_FORMAT also for loss_scale != 1.
  */
@@ -411,10 +414,10 @@ int qfmt_conv_tile_policy(int policy);
  * most 128, and at most 32 for the filter gradient; every tensor below 2^30 elements per
  * dimension product used as a GEMM extent.  Violations return QFMT_ERR_BAD_ARG.
  *   d_workspace  device, 16-byte aligned, >= qfmt_conv_workspace_bytes(op, geom) bytes: status
- *                word, and for the filter gradient the split-K partial sums (the long pixel
+ *                area, and for the filter gradient the split-K partial sums (the long pixel
  *                dimension is split over CTAs and the parts are added in a fixed pairwise order,
  *                so results are reproducible).
- * Errors and the bounded-wait status word: as qfmt_gemm.
+ * Errors and the bounded-wait status area: as qfmt_gemm.
  */
 typedef struct {
     int32_t n, c_in, h, w, c_out, r, s, pad_h, pad_w;
@@ -438,14 +441,15 @@ size_t qfmt_conv_workspace_bytes(int32_t op, const qfmt_conv_t* geom);  /* 0 if 
  * ends.  The call itself performs no cudaMalloc / cudaFree and uses no allocating library routine.
  *
  * Arguments A, B, d_C, ldc, fmt, stream: exactly as for qfmt_gemm, same results bit for bit.
- *   d_status_out  device, 4-byte aligned, or NULL.  If given, the kernel's status word
- *                 (QFMT_OK or QFMT_ERR_TIMEOUT) is copied there on `stream` after the product;
- *                 read it with qfmt_device_status(d_status_out, stream) or your own copy.
+ *   d_status_out  device, 4-byte aligned, or NULL.  If given, the product's status (QFMT_OK or
+ *                 QFMT_ERR_TIMEOUT, one int32: what qfmt_device_status would report for a
+ *                 caller-owned workspace) is written there on `stream` after the product; read it
+ *                 with a copy of your own.
  * Limits and rules
  *   - A problem for which qfmt_gemm_workspace_bytes(A, B) exceeds 16 MiB (16 777 216 bytes) is
  *     refused with QFMT_ERR_SCRATCH_LIMIT and nothing is enqueued; use qfmt_gemm with your own
  *     workspace.  That figure counts the whole workspace: the 256-byte header that holds the
- *     status word as well as the partial sums of a product whose K dimension is split, so a
+ *     status area as well as the partial sums of a product whose K dimension is split, so a
  *     product whose partial sums take exactly 16 MiB (1024 x 1024 outputs in four splits, say) is
  *     refused by those 256 bytes.  All argument checks of qfmt_gemm run before anything is
  *     enqueued, so every error return of this call leaves the stream untouched.
@@ -465,15 +469,15 @@ int qfmt_gemm_builtin_scratch(const qfmt_matrix_t* A, const qfmt_matrix_t* B, fl
  * (every wait in them is bounded; see QFMT_ERR_TIMEOUT).  Launches one small block that waits, with
  * the same primitives, on a barrier nothing ever arrives on; the wait gives up after
  * `limit_cycles` SM cycles (1 .. 2^24, i.e. at most a few milliseconds), the block records
- * QFMT_ERR_TIMEOUT in *d_status exactly as a contraction kernel would, its other warp notices the
- * block-wide abort flag, and the kernel returns normally: the context stays usable.
- *   d_status  device, 4-byte aligned: receives QFMT_ERR_TIMEOUT (cleared first); read it with
- *             qfmt_device_status(d_status, stream)
+ * QFMT_ERR_TIMEOUT in the status area exactly as a contraction kernel would, its other warp notices
+ * the block-wide abort flag, and the kernel returns normally: the context stays usable.
+ *   d_status  device, 8-byte aligned, 16 bytes: a status area as at the head of a workspace (any
+ *             contents); afterwards qfmt_device_status(d_status, stream) returns QFMT_ERR_TIMEOUT
  *   d_trace   device, four int32: [0] = 1 the waiting warp saw its wait expire, [1] = 1 the other warp
  *             left because of the abort flag, [2] = cycles waited, [3] unused
  * The paper has no counterpart; this is a diagnostic of the library.
  */
-int qfmt_selftest_bounded_wait(int32_t* d_status, uint32_t limit_cycles, int32_t* d_trace, void* stream);
+int qfmt_selftest_bounded_wait(void* d_status, uint32_t limit_cycles, int32_t* d_trace, void* stream);
 
 /*
  * Host-only view of the balanced schedule of the CTA-pair kernels (tile policy 3, and the forward /
@@ -490,8 +494,10 @@ int qfmt_selftest_bounded_wait(int32_t* d_status, uint32_t limit_cycles, int32_t
 int qfmt_selftest_pair_schedule(int64_t tiles, int32_t chunks_per_tile, int32_t pair, int32_t j, int32_t* out);
 
 /*
- * Synchronises `stream` and returns the status word of a workspace: QFMT_OK, or the error a
- * kernel recorded (QFMT_ERR_TIMEOUT), or QFMT_ERR_CUDA if the copy itself failed.
+ * Synchronises `stream` and returns what the status area at the head of a workspace (8-byte
+ * aligned, 16 bytes) says about the launch that last used it: QFMT_OK, or the error that launch
+ * recorded (QFMT_ERR_TIMEOUT), or QFMT_ERR_CUDA if the copy itself failed.  An area no launch has
+ * used yet, whatever it holds, reads as QFMT_OK unless its two words happen to agree (2^-48).
  */
 int qfmt_device_status(void* d_workspace, void* stream);
 

@@ -82,7 +82,12 @@ struct GemmParams {
     int M, N, K;
     long long ldc;
     float* C;
-    int* status;
+    // Status area at the head of the workspace: two 64-bit words.  Word 1 receives the launch's tag when
+    // the kernel starts; an error is recorded in word 0 as (tag << 16) | code.  A reader takes word 0 for
+    // an error only if its tag is word 1's, so nothing has to be cleared before a launch and whatever an
+    // earlier call (or nobody) left there reads as "no error".
+    unsigned long long* status;
+    unsigned long long launch_tag;
     int a_mn_major;  // op(A) stored with M contiguous
     int b_mn_major;  // op(B) stored with N contiguous
     int tiles_m, tiles_n;
@@ -264,13 +269,19 @@ __device__ __forceinline__ uint32_t make_idesc(int a_mn, int b_mn) {
 }
 
 // What a role does when one of its bounded waits runs out: the CTA-wide flag tells the other roles
-// to stop at their next check, the status word (first error wins) tells the host.
-__device__ __forceinline__ void raise_timeout(int* status, volatile int* abort_flag) {
+// to stop at their next check, the status area (first error of the launch wins) tells the host.
+__device__ __forceinline__ void raise_timeout(unsigned long long* status, unsigned long long tag, volatile int* abort_flag) {
     *abort_flag = 1;
-    atomicCAS(status, 0, (int)QFMT_ERR_TIMEOUT);
+    const unsigned long long seen = *reinterpret_cast<volatile unsigned long long*>(status);
+    if ((seen >> 16) != tag)  // no error of this launch yet; if another role gets in first, its error stands
+        atomicCAS(status, seen, (tag << 16) | (unsigned long long)(-(int)QFMT_ERR_TIMEOUT));
 }
 __device__ __forceinline__ void raise_timeout(const GemmParams& p, volatile int* abort_flag) {
-    raise_timeout(p.status, abort_flag);
+    raise_timeout(p.status, p.launch_tag, abort_flag);
+}
+// The first thread of the grid names the launch in the status area (see GemmParams::status).
+__device__ __forceinline__ void announce_launch(unsigned long long* status, unsigned long long tag) {
+    if (blockIdx.x == 0 && threadIdx.x == 0) *reinterpret_cast<volatile unsigned long long*>(status + 1) = tag;
 }
 
 // Self-test of the bounded-wait path with the primitives the GEMM kernels use, on a barrier that
@@ -281,7 +292,8 @@ __device__ __forceinline__ void raise_timeout(const GemmParams& p, volatile int*
 // trace[0] = 1 if warp 0's wait returned false, trace[1] = 1 if warp 1 left because of the flag,
 // trace[2] = cycles warp 0 waited.
 __global__ void __launch_bounds__(64, 1)
-bounded_wait_selftest_kernel(int* status, uint32_t limit, int* trace) {
+bounded_wait_selftest_kernel(unsigned long long* status, unsigned long long tag, uint32_t limit, int* trace) {
+    announce_launch(status, tag);
     __shared__ __align__(8) unsigned long long bar_storage;
     __shared__ int abort_word;
     volatile int* abort_flag = &abort_word;
@@ -299,7 +311,7 @@ bounded_wait_selftest_kernel(int* status, uint32_t limit, int* trace) {
             const bool ok = ptx::mbar_wait_bounded(bar, 0u, limit);  // phase 0 never completes
             trace[2] = (int)(clock64() - t0);
             if (!ok) {
-                raise_timeout(status, abort_flag);
+                raise_timeout(status, tag, abort_flag);
                 trace[0] = 1;
             }
         }
@@ -386,6 +398,7 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                  const __grid_constant__ CUtensorMap tmap_c, const __grid_constant__ CUtensorMap tmap_p,
                  const __grid_constant__ RowMaps row_maps, const GemmParams p) {
     extern __shared__ uint8_t smem_raw[];
+    announce_launch(p.status, p.launch_tag);
     const uint32_t raw = ptx::smem_addr(smem_raw);
     const uint32_t tiles = (raw + 1023u) & ~1023u;  // swizzled tiles need 1024-byte alignment
     const uint32_t out_stage = tiles + kStages * kStageBytes;
@@ -782,7 +795,7 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
             }
             if (dead) break;
         }
-        if (lane == 0) ptx::bulk_wait_all();  // shared memory stays valid until the last copy has read it
+        if (lane == 0) ptx::bulk_wait_read_all();  // shared memory stays valid until the last copy has read it
         __syncwarp();
     }
 
@@ -865,6 +878,7 @@ template <bool kEpi, int kKind, int kMode, bool kSk>
 __device__ __forceinline__ void pair_body(const CUtensorMap& tmap_a, const CUtensorMap& tmap_b, const CUtensorMap& tmap_c,
                                           const CUtensorMap* tmap_c2, const CUtensorMap* row_maps, const GemmParams& p) {
     extern __shared__ uint8_t smem_raw[];
+    announce_launch(p.status, p.launch_tag);
     const uint32_t raw = ptx::smem_addr(smem_raw);
     const uint32_t tiles = (raw + 1023u) & ~1023u;
     const uint32_t out_stage = tiles + kPStages * kPStageBytes;
@@ -1343,7 +1357,9 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmap_a, const CUten
                 __syncwarp();
             }
         }
-        if (lane == 0) ptx::bulk_wait_all();
+        // shared memory stays valid until the last copy has read it; the copies' writes are complete when
+        // the kernel is
+        if (lane == 0) ptx::bulk_wait_read_all();
         __syncwarp();
     }
 
@@ -1530,7 +1546,12 @@ void launch_splitk_reduce(const float* part, float* C, long long rows, long long
     else launch_splitk_reduce_as<float>(part, C, rows, cols, ldc, splits, sm_count, stream);
 }
 
-constexpr size_t kWorkspaceHeader = 256;  // status word and padding ahead of the partial sums
+constexpr size_t kWorkspaceHeader = 256;  // status area and padding ahead of the partial sums
+// Tag of the next launch (GemmParams::launch_tag): process-wide, never zero, 48 bits.
+unsigned long long next_launch_tag() {
+    static std::atomic<unsigned long long> counter{0};
+    return (counter.fetch_add(1) % ((1ull << 48) - 1)) + 1;
+}
 constexpr int kMaxSplits = 32;
 
 // Balanced schedule, second pass: CTA b's first piece began inside a tile and sits in slot b; add it
@@ -1745,7 +1766,7 @@ bool pair_schedule_fits(long long tiles, long long cpt) {
 }
 
 // Turns the balanced schedule of the pair kernel on: chunks per tile, the most pieces a pair can have,
-// and the flag words behind the workspace header (cleared on the stream, with the status word).
+// and the flag words behind the workspace header (cleared on the stream).
 int enable_pair_schedule(GemmParams* p, void* d_workspace, cudaStream_t stream) {
     p->sk_cpt = (p->kb_total + kChunkKB - 1) / kChunkKB;
     const long long total = (long long)p->tiles_m * p->tiles_n * p->sk_cpt;
@@ -1798,9 +1819,8 @@ int gemm_device(const qfmt_matrix_t* A, const qfmt_matrix_t* B, float* d_C, int6
     rc = current_device(&dev);
     if (rc != QFMT_OK) return rc;
 
-    int* status = reinterpret_cast<int*>(d_workspace);
-    QFMT_CUDA_TRY(cudaMemsetAsync(status, 0, 16, stream));
-    if (K == 0) {
+    if (K == 0) {  // no kernel: the status area itself says "no error"
+        QFMT_CUDA_TRY(cudaMemsetAsync(d_workspace, 0, 16, stream));
         QFMT_CUDA_TRY(cudaMemset2DAsync(d_C, (size_t)ldc * sizeof(float), 0, (size_t)N * sizeof(float), (size_t)M, stream));
         return QFMT_OK;
     }
@@ -1810,7 +1830,8 @@ int gemm_device(const qfmt_matrix_t* A, const qfmt_matrix_t* B, float* d_C, int6
     p.M = (int)M; p.N = (int)N; p.K = (int)K;
     p.ldc = ldc;
     p.C = d_C;
-    p.status = status;
+    p.status = reinterpret_cast<unsigned long long*>(d_workspace);
+    p.launch_tag = next_launch_tag();
     p.a_mn_major = A->trans ? 1 : 0;
     p.b_mn_major = B->trans ? 0 : 1;
     const DensePlan plan = plan_dense(M, N, K);
@@ -1925,9 +1946,8 @@ int gemm16_device(const qfmt_matrix16_t* A, const qfmt_matrix16_t* B, float* d_C
     DeviceInfo dev;
     rc = current_device(&dev);
     if (rc != QFMT_OK) return rc;
-    int* status = reinterpret_cast<int*>(d_workspace);
-    QFMT_CUDA_TRY(cudaMemsetAsync(status, 0, 16, stream));
     if (K == 0) {
+        QFMT_CUDA_TRY(cudaMemsetAsync(d_workspace, 0, 16, stream));
         QFMT_CUDA_TRY(cudaMemset2DAsync(d_C, (size_t)ldc * sizeof(float), 0, (size_t)N * sizeof(float), (size_t)M, stream));
         return QFMT_OK;
     }
@@ -1936,7 +1956,8 @@ int gemm16_device(const qfmt_matrix16_t* A, const qfmt_matrix16_t* B, float* d_C
     p.M = (int)M; p.N = (int)N; p.K = (int)K;
     p.ldc = ldc;
     p.C = d_C;
-    p.status = status;
+    p.status = reinterpret_cast<unsigned long long*>(d_workspace);
+    p.launch_tag = next_launch_tag();
     p.a_mn_major = A->trans ? 1 : 0;
     p.b_mn_major = B->trans ? 0 : 1;
     p.tile_rows = 2 * kBM;
@@ -2139,14 +2160,12 @@ int conv_device(int op, const qfmt_conv_t* g, const float* d_p, const float* d_q
         pointwise_operands(op, g, d_p, d_q, &A, &B, &ldc);
         return gemm_device(&A, &B, d_out, ldc, fmt, d_workspace, workspace_bytes, stream);
     }
-    int* status = reinterpret_cast<int*>(d_workspace);
-    QFMT_CUDA_TRY(cudaMemsetAsync(status, 0, 16, stream));
-
     const uint64_t N = g->n, CI = g->c_in, H = g->h, W = g->w, CO = g->c_out, R = g->r, S = g->s;
     const uint64_t OH = plan.oh, OW = plan.ow, TAPS = R * S;
     GemmParams p;
     dense_defaults(&p);
-    p.status = status;
+    p.status = reinterpret_cast<unsigned long long*>(d_workspace);
+    p.launch_tag = next_launch_tag();
     p.taps = (int)TAPS;
     p.taps_s = (int)S;
     p.tma_store = 1;  // channel counts are multiples of 32 and the bases 16-byte aligned
@@ -2388,7 +2407,7 @@ int linear_forward_device(const qfmt_matrix_t* A, const qfmt_matrix_t* B, const 
     if (d_workspace == nullptr || (reinterpret_cast<uintptr_t>(d_workspace) & 15u)) return QFMT_ERR_BAD_ARG;
     const size_t bias_bytes = linear_bias_bytes(N);
     if (workspace_bytes < kWorkspaceHeader + bias_bytes + 256) return QFMT_ERR_BAD_ARG;
-    // layout: [status word and padding | GEMM partial sums (unfused path) ... | rounded bias at the end,
+    // layout: [status area and padding | GEMM partial sums (unfused path) ... | rounded bias at the end,
     // on a 256-byte boundary]
     const size_t gemm_bytes = (workspace_bytes - bias_bytes) & ~(size_t)255u;
     float* rbias = reinterpret_cast<float*>(reinterpret_cast<char*>(d_workspace) + gemm_bytes);
@@ -2482,23 +2501,26 @@ extern "C" size_t qfmt_gemm_packed16_workspace_bytes(const qfmt_matrix16_t* A, c
 
 extern "C" int qfmt_device_status(void* d_workspace, void* stream) {
     if (d_workspace == nullptr) return QFMT_ERR_BAD_ARG;
-    int st = 0;
-    QFMT_CUDA_TRY(cudaMemcpyAsync(&st, d_workspace, sizeof(int), cudaMemcpyDeviceToHost, (cudaStream_t)stream));
+    if (reinterpret_cast<uintptr_t>(d_workspace) & 7u) return QFMT_ERR_BAD_ARG;
+    unsigned long long words[2] = {0, 0};
+    QFMT_CUDA_TRY(cudaMemcpyAsync(words, d_workspace, sizeof(words), cudaMemcpyDeviceToHost, (cudaStream_t)stream));
     QFMT_CUDA_TRY(cudaStreamSynchronize((cudaStream_t)stream));
-    return st;
+    // an error counts only if it carries the tag of the launch that last used the area (GemmParams::status)
+    if (words[1] != 0 && (words[0] >> 16) == words[1]) return -(int)(words[0] & 0xFFFFu);
+    return QFMT_OK;
 }
 
 
-extern "C" int qfmt_selftest_bounded_wait(int32_t* d_status, uint32_t limit_cycles, int32_t* d_trace, void* stream) {
+extern "C" int qfmt_selftest_bounded_wait(void* d_status, uint32_t limit_cycles, int32_t* d_trace, void* stream) {
     if (d_status == nullptr || d_trace == nullptr) return QFMT_ERR_BAD_ARG;
-    if ((reinterpret_cast<uintptr_t>(d_status) & 3u) || (reinterpret_cast<uintptr_t>(d_trace) & 3u)) return QFMT_ERR_BAD_ARG;
+    if ((reinterpret_cast<uintptr_t>(d_status) & 7u) || (reinterpret_cast<uintptr_t>(d_trace) & 3u)) return QFMT_ERR_BAD_ARG;
     if (limit_cycles == 0 || limit_cycles > (1u << 24)) return QFMT_ERR_BAD_ARG;  // at most a few milliseconds
     qfmt::DeviceInfo dev;
     int rc = qfmt::current_device(&dev);
     if (rc != QFMT_OK) return rc;
-    QFMT_CUDA_TRY(cudaMemsetAsync(d_status, 0, sizeof(int32_t), (cudaStream_t)stream));
     QFMT_CUDA_TRY(cudaMemsetAsync(d_trace, 0, 4 * sizeof(int32_t), (cudaStream_t)stream));
-    qfmt::bounded_wait_selftest_kernel<<<1, 64, 0, (cudaStream_t)stream>>>(d_status, limit_cycles, d_trace);
+    qfmt::bounded_wait_selftest_kernel<<<1, 64, 0, (cudaStream_t)stream>>>(
+        reinterpret_cast<unsigned long long*>(d_status), qfmt::next_launch_tag(), limit_cycles, d_trace);
     QFMT_CUDA_TRY(cudaGetLastError());
     return QFMT_OK;
 }
@@ -2510,6 +2532,12 @@ namespace qfmt {
 namespace {
 
 constexpr size_t kBuiltinScratchBytes = (size_t)16 << 20;  // 16 MiB per GPU that loads the library
+
+// The status area's verdict as one int32 (what qfmt_device_status computes on the host).
+__global__ void status_word_kernel(const unsigned long long* status, int32_t* out) {
+    const unsigned long long w0 = status[0], w1 = status[1];
+    *out = (w1 != 0 && (w0 >> 16) == w1) ? -(int32_t)(w0 & 0xFFFFu) : 0;
+}
 
 // Lives in every device's copy of the module.  In host code this name is only a handle for
 // cudaGetSymbolAddress: it is not a device address and must never be handed to a kernel.
@@ -2548,14 +2576,17 @@ extern "C" int qfmt_gemm_builtin_scratch(const qfmt_matrix_t* A, const qfmt_matr
     void* scratch = nullptr;
     rc = qfmt::builtin_scratch_address(&scratch);
     if (rc != QFMT_OK) return rc;
-    // The array still holds what the previous call left.  Only the status word at its head has to
-    // start at zero; a product with work to do clears it itself, so it is cleared here only for
-    // the call that enqueues no kernel (M or N zero), which must not report an older call's status.
+    // The array still holds what the previous call left.  A product with work to do names its launch in
+    // the status area at the array's head, which makes older entries there void; the area is cleared
+    // here only for the call that enqueues no kernel (M or N zero), which must not report an older
+    // call's status.
     if (M == 0 || N == 0) QFMT_CUDA_TRY(cudaMemsetAsync(scratch, 0, 16, (cudaStream_t)stream));
     rc = qfmt::gemm_device(A, B, d_C, ldc, fmt, scratch, qfmt::kBuiltinScratchBytes, (cudaStream_t)stream);
     if (rc != QFMT_OK) return rc;
-    if (d_status_out != nullptr)
-        QFMT_CUDA_TRY(cudaMemcpyAsync(d_status_out, scratch, sizeof(int32_t), cudaMemcpyDeviceToDevice,
-                                      (cudaStream_t)stream));
+    if (d_status_out != nullptr) {
+        qfmt::status_word_kernel<<<1, 1, 0, (cudaStream_t)stream>>>(reinterpret_cast<const unsigned long long*>(scratch),
+                                                                    d_status_out);
+        QFMT_CUDA_TRY(cudaGetLastError());
+    }
     return QFMT_OK;
 }
