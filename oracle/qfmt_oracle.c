@@ -23,6 +23,9 @@
  *     (fp64 accumulation of exact products) together with sum |a||b| for the error bound.
  *   - Section III-B, FMAC, a16 = round(a16 + x16*y16), and Algorithm 1 (FMAC-8): the exact value
  *     of a + x*y is formed in integers and rounded once; the master accumulator adds in fp32.
+ *   - Section IV-A: FMAC-8 also names a convolution whose sums are accumulated as in
+ *     Algorithm 1; the order in which a convolution's reduction is walked is a reading, stated
+ *     where oracle_conv_fmac8 is defined.
  *   - Section IV-A's layer formula Y = R(R(W^T X) + R(B)): exact sum of the two rounded
  *     terms, rounded once more.
  *   - Section V: "denormal fraction" of each tensor is the logged statistic.
@@ -758,6 +761,112 @@ void oracle_conv(int which, const int64_t *geom, const float *P, const float *Q,
         } else {
             int64_t s = f % g.s, r = (f / g.s) % g.r, ci = (f / (g.s * g.r)) % g.ci, co = f / (g.s * g.r * g.ci);
             conv_wgrad_one(&g, P, Q, co, ci, r, s, &c[k], tk);
+        }
+    }
+}
+
+/* ------------------------------------------------------------------------------------------ */
+/* FMAC-8 for convolution layers.  Section IV-A counts as FMAC-8 "a matrix multiplication or    */
+/* convolution" whose sums are accumulated as in Algorithm 1: runs of `group` fused multiply-    */
+/* accumulates in the 16-bit format, each run's sum added in fp32 to a single-precision total,   */
+/* one rounding of the total at the end.  The paper does not say in which order a convolution's  */
+/* reduction index is walked; the reading taken here (the order of an unfolded, channels-last   */
+/* operand matrix):                                                                              */
+/*   forward          filter taps row by row (r, then s), within a tap the input channels        */
+/*   data gradient    filter taps row by row (r, then s), within a tap the output channels       */
+/*   filter gradient  images, within an image the output rows, within a row the output pixels    */
+/* A term whose input position lies in the zero padding is a term with a zero factor: it keeps   */
+/* its place in its run (an FMAC with a zero factor leaves the accumulator as it is).            */
+/* ------------------------------------------------------------------------------------------ */
+typedef struct {
+    uint32_t total;   /* fp32 word of the single-precision total */
+    uint32_t run_sum; /* the 16-bit accumulator, as the fp32 word of its value */
+    int in_run, group, e, m, keep;
+} fmac8_state;
+
+static void fmac8_begin(fmac8_state *st, int e, int m, int keep, int group) {
+    st->total = 0; st->run_sum = 0; st->in_run = 0;
+    st->group = group; st->e = e; st->m = m; st->keep = keep;
+}
+static void fmac8_term(fmac8_state *st, float x, float y) {
+    st->run_sum = oracle_fmac_bits(st->run_sum, word_of(x), word_of(y), st->e, st->m, st->keep);
+    if (++st->in_run == st->group) {
+        st->total = f32_add_bits(st->total, st->run_sum);
+        st->run_sum = 0;
+        st->in_run = 0;
+    }
+}
+static uint32_t fmac8_end(fmac8_state *st) {
+    if (st->in_run > 0) st->total = f32_add_bits(st->total, st->run_sum);
+    return oracle_quantize_bits(st->total, st->e, st->m, st->keep, NULL);
+}
+
+static uint32_t conv_fmac8_fwd_one(const conv_t *g, const float *X, const float *Wt, int64_t n, int64_t co,
+                                   int64_t oh, int64_t ow, int e, int m, int keep, int group) {
+    fmac8_state st;
+    fmac8_begin(&st, e, m, keep, group);
+    for (int64_t r = 0; r < g->r; ++r)
+        for (int64_t s = 0; s < g->s; ++s)
+            for (int64_t ci = 0; ci < g->ci; ++ci) {
+                int64_t ih = oh + r - g->pad_h, iw = ow + s - g->pad_w;
+                int inside = ih >= 0 && ih < g->h && iw >= 0 && iw < g->w;
+                float x = inside ? X[((n * g->ci + ci) * g->h + ih) * g->w + iw] : 0.0f;
+                fmac8_term(&st, x, Wt[((co * g->ci + ci) * g->r + r) * g->s + s]);
+            }
+    return fmac8_end(&st);
+}
+
+static uint32_t conv_fmac8_dgrad_one(const conv_t *g, const float *dY, const float *Wt, int64_t n, int64_t ci,
+                                     int64_t ih, int64_t iw, int e, int m, int keep, int group) {
+    int64_t OH = conv_oh(g), OW = conv_ow(g);
+    fmac8_state st;
+    fmac8_begin(&st, e, m, keep, group);
+    for (int64_t r = 0; r < g->r; ++r)
+        for (int64_t s = 0; s < g->s; ++s)
+            for (int64_t co = 0; co < g->co; ++co) {
+                int64_t oh = ih - r + g->pad_h, ow = iw - s + g->pad_w;
+                int inside = oh >= 0 && oh < OH && ow >= 0 && ow < OW;
+                float x = inside ? dY[((n * g->co + co) * OH + oh) * OW + ow] : 0.0f;
+                fmac8_term(&st, x, Wt[((co * g->ci + ci) * g->r + r) * g->s + s]);
+            }
+    return fmac8_end(&st);
+}
+
+static uint32_t conv_fmac8_wgrad_one(const conv_t *g, const float *dY, const float *X, int64_t co, int64_t ci,
+                                     int64_t r, int64_t s, int e, int m, int keep, int group) {
+    int64_t OH = conv_oh(g), OW = conv_ow(g);
+    fmac8_state st;
+    fmac8_begin(&st, e, m, keep, group);
+    for (int64_t n = 0; n < g->n; ++n)
+        for (int64_t oh = 0; oh < OH; ++oh)
+            for (int64_t ow = 0; ow < OW; ++ow) {
+                int64_t ih = oh + r - g->pad_h, iw = ow + s - g->pad_w;
+                int inside = ih >= 0 && ih < g->h && iw >= 0 && iw < g->w;
+                float y = inside ? X[((n * g->ci + ci) * g->h + ih) * g->w + iw] : 0.0f;
+                fmac8_term(&st, dY[((n * g->co + co) * OH + oh) * OW + ow], y);
+            }
+    return fmac8_end(&st);
+}
+
+/* Same index conventions as oracle_conv; out receives the fp32 words of the rounded results. */
+void oracle_conv_fmac8(int which, const int64_t *geom, const float *P, const float *Q, int e, int m,
+                       int keep_denormals, int group, const int64_t *idx, int64_t count, uint32_t *out) {
+    conv_t g;
+    g.n = geom[0]; g.ci = geom[1]; g.h = geom[2]; g.w = geom[3]; g.co = geom[4];
+    g.r = geom[5]; g.s = geom[6]; g.pad_h = geom[7]; g.pad_w = geom[8];
+    int64_t OH = conv_oh(&g), OW = conv_ow(&g);
+#pragma omp parallel for schedule(static)
+    for (int64_t k = 0; k < count; ++k) {
+        int64_t f = idx ? idx[k] : k;
+        if (which == 0) {
+            int64_t ow = f % OW, oh = (f / OW) % OH, co = (f / (OW * OH)) % g.co, n = f / (OW * OH * g.co);
+            out[k] = conv_fmac8_fwd_one(&g, P, Q, n, co, oh, ow, e, m, keep_denormals, group);
+        } else if (which == 1) {
+            int64_t iw = f % g.w, ih = (f / g.w) % g.h, ci = (f / (g.w * g.h)) % g.ci, n = f / (g.w * g.h * g.ci);
+            out[k] = conv_fmac8_dgrad_one(&g, P, Q, n, ci, ih, iw, e, m, keep_denormals, group);
+        } else {
+            int64_t s = f % g.s, r = (f / g.s) % g.r, ci = (f / (g.s * g.r)) % g.ci, co = f / (g.s * g.r * g.ci);
+            out[k] = conv_fmac8_wgrad_one(&g, P, Q, co, ci, r, s, e, m, keep_denormals, group);
         }
     }
 }
