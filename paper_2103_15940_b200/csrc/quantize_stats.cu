@@ -206,6 +206,7 @@ quantize_stats_transpose_kernel(const uint32_t* __restrict__ in, uint32_t* __res
 // 16-bit storage (Section II: activations and gradients are kept in 16 bits, halving storage and
 // bandwidth): the rounding pass writing packed codes instead of fp32 containers, 4 bytes read and
 // 2 written per element, and the pass that expands codes back to containers for the contraction.
+// A thread takes eight consecutive elements: two 128-bit loads, one 128-bit store.
 // kRare: results below the smallest normal are expected to be rare (formats with e >= 6): the denormal
 // grid sits behind a branch (quantize_pack_one_rare_denormals).
 template <bool kStats, bool kScale, bool kRare>
@@ -219,36 +220,38 @@ quantize_stats_pack16_kernel(const uint32_t* __restrict__ in, uint16_t* __restri
         for (int i = threadIdx.x; i < nbins * 32; i += kThreads) lane_hist[i] = 0u;
         __syncthreads();
     }
-    // vector body: a thread takes four consecutive elements per step (one 128-bit load, one 64-bit
-    // store), a warp 512 consecutive bytes in and 256 out, kUnroll loads in flight per thread
-    const unsigned long long n4 = vec ? n / 4 : 0ull;
-    const unsigned long long stride = (unsigned long long)gridDim.x * (kThreads * kUnroll);
-    for (unsigned long long base = (unsigned long long)blockIdx.x * (kThreads * kUnroll); base < n4; base += stride) {
-        uint4 v[kUnroll];
+    const unsigned long long n8 = vec ? n / 8 : 0ull;
+    const unsigned long long stride = (unsigned long long)gridDim.x * (kThreads * 2);
+    for (unsigned long long base = (unsigned long long)blockIdx.x * (kThreads * 2); base < n8; base += stride) {
+        uint4 v[2][2];
 #pragma unroll
-        for (int u = 0; u < kUnroll; ++u) {
+        for (int u = 0; u < 2; ++u) {
             const unsigned long long idx = base + (unsigned long long)u * kThreads + threadIdx.x;
-            if (idx < n4) v[u] = load_stream(reinterpret_cast<const uint4*>(in) + idx);
+            if (idx < n8) {
+                v[u][0] = load_stream(reinterpret_cast<const uint4*>(in) + 2 * idx);
+                v[u][1] = load_stream(reinterpret_cast<const uint4*>(in) + 2 * idx + 1);
+            }
         }
 #pragma unroll
-        for (int u = 0; u < kUnroll; ++u) {
+        for (int u = 0; u < 2; ++u) {
             const unsigned long long idx = base + (unsigned long long)u * kThreads + threadIdx.x;
-            if (idx < n4) {
-                const uint32_t w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
-                uint32_t c[4];
+            if (idx < n8) {
+                const uint32_t w[8] = {v[u][0].x, v[u][0].y, v[u][0].z, v[u][0].w, v[u][1].x, v[u][1].y, v[u][1].z, v[u][1].w};
+                uint32_t c[8];
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
+                for (int j = 0; j < 8; ++j) {
                     int b;
                     c[j] = kRare ? quantize_pack_one_rare_denormals<kScale>(w[j], p, sign_shift, b)
                                  : quantize_pack_one<kScale>(w[j], p, sign_shift, b);
                     if (kStats) atomicAdd(&lane_hist[b * 32 + lane], 1u);
                 }
-                store_stream(reinterpret_cast<uint2*>(codes) + idx, make_uint2(c[0] | (c[1] << 16), c[2] | (c[3] << 16)));
+                store_stream(reinterpret_cast<uint4*>(codes) + idx,
+                             make_uint4(c[0] | (c[1] << 16), c[2] | (c[3] << 16), c[4] | (c[5] << 16), c[6] | (c[7] << 16)));
             }
         }
     }
     // what the vector body leaves (everything when the pointers are not 16-byte aligned)
-    const unsigned long long done = n4 * 4;
+    const unsigned long long done = n8 * 8;
     for (unsigned long long i = done + (unsigned long long)blockIdx.x * kThreads + threadIdx.x; i < n;
          i += (unsigned long long)gridDim.x * kThreads) {
         int b;
