@@ -428,6 +428,31 @@ int qfmt_conv(int32_t op, const qfmt_conv_t* geom, const float* d_p, const float
 size_t qfmt_conv_workspace_bytes(int32_t op, const qfmt_conv_t* geom);  /* 0 if geom is unsupported */
 
 /*
+ * The three products of a convolution layer with FMAC-8 accumulation (Section IV-A: FMAC-8 means
+ * Algorithm 1 "or a matrix multiplication or convolution" whose sums are accumulated in its manner;
+ * Table II's convolutional networks are trained this way).  Same tensors, layouts and operand order as
+ * qfmt_conv (channels-last; unit stride, zero padding), same accumulation and output rules as
+ * qfmt_gemm_fmac8: runs of eight FMACs in the 16-bit format, every run's sum added in fp32 to a
+ * single-precision total, the total rounded to the format at the end; d_out holds format values and
+ * is bit-exact against that definition.
+ * The paper does not fix the order in which a convolution's reduction index is walked.  This library
+ * walks it as the unfolded channels-last operand matrix would be:
+ *     forward          filter taps row by row (r, then s), within a tap the input channels
+ *     data gradient    filter taps row by row (r, then s), within a tap the output channels
+ *     filter gradient  images, within an image the output rows, within a row the output pixels
+ * A term whose input position lies in the zero padding is a term with a zero factor: it keeps its place
+ * in its run of eight.
+ *   geom     any positive sizes (no multiple-of-32 rule here); every tensor below 2^31 elements
+ *   d_p, d_q, d_out   as for qfmt_conv, 4-byte aligned; operands hold values of the format
+ *   fmt, d_stats, accumulate, path   as for qfmt_gemm_fmac8 (statistics of the output tensor)
+ * Plain-ALU work, like qfmt_gemm_fmac8; the activation-like operand is gathered at the taps' offsets
+ * while it is staged, nothing is unfolded in memory.
+ * Errors: QFMT_ERR_BAD_FORMAT, QFMT_ERR_BAD_ARG, QFMT_ERR_UNSUPPORTED_ARCH, QFMT_ERR_CUDA.
+ */
+int qfmt_conv_fmac8(int32_t op, const qfmt_conv_t* geom, const float* d_p, const float* d_q, float* d_out,
+                    const qfmt_format_t* fmt, qfmt_stats_t* d_stats, int accumulate, int path, void* stream);
+
+/*
  * qfmt_gemm for callers that cannot allocate device memory.  (The paper has no counterpart of
  * this call; it exists for the way the library gets embedded.)
  *

@@ -80,7 +80,7 @@ def _L() -> ctypes.CDLL:
         lib.oracle_unpack16.restype = None
         lib.oracle_dls_update.argtypes = [vp, vp, i64]
         lib.oracle_dls_update.restype = None
-        lib.oracle_conv_fmac8.argtypes = [i32, vp, vp, vp, i32, i32, i32, i32, vp, i64, vp]
+        lib.oracle_conv_fmac8.argtypes = [i32, vp, vp, vp, i32, i32, i32, i32, vp, i64, vp, vp]
         lib.oracle_conv_fmac8.restype = None
         _lib = lib
     return _lib
@@ -310,10 +310,11 @@ def conv(which: int, P: np.ndarray, Q: np.ndarray, geom, idx: Optional[np.ndarra
 
 
 def conv_fmac8(which: int, P: np.ndarray, Q: np.ndarray, geom, e: int, m: int, denormals: int = 1, group: int = 8,
-               idx: Optional[np.ndarray] = None) -> np.ndarray:
+               idx: Optional[np.ndarray] = None, want_master: bool = False):
     """Algorithm 1 applied to a convolution's sums (NCHW tensors, operands and index spaces as for
     ``conv``): runs of ``group`` FMACs along the reduction in the order stated in qfmt_oracle.c, padding
-    positions as zero factors.  Returns the rounded results as float32, flat."""
+    positions as zero factors.  Returns the rounded results as float32, flat (and, if asked, the fp32
+    totals before the final rounding)."""
     n, ci, h, w, co, r, s, ph, pw = [int(v) for v in geom]
     oh, ow = h + 2 * ph - r + 1, w + 2 * pw - s + 1
     total = {CONV_FWD: n * co * oh * ow, CONV_DGRAD: n * ci * h * w, CONV_WGRAD: co * ci * r * s}[which]
@@ -328,6 +329,8 @@ def conv_fmac8(which: int, P: np.ndarray, Q: np.ndarray, geom, e: int, m: int, d
     else:
         count = total
     out = np.empty(count, dtype=np.uint32)
+    master = np.empty(count, dtype=np.uint32) if want_master else None
     _L().oracle_conv_fmac8(which, g.ctypes.data, P.ctypes.data, Q.ctypes.data, e, m, int(denormals), int(group),
-                           idx.ctypes.data if idx is not None else None, count, out.ctypes.data)
-    return out.view(np.float32)
+                           idx.ctypes.data if idx is not None else None, count, out.ctypes.data,
+                           master.ctypes.data if want_master else None)
+    return (out.view(np.float32), master.view(np.float32)) if want_master else out.view(np.float32)

@@ -796,13 +796,14 @@ static void fmac8_term(fmac8_state *st, float x, float y) {
         st->in_run = 0;
     }
 }
-static uint32_t fmac8_end(fmac8_state *st) {
+static uint32_t fmac8_end(fmac8_state *st, uint32_t *total_out) {
     if (st->in_run > 0) st->total = f32_add_bits(st->total, st->run_sum);
+    if (total_out) *total_out = st->total; /* the single-precision total before the final rounding */
     return oracle_quantize_bits(st->total, st->e, st->m, st->keep, NULL);
 }
 
 static uint32_t conv_fmac8_fwd_one(const conv_t *g, const float *X, const float *Wt, int64_t n, int64_t co,
-                                   int64_t oh, int64_t ow, int e, int m, int keep, int group) {
+                                   int64_t oh, int64_t ow, int e, int m, int keep, int group, uint32_t *total_out) {
     fmac8_state st;
     fmac8_begin(&st, e, m, keep, group);
     for (int64_t r = 0; r < g->r; ++r)
@@ -813,11 +814,11 @@ static uint32_t conv_fmac8_fwd_one(const conv_t *g, const float *X, const float 
                 float x = inside ? X[((n * g->ci + ci) * g->h + ih) * g->w + iw] : 0.0f;
                 fmac8_term(&st, x, Wt[((co * g->ci + ci) * g->r + r) * g->s + s]);
             }
-    return fmac8_end(&st);
+    return fmac8_end(&st, total_out);
 }
 
 static uint32_t conv_fmac8_dgrad_one(const conv_t *g, const float *dY, const float *Wt, int64_t n, int64_t ci,
-                                     int64_t ih, int64_t iw, int e, int m, int keep, int group) {
+                                     int64_t ih, int64_t iw, int e, int m, int keep, int group, uint32_t *total_out) {
     int64_t OH = conv_oh(g), OW = conv_ow(g);
     fmac8_state st;
     fmac8_begin(&st, e, m, keep, group);
@@ -829,11 +830,11 @@ static uint32_t conv_fmac8_dgrad_one(const conv_t *g, const float *dY, const flo
                 float x = inside ? dY[((n * g->co + co) * OH + oh) * OW + ow] : 0.0f;
                 fmac8_term(&st, x, Wt[((co * g->ci + ci) * g->r + r) * g->s + s]);
             }
-    return fmac8_end(&st);
+    return fmac8_end(&st, total_out);
 }
 
 static uint32_t conv_fmac8_wgrad_one(const conv_t *g, const float *dY, const float *X, int64_t co, int64_t ci,
-                                     int64_t r, int64_t s, int e, int m, int keep, int group) {
+                                     int64_t r, int64_t s, int e, int m, int keep, int group, uint32_t *total_out) {
     int64_t OH = conv_oh(g), OW = conv_ow(g);
     fmac8_state st;
     fmac8_begin(&st, e, m, keep, group);
@@ -845,12 +846,14 @@ static uint32_t conv_fmac8_wgrad_one(const conv_t *g, const float *dY, const flo
                 float y = inside ? X[((n * g->ci + ci) * g->h + ih) * g->w + iw] : 0.0f;
                 fmac8_term(&st, dY[((n * g->co + co) * OH + oh) * OW + ow], y);
             }
-    return fmac8_end(&st);
+    return fmac8_end(&st, total_out);
 }
 
-/* Same index conventions as oracle_conv; out receives the fp32 words of the rounded results. */
+/* Same index conventions as oracle_conv; out receives the fp32 words of the rounded results and     */
+/* master (may be NULL) those of the single-precision totals before the final rounding.              */
 void oracle_conv_fmac8(int which, const int64_t *geom, const float *P, const float *Q, int e, int m,
-                       int keep_denormals, int group, const int64_t *idx, int64_t count, uint32_t *out) {
+                       int keep_denormals, int group, const int64_t *idx, int64_t count, uint32_t *out,
+                       uint32_t *master) {
     conv_t g;
     g.n = geom[0]; g.ci = geom[1]; g.h = geom[2]; g.w = geom[3]; g.co = geom[4];
     g.r = geom[5]; g.s = geom[6]; g.pad_h = geom[7]; g.pad_w = geom[8];
@@ -860,13 +863,13 @@ void oracle_conv_fmac8(int which, const int64_t *geom, const float *P, const flo
         int64_t f = idx ? idx[k] : k;
         if (which == 0) {
             int64_t ow = f % OW, oh = (f / OW) % OH, co = (f / (OW * OH)) % g.co, n = f / (OW * OH * g.co);
-            out[k] = conv_fmac8_fwd_one(&g, P, Q, n, co, oh, ow, e, m, keep_denormals, group);
+            out[k] = conv_fmac8_fwd_one(&g, P, Q, n, co, oh, ow, e, m, keep_denormals, group, master ? &master[k] : NULL);
         } else if (which == 1) {
             int64_t iw = f % g.w, ih = (f / g.w) % g.h, ci = (f / (g.w * g.h)) % g.ci, n = f / (g.w * g.h * g.ci);
-            out[k] = conv_fmac8_dgrad_one(&g, P, Q, n, ci, ih, iw, e, m, keep_denormals, group);
+            out[k] = conv_fmac8_dgrad_one(&g, P, Q, n, ci, ih, iw, e, m, keep_denormals, group, master ? &master[k] : NULL);
         } else {
             int64_t s = f % g.s, r = (f / g.s) % g.r, ci = (f / (g.s * g.r)) % g.ci, co = f / (g.s * g.r * g.ci);
-            out[k] = conv_fmac8_wgrad_one(&g, P, Q, co, ci, r, s, e, m, keep_denormals, group);
+            out[k] = conv_fmac8_wgrad_one(&g, P, Q, co, ci, r, s, e, m, keep_denormals, group, master ? &master[k] : NULL);
         }
     }
 }

@@ -143,6 +143,8 @@ def _bind_optional(L: ctypes.CDLL) -> None:
     L.qfmt_conv.restype = ci
     L.qfmt_conv_workspace_bytes.argtypes = [ctypes.c_int32, convp]
     L.qfmt_conv_workspace_bytes.restype = sz
+    L.qfmt_conv_fmac8.argtypes = [ctypes.c_int32, convp, vp, vp, vp, ctypes.POINTER(qfmt_format_t), vp, ci, ci, vp]
+    L.qfmt_conv_fmac8.restype = ci
     L.qfmt_gemm_builtin_scratch.argtypes = [matp, matp, vp, ctypes.c_int64, ctypes.POINTER(qfmt_format_t), vp, vp]
     L.qfmt_gemm_builtin_scratch.restype = ci
     L.qfmt_selftest_bounded_wait.argtypes = [vp, ctypes.c_uint32, vp, vp]
@@ -356,6 +358,14 @@ def qfmt_conv(op: int, geom: qfmt_conv_t, d_p, d_q, d_out, fmt: qfmt_format_t, d
     see qfmt_conv in include/qfmt.h."""
     _check(lib().qfmt_conv(int(op), ctypes.byref(geom), _ptr(d_p), _ptr(d_q), _ptr(d_out), ctypes.byref(fmt),
                            _ptr(d_workspace), int(workspace_bytes), _stream_handle(stream)), "qfmt_conv")
+
+
+def qfmt_conv_fmac8(op: int, geom: qfmt_conv_t, d_p, d_q, d_out, fmt: qfmt_format_t, d_stats=None, accumulate: int = 0,
+                    path: int = 0, stream=None) -> None:
+    """A convolution's forward / data-gradient / filter-gradient product with FMAC-8 accumulation; see
+    qfmt_conv_fmac8 in include/qfmt.h."""
+    _check(lib().qfmt_conv_fmac8(int(op), ctypes.byref(geom), _ptr(d_p), _ptr(d_q), _ptr(d_out), ctypes.byref(fmt),
+                                 _ptr(d_stats), int(accumulate), int(path), _stream_handle(stream)), "qfmt_conv_fmac8")
 
 
 def qfmt_conv_tile_policy(policy: int) -> None:

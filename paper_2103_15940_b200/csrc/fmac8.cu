@@ -18,6 +18,16 @@
 //     smallest normal afterwards.
 // They keep a 64 x 64 (resp. 64 x 128) tile of outputs per block in registers and stream
 // 32-deep slices of the operands through shared memory.
+//
+// Convolution layers (Section IV-A: FMAC-8 also names a convolution whose sums are accumulated this
+// way).  The three products of a unit-stride, zero-padded convolution on channels-last tensors run on
+// the same kernels (their kConv instantiations) as matrix products whose activation-like operand is
+// gathered at the filter taps' offsets while a slice is staged; a position in the padding is a zero
+// factor that keeps its place in its run of eight.  Order of the reduction index (the paper leaves it
+// open; this is the order of the unfolded channels-last operand matrix):
+//   forward          taps (r, then s), within a tap the input channels
+//   data gradient    taps (r, then s), within a tap the output channels
+//   filter gradient  images, within an image the output rows, within a row the output pixels
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -32,6 +42,19 @@ constexpr int kFmThreads = 256;
 constexpr int kFmBK = 32;    // K elements per shared-memory slice: four groups of eight
 constexpr int kGroup = 8;    // FMACs per group (Algorithm 1)
 
+// How the gathered operand of a convolution product is addressed.  A pixel index runs over
+// [image][PH][PW]; a tap-and-channel index is tap * C + channel with tap = r * S + s.  The element for
+// pixel (b, y, x) and (r, s, c) is src[((b * H + y + sign * r + off_h) * W + x + sign * s + off_w) * C + c],
+// zero when that row or column lies outside the tensor.
+struct ConvGather {
+    int mode;             // 0 plain matrices, 1 forward, 2 data gradient, 3 filter gradient
+    int H, W, C;          // the gathered tensor [n][H][W][C]
+    int PH, PW, pixels;   // the pixel space and its size n * PH * PW
+    int S, taps;          // filter taps per row, taps in all
+    int sign, off_h, off_w;
+    int filt_n, filt_k;   // data gradient: filters [filt_k = c_out][taps][filt_n = c_in]
+};
+
 struct FmacParams {
     const float* A;
     const float* B;
@@ -41,7 +64,77 @@ struct FmacParams {
     int transA, transB;
     int vec_store;  // C rows 16-byte aligned
     int vec_a, vec_b;  // operand base and leading dimension allow 128-bit loads
+    ConvGather cv;
 };
+
+// Table entries of the gather: a pixel as {offset of its image, y, x, inside the pixel space}, a
+// tap-and-channel index as {row offset, column offset, channel, inside the index range}.
+__device__ __forceinline__ int4 pixel_entry(const ConvGather& cv, int pix) {
+    const int x = pix % cv.PW, q = pix / cv.PW;
+    return make_int4((q / cv.PH) * cv.H * cv.W * cv.C, q % cv.PH, x, pix < cv.pixels ? 1 : 0);
+}
+__device__ __forceinline__ int4 tap_entry(const ConvGather& cv, int tc) {
+    const int c = tc % cv.C, tap = tc / cv.C;
+    return make_int4(cv.sign * (tap / cv.S) + cv.off_h, cv.sign * (tap % cv.S) + cv.off_w, c, tap < cv.taps ? 1 : 0);
+}
+__device__ __forceinline__ float gather_element(const ConvGather& cv, const float* src, const int4& px, const int4& tc) {
+    const int ih = px.y + tc.x, iw = px.z + tc.y;
+    if (!(px.w & tc.w) || (unsigned)ih >= (unsigned)cv.H || (unsigned)iw >= (unsigned)cv.W) return 0.0f;
+    return src[px.x + (ih * cv.W + iw) * cv.C + tc.z];
+}
+// Data gradient: offset of filter row k = tap * c_out + o, i.e. of W[o][tap][0], or -1 past the end.
+__device__ __forceinline__ int filter_row_entry(const ConvGather& cv, int k) {
+    const int o = k % cv.filt_k, tap = k / cv.filt_k;
+    return tap < cv.taps ? (o * cv.taps + tap) * cv.filt_n : -1;
+}
+// Tables of a convolution product in shared memory: 64 pixels or 32, 128 tap-and-channel indices or 32.
+struct ConvTables {
+    int4 pix[64];
+    int4 tap[128];
+    int filt[kFmBK];
+};
+// Per tile (slice = false) and per slice (slice = true): the entries that depend on the tile's rows /
+// columns, and those that depend on the slice's k range.  kCols is the tile's width.
+template <int kRows, int kCols>
+__device__ __forceinline__ void conv_tables(ConvTables& t, const ConvGather& cv, bool slice, int m0, int n0, int k0) {
+    const int i = threadIdx.x;
+    if (!slice) {
+        if (cv.mode != 3) { if (i < kRows) t.pix[i] = pixel_entry(cv, m0 + i); }
+        else if (i < kCols) t.tap[i] = tap_entry(cv, n0 + i);
+    } else if (i < kFmBK) {
+        if (cv.mode != 3) t.tap[i] = tap_entry(cv, k0 + i);
+        else t.pix[i] = pixel_entry(cv, k0 + i);
+        if (cv.mode == 2) t.filt[i] = filter_row_entry(cv, k0 + i);
+    }
+}
+// A convolution's slice of op(A) (kIsA) or op(B) as [k][row or column], converted by `convert`.
+template <int kRows, int kLd, bool kIsA, typename T, typename F>
+__device__ __forceinline__ void load_slice_conv(T (*dst)[kLd], const FmacParams& g, const ConvTables& t, int r0, int k0,
+                                                F convert) {
+    const ConvGather& cv = g.cv;
+    const bool gathered = kIsA ? cv.mode != 3 : cv.mode == 3;
+    for (int idx = threadIdx.x; idx < kRows * kFmBK; idx += kFmThreads) {
+        float v;
+        int r, k;
+        if (gathered && kIsA) {            // consecutive k are consecutive channels of a pixel
+            k = idx % kFmBK; r = idx / kFmBK;
+            v = gather_element(cv, g.A, t.pix[r], t.tap[k]);
+        } else if (gathered) {             // filter gradient: consecutive columns are consecutive channels
+            r = idx % kRows; k = idx / kRows;
+            v = gather_element(cv, g.B, t.pix[k], t.tap[r]);
+        } else if (kIsA) {                 // filter gradient: dY as [pixel][c_out], op(A)[i][k] = dY[k][i]
+            r = idx % kRows; k = idx / kRows;
+            v = (r0 + r < g.M && k0 + k < g.K) ? g.A[(long long)(k0 + k) * g.lda + (r0 + r)] : 0.0f;
+        } else if (cv.mode == 1) {         // forward: filters [c_out][taps * c_in], k contiguous
+            k = idx % kFmBK; r = idx / kFmBK;
+            v = (r0 + r < g.N && k0 + k < g.K) ? g.B[(long long)(r0 + r) * g.ldb + (k0 + k)] : 0.0f;
+        } else {                           // data gradient: filters [c_out][taps][c_in], row k = (tap, c_out)
+            r = idx % kRows; k = idx / kRows;
+            v = (t.filt[k] >= 0 && r0 + r < g.N) ? g.B[t.filt[k] + r0 + r] : 0.0f;
+        }
+        dst[k][r] = convert(v);
+    }
+}
 
 // a + x*y rounded to 24 bits with round-to-odd.  The two directed fused multiply-adds (exact
 // product, one rounding) are equal when the value is exact and adjacent fp32 numbers otherwise,
@@ -166,11 +259,12 @@ __device__ __forceinline__ void merge_block_hist(qfmt_stats_t* stats, const Quan
 constexpr int kFmBM = 64, kFmBN = 64, kFmTM = 4, kFmTN = 4;
 constexpr int kFmBlocksPerSm = 4;
 
-template <bool kStats, bool kFlush, int kWide>
+template <bool kStats, bool kFlush, int kWide, bool kConv>
 __global__ void __launch_bounds__(kFmThreads, kFmBlocksPerSm)
 fmac8_kernel(FmacParams g, QuantParams p, qfmt_stats_t* __restrict__ stats) {
     __shared__ __align__(16) float As[kFmBK][kFmBM + 4];
     __shared__ __align__(16) float Bs[kFmBK][kFmBN + 4];
+    __shared__ ConvTables tabs[1];  // used by the convolution instantiations only
     extern __shared__ uint32_t lane_hist[];  // [(top + kExtraBins)][32]
     const int nbins = p.top + kExtraBins;
     const int lane = threadIdx.x & 31;
@@ -196,10 +290,18 @@ fmac8_kernel(FmacParams g, QuantParams p, qfmt_stats_t* __restrict__ stats) {
         for (int i = 0; i < kFmTM; ++i)
 #pragma unroll
             for (int j = 0; j < kFmTN; ++j) master[i][j] = 0.0f, small[i][j] = 0.0f;
+        if (kConv) conv_tables<kFmBM, kFmBN>(tabs[0], g.cv, false, m0, n0, 0);  // read after the next barrier
         for (int k0 = 0; k0 < g.K; k0 += kFmBK) {
             __syncthreads();  // the previous slice is no longer read
-            load_slice<kFmBM, kFmBM + 4>(As, g.A, g.lda, !g.transA, m0, g.M, k0, g.K, same);
-            load_slice<kFmBN, kFmBN + 4>(Bs, g.B, g.ldb, g.transB, n0, g.N, k0, g.K, same);
+            if (kConv) {
+                conv_tables<kFmBM, kFmBN>(tabs[0], g.cv, true, m0, n0, k0);
+                __syncthreads();
+                load_slice_conv<kFmBM, kFmBM + 4, true>(As, g, tabs[0], m0, k0, same);
+                load_slice_conv<kFmBN, kFmBN + 4, false>(Bs, g, tabs[0], n0, k0, same);
+            } else {
+                load_slice<kFmBM, kFmBM + 4>(As, g.A, g.lda, !g.transA, m0, g.M, k0, g.K, same);
+                load_slice<kFmBN, kFmBN + 4>(Bs, g.B, g.ldb, g.transB, n0, g.N, k0, g.K, same);
+            }
             __syncthreads();
             const int kmax = g.K - k0 < kFmBK ? g.K - k0 : kFmBK;
 #pragma unroll 1
@@ -302,11 +404,12 @@ __device__ __forceinline__ void fetch_slice(float4 (&v)[kRows * kFmBK / (4 * kFm
     }
 }
 
-template <bool kStats, bool kFlush, bool kBf16>
+template <bool kStats, bool kFlush, bool kBf16, bool kConv>
 __global__ void __launch_bounds__(kFmThreads, kHfBlocksPerSm)
 fmac8_f16_kernel(FmacParams g, QuantParams p, qfmt_stats_t* __restrict__ stats) {
     __shared__ __align__(16) uint32_t As2[kFmBK][kHfBM + 4];  // each A value twice: {a, a} as f16x2
     __shared__ __align__(16) uint16_t Bs[kFmBK][kHfBN + 8];
+    __shared__ ConvTables tabs[1];  // used by the convolution instantiations only
     extern __shared__ uint32_t lane_hist[];
     const int nbins = p.top + kExtraBins;
     const int lane = threadIdx.x & 31;
@@ -330,13 +433,24 @@ fmac8_f16_kernel(FmacParams g, QuantParams p, qfmt_stats_t* __restrict__ stats) 
             for (int j = 0; j < kHfTN / 2; ++j) small[i][j] = zero2;
         }
         float4 fa[kPerA], fb[kPerB];  // the next slice, on its way from global memory while this one is used
-        fetch_slice<kHfBM>(fa, g.A, g.lda, !g.transA, g.vec_a, m0, g.M, 0, g.K);
-        fetch_slice<kHfBN>(fb, g.B, g.ldb, g.transB, g.vec_b, n0, g.N, 0, g.K);
+        if (kConv) {
+            conv_tables<kHfBM, kHfBN>(tabs[0], g.cv, false, m0, n0, 0);  // read after the next barrier
+        } else {
+            fetch_slice<kHfBM>(fa, g.A, g.lda, !g.transA, g.vec_a, m0, g.M, 0, g.K);
+            fetch_slice<kHfBN>(fb, g.B, g.ldb, g.transB, g.vec_b, n0, g.N, 0, g.K);
+        }
         for (int k0 = 0; k0 < g.K; k0 += kFmBK) {
             __syncthreads();  // the previous slice is no longer read
+            if (kConv) {  // gathered straight into the staged form
+                conv_tables<kHfBM, kHfBN>(tabs[0], g.cv, true, m0, n0, k0);
+                __syncthreads();
+                load_slice_conv<kHfBM, kHfBM + 4, true>(As2, g, tabs[0], m0, k0,
+                                                        [](float v) { const uint32_t h = to_16<kBf16>(v); return h | (h << 16); });
+                load_slice_conv<kHfBN, kHfBN + 8, false>(Bs, g, tabs[0], n0, k0, [](float v) { return (uint16_t)to_16<kBf16>(v); });
+            }
             // the conversions are exact: operands hold values of the 16-bit type
 #pragma unroll
-            for (int t = 0; t < kPerA; ++t) {
+            for (int t = 0; t < (kConv ? 0 : kPerA); ++t) {
                 int r, k;
                 group_position<kHfBM>(threadIdx.x + t * kFmThreads, !g.transA, r, k);
                 const uint32_t h0 = to_16<kBf16>(fa[t].x), h1 = to_16<kBf16>(fa[t].y), h2 = to_16<kBf16>(fa[t].z),
@@ -352,7 +466,7 @@ fmac8_f16_kernel(FmacParams g, QuantParams p, qfmt_stats_t* __restrict__ stats) 
                 }
             }
 #pragma unroll
-            for (int t = 0; t < kPerB; ++t) {
+            for (int t = 0; t < (kConv ? 0 : kPerB); ++t) {
                 int r, k;
                 group_position<kHfBN>(threadIdx.x + t * kFmThreads, g.transB, r, k);
                 const uint32_t h0 = to_16<kBf16>(fb[t].x), h1 = to_16<kBf16>(fb[t].y), h2 = to_16<kBf16>(fb[t].z),
@@ -367,7 +481,7 @@ fmac8_f16_kernel(FmacParams g, QuantParams p, qfmt_stats_t* __restrict__ stats) 
                 }
             }
             __syncthreads();
-            if (k0 + kFmBK < g.K) {
+            if (!kConv && k0 + kFmBK < g.K) {
                 fetch_slice<kHfBM>(fa, g.A, g.lda, !g.transA, g.vec_a, m0, g.M, k0 + kFmBK, g.K);
                 fetch_slice<kHfBN>(fb, g.B, g.ldb, g.transB, g.vec_b, n0, g.N, k0 + kFmBK, g.K);
             }
@@ -408,6 +522,64 @@ fmac8_f16_kernel(FmacParams g, QuantParams p, qfmt_stats_t* __restrict__ stats) 
 
 }  // namespace
 
+// Launches the kernel for a product described by g (plain matrices, or a convolution when g.cv.mode != 0).
+int launch_fmac8(const FmacParams& g, const QuantParams& p, const qfmt_format_t* fmt, qfmt_stats_t* d_stats,
+                 bool use_native, bool bf16, const DeviceInfo& dev, cudaStream_t stream) {
+    const bool conv = g.cv.mode != 0;
+    const bool has_stats = d_stats != nullptr;
+    const size_t smem = has_stats ? (size_t)(p.top + kExtraBins) * 32 * sizeof(uint32_t) : 0;
+    if (use_native) {
+        const long long tiles = (((long long)g.M + kHfBM - 1) / kHfBM) * (((long long)g.N + kHfBN - 1) / kHfBN);
+        const long long slots = (long long)dev.sm_count * kHfBlocksPerSm;
+        const unsigned grid = (unsigned)(tiles < slots ? tiles : slots);
+        const bool flush = fmt->denormals == 0;
+        const size_t sm = has_stats ? smem : 0;
+        // 256-bin histograms (bfloat16) put static + dynamic shared memory past the 48 KB that need no opt-in
+#define QFMT_HLAUNCH(S, F, B, C)                                                                            \
+    do {                                                                                                   \
+        if (sm > 16 * 1024)                                                                                \
+            QFMT_CUDA_TRY(cudaFuncSetAttribute(fmac8_f16_kernel<S, F, B, C>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm)); \
+        fmac8_f16_kernel<S, F, B, C><<<grid, kFmThreads, sm, stream>>>(g, p, d_stats);                      \
+    } while (0)
+#define QFMT_HTYPE(S, F)                                                                                   \
+    do {                                                                                                   \
+        if (bf16) { if (conv) QFMT_HLAUNCH(S, F, true, true); else QFMT_HLAUNCH(S, F, true, false); }      \
+        else { if (conv) QFMT_HLAUNCH(S, F, false, true); else QFMT_HLAUNCH(S, F, false, false); }         \
+    } while (0)
+        if (has_stats) { if (flush) QFMT_HTYPE(true, true); else QFMT_HTYPE(true, false); }
+        else { if (flush) QFMT_HTYPE(false, true); else QFMT_HTYPE(false, false); }
+#undef QFMT_HTYPE
+#undef QFMT_HLAUNCH
+    } else {
+        const long long tiles = (((long long)g.M + kFmBM - 1) / kFmBM) * (((long long)g.N + kFmBN - 1) / kFmBN);
+        const long long cap = (long long)dev.sm_count * kFmBlocksPerSm;
+        const unsigned grid = (unsigned)(tiles < cap ? tiles : cap);
+        const bool flush = fmt->denormals == 0;
+        const int wide = fmt->e == 8 ? 2 : (fmt->e == 7 ? 1 : 0);
+        const size_t sm = has_stats ? smem : 0;
+        // 256-bin histograms (e = 8) put static + dynamic shared memory past the 48 KB that need no opt-in
+#define QFMT_FLAUNCH(S, F, W)                                                                              \
+    do {                                                                                                   \
+        if (sm > 16 * 1024) {                                                                              \
+            QFMT_CUDA_TRY(cudaFuncSetAttribute(fmac8_kernel<S, F, W, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm)); \
+            QFMT_CUDA_TRY(cudaFuncSetAttribute(fmac8_kernel<S, F, W, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm)); \
+        }                                                                                                  \
+        if (conv) fmac8_kernel<S, F, W, true><<<grid, kFmThreads, sm, stream>>>(g, p, d_stats);             \
+        else fmac8_kernel<S, F, W, false><<<grid, kFmThreads, sm, stream>>>(g, p, d_stats);                 \
+    } while (0)
+#define QFMT_FWIDE(S, F)                                                                                   \
+    do {                                                                                                   \
+        if (wide == 2) QFMT_FLAUNCH(S, F, 2); else if (wide == 1) QFMT_FLAUNCH(S, F, 1); else QFMT_FLAUNCH(S, F, 0); \
+    } while (0)
+        if (has_stats) { if (flush) QFMT_FWIDE(true, true); else QFMT_FWIDE(true, false); }
+        else { if (flush) QFMT_FWIDE(false, true); else QFMT_FWIDE(false, false); }
+#undef QFMT_FWIDE
+#undef QFMT_FLAUNCH
+    }
+    QFMT_CUDA_TRY(cudaGetLastError());
+    return QFMT_OK;
+}
+
 int gemm_fmac8_device(const qfmt_matrix_t* A, const qfmt_matrix_t* B, float* d_C, int64_t ldc, const qfmt_format_t* fmt,
                       qfmt_stats_t* d_stats, int accumulate, int path, cudaStream_t stream) {
     int rc = validate_format(fmt);
@@ -446,55 +618,73 @@ int gemm_fmac8_device(const qfmt_matrix_t* A, const qfmt_matrix_t* B, float* d_C
     g.vec_store = (ldc % 4 == 0) && !(reinterpret_cast<uintptr_t>(d_C) & 15u);
     g.vec_a = (A->ld % 4 == 0) && !(reinterpret_cast<uintptr_t>(A->ptr) & 15u);
     g.vec_b = (B->ld % 4 == 0) && !(reinterpret_cast<uintptr_t>(B->ptr) & 15u);
-    const bool has_stats = d_stats != nullptr;
-    const size_t smem = has_stats ? (size_t)(p.top + kExtraBins) * 32 * sizeof(uint32_t) : 0;
-    const bool use_native = native && path != 1;
-    if (use_native) {
-        const long long tiles = ((M + kHfBM - 1) / kHfBM) * ((N + kHfBN - 1) / kHfBN);
-        const long long slots = (long long)dev.sm_count * kHfBlocksPerSm;
-        const unsigned grid = (unsigned)(tiles < slots ? tiles : slots);
-        const bool flush = fmt->denormals == 0;
-        const size_t sm = has_stats ? smem : 0;
-        // 256-bin histograms (bfloat16) put static + dynamic shared memory past the 48 KB that need no opt-in
-#define QFMT_HLAUNCH(S, F, B)                                                                               \
-    do {                                                                                                   \
-        if (sm > 24 * 1024)                                                                                \
-            QFMT_CUDA_TRY(cudaFuncSetAttribute(fmac8_f16_kernel<S, F, B>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm)); \
-        fmac8_f16_kernel<S, F, B><<<grid, kFmThreads, sm, stream>>>(g, p, d_stats);                         \
-    } while (0)
-#define QFMT_HTYPE(S, F)                                                                                   \
-    do {                                                                                                   \
-        if (bf16) QFMT_HLAUNCH(S, F, true); else QFMT_HLAUNCH(S, F, false);                                \
-    } while (0)
-        if (has_stats) { if (flush) QFMT_HTYPE(true, true); else QFMT_HTYPE(true, false); }
-        else { if (flush) QFMT_HTYPE(false, true); else QFMT_HTYPE(false, false); }
-#undef QFMT_HTYPE
-#undef QFMT_HLAUNCH
-    } else {
-        const long long tiles = ((M + kFmBM - 1) / kFmBM) * ((N + kFmBN - 1) / kFmBN);
-        const long long cap = (long long)dev.sm_count * kFmBlocksPerSm;
-        const unsigned grid = (unsigned)(tiles < cap ? tiles : cap);
-        const bool flush = fmt->denormals == 0;
-        const int wide = fmt->e == 8 ? 2 : (fmt->e == 7 ? 1 : 0);
-        const size_t sm = has_stats ? smem : 0;
-        // 256-bin histograms (e = 8) put static + dynamic shared memory past the 48 KB that need no opt-in
-#define QFMT_FLAUNCH(S, F, W)                                                                              \
-    do {                                                                                                   \
-        if (sm > 24 * 1024)                                                                                \
-            QFMT_CUDA_TRY(cudaFuncSetAttribute(fmac8_kernel<S, F, W>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm)); \
-        fmac8_kernel<S, F, W><<<grid, kFmThreads, sm, stream>>>(g, p, d_stats);                             \
-    } while (0)
-#define QFMT_FWIDE(S, F)                                                                                   \
-    do {                                                                                                   \
-        if (wide == 2) QFMT_FLAUNCH(S, F, 2); else if (wide == 1) QFMT_FLAUNCH(S, F, 1); else QFMT_FLAUNCH(S, F, 0); \
-    } while (0)
-        if (has_stats) { if (flush) QFMT_FWIDE(true, true); else QFMT_FWIDE(true, false); }
-        else { if (flush) QFMT_FWIDE(false, true); else QFMT_FWIDE(false, false); }
-#undef QFMT_FWIDE
-#undef QFMT_FLAUNCH
+    g.cv = ConvGather{};  // mode 0: plain matrices
+    return launch_fmac8(g, p, fmt, d_stats, native && path != 1, bf16, dev, stream);
+}
+
+// The three products of a convolution with FMAC-8 accumulation, on channels-last tensors (see the
+// head of this file for the order of the reduction).
+int conv_fmac8_device(int op, const qfmt_conv_t* geom, const float* d_p, const float* d_q, float* d_out,
+                      const qfmt_format_t* fmt, qfmt_stats_t* d_stats, int accumulate, int path, cudaStream_t stream) {
+    int rc = validate_format(fmt);
+    if (rc != QFMT_OK) return rc;
+    if (fmt->m > 10) return QFMT_ERR_BAD_FORMAT;
+    if (geom == nullptr || op < QFMT_CONV_FWD || op > QFMT_CONV_WGRAD) return QFMT_ERR_BAD_ARG;
+    if (accumulate != 0 && accumulate != 1) return QFMT_ERR_BAD_ARG;
+    if (path < 0 || path > 2) return QFMT_ERR_BAD_ARG;
+    const qfmt_conv_t& c = *geom;
+    if (c.n <= 0 || c.c_in <= 0 || c.h <= 0 || c.w <= 0 || c.c_out <= 0 || c.r <= 0 || c.s <= 0 || c.pad_h < 0 || c.pad_w < 0)
+        return QFMT_ERR_BAD_ARG;
+    const int64_t oh = (int64_t)c.h + 2 * c.pad_h - c.r + 1, ow = (int64_t)c.w + 2 * c.pad_w - c.s + 1;
+    if (oh <= 0 || ow <= 0) return QFMT_ERR_BAD_ARG;
+    const int64_t taps = (int64_t)c.r * c.s, in_px = (int64_t)c.n * c.h * c.w, out_px = (int64_t)c.n * oh * ow;
+    // every tensor, and every index the kernel forms, stays below 2^31
+    const int64_t lim = 0x7FFFFFFF;
+    if (in_px * c.c_in > lim || out_px * c.c_out > lim || taps * c.c_in * c.c_out > lim ||
+        (taps + 32) * ((int64_t)c.c_in + c.c_out) > lim || in_px + 64 > lim || out_px + 64 > lim)
+        return QFMT_ERR_BAD_ARG;
+    if (d_p == nullptr || d_q == nullptr || d_out == nullptr) return QFMT_ERR_BAD_ARG;
+    if ((reinterpret_cast<uintptr_t>(d_p) & 3u) || (reinterpret_cast<uintptr_t>(d_q) & 3u) ||
+        (reinterpret_cast<uintptr_t>(d_out) & 3u) || (reinterpret_cast<uintptr_t>(d_stats) & 7u))
+        return QFMT_ERR_BAD_ARG;
+    const bool bf16 = fmt->e == 8 && fmt->m == 7;
+    const bool native = (fmt->e == 5 && fmt->m == 10) || bf16;
+    if (path == 2 && !native) return QFMT_ERR_BAD_FORMAT;
+    DeviceInfo dev;
+    rc = current_device(&dev);
+    if (rc != QFMT_OK) return rc;
+    if (d_stats != nullptr && accumulate == 0) QFMT_CUDA_TRY(cudaMemsetAsync(d_stats, 0, sizeof(qfmt_stats_t), stream));
+
+    qfmt_format_t f = *fmt;
+    f.loss_scale = 1.0f;
+    const QuantParams p = make_params(f);
+    FmacParams g;
+    g.A = d_p; g.B = d_q; g.C = d_out;
+    g.transA = 0; g.transB = 0; g.vec_a = g.vec_b = 0;
+    ConvGather& cv = g.cv;
+    cv.S = c.s; cv.taps = (int)taps;
+    cv.filt_n = c.c_in; cv.filt_k = c.c_out;
+    if (op == QFMT_CONV_FWD) {          // Y[pixel][c_out] = sum over (tap, c_in) of X gathered . W[c_out][(tap, c_in)]
+        cv.mode = 1;
+        cv.H = c.h; cv.W = c.w; cv.C = c.c_in; cv.PH = (int)oh; cv.PW = (int)ow; cv.pixels = (int)out_px;
+        cv.sign = 1; cv.off_h = -c.pad_h; cv.off_w = -c.pad_w;
+        g.M = (int)out_px; g.N = c.c_out; g.K = (int)(taps * c.c_in);
+        g.lda = 0; g.ldb = g.K; g.ldc = c.c_out;
+    } else if (op == QFMT_CONV_DGRAD) { // dX[pixel][c_in] = sum over (tap, c_out) of dY gathered . W[c_out][tap][c_in]
+        cv.mode = 2;
+        cv.H = (int)oh; cv.W = (int)ow; cv.C = c.c_out; cv.PH = c.h; cv.PW = c.w; cv.pixels = (int)in_px;
+        cv.sign = -1; cv.off_h = c.pad_h; cv.off_w = c.pad_w;
+        g.M = (int)in_px; g.N = c.c_in; g.K = (int)(taps * c.c_out);
+        g.lda = 0; g.ldb = 0; g.ldc = c.c_in;
+    } else {                            // dW[c_out][(tap, c_in)] = sum over output pixels of dY[pixel][c_out] . X gathered
+        cv.mode = 3;
+        cv.H = c.h; cv.W = c.w; cv.C = c.c_in; cv.PH = (int)oh; cv.PW = (int)ow; cv.pixels = (int)out_px;
+        cv.sign = 1; cv.off_h = -c.pad_h; cv.off_w = -c.pad_w;
+        g.M = c.c_out; g.N = (int)(taps * c.c_in); g.K = (int)out_px;
+        g.lda = c.c_out; g.ldb = 0; g.ldc = g.N;
     }
-    QFMT_CUDA_TRY(cudaGetLastError());
-    return QFMT_OK;
+    g.vec_store = (g.ldc % 4 == 0) && !(reinterpret_cast<uintptr_t>(d_out) & 15u);
+    return launch_fmac8(g, p, fmt, d_stats, native && path != 1, bf16, dev, stream);
 }
 
 }  // namespace qfmt
@@ -502,4 +692,9 @@ int gemm_fmac8_device(const qfmt_matrix_t* A, const qfmt_matrix_t* B, float* d_C
 extern "C" int qfmt_gemm_fmac8(const qfmt_matrix_t* A, const qfmt_matrix_t* B, float* d_C, int64_t ldc,
                                const qfmt_format_t* fmt, qfmt_stats_t* d_stats, int accumulate, int path, void* stream) {
     return qfmt::gemm_fmac8_device(A, B, d_C, ldc, fmt, d_stats, accumulate, path, (cudaStream_t)stream);
+}
+
+extern "C" int qfmt_conv_fmac8(int32_t op, const qfmt_conv_t* geom, const float* d_p, const float* d_q, float* d_out,
+                               const qfmt_format_t* fmt, qfmt_stats_t* d_stats, int accumulate, int path, void* stream) {
+    return qfmt::conv_fmac8_device(op, geom, d_p, d_q, d_out, fmt, d_stats, accumulate, path, (cudaStream_t)stream);
 }
