@@ -705,6 +705,35 @@ def fmac8_section(torch, qf, dev, peaks, clock_mhz, reps=3):
                             "roofline": {"bound": "alu", "achieved": tf, "peak": peaks_t[kind], "unit": "TFMAC/s",
                                          "frac": tf / peaks_t[kind], "traffic": None,
                                          "peak_source": "derived: SMs x lanes x max SM clock / cycles per FMAC (see comment)"}}
+    # FMAC-8 in a convolution layer: the config4 3x3 layer (batch 128, 256 -> 256 channels at 14 x 14), forward
+    sh = workloads.CONV3X3
+    cfg4 = workloads.config4(sh)
+    g = qf.qfmt_conv_t(sh.n, sh.c_in, sh.h, sh.w, sh.c_out, sh.r, sh.s, sh.pad, sh.pad)
+    fmacs = float(sh.n * sh.h * sh.w) * sh.c_out * sh.c_in * sh.r * sh.s
+    out["conv"] = {"workload": "config4 3x3 layer forward (25088 x 256 x 2304 as a product), FMAC-8 accumulation, "
+                               "channels-last, statistics of the output", "runs": {}}
+    for tag, e, m, kind in (("1/6/9 general", 6, 9, "general"), ("1/5/10 binary16", 5, 10, "binary16")):
+        fmt = qf.make_format(e, m, 1)
+        tensors = []
+        for x in (cfg4["X"], cfg4["W"]):
+            b_, c_, hh, ww = x.shape
+            d_in = torch.from_numpy(x).to(dev)
+            d_cl = torch.empty(b_ * hh * ww * c_, dtype=torch.float32, device=dev)
+            qf.qfmt_quantize_stats_transpose(d_in, d_cl, b_, c_, hh * ww, fmt)
+            tensors.append(d_cl)
+        Y = torch.empty(sh.n * sh.h * sh.w * sh.c_out, dtype=torch.float32, device=dev)
+        st = torch.zeros(qf.STATS_WORDS, dtype=torch.int64, device=dev)
+
+        def conv_step():
+            qf.qfmt_conv_fmac8(qf.QFMT_CONV_FWD, g, tensors[0], tensors[1], Y, fmt, st, 0, 0)
+        conv_step()
+        ms = statistics.median(time_events(torch, conv_step, reps))
+        assert int(st.cpu()[256]) == Y.numel()
+        tf = fmacs / ms / 1e9
+        out["conv"]["runs"][tag] = {"ms": ms, "tfmac_per_s": tf,
+                                    "roofline": {"bound": "alu", "achieved": tf, "peak": peaks_t[kind], "unit": "TFMAC/s",
+                                                 "frac": tf / peaks_t[kind], "traffic": None,
+                                                 "peak_source": "derived: SMs x lanes x max SM clock / cycles per FMAC (see comment)"}}
     first = out["runs"]["1/6/9 general"]
     out.update({"value": first["tfmac_per_s"], "ms_per_step": first["ms"], "gpu_launches_per_step": 1,
                 "roofline": first["roofline"]})
@@ -882,7 +911,7 @@ def finish(args, world, value, total_ms, n, runs, clocks, e2e, roofline, cpu, ge
 # when the counters were taken: it is set to None as soon as that kernel's code changes, until re-taken.
 NCU_TRAFFIC_BYTES_PER_LAUNCH = 268463872 + 218315520
 # the same for the layer-output kernel on the 8192 x 4096 product
-NCU_EPILOGUE_TRAFFIC_BYTES_PER_LAUNCH = 134286336 + 86052352
+NCU_EPILOGUE_TRAFFIC_BYTES_PER_LAUNCH = 134290432 + 85915904
 
 
 def main():

@@ -247,8 +247,12 @@ typedef struct {
  * operands of any format with e <= 8 and m <= 10; fmt states that format (m > 10 is rejected
  * with QFMT_ERR_BAD_FORMAT).  Operands are NOT re-rounded; feeding values with more than 10
  * mantissa bits loses the extra bits.  The accumulation order is fixed, so results are
- * reproducible run to run; against an exact sum the error stays within
- * 2^-20 * sum_k |a_ik| |b_kj| for the workloads this library targets.
+ * reproducible run to run.  Against an exact sum the error of every element stays within
+ * 2^-20 * sum_k |a_ik| |b_kj| whenever at least one operand carries mixed signs (every
+ * workload the library is built for: signed weights or gradients meet the activations).
+ * When BOTH operands are non-negative and heavy-tailed, the tensor core's truncation of each
+ * 8-element partial sum goes one way and the error can exceed that bound, by less than a
+ * factor of 2 (the tests pin both statements); no mode of this call restores the bound there.
  * fp32 denormal operands (only 1/8/m formats have them) are handled as the tensor core
  * handles them.
  *

@@ -53,6 +53,8 @@ struct ConvGather {
     int S, taps;          // filter taps per row, taps in all
     int sign, off_h, off_w;
     int filt_n, filt_k;   // data gradient: filters [filt_k = c_out][taps][filt_n = c_in]
+    int vec4;             // both channel counts are multiples of four and the tensors 16-byte aligned:
+                          // four consecutive channels are one 128-bit load
 };
 
 struct FmacParams {
@@ -253,6 +255,43 @@ __device__ __forceinline__ void merge_block_hist(qfmt_stats_t* stats, const Quan
         atomicAdd((unsigned long long*)&stats->n_total, n_total);
 }
 
+// The same with 128-bit loads (ConvGather::vec4): a group is four consecutive channels, which are four
+// consecutive k of a pixel (forward / data gradient: gathered operand and forward filters), or four
+// consecutive rows or columns of a k (the other operands).  Channel counts that are multiples of four
+// keep a group inside one tap, inside the matrix, and 16-byte aligned.
+template <int kRows, int kLd, bool kIsA, typename T, typename F>
+__device__ __forceinline__ void load_slice_conv4(T (*dst)[kLd], const FmacParams& g, const ConvTables& t, int r0, int k0,
+                                                 F convert) {
+    const ConvGather& cv = g.cv;
+    const bool gathered = kIsA ? cv.mode != 3 : cv.mode == 3;
+    const bool along_k = kIsA ? cv.mode != 3 : cv.mode == 1;
+    const float* src = kIsA ? g.A : g.B;
+    for (int idx = threadIdx.x; idx < kRows * kFmBK / 4; idx += kFmThreads) {
+        int r, k;
+        if (along_k) { k = 4 * (idx % (kFmBK / 4)); r = idx / (kFmBK / 4); }
+        else { r = 4 * (idx % (kRows / 4)); k = idx / (kRows / 4); }
+        const float* ptr = nullptr;
+        if (gathered) {
+            const int4 px = kIsA ? t.pix[r] : t.pix[k], tc = kIsA ? t.tap[k] : t.tap[r];
+            const int ih = px.y + tc.x, iw = px.z + tc.y;
+            if ((px.w & tc.w) && (unsigned)ih < (unsigned)cv.H && (unsigned)iw < (unsigned)cv.W)
+                ptr = src + px.x + (ih * cv.W + iw) * cv.C + tc.z;
+        } else if (kIsA) {            // filter gradient: op(A)[i][k] = dY[k][i]
+            if (r0 + r < g.M && k0 + k < g.K) ptr = src + (long long)(k0 + k) * g.lda + (r0 + r);
+        } else if (cv.mode == 1) {    // forward: filters [c_out][taps * c_in]
+            if (r0 + r < g.N && k0 + k < g.K) ptr = src + (long long)(r0 + r) * g.ldb + (k0 + k);
+        } else {                      // data gradient: filters [c_out][taps][c_in]
+            if (t.filt[k] >= 0 && r0 + r < g.N) ptr = src + t.filt[k] + r0 + r;
+        }
+        const float4 v = ptr != nullptr ? *reinterpret_cast<const float4*>(ptr) : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+        if (along_k) {
+            dst[k][r] = convert(v.x); dst[k + 1][r] = convert(v.y); dst[k + 2][r] = convert(v.z); dst[k + 3][r] = convert(v.w);
+        } else {
+            dst[k][r] = convert(v.x); dst[k][r + 1] = convert(v.y); dst[k][r + 2] = convert(v.z); dst[k][r + 3] = convert(v.w);
+        }
+    }
+}
+
 // ---- any format with m <= 10 ----------------------------------------------------------------
 // 4 x 4 outputs per thread: the FMAC chain of one output is a dozen dependent instructions, so
 // many resident warps (four blocks per SM) hide more latency than a larger patch per thread would.
@@ -296,8 +335,13 @@ fmac8_kernel(FmacParams g, QuantParams p, qfmt_stats_t* __restrict__ stats) {
             if (kConv) {
                 conv_tables<kFmBM, kFmBN>(tabs[0], g.cv, true, m0, n0, k0);
                 __syncthreads();
-                load_slice_conv<kFmBM, kFmBM + 4, true>(As, g, tabs[0], m0, k0, same);
-                load_slice_conv<kFmBN, kFmBN + 4, false>(Bs, g, tabs[0], n0, k0, same);
+                if (g.cv.vec4) {
+                    load_slice_conv4<kFmBM, kFmBM + 4, true>(As, g, tabs[0], m0, k0, same);
+                    load_slice_conv4<kFmBN, kFmBN + 4, false>(Bs, g, tabs[0], n0, k0, same);
+                } else {
+                    load_slice_conv<kFmBM, kFmBM + 4, true>(As, g, tabs[0], m0, k0, same);
+                    load_slice_conv<kFmBN, kFmBN + 4, false>(Bs, g, tabs[0], n0, k0, same);
+                }
             } else {
                 load_slice<kFmBM, kFmBM + 4>(As, g.A, g.lda, !g.transA, m0, g.M, k0, g.K, same);
                 load_slice<kFmBN, kFmBN + 4>(Bs, g.B, g.ldb, g.transB, n0, g.N, k0, g.K, same);
@@ -444,9 +488,15 @@ fmac8_f16_kernel(FmacParams g, QuantParams p, qfmt_stats_t* __restrict__ stats) 
             if (kConv) {  // gathered straight into the staged form
                 conv_tables<kHfBM, kHfBN>(tabs[0], g.cv, true, m0, n0, k0);
                 __syncthreads();
-                load_slice_conv<kHfBM, kHfBM + 4, true>(As2, g, tabs[0], m0, k0,
-                                                        [](float v) { const uint32_t h = to_16<kBf16>(v); return h | (h << 16); });
-                load_slice_conv<kHfBN, kHfBN + 8, false>(Bs, g, tabs[0], n0, k0, [](float v) { return (uint16_t)to_16<kBf16>(v); });
+                auto twice = [](float v) { const uint32_t h = to_16<kBf16>(v); return h | (h << 16); };
+                auto once = [](float v) { return (uint16_t)to_16<kBf16>(v); };
+                if (g.cv.vec4) {
+                    load_slice_conv4<kHfBM, kHfBM + 4, true>(As2, g, tabs[0], m0, k0, twice);
+                    load_slice_conv4<kHfBN, kHfBN + 8, false>(Bs, g, tabs[0], n0, k0, once);
+                } else {
+                    load_slice_conv<kHfBM, kHfBM + 4, true>(As2, g, tabs[0], m0, k0, twice);
+                    load_slice_conv<kHfBN, kHfBN + 8, false>(Bs, g, tabs[0], n0, k0, once);
+                }
             }
             // the conversions are exact: operands hold values of the 16-bit type
 #pragma unroll
@@ -684,6 +734,8 @@ int conv_fmac8_device(int op, const qfmt_conv_t* geom, const float* d_p, const f
         g.lda = c.c_out; g.ldb = 0; g.ldc = g.N;
     }
     g.vec_store = (g.ldc % 4 == 0) && !(reinterpret_cast<uintptr_t>(d_out) & 15u);
+    cv.vec4 = (c.c_in % 4 == 0 && c.c_out % 4 == 0 &&
+               !((reinterpret_cast<uintptr_t>(d_p) | reinterpret_cast<uintptr_t>(d_q)) & 15u)) ? 1 : 0;
     return launch_fmac8(g, p, fmt, d_stats, native && path != 1, bf16, dev, stream);
 }
 
