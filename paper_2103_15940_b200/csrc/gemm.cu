@@ -871,7 +871,10 @@ __device__ __forceinline__ uint32_t make_idesc_pair(int a_mn, int b_mn, int kind
 // CTA of the pair owns one M-tile of whole image rows (p.rows_per_blk rows, p.conv_rows pixels) and
 // half of the 256 filter columns; its pixel operand arrives as one box per image touched from
 // row_maps, C is written through tmap_c ({32, conv_rows, N / 32, complete tiles}: rows past the tile
-// are clipped) or, for the incomplete last tile, tmap_c2.
+// are clipped) or, for the incomplete last tile, tmap_c2.  kMode 2: filter gradient of a convolution with
+// padded stages (GemmParams::wg_padded): a dense product of two MN-major operands whose stages are
+// gathered pixel rows, C_out is M (128 rows per CTA), (tap, C_in) is N (128 columns per CTA, inside one
+// tap), one rank-5 copy per operand and stage.
 // kSk: the balanced schedule (GemmParams::sk_flags) is compiled in; products that do not use it run an
 // instantiation without any of its code.
 template <bool kEpi, int kKind, int kMode, bool kSk>
@@ -1051,6 +1054,18 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmap_a, const CUten
                         continue;
                     }
                     ptx::mbar_expect_tx_cluster(bar, kPStageBytes);
+                    if (kMode == 2) {
+                        // stage kb = rows_per_blk output rows of one image, each padded to a power-of-two number of
+                        // K rows; A = output gradient, B = activations at the tap this CTA's columns belong to
+                        const int q = kb * p.rows_per_blk;
+                        const int oh = q % p.img_rows, img = q / p.img_rows;
+                        const int tap = n0 / p.ck, ci = n0 % p.ck;
+                        ptx::tma_load_5d_pair(sa, &tmap_a, bar, 0, 0, oh, img, m0 >> 5);
+                        ptx::tma_load_5d_pair(sb, &tmap_b, bar, 0, tap % p.taps_s + p.off_w, oh + tap / p.taps_s + p.off_h, img,
+                                              ci >> 5);
+                        if (++stage == kPStages) { stage = 0; phase ^= 1u; }
+                        continue;
+                    }
                     // an MN-major operand arrives as column blocks of one 128-byte row per K element:
                     // 32 columns x 32 K rows (TF32) or 64 columns x 64 K rows (16-bit codes)
                     constexpr int kBlkShift = kKind == kKindTf32 ? 5 : 6, kBlk = 1 << kBlkShift;
@@ -1386,6 +1401,13 @@ gemm_tf32_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_c
 
 // Forward / data gradient of a convolution on CTA pairs (its own instantiation, so that the dense
 // products carry none of its code).
+// Filter gradient of a convolution on CTA pairs (padded stages; its own instantiation).
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+gemm_wgrad_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+                       const __grid_constant__ CUtensorMap tmap_c, const GemmParams p) {
+    pair_body<false, kKindTf32, 2, false>(tmap_a, tmap_b, tmap_c, nullptr, nullptr, p);
+}
+
 template <bool kSk>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 gemm_conv_pair_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_constant__ CUtensorMap tmap_c,
@@ -1748,6 +1770,21 @@ int launch_conv_pair(const CUtensorMap& mb, const CUtensorMap& mc, const CUtenso
     return QFMT_OK;
 }
 
+int launch_wgrad_pair(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc, const GemmParams& p,
+                      const DeviceInfo& dev, cudaStream_t stream) {
+    static bool attr_set[64] = {};
+    if (dev.ordinal < 0 || dev.ordinal >= 64 || !attr_set[dev.ordinal]) {
+        QFMT_CUDA_TRY(cudaFuncSetAttribute(gemm_wgrad_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           (int)kPairSmemBytes));
+        if (dev.ordinal >= 0 && dev.ordinal < 64) attr_set[dev.ordinal] = true;
+    }
+    const long long work = (long long)p.tiles_m * p.tiles_n * p.splits;
+    const long long clusters = work < dev.sm_count / 2 ? work : dev.sm_count / 2;
+    gemm_wgrad_pair_kernel<<<(unsigned)(2 * clusters), kThreads, kPairSmemBytes, stream>>>(ma, mb, mc, p);
+    QFMT_CUDA_TRY(cudaGetLastError());
+    return QFMT_OK;
+}
+
 // Layer-output epilogue request for gemm_device: the rounded, zero-padded bias and the record.
 struct EpiArgs {
     const float* rbias;
@@ -2013,6 +2050,7 @@ struct ConvPlan {
     int64_t oh, ow;
     bool pair;       // forward / data gradient on CTA pairs (two M-tiles of whole image rows per pair)
     bool pair_sk;    // ... under the balanced schedule of the pair kernel
+    bool pair_wgrad; // filter gradient on CTA pairs (padded stages, C_out of at least 256)
     int splits;
     int sk_cpt;      // forward / data gradient: chunks per tile when the balanced schedule is used, else 0
     int sk_pieces;
@@ -2043,6 +2081,7 @@ int plan_conv(int op, const qfmt_conv_t* g, ConvPlan* plan) {
     plan->splits = 1;
     plan->pair = false;
     plan->pair_sk = false;
+    plan->pair_wgrad = false;
     plan->sk_cpt = 0;
     plan->sk_pieces = 1;
     plan->workspace = kWorkspaceHeader;
@@ -2095,10 +2134,15 @@ int plan_conv(int op, const qfmt_conv_t* g, ConvPlan* plan) {
     }
     if (op == QFMT_CONV_WGRAD) {
         if (plan->ow > kBK) return QFMT_ERR_BAD_ARG;                      // a stage is made of whole output rows
-        const int rows_per_blk = wgrad_rows_per_stage(plan->oh, plan->ow, g->c_in, nullptr);
+        int padded_row = 0;
+        const int rows_per_blk = wgrad_rows_per_stage(plan->oh, plan->ow, g->c_in, &padded_row);
         const int64_t kb_total = ((int64_t)g->n * plan->oh + rows_per_blk - 1) / rows_per_blk;
-        const int64_t tiles = (((int64_t)g->c_out + kBM - 1) / kBM) * (((int64_t)g->r * g->s * g->c_in + kBN - 1) / kBN);
-        int64_t splits = kPlanSms / tiles;
+        // CTA pairs (each CTA 128 rows of C_out and 128 columns of a tap) when the stages are padded, so that
+        // one copy per operand fills a stage, and C_out fills a pair's 256 rows
+        plan->pair_wgrad = padded_row > 0 && g->c_out >= 2 * kBM && g_conv_pair_policy.load() != 1;
+        const int64_t tile_rows = plan->pair_wgrad ? 2 * kBM : kBM, units = plan->pair_wgrad ? kPlanPairs : kPlanSms;
+        const int64_t tiles = (((int64_t)g->c_out + tile_rows - 1) / tile_rows) * (((int64_t)g->r * g->s * g->c_in + kBN - 1) / kBN);
+        int64_t splits = units / tiles;
         if (splits > kMaxSplits) splits = kMaxSplits;
         if (splits > kb_total / 8) splits = kb_total / 8;   // at least eight stages per split
         if (splits < 1) splits = 1;
@@ -2292,7 +2336,9 @@ int conv_device(int op, const qfmt_conv_t* g, const float* d_p, const float* d_q
     p.ck = (int)CI;
     p.off_h = -g->pad_h;
     p.off_w = -g->pad_w;
-    p.tiles_m = (int)((CO + kBM - 1) / kBM);
+    const bool pair_wgrad = plan.pair_wgrad && p.wg_padded;
+    p.tile_rows = pair_wgrad ? 2 * kBM : kBM;
+    p.tiles_m = (int)((CO + p.tile_rows - 1) / p.tile_rows);
     p.tiles_n = (p.N + kBN - 1) / kBN;
     p.kb_total = (p.total_q + p.rows_per_blk - 1) / p.rows_per_blk;
     p.splits = plan.splits;
@@ -2314,7 +2360,7 @@ int conv_device(int op, const qfmt_conv_t* g, const float* d_p, const float* d_q
         rc = make_map(&ma, d_p, 5, da, sa_, ba, true);
         if (rc != QFMT_OK) return rc;
         const uint64_t db[5] = {32, W, H, N, CI / 32}, sb_[4] = {CI, W * CI, H * W * CI, 32};
-        const uint32_t bb[5] = {32, wpad, (uint32_t)p.rows_per_blk, 1, kBN / 32};
+        const uint32_t bb[5] = {32, wpad, (uint32_t)p.rows_per_blk, 1, (uint32_t)((pair_wgrad ? kBN / 2 : kBN) / 32)};
         rc = make_map(&mb, d_q, 5, db, sb_, bb, true);
         if (rc != QFMT_OK) return rc;
     } else {
@@ -2331,11 +2377,18 @@ int conv_device(int op, const qfmt_conv_t* g, const float* d_p, const float* d_q
         if (rc != QFMT_OK) return rc;
     }
     }
-    rc = make_map_c(&mc, p.C, (uint64_t)p.N, (uint64_t)p.M, (uint64_t)p.splits, (uint64_t)p.N, (uint64_t)p.M * p.N);
-    if (rc != QFMT_OK) return rc;
-    RowMaps rows;
-    for (int i = 0; i < kMaxRowMaps; ++i) rows.m[i] = ma;  // unused by the filter gradient
-    rc = launch_gemm(ma, mb, mc, mc, rows, p, dev, stream);
+    if (pair_wgrad) {
+        p.c_blocked = 1;  // N = taps * C_in is a multiple of 32
+        rc = make_map_c_blocked(&mc, p.C, (uint64_t)p.N, (uint64_t)p.M, (uint64_t)p.splits, (uint64_t)p.N, (uint64_t)p.M * p.N);
+        if (rc != QFMT_OK) return rc;
+        rc = launch_wgrad_pair(ma, mb, mc, p, dev, stream);
+    } else {
+        rc = make_map_c(&mc, p.C, (uint64_t)p.N, (uint64_t)p.M, (uint64_t)p.splits, (uint64_t)p.N, (uint64_t)p.M * p.N);
+        if (rc != QFMT_OK) return rc;
+        RowMaps rows;
+        for (int i = 0; i < kMaxRowMaps; ++i) rows.m[i] = ma;  // unused by the filter gradient
+        rc = launch_gemm(ma, mb, mc, mc, rows, p, dev, stream);
+    }
     if (rc != QFMT_OK) return rc;
     if (p.splits > 1) {
         launch_splitk_reduce(partials, d_out, p.M, p.N, p.N, p.splits, dev.sm_count, stream);

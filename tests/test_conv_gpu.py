@@ -82,6 +82,8 @@ SMALL = [
     (2, 256, 10, 9, 32, 3, 3, 0, 0),      # the same without zero padding: the pad rows of B hold real pixels
     (2, 512, 4, 14, 32, 1, 1, 0, 0),      # padded stages, two 256-column tiles per tap
     (64, 32, 3, 3, 64, 3, 3, 1, 1),       # 42 three-pixel rows per M-tile: fourteen images (copies) per tile and stage
+    (2, 256, 4, 7, 256, 3, 3, 1, 1),      # filter gradient on CTA pairs: padded stages and 256 output channels
+    (1, 256, 8, 8, 320, 3, 3, 1, 1),      # the same with a second, incomplete row of pair tiles (320 output channels)
 ]
 
 
