@@ -415,7 +415,8 @@ int qfmt_conv_tile_policy(int policy);
  *   op = QFMT_CONV_DGRAD  d_p = dY, d_q = W   d_out = dX  dX[n,h,w,ci] = sum dY[n,h-r+pad_h,w-s+pad_w,co] W[co,r,s,ci]
  *   op = QFMT_CONV_WGRAD  d_p = dY, d_q = X   d_out = dW  dW[co,r,s,ci] = sum dY[n,oh,ow,co] X[n,oh+r-pad_h,ow+s-pad_w,ci]
  * Limits: c_in and c_out multiples of 32; output row length (ow; w for the data gradient) at
- * most 128, and at most 32 for the filter gradient; every tensor below 2^30 elements per
+ * most 128 for the forward pass and the data gradient (none for the filter gradient, which takes
+ * rows longer than 32 pixels in 32-pixel pieces); every tensor below 2^30 elements per
  * dimension product used as a GEMM extent.  Violations return QFMT_ERR_BAD_ARG.
  *   d_workspace  device, 16-byte aligned, >= qfmt_conv_workspace_bytes(op, geom) bytes: status
  *                area, and for the filter gradient the split-K partial sums (the long pixel

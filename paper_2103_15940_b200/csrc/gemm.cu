@@ -114,6 +114,7 @@ struct GemmParams {
                      // (the copy engine zero-fills the columns past the image), a stage is 32 K rows
                      // exactly, and one rank-5 copy per operand brings all of its channel blocks
     int rows_box;    // filter gradient: image rows fetched by one copy (rows_per_blk when it divides the image height, else 1)
+    int wg_segs;     // filter gradient: K stages per output row (1; more when a row is longer than a stage's 32 pixels)
     int a_blocked, b_blocked;  // dense MN-major operand whose extent is a multiple of 32: its map is
                                // rank 3, {32, K, extent / 32}, and one copy fetches a stage's 32-wide blocks
     // ---- work decomposition
@@ -569,18 +570,21 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                         // Filter gradient: K = pixels.  A = output gradient (C_out is M), B = activations
                         // read at the tap that the N column block belongs to (C_in within a tap is N).
                         const int per_row = kBM / 32 + kBN / 32;
+                        // A row longer than 32 pixels takes wg_segs stages of 32 pixels each (one image row per
+                        // stage then); the last one reaches past the row's end, where the copy of A fills zeros.
+                        const int x0 = (kb % p.wg_segs) * kBK, q0 = (kb / p.wg_segs) * p.rows_per_blk;
                         for (int i = lane; i < (p.rows_per_blk / p.rows_box) * per_row; i += 32) {
                             const int j = (i / per_row) * p.rows_box, c = i % per_row;
-                            const int q = kb * p.rows_per_blk + j;
+                            const int q = q0 + j;
                             const int oh = q % p.img_rows, img = q / p.img_rows;
                             const uint32_t row_off = (uint32_t)(j * p.img_w) * 128u;
                             if (c < kBM / 32) {
-                                ptx::tma_load_4d(sa + c * 4096u + row_off, &tmap_a, bar, m0 + c * 32, 0, oh, img);
+                                ptx::tma_load_4d(sa + c * 4096u + row_off, &tmap_a, bar, m0 + c * 32, x0, oh, img);
                             } else {
                                 const int col = n0 + (c - kBM / 32) * 32;
                                 const int tap = col / p.ck, ci = col % p.ck;
                                 ptx::tma_load_4d(sb + (c - kBM / 32) * 4096u + row_off, &tmap_b, bar, ci,
-                                                 tap % p.taps_s + p.off_w, oh + tap / p.taps_s + p.off_h, img);
+                                                 x0 + tap % p.taps_s + p.off_w, oh + tap / p.taps_s + p.off_h, img);
                             }
                         }
                     }
@@ -1639,6 +1643,7 @@ void dense_defaults(GemmParams* p) {
     p->a_blocked = p->b_blocked = 0;
     p->c_blocked = 0;
     p->rows_box = 1;
+    p->wg_segs = 1;
     p->wg_padded = 0;
     p->sk_cpt = 0;
     p->sk_pieces = 1;
@@ -2063,8 +2068,11 @@ int wgrad_rows_per_stage(int64_t oh, int64_t ow, int64_t c_in, int* padded_row) 
     while (wpad < ow) wpad *= 2;
     const bool padded = wpad <= kBK && oh % (kBK / wpad) == 0 && c_in % kBN == 0;
     if (padded_row != nullptr) *padded_row = padded ? wpad : 0;
+    if (ow > kBK) return 1;
     return padded ? kBK / wpad : kBK / (int)ow;
 }
+// K stages per output row of the filter gradient: rows longer than a stage's 32 pixels are cut into 32-pixel pieces.
+int wgrad_row_segments(int64_t ow) { return ow > kBK ? (int)((ow + kBK - 1) / kBK) : 1; }
 constexpr int kPlanSms = 148;  // B200; the split factor is planned for it so that it does not vary
 int plan_conv(int op, const qfmt_conv_t* g, ConvPlan* plan) {
     if (g == nullptr || op < QFMT_CONV_FWD || op > QFMT_CONV_WGRAD) return QFMT_ERR_BAD_ARG;
@@ -2133,10 +2141,9 @@ int plan_conv(int op, const qfmt_conv_t* g, ConvPlan* plan) {
         }
     }
     if (op == QFMT_CONV_WGRAD) {
-        if (plan->ow > kBK) return QFMT_ERR_BAD_ARG;                      // a stage is made of whole output rows
         int padded_row = 0;
         const int rows_per_blk = wgrad_rows_per_stage(plan->oh, plan->ow, g->c_in, &padded_row);
-        const int64_t kb_total = ((int64_t)g->n * plan->oh + rows_per_blk - 1) / rows_per_blk;
+        const int64_t kb_total = (((int64_t)g->n * plan->oh + rows_per_blk - 1) / rows_per_blk) * wgrad_row_segments(plan->ow);
         // CTA pairs (each CTA 128 rows of C_out and 128 columns of a tap) when the stages are padded, so that
         // one copy per operand fills a stage, and C_out fills a pair's 256 rows
         plan->pair_wgrad = padded_row > 0 && g->c_out >= 2 * kBM && g_conv_pair_policy.load() != 1;
@@ -2340,13 +2347,16 @@ int conv_device(int op, const qfmt_conv_t* g, const float* d_p, const float* d_q
     p.tile_rows = pair_wgrad ? 2 * kBM : kBM;
     p.tiles_m = (int)((CO + p.tile_rows - 1) / p.tile_rows);
     p.tiles_n = (p.N + kBN - 1) / kBN;
-    p.kb_total = (p.total_q + p.rows_per_blk - 1) / p.rows_per_blk;
+    p.wg_segs = wgrad_row_segments((int64_t)OW);
+    p.kb_total = ((p.total_q + p.rows_per_blk - 1) / p.rows_per_blk) * p.wg_segs;
     p.splits = plan.splits;
     p.kb_per_split = (p.kb_total + p.splits - 1) / p.splits;
     p.a_mn_major = 1;
     p.b_mn_major = 1;
-    p.a_bytes = p.wg_padded ? kABytes : (uint32_t)((kBM / 32) * p.rows_per_blk * (int)OW * 128);
-    p.b_bytes = p.wg_padded ? kBBytes : (uint32_t)((kBN / 32) * p.rows_per_blk * (int)OW * 128);
+    // pixels a copy brings per image row: the whole row, or a 32-pixel piece of a longer one (zero-filled past its end)
+    const uint32_t box_w = p.wg_segs > 1 ? (uint32_t)kBK : (uint32_t)OW;
+    p.a_bytes = p.wg_padded ? kABytes : (uint32_t)(kBM / 32) * (uint32_t)p.rows_per_blk * box_w * 128u;
+    p.b_bytes = p.wg_padded ? kBBytes : (uint32_t)(kBN / 32) * (uint32_t)p.rows_per_blk * box_w * 128u;
     float* partials = reinterpret_cast<float*>(reinterpret_cast<char*>(d_workspace) + kWorkspaceHeader);
     p.ldc = (long long)p.N;
     p.C = p.splits > 1 ? partials : d_out;
@@ -2366,13 +2376,13 @@ int conv_device(int op, const qfmt_conv_t* g, const float* d_p, const float* d_q
     } else {
     {
         const uint64_t dims[4] = {CO, OW, OH, N}, st[3] = {CO, OW * CO, OH * OW * CO};
-        const uint32_t box[4] = {32, (uint32_t)OW, (uint32_t)p.rows_box, 1};
+        const uint32_t box[4] = {32, box_w, (uint32_t)p.rows_box, 1};
         rc = make_map(&ma, d_p, 4, dims, st, box, true);
         if (rc != QFMT_OK) return rc;
     }
     {
         const uint64_t dims[4] = {CI, W, H, N}, st[3] = {CI, W * CI, H * W * CI};
-        const uint32_t box[4] = {32, (uint32_t)OW, (uint32_t)p.rows_box, 1};
+        const uint32_t box[4] = {32, box_w, (uint32_t)p.rows_box, 1};
         rc = make_map(&mb, d_q, 4, dims, st, box, true);
         if (rc != QFMT_OK) return rc;
     }

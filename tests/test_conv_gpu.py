@@ -84,6 +84,9 @@ SMALL = [
     (64, 32, 3, 3, 64, 3, 3, 1, 1),       # 42 three-pixel rows per M-tile: fourteen images (copies) per tile and stage
     (2, 256, 4, 7, 256, 3, 3, 1, 1),      # filter gradient on CTA pairs: padded stages and 256 output channels
     (1, 256, 8, 8, 320, 3, 3, 1, 1),      # the same with a second, incomplete row of pair tiles (320 output channels)
+    (1, 64, 5, 40, 32, 3, 3, 1, 1),       # 40-pixel rows: two filter-gradient stages per row, the second 8 pixels and zeros
+    (2, 64, 6, 56, 64, 3, 3, 1, 1),       # 56-pixel rows (the first stage of a ResNet-50-shaped network), split K
+    (1, 32, 3, 70, 32, 1, 3, 0, 0),       # 68-pixel output rows without padding: three stages per row, the last 4 pixels
 ]
 
 
@@ -170,7 +173,7 @@ def test_unsupported_geometries_are_refused():
     fmt = qf.make_format(6, 9)
     for geom, op in (((1, 30, 8, 8, 32, 3, 3, 1, 1), qf.QFMT_CONV_FWD),     # channels not a multiple of 32
                      ((1, 32, 8, 200, 32, 3, 3, 1, 1), qf.QFMT_CONV_FWD),    # rows longer than an M-tile
-                     ((1, 32, 8, 40, 32, 3, 3, 1, 1), qf.QFMT_CONV_WGRAD),   # rows longer than a stage
+                     ((1, 32, 8, 200, 32, 3, 3, 1, 1), qf.QFMT_CONV_DGRAD),  # the same for the data gradient
                      ((1, 32, 2, 2, 32, 5, 5, 0, 0), qf.QFMT_CONV_FWD)):     # empty output
         g = qf.qfmt_conv_t(*geom)
         assert qf.qfmt_conv_workspace_bytes(op, g) == 0
