@@ -399,7 +399,6 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                  const __grid_constant__ CUtensorMap tmap_c, const __grid_constant__ CUtensorMap tmap_p,
                  const __grid_constant__ RowMaps row_maps, const GemmParams p) {
     extern __shared__ uint8_t smem_raw[];
-    announce_launch(p.status, p.launch_tag);
     const uint32_t raw = ptx::smem_addr(smem_raw);
     const uint32_t tiles = (raw + 1023u) & ~1023u;  // swizzled tiles need 1024-byte alignment
     const uint32_t out_stage = tiles + kStages * kStageBytes;
@@ -452,9 +451,14 @@ gemm_tf32_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
         ptx::tmem_alloc(ptx::smem_addr(const_cast<uint32_t*>(tmem_slot)), kTmemCols);
         ptx::tmem_relinquish();
     }
+    // Everything above touched shared and tensor memory only and may run while the kernel before this one
+    // in the stream drains; from here on global memory is read and written.
+    grid_dependency_wait();
+    announce_launch(p.status, p.launch_tag);
     ptx::tc_fence_before_sync();
     __syncthreads();
     ptx::tc_fence_after_sync();
+    grid_launch_dependents();
     const uint32_t tmem_base = *tmem_slot;
 
     const int num_work = p.sk_cpt > 0 ? p.sk_pieces * (int)gridDim.x : p.tiles_m * p.tiles_n * p.splits;
@@ -885,7 +889,6 @@ template <bool kEpi, int kKind, int kMode, bool kSk>
 __device__ __forceinline__ void pair_body(const CUtensorMap& tmap_a, const CUtensorMap& tmap_b, const CUtensorMap& tmap_c,
                                           const CUtensorMap* tmap_c2, const CUtensorMap* row_maps, const GemmParams& p) {
     extern __shared__ uint8_t smem_raw[];
-    announce_launch(p.status, p.launch_tag);
     const uint32_t raw = ptx::smem_addr(smem_raw);
     const uint32_t tiles = (raw + 1023u) & ~1023u;
     const uint32_t out_stage = tiles + kPStages * kPStageBytes;
@@ -940,10 +943,15 @@ __device__ __forceinline__ void pair_body(const CUtensorMap& tmap_a, const CUten
         ptx::tmem_alloc_pair(ptx::smem_addr(const_cast<uint32_t*>(tmem_slot)), kTmemCols);
         ptx::tmem_relinquish_pair();
     }
+    // Everything above touched shared and tensor memory only and may run while the kernel before this one
+    // in the stream drains; from here on global memory is read and written.
+    grid_dependency_wait();
+    announce_launch(p.status, p.launch_tag);
     ptx::tc_fence_before_sync();
     __syncthreads();
     ptx::cluster_sync();  // the peer's barriers exist before anything is signalled to them
     ptx::tc_fence_after_sync();
+    grid_launch_dependents();
     const uint32_t tmem_base = *tmem_slot;
     // work items of this pair: its pieces under the balanced schedule (t = 0, 1, ...), else every
     // num_clusters-th tile (t = cluster_id, cluster_id + num_clusters, ...)
@@ -1532,6 +1540,8 @@ template <typename T, int kMax>
 __global__ void __launch_bounds__(256)
 splitk_reduce_kernel(const T* __restrict__ part, T* __restrict__ C, long long rows, long long cols,
                      long long ldc, int splits) {
+    grid_dependency_wait();   // the partial sums come from the kernel before this one
+    grid_launch_dependents();
     const long long total = rows * cols;
     for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total;
          i += (long long)gridDim.x * blockDim.x) {
@@ -1556,11 +1566,11 @@ void launch_splitk_reduce_as(const float* part, float* C, long long rows, long l
     const int blocks = (int)(want < cap ? want : cap);
     const T* p = reinterpret_cast<const T*>(part);
     T* c = reinterpret_cast<T*>(C);
-    if (splits <= 2) splitk_reduce_kernel<T, 2><<<blocks, 256, 0, stream>>>(p, c, rows, cols, ldc, splits);
-    else if (splits <= 4) splitk_reduce_kernel<T, 4><<<blocks, 256, 0, stream>>>(p, c, rows, cols, ldc, splits);
-    else if (splits <= 8) splitk_reduce_kernel<T, 8><<<blocks, 256, 0, stream>>>(p, c, rows, cols, ldc, splits);
-    else if (splits <= 16) splitk_reduce_kernel<T, 16><<<blocks, 256, 0, stream>>>(p, c, rows, cols, ldc, splits);
-    else splitk_reduce_kernel<T, 32><<<blocks, 256, 0, stream>>>(p, c, rows, cols, ldc, splits);
+    if (splits <= 2) (void)launch_overlapping(splitk_reduce_kernel<T, 2>, (unsigned)blocks, 256u, 0, stream, p, c, rows, cols, ldc, splits);
+    else if (splits <= 4) (void)launch_overlapping(splitk_reduce_kernel<T, 4>, (unsigned)blocks, 256u, 0, stream, p, c, rows, cols, ldc, splits);
+    else if (splits <= 8) (void)launch_overlapping(splitk_reduce_kernel<T, 8>, (unsigned)blocks, 256u, 0, stream, p, c, rows, cols, ldc, splits);
+    else if (splits <= 16) (void)launch_overlapping(splitk_reduce_kernel<T, 16>, (unsigned)blocks, 256u, 0, stream, p, c, rows, cols, ldc, splits);
+    else (void)launch_overlapping(splitk_reduce_kernel<T, 32>, (unsigned)blocks, 256u, 0, stream, p, c, rows, cols, ldc, splits);
 }
 // splits <= 32 (kMaxSplits).  The partials are dense, so groups of four stay inside a row when cols % 4 == 0.
 void launch_splitk_reduce(const float* part, float* C, long long rows, long long cols, long long ldc, int splits,
@@ -1616,8 +1626,8 @@ int launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap&
     }
     const long long work = (long long)p.tiles_m * p.tiles_n * p.splits;
     const int grid = work < dev.sm_count ? (int)work : dev.sm_count;
-    if (p.epi) gemm_tf32_kernel<true><<<grid, kThreads, kSmemBytes, stream>>>(ma, mb, mc, mp, rows, p);
-    else gemm_tf32_kernel<false><<<grid, kThreads, kSmemBytes, stream>>>(ma, mb, mc, mp, rows, p);
+    if (p.epi) QFMT_CUDA_TRY(launch_overlapping(gemm_tf32_kernel<true>, (unsigned)grid, (unsigned)kThreads, kSmemBytes, stream, ma, mb, mc, mp, rows, p));
+    else QFMT_CUDA_TRY(launch_overlapping(gemm_tf32_kernel<false>, (unsigned)grid, (unsigned)kThreads, kSmemBytes, stream, ma, mb, mc, mp, rows, p));
     QFMT_CUDA_TRY(cudaGetLastError());
     if (p.sk_cpt > 0) {
         streamk_fixup_kernel<<<grid * kFixupParts, 64, 0, stream>>>(p.sk_partials, p.C, grid, p.tiles_m * p.tiles_n, p.tiles_m,
@@ -1744,7 +1754,8 @@ int launch_pair(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap&
     const long long clusters = p.sk_flags != nullptr ? kPlanPairs : (work < dev.sm_count / 2 ? work : dev.sm_count / 2);
     const unsigned grid = (unsigned)(2 * clusters);
     const bool sk = p.sk_flags != nullptr;
-#define QFMT_PAIR_LAUNCH(...) gemm_tf32_pair_kernel<__VA_ARGS__><<<grid, kThreads, kPairSmemBytes, stream>>>(ma, mb, mc, p)
+#define QFMT_PAIR_LAUNCH(...) \
+    QFMT_CUDA_TRY(launch_overlapping(gemm_tf32_pair_kernel<__VA_ARGS__>, grid, (unsigned)kThreads, kPairSmemBytes, stream, ma, mb, mc, p))
     if (kind == kKindF16) { if (sk) QFMT_PAIR_LAUNCH(false, kKindF16, true); else QFMT_PAIR_LAUNCH(false, kKindF16, false); }
     else if (kind == kKindBf16) { if (sk) QFMT_PAIR_LAUNCH(false, kKindBf16, true); else QFMT_PAIR_LAUNCH(false, kKindBf16, false); }
     else if (p.epi) QFMT_PAIR_LAUNCH(true, kKindTf32, false);
@@ -1768,9 +1779,11 @@ int launch_conv_pair(const CUtensorMap& mb, const CUtensorMap& mc, const CUtenso
     const long long work = (long long)p.tiles_m * p.tiles_n;
     const long long clusters = p.sk_flags != nullptr ? kPlanPairs : (work < dev.sm_count / 2 ? work : dev.sm_count / 2);
     if (p.sk_flags != nullptr)
-        gemm_conv_pair_kernel<true><<<(unsigned)(2 * clusters), kThreads, kPairSmemBytes, stream>>>(mb, mc, mc2, rows, p);
+        QFMT_CUDA_TRY(launch_overlapping(gemm_conv_pair_kernel<true>, (unsigned)(2 * clusters), (unsigned)kThreads, kPairSmemBytes, stream,
+                                         mb, mc, mc2, rows, p));
     else
-        gemm_conv_pair_kernel<false><<<(unsigned)(2 * clusters), kThreads, kPairSmemBytes, stream>>>(mb, mc, mc2, rows, p);
+        QFMT_CUDA_TRY(launch_overlapping(gemm_conv_pair_kernel<false>, (unsigned)(2 * clusters), (unsigned)kThreads, kPairSmemBytes, stream,
+                                         mb, mc, mc2, rows, p));
     QFMT_CUDA_TRY(cudaGetLastError());
     return QFMT_OK;
 }
@@ -1785,7 +1798,7 @@ int launch_wgrad_pair(const CUtensorMap& ma, const CUtensorMap& mb, const CUtens
     }
     const long long work = (long long)p.tiles_m * p.tiles_n * p.splits;
     const long long clusters = work < dev.sm_count / 2 ? work : dev.sm_count / 2;
-    gemm_wgrad_pair_kernel<<<(unsigned)(2 * clusters), kThreads, kPairSmemBytes, stream>>>(ma, mb, mc, p);
+    QFMT_CUDA_TRY(launch_overlapping(gemm_wgrad_pair_kernel, (unsigned)(2 * clusters), (unsigned)kThreads, kPairSmemBytes, stream, ma, mb, mc, p));
     QFMT_CUDA_TRY(cudaGetLastError());
     return QFMT_OK;
 }
@@ -1809,6 +1822,16 @@ bool pair_schedule_fits(long long tiles, long long cpt) {
 
 // Turns the balanced schedule of the pair kernel on: chunks per tile, the most pieces a pair can have,
 // and the flag words behind the workspace header (cleared on the stream).
+// Zeroes the hand-over words of the balanced schedule.  A kernel rather than a memset so that the launches
+// around it can overlap (launch_overlapping): it lets the product that follows be placed at once, then waits
+// for the kernel before it (which may be a product still reading these words), then clears them; the product
+// that follows waits for this kernel, and so for both.
+__global__ void __launch_bounds__(256) zero_words_kernel(int* words, int n) {
+    grid_launch_dependents();
+    grid_dependency_wait();
+    for (int i = threadIdx.x; i < n; i += 256) words[i] = 0;
+}
+
 int enable_pair_schedule(GemmParams* p, void* d_workspace, cudaStream_t stream) {
     p->sk_cpt = (p->kb_total + kChunkKB - 1) / kChunkKB;
     const long long total = (long long)p->tiles_m * p->tiles_n * p->sk_cpt;
@@ -1817,7 +1840,7 @@ int enable_pair_schedule(GemmParams* p, void* d_workspace, cudaStream_t stream) 
     p->sk_q = (int)(total / kPlanPairs);
     p->sk_r = (int)(total % kPlanPairs);
     p->sk_flags = reinterpret_cast<int*>(reinterpret_cast<char*>(d_workspace) + kWorkspaceHeader);
-    QFMT_CUDA_TRY(cudaMemsetAsync(p->sk_flags, 0, kSkFlagBytes, stream));
+    QFMT_CUDA_TRY(launch_overlapping(zero_words_kernel, 1u, 256u, 0, stream, p->sk_flags, (int)(kSkFlagBytes / sizeof(int))));
     return QFMT_OK;
 }
 

@@ -59,6 +59,7 @@ quantize_stats_kernel(const uint32_t* in, uint32_t* out, uint32_t head,
                       unsigned long long n4, uint32_t tail, QuantParams p, qfmt_stats_t* __restrict__ stats,
                       unsigned long long n_total, const float* __restrict__ d_scale) {
     extern __shared__ uint32_t lane_hist[];  // [(top + kExtraBins)][32]
+    grid_launch_dependents();  // a product launched after this pass may take the SMs as this grid leaves them
     if (kScale && d_scale != nullptr) p.scale = *d_scale;  // loss scale kept on the device (dynamic loss scaling)
     const int nbins = p.top + kExtraBins;
     const int lane = threadIdx.x & 31;
@@ -430,6 +431,8 @@ bias_quantize_stats_kernel(const uint32_t* acc, long long ld_acc, const uint32_t
     const uint32_t inf_bits = p.top < 255 ? (uint32_t)(p.top + p.code_off) << 23 : 0u;  // 2^(E_max+1); 0 = 1/8/m
     // fast path: exponent fields from E_min up to E_max - 1 (see bias_round_fast)
     const uint32_t lo2 = p.min_normal << 1, span2 = (inf_bits - (1u << 23) - p.min_normal) << 1;
+    grid_dependency_wait();    // the sums come from the product launched before this pass
+    grid_launch_dependents();
     if (kStats) {
         for (int i = threadIdx.x; i < nbins * 32; i += kThreads) lane_hist[i] = 0u;
         __syncthreads();
@@ -718,7 +721,7 @@ int bias_quantize_stats_device(const float* d_acc, int64_t ld_acc, const float* 
         const unsigned long long cap = (unsigned long long)dev.sm_count * 2;  // 64 registers: two blocks per SM
         if (want > cap) want = cap;
 #define QFMT_BLAUNCH(S, C, P)                                                                                     \
-    bias_quantize_stats_kernel<S, C, P><<<(unsigned)want, kThreads, smem, stream>>>(                              \
+    err = launch_overlapping(bias_quantize_stats_kernel<S, C, P>, (unsigned)want, (unsigned)kThreads, smem, stream, \
         acc, (long long)ld_acc, bias, out, (long long)ld_out, (unsigned long long)rows, c4, cw, rpp, p, d_stats, sign_shift)
 #define QFMT_BLAUNCH2(S, C) do { if (pack) QFMT_BLAUNCH(S, C, true); else QFMT_BLAUNCH(S, C, false); } while (0)
         if (has_stats) { if (has_scale) QFMT_BLAUNCH2(true, true); else QFMT_BLAUNCH2(true, false); }
