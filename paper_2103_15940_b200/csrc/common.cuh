@@ -64,4 +64,14 @@ cudaError_t launch_overlapping(void (*kernel)(P...), unsigned grid, unsigned blo
     return cudaLaunchKernelEx(&cfg, kernel, std::forward<A>(args)...);
 }
 
+// Zeroes a few words (the hand-over words of the balanced schedule, a statistics record).  A kernel rather than a memset so that the launches
+// around it can overlap (launch_overlapping): it lets the product that follows be placed at once, then waits
+// for the kernel before it (which may be a product still reading these words), then clears them; the product
+// that follows waits for this kernel, and so for both.
+static __global__ void __launch_bounds__(256) zero_words_kernel(int* words, int n) {
+    grid_launch_dependents();
+    grid_dependency_wait();
+    for (int i = threadIdx.x; i < n; i += 256) words[i] = 0;
+}
+
 }  // namespace qfmt

@@ -1822,16 +1822,6 @@ bool pair_schedule_fits(long long tiles, long long cpt) {
 
 // Turns the balanced schedule of the pair kernel on: chunks per tile, the most pieces a pair can have,
 // and the flag words behind the workspace header (cleared on the stream).
-// Zeroes the hand-over words of the balanced schedule.  A kernel rather than a memset so that the launches
-// around it can overlap (launch_overlapping): it lets the product that follows be placed at once, then waits
-// for the kernel before it (which may be a product still reading these words), then clears them; the product
-// that follows waits for this kernel, and so for both.
-__global__ void __launch_bounds__(256) zero_words_kernel(int* words, int n) {
-    grid_launch_dependents();
-    grid_dependency_wait();
-    for (int i = threadIdx.x; i < n; i += 256) words[i] = 0;
-}
-
 int enable_pair_schedule(GemmParams* p, void* d_workspace, cudaStream_t stream) {
     p->sk_cpt = (p->kb_total + kChunkKB - 1) / kChunkKB;
     const long long total = (long long)p->tiles_m * p->tiles_n * p->sk_cpt;

@@ -696,7 +696,10 @@ int bias_quantize_stats_device(const float* d_acc, int64_t ld_acc, const float* 
     DeviceInfo dev;
     rc = current_device(&dev);
     if (rc != QFMT_OK) return rc;
-    if (d_stats != nullptr && accumulate == 0) QFMT_CUDA_TRY(cudaMemsetAsync(d_stats, 0, sizeof(qfmt_stats_t), stream));
+    // cleared by a kernel that the pass behind it can overlap (see zero_words_kernel), not by a memset
+    if (d_stats != nullptr && accumulate == 0)
+        QFMT_CUDA_TRY(launch_overlapping(zero_words_kernel, 1u, 256u, 0, stream, reinterpret_cast<int*>(d_stats),
+                                         (int)(sizeof(qfmt_stats_t) / sizeof(int))));
     if (n == 0) return QFMT_OK;
 
     const QuantParams p = make_params(*fmt);
