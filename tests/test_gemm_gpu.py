@@ -445,3 +445,49 @@ def test_balanced_schedule_real_values_within_bound_and_reproducible(balanced_sc
     for _ in range(3):
         C2 = gpu_gemm(A, B)
         assert np.array_equal(C1.view(np.uint32), C2.view(np.uint32))
+
+
+# ---------------------------------------------------------------------------------------------
+# Products that feed one another, launched back to back.  A product may be placed on the GPU while
+# the kernel before it still runs; it must not read its operands before that kernel has finished.
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("policy", [0, 3], ids=["automatic", "balanced"])
+def test_dependent_products_back_to_back(policy):
+    """C1 = A B, C2 = C1 D, C3 = C2^T E with no synchronisation in between, C1 and C2 refilled with
+    other values before every round.  Entries in -1..1 keep every value an integer that the format
+    holds (|C1| <= 512 needs ten bits) and every sum exact, so C3 is exact iff every product saw
+    the finished output of the one before it (the third one through split K and its reduction)."""
+    rng = np.random.default_rng(11)
+    M, K, N1, N2, N3 = 2560, 512, 2560, 256, 128
+    gen = lambda s: rng.integers(-1, 2, size=s).astype(np.float32)
+    A, B = gen((M, K)), gen((K, N1))
+    D = np.zeros((N1, N2), dtype=np.float32)          # sparse, so that C2 stays within the format's ten bits
+    D[rng.integers(0, N1, size=N2), np.arange(N2)] = 1.0
+    E = gen((M, N3))
+    C1_ref = A.astype(np.int64) @ B.astype(np.int64)
+    C2_ref = C1_ref @ D.astype(np.int64)
+    C3_ref = C2_ref.T @ E.astype(np.int64)
+    assert np.abs(C1_ref).max() < 1024 and np.abs(C2_ref).max() < 1024 and np.abs(C3_ref).max() < 2 ** 24
+    dA, dB, dD, dE = (torch.from_numpy(t).to(DEV) for t in (A, B, D, E))
+    C1 = torch.empty(M, N1, dtype=torch.float32, device=DEV)
+    C2 = torch.empty(M, N2, dtype=torch.float32, device=DEV)
+    C3 = torch.empty(N2, N3, dtype=torch.float32, device=DEV)
+    fmt = qf.make_format(6, 9)
+    ops = [(qf.make_matrix(dA), qf.make_matrix(dB), C1, N1), (qf.make_matrix(C1), qf.make_matrix(dD), C2, N2),
+           (qf.make_matrix(C2, True), qf.make_matrix(dE), C3, N3)]
+    qf.qfmt_gemm_tile_policy(policy)
+    try:
+        wss = [torch.zeros(max(256, qf.qfmt_gemm_workspace_bytes(a, b)), dtype=torch.uint8, device=DEV) for a, b, _, _ in ops]
+        assert wss[2].numel() > 256 + 2 * N2 * N3 * 4          # the third product is split along K
+        for rnd in range(6):
+            C1.fill_(float(rnd + 2))
+            C2.fill_(float(-rnd - 3))
+            C3.fill_(float("nan"))
+            for (a, b, C, ldc), ws in zip(ops, wss):
+                qf.qfmt_gemm(a, b, C, ldc, fmt, ws, ws.numel())
+            for ws in wss:
+                assert qf.qfmt_device_status(ws) == qf.QFMT_OK
+            assert np.array_equal(C3.cpu().numpy().astype(np.int64), C3_ref), rnd
+            assert np.array_equal(C1.cpu().numpy().astype(np.int64), C1_ref), rnd
+    finally:
+        qf.qfmt_gemm_tile_policy(0)
