@@ -407,10 +407,15 @@ __device__ __forceinline__ uint32_t to_16(float v) {
     return kBf16 ? (__float_as_uint(v) >> 16) : (uint32_t)__half_as_ushort(__float2half_rn(v));
 }
 
+// master + h in fp32, h a 16-bit value: the mixed-precision add converts h exactly and rounds the sum
+// once (to nearest even, denormals kept), which is what a conversion followed by an fp32 addition does,
+// in one instruction.
 template <bool kBf16>
-__device__ __forceinline__ float2 pair_to_float2(uint32_t u) {
-    if (kBf16) return make_float2(__uint_as_float(u << 16), __uint_as_float(u & 0xFFFF0000u));
-    return __half22float2(*reinterpret_cast<const __half2*>(&u));
+__device__ __forceinline__ float add_16_to_master(float master, unsigned short h) {
+    float r;
+    if (kBf16) asm("add.rn.f32.bf16 %0, %1, %2;" : "=f"(r) : "h"(h), "f"(master));
+    else asm("add.rn.f32.f16 %0, %1, %2;" : "=f"(r) : "h"(h), "f"(master));
+    return r;
 }
 
 // The part of a 32-deep slice of an operand tile (kRows rows of op(A), or columns of op(B)) that a
@@ -558,9 +563,8 @@ fmac8_f16_kernel(FmacParams g, QuantParams p, qfmt_stats_t* __restrict__ stats) 
                 for (int i = 0; i < kHfTM; ++i)
 #pragma unroll
                     for (int j = 0; j < kHfTN / 2; ++j) {
-                        const float2 v = pair_to_float2<kBf16>(small[i][j]);
-                        master[i][2 * j] = add_ieee(master[i][2 * j], v.x);
-                        master[i][2 * j + 1] = add_ieee(master[i][2 * j + 1], v.y);
+                        master[i][2 * j] = add_16_to_master<kBf16>(master[i][2 * j], (unsigned short)(small[i][j] & 0xFFFFu));
+                        master[i][2 * j + 1] = add_16_to_master<kBf16>(master[i][2 * j + 1], (unsigned short)(small[i][j] >> 16));
                         small[i][j] = zero2;
                     }
             }
