@@ -76,6 +76,61 @@ __device__ __forceinline__ uint32_t quantize_one(uint32_t xb, const QuantParams&
     return sign | qa;
 }
 
+// Two elements of binary16 (1/5/10) or bfloat16 (1/8/7) at once: for these two formats the rounding of
+// Section IV-A (nearest even onto the format's grid, denormals included, overflow to infinity at
+// 2^(E_max+1)) is the IEEE conversion the hardware has, so one packed conversion replaces the integer
+// rounding of quantize_one; the classification into bins and the treatment of specials are the same.
+// Returns the same containers and bins as quantize_one does, element by element.
+template <bool kScale, bool kBf16>
+__device__ __forceinline__ void quantize_pair_native(uint32_t xb0, uint32_t xb1, const QuantParams& p, uint32_t& q0,
+                                                     uint32_t& q1, int& bin0, int& bin1) {
+    constexpr int kM = kBf16 ? 7 : 10;
+    constexpr uint32_t kTop = kBf16 ? 255u : 31u;
+    const float y0 = kScale ? mul_ieee(__uint_as_float(xb0), p.scale) : __uint_as_float(xb0);
+    const float y1 = kScale ? mul_ieee(__uint_as_float(xb1), p.scale) : __uint_as_float(xb1);
+    uint32_t pk;  // y1's code in the upper half, y0's in the lower
+    if (kBf16) asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(pk) : "f"(y1), "f"(y0));
+    else asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(pk) : "f"(y1), "f"(y0));
+    uint32_t c0, c1;  // containers of the two codes (exact)
+    if (kBf16) {
+        c0 = pk << 16;
+        c1 = pk & 0xFFFF0000u;
+    } else {
+        float f0, f1;
+        asm("{ .reg .b16 lo, hi; mov.b32 {lo, hi}, %2; cvt.f32.f16 %0, lo; cvt.f32.f16 %1, hi; }"
+            : "=f"(f0), "=f"(f1) : "r"(pk));
+        c0 = __float_as_uint(f0);
+        c1 = __float_as_uint(f1);
+    }
+    const uint32_t e0 = (pk >> kM) & kTop, e1 = (pk >> (16 + kM)) & kTop;
+    bin0 = (int)e0;
+    bin1 = (int)e1;
+    if (e0 - 1u >= kTop - 1u) {
+        const uint32_t ax = xb0 & 0x7FFFFFFFu, sign = xb0 & 0x80000000u;  // a NaN's sign does not survive the multiply
+        if (e0 == kTop) {
+            const bool is_nan = ax > 0x7F800000u;
+            c0 = sign | (is_nan ? 0x7FC00000u : 0x7F800000u);
+            bin0 = p.top + (is_nan ? kBinNanIn : (ax == 0x7F800000u ? kBinInfIn : kBinOverflow));
+        } else {
+            bin0 = p.top + (ax == 0u ? kBinZeroIn : ((pk & 0x7FFFu) == 0u ? kBinRoundedToZero : kBinDenormal));
+            if (!p.keep_denormals) c0 = sign;
+        }
+    }
+    if (e1 - 1u >= kTop - 1u) {
+        const uint32_t ax = xb1 & 0x7FFFFFFFu, sign = xb1 & 0x80000000u;
+        if (e1 == kTop) {
+            const bool is_nan = ax > 0x7F800000u;
+            c1 = sign | (is_nan ? 0x7FC00000u : 0x7F800000u);
+            bin1 = p.top + (is_nan ? kBinNanIn : (ax == 0x7F800000u ? kBinInfIn : kBinOverflow));
+        } else {
+            bin1 = p.top + (ax == 0u ? kBinZeroIn : ((pk & 0x7FFF0000u) == 0u ? kBinRoundedToZero : kBinDenormal));
+            if (!p.keep_denormals) c1 = sign;
+        }
+    }
+    q0 = c0;
+    q1 = c1;
+}
+
 // R(S * x) without statistics, for formats with e <= 7: the first rounding of the layer formula.
 // The integer pipe runs at half the float pipe's rate, so the rounding is two float operations:
 // with C = 1.5 * 2^(max(floor(log2|y|), E_min) + 23 - m) the sum y + C lies in C's binade, whose
