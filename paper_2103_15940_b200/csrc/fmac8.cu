@@ -378,7 +378,11 @@ fmac8_kernel(FmacParams g, QuantParams p, qfmt_stats_t* __restrict__ stats) {
 
 // ---- 1/5/10 and 1/8/7: the hardware's own 16-bit fused multiply-adds --------------------------
 constexpr int kHfBM = 64, kHfBN = 128, kHfTM = 4, kHfTN = 8;
-constexpr int kHfBlocksPerSm = 2;
+// Resident blocks per SM: two for matrix products (the next operand slice waits in registers while this one
+// is used: 120 registers a thread), three for convolutions (their gathered slices are not fetched ahead, so
+// a third block hides more of the gather: 14.3 -> 15.5 TFMAC/s on a 3 x 3 layer, where matrix products lose:
+// 19.7 -> 18.5).
+constexpr int kHfBlocksPerSm = 2, kHfConvBlocksPerSm = 3;
 
 // two FMACs: {a.lo * b.lo + c.lo, a.hi * b.hi + c.hi}, each rounded once to the 16-bit type
 template <bool kBf16>
@@ -454,7 +458,7 @@ __device__ __forceinline__ void fetch_slice(float4 (&v)[kRows * kFmBK / (4 * kFm
 }
 
 template <bool kStats, bool kFlush, bool kBf16, bool kConv>
-__global__ void __launch_bounds__(kFmThreads, kHfBlocksPerSm)
+__global__ void __launch_bounds__(kFmThreads, kConv ? kHfConvBlocksPerSm : kHfBlocksPerSm)
 fmac8_f16_kernel(FmacParams g, QuantParams p, qfmt_stats_t* __restrict__ stats) {
     __shared__ __align__(16) uint32_t As2[kFmBK][kHfBM + 4];  // each A value twice: {a, a} as f16x2
     __shared__ __align__(16) uint16_t Bs[kFmBK][kHfBN + 8];
@@ -584,7 +588,7 @@ int launch_fmac8(const FmacParams& g, const QuantParams& p, const qfmt_format_t*
     const size_t smem = has_stats ? (size_t)(p.top + kExtraBins) * 32 * sizeof(uint32_t) : 0;
     if (use_native) {
         const long long tiles = (((long long)g.M + kHfBM - 1) / kHfBM) * (((long long)g.N + kHfBN - 1) / kHfBN);
-        const long long slots = (long long)dev.sm_count * kHfBlocksPerSm;
+        const long long slots = (long long)dev.sm_count * (conv ? kHfConvBlocksPerSm : kHfBlocksPerSm);
         const unsigned grid = (unsigned)(tiles < slots ? tiles : slots);
         const bool flush = fmt->denormals == 0;
         const size_t sm = has_stats ? smem : 0;
