@@ -911,9 +911,9 @@ def finish(args, world, value, total_ms, n, runs, clocks, e2e, roofline, cpu, ge
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the quantize+stats kernel on the 64 Mi-element
 # tensor, from one ncu capture of that kernel (read + write).  A figure here belongs to the kernel as it was
 # when the counters were taken: it is set to None as soon as that kernel's code changes, until re-taken.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 268463872 + 218315520
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 268463872 + 218982144
 # the same for the layer-output kernel on the 8192 x 4096 product
-NCU_EPILOGUE_TRAFFIC_BYTES_PER_LAUNCH = 134290432 + 85915904
+NCU_EPILOGUE_TRAFFIC_BYTES_PER_LAUNCH = 134294528 + 84735232
 
 
 def main():
