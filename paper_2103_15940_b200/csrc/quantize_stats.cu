@@ -215,9 +215,10 @@ quantize_stats_transpose_kernel(const uint32_t* __restrict__ in, uint32_t* __res
 // bandwidth): the rounding pass writing packed codes instead of fp32 containers, 4 bytes read and
 // 2 written per element, and the pass that expands codes back to containers for the contraction.
 // A thread takes eight consecutive elements: two 128-bit loads, one 128-bit store.
-// kRare: results below the smallest normal are expected to be rare (formats with e >= 6): the denormal
-// grid sits behind a branch (quantize_pack_one_rare_denormals).
-template <bool kStats, bool kScale, bool kRare>
+// kMode 1: results below the smallest normal are expected to be rare (formats with e >= 6): the denormal
+// grid sits behind a branch (quantize_pack_one_rare_denormals).  kMode 2 / 3: binary16 / bfloat16 by the
+// hardware's conversion in the vector body (quantize_pack_pair_native).  kMode 0: every other format.
+template <bool kStats, bool kScale, int kMode>
 __global__ void __launch_bounds__(kThreads)
 quantize_stats_pack16_kernel(const uint32_t* __restrict__ in, uint16_t* __restrict__ codes, unsigned long long n,
                              int vec, QuantParams p, int sign_shift, qfmt_stats_t* __restrict__ stats) {
@@ -245,16 +246,30 @@ quantize_stats_pack16_kernel(const uint32_t* __restrict__ in, uint16_t* __restri
             const unsigned long long idx = base + (unsigned long long)u * kThreads + threadIdx.x;
             if (idx < n8) {
                 const uint32_t w[8] = {v[u][0].x, v[u][0].y, v[u][0].z, v[u][0].w, v[u][1].x, v[u][1].y, v[u][1].z, v[u][1].w};
-                uint32_t c[8];
+                if (kMode >= 2) {
+                    uint32_t pk[4];
 #pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    int b;
-                    c[j] = kRare ? quantize_pack_one_rare_denormals<kScale>(w[j], p, sign_shift, b)
-                                 : quantize_pack_one<kScale>(w[j], p, sign_shift, b);
-                    if (kStats) atomicAdd(&lane_hist[b * 32 + lane], 1u);
+                    for (int j = 0; j < 4; ++j) {
+                        int b0, b1;
+                        pk[j] = quantize_pack_pair_native<kScale, kMode == 3>(w[2 * j], w[2 * j + 1], p, b0, b1);
+                        if (kStats) {
+                            atomicAdd(&lane_hist[b0 * 32 + lane], 1u);
+                            atomicAdd(&lane_hist[b1 * 32 + lane], 1u);
+                        }
+                    }
+                    store_stream(reinterpret_cast<uint4*>(codes) + idx, make_uint4(pk[0], pk[1], pk[2], pk[3]));
+                } else {
+                    uint32_t c[8];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        int b;
+                        c[j] = kMode == 1 ? quantize_pack_one_rare_denormals<kScale>(w[j], p, sign_shift, b)
+                                          : quantize_pack_one<kScale>(w[j], p, sign_shift, b);
+                        if (kStats) atomicAdd(&lane_hist[b * 32 + lane], 1u);
+                    }
+                    store_stream(reinterpret_cast<uint4*>(codes) + idx,
+                                 make_uint4(c[0] | (c[1] << 16), c[2] | (c[3] << 16), c[4] | (c[5] << 16), c[6] | (c[7] << 16)));
                 }
-                store_stream(reinterpret_cast<uint4*>(codes) + idx,
-                             make_uint4(c[0] | (c[1] << 16), c[2] | (c[3] << 16), c[4] | (c[5] << 16), c[6] | (c[7] << 16)));
             }
         }
     }
@@ -263,8 +278,8 @@ quantize_stats_pack16_kernel(const uint32_t* __restrict__ in, uint16_t* __restri
     for (unsigned long long i = done + (unsigned long long)blockIdx.x * kThreads + threadIdx.x; i < n;
          i += (unsigned long long)gridDim.x * kThreads) {
         int b;
-        codes[i] = (uint16_t)(kRare ? quantize_pack_one_rare_denormals<kScale>(in[i], p, sign_shift, b)
-                                    : quantize_pack_one<kScale>(in[i], p, sign_shift, b));
+        codes[i] = (uint16_t)(kMode == 1 ? quantize_pack_one_rare_denormals<kScale>(in[i], p, sign_shift, b)
+                                         : quantize_pack_one<kScale>(in[i], p, sign_shift, b));
         if (kStats) atomicAdd(&lane_hist[b * 32 + lane], 1u);
     }
     if (kStats) {
@@ -789,17 +804,20 @@ int quantize_stats_pack16_device(const float* d_in, uint16_t* d_codes, size_t n,
     const int sign_shift = fmt->e + fmt->m;
     // 1/5/m tensors of small gradients are mostly denormal (the paper's observation on binary16), so
     // only wider exponents take the kernel that branches on results below the smallest normal
-    const bool rare = fmt->e >= 6;
+    const int mode = (fmt->e == 5 && fmt->m == 10) ? 2 : (fmt->e == 8 && fmt->m == 7) ? 3 : (fmt->e >= 6 ? 1 : 0);
+#define QFMT_PLAUNCH1(S, C, M) \
+    quantize_stats_pack16_kernel<S, C, M><<<(unsigned)want, kThreads, smem, stream>>>(in, d_codes, n, vec, p, sign_shift, d_stats)
 #define QFMT_PLAUNCH(S, C)                                                                                         \
     do {                                                                                                           \
-        if (rare) quantize_stats_pack16_kernel<S, C, true><<<(unsigned)want, kThreads, smem, stream>>>(            \
-                      in, d_codes, n, vec, p, sign_shift, d_stats);                                                \
-        else quantize_stats_pack16_kernel<S, C, false><<<(unsigned)want, kThreads, smem, stream>>>(               \
-                      in, d_codes, n, vec, p, sign_shift, d_stats);                                                \
+        if (mode == 3) QFMT_PLAUNCH1(S, C, 3);                                                                     \
+        else if (mode == 2) QFMT_PLAUNCH1(S, C, 2);                                                                \
+        else if (mode == 1) QFMT_PLAUNCH1(S, C, 1);                                                                \
+        else QFMT_PLAUNCH1(S, C, 0);                                                                               \
     } while (0)
     if (has_stats) { if (has_scale) QFMT_PLAUNCH(true, true); else QFMT_PLAUNCH(true, false); }
     else { if (has_scale) QFMT_PLAUNCH(false, true); else QFMT_PLAUNCH(false, false); }
 #undef QFMT_PLAUNCH
+#undef QFMT_PLAUNCH1
     QFMT_CUDA_TRY(cudaGetLastError());
     return QFMT_OK;
 }

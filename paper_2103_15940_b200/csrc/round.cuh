@@ -131,6 +131,51 @@ __device__ __forceinline__ void quantize_pair_native(uint32_t xb0, uint32_t xb1,
     q1 = c1;
 }
 
+// The packed 16-bit codes of two elements of binary16 / bfloat16 by the same conversion: the code of a
+// finite result IS the converted half, so only the specials are touched (the library's NaN code, the
+// input's sign on it, the flush of denormals).  Same codes and bins as quantize_pack_one.
+template <bool kScale, bool kBf16>
+__device__ __forceinline__ uint32_t quantize_pack_pair_native(uint32_t xb0, uint32_t xb1, const QuantParams& p, int& bin0,
+                                                              int& bin1) {
+    constexpr int kM = kBf16 ? 7 : 10;
+    constexpr uint32_t kTop = kBf16 ? 255u : 31u;
+    const float y0 = kScale ? mul_ieee(__uint_as_float(xb0), p.scale) : __uint_as_float(xb0);
+    const float y1 = kScale ? mul_ieee(__uint_as_float(xb1), p.scale) : __uint_as_float(xb1);
+    uint32_t pk;  // y1's code in the upper half, y0's in the lower
+    if (kBf16) asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(pk) : "f"(y1), "f"(y0));
+    else asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(pk) : "f"(y1), "f"(y0));
+    const uint32_t e0 = (pk >> kM) & kTop, e1 = (pk >> (16 + kM)) & kTop;
+    bin0 = (int)e0;
+    bin1 = (int)e1;
+    if (e0 - 1u >= kTop - 1u) {
+        const uint32_t ax = xb0 & 0x7FFFFFFFu, sign = (xb0 >> 31) << 15;
+        uint32_t c = pk & 0xFFFFu;
+        if (e0 == kTop) {
+            const bool is_nan = ax > 0x7F800000u;
+            c = sign | (kTop << kM) | (is_nan ? (1u << (kM - 1)) : 0u);
+            bin0 = p.top + (is_nan ? kBinNanIn : (ax == 0x7F800000u ? kBinInfIn : kBinOverflow));
+        } else {
+            bin0 = p.top + (ax == 0u ? kBinZeroIn : ((pk & 0x7FFFu) == 0u ? kBinRoundedToZero : kBinDenormal));
+            if (!p.keep_denormals) c = sign;
+        }
+        pk = (pk & 0xFFFF0000u) | c;
+    }
+    if (e1 - 1u >= kTop - 1u) {
+        const uint32_t ax = xb1 & 0x7FFFFFFFu, sign = (xb1 >> 31) << 15;
+        uint32_t c = pk >> 16;
+        if (e1 == kTop) {
+            const bool is_nan = ax > 0x7F800000u;
+            c = sign | (kTop << kM) | (is_nan ? (1u << (kM - 1)) : 0u);
+            bin1 = p.top + (is_nan ? kBinNanIn : (ax == 0x7F800000u ? kBinInfIn : kBinOverflow));
+        } else {
+            bin1 = p.top + (ax == 0u ? kBinZeroIn : ((pk & 0x7FFF0000u) == 0u ? kBinRoundedToZero : kBinDenormal));
+            if (!p.keep_denormals) c = sign;
+        }
+        pk = (pk & 0xFFFFu) | (c << 16);
+    }
+    return pk;
+}
+
 // R(S * x) without statistics, for formats with e <= 7: the first rounding of the layer formula.
 // The integer pipe runs at half the float pipe's rate, so the rounding is two float operations:
 // with C = 1.5 * 2^(max(floor(log2|y|), E_min) + 23 - m) the sum y + C lies in C's binade, whose
