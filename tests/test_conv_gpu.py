@@ -167,6 +167,25 @@ def test_config4_resnet50_shaped_layers(shape):
     print("config4", shape.r, worst)
 
 
+def test_56x56_stage_sampled():
+    """A layer shaped like the first stage of a ResNet-50 (64 -> 64 channels at 56 x 56, 3 x 3, batch 8):
+    the filter gradient runs two 32-pixel stages per output row over 448 rows and splits K; forward and data
+    gradient have two image rows per tile.  Integers first (exact), then values of the format within the bound,
+    on sampled outputs."""
+    geom = (8, 64, 56, 56, 64, 3, 3, 1, 1)
+    n, ci, h, w, co, r, s, ph, pw = geom
+    rng = np.random.default_rng(56)
+    X = rng.integers(-2, 3, size=(n, ci, h, w)).astype(np.float32)
+    Wt = rng.integers(-2, 3, size=(co, ci, r, s)).astype(np.float32)
+    dY = rng.integers(-1, 2, size=(n, co, h, w)).astype(np.float32)
+    all_three(geom, X, Wt, dY, exact=True, sample=20000, seed=7)
+    rng = workloads.rng_for(56, 3)
+    X = workloads.lognormal_tensor(rng, (n, ci, h, w), -2.0, 2.0, p_zero=0.5, positive=True)
+    Wt = workloads.normal_tensor(rng, (co, ci, r, s), 0.05)
+    dY = workloads.lognormal_tensor(rng, (n, co, h, w), -20.0, 4.0)
+    all_three(geom, X, Wt, dY, grad_scale=2.0 ** 10, sample=20000, seed=8)
+
+
 def test_unsupported_geometries_are_refused():
     d = torch.zeros(1 << 16, dtype=torch.float32, device=DEV)
     ws = torch.zeros(1 << 20, dtype=torch.uint8, device=DEV)
