@@ -108,3 +108,27 @@ def test_builtin_scratch_refuses_on_the_host_what_does_not_fit(lib):
                                          ctypes.byref(fmt), None, None) == qf.QFMT_ERR_BAD_ARG  # ldc < N
     assert lib.qfmt_gemm_builtin_scratch(ctypes.byref(a), ctypes.byref(b), ctypes.c_void_p(0x30002), 1024,
                                          ctypes.byref(fmt), None, None) == qf.QFMT_ERR_BAD_ARG  # misaligned C
+
+
+def test_conv_workspace_planning_without_a_gpu(lib):
+    """qfmt_conv_workspace_bytes is host arithmetic: 0 for geometries the kernels refuse, the status
+    header otherwise, plus the split-K partial sums of a filter gradient."""
+    fwd, dgrad, wgrad = qf.QFMT_CONV_FWD, qf.QFMT_CONV_DGRAD, qf.QFMT_CONV_WGRAD
+    ws = qf.qfmt_conv_workspace_bytes
+    assert ws(fwd, qf.qfmt_conv_t(1, 30, 8, 8, 32, 3, 3, 1, 1)) == 0      # channels not a multiple of 32
+    assert ws(fwd, qf.qfmt_conv_t(1, 32, 8, 200, 32, 3, 3, 1, 1)) == 0    # forward rows longer than a tile
+    assert ws(dgrad, qf.qfmt_conv_t(1, 32, 8, 200, 32, 3, 3, 1, 1)) == 0
+    assert ws(fwd, qf.qfmt_conv_t(1, 32, 2, 2, 32, 5, 5, 0, 0)) == 0      # empty output
+    assert ws(7, qf.qfmt_conv_t(1, 32, 8, 8, 32, 3, 3, 1, 1)) == 0        # no such product
+    # filter gradients take rows of any length (32-pixel stages); long pixel dimensions are split
+    small = ws(wgrad, qf.qfmt_conv_t(1, 32, 2, 40, 32, 3, 3, 1, 1))
+    assert 256 <= small < 256 + 2 * 32 * 9 * 32 * 4                        # four stages: one split, no partial sums
+    g = qf.qfmt_conv_t(8, 64, 56, 56, 64, 3, 3, 1, 1)
+    big = ws(wgrad, g)
+    out_bytes = 64 * 9 * 64 * 4
+    assert big >= 256 + 2 * out_bytes and (big - 256) % out_bytes == 0     # whole partial results behind the header
+    assert (big - 256) // out_bytes <= 32                                  # at most 32 splits
+    assert ws(wgrad, qf.qfmt_conv_t(1, 32, 8, 200, 32, 3, 3, 1, 1)) > 0
+    # forward / data gradient: header, and the hand-over words when CTA pairs may run the balanced schedule
+    assert 256 <= ws(fwd, g) <= 256 + 8192
+    assert 256 <= ws(dgrad, g) <= 256 + 8192
